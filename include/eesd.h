@@ -1,0 +1,241 @@
+/*
+ * eesd.h -- C ABI of the EESD decode-round library for NVIDIA B200 (sm_100a).
+ *
+ * EESD = Early-exiting Speculative Decoding (Liu et al., arXiv 2406.03853).  One decode
+ * round drafts K tokens with the draft model of Eq. 1 (first N decoder layers of the target
+ * model, one early-exit decoder layer, RMSNorm, own vocabulary head), then verifies them in
+ * ONE forward pass of the target model over K+1 rows (Algorithm 1, verification step) and
+ * applies lossless speculative acceptance; a Thompson-sampling controller with a Beta
+ * posterior (Sec. 3.3, Eq. 3-4, Algorithm 2) decides when drafting stops.
+ *
+ * Conventions
+ *   - every function returns an int status: EESD_OK (0) or a negative EESD_ERR_* value; no
+ *     function throws, aborts or traps the device.  eesd_strerror() gives a text.
+ *   - "device" pointers are CUDA global-memory addresses of the current device; "host"
+ *     pointers are ordinary process memory.  The library never allocates or frees device
+ *     memory: all of it is passed in through eesd_buffers and stays owned by the caller, who
+ *     must keep it alive until eesd_destroy().
+ *   - matrices are row-major [out_features][in_features] (the input dimension is contiguous).
+ *   - batch size is 1 sequence per context (the paper's setting, Sec. 4.1); the standalone
+ *     acceptance entry points take a batch of independent sequences.
+ *   - all work is enqueued on the CUDA stream given at eesd_init(); calls that return
+ *     host-visible results synchronise that stream before returning.
+ *   - a context is not thread-safe; use one per host thread / stream.
+ */
+#ifndef EESD_H
+#define EESD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    EESD_OK = 0,
+    EESD_ERR_BADARG = -1,      /* null pointer, non-positive size, inconsistent shape         */
+    EESD_ERR_NOMEM = -2,       /* a caller-provided buffer is smaller than required            */
+    EESD_ERR_CUDA = -3,        /* a CUDA runtime call failed (see eesd_last_cuda_error)        */
+    EESD_ERR_STATE = -4,       /* call not valid in the current state (e.g. verify w/o draft)  */
+    EESD_ERR_CTX_FULL = -5,    /* the round would exceed max_ctx or the KV page pool           */
+    EESD_ERR_RNG = -6,         /* a uniform stream is missing or exhausted                     */
+    EESD_ERR_DEVICE = -7,      /* a kernel reported an error word (bad token id, bounded wait) */
+    EESD_ERR_UNSUPPORTED = -8  /* shape outside what the kernels support                       */
+};
+
+enum { EESD_F32 = 0, EESD_BF16 = 1 };
+enum { EESD_CTRL_FIXED_K = 0, EESD_CTRL_BETA_TS = 1 };
+enum { EESD_TS_RULE_PAPER = 0, EESD_TS_RULE_SINGLE_FAILURE = 1 };
+
+#define EESD_MAX_ROWS 16 /* most token rows one pass processes (k_cap + 1 <= 16) */
+
+/* Model and round configuration (plain data, copied by eesd_init). */
+typedef struct eesd_config {
+    int32_t d_model;      /* d: residual width (multiple of 8)                                  */
+    int32_t n_heads;      /* H: query heads                                                     */
+    int32_t n_kv_heads;   /* H_kv: key/value heads (H % H_kv == 0)                              */
+    int32_t head_dim;     /* D: 64 or 128                                                       */
+    int32_t ffn_dim;      /* F: SwiGLU hidden width (multiple of 8)                             */
+    int32_t vocab;        /* V                                                                  */
+    int32_t n_layers;     /* L: decoder layers of the target model                              */
+    int32_t n_early;      /* N: first layers shared by the draft model (Sec. 3.1), 1 <= N <= L  */
+    int32_t dtype;        /* EESD_F32 or EESD_BF16: weights, projection inputs and KV cache     */
+    int32_t tie_exit_head;/* 1: the exit head W of Eq. 1 is the target LM head (same storage)   */
+    float rms_eps;        /* RMSNorm epsilon                                                    */
+    float rope_theta;     /* rotary base; pairs (2i, 2i+1) turn by pos * theta^(-2i/D)          */
+    int32_t page_tokens;  /* tokens per KV page (power of two, >= 8)                            */
+    int32_t max_ctx;      /* most tokens a sequence may hold (prompt + generated + drafts)      */
+    int32_t k_cap;        /* most draft tokens per round, 1 <= k_cap <= EESD_MAX_ROWS - 1       */
+    float temperature;    /* 0: greedy (draft top-1, accept while equal to target top-1)        */
+    int32_t controller;   /* EESD_CTRL_FIXED_K or EESD_CTRL_BETA_TS                             */
+    int32_t fixed_k;      /* draft length for EESD_CTRL_FIXED_K                                 */
+    int32_t alpha0;       /* Beta prior (Algorithm 2, initialisation); positive integers        */
+    int32_t beta0;
+    int32_t ts_update_rule; /* EESD_TS_RULE_PAPER: r = |Q_v|-1, n = min(|Q_v|+1, |Q_d|)          */
+} eesd_config;
+
+/* Byte offsets inside the weight buffer.  A decoder layer holds, in this order:
+ *   g_attn f32[d] | wqkv [(H+2H_kv)D][d] (q heads, k heads, v heads) | wo [d][H*D] |
+ *   g_ffn f32[d]  | wgu [2F][d] (gate rows then up rows) | wd [d][F]
+ * matrices in the configured dtype, gains always fp32.  Target layer l starts at
+ * layer0 + l * layer_stride; the early-exit layer (Eq. 1, Transformer^e) at exit_layer. */
+typedef struct eesd_layout {
+    size_t embed;        /* [V][d] token embedding                                              */
+    size_t layer0, layer_stride;
+    size_t off_g_attn, off_wqkv, off_wo, off_g_ffn, off_wgu, off_wd; /* within a layer          */
+    size_t final_norm;   /* f32[d]                                                              */
+    size_t lm_head;      /* [V][d]                                                              */
+    size_t exit_layer;   /* one decoder layer                                                   */
+    size_t exit_norm;    /* f32[d], the RMSNorm before the exit head                            */
+    size_t exit_head;    /* [V][d]; equals lm_head when tie_exit_head                           */
+    size_t total_bytes;
+} eesd_layout;
+
+typedef struct eesd_sizes {
+    size_t weights_bytes;
+    size_t kv_page_bytes;   /* bytes of ONE page across all L+1 cache slots                     */
+    int64_t min_pages;      /* pages needed to hold max_ctx tokens                              */
+    size_t workspace_bytes;
+} eesd_sizes;
+
+/* Caller-owned device memory.  kv_pool holds P = floor(kv_bytes / kv_page_bytes) pages laid
+ * out [slot 0..L][page 0..P-1][K|V][H_kv][page_tokens][D]; slot L is the early-exit layer's
+ * cache.  The workspace must be zero-filled by the caller before eesd_init. */
+typedef struct eesd_buffers {
+    void *weights;   size_t weights_bytes;
+    void *kv_pool;   size_t kv_bytes;
+    void *workspace; size_t workspace_bytes;
+} eesd_buffers;
+
+/* Host arrays of uniforms in [0,1) of the form m * 2^-24 (random numbers are inputs, never
+ * drawn inside the library).  u_draft[p] / u_accept[p]: used when the token that would take
+ * context position p is drafted / tested; u_resample[p]: used by the round whose first
+ * drafted token takes position p; each needs max_ctx entries.  u_ctrl is consumed in order by
+ * the controller (alpha + beta + 1 values per decision). */
+typedef struct eesd_uniforms {
+    const float *u_draft, *u_accept, *u_resample;
+    const float *u_ctrl; int64_t n_ctrl;
+} eesd_uniforms;
+
+typedef struct eesd_round { int32_t k, n_accept, next_token; } eesd_round;
+
+/* Counters of one eesd_generate call.  v_d = accepted / drafted and r_d = accepted / emitted
+ * are the paper's acceptance rate and draft proportion (metrics paragraph of Sec. 4.1). */
+typedef struct eesd_stats {
+    int64_t rounds, drafted, accepted, emitted;
+    double ms_prefill, ms_draft, ms_verify, ms_total; /* device time, CUDA events               */
+    int64_t kernel_launches;
+    int64_t alpha, beta;                               /* posterior after the last round         */
+} eesd_stats;
+
+typedef struct eesd_ctx eesd_ctx;
+
+const char *eesd_strerror(int status);
+/* Text of the last CUDA error seen by this context (empty string if none). */
+const char *eesd_last_cuda_error(const eesd_ctx *ctx);
+
+/* Fills the weight-buffer layout for a configuration.  EESD_ERR_BADARG on invalid shapes. */
+int eesd_weight_layout(const eesd_config *cfg, eesd_layout *out);
+/* Sizes of the three device buffers eesd_init needs for a configuration. */
+int eesd_required_bytes(const eesd_config *cfg, eesd_sizes *out);
+
+/* Creates a context over caller-owned device buffers (weights already filled by the caller).
+ * `cuda_stream` is a cudaStream_t (borrowed; NULL = default stream).  Builds the rotary table
+ * and the KV page allocator; enqueues small set-up kernels on the stream.
+ * Errors: BADARG (shape), NOMEM (a buffer too small), UNSUPPORTED, CUDA. */
+int eesd_init(const eesd_config *cfg, const eesd_buffers *bufs, void *cuda_stream, eesd_ctx **out);
+/* Frees host state only. */
+int eesd_destroy(eesd_ctx *ctx);
+/* Forgets the sequence: context length 0, all KV pages free, posterior back to the prior. */
+int eesd_reset(eesd_ctx *ctx);
+
+/* Algorithm 1, initialisation of Q_g with the prompt: runs prompt tokens 0..n-2 through all L
+ * target layers (and writes the early-exit layer's keys/values for them), leaving the last
+ * prompt token pending, i.e. it is the first row of the next draft step and verify pass.
+ * `prompt` is a host pointer, borrowed for the call.  Resets the sequence first.
+ * Errors: BADARG (n_prompt < 1 or a token id outside [0, V)), CTX_FULL. */
+int eesd_prefill(eesd_ctx *ctx, const int32_t *prompt, int n_prompt);
+
+/* Algorithm 1, draft loop body (Eq. 1): k more draft steps of the current round.  Each step
+ * feeds the newest token through the first N layers (writing their shared KV rows) and the
+ * early-exit layer, and picks x_i = argmax q_i (temperature 0) or x_i ~ softmax(q_i / T) with
+ * uniform u_draft[i] (host array of k values, may be NULL when greedy).  The draft logits stay
+ * on the device for verification.  out_tokens (host, k entries, may be NULL) receives the
+ * tokens.  May be called repeatedly within a round, so a host controller can interleave.
+ * Errors: STATE (no prefill), CTX_FULL (round longer than k_cap or context full), RNG. */
+int eesd_draft(eesd_ctx *ctx, int k, const float *u_draft, int32_t *out_tokens);
+
+/* Algorithm 1, verification step with lossless acceptance: one pass of the K+1 rows
+ * (pending token, x_1..x_K) through all L layers against the KV cache, then for i = 1..K
+ * accept x_i iff u_accept[i-1] * q_i(x_i) < p_i(x_i); at the first rejection j the next token is
+ * drawn from normalize(max(0, p_j - q_j)), with no rejection from p_{K+1}, both with
+ * u_resample.  Greedy: accept while x_i = argmax p_i, next token = argmax of the first
+ * disagreeing row.  KV rows of rejected tokens are rolled back (pages past the end freed).
+ * Afterwards the context holds the accepted tokens plus next_token, which is pending.
+ * u_accept: host array of K values (may be NULL when greedy).  Errors: STATE (nothing drafted). */
+int eesd_verify_accept(eesd_ctx *ctx, const float *u_accept, float u_resample,
+                       int *n_accept, int32_t *next_token);
+
+/* Algorithm 1 end to end: prefill, then rounds of {draft until the controller stops or k_cap,
+ * verify, accept, posterior update (Eq. 3-4)} until max_new tokens exist; the output is cut to
+ * exactly max_new tokens.  k_schedule (host, may be NULL) forces the draft length of round r
+ * to k_schedule[r] for r < n_schedule (then the configured controller takes over).
+ * `u` may be NULL only for greedy decoding with a fixed K.  out: host, max_new entries.
+ * stats / trace / n_rounds may be NULL; trace receives at most trace_cap rounds.
+ * One host<->device synchronisation per round (to read n_accept and the next token). */
+int eesd_generate(eesd_ctx *ctx, const int32_t *prompt, int n_prompt, int max_new,
+                  const int32_t *k_schedule, int n_schedule, const eesd_uniforms *u,
+                  int32_t *out, eesd_stats *stats, eesd_round *trace, int trace_cap, int *n_rounds);
+
+/* ---- additions beyond the five calls above (testing and measurement) ---- */
+
+/* Context length in tokens (including the pending one), and KV pages in use. */
+int eesd_context_len(const eesd_ctx *ctx, int *n_tokens, int *pages_in_use);
+/* Posterior parameters of the controller. */
+int eesd_posterior(const eesd_ctx *ctx, int64_t *alpha, int64_t *beta);
+
+/* Declares that the KV cache already holds n_ctx - 1 valid rows (whatever bytes the pool
+ * contains) and that `pending` is the pending token: allocates pages, sets the length.  Used to
+ * time a verify pass against a cache of a chosen length without running a prefill. */
+int eesd_assume_context(eesd_ctx *ctx, int n_ctx, int32_t pending);
+
+/* One verification pass of M rows (tokens: host, M entries; row 0 replaces the pending token)
+ * at the current position WITHOUT acceptance: logits stay in the context (eesd_logits), the
+ * context length is unchanged afterwards.  The verify pass of Algorithm 1 at a forced M.
+ * Asynchronous: enqueues on the context's stream and returns. */
+int eesd_verify_only(eesd_ctx *ctx, const int32_t *tokens, int M);
+
+/* Device pointers of the fp32 logits of the last verify pass ([rows][V], which = 0) and of
+ * the current round's draft steps ([k][V], which = 1). */
+int eesd_logits(const eesd_ctx *ctx, int which, const float **device_ptr);
+
+/* When set (device buffer of (L + 2) * EESD_MAX_ROWS * d floats, or NULL to stop), every
+ * pass stores the residual stream after the embedding (index 0), after target layer l
+ * (index l + 1) and, in draft steps, after the early-exit layer (index L + 1) as
+ * [index][row][d] fp32. */
+int eesd_capture_hidden(eesd_ctx *ctx, float *device_buf, size_t bytes);
+
+/* Kernel launches issued by this context since creation. */
+int eesd_launch_count(const eesd_ctx *ctx, int64_t *n);
+
+/* Standalone fused softmax / accept / residual-resample over a batch of B independent
+ * sequences (the acceptance step of eesd_verify_accept).  All pointers are device pointers:
+ * p_logits [B][K+1][V] f32, q_logits [B][K][V] f32, tokens [B][K] i32 (the drafted x_i),
+ * u_accept [B][K], u_resample [B]; outputs n_accept [B], next_token [B] (i32).  scratch: at
+ * least eesd_accept_scratch_bytes(B, K) bytes.  Asynchronous on `cuda_stream`. */
+size_t eesd_accept_scratch_bytes(int B, int K);
+int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *q_logits,
+                         const int32_t *tokens, const float *u_accept, const float *u_resample,
+                         int B, int K, int V, float temperature, void *scratch, size_t scratch_bytes,
+                         int32_t *n_accept, int32_t *next_token);
+
+/* Draws one token per row: argmax (temperature 0) or x ~ softmax(logits / T) by inverse CDF
+ * with u[b].  logits [B][V] f32, u [B] (may be NULL when greedy), out [B] i32; device pointers. */
+int eesd_sample_rows(void *cuda_stream, const float *logits, const float *u, int B, int V,
+                     float temperature, int32_t *out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EESD_H */
