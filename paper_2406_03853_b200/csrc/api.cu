@@ -1,0 +1,746 @@
+// C ABI of the EESD decode-round library: context, KV page allocator, pass assembly,
+// generation loop (Algorithm 1) and the host-side Thompson-sampling controller (Algorithm 2).
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/eesd.h"
+#include "kernels.cuh"
+
+using namespace eesd;
+
+namespace {
+
+struct LayerW {
+    const float *g_attn, *g_ffn;
+    const char *wqkv, *wo, *wgu, *wd;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int check_config(const eesd_config *c) {
+    if (!c) return EESD_ERR_BADARG;
+    if (c->d_model <= 0 || c->n_heads <= 0 || c->n_kv_heads <= 0 || c->ffn_dim <= 0 || c->vocab <= 0 ||
+        c->n_layers <= 0 || c->max_ctx <= 1)
+        return EESD_ERR_BADARG;
+    if (c->n_heads % c->n_kv_heads) return EESD_ERR_BADARG;
+    if (c->n_early < 1 || c->n_early > c->n_layers) return EESD_ERR_BADARG;
+    if (c->dtype != EESD_F32 && c->dtype != EESD_BF16) return EESD_ERR_BADARG;
+    if (c->head_dim != 64 && c->head_dim != 128) return EESD_ERR_UNSUPPORTED;
+    if (c->d_model % 8 || c->ffn_dim % 8 || (c->n_heads * c->head_dim) % 8) return EESD_ERR_UNSUPPORTED;
+    if (c->page_tokens < 8 || (c->page_tokens & (c->page_tokens - 1))) return EESD_ERR_BADARG;
+    if (c->k_cap < 1 || c->k_cap > EESD_MAX_ROWS - 1) return EESD_ERR_BADARG;
+    if (c->temperature < 0.f) return EESD_ERR_BADARG;
+    if (c->controller != EESD_CTRL_FIXED_K && c->controller != EESD_CTRL_BETA_TS) return EESD_ERR_BADARG;
+    if (c->controller == EESD_CTRL_FIXED_K && c->fixed_k < 1) return EESD_ERR_BADARG;
+    if (c->alpha0 < 1 || c->beta0 < 1) return EESD_ERR_BADARG;
+    if (c->rms_eps < 0.f || c->rope_theta <= 1.f) return EESD_ERR_BADARG;
+    return EESD_OK;
+}
+
+struct Workspace {
+    size_t x, xn, q, attn, h, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
+        accept, total;
+};
+
+constexpr int kPartSplits = 8;   // room for K-split partial sums of one projection
+constexpr int kAttnSplits = 8;   // KV splits per head in attention
+constexpr int kIntSlots = 64;    // small device integer area
+
+Workspace carve(const eesd_config *c) {
+    Workspace w;
+    const size_t es = c->dtype == EESD_F32 ? 4 : 2;
+    const size_t R = EESD_MAX_ROWS;
+    const size_t qd = (size_t)c->n_heads * c->head_dim, kvd = (size_t)c->n_kv_heads * c->head_dim;
+    size_t maxR = qd + 2 * kvd;
+    if ((size_t)2 * c->ffn_dim > maxR) maxR = (size_t)2 * c->ffn_dim;
+    if ((size_t)c->vocab > maxR) maxR = c->vocab;
+    if ((size_t)c->d_model > maxR) maxR = c->d_model;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    w.x = take(R * c->d_model * 4);
+    w.xn = take(R * c->d_model * es);
+    w.q = take(R * qd * 4);
+    w.attn = take(R * qd * es);
+    w.h = take(R * (size_t)c->ffn_dim * es);
+    w.part = take((size_t)kPartSplits * R * maxR * 4);
+    w.apart = take((size_t)c->n_heads * kAttnSplits * R * (c->head_dim + 2) * 4);
+    w.logits_p = take(R * (size_t)c->vocab * 4);
+    w.logits_q = take(R * (size_t)c->vocab * 4);
+    w.rope = take((size_t)c->max_ctx * (c->head_dim / 2) * 8);
+    w.page_table = take(((size_t)c->max_ctx / c->page_tokens + 2) * 4);
+    w.ints = take(kIntSlots * 4);
+    w.u_dev = take((size_t)3 * c->max_ctx * 4);
+    w.u_stage = take(64 * 4);
+    w.err = take(16);
+    w.accept = take(accept_scratch_bytes(1, EESD_MAX_ROWS));
+    w.total = o;
+    return w;
+}
+
+// offsets inside the device integer area
+constexpr int kRoundTok = 0;   // [17]: pending token, then the round's draft tokens
+constexpr int kRowTok = 20;    // [16]: token rows of a prefill chunk / verify_only
+constexpr int kResult = 40;    // [2]: n_accept, next token
+
+}  // namespace
+
+struct eesd_ctx {
+    eesd_config cfg;
+    eesd_buffers buf;
+    eesd_layout lay;
+    cudaStream_t stream;
+    size_t es;
+    // device pointers
+    float *x, *q, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
+    void *xn, *attn, *h, *accept_scratch;
+    float2 *rope;
+    int32_t *page_table, *ints;
+    int *err;
+    std::vector<LayerW> layers;  // L target layers + exit layer at index L
+    const void *embed, *lm_head, *exit_head;
+    const float *g_final, *g_exit;
+    // KV pool
+    int64_t n_pages_total;
+    size_t slot_bytes;
+    std::vector<int32_t> free_pages, page_of;
+    // sequence state
+    std::vector<int32_t> tokens;
+    bool prefilled;
+    int round_k;
+    int64_t alpha, beta;
+    int64_t launches;
+    int32_t *h_result;  // pinned: [0] n_accept, [1] next token, [2] error word, [8..23] draft tokens
+    cudaEvent_t ev[5];  // prefill start / end, draft start, verify start, round end
+    char cuda_err[256];
+};
+
+namespace {
+
+#define CU(ctx, call)                                                                       \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess) {                                                            \
+            snprintf((ctx)->cuda_err, sizeof((ctx)->cuda_err), "%s: %s", #call, cudaGetErrorString(e_)); \
+            return EESD_ERR_CUDA;                                                           \
+        }                                                                                   \
+    } while (0)
+
+int check_launch(eesd_ctx *c) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        snprintf(c->cuda_err, sizeof(c->cuda_err), "kernel launch: %s", cudaGetErrorString(e));
+        return EESD_ERR_CUDA;
+    }
+    return EESD_OK;
+}
+
+KvGeom kv_geom(eesd_ctx *c, int slot) {
+    KvGeom g;
+    g.slot_base = (char *)c->buf.kv_pool + (size_t)slot * c->slot_bytes;
+    g.page_table = c->page_table;
+    g.Hkv = c->cfg.n_kv_heads;
+    g.D = c->cfg.head_dim;
+    g.page_tokens = c->cfg.page_tokens;
+    g.n_pages_total = (int)c->n_pages_total;
+    return g;
+}
+
+// make sure pages exist for `n_tokens` cache rows; pushes new table entries to the device
+int ensure_pages(eesd_ctx *c, int n_tokens) {
+    const int PT = c->cfg.page_tokens;
+    const int need = (n_tokens + PT - 1) / PT;
+    while ((int)c->page_of.size() < need) {
+        IntList16 l;
+        int first = (int)c->page_of.size(), n = 0;
+        while ((int)c->page_of.size() < need && n < 16) {
+            if (c->free_pages.empty()) return EESD_ERR_CTX_FULL;
+            int32_t p = c->free_pages.back();
+            c->free_pages.pop_back();
+            c->page_of.push_back(p);
+            l.v[n++] = p;
+        }
+        launch_set_ints(c->stream, c->page_table + first, l, n);
+        c->launches++;
+    }
+    return EESD_OK;
+}
+
+// give back pages that hold no valid row when only `n_tokens` rows are valid
+void trim_pages(eesd_ctx *c, int n_tokens) {
+    const int PT = c->cfg.page_tokens;
+    const int need = (n_tokens + PT - 1) / PT;
+    while ((int)c->page_of.size() > need) {
+        c->free_pages.push_back(c->page_of.back());
+        c->page_of.pop_back();
+    }
+}
+
+// one decoder layer on M rows at positions pos0.. ; on entry xn = RMSNorm(x) * g_attn of this
+// layer; on exit x holds the layer output and, when g_next is given, xn = RMSNorm(x) * g_next.
+void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const float *g_next, float *cap) {
+    const eesd_config &f = c->cfg;
+    const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim, d = f.d_model, F = f.ffn_dim;
+    cudaStream_t s = c->stream;
+    KvGeom kv = kv_geom(c, slot);
+    int S = launch_gemm(s, f.dtype, c->xn, w.wqkv, c->part, M, qd + 2 * kvd, d);
+    launch_qkv_post(s, f.dtype, c->part, S, M, pos0, f.n_heads, kv, c->rope, c->q, false, c->err);
+    launch_attention(s, f.dtype, c->q, kv, c->apart, c->attn, M, pos0, f.n_heads, kAttnSplits);
+    S = launch_gemm(s, f.dtype, c->attn, w.wo, c->part, M, d, qd);
+    launch_resid_norm(s, f.dtype, c->x, c->part, S, w.g_ffn, c->xn, nullptr, M, d, f.rms_eps);
+    S = launch_gemm(s, f.dtype, c->xn, w.wgu, c->part, M, 2 * F, d);
+    launch_swiglu(s, f.dtype, c->part, S, c->h, M, F);
+    S = launch_gemm(s, f.dtype, c->h, w.wd, c->part, M, d, F);
+    launch_resid_norm(s, f.dtype, c->x, c->part, S, g_next, c->xn, cap, M, d, f.rms_eps);
+    c->launches += 10;
+}
+
+float *cap_slot(eesd_ctx *c, int index) {
+    return c->capture ? c->capture + (size_t)index * EESD_MAX_ROWS * c->cfg.d_model : nullptr;
+}
+
+// Target model on M rows (device token ids) at positions pos0.. : all L layers, the exit
+// layer's keys/values after layer N, and (optionally) final norm + LM head into logits_p.
+int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_logits) {
+    const eesd_config &f = c->cfg;
+    cudaStream_t s = c->stream;
+    const int L = f.n_layers, d = f.d_model;
+    launch_embed(s, f.dtype, d_tok, c->embed, c->x, cap_slot(c, 0), M, d, f.vocab, c->err);
+    launch_resid_norm(s, f.dtype, c->x, nullptr, 0, c->layers[0].g_attn, c->xn, nullptr, M, d, f.rms_eps);
+    c->launches += 2;
+    for (int l = 0; l < L; l++) {
+        const bool exit_here = (l == f.n_early - 1);
+        const float *g_after = exit_here ? c->layers[L].g_attn : (l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
+        run_layer(c, c->layers[l], l, M, pos0, g_after, cap_slot(c, l + 1));
+        if (exit_here) {
+            // keys / values of the early-exit layer for these rows: they depend on H^N only
+            const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim;
+            const char *wkv = c->layers[L].wqkv + (size_t)qd * d * c->es;
+            int S = launch_gemm(s, f.dtype, c->xn, wkv, c->part, M, 2 * kvd, d);
+            launch_qkv_post(s, f.dtype, c->part, S, M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err);
+            const float *g_next = l + 1 < L ? c->layers[l + 1].g_attn : c->g_final;
+            launch_resid_norm(s, f.dtype, c->x, nullptr, 0, g_next, c->xn, nullptr, M, d, f.rms_eps);
+            c->launches += 3;
+        }
+    }
+    if (want_logits) {
+        int S = launch_gemm(s, f.dtype, c->xn, c->lm_head, c->part, M, f.vocab, d);
+        launch_reduce_partials(s, c->part, S, c->logits_p, M, f.vocab);
+        c->launches += 2;
+    }
+    return check_launch(c);
+}
+
+// Draft model (Eq. 1) on one row: token ints[kRoundTok + i] at position pos, logits into
+// logits_q[i], chosen token into ints[kRoundTok + i + 1].
+int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
+    const eesd_config &f = c->cfg;
+    cudaStream_t s = c->stream;
+    const int L = f.n_layers, d = f.d_model, N = f.n_early;
+    launch_embed(s, f.dtype, c->ints + kRoundTok + i, c->embed, c->x, cap_slot(c, 0), 1, d, f.vocab, c->err);
+    launch_resid_norm(s, f.dtype, c->x, nullptr, 0, c->layers[0].g_attn, c->xn, nullptr, 1, d, f.rms_eps);
+    for (int l = 0; l < N; l++) {
+        const float *g_after = l + 1 < N ? c->layers[l + 1].g_attn : c->layers[L].g_attn;
+        run_layer(c, c->layers[l], l, 1, pos, g_after, cap_slot(c, l + 1));
+    }
+    run_layer(c, c->layers[L], L, 1, pos, c->g_exit, cap_slot(c, L + 1));
+    float *lq = c->logits_q + (size_t)i * f.vocab;
+    int S = launch_gemm(s, f.dtype, c->xn, c->exit_head, c->part, 1, f.vocab, d);
+    launch_reduce_partials(s, c->part, S, lq, 1, f.vocab);
+    launch_sample_rows(s, lq, d_u, 1, f.vocab, f.temperature, c->ints + kRoundTok + i + 1);
+    c->launches += 5;
+    return check_launch(c);
+}
+
+int set_device_ints(eesd_ctx *c, int slot, const int32_t *vals, int n) {
+    IntList16 l;
+    for (int i = 0; i < n; i++) l.v[i] = vals[i];
+    launch_set_ints(c->stream, c->ints + slot, l, n);
+    c->launches++;
+    return check_launch(c);
+}
+
+int read_error_word(eesd_ctx *c) {
+    // h_result[2] was copied from the device error word together with the round result
+    return c->h_result[2] ? EESD_ERR_DEVICE : EESD_OK;
+}
+
+// theta ~ Beta(alpha, beta) through two Gamma sums of -ln u, chi ~ Bernoulli(theta)
+int ts_continue(eesd_ctx *c, const eesd_uniforms *u, int64_t *cursor) {
+    if (!u || !u->u_ctrl) return EESD_ERR_RNG;
+    if (*cursor + c->alpha + c->beta + 1 > u->n_ctrl) return EESD_ERR_RNG;
+    auto nl = [](float v) { return -log(v > 0.0f ? (double)v : 2.98023223876953125e-08); };
+    double X = 0.0, Y = 0.0;
+    for (int64_t i = 0; i < c->alpha; i++) X += nl(u->u_ctrl[(*cursor)++]);
+    for (int64_t i = 0; i < c->beta; i++) Y += nl(u->u_ctrl[(*cursor)++]);
+    const double theta = X / (X + Y);
+    return (double)u->u_ctrl[(*cursor)++] < theta ? 1 : 0;
+}
+
+// Eq. 3-4 with r = |Q_v| - 1 and n = min(|Q_v| + 1, |Q_d|) (Algorithm 2, update steps)
+void ts_update(eesd_ctx *c, int q_v, int n_draft) {
+    const int64_t r = q_v - 1;
+    int64_t n = c->cfg.ts_update_rule == EESD_TS_RULE_PAPER ? (q_v + 1 < n_draft ? q_v + 1 : n_draft)
+                                                            : (q_v < n_draft ? q_v : n_draft);
+    if (n < r) n = r;
+    c->alpha += r;
+    c->beta += n - r;
+}
+
+void reset_sequence(eesd_ctx *c) {
+    trim_pages(c, 0);
+    c->tokens.clear();
+    c->prefilled = false;
+    c->round_k = 0;
+    c->alpha = c->cfg.alpha0;
+    c->beta = c->cfg.beta0;
+}
+
+int prefill_impl(eesd_ctx *c, const int32_t *prompt, int n_prompt) {
+    if (!prompt || n_prompt < 1) return EESD_ERR_BADARG;
+    if (n_prompt >= c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
+    for (int i = 0; i < n_prompt; i++)
+        if (prompt[i] < 0 || prompt[i] >= c->cfg.vocab) return EESD_ERR_BADARG;
+    reset_sequence(c);
+    int st = ensure_pages(c, n_prompt);
+    if (st) return st;
+    for (int p = 0; p < n_prompt - 1; p += EESD_MAX_ROWS) {
+        int M = n_prompt - 1 - p;
+        if (M > EESD_MAX_ROWS) M = EESD_MAX_ROWS;
+        st = set_device_ints(c, kRowTok, prompt + p, M);
+        if (st) return st;
+        st = run_target(c, c->ints + kRowTok, M, p, false);
+        if (st) return st;
+    }
+    st = set_device_ints(c, kRoundTok, prompt + n_prompt - 1, 1);
+    if (st) return st;
+    c->tokens.assign(prompt, prompt + n_prompt);
+    c->prefilled = true;
+    return EESD_OK;
+}
+
+// draft steps round_k .. round_k + k - 1 of the current round; d_u: device uniforms, one per step
+int draft_impl(eesd_ctx *c, int k, const float *d_u, int u_stride) {
+    const int T = (int)c->tokens.size();
+    if (c->round_k + k > c->cfg.k_cap) return EESD_ERR_CTX_FULL;
+    if (T + c->round_k + k > c->cfg.max_ctx - 1) return EESD_ERR_CTX_FULL;
+    int st = ensure_pages(c, T + c->round_k + k);
+    if (st) return st;
+    for (int j = 0; j < k; j++) {
+        const int i = c->round_k;
+        st = run_draft_step(c, i, T - 1 + i, d_u ? d_u + (size_t)j * u_stride : nullptr);
+        if (st) return st;
+        c->round_k++;
+    }
+    return EESD_OK;
+}
+
+// verify pass + acceptance; leaves (n_accept, next token, error word) in h_result after a sync
+int verify_impl(eesd_ctx *c, const float *d_u_acc, const float *d_u_res) {
+    const eesd_config &f = c->cfg;
+    const int T = (int)c->tokens.size(), K = c->round_k;
+    int st = ensure_pages(c, T + K);
+    if (st) return st;
+    st = run_target(c, c->ints + kRoundTok, K + 1, T - 1, true);
+    if (st) return st;
+    launch_accept(c->stream, c->logits_p, c->logits_q, c->ints + kRoundTok + 1, d_u_acc, d_u_res, 1, K, f.vocab,
+                  f.temperature, c->accept_scratch, c->ints + kResult, c->ints + kResult + 1, c->ints + kRoundTok);
+    c->launches++;
+    st = check_launch(c);
+    if (st) return st;
+    CU(c, cudaMemcpyAsync(c->h_result, c->ints + kResult, 8, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaMemcpyAsync(c->h_result + 2, c->err, 4, cudaMemcpyDeviceToHost, c->stream));
+    return EESD_OK;
+}
+
+// host bookkeeping after the round's result has arrived
+int finish_round(eesd_ctx *c, const int32_t *draft_tokens_host, int *n_accept, int32_t *next) {
+    const int K = c->round_k;
+    const int a = c->h_result[0], y = c->h_result[1];
+    if (read_error_word(c)) return EESD_ERR_DEVICE;
+    if (a < 0 || a > K || y < 0 || y >= c->cfg.vocab) return EESD_ERR_DEVICE;
+    for (int i = 0; i < a; i++) c->tokens.push_back(draft_tokens_host[i]);
+    c->tokens.push_back(y);
+    c->round_k = 0;
+    trim_pages(c, (int)c->tokens.size() - 1);  // rows of rejected tokens are dropped
+    if (n_accept) *n_accept = a;
+    if (next) *next = y;
+    return EESD_OK;
+}
+
+}  // namespace
+
+// =====================================================================================  C ABI
+extern "C" {
+
+const char *eesd_strerror(int status) {
+    switch (status) {
+        case EESD_OK: return "ok";
+        case EESD_ERR_BADARG: return "bad argument";
+        case EESD_ERR_NOMEM: return "caller-provided buffer too small";
+        case EESD_ERR_CUDA: return "CUDA runtime error";
+        case EESD_ERR_STATE: return "call not valid in the current state";
+        case EESD_ERR_CTX_FULL: return "context, round or KV page pool full";
+        case EESD_ERR_RNG: return "uniform stream missing or exhausted";
+        case EESD_ERR_DEVICE: return "device-side error word set";
+        case EESD_ERR_UNSUPPORTED: return "unsupported shape";
+        default: return "unknown status";
+    }
+}
+
+const char *eesd_last_cuda_error(const eesd_ctx *ctx) { return ctx ? ctx->cuda_err : ""; }
+
+int eesd_weight_layout(const eesd_config *c, eesd_layout *out) {
+    int st = check_config(c);
+    if (st) return st;
+    if (!out) return EESD_ERR_BADARG;
+    const size_t es = c->dtype == EESD_F32 ? 4 : 2;
+    const size_t d = c->d_model, F = c->ffn_dim, V = c->vocab;
+    const size_t qd = (size_t)c->n_heads * c->head_dim, kvd = (size_t)c->n_kv_heads * c->head_dim;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    out->off_g_attn = take(d * 4);
+    out->off_wqkv = take((qd + 2 * kvd) * d * es);
+    out->off_wo = take(d * qd * es);
+    out->off_g_ffn = take(d * 4);
+    out->off_wgu = take(2 * F * d * es);
+    out->off_wd = take(d * F * es);
+    out->layer_stride = o;
+    o = 0;
+    out->embed = take(V * d * es);
+    out->layer0 = o;
+    o += out->layer_stride * (size_t)c->n_layers;
+    out->final_norm = take(d * 4);
+    out->lm_head = take(V * d * es);
+    out->exit_layer = o;
+    o += out->layer_stride;
+    out->exit_norm = take(d * 4);
+    out->exit_head = c->tie_exit_head ? out->lm_head : take(V * d * es);
+    out->total_bytes = o;
+    return EESD_OK;
+}
+
+int eesd_required_bytes(const eesd_config *c, eesd_sizes *out) {
+    eesd_layout lay;
+    int st = eesd_weight_layout(c, &lay);
+    if (st) return st;
+    if (!out) return EESD_ERR_BADARG;
+    const size_t es = c->dtype == EESD_F32 ? 4 : 2;
+    out->weights_bytes = lay.total_bytes;
+    out->kv_page_bytes = (size_t)(c->n_layers + 1) * 2 * c->n_kv_heads * c->page_tokens * c->head_dim * es;
+    out->min_pages = (c->max_ctx + c->page_tokens - 1) / c->page_tokens;
+    out->workspace_bytes = carve(c).total;
+    return EESD_OK;
+}
+
+int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, eesd_ctx **out) {
+    eesd_layout lay;
+    eesd_sizes sz;
+    int st = eesd_required_bytes(cfg, &sz);
+    if (st) return st;
+    eesd_weight_layout(cfg, &lay);
+    if (!b || !out || !b->weights || !b->kv_pool || !b->workspace) return EESD_ERR_BADARG;
+    if (b->weights_bytes < sz.weights_bytes || b->workspace_bytes < sz.workspace_bytes) return EESD_ERR_NOMEM;
+    const int64_t pages = (int64_t)(b->kv_bytes / sz.kv_page_bytes);
+    if (pages < sz.min_pages) return EESD_ERR_NOMEM;
+    eesd_ctx *c = new (std::nothrow) eesd_ctx();
+    if (!c) return EESD_ERR_NOMEM;
+    c->cfg = *cfg;
+    c->buf = *b;
+    c->lay = lay;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->es = cfg->dtype == EESD_F32 ? 4 : 2;
+    c->cuda_err[0] = 0;
+    c->capture = nullptr;
+    c->launches = 0;
+    c->n_pages_total = pages > 0x7fffffff ? 0x7fffffff : pages;
+    c->slot_bytes = (size_t)c->n_pages_total * 2 * cfg->n_kv_heads * cfg->page_tokens * cfg->head_dim * c->es;
+    Workspace w = carve(cfg);
+    char *ws = (char *)b->workspace;
+    c->x = (float *)(ws + w.x); c->xn = ws + w.xn; c->q = (float *)(ws + w.q); c->attn = ws + w.attn;
+    c->h = ws + w.h; c->part = (float *)(ws + w.part); c->apart = (float *)(ws + w.apart);
+    c->logits_p = (float *)(ws + w.logits_p); c->logits_q = (float *)(ws + w.logits_q);
+    c->rope = (float2 *)(ws + w.rope); c->page_table = (int32_t *)(ws + w.page_table);
+    c->ints = (int32_t *)(ws + w.ints); c->u_dev = (float *)(ws + w.u_dev); c->u_stage = (float *)(ws + w.u_stage);
+    c->err = (int *)(ws + w.err); c->accept_scratch = ws + w.accept;
+    const char *wb = (const char *)b->weights;
+    c->layers.resize(cfg->n_layers + 1);
+    for (int l = 0; l <= cfg->n_layers; l++) {
+        const char *base = wb + (l < cfg->n_layers ? lay.layer0 + (size_t)l * lay.layer_stride : lay.exit_layer);
+        LayerW &lw = c->layers[l];
+        lw.g_attn = (const float *)(base + lay.off_g_attn); lw.wqkv = base + lay.off_wqkv; lw.wo = base + lay.off_wo;
+        lw.g_ffn = (const float *)(base + lay.off_g_ffn); lw.wgu = base + lay.off_wgu; lw.wd = base + lay.off_wd;
+    }
+    c->embed = wb + lay.embed; c->lm_head = wb + lay.lm_head; c->exit_head = wb + lay.exit_head;
+    c->g_final = (const float *)(wb + lay.final_norm); c->g_exit = (const float *)(wb + lay.exit_norm);
+    // free list in descending order: the first pages handed out are the highest, so logical
+    // and physical page numbers differ and the page table is really exercised
+    for (int64_t p = 0; p < c->n_pages_total; p++) c->free_pages.push_back((int32_t)p);
+    reset_sequence(c);
+    c->h_result = nullptr;
+    for (auto &e : c->ev) e = nullptr;
+    cudaError_t e = cudaHostAlloc((void **)&c->h_result, 256, cudaHostAllocDefault);
+    for (int i = 0; i < 5 && e == cudaSuccess; i++) e = cudaEventCreate(&c->ev[i]);
+    if (e != cudaSuccess) {
+        eesd_destroy(c);
+        return EESD_ERR_CUDA;
+    }
+    memset(c->h_result, 0, 256);
+    cudaMemsetAsync(c->err, 0, 16, c->stream);
+    cudaMemsetAsync(c->ints, 0, kIntSlots * 4, c->stream);
+    cudaMemsetAsync(c->accept_scratch, 0, accept_scratch_bytes(1, EESD_MAX_ROWS), c->stream);
+    launch_rope_table(c->stream, c->rope, cfg->max_ctx, cfg->head_dim, cfg->rope_theta);
+    c->launches++;
+    st = check_launch(c);
+    if (st) {
+        eesd_destroy(c);
+        return st;
+    }
+    *out = c;
+    return EESD_OK;
+}
+
+int eesd_destroy(eesd_ctx *c) {
+    if (!c) return EESD_OK;
+    if (c->h_result) cudaFreeHost(c->h_result);
+    for (auto &e : c->ev)
+        if (e) cudaEventDestroy(e);
+    delete c;
+    return EESD_OK;
+}
+
+int eesd_reset(eesd_ctx *c) {
+    if (!c) return EESD_ERR_BADARG;
+    reset_sequence(c);
+    return EESD_OK;
+}
+
+int eesd_prefill(eesd_ctx *c, const int32_t *prompt, int n_prompt) {
+    if (!c) return EESD_ERR_BADARG;
+    int st = prefill_impl(c, prompt, n_prompt);
+    if (st) return st;
+    CU(c, cudaMemcpyAsync(c->h_result + 2, c->err, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    return read_error_word(c);
+}
+
+int eesd_draft(eesd_ctx *c, int k, const float *u_draft, int32_t *out_tokens) {
+    if (!c || k < 1) return EESD_ERR_BADARG;
+    if (!c->prefilled) return EESD_ERR_STATE;
+    if (c->round_k + k > c->cfg.k_cap) return EESD_ERR_CTX_FULL;
+    const bool greedy = c->cfg.temperature == 0.f;
+    if (!greedy && !u_draft) return EESD_ERR_RNG;
+    const int first = c->round_k;
+    float *d_u = nullptr;
+    if (!greedy) {
+        d_u = c->u_stage + first;
+        CU(c, cudaMemcpyAsync(d_u, u_draft, (size_t)k * 4, cudaMemcpyHostToDevice, c->stream));
+    }
+    int st = draft_impl(c, k, d_u, 1);
+    if (st) return st;
+    if (out_tokens) {
+        CU(c, cudaMemcpyAsync(out_tokens, c->ints + kRoundTok + 1 + first, (size_t)k * 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(c, cudaStreamSynchronize(c->stream));
+    }
+    return EESD_OK;
+}
+
+int eesd_verify_accept(eesd_ctx *c, const float *u_accept, float u_resample, int *n_accept, int32_t *next_token) {
+    if (!c) return EESD_ERR_BADARG;
+    if (!c->prefilled || c->round_k < 1) return EESD_ERR_STATE;
+    const bool greedy = c->cfg.temperature == 0.f;
+    if (!greedy && !u_accept) return EESD_ERR_RNG;
+    const int K = c->round_k;
+    float *d_acc = c->u_stage + 16, *d_res = c->u_stage + 32;
+    if (!greedy) {
+        CU(c, cudaMemcpyAsync(d_acc, u_accept, (size_t)K * 4, cudaMemcpyHostToDevice, c->stream));
+        CU(c, cudaMemcpyAsync(d_res, &u_resample, 4, cudaMemcpyHostToDevice, c->stream));
+    }
+    int32_t *drafts = c->h_result + 8;
+    int st = verify_impl(c, d_acc, d_res);
+    if (st) return st;
+    CU(c, cudaMemcpyAsync(drafts, c->ints + kRoundTok + 1, (size_t)K * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    return finish_round(c, drafts, n_accept, next_token);
+}
+
+int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new, const int32_t *k_schedule,
+                  int n_schedule, const eesd_uniforms *u, int32_t *out, eesd_stats *stats, eesd_round *trace,
+                  int trace_cap, int *n_rounds) {
+    if (!c || !out || max_new < 1) return EESD_ERR_BADARG;
+    const eesd_config &f = c->cfg;
+    const bool greedy = f.temperature == 0.f;
+    if (!greedy && (!u || !u->u_draft || !u->u_accept || !u->u_resample)) return EESD_ERR_RNG;
+    if (f.controller == EESD_CTRL_BETA_TS && (!u || !u->u_ctrl)) return EESD_ERR_RNG;
+    if (n_prompt + max_new + 1 > f.max_ctx) return EESD_ERR_CTX_FULL;
+    const int64_t launches0 = c->launches;
+    float *d_ud = c->u_dev, *d_ua = c->u_dev + f.max_ctx, *d_ur = c->u_dev + 2 * (size_t)f.max_ctx;
+    if (!greedy) {
+        CU(c, cudaMemcpyAsync(d_ud, u->u_draft, (size_t)f.max_ctx * 4, cudaMemcpyHostToDevice, c->stream));
+        CU(c, cudaMemcpyAsync(d_ua, u->u_accept, (size_t)f.max_ctx * 4, cudaMemcpyHostToDevice, c->stream));
+        CU(c, cudaMemcpyAsync(d_ur, u->u_resample, (size_t)f.max_ctx * 4, cudaMemcpyHostToDevice, c->stream));
+    }
+    CU(c, cudaEventRecord(c->ev[0], c->stream));
+    int st = prefill_impl(c, prompt, n_prompt);
+    if (st) return st;
+    CU(c, cudaEventRecord(c->ev[1], c->stream));
+    eesd_stats sacc;
+    memset(&sacc, 0, sizeof(sacc));
+    int64_t cursor = 0;
+    int t = 0, rounds = 0;
+    int32_t *drafts = c->h_result + 8;
+    float ms_p = 0.f;
+    while (t < max_new) {
+        const int T = (int)c->tokens.size();
+        // draft length of this round: the controller's decisions depend on the posterior only,
+        // so they are taken before the round is enqueued (Algorithm 2, draft loop)
+        int cap = f.k_cap;
+        if (f.max_ctx - 1 - T < cap) cap = f.max_ctx - 1 - T;
+        if (cap < 1) return EESD_ERR_CTX_FULL;
+        int K;
+        if (k_schedule && rounds < n_schedule) K = k_schedule[rounds];
+        else if (f.controller == EESD_CTRL_FIXED_K) K = f.fixed_k;
+        else {
+            K = 1;
+            while (K < cap) {
+                int chi = ts_continue(c, u, &cursor);
+                if (chi < 0) return chi;
+                if (!chi) break;
+                K++;
+            }
+        }
+        if (K < 1) K = 1;
+        if (K > cap) K = cap;
+        CU(c, cudaEventRecord(c->ev[2], c->stream));
+        st = draft_impl(c, K, greedy ? nullptr : d_ud + T, 1);
+        if (st) return st;
+        CU(c, cudaEventRecord(c->ev[3], c->stream));
+        st = verify_impl(c, d_ua + T, d_ur + T);
+        if (st) return st;
+        CU(c, cudaMemcpyAsync(drafts, c->ints + kRoundTok + 1, (size_t)K * 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(c, cudaEventRecord(c->ev[4], c->stream));
+        CU(c, cudaStreamSynchronize(c->stream));
+        int a;
+        int32_t y;
+        st = finish_round(c, drafts, &a, &y);
+        if (st) return st;
+        float ms_d = 0.f, ms_v = 0.f;
+        cudaEventElapsedTime(&ms_d, c->ev[2], c->ev[3]);
+        cudaEventElapsedTime(&ms_v, c->ev[3], c->ev[4]);
+        if (rounds == 0) cudaEventElapsedTime(&ms_p, c->ev[0], c->ev[1]);
+        sacc.ms_draft += ms_d;
+        sacc.ms_verify += ms_v;
+        sacc.drafted += K;
+        sacc.accepted += a;
+        ts_update(c, a + 1, K);
+        if (trace && rounds < trace_cap) { trace[rounds].k = K; trace[rounds].n_accept = a; trace[rounds].next_token = y; }
+        t += a + 1;
+        rounds++;
+    }
+    for (int i = 0; i < max_new; i++) out[i] = c->tokens[n_prompt + i];
+    if (n_rounds) *n_rounds = rounds;
+    if (stats) {
+        sacc.rounds = rounds;
+        sacc.emitted = max_new;
+        sacc.ms_prefill = ms_p;
+        sacc.ms_total = sacc.ms_prefill + sacc.ms_draft + sacc.ms_verify;
+        sacc.kernel_launches = c->launches - launches0;
+        sacc.alpha = c->alpha;
+        sacc.beta = c->beta;
+        *stats = sacc;
+    }
+    return EESD_OK;
+}
+
+int eesd_context_len(const eesd_ctx *c, int *n_tokens, int *pages_in_use) {
+    if (!c) return EESD_ERR_BADARG;
+    if (n_tokens) *n_tokens = (int)c->tokens.size();
+    if (pages_in_use) *pages_in_use = (int)c->page_of.size();
+    return EESD_OK;
+}
+
+int eesd_posterior(const eesd_ctx *c, int64_t *alpha, int64_t *beta) {
+    if (!c) return EESD_ERR_BADARG;
+    if (alpha) *alpha = c->alpha;
+    if (beta) *beta = c->beta;
+    return EESD_OK;
+}
+
+int eesd_assume_context(eesd_ctx *c, int n_ctx, int32_t pending) {
+    if (!c || n_ctx < 1 || pending < 0 || pending >= c->cfg.vocab) return EESD_ERR_BADARG;
+    if (n_ctx >= c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
+    reset_sequence(c);
+    int st = ensure_pages(c, n_ctx);
+    if (st) return st;
+    c->tokens.assign(n_ctx, 0);
+    c->tokens[n_ctx - 1] = pending;
+    st = set_device_ints(c, kRoundTok, &pending, 1);
+    if (st) return st;
+    c->prefilled = true;
+    return EESD_OK;
+}
+
+int eesd_verify_only(eesd_ctx *c, const int32_t *tokens, int M) {
+    if (!c || !tokens || M < 1 || M > EESD_MAX_ROWS) return EESD_ERR_BADARG;
+    if (!c->prefilled) return EESD_ERR_STATE;
+    const int T = (int)c->tokens.size();
+    if (T - 1 + M > c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
+    int st = ensure_pages(c, T - 1 + M);
+    if (st) return st;
+    st = set_device_ints(c, kRowTok, tokens, M);
+    if (st) return st;
+    return run_target(c, c->ints + kRowTok, M, T - 1, true);
+}
+
+int eesd_logits(const eesd_ctx *c, int which, const float **device_ptr) {
+    if (!c || !device_ptr || (which != 0 && which != 1)) return EESD_ERR_BADARG;
+    *device_ptr = which == 0 ? c->logits_p : c->logits_q;
+    return EESD_OK;
+}
+
+int eesd_capture_hidden(eesd_ctx *c, float *device_buf, size_t bytes) {
+    if (!c) return EESD_ERR_BADARG;
+    if (device_buf && bytes < (size_t)(c->cfg.n_layers + 2) * EESD_MAX_ROWS * c->cfg.d_model * 4) return EESD_ERR_NOMEM;
+    c->capture = device_buf;
+    return EESD_OK;
+}
+
+int eesd_launch_count(const eesd_ctx *c, int64_t *n) {
+    if (!c || !n) return EESD_ERR_BADARG;
+    *n = c->launches;
+    return EESD_OK;
+}
+
+size_t eesd_accept_scratch_bytes(int B, int K) {
+    if (B < 1 || K < 1) return 0;
+    return accept_scratch_bytes(B, K);
+}
+
+int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *q_logits, const int32_t *tokens,
+                         const float *u_accept, const float *u_resample, int B, int K, int V, float temperature,
+                         void *scratch, size_t scratch_bytes, int32_t *n_accept, int32_t *next_token) {
+    if (!p_logits || !q_logits || !tokens || !scratch || !n_accept || !next_token) return EESD_ERR_BADARG;
+    if (B < 1 || K < 1 || V < 1 || temperature < 0.f) return EESD_ERR_BADARG;
+    if (temperature != 0.f && (!u_accept || !u_resample)) return EESD_ERR_RNG;
+    if ((long long)B * (2 * K + 1) > 0x7fffffffLL) return EESD_ERR_UNSUPPORTED;
+    const size_t need = accept_scratch_bytes(B, K);
+    if (scratch_bytes < need) return EESD_ERR_NOMEM;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(scratch, 0, need, s) != cudaSuccess) return EESD_ERR_CUDA;
+    launch_accept(s, p_logits, q_logits, tokens, u_accept, u_resample, B, K, V, temperature, scratch, n_accept,
+                  next_token, nullptr);
+    return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
+}
+
+int eesd_sample_rows(void *cuda_stream, const float *logits, const float *u, int B, int V, float temperature,
+                     int32_t *out) {
+    if (!logits || !out || B < 1 || V < 1 || temperature < 0.f) return EESD_ERR_BADARG;
+    if (temperature != 0.f && !u) return EESD_ERR_RNG;
+    launch_sample_rows((cudaStream_t)cuda_stream, logits, u, B, V, temperature, out);
+    return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
+}
+
+}  // extern "C"

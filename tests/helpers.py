@@ -21,3 +21,42 @@ def np_softmax(x):
     x = np.asarray(x, np.float64)
     e = np.exp(x - x.max(-1, keepdims=True))
     return e / e.sum(-1, keepdims=True)
+
+
+# ------------------------------------------------------------------ CUDA engine from a spec
+def config_from_spec(spec, n_layers=None, **kw):
+    from paper_2406_03853_b200 import binding as b
+    L = spec.n_layers if n_layers is None else n_layers
+    return b.make_config(d_model=spec.d_model, n_heads=spec.n_heads, n_kv_heads=spec.n_kv_heads,
+                         head_dim=spec.head_dim, ffn_dim=spec.ffn_dim, vocab=spec.vocab, n_layers=L,
+                         n_early=min(spec.n_early, L), dtype=spec.dtype, tie_exit_head=spec.tie_exit_head,
+                         rms_eps=spec.rms_eps, rope_theta=spec.rope_theta, **kw)
+
+
+def fill_engine(engine, spec, seed=synth.SEED):
+    """Writes the synthetic weights of `spec` into the engine's weight buffer (generated on
+    the engine's device by the shared generator, so the oracle sees the same bits)."""
+    dev = engine.device
+    L = engine.cfg.n_layers
+    for l in range(L):
+        views = engine.layer_views(l)
+        for k, v in synth.layer_weights(spec, l, seed, dev).items():
+            views[k].copy_(v)
+    views = engine.layer_views(L)
+    for k, v in synth.exit_layer_weights(spec, seed, dev).items():
+        views[k].copy_(v)
+    g = engine.global_views()
+    g["embed"].copy_(synth.embedding(spec, seed, dev))
+    head = synth.lm_head(spec, seed, dev)
+    g["lm_head"].copy_(head)
+    if not engine.cfg.tie_exit_head:
+        g["exit_head"].copy_(head)
+    g["g_final"].fill_(1.0)
+    g["g_exit"].fill_(1.0)
+
+
+def engine_from_spec(spec, n_layers=None, seed=synth.SEED, kv_pages=None, **kw):
+    from paper_2406_03853_b200 import Engine
+    eng = Engine(config_from_spec(spec, n_layers, **kw), kv_pages=kv_pages)
+    fill_engine(eng, spec, seed)
+    return eng

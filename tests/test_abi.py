@@ -1,0 +1,64 @@
+"""The C-ABI library loads and exports every symbol include/eesd.h declares; host-side
+argument checking works without a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2406_03853_b200 import build
+    build.build()
+    import paper_2406_03853_b200 as eesd
+    return eesd.lib()
+
+
+def test_every_declared_symbol_is_exported(L):
+    hdr = open(os.path.join(ROOT, "include", "eesd.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    names = set(re.findall(r"\b(eesd_[a-z_]+)\s*\(", hdr))
+    assert {"eesd_init", "eesd_prefill", "eesd_draft", "eesd_verify_accept", "eesd_generate"} <= names
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_layout_sizes_and_config_checks(L):
+    from paper_2406_03853_b200 import binding as b
+    import eesd_synth as synth
+    from tests.helpers import config_from_spec
+    for spec in (synth.TINY, synth.LLAMA2_13B, synth.LLAMA2_70B):
+        cfg = config_from_spec(spec, max_ctx=1536)
+        lay, sz = b.Layout(), b.Sizes()
+        assert L.eesd_weight_layout(C.byref(cfg), C.byref(lay)) == 0
+        assert L.eesd_required_bytes(C.byref(cfg), C.byref(sz)) == 0
+        es = 4 if spec.dtype == "f32" else 2
+        params = (spec.n_layers + 1) * spec.layer_params + (2 if spec.tie_exit_head else 3) * spec.vocab * spec.d_model
+        assert params * es <= sz.weights_bytes <= params * es * 1.001 + (1 << 20)
+        assert sz.kv_page_bytes == (spec.n_layers + 1) * 2 * spec.kv_dim * 16 * es
+        assert sz.min_pages == 96
+        assert (lay.exit_head == lay.lm_head) == spec.tie_exit_head
+    bad = config_from_spec(synth.TINY)
+    bad.n_kv_heads = 3
+    assert L.eesd_weight_layout(C.byref(bad), C.byref(lay)) == -1
+    bad = config_from_spec(synth.TINY)
+    bad.head_dim = 80
+    assert L.eesd_required_bytes(C.byref(bad), C.byref(sz)) == -8
+    bad = config_from_spec(synth.TINY, k_cap=16)
+    assert L.eesd_required_bytes(C.byref(bad), C.byref(sz)) == -1
+    assert L.eesd_strerror(-5).decode().startswith("context")
+    assert L.eesd_prefill(None, None, 0) == -1 and L.eesd_generate(None, None, 0, 0, None, 0, None, None, None, None, 0, None) == -1
+
+
+def test_binding_refuses_to_run_without_cuda():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("CUDA present")
+    import paper_2406_03853_b200 as eesd
+    from tests.helpers import config_from_spec
+    import eesd_synth as synth
+    with pytest.raises(RuntimeError):
+        eesd.Engine(config_from_spec(synth.TINY))

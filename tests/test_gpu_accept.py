@@ -1,0 +1,72 @@
+"""GPU parity: fused softmax / accept / residual-resample kernel and the draft sampler against
+the CPU oracle, bit-exact on identical logits and uniforms (accept sweep configuration)."""
+import numpy as np
+import pytest
+import torch
+
+import eesd_synth as synth
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+CASES = [(s, d) for s in (1.0, 3.0) for d in (0.1, 1.0, 3.0)]
+
+
+def _run_case(case, B, K, V, sigma, delta, T):
+    import paper_2406_03853_b200 as eesd
+    p, q, ua, ur, ud = synth.accept_case(case, B, K, V, sigma, delta, device="cuda")
+    # draft tokens x_i ~ q_i by the sampler under test, checked against the oracle's sampler
+    x = eesd.sample_rows(q.view(B * K, V), ud.view(B * K), T).view(B, K)
+    qc, udc = q.cpu().numpy(), ud.cpu().numpy()
+    if T == 0.0:
+        x_ref = qc.reshape(B * K, V).argmax(1)
+    else:
+        x_ref = np.array([oracle.sample_logits(qc[b, i], T, float(udc[b, i])) for b in range(B) for i in range(K)])
+    np.testing.assert_array_equal(x.cpu().numpy().reshape(-1), x_ref)
+    n, y = eesd.accept_resample(p, q, x.contiguous(), ua, ur, T)
+    n_ref, y_ref = oracle.accept_resample_batch(p.cpu().numpy(), qc, x.cpu().numpy(), ua.cpu().numpy(),
+                                                ur.cpu().numpy(), T)
+    np.testing.assert_array_equal(n.cpu().numpy(), n_ref)
+    np.testing.assert_array_equal(y.cpu().numpy(), y_ref)
+    return n_ref
+
+
+@pytest.mark.parametrize("B,K", [(1, 1), (1, 4), (8, 8), (64, 16), (8, 1), (64, 4), (1, 16)])
+def test_accept_sweep_bit_exact(B, K):
+    seen = []
+    for ci, (sigma, delta) in enumerate(CASES):
+        seen.append(_run_case(ci * 100 + B * 17 + K, B, K, 32000, sigma, delta, 1.0).mean() / K)
+    if B * K >= 64:
+        assert max(seen) > 0.5 and min(seen) < 0.5  # the sweep spans high and low acceptance
+
+
+def test_accept_greedy_and_temperature_and_ragged_vocab():
+    _run_case(900, 8, 4, 32000, 3.0, 0.1, 0.0)
+    _run_case(901, 4, 4, 32000, 1.0, 1.0, 0.7)
+    for V in (1, 2, 17, 1024, 1025, 50257):
+        _run_case(902 + V, 3, 3, V, 2.0, 1.0, 1.0)
+
+
+def test_accept_p_equals_q_accepts_all_and_scratch_is_reusable():
+    import paper_2406_03853_b200 as eesd
+    B, K, V = 4, 5, 4096
+    p, _, ua, ur, ud = synth.accept_case(77, B, K, V, 2.0, 0.0, device="cuda")
+    q = p[:, :K].contiguous()
+    x = eesd.sample_rows(q.view(B * K, V), ud.view(B * K), 1.0).view(B, K).contiguous()
+    scratch = torch.empty(eesd.lib().eesd_accept_scratch_bytes(B, K), dtype=torch.uint8, device="cuda")
+    for _ in range(3):
+        n, y = eesd.accept_resample(p, q, x, ua, ur, 1.0, scratch=scratch)
+        assert (n.cpu().numpy() == K).all()
+    y_ref = [oracle.sample_logits(p[b, K].cpu().numpy(), 1.0, float(ur[b])) for b in range(B)]
+    np.testing.assert_array_equal(y.cpu().numpy(), y_ref)
+
+
+def test_bad_arguments_are_rejected():
+    import paper_2406_03853_b200 as eesd
+    L = eesd.lib()
+    assert L.eesd_accept_resample(None, None, None, None, None, None, 1, 1, 8, 1.0, None, 0, None, None) == -1
+    t = torch.zeros(64, device="cuda")
+    i = torch.zeros(8, dtype=torch.int32, device="cuda")
+    assert L.eesd_accept_resample(None, t.data_ptr(), t.data_ptr(), i.data_ptr(), t.data_ptr(), t.data_ptr(),
+                                  1, 1, 8, 1.0, t.data_ptr(), 4, i.data_ptr(), i.data_ptr()) == -2  # scratch too small
+    assert L.eesd_sample_rows(None, t.data_ptr(), None, 1, 8, 1.0, i.data_ptr()) == -6        # needs uniforms
