@@ -222,8 +222,9 @@ int eesd_launch_count(const eesd_ctx *ctx, int64_t *n);
 /* Standalone fused softmax / accept / residual-resample over a batch of B independent
  * sequences (the acceptance step of eesd_verify_accept).  All pointers are device pointers:
  * p_logits [B][K+1][V] f32, q_logits [B][K][V] f32, tokens [B][K] i32 (the drafted x_i),
- * u_accept [B][K], u_resample [B]; outputs n_accept [B], next_token [B] (i32).  scratch: at
- * least eesd_accept_scratch_bytes(B, K) bytes.  Asynchronous on `cuda_stream`. */
+ * u_accept [B][K], u_resample [B]; outputs n_accept [B], next_token [B] (i32).  scratch: 16-byte
+ * aligned, at least eesd_accept_scratch_bytes(B, K) bytes, contents irrelevant (the call clears
+ * what it needs).  Asynchronous on `cuda_stream`.  Errors: BADARG, NOMEM (scratch), RNG. */
 size_t eesd_accept_scratch_bytes(int B, int K);
 int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *q_logits,
                          const int32_t *tokens, const float *u_accept, const float *u_resample,

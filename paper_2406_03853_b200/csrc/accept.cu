@@ -209,8 +209,9 @@ __device__ int block_draw(const float *lp, const RowStat &sp, const float *lq, c
 }
 
 // ---- accept kernel -------------------------------------------------------------------------------
-// scratch per sequence: RowStat[2K+1] (p rows 0..K, then q rows 0..K-1) followed by one
-// 32-bit arrival counter per sequence (zero on entry, reset to zero by the finishing block).
+// scratch: one 32-bit arrival counter per sequence (zero on entry, reset to zero by the
+// finishing block; at the start so its place does not move with K), then per sequence
+// RowStat[2K+1] (p rows 0..K, then q rows 0..K-1).
 // grid = B * (2K+1) blocks.  Each block computes the statistics of one row; the block that
 // arrives last for its sequence runs the acceptance tests and the draw.
 __global__ void __launch_bounds__(kAccThreads) accept_kernel(const float *p_logits, const float *q_logits,
@@ -282,15 +283,15 @@ __global__ void __launch_bounds__(kAccThreads) accept_kernel(const float *p_logi
 }
 
 size_t accept_scratch_bytes(int B, int K) {
-    size_t stats = (size_t)B * (2 * K + 1) * sizeof(RowStat);
-    return stats + (size_t)B * sizeof(unsigned int) + 16;
+    size_t counters = ((size_t)B * sizeof(unsigned int) + 15) / 16 * 16;
+    return counters + (size_t)B * (2 * K + 1) * sizeof(RowStat);
 }
 
 void launch_accept(cudaStream_t s, const float *p_logits, const float *q_logits, const int32_t *tokens,
                    const float *u_acc, const float *u_res, int B, int K, int V, float T, void *scratch,
                    int32_t *n_acc, int32_t *y, int32_t *pending_out) {
-    RowStat *stats = (RowStat *)scratch;
-    unsigned int *counters = (unsigned int *)((char *)scratch + (size_t)B * (2 * K + 1) * sizeof(RowStat));
+    unsigned int *counters = (unsigned int *)scratch;
+    RowStat *stats = (RowStat *)((char *)scratch + ((size_t)B * sizeof(unsigned int) + 15) / 16 * 16);
     accept_kernel<<<B * (2 * K + 1), kAccThreads, 0, s>>>(p_logits, q_logits, tokens, u_acc, u_res, K, V, T,
                                                          stats, counters, n_acc, y, pending_out);
 }

@@ -360,8 +360,11 @@ int verify_impl(eesd_ctx *c, const float *d_u_acc, const float *d_u_res) {
 int finish_round(eesd_ctx *c, const int32_t *draft_tokens_host, int *n_accept, int32_t *next) {
     const int K = c->round_k;
     const int a = c->h_result[0], y = c->h_result[1];
-    if (read_error_word(c)) return EESD_ERR_DEVICE;
-    if (a < 0 || a > K || y < 0 || y >= c->cfg.vocab) return EESD_ERR_DEVICE;
+    if (read_error_word(c) || a < 0 || a > K || y < 0 || y >= c->cfg.vocab) {
+        snprintf(c->cuda_err, sizeof(c->cuda_err), "device error word 0x%x, round result n_accept=%d next=%d (K=%d)",
+                 c->h_result[2], a, y, K);
+        return EESD_ERR_DEVICE;
+    }
     for (int i = 0; i < a; i++) c->tokens.push_back(draft_tokens_host[i]);
     c->tokens.push_back(y);
     c->round_k = 0;
@@ -729,7 +732,7 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
     const size_t need = accept_scratch_bytes(B, K);
     if (scratch_bytes < need) return EESD_ERR_NOMEM;
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    if (cudaMemsetAsync(scratch, 0, need, s) != cudaSuccess) return EESD_ERR_CUDA;
+    if (cudaMemsetAsync(scratch, 0, (size_t)B * sizeof(unsigned int), s) != cudaSuccess) return EESD_ERR_CUDA;
     launch_accept(s, p_logits, q_logits, tokens, u_accept, u_resample, B, K, V, temperature, scratch, n_accept,
                   next_token, nullptr);
     return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
