@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""EESD decode benchmark on B200.
+
+One "step" is one full decode of `max_new` tokens by Early-exiting Speculative Decoding
+(draft steps through the first N layers + exit layer + exit head, one verify pass of K+1 rows
+through every layer, lossless acceptance, Thompson-sampling draft length) on a synthetic
+random-init model of the named LLaMA-2 shape, batch 1.
+
+  value  tokens/s of the decode loop (eesd_decode) with the prompt already prefilled: every
+         input resident in HBM when the timed region starts.
+  e2e    tokens/s of eesd_generate called with host buffers: prompt upload, prefill, uniform
+         streams upload, decode, per-round result read-back, all inside the timed region.
+  roofline  the dominant kernel (the skinny projection that streams the weights), timed by
+         CUDA events over the layers' real weight matrices, against the measured HBM copy rate.
+  cpu_baseline  the CPU oracle timed on a bounded slice of the same workload.
+
+Multi-GPU (--gpus N under torchrun): N independent replicas, no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import eesd_synth as synth
+
+WORKLOADS = {
+    # name: (spec, prompt length, generated tokens, damp alpha, kv cache length for the verify-pass leg)
+    "13b-eesd": ("13b", 512, 256, 0.2, 1024),
+    "70b-eesd": ("70b", 1024, 256, 0.2, 1024),
+    "tiny-eesd": ("tiny", 32, 64, 0.1, 64),
+}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_engine(wl, temperature, controller, device):
+    from paper_2406_03853_b200 import Engine
+    from paper_2406_03853_b200 import binding as b
+    spec_name, n_prompt, max_new, damp, _ = WORKLOADS[wl]
+    spec = synth.SPECS[spec_name].with_(damp=damp)
+    max_ctx = max(n_prompt + max_new + 16, 1024 + 32)
+    cfg = b.make_config(d_model=spec.d_model, n_heads=spec.n_heads, n_kv_heads=spec.n_kv_heads, head_dim=spec.head_dim,
+                        ffn_dim=spec.ffn_dim, vocab=spec.vocab, n_layers=spec.n_layers, n_early=spec.n_early,
+                        dtype=spec.dtype, tie_exit_head=spec.tie_exit_head, max_ctx=max_ctx, k_cap=10,
+                        temperature=temperature, controller=controller, fixed_k=5, page_tokens=16)
+    eng = Engine(cfg, device=device)
+    # synthetic weights, generated on the device by the shared seeded generator
+    for l in range(spec.n_layers):
+        v = eng.layer_views(l)
+        for k, t in synth.layer_weights(spec, l, synth.SEED, device).items():
+            v[k].copy_(t)
+    v = eng.layer_views(spec.n_layers)
+    for k, t in synth.exit_layer_weights(spec, synth.SEED, device).items():
+        v[k].copy_(t)
+    g = eng.global_views()
+    g["embed"].copy_(synth.embedding(spec, synth.SEED, device))
+    head = synth.lm_head(spec, synth.SEED, device)
+    g["lm_head"].copy_(head)
+    if not spec.tie_exit_head:
+        g["exit_head"].copy_(head)
+    g["g_final"].fill_(1.0)
+    g["g_exit"].fill_(1.0)
+    torch.cuda.synchronize(device)
+    return eng, spec, n_prompt, max_new
+
+
+def pass_bytes(spec, rows_ctx):
+    """Algorithmic HBM bytes of one verify pass and one draft step: every weight of the layers
+    used plus the vocabulary head once, plus the KV rows read (cache of rows_ctx tokens)."""
+    es = 2 if spec.dtype == "bf16" else 4
+    layer = spec.layer_params * es
+    head = spec.vocab * spec.d_model * es
+    kv_tok = 2 * spec.kv_dim * es
+    verify = spec.n_layers * layer + head + spec.n_layers * rows_ctx * kv_tok
+    draft = (spec.n_early + 1) * layer + head + (spec.n_early + 1) * rows_ctx * kv_tok
+    return verify, draft
+
+
+def time_projection(eng, spec, M, reps=3):
+    """Dominant kernel in isolation: the gate/up projection of every layer, back to back, over
+    the layers' own weights (so consecutive launches never re-read a matrix from L2)."""
+    import paper_2406_03853_b200 as eesd
+    A = synth.normal_f32(3, 3, M * spec.d_model, eng.device).view(M, spec.d_model)
+    out = torch.empty(8, M, 2 * spec.ffn_dim, dtype=torch.float32, device=eng.device)
+    Ws = [eng.layer_views(l)["wgu"] for l in range(spec.n_layers)]
+    for W in Ws[:3]:
+        eesd.project_rows(A, W, out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    best = []
+    for _ in range(reps):
+        e0.record()
+        for W in Ws:
+            eesd.project_rows(A, W, out)
+        e1.record()
+        torch.cuda.synchronize()
+        best.append(e0.elapsed_time(e1) / len(Ws))
+    es = 2 if spec.dtype == "bf16" else 4
+    nbytes = 2 * spec.ffn_dim * spec.d_model * es
+    ms = statistics.median(best)
+    return nbytes, ms
+
+
+def time_verify_pass(eng, spec, ctx_len, M, reps=5):
+    toks = synth.prompt_tokens(5, M, spec.vocab).numpy()
+    eng.assume_context(ctx_len, int(toks[0]))
+    for _ in range(2):
+        eng.verify_only(toks)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ts = []
+    for _ in range(reps):
+        e0.record()
+        eng.verify_only(toks)
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    return statistics.median(ts)
+
+
+def oracle_sample(spec, mean_k, mean_emit, threads_note=True):
+    """CPU oracle on a bounded slice: one decoder layer of this shape on (mean_k + 1) rows
+    against a 512-token cache, and the vocabulary head on one row; scaled to a whole round."""
+    import oracle
+    L1 = spec.with_(n_layers=1, n_early=1, vocab=64)
+    lw = {k: v for k, v in synth.layer_weights(spec, 0).items()}
+    emb = np.zeros((64, spec.d_model), np.float32)
+    m = oracle.model_from_weights(L1, [lw], lw, emb, emb, max_ctx=640)
+    rows = max(2, int(round(mean_k)) + 1)
+    x = np.asarray(synth.normal_f32(1, 1, rows * spec.d_model).view(rows, spec.d_model), np.float64)
+    t0 = time.time()
+    m.layer_fwd(0, 0, x, 512)
+    t_layer_rows = time.time() - t0
+    t0 = time.time()
+    m.layer_fwd(0, 0, x[:1], 512)
+    t_layer_1 = time.time() - t0
+    head_rows = spec.vocab * spec.d_model / spec.layer_params  # head cost in units of one layer-row
+    per_row = t_layer_rows / rows
+    t_verify = spec.n_layers * t_layer_rows + rows * head_rows * per_row
+    t_draft = (rows - 1) * ((spec.n_early + 1) * t_layer_1 + head_rows * t_layer_1)
+    tok_s = mean_emit / (t_verify + t_draft)
+    return tok_s, t_layer_rows + t_layer_1, rows
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle as it stands, timed on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    spec_name, n_prompt, max_new, damp, _ = WORKLOADS[args.workload]
+    spec = synth.SPECS[spec_name].with_(damp=damp)
+    vals, ms = [], []
+    for i in range(args.warmup + args.steps):
+        t0 = time.time()
+        tok_s, _, rows = oracle_sample(spec, 5.0, 3.0)
+        if i >= args.warmup:
+            vals.append(tok_s)
+            ms.append((time.time() - t0) * 1e3)
+    v = statistics.median(vals)
+    sample = (f"one {spec.name}-shaped decoder layer on {rows} rows + on 1 row against a 512-token cache, scaled to "
+              f"a round of K=5 drafts emitting 3 tokens ({spec.n_layers} layers verify, {spec.n_early + 1} layers per "
+              f"draft step, vocabulary heads by parameter count); extrapolated, not a full-model run")
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    print(json.dumps({"impl": "reference", "metric": "eesd_decode_tokens_per_s", "value": v, "unit": "tokens/s",
+                      "n_gpus": 0, "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.median(ms),
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                      "config": {"workload": args.workload},
+                      "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+                      "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="13b-eesd", choices=sorted(WORKLOADS))
+    ap.add_argument("--temperature", type=float, default=0.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    device = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2406_03853_b200 import binding as b
+    eng, spec, n_prompt, max_new = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device)
+    prompt = synth.prompt_tokens(synth.SEED, n_prompt, spec.vocab).numpy()
+    u = {k: v.numpy() for k, v in synth.generate_uniforms(eng.cfg.max_ctx, 1 << 20).items()}
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- value: decode loop only, prompt prefilled, everything resident
+    for _ in range(args.warmup):
+        eng.prefill(prompt)
+        eng.decode(max_new, uniforms=u)
+    clocks = ClockSampler(local)
+    stats, dec_ms = [], 0.0
+    launches0 = eng.launch_count()
+    barrier()
+    clocks.start()
+    for _ in range(args.steps):
+        eng.prefill(prompt)       # untimed: rebuilds the KV cache of the prompt
+        torch.cuda.synchronize()
+        e0.record()
+        out, trace, st = eng.decode(max_new, uniforms=u)
+        e1.record()
+        torch.cuda.synchronize()
+        dec_ms += e0.elapsed_time(e1)
+        stats.append(st.as_dict())
+    clk = clocks.stop()
+    barrier()
+    launches = eng.launch_count() - launches0
+    t = torch.tensor([dec_ms], dtype=torch.float64, device=device)
+    if dist:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dec_ms = float(t.item())
+    value = world * args.steps * max_new / (dec_ms / 1e3)
+
+    # ---- e2e: eesd_generate with host buffers (prefill and all copies inside the timed region)
+    e2e_ms = 0.0
+    barrier()
+    for _ in range(args.steps):
+        e0.record()
+        out2, trace2, st2 = eng.generate(prompt, max_new, uniforms=u)
+        e1.record()
+        torch.cuda.synchronize()
+        e2e_ms += e0.elapsed_time(e1)
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
+    if dist:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item())
+    e2e_value = world * args.steps * max_new / (e2e_ms / 1e3)
+    greedy = args.temperature == 0.0
+    h2d = n_prompt * 4 + (0 if greedy else 3 * eng.cfg.max_ctx * 4)
+    d2h = sum(12 + 4 * k for k, _, _ in trace2)
+
+    if rank != 0:
+        return
+    # ---- dominant kernel and verify pass against the HBM roofline
+    peaks, peak_kind = measured_peaks()
+    mean_k = sum(s["drafted"] for s in stats) / max(1, sum(s["rounds"] for s in stats))
+    mean_emit = sum(s["emitted"] for s in stats) / max(1, sum(s["rounds"] for s in stats))
+    M_typ = min(16, int(round(mean_k)) + 1)
+    kbytes, kms = time_projection(eng, spec, M_typ)
+    achieved = kbytes / (kms * 1e-3) / 1e9
+    kv_len = WORKLOADS[args.workload][4]
+    bv, bd = pass_bytes(spec, kv_len)
+    vp = {}
+    for M in (1, M_typ, 16):
+        ms = time_verify_pass(eng, spec, kv_len, M)
+        vp[f"M{M}"] = {"ms": round(ms, 4), "gbs": round(bv / (ms * 1e-3) / 1e9, 1),
+                       "frac_of_measured_copy": round(bv / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                       "frac_of_8tbs": round(bv / (ms * 1e-3) / 1e9 / 8000.0, 4)}
+    s0 = stats[-1]
+    v_d = s0["accepted"] / max(1, s0["drafted"])
+    r_d = s0["accepted"] / max(1, s0["emitted"])
+    line = {
+        "metric": "eesd_decode_tokens_per_s", "value": round(value, 3), "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dec_ms / args.steps, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": spec.dtype, "data": "synthetic",
+        "config": {"workload": args.workload, "shape": spec.name, "prompt_tokens": n_prompt, "new_tokens": max_new,
+                   "batch": 1, "early_layers": spec.n_early, "damp_alpha": spec.damp, "controller": "beta_ts",
+                   "k_cap": 10, "temperature": args.temperature, "parallelism": f"replicas x{world}",
+                   "l2_policy": "inputs larger than L2 (each pass streams every weight once)"},
+        "e2e": {"value": round(e2e_value, 3), "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": round(e2e_ms / args.steps, 3)},
+        "gpu_launches": int(launches),
+        "clocks": clk,
+        "roofline": {"bound": "hbm", "kernel": "skinny projection (gate/up shape, M=%d)" % M_typ,
+                     "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
+                     "bytes_per_launch": kbytes, "ms_per_launch": round(kms, 5)},
+        "verify_pass": {"kv_len": kv_len, "bytes": bv, **vp},
+        "draft_step_bytes": bd,
+        "round_stats": {"rounds": s0["rounds"], "mean_k": round(mean_k, 3), "v_d": round(v_d, 4), "r_d": round(r_d, 4),
+                        "hm": round(2 * v_d * r_d / max(1e-9, v_d + r_d), 4),
+                        "ms_draft": round(s0["ms_draft"], 3), "ms_verify": round(s0["ms_verify"], 3),
+                        "ms_prefill_e2e": round(st2.ms_prefill, 3)},
+    }
+    if not args.no_cpu_baseline and world == 1:
+        import oracle
+        oracle.build()
+        tok_s, secs, rows = oracle_sample(spec, mean_k, mean_emit)
+        line["cpu_baseline"] = {
+            "value": round(tok_s, 5), "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"one {spec.name}-shaped decoder layer on {rows} rows and on 1 row against a 512-token cache "
+                      f"({secs:.1f} s of CPU work), scaled to a round of mean K={mean_k:.2f} emitting {mean_emit:.2f} "
+                      f"tokens; extrapolated"}
+    print(json.dumps(line))
+    eng.close()
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

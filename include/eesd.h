@@ -60,7 +60,7 @@ typedef struct eesd_config {
     int32_t vocab;        /* V                                                                  */
     int32_t n_layers;     /* L: decoder layers of the target model                              */
     int32_t n_early;      /* N: first layers shared by the draft model (Sec. 3.1), 1 <= N <= L  */
-    int32_t dtype;        /* EESD_F32 or EESD_BF16: weights, projection inputs and KV cache     */
+    int32_t dtype;        /* EESD_F32 or EESD_BF16: weights and KV cache (activations are fp32) */
     int32_t tie_exit_head;/* 1: the exit head W of Eq. 1 is the target LM head (same storage)   */
     float rms_eps;        /* RMSNorm epsilon                                                    */
     float rope_theta;     /* rotary base; pairs (2i, 2i+1) turn by pos * theta^(-2i/D)          */
@@ -190,6 +190,13 @@ int eesd_generate(eesd_ctx *ctx, const int32_t *prompt, int n_prompt, int max_ne
 
 /* ---- additions beyond the five calls above (testing and measurement) ---- */
 
+/* The decode loop of eesd_generate without its prefill: continues from the current context
+ * (after eesd_prefill, or a previous eesd_decode / eesd_verify_accept) for max_new more tokens.
+ * Same arguments and errors as eesd_generate; STATE if no prefill or a round is half drafted. */
+int eesd_decode(eesd_ctx *ctx, int max_new, const int32_t *k_schedule, int n_schedule,
+                const eesd_uniforms *u, int32_t *out, eesd_stats *stats, eesd_round *trace,
+                int trace_cap, int *n_rounds);
+
 /* Context length in tokens (including the pending one), and KV pages in use. */
 int eesd_context_len(const eesd_ctx *ctx, int *n_tokens, int *pages_in_use);
 /* Posterior parameters of the controller. */
@@ -230,6 +237,15 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
                          const int32_t *tokens, const float *u_accept, const float *u_resample,
                          int B, int K, int V, float temperature, void *scratch, size_t scratch_bytes,
                          int32_t *n_accept, int32_t *next_token);
+
+/* The skinny projection used by every weight-streaming step of a pass (QKV, attention output,
+ * SwiGLU gate/up and down, vocabulary heads): out[s][m][r] = sum over the s-th slice of k of
+ * A[m][k] * W[r][k], M <= EESD_MAX_ROWS rows, fp32 results.  A [M][K] fp32, W [R][K] in `dtype`
+ * (device), out: device, room for EESD_MAX_SPLITS * M * R floats.  *n_splits (host) receives the
+ * number of k slices written; the caller sums them in index order.  Asynchronous. */
+#define EESD_MAX_SPLITS 8
+int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *W, float *out,
+                      int M, int R, int K, int *n_splits);
 
 /* Draws one token per row: argmax (temperature 0) or x ~ softmax(logits / T) by inverse CDF
  * with u[b].  logits [B][V] f32, u [B] (may be NULL when greedy), out [B] i32; device pointers. */

@@ -28,7 +28,7 @@ def build(force: bool = False) -> str:
 
 class _Cfg(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("d", "H", "Hkv", "D", "F", "V", "L", "N", "max_ctx")] + \
-               [("eps", C.c_double), ("theta", C.c_double)]
+               [("eps", C.c_double), ("theta", C.c_double), ("kv_bf16", C.c_int)]
 
 
 class _GenCfg(C.Structure):
@@ -55,6 +55,8 @@ def lib():
         L.orc_set_globals.argtypes = [C.c_void_p] + [C.c_void_p] * 5
         L.orc_rmsnorm.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_double, C.c_void_p]
         L.orc_rope.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_double]
+        L.orc_bf16_round.restype = C.c_double
+        L.orc_bf16_round.argtypes = [C.c_double]
         L.orc_layer_fwd.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int]
         L.orc_embed.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_head.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -176,9 +178,9 @@ class OracleModel:
     """
 
     def __init__(self, *, d, H, Hkv, D, F, V, N, max_ctx, layers: Sequence[Dict], exit_layer: Dict,
-                 embed, g_final, lm_head, g_exit, exit_head, eps=1e-5, theta=10000.0):
+                 embed, g_final, lm_head, g_exit, exit_head, eps=1e-5, theta=10000.0, kv_bf16=False):
         self.L = len(layers)
-        self.cfg = _Cfg(d, H, Hkv, D, F, V, self.L, N, max_ctx, eps, theta)
+        self.cfg = _Cfg(d, H, Hkv, D, F, V, self.L, N, max_ctx, eps, theta, int(kv_bf16))
         self.d, self.V, self.F, self.N, self.max_ctx = d, V, F, N, max_ctx
         self._keep = []
         self.h = C.c_void_p(lib().orc_model_new(C.byref(self.cfg)))
@@ -257,8 +259,12 @@ class OracleModel:
         return out, [(trace[i].k, trace[i].n_acc, trace[i].y) for i in range(n)], (a.value, b.value)
 
 
+def bf16_round(x: float) -> float:
+    return float(lib().orc_bf16_round(float(x)))
+
+
 def model_from_weights(spec_like, layers, exit_layer, embed, lm_head, exit_head=None, max_ctx=256,
-                       g_final=None, g_exit=None) -> OracleModel:
+                       g_final=None, g_exit=None, kv_bf16=None) -> OracleModel:
     """Convenience: build an OracleModel from shape fields (d_model, n_heads, ...) and weights."""
     s = spec_like
     ones = np.ones(s.d_model, np.float32)
@@ -267,4 +273,5 @@ def model_from_weights(spec_like, layers, exit_layer, embed, lm_head, exit_head=
                        g_final=ones if g_final is None else g_final, lm_head=lm_head,
                        g_exit=ones if g_exit is None else g_exit,
                        exit_head=lm_head if exit_head is None else exit_head,
-                       eps=s.rms_eps, theta=s.rope_theta)
+                       eps=s.rms_eps, theta=s.rope_theta,
+                       kv_bf16=(getattr(s, 'dtype', 'f32') == 'bf16') if kv_bf16 is None else kv_bf16)

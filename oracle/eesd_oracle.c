@@ -9,7 +9,9 @@
  * acceptance, and the Beta-posterior Thompson-sampling controller (Eq. 3-4, Algorithm 2).
  *
  * Precision: weights and logits are fp32 values; every activation, dot product, norm and
- * attention softmax is carried in fp64.  The acceptance / sampling arithmetic is the one
+ * attention softmax is carried in fp64.  Storage formats are part of a configuration: bf16
+ * configurations hand this file bf16-rounded weight values and set kv_bf16, which rounds keys
+ * and values to bfloat16 when they enter the cache.  The acceptance / sampling arithmetic is the one
  * place where fp32 is fixed, step by step (see "canonical sampling arithmetic" below), so
  * that an independent implementation can reproduce it bit for bit.
  *
@@ -28,6 +30,8 @@ typedef struct {
     int d, H, Hkv, D, F, V, L, N; /* L target layers, N early layers shared with the draft */
     int max_ctx;
     double eps, theta;
+    int kv_bf16; /* 1: cached keys/values are stored rounded to bfloat16 (the storage format of
+                    the bf16 configurations); arithmetic on them stays fp64 */
 } orc_cfg;
 
 typedef struct {
@@ -96,6 +100,16 @@ static void matvec(const float *W, const double *x, int rows, int cols, double *
     }
 }
 
+/* value of x after storage as bfloat16: round to nearest even on the upper 16 bits of fp32 */
+double orc_bf16_round(double x) {
+    union { float f; uint32_t u; } v;
+    v.f = (float)x;
+    if ((v.u & 0x7F800000u) == 0x7F800000u) return (double)v.f; /* inf / nan unchanged */
+    v.u += 0x7FFFu + ((v.u >> 16) & 1u);
+    v.u &= 0xFFFF0000u;
+    return (double)v.f;
+}
+
 static double *cache_row(double *base, const orc_cfg *c, int slot, int pos) {
     return base + ((size_t)slot * c->max_ctx + pos) * ((size_t)c->Hkv * c->D);
 }
@@ -119,6 +133,8 @@ static void project_qkv(orc_model *m, const orc_layer *lw, int slot, const doubl
             matvec(lw->wqkv + (size_t)qd * c->d, n, 2 * kvd, c->d, qkv + qd);
         }
         for (int h = 0; h < c->Hkv; h++) orc_rope(qkv + qd + h * c->D, c->D, pos, c->theta);
+        if (c->kv_bf16)
+            for (int i = 0; i < 2 * kvd; i++) qkv[qd + i] = orc_bf16_round(qkv[qd + i]);
         memcpy(cache_row(m->kc, c, slot, pos), qkv + qd, sizeof(double) * kvd);
         memcpy(cache_row(m->vc, c, slot, pos), qkv + qd + kvd, sizeof(double) * kvd);
     }

@@ -99,6 +99,8 @@ def lib():
         L.eesd_verify_accept.argtypes = [vp, vp, C.c_float, C.POINTER(C.c_int), i32p]
         L.eesd_generate.argtypes = [vp, vp, C.c_int, C.c_int, vp, C.c_int, C.POINTER(Uniforms), vp,
                                     C.POINTER(Stats), vp, C.c_int, C.POINTER(C.c_int)]
+        L.eesd_decode.argtypes = [vp, C.c_int, vp, C.c_int, C.POINTER(Uniforms), vp, C.POINTER(Stats), vp, C.c_int,
+                                  C.POINTER(C.c_int)]
         L.eesd_context_len.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.eesd_posterior.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.eesd_assume_context.argtypes = [vp, C.c_int, C.c_int32]
@@ -110,6 +112,7 @@ def lib():
         L.eesd_accept_scratch_bytes.argtypes = [C.c_int, C.c_int]
         L.eesd_accept_resample.argtypes = [vp, vp, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_float, vp,
                                            C.c_size_t, vp, vp]
+        L.eesd_project_rows.argtypes = [vp, C.c_int, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
         L.eesd_sample_rows.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_float, vp]
         _lib = L
     return _lib
@@ -236,22 +239,26 @@ class Engine:
                                              C.byref(n), C.byref(y)), "eesd_verify_accept")
         return n.value, y.value
 
+    def _uniforms(self, uniforms: Optional[Dict]):
+        if uniforms is None:
+            return None, []
+        U, keep = Uniforms(), []
+        for name in ("u_draft", "u_accept", "u_resample", "u_ctrl"):
+            a = _np_f32(uniforms[name])
+            keep.append(a)
+            setattr(U, name, a.ctypes.data)
+        U.n_ctrl = len(keep[-1])
+        for a in keep[:3]:
+            if len(a) < self.cfg.max_ctx:
+                raise ValueError("position-indexed uniform streams need max_ctx entries")
+        return U, keep
+
     def generate(self, prompt, max_new: int, k_schedule=None, uniforms: Optional[Dict] = None):
-        """Returns (tokens[max_new], trace[(k, n_accept, next_token)], Stats)."""
+        """eesd_generate.  Returns (tokens[max_new], trace[(k, n_accept, next_token)], Stats)."""
         p = _np_i32(prompt)
         out = np.empty(max_new, np.int32)
         ks = None if k_schedule is None else _np_i32(k_schedule)
-        U, keep = None, []
-        if uniforms is not None:
-            U = Uniforms()
-            for name in ("u_draft", "u_accept", "u_resample", "u_ctrl"):
-                a = _np_f32(uniforms[name])
-                keep.append(a)
-                setattr(U, name, a.ctypes.data)
-            U.n_ctrl = len(keep[-1])
-            for a in keep[:3]:
-                if len(a) < self.cfg.max_ctx:
-                    raise ValueError("position-indexed uniform streams need max_ctx entries")
+        U, keep = self._uniforms(uniforms)
         cap = max_new + 1
         trace = (Round * cap)()
         st, nr = Stats(), C.c_int()
@@ -259,6 +266,20 @@ class Engine:
                                         None if ks is None else ks.ctypes.data, 0 if ks is None else len(ks),
                                         None if U is None else C.byref(U), out.ctypes.data, C.byref(st),
                                         C.cast(trace, C.c_void_p), cap, C.byref(nr)), "eesd_generate")
+        return out, [(trace[i].k, trace[i].n_accept, trace[i].next_token) for i in range(nr.value)], st
+
+    def decode(self, max_new: int, k_schedule=None, uniforms: Optional[Dict] = None):
+        """eesd_decode: the decode loop from the current context (no prefill)."""
+        out = np.empty(max_new, np.int32)
+        ks = None if k_schedule is None else _np_i32(k_schedule)
+        U, keep = self._uniforms(uniforms)
+        cap = max_new + 1
+        trace = (Round * cap)()
+        st, nr = Stats(), C.c_int()
+        self._check(lib().eesd_decode(self.h, max_new, None if ks is None else ks.ctypes.data,
+                                      0 if ks is None else len(ks), None if U is None else C.byref(U),
+                                      out.ctypes.data, C.byref(st), C.cast(trace, C.c_void_p), cap, C.byref(nr)),
+                    "eesd_decode")
         return out, [(trace[i].k, trace[i].n_accept, trace[i].next_token) for i in range(nr.value)], st
 
     # ---- additions
@@ -335,3 +356,19 @@ def sample_rows(logits: torch.Tensor, u: Optional[torch.Tensor], temperature: fl
     if st:
         raise EesdError(st, "eesd_sample_rows")
     return out
+
+
+def project_rows(A: torch.Tensor, W: torch.Tensor, out: Optional[torch.Tensor] = None):
+    """eesd_project_rows: returns (partials [8, M, R] fp32 tensor, n_splits); sum partials[:n_splits]."""
+    _need_cuda()
+    M, K = A.shape
+    R = W.shape[0]
+    assert W.shape[1] == K and A.dtype == torch.float32 and A.is_contiguous() and W.is_contiguous() and A.is_cuda
+    dt = F32 if W.dtype == torch.float32 else BF16
+    if out is None:
+        out = torch.empty(8, M, R, dtype=torch.float32, device=A.device)
+    ns = C.c_int()
+    st = lib().eesd_project_rows(_stream_ptr(), dt, A.data_ptr(), W.data_ptr(), out.data_ptr(), M, R, K, C.byref(ns))
+    if st:
+        raise EesdError(st, "eesd_project_rows")
+    return out, ns.value

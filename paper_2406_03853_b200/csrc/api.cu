@@ -46,7 +46,7 @@ struct Workspace {
         accept, total;
 };
 
-constexpr int kPartSplits = 8;   // room for K-split partial sums of one projection
+constexpr int kPartSplits = EESD_MAX_SPLITS;   // room for K-split partial sums of one projection
 constexpr int kAttnSplits = 8;   // KV splits per head in attention
 constexpr int kIntSlots = 64;    // small device integer area
 
@@ -62,10 +62,10 @@ Workspace carve(const eesd_config *c) {
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     w.x = take(R * c->d_model * 4);
-    w.xn = take(R * c->d_model * es);
+    w.xn = take(R * c->d_model * 4);
     w.q = take(R * qd * 4);
-    w.attn = take(R * qd * es);
-    w.h = take(R * (size_t)c->ffn_dim * es);
+    w.attn = take(R * qd * 4);
+    w.h = take(R * (size_t)c->ffn_dim * 4);
     w.part = take((size_t)kPartSplits * R * maxR * 4);
     w.apart = take((size_t)c->n_heads * kAttnSplits * R * (c->head_dim + 2) * 4);
     w.logits_p = take(R * (size_t)c->vocab * 4);
@@ -95,8 +95,8 @@ struct eesd_ctx {
     cudaStream_t stream;
     size_t es;
     // device pointers
-    float *x, *q, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
-    void *xn, *attn, *h, *accept_scratch;
+    float *x, *xn, *q, *attn, *h, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
+    void *accept_scratch;
     float2 *rope;
     int32_t *page_table, *ints;
     int *err;
@@ -190,11 +190,11 @@ void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const fl
     launch_qkv_post(s, f.dtype, c->part, S, M, pos0, f.n_heads, kv, c->rope, c->q, false, c->err);
     launch_attention(s, f.dtype, c->q, kv, c->apart, c->attn, M, pos0, f.n_heads, kAttnSplits);
     S = launch_gemm(s, f.dtype, c->attn, w.wo, c->part, M, d, qd);
-    launch_resid_norm(s, f.dtype, c->x, c->part, S, w.g_ffn, c->xn, nullptr, M, d, f.rms_eps);
+    launch_resid_norm(s, c->x, c->part, S, w.g_ffn, c->xn, nullptr, M, d, f.rms_eps);
     S = launch_gemm(s, f.dtype, c->xn, w.wgu, c->part, M, 2 * F, d);
-    launch_swiglu(s, f.dtype, c->part, S, c->h, M, F);
+    launch_swiglu(s, c->part, S, c->h, M, F);
     S = launch_gemm(s, f.dtype, c->h, w.wd, c->part, M, d, F);
-    launch_resid_norm(s, f.dtype, c->x, c->part, S, g_next, c->xn, cap, M, d, f.rms_eps);
+    launch_resid_norm(s, c->x, c->part, S, g_next, c->xn, cap, M, d, f.rms_eps);
     c->launches += 10;
 }
 
@@ -209,7 +209,7 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
     cudaStream_t s = c->stream;
     const int L = f.n_layers, d = f.d_model;
     launch_embed(s, f.dtype, d_tok, c->embed, c->x, cap_slot(c, 0), M, d, f.vocab, c->err);
-    launch_resid_norm(s, f.dtype, c->x, nullptr, 0, c->layers[0].g_attn, c->xn, nullptr, M, d, f.rms_eps);
+    launch_resid_norm(s, c->x, nullptr, 0, c->layers[0].g_attn, c->xn, nullptr, M, d, f.rms_eps);
     c->launches += 2;
     for (int l = 0; l < L; l++) {
         const bool exit_here = (l == f.n_early - 1);
@@ -222,7 +222,7 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
             int S = launch_gemm(s, f.dtype, c->xn, wkv, c->part, M, 2 * kvd, d);
             launch_qkv_post(s, f.dtype, c->part, S, M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err);
             const float *g_next = l + 1 < L ? c->layers[l + 1].g_attn : c->g_final;
-            launch_resid_norm(s, f.dtype, c->x, nullptr, 0, g_next, c->xn, nullptr, M, d, f.rms_eps);
+            launch_resid_norm(s, c->x, nullptr, 0, g_next, c->xn, nullptr, M, d, f.rms_eps);
             c->launches += 3;
         }
     }
@@ -241,7 +241,7 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
     cudaStream_t s = c->stream;
     const int L = f.n_layers, d = f.d_model, N = f.n_early;
     launch_embed(s, f.dtype, c->ints + kRoundTok + i, c->embed, c->x, cap_slot(c, 0), 1, d, f.vocab, c->err);
-    launch_resid_norm(s, f.dtype, c->x, nullptr, 0, c->layers[0].g_attn, c->xn, nullptr, 1, d, f.rms_eps);
+    launch_resid_norm(s, c->x, nullptr, 0, c->layers[0].g_attn, c->xn, nullptr, 1, d, f.rms_eps);
     for (int l = 0; l < N; l++) {
         const float *g_after = l + 1 < N ? c->layers[l + 1].g_attn : c->layers[L].g_attn;
         run_layer(c, c->layers[l], l, 1, pos, g_after, cap_slot(c, l + 1));
@@ -463,8 +463,8 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->slot_bytes = (size_t)c->n_pages_total * 2 * cfg->n_kv_heads * cfg->page_tokens * cfg->head_dim * c->es;
     Workspace w = carve(cfg);
     char *ws = (char *)b->workspace;
-    c->x = (float *)(ws + w.x); c->xn = ws + w.xn; c->q = (float *)(ws + w.q); c->attn = ws + w.attn;
-    c->h = ws + w.h; c->part = (float *)(ws + w.part); c->apart = (float *)(ws + w.apart);
+    c->x = (float *)(ws + w.x); c->xn = (float *)(ws + w.xn); c->q = (float *)(ws + w.q); c->attn = (float *)(ws + w.attn);
+    c->h = (float *)(ws + w.h); c->part = (float *)(ws + w.part); c->apart = (float *)(ws + w.apart);
     c->logits_p = (float *)(ws + w.logits_p); c->logits_q = (float *)(ws + w.logits_q);
     c->rope = (float2 *)(ws + w.rope); c->page_table = (int32_t *)(ws + w.page_table);
     c->ints = (int32_t *)(ws + w.ints); c->u_dev = (float *)(ws + w.u_dev); c->u_stage = (float *)(ws + w.u_stage);
@@ -570,32 +570,28 @@ int eesd_verify_accept(eesd_ctx *c, const float *u_accept, float u_resample, int
     return finish_round(c, drafts, n_accept, next_token);
 }
 
-int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new, const int32_t *k_schedule,
-                  int n_schedule, const eesd_uniforms *u, int32_t *out, eesd_stats *stats, eesd_round *trace,
-                  int trace_cap, int *n_rounds) {
-    if (!c || !out || max_new < 1) return EESD_ERR_BADARG;
+// rounds of {draft, verify, accept, posterior update} from the current context until max_new
+// tokens exist (Algorithm 1, outer loop)
+static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int n_schedule, const eesd_uniforms *u,
+                       int32_t *out, eesd_stats *stats, eesd_round *trace, int trace_cap, int *n_rounds,
+                       int64_t launches0, float ms_prefill) {
     const eesd_config &f = c->cfg;
     const bool greedy = f.temperature == 0.f;
     if (!greedy && (!u || !u->u_draft || !u->u_accept || !u->u_resample)) return EESD_ERR_RNG;
     if (f.controller == EESD_CTRL_BETA_TS && (!u || !u->u_ctrl)) return EESD_ERR_RNG;
-    if (n_prompt + max_new + 1 > f.max_ctx) return EESD_ERR_CTX_FULL;
-    const int64_t launches0 = c->launches;
+    const int n0 = (int)c->tokens.size();
+    if (n0 + max_new + 1 > f.max_ctx) return EESD_ERR_CTX_FULL;
     float *d_ud = c->u_dev, *d_ua = c->u_dev + f.max_ctx, *d_ur = c->u_dev + 2 * (size_t)f.max_ctx;
     if (!greedy) {
         CU(c, cudaMemcpyAsync(d_ud, u->u_draft, (size_t)f.max_ctx * 4, cudaMemcpyHostToDevice, c->stream));
         CU(c, cudaMemcpyAsync(d_ua, u->u_accept, (size_t)f.max_ctx * 4, cudaMemcpyHostToDevice, c->stream));
         CU(c, cudaMemcpyAsync(d_ur, u->u_resample, (size_t)f.max_ctx * 4, cudaMemcpyHostToDevice, c->stream));
     }
-    CU(c, cudaEventRecord(c->ev[0], c->stream));
-    int st = prefill_impl(c, prompt, n_prompt);
-    if (st) return st;
-    CU(c, cudaEventRecord(c->ev[1], c->stream));
     eesd_stats sacc;
     memset(&sacc, 0, sizeof(sacc));
     int64_t cursor = 0;
-    int t = 0, rounds = 0;
+    int t = 0, rounds = 0, st;
     int32_t *drafts = c->h_result + 8;
-    float ms_p = 0.f;
     while (t < max_new) {
         const int T = (int)c->tokens.size();
         // draft length of this round: the controller's decisions depend on the posterior only,
@@ -633,22 +629,21 @@ int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new,
         float ms_d = 0.f, ms_v = 0.f;
         cudaEventElapsedTime(&ms_d, c->ev[2], c->ev[3]);
         cudaEventElapsedTime(&ms_v, c->ev[3], c->ev[4]);
-        if (rounds == 0) cudaEventElapsedTime(&ms_p, c->ev[0], c->ev[1]);
         sacc.ms_draft += ms_d;
         sacc.ms_verify += ms_v;
         sacc.drafted += K;
-        sacc.accepted += a;
+        sacc.accepted += a < max_new - t ? a : max_new - t;
         ts_update(c, a + 1, K);
         if (trace && rounds < trace_cap) { trace[rounds].k = K; trace[rounds].n_accept = a; trace[rounds].next_token = y; }
         t += a + 1;
         rounds++;
     }
-    for (int i = 0; i < max_new; i++) out[i] = c->tokens[n_prompt + i];
+    for (int i = 0; i < max_new; i++) out[i] = c->tokens[n0 + i];
     if (n_rounds) *n_rounds = rounds;
     if (stats) {
         sacc.rounds = rounds;
         sacc.emitted = max_new;
-        sacc.ms_prefill = ms_p;
+        sacc.ms_prefill = ms_prefill;
         sacc.ms_total = sacc.ms_prefill + sacc.ms_draft + sacc.ms_verify;
         sacc.kernel_launches = c->launches - launches0;
         sacc.alpha = c->alpha;
@@ -656,6 +651,29 @@ int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new,
         *stats = sacc;
     }
     return EESD_OK;
+}
+
+int eesd_decode(eesd_ctx *c, int max_new, const int32_t *k_schedule, int n_schedule, const eesd_uniforms *u,
+                int32_t *out, eesd_stats *stats, eesd_round *trace, int trace_cap, int *n_rounds) {
+    if (!c || !out || max_new < 1) return EESD_ERR_BADARG;
+    if (!c->prefilled || c->round_k != 0) return EESD_ERR_STATE;
+    return decode_impl(c, max_new, k_schedule, n_schedule, u, out, stats, trace, trace_cap, n_rounds, c->launches, 0.f);
+}
+
+int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new, const int32_t *k_schedule,
+                  int n_schedule, const eesd_uniforms *u, int32_t *out, eesd_stats *stats, eesd_round *trace,
+                  int trace_cap, int *n_rounds) {
+    if (!c || !out || max_new < 1) return EESD_ERR_BADARG;
+    if (n_prompt + max_new + 1 > c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
+    const int64_t launches0 = c->launches;
+    CU(c, cudaEventRecord(c->ev[0], c->stream));
+    int st = prefill_impl(c, prompt, n_prompt);
+    if (st) return st;
+    CU(c, cudaEventRecord(c->ev[1], c->stream));
+    CU(c, cudaEventSynchronize(c->ev[1]));
+    float ms_p = 0.f;
+    cudaEventElapsedTime(&ms_p, c->ev[0], c->ev[1]);
+    return decode_impl(c, max_new, k_schedule, n_schedule, u, out, stats, trace, trace_cap, n_rounds, launches0, ms_p);
 }
 
 int eesd_context_len(const eesd_ctx *c, int *n_tokens, int *pages_in_use) {
@@ -735,6 +753,15 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
     if (cudaMemsetAsync(scratch, 0, (size_t)B * sizeof(unsigned int), s) != cudaSuccess) return EESD_ERR_CUDA;
     launch_accept(s, p_logits, q_logits, tokens, u_accept, u_resample, B, K, V, temperature, scratch, n_accept,
                   next_token, nullptr);
+    return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
+}
+
+int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *W, float *out, int M, int R, int K,
+                      int *n_splits) {
+    if (!A || !W || !out || !n_splits) return EESD_ERR_BADARG;
+    if (M < 1 || M > EESD_MAX_ROWS || R < 1 || K < 8 || (K % 8)) return EESD_ERR_BADARG;
+    if (dtype != EESD_F32 && dtype != EESD_BF16) return EESD_ERR_BADARG;
+    *n_splits = launch_gemm((cudaStream_t)cuda_stream, dtype, A, W, out, M, R, K);
     return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
 }
 

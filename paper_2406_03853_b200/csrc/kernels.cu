@@ -57,9 +57,8 @@ void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, 
 
 // ------------------------------------------------------------------------------------ residual + RMSNorm
 // One block per token row.  x[m] += sum_s part[s][m]; xn[m] = RMSNorm(x[m]) * g.
-template <typename AT>
 __global__ void __launch_bounds__(256) resid_norm_kernel(float *x, const float *part, int S, size_t part_stride,
-                                                         const float *g, AT *xn, float *cap, int d, float eps) {
+                                                         const float *g, float *xn, float *cap, int d, float eps) {
     extern __shared__ float row[];  // d floats + 33 scratch
     float *scratch = row + d;
     const int m = blockIdx.x;
@@ -76,15 +75,14 @@ __global__ void __launch_bounds__(256) resid_norm_kernel(float *x, const float *
     if (!g) return;
     ss = block_sum(ss, scratch);
     const float rstd = 1.0f / sqrtf(ss / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) xn[(size_t)m * d + i] = from_f<AT>(row[i] * rstd * g[i]);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) xn[(size_t)m * d + i] = row[i] * rstd * g[i];
 }
-void launch_resid_norm(cudaStream_t s, int dtype, float *x, const float *part, int S, const float *g,
-                       void *xn, float *cap, int M, int d, float eps) {
+void launch_resid_norm(cudaStream_t s, float *x, const float *part, int S, const float *g, float *xn, float *cap,
+                       int M, int d, float eps) {
     size_t smem = (size_t)(d + 33) * sizeof(float);
     size_t stride = (size_t)M * d;
     if (!part) S = 0;
-    if (dtype == 0) resid_norm_kernel<float><<<M, 256, smem, s>>>(x, part, S, stride, g, (float *)xn, cap, d, eps);
-    else resid_norm_kernel<bf16><<<M, 256, smem, s>>>(x, part, S, stride, g, (bf16 *)xn, cap, d, eps);
+    resid_norm_kernel<<<M, 256, smem, s>>>(x, part, S, stride, g, xn, cap, d, eps);
 }
 
 // ------------------------------------------------------------------------------------ skinny projection (SIMT)
@@ -162,9 +160,9 @@ static void gemm_simt_dispatch(cudaStream_t s, const void *A, const void *W, flo
     else gemm_simt_kernel<WT, AT, 16><<<grid, 256, 0, s>>>(a, w, out, M, R, K);
 }
 
-int launch_gemm(cudaStream_t s, int dtype, const void *A, const void *W, float *out, int M, int R, int K) {
+int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float *out, int M, int R, int K) {
     if (dtype == 0) gemm_simt_dispatch<float, float>(s, A, W, out, M, R, K);
-    else gemm_simt_dispatch<bf16, bf16>(s, A, W, out, M, R, K);
+    else gemm_simt_dispatch<bf16, float>(s, A, W, out, M, R, K);
     return 1;
 }
 
@@ -340,8 +338,7 @@ __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, 
 }
 
 // grid (H, M), block D: merge the splits of one (head, row)
-template <typename AT>
-__global__ void attn_combine_kernel(const float *apart, AT *out, int H, int D, int n_split) {
+__global__ void attn_combine_kernel(const float *apart, float *out, int H, int D, int n_split) {
     const int h = blockIdx.x, m = blockIdx.y, dd = threadIdx.x;
     const float *src = apart + (size_t)h * n_split * kMaxRows * (D + 2) + (size_t)m * (D + 2);
     const size_t sstride = (size_t)kMaxRows * (D + 2);
@@ -355,27 +352,25 @@ __global__ void attn_combine_kernel(const float *apart, AT *out, int H, int D, i
         num = fmaf(w, src[s * sstride + dd], num);
         den = fmaf(w, src[s * sstride + D + 1], den);
     }
-    out[(size_t)m * H * D + (size_t)h * D + dd] = from_f<AT>(den > 0.f ? num / den : 0.f);
+    out[(size_t)m * H * D + (size_t)h * D + dd] = den > 0.f ? num / den : 0.f;
 }
 
 void launch_attention(cudaStream_t s, int dtype, const float *q, const KvGeom &kv, float *apart,
-                      void *attn_out, int M, int pos0, int H, int n_split) {
+                      float *attn_out, int M, int pos0, int H, int n_split) {
     dim3 grid(H, n_split);
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (dtype == 0) {
         if (kv.D == 64) attn_kernel<float, 64><<<grid, 256, 0, s>>>(q, kv, apart, M, pos0, H, n_split, scale);
         else attn_kernel<float, 128><<<grid, 256, 0, s>>>(q, kv, apart, M, pos0, H, n_split, scale);
-        attn_combine_kernel<float><<<dim3(H, M), kv.D, 0, s>>>(apart, (float *)attn_out, H, kv.D, n_split);
     } else {
         if (kv.D == 64) attn_kernel<bf16, 64><<<grid, 256, 0, s>>>(q, kv, apart, M, pos0, H, n_split, scale);
         else attn_kernel<bf16, 128><<<grid, 256, 0, s>>>(q, kv, apart, M, pos0, H, n_split, scale);
-        attn_combine_kernel<bf16><<<dim3(H, M), kv.D, 0, s>>>(apart, (bf16 *)attn_out, H, kv.D, n_split);
     }
+    attn_combine_kernel<<<dim3(H, M), kv.D, 0, s>>>(apart, attn_out, H, kv.D, n_split);
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU, partial sums
-template <typename AT>
-__global__ void swiglu_kernel(const float *part, int S, size_t part_stride, AT *h, int F) {
+__global__ void swiglu_kernel(const float *part, int S, size_t part_stride, float *h, int F) {
     const int m = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= F) return;
     float g = 0.f, u = 0.f;
@@ -385,13 +380,12 @@ __global__ void swiglu_kernel(const float *part, int S, size_t part_stride, AT *
         u += p[F + i];
     }
     const float sg = g / (1.0f + expf(-g));
-    h[(size_t)m * F + i] = from_f<AT>(sg * u);
+    h[(size_t)m * F + i] = sg * u;
 }
-void launch_swiglu(cudaStream_t s, int dtype, const float *part, int S, void *h, int M, int F) {
+void launch_swiglu(cudaStream_t s, const float *part, int S, float *h, int M, int F) {
     dim3 grid((F + 255) / 256, M);
     size_t stride = (size_t)M * 2 * F;
-    if (dtype == 0) swiglu_kernel<float><<<grid, 256, 0, s>>>(part, S, stride, (float *)h, F);
-    else swiglu_kernel<bf16><<<grid, 256, 0, s>>>(part, S, stride, (bf16 *)h, F);
+    swiglu_kernel<<<grid, 256, 0, s>>>(part, S, stride, h, F);
 }
 
 __global__ void reduce_partials_kernel(const float *part, int S, size_t stride, float *out, size_t n) {

@@ -5,7 +5,7 @@ import eesd_synth as synth
 import oracle
 
 
-def oracle_from_spec(spec, max_ctx=256, n_layers=None, device="cpu", seed=synth.SEED):
+def oracle_from_spec(spec, max_ctx=256, n_layers=None, device="cpu", seed=synth.SEED, kv_bf16=None):
     """Oracle model with the synthetic weights of `spec` (optionally only the first n_layers;
     the exit layer is then still the copy of the spec's last layer)."""
     L = spec.n_layers if n_layers is None else n_layers
@@ -14,7 +14,7 @@ def oracle_from_spec(spec, max_ctx=256, n_layers=None, device="cpu", seed=synth.
     emb = synth.embedding(spec, seed, device).cpu()
     head = synth.lm_head(spec, seed, device).cpu()
     s = spec.with_(n_layers=L)
-    return oracle.model_from_weights(s, layers, ex, emb, head, max_ctx=max_ctx)
+    return oracle.model_from_weights(s, layers, ex, emb, head, max_ctx=max_ctx, kv_bf16=kv_bf16)
 
 
 def np_softmax(x):

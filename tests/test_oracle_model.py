@@ -188,3 +188,23 @@ def test_parameter_counts_match_the_papers_tables():
     # the shapes the oracle is built with carry exactly these counts
     lw = synth.layer_weights(synth.TINY, 0)
     assert sum(v.numel() for k, v in lw.items() if k.startswith("w")) == synth.TINY.layer_params
+
+
+def test_bf16_storage_rounding_matches_library_conversion_and_only_touches_the_cache():
+    import torch
+    xs = np.concatenate([synth.normal_f32(8, 1, 20000).numpy().astype(np.float64) * 3.0,
+                         [0.0, 1.0, 1.00390625, 1.001953125, 1.005859375, -2.5e-7, 3.0e38, 65504.0]])
+    got = np.array([oracle.bf16_round(x) for x in xs])
+    ref = torch.tensor(xs, dtype=torch.float32).to(torch.bfloat16).double().numpy()  # round-to-nearest-even
+    np.testing.assert_array_equal(got, ref)
+    # with one cached position attention returns v exactly, so the layer output moves by exactly
+    # Wo (bf16(v) - v); with more positions a bf16 cache stays within bf16 rounding of the fp64 one
+    spec = synth.TINY.with_(n_layers=1, n_early=1)
+    lw = synth.layer_weights(spec, 0)
+    emb, head = synth.embedding(spec), synth.lm_head(spec)
+    a = oracle.model_from_weights(spec, [lw], lw, emb, head, max_ctx=16, kv_bf16=False)
+    b = oracle.model_from_weights(spec, [lw], lw, emb, head, max_ctx=16, kv_bf16=True)
+    x0 = a.embed([5, 6, 7, 8]) * 30.0
+    ya, yb = a.layer_fwd(0, 0, x0, 0), b.layer_fwd(0, 0, x0, 0)
+    d = np.abs(ya - yb).max()
+    assert 0 < d < 2.0 ** -7 * np.abs(ya).max()
