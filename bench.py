@@ -94,11 +94,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_engine(wl, temperature, controller, device):
+def build_engine(wl, temperature, controller, device, n_layers=0):
     from paper_2406_03853_b200 import Engine
     from paper_2406_03853_b200 import binding as b
     spec_name, n_prompt, max_new, damp, _ = WORKLOADS[wl]
     spec = synth.SPECS[spec_name].with_(damp=damp)
+    if n_layers:
+        spec = spec.with_(n_layers=n_layers, n_early=min(spec.n_early, n_layers))
     max_ctx = max(n_prompt + max_new + 16, 1024 + 32)
     cfg = b.make_config(d_model=spec.d_model, n_heads=spec.n_heads, n_kv_heads=spec.n_kv_heads, head_dim=spec.head_dim,
                         ffn_dim=spec.ffn_dim, vocab=spec.vocab, n_layers=spec.n_layers, n_early=spec.n_early,
@@ -138,28 +140,11 @@ def pass_bytes(spec, rows_ctx):
 
 
 def time_projection(eng, spec, M, reps=3):
-    """Dominant kernel in isolation: the gate/up projection of every layer, back to back, over
-    the layers' own weights (so consecutive launches never re-read a matrix from L2)."""
-    import paper_2406_03853_b200 as eesd
-    A = synth.normal_f32(3, 3, M * spec.d_model, eng.device).view(M, spec.d_model)
-    out = torch.empty(8, M, 2 * spec.ffn_dim, dtype=torch.float32, device=eng.device)
-    Ws = [eng.layer_views(l)["wgu"] for l in range(spec.n_layers)]
-    for W in Ws[:3]:
-        eesd.project_rows(A, W, out)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    best = []
-    for _ in range(reps):
-        e0.record()
-        for W in Ws:
-            eesd.project_rows(A, W, out)
-        e1.record()
-        torch.cuda.synchronize()
-        best.append(e0.elapsed_time(e1) / len(Ws))
-    es = 2 if spec.dtype == "bf16" else 4
-    nbytes = 2 * spec.ffn_dim * spec.d_model * es
-    ms = statistics.median(best)
-    return nbytes, ms
+    """Dominant kernel as the passes launch it: the gate/up projection of every layer, back to
+    back over the layers' own weights (consecutive launches never re-read a matrix from L2),
+    bracketed by CUDA events on the library's stream (eesd_time_projection)."""
+    ms = [eng.time_projection(2, M) for _ in range(reps)]
+    return ms[0][1], statistics.median(m for m, _ in ms)
 
 
 def time_verify_pass(eng, spec, ctx_len, M, reps=5):
@@ -203,6 +188,24 @@ def oracle_sample(spec, mean_k, mean_emit, threads_note=True):
     return tok_s, t_layer_rows + t_layer_1, rows
 
 
+def profile_pass(args, device):
+    """Verify passes and draft steps between cudaProfilerStart/Stop (for the ncu recipes)."""
+    from paper_2406_03853_b200 import binding as b
+    eng, spec, _, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, args.layers)
+    kv_len = WORKLOADS[args.workload][4]
+    toks = synth.prompt_tokens(5, args.profile_pass, spec.vocab).numpy()
+    eng.assume_context(kv_len, int(toks[0]))
+    eng.verify_only(toks)
+    torch.cuda.synchronize()
+    torch.cuda.profiler.start()
+    eng.verify_only(toks)
+    eng.draft(1)
+    torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
+    print("profiled: 1 verify pass of %d rows + 1 draft step, %s, %d layers" % (args.profile_pass, spec.name, spec.n_layers))
+    eng.close()
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle as it stands, timed on the host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -241,6 +244,10 @@ def main():
     ap.add_argument("--workload", default="13b-eesd", choices=sorted(WORKLOADS))
     ap.add_argument("--temperature", type=float, default=0.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-pass", type=int, default=0, metavar="M",
+                    help="only run verify passes of M rows (and draft steps) inside a cudaProfilerStart/Stop "
+                         "bracket, for ncu --profile-from-start off")
+    ap.add_argument("--layers", type=int, default=0, help="with --profile-pass: keep only this many layers")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -259,6 +266,8 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     from paper_2406_03853_b200 import binding as b
+    if args.profile_pass:
+        return profile_pass(args, device)
     eng, spec, n_prompt, max_new = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device)
     prompt = synth.prompt_tokens(synth.SEED, n_prompt, spec.vocab).numpy()
     u = {k: v.numpy() for k, v in synth.generate_uniforms(eng.cfg.max_ctx, 1 << 20).items()}

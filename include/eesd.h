@@ -64,7 +64,7 @@ typedef struct eesd_config {
     int32_t tie_exit_head;/* 1: the exit head W of Eq. 1 is the target LM head (same storage)   */
     float rms_eps;        /* RMSNorm epsilon                                                    */
     float rope_theta;     /* rotary base; pairs (2i, 2i+1) turn by pos * theta^(-2i/D)          */
-    int32_t page_tokens;  /* tokens per KV page (power of two, >= 8)                            */
+    int32_t page_tokens;  /* tokens per KV page (power of two, 8..128)                          */
     int32_t max_ctx;      /* most tokens a sequence may hold (prompt + generated + drafts)      */
     int32_t k_cap;        /* most draft tokens per round, 1 <= k_cap <= EESD_MAX_ROWS - 1       */
     float temperature;    /* 0: greedy (draft top-1, accept while equal to target top-1)        */
@@ -239,13 +239,22 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
                          int32_t *n_accept, int32_t *next_token);
 
 /* The skinny projection used by every weight-streaming step of a pass (QKV, attention output,
- * SwiGLU gate/up and down, vocabulary heads): out[s][m][r] = sum over the s-th slice of k of
- * A[m][k] * W[r][k], M <= EESD_MAX_ROWS rows, fp32 results.  A [M][K] fp32, W [R][K] in `dtype`
- * (device), out: device, room for EESD_MAX_SPLITS * M * R floats.  *n_splits (host) receives the
- * number of k slices written; the caller sums them in index order.  Asynchronous. */
-#define EESD_MAX_SPLITS 8
+ * SwiGLU gate/up and down, vocabulary heads): out[m][r] = sum_k A[m][k] * W[r][k] for
+ * M <= EESD_MAX_ROWS rows.  A [M][K] fp32, W [R][K] in `dtype`, out [M][R] fp32, all device.
+ * bf16 weights with R % 128 == 0 and K % 64 == 0 take the tensor-core path (the rows are split
+ * into two bf16 terms first), everything else the SIMT path.  scratch: device, 256-byte
+ * aligned, at least eesd_project_scratch_bytes(R, K) bytes; afterwards its first 4 bytes hold
+ * an error word (0 = none).  Asynchronous on `cuda_stream`.  K must be a multiple of 8. */
+size_t eesd_project_scratch_bytes(int R, int K);
 int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *W, float *out,
-                      int M, int R, int K, int *n_splits);
+                      int M, int R, int K, void *scratch, size_t scratch_bytes);
+
+/* Times the projection kernel of one kind (0 QKV, 1 attention output, 2 gate/up, 3 down) as
+ * the passes launch it: once over every target layer's matrix untimed, then once more
+ * bracketed by CUDA events on the context's stream.  Returns the mean device time per launch
+ * and the weight bytes one launch streams.  Synchronises.  The activation content is whatever
+ * the last pass left in the context. */
+int eesd_time_projection(eesd_ctx *ctx, int which, int M, float *ms_per_launch, size_t *bytes_per_launch);
 
 /* Draws one token per row: argmax (temperature 0) or x ~ softmax(logits / T) by inverse CDF
  * with u[b].  logits [B][V] f32, u [B] (may be NULL when greedy), out [B] i32; device pointers. */

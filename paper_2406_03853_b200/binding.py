@@ -112,7 +112,10 @@ def lib():
         L.eesd_accept_scratch_bytes.argtypes = [C.c_int, C.c_int]
         L.eesd_accept_resample.argtypes = [vp, vp, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_float, vp,
                                            C.c_size_t, vp, vp]
-        L.eesd_project_rows.argtypes = [vp, C.c_int, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
+        L.eesd_project_scratch_bytes.restype = C.c_size_t
+        L.eesd_project_scratch_bytes.argtypes = [C.c_int, C.c_int]
+        L.eesd_project_rows.argtypes = [vp, C.c_int, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, C.c_size_t]
+        L.eesd_time_projection.argtypes = [vp, C.c_int, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_size_t)]
         L.eesd_sample_rows.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_float, vp]
         _lib = L
     return _lib
@@ -320,6 +323,12 @@ class Engine:
             self._capture = None
         return self._capture
 
+    def time_projection(self, which: int, M: int):
+        """(ms per launch, weight bytes per launch) of projection kind `which` over all layers."""
+        ms, nb = C.c_float(), C.c_size_t()
+        self._check(lib().eesd_time_projection(self.h, which, M, C.byref(ms), C.byref(nb)), "eesd_time_projection")
+        return ms.value, nb.value
+
     def launch_count(self) -> int:
         n = C.c_int64()
         self._check(lib().eesd_launch_count(self.h, C.byref(n)), "eesd_launch_count")
@@ -358,17 +367,19 @@ def sample_rows(logits: torch.Tensor, u: Optional[torch.Tensor], temperature: fl
     return out
 
 
-def project_rows(A: torch.Tensor, W: torch.Tensor, out: Optional[torch.Tensor] = None):
-    """eesd_project_rows: returns (partials [8, M, R] fp32 tensor, n_splits); sum partials[:n_splits]."""
+def project_rows(A: torch.Tensor, W: torch.Tensor, scratch: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """eesd_project_rows: A [M, K] fp32 times W [R, K]^T (fp32 or bf16) -> [M, R] fp32."""
     _need_cuda()
     M, K = A.shape
     R = W.shape[0]
     assert W.shape[1] == K and A.dtype == torch.float32 and A.is_contiguous() and W.is_contiguous() and A.is_cuda
     dt = F32 if W.dtype == torch.float32 else BF16
-    if out is None:
-        out = torch.empty(8, M, R, dtype=torch.float32, device=A.device)
-    ns = C.c_int()
-    st = lib().eesd_project_rows(_stream_ptr(), dt, A.data_ptr(), W.data_ptr(), out.data_ptr(), M, R, K, C.byref(ns))
+    need = lib().eesd_project_scratch_bytes(R, K)
+    if scratch is None:
+        scratch = torch.empty(need, dtype=torch.uint8, device=A.device)
+    out = torch.empty(M, R, dtype=torch.float32, device=A.device)
+    st = lib().eesd_project_rows(_stream_ptr(), dt, A.data_ptr(), W.data_ptr(), out.data_ptr(), M, R, K,
+                                 scratch.data_ptr(), scratch.numel())
     if st:
         raise EesdError(st, "eesd_project_rows")
-    return out, ns.value
+    return out

@@ -17,7 +17,11 @@ namespace {
 struct LayerW {
     const float *g_attn, *g_ffn;
     const char *wqkv, *wo, *wgu, *wd;
+    CUtensorMap m_qkv, m_o, m_gu, m_d;  // tensor-core path only
 };
+
+// which activation matrix feeds a projection
+enum { X_NORM = 0, X_ATTN = 1, X_FFN = 2 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -31,7 +35,7 @@ int check_config(const eesd_config *c) {
     if (c->dtype != EESD_F32 && c->dtype != EESD_BF16) return EESD_ERR_BADARG;
     if (c->head_dim != 64 && c->head_dim != 128) return EESD_ERR_UNSUPPORTED;
     if (c->d_model % 8 || c->ffn_dim % 8 || (c->n_heads * c->head_dim) % 8) return EESD_ERR_UNSUPPORTED;
-    if (c->page_tokens < 8 || (c->page_tokens & (c->page_tokens - 1))) return EESD_ERR_BADARG;
+    if (c->page_tokens < 8 || c->page_tokens > 128 || (c->page_tokens & (c->page_tokens - 1))) return EESD_ERR_BADARG;
     if (c->k_cap < 1 || c->k_cap > EESD_MAX_ROWS - 1) return EESD_ERR_BADARG;
     if (c->temperature < 0.f) return EESD_ERR_BADARG;
     if (c->controller != EESD_CTRL_FIXED_K && c->controller != EESD_CTRL_BETA_TS) return EESD_ERR_BADARG;
@@ -42,13 +46,14 @@ int check_config(const eesd_config *c) {
 }
 
 struct Workspace {
-    size_t x, xn, q, attn, h, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
+    size_t x, xn, q, attn, h, xs[3], part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
         accept, total;
 };
 
-constexpr int kPartSplits = EESD_MAX_SPLITS;   // room for K-split partial sums of one projection
-constexpr int kAttnSplits = 8;   // KV splits per head in attention
+constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
+constexpr int kAttnSplits = 64;  // most KV slices per head in attention
 constexpr int kIntSlots = 64;    // small device integer area
+constexpr int kMaxSm = 256;      // upper bound on CTAs of the persistent projection kernel
 
 Workspace carve(const eesd_config *c) {
     Workspace w;
@@ -66,7 +71,16 @@ Workspace carve(const eesd_config *c) {
     w.q = take(R * qd * 4);
     w.attn = take(R * qd * 4);
     w.h = take(R * (size_t)c->ffn_dim * 4);
-    w.part = take((size_t)kPartSplits * R * maxR * 4);
+    // the same three activation matrices as two bf16 terms, [32][K] (tensor-core path)
+    w.xs[X_NORM] = take(2 * R * (size_t)c->d_model * 2);
+    w.xs[X_ATTN] = take(2 * R * qd * 2);
+    w.xs[X_FFN] = take(2 * R * (size_t)c->ffn_dim * 2);
+    {   // partial sums: SIMT layout [splits][16][maxR], or stream-K blocks of the widest projection
+        size_t part_floats = (size_t)kPartSplits * R * maxR;
+        const size_t sk_floats = (maxR / 128 + 3 * (size_t)kMaxSm) * R * 128;  // >= G * max_seg blocks
+        if (sk_floats > part_floats) part_floats = sk_floats;
+        w.part = take(part_floats * 4);
+    }
     w.apart = take((size_t)c->n_heads * kAttnSplits * R * (c->head_dim + 2) * 4);
     w.logits_p = take(R * (size_t)c->vocab * 4);
     w.logits_q = take(R * (size_t)c->vocab * 4);
@@ -97,6 +111,11 @@ struct eesd_ctx {
     // device pointers
     float *x, *xn, *q, *attn, *h, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
     void *accept_scratch;
+    void *xs[3];                 // bf16 hi/lo copies of xn, attn, h
+    CUtensorMap m_x[3];
+    CUtensorMap m_exit_kv, m_lm_head, m_exit_head;
+    bool use_tc;
+    int n_sm;
     float2 *rope;
     int32_t *page_table, *ints;
     int *err;
@@ -179,6 +198,26 @@ void trim_pages(eesd_ctx *c, int n_tokens) {
     }
 }
 
+// One projection: out = X[which] . W^T.  Tensor-core stream-K kernel when the context uses it
+// (bf16, tile-aligned shapes), else the SIMT kernel.  Returns where the partial sums are.
+PartView run_proj(eesd_ctx *c, const void *W, const CUtensorMap *mW, int which, int M, int R, int K) {
+    PartView pv = {};
+    pv.base = c->part;
+    pv.R = R;
+    if (c->use_tc) {
+        pv.mode = 1;
+        pv.sk = tc_plan(R, K, c->n_sm);
+        launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, pv.sk, M, c->err);
+    } else {
+        const float *A = which == X_NORM ? c->xn : which == X_ATTN ? c->attn : c->h;
+        pv.mode = 0;
+        pv.S = launch_gemm(c->stream, c->cfg.dtype, A, W, c->part, M, R, K);
+        pv.split_stride = (size_t)M * R;
+    }
+    c->launches++;
+    return pv;
+}
+
 // one decoder layer on M rows at positions pos0.. ; on entry xn = RMSNorm(x) * g_attn of this
 // layer; on exit x holds the layer output and, when g_next is given, xn = RMSNorm(x) * g_next.
 void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const float *g_next, float *cap) {
@@ -186,16 +225,16 @@ void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const fl
     const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim, d = f.d_model, F = f.ffn_dim;
     cudaStream_t s = c->stream;
     KvGeom kv = kv_geom(c, slot);
-    int S = launch_gemm(s, f.dtype, c->xn, w.wqkv, c->part, M, qd + 2 * kvd, d);
-    launch_qkv_post(s, f.dtype, c->part, S, M, pos0, f.n_heads, kv, c->rope, c->q, false, c->err);
-    launch_attention(s, f.dtype, c->q, kv, c->apart, c->attn, M, pos0, f.n_heads, kAttnSplits);
-    S = launch_gemm(s, f.dtype, c->attn, w.wo, c->part, M, d, qd);
-    launch_resid_norm(s, c->x, c->part, S, w.g_ffn, c->xn, nullptr, M, d, f.rms_eps);
-    S = launch_gemm(s, f.dtype, c->xn, w.wgu, c->part, M, 2 * F, d);
-    launch_swiglu(s, c->part, S, c->h, M, F);
-    S = launch_gemm(s, f.dtype, c->h, w.wd, c->part, M, d, F);
-    launch_resid_norm(s, c->x, c->part, S, g_next, c->xn, cap, M, d, f.rms_eps);
-    c->launches += 10;
+    PartView pv = run_proj(c, w.wqkv, &w.m_qkv, X_NORM, M, qd + 2 * kvd, d);
+    launch_qkv_post(s, f.dtype, pv, M, pos0, f.n_heads, kv, c->rope, c->q, false, c->err);
+    launch_attention(s, f.dtype, c->q, kv, c->apart, c->attn, c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, c->err);
+    pv = run_proj(c, w.wo, &w.m_o, X_ATTN, M, d, qd);
+    launch_resid_norm(s, c->x, &pv, w.g_ffn, c->xn, c->xs[X_NORM], nullptr, M, d, f.rms_eps);
+    pv = run_proj(c, w.wgu, &w.m_gu, X_NORM, M, 2 * F, d);
+    launch_swiglu(s, pv, c->h, c->xs[X_FFN], M, F);
+    pv = run_proj(c, w.wd, &w.m_d, X_FFN, M, d, F);
+    launch_resid_norm(s, c->x, &pv, g_next, c->xn, c->xs[X_NORM], cap, M, d, f.rms_eps);
+    c->launches += 6;
 }
 
 float *cap_slot(eesd_ctx *c, int index) {
@@ -209,7 +248,7 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
     cudaStream_t s = c->stream;
     const int L = f.n_layers, d = f.d_model;
     launch_embed(s, f.dtype, d_tok, c->embed, c->x, cap_slot(c, 0), M, d, f.vocab, c->err);
-    launch_resid_norm(s, c->x, nullptr, 0, c->layers[0].g_attn, c->xn, nullptr, M, d, f.rms_eps);
+    launch_resid_norm(s, c->x, nullptr, c->layers[0].g_attn, c->xn, c->xs[X_NORM], nullptr, M, d, f.rms_eps);
     c->launches += 2;
     for (int l = 0; l < L; l++) {
         const bool exit_here = (l == f.n_early - 1);
@@ -219,17 +258,17 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
             // keys / values of the early-exit layer for these rows: they depend on H^N only
             const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim;
             const char *wkv = c->layers[L].wqkv + (size_t)qd * d * c->es;
-            int S = launch_gemm(s, f.dtype, c->xn, wkv, c->part, M, 2 * kvd, d);
-            launch_qkv_post(s, f.dtype, c->part, S, M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err);
+            PartView pv = run_proj(c, wkv, &c->m_exit_kv, X_NORM, M, 2 * kvd, d);
+            launch_qkv_post(s, f.dtype, pv, M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err);
             const float *g_next = l + 1 < L ? c->layers[l + 1].g_attn : c->g_final;
-            launch_resid_norm(s, c->x, nullptr, 0, g_next, c->xn, nullptr, M, d, f.rms_eps);
-            c->launches += 3;
+            launch_resid_norm(s, c->x, nullptr, g_next, c->xn, c->xs[X_NORM], nullptr, M, d, f.rms_eps);
+            c->launches += 2;
         }
     }
     if (want_logits) {
-        int S = launch_gemm(s, f.dtype, c->xn, c->lm_head, c->part, M, f.vocab, d);
-        launch_reduce_partials(s, c->part, S, c->logits_p, M, f.vocab);
-        c->launches += 2;
+        PartView pv = run_proj(c, c->lm_head, &c->m_lm_head, X_NORM, M, f.vocab, d);
+        launch_reduce_partials(s, pv, c->logits_p, M, f.vocab);
+        c->launches += 1;
     }
     return check_launch(c);
 }
@@ -241,17 +280,17 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
     cudaStream_t s = c->stream;
     const int L = f.n_layers, d = f.d_model, N = f.n_early;
     launch_embed(s, f.dtype, c->ints + kRoundTok + i, c->embed, c->x, cap_slot(c, 0), 1, d, f.vocab, c->err);
-    launch_resid_norm(s, c->x, nullptr, 0, c->layers[0].g_attn, c->xn, nullptr, 1, d, f.rms_eps);
+    launch_resid_norm(s, c->x, nullptr, c->layers[0].g_attn, c->xn, c->xs[X_NORM], nullptr, 1, d, f.rms_eps);
     for (int l = 0; l < N; l++) {
         const float *g_after = l + 1 < N ? c->layers[l + 1].g_attn : c->layers[L].g_attn;
         run_layer(c, c->layers[l], l, 1, pos, g_after, cap_slot(c, l + 1));
     }
     run_layer(c, c->layers[L], L, 1, pos, c->g_exit, cap_slot(c, L + 1));
     float *lq = c->logits_q + (size_t)i * f.vocab;
-    int S = launch_gemm(s, f.dtype, c->xn, c->exit_head, c->part, 1, f.vocab, d);
-    launch_reduce_partials(s, c->part, S, lq, 1, f.vocab);
+    PartView pv = run_proj(c, c->exit_head, &c->m_exit_head, X_NORM, 1, f.vocab, d);
+    launch_reduce_partials(s, pv, lq, 1, f.vocab);
     launch_sample_rows(s, lq, d_u, 1, f.vocab, f.temperature, c->ints + kRoundTok + i + 1);
-    c->launches += 5;
+    c->launches += 4;
     return check_launch(c);
 }
 
@@ -469,6 +508,18 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->rope = (float2 *)(ws + w.rope); c->page_table = (int32_t *)(ws + w.page_table);
     c->ints = (int32_t *)(ws + w.ints); c->u_dev = (float *)(ws + w.u_dev); c->u_stage = (float *)(ws + w.u_stage);
     c->err = (int *)(ws + w.err); c->accept_scratch = ws + w.accept;
+    for (int i = 0; i < 3; i++) c->xs[i] = nullptr;
+    c->n_sm = 1;
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, dev);
+        if (c->n_sm > kMaxSm) c->n_sm = kMaxSm;
+    }
+    const int qd_ = cfg->n_heads * cfg->head_dim, kvd_ = cfg->n_kv_heads * cfg->head_dim;
+    c->use_tc = cfg->dtype == EESD_BF16 && tc_shape_ok(qd_ + 2 * kvd_, cfg->d_model) && tc_shape_ok(cfg->d_model, qd_) &&
+                tc_shape_ok(2 * cfg->ffn_dim, cfg->d_model) && tc_shape_ok(cfg->d_model, cfg->ffn_dim) &&
+                tc_shape_ok(2 * kvd_, cfg->d_model) && tc_shape_ok(cfg->vocab, cfg->d_model) && tc_init() == 0;
     const char *wb = (const char *)b->weights;
     c->layers.resize(cfg->n_layers + 1);
     for (int l = 0; l <= cfg->n_layers; l++) {
@@ -478,6 +529,27 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         lw.g_ffn = (const float *)(base + lay.off_g_ffn); lw.wgu = base + lay.off_wgu; lw.wd = base + lay.off_wd;
     }
     c->embed = wb + lay.embed; c->lm_head = wb + lay.lm_head; c->exit_head = wb + lay.exit_head;
+    if (c->use_tc) {
+        const int d = cfg->d_model, F = cfg->ffn_dim, R2 = 2 * EESD_MAX_ROWS;
+        bool ok = true;
+        for (int i = 0; i < 3; i++) c->xs[i] = ws + w.xs[i];
+        ok = ok && tc_make_map(&c->m_x[X_NORM], c->xs[X_NORM], R2, d, R2);
+        ok = ok && tc_make_map(&c->m_x[X_ATTN], c->xs[X_ATTN], R2, qd_, R2);
+        ok = ok && tc_make_map(&c->m_x[X_FFN], c->xs[X_FFN], R2, F, R2);
+        for (auto &lw : c->layers) {
+            ok = ok && tc_make_map(&lw.m_qkv, lw.wqkv, qd_ + 2 * kvd_, d, 128);
+            ok = ok && tc_make_map(&lw.m_o, lw.wo, d, qd_, 128);
+            ok = ok && tc_make_map(&lw.m_gu, lw.wgu, 2 * F, d, 128);
+            ok = ok && tc_make_map(&lw.m_d, lw.wd, d, F, 128);
+        }
+        ok = ok && tc_make_map(&c->m_exit_kv, c->layers[cfg->n_layers].wqkv + (size_t)qd_ * d * 2, 2 * kvd_, d, 128);
+        ok = ok && tc_make_map(&c->m_lm_head, c->lm_head, cfg->vocab, d, 128);
+        ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128);
+        if (!ok) {
+            delete c;
+            return EESD_ERR_CUDA;
+        }
+    }
     c->g_final = (const float *)(wb + lay.final_norm); c->g_exit = (const float *)(wb + lay.exit_norm);
     // free list in descending order: the first pages handed out are the highest, so logical
     // and physical page numbers differ and the page table is really exercised
@@ -756,13 +828,86 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
     return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
 }
 
+static size_t project_scratch_layout(int R, int K, size_t *off_xs, size_t *off_part) {
+    size_t o = 256;  // error word
+    *off_xs = o;
+    o = align_up(o + (size_t)2 * EESD_MAX_ROWS * K * 2, 256);
+    *off_part = o;
+    size_t floats = (size_t)EESD_MAX_ROWS * R;
+    const size_t sk = ((size_t)R / 128 + 3 * (size_t)kMaxSm) * EESD_MAX_ROWS * 128;
+    if (sk > floats) floats = sk;
+    return o + floats * 4;
+}
+
+size_t eesd_project_scratch_bytes(int R, int K) {
+    if (R < 1 || K < 1) return 0;
+    size_t a, b;
+    return project_scratch_layout(R, K, &a, &b);
+}
+
 int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *W, float *out, int M, int R, int K,
-                      int *n_splits) {
-    if (!A || !W || !out || !n_splits) return EESD_ERR_BADARG;
+                      void *scratch, size_t scratch_bytes) {
+    if (!A || !W || !out || !scratch) return EESD_ERR_BADARG;
     if (M < 1 || M > EESD_MAX_ROWS || R < 1 || K < 8 || (K % 8)) return EESD_ERR_BADARG;
     if (dtype != EESD_F32 && dtype != EESD_BF16) return EESD_ERR_BADARG;
-    *n_splits = launch_gemm((cudaStream_t)cuda_stream, dtype, A, W, out, M, R, K);
+    size_t off_xs, off_part;
+    if (scratch_bytes < project_scratch_layout(R, K, &off_xs, &off_part)) return EESD_ERR_NOMEM;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    char *sc = (char *)scratch;
+    float *part = (float *)(sc + off_part);
+    PartView pv = {};
+    pv.base = part;
+    pv.R = R;
+    if (dtype == EESD_BF16 && tc_shape_ok(R, K) && tc_init() == 0) {
+        int dev = 0, n_sm = 1;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        if (n_sm > kMaxSm) n_sm = kMaxSm;
+        CUtensorMap mW, mX;
+        if (!tc_make_map(&mW, W, R, K, 128) || !tc_make_map(&mX, sc + off_xs, 2 * EESD_MAX_ROWS, K, 2 * EESD_MAX_ROWS))
+            return EESD_ERR_CUDA;
+        if (cudaMemsetAsync(sc, 0, 16, s) != cudaSuccess) return EESD_ERR_CUDA;
+        launch_split_rows(s, A, sc + off_xs, M, K);
+        pv.mode = 1;
+        pv.sk = tc_plan(R, K, n_sm);
+        launch_gemm_tc(s, mW, mX, part, pv.sk, M, (int *)sc);
+    } else {
+        pv.mode = 0;
+        pv.S = launch_gemm(s, dtype, A, W, part, M, R, K);
+        pv.split_stride = (size_t)M * R;
+    }
+    launch_reduce_partials(s, pv, out, M, R);
     return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
+}
+
+int eesd_time_projection(eesd_ctx *c, int which, int M, float *ms_per_launch, size_t *bytes_per_launch) {
+    if (!c || which < 0 || which > 3 || M < 1 || M > EESD_MAX_ROWS || !ms_per_launch || !bytes_per_launch)
+        return EESD_ERR_BADARG;
+    const eesd_config &f = c->cfg;
+    const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim, d = f.d_model, F = f.ffn_dim;
+    const int R = which == 0 ? qd + 2 * kvd : which == 2 ? 2 * F : d;
+    const int K = which == 1 ? qd : which == 3 ? F : d;
+    const int X = which == 1 ? X_ATTN : which == 3 ? X_FFN : X_NORM;
+    for (int pass = 0; pass < 2; pass++) {
+        if (pass == 1) CU(c, cudaEventRecord(c->ev[0], c->stream));
+        for (int l = 0; l < f.n_layers; l++) {
+            const LayerW &w = c->layers[l];
+            const void *W = which == 0 ? w.wqkv : which == 1 ? w.wo : which == 2 ? w.wgu : w.wd;
+            const CUtensorMap *m = which == 0 ? &w.m_qkv : which == 1 ? &w.m_o : which == 2 ? &w.m_gu : &w.m_d;
+            run_proj(c, W, m, X, M, R, K);
+        }
+        if (pass == 1) CU(c, cudaEventRecord(c->ev[1], c->stream));
+    }
+    int st = check_launch(c);
+    if (st) return st;
+    CU(c, cudaEventSynchronize(c->ev[1]));
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]);
+    *ms_per_launch = ms / f.n_layers;
+    *bytes_per_launch = (size_t)R * K * c->es;
+    CU(c, cudaMemcpyAsync(c->h_result + 2, c->err, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    return read_error_word(c);
 }
 
 int eesd_sample_rows(void *cuda_stream, const float *logits, const float *u, int B, int V, float temperature,

@@ -77,4 +77,11 @@ __device__ __forceinline__ float block_sum(float v, float *scratch /* >= 33 floa
     return scratch[32];
 }
 
+// writes v as two bf16 terms into a [2 * kMaxRows][K] matrix: row m gets hi, row kMaxRows + m gets lo
+__device__ __forceinline__ void store_split(__nv_bfloat16 *xs, int m, size_t K, size_t i, float v) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    xs[(size_t)m * K + i] = hi;
+    xs[(size_t)(kMaxRows + m) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
 }  // namespace eesd

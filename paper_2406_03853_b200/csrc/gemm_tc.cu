@@ -1,0 +1,326 @@
+// Weight-streaming skinny projection on the Blackwell tensor cores (sm_100a).
+//
+//   out[m][r] = sum_k X[m][k] * W[r][k],   m < M <= 16 token rows,  W bf16 [R][K] row-major
+//
+// HBM-bound: every weight byte is read exactly once per pass, the token rows are tiny.  The
+// kernel therefore exists to keep the memory system full:
+//   * persistent grid (one CTA per SM), work = (128-row weight tile, 64-wide k block) units
+//     dealt out as one contiguous, equal range per CTA ("stream-K"), so every SM streams the
+//     same number of bytes whatever R and K are;
+//   * a 10-stage TMA ring (16 KB weight tile + 4 KB token tile per stage, 128-byte swizzle)
+//     fed by one producer thread; nothing but mbarriers between HBM and the tensor core;
+//   * tcgen05.mma with the weight tile as the 128-row A operand and the token rows as the
+//     32-column B operand; fp32 accumulators in tensor memory, two buffers so the epilogue of
+//     one segment overlaps the MMAs of the next;
+//   * token rows are fp32 values split into two bf16 terms (hi + lo, rows 0..15 and 16..31 of
+//     the B operand): products are exact, accumulation is fp32, and the result equals an fp32
+//     activation times a bf16 weight to about 2^-17 relative.  The extra columns cost tensor
+//     time only, which this kernel has to spare.
+// Each segment (part of one tile's k range done by one CTA) is written as an fp32 partial;
+// consumers add the partials of a tile in CTA order, so results are bit-reproducible and do
+// not depend on M.
+//
+// Every wait is bounded: on expiry the thread raises the error word, the CTA drains its
+// outstanding TMA copies (bounded as well), frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace eesd {
+
+namespace tc {
+
+constexpr int BM = 128, BK = 64, BN = 32;
+constexpr int STAGES = 10;
+constexpr int STAGE_W = BM * BK * 2, STAGE_X = BN * BK * 2;
+constexpr int STAGE_BYTES = STAGE_W + STAGE_X;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int THREADS = 192;  // warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA issuer
+constexpr uint32_t TMEM_COLS = 64;   // two 128 x 32 fp32 accumulators
+constexpr uint32_t SPIN_LIMIT = 1u << 25;  // polls of a barrier before a wait gives up (about a second)
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait; false (and the abort flag set) when the limit is reached or another role gave up
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          uint32_t sleep_ns = 0) {
+    for (uint32_t i = 0; i < SPIN_LIMIT; i++) {
+        if (mbar_try(bar, parity)) return true;   // non-blocking poll
+        if (sleep_ns) __nanosleep(sleep_ns);
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+
+// shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row
+// groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                          // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version for this architecture
+    d |= (uint64_t)2 << 61;                          // 128-byte swizzle
+    return d;
+}
+
+// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 32
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+               float *__restrict__ part, StreamK sk, int M, int *err) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *sbase = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sW = sbase;
+    uint8_t *sX = sbase + STAGES * STAGE_W;
+    uint64_t *full = (uint64_t *)(sbase + STAGES * STAGE_BYTES);
+    uint64_t *empty = full + STAGES;
+    uint64_t *acc_full = empty + STAGES;   // [2]
+    uint64_t *acc_empty = acc_full + 2;    // [2]
+    uint32_t *tmem_slot = (uint32_t *)(acc_empty + 2);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x;
+    const int u0 = sk.start(cta), u1 = sk.start(cta + 1);
+
+    if (tid == 0) {
+        for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < 2; i++) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 4) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            int issued = 0;
+            bool ok = true;
+            for (int u = u0; u < u1 && ok; u++, issued++) {
+                const int s = issued % STAGES, round = issued / STAGES;
+                ok = mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                const int tile = u / sk.KB, kb = u - tile * sk.KB;
+                mbar_expect_tx(&full[s], STAGE_BYTES);
+                tma_load_2d(sW + s * STAGE_W, &tmW, &full[s], kb * BK, tile * BM);
+                tma_load_2d(sX + s * STAGE_X, &tmX, &full[s], kb * BK, 0);
+            }
+            if (*abort_flag) {
+                // let every copy still in flight land before the CTA's shared memory is released
+                const int first = issued > STAGES ? issued - STAGES : 0;
+                for (int i = first; i < issued; i++) {
+                    uint64_t *b = &full[i % STAGES];
+                    const uint32_t par = (uint32_t)((i / STAGES) & 1);
+                    for (uint32_t t = 0; t < SPIN_LIMIT && !mbar_try(b, par); t++) {}
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            int it = 0, seg = 0;
+            bool ok = true;
+            for (int u = u0; u < u1 && ok; seg++) {
+                const int tile = u / sk.KB;
+                const int u_end = min(u1, (tile + 1) * sk.KB);
+                const int b = seg & 1, use = seg >> 1;
+                ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_addr = tmem_base + (uint32_t)(b * BN);
+                for (int uu = u; uu < u_end; uu++, it++) {
+                    const int s = it % STAGES, round = it / STAGES;
+                    ok = mbar_wait(&full[s], round & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t da = smem_desc(smem_u32(sW + s * STAGE_W));
+                    const uint64_t db = smem_desc(smem_u32(sX + s * STAGE_X));
+#pragma unroll
+                    for (int j = 0; j < BK / 16; j++)
+                        mma_bf16(d_addr, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), (uu > u || j > 0) ? 1u : 0u);
+                    mma_commit(&empty[s]);   // the stage may be refilled once these MMAs have read it
+                }
+                if (!ok) break;
+                mma_commit(&acc_full[b]);    // accumulator complete
+                u = u_end;
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (warps 0-3)
+        int seg = 0;
+        bool ok = true;
+        for (int u = u0; u < u1 && ok; seg++) {
+            const int tile = u / sk.KB;
+            const int u_end = min(u1, (tile + 1) * sk.KB);
+            const int b = seg & 1, use = seg >> 1;
+            ok = mbar_wait(&acc_full[b], use & 1, abort_flag, 64);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t r[32];
+            tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * BN), r);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[b]);
+            float *dst = part + ((size_t)(cta * sk.max_seg + (tile - sk.first_tile(cta))) * kMaxRows) * BM + warp * 32 + lane;
+#pragma unroll
+            for (int m = 0; m < kMaxRows; m++)
+                if (m < M) dst[(size_t)m * BM] = __uint_as_float(r[m]) + __uint_as_float(r[16 + m]);
+            u = u_end;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && *abort_flag) atomicOr(err, kErrWaitTimeout);
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace tc
+
+// ---------------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                             const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeFn encode_fn() {
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeFn)p;
+    }
+    return fn;
+}
+
+bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    if (((uintptr_t)base & 15) || (cols % 8)) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
+                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool tc_shape_ok(int R, int K) { return R > 0 && K > 0 && R % tc::BM == 0 && K % tc::BK == 0; }
+
+StreamK tc_plan(int R, int K, int n_sm) {
+    StreamK sk;
+    sk.KB = K / tc::BK;
+    sk.U = (R / tc::BM) * sk.KB;
+    sk.G = sk.U < n_sm ? sk.U : n_sm;
+    sk.base = sk.U / sk.G;
+    sk.rem = sk.U % sk.G;
+    sk.max_seg = (sk.base + 1 + sk.KB - 1) / sk.KB + 1;
+    return sk;
+}
+
+size_t tc_partial_floats(const StreamK &sk) { return (size_t)sk.G * sk.max_seg * kMaxRows * tc::BM; }
+
+int tc_init() {
+    static int done = 0;
+    if (!done) {
+        if (cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess)
+            return -1;
+        if (!encode_fn()) return -1;
+        done = 1;
+    }
+    return 0;
+}
+
+void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
+                    int M, int *err) {
+    tc::gemm_tc_kernel<<<sk.G, tc::THREADS, tc::SMEM_BYTES, s>>>(mW, mX, part, sk, M, err);
+}
+
+// fp32 rows -> two bf16 terms: rows 0..15 hold hi = bf16(x), rows 16..31 hold lo = bf16(x - hi)
+__global__ void split_rows_kernel(const float *x, __nv_bfloat16 *xs, int K) {
+    const int m = blockIdx.y;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= K) return;
+    const float v = x[(size_t)m * K + i];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    xs[(size_t)m * K + i] = hi;
+    xs[(size_t)(kMaxRows + m) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+void launch_split_rows(cudaStream_t s, const float *x, void *xs, int M, int K) {
+    split_rows_kernel<<<dim3((K + 255) / 256, M), 256, 0, s>>>(x, (__nv_bfloat16 *)xs, K);
+}
+
+}  // namespace eesd

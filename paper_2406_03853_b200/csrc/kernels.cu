@@ -10,6 +10,42 @@ namespace eesd {
 
 typedef __nv_bfloat16 bf16;
 
+// sum of the partial results of output element (m, r), in a fixed order
+__device__ __forceinline__ float part_gather(const PartView &pv, int m, int r) {
+    float v = 0.f;
+    if (pv.mode == 0) {
+        for (int s = 0; s < pv.S; s++) v += pv.base[(size_t)s * pv.split_stride + (size_t)m * pv.R + r];
+    } else {
+        const StreamK &sk = pv.sk;
+        const int t = r >> 7, rr = r & 127;
+        const int c0 = sk.owner(t * sk.KB), c1 = sk.owner((t + 1) * sk.KB - 1);
+        for (int c = c0; c <= c1; c++)
+            v += pv.base[((size_t)(c * sk.max_seg + (t - sk.first_tile(c))) * kMaxRows + m) * 128 + rr];
+    }
+    return v;
+}
+
+// the same for four consecutive outputs r..r+3 (r % 4 == 0, so they share a weight tile)
+__device__ __forceinline__ float4 part_gather4(const PartView &pv, int m, int r) {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (pv.mode == 0) {
+        for (int s = 0; s < pv.S; s++) {
+            const float4 t = *reinterpret_cast<const float4 *>(pv.base + (size_t)s * pv.split_stride + (size_t)m * pv.R + r);
+            v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+        }
+    } else {
+        const StreamK &sk = pv.sk;
+        const int t = r >> 7, rr = r & 127;
+        const int c0 = sk.owner(t * sk.KB), c1 = sk.owner((t + 1) * sk.KB - 1);
+        for (int c = c0; c <= c1; c++) {
+            const float4 a = __ldcg(reinterpret_cast<const float4 *>(
+                pv.base + ((size_t)(c * sk.max_seg + (t - sk.first_tile(c))) * kMaxRows + m) * 128 + rr));
+            v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+        }
+    }
+    return v;
+}
+
 // ------------------------------------------------------------------------------------ small utilities
 __global__ void set_ints_kernel(int32_t *dst, IntList16 vals, int n) {
     if (threadIdx.x < n) dst[threadIdx.x] = vals.v[threadIdx.x];
@@ -56,33 +92,45 @@ void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, 
 }
 
 // ------------------------------------------------------------------------------------ residual + RMSNorm
-// One block per token row.  x[m] += sum_s part[s][m]; xn[m] = RMSNorm(x[m]) * g.
-__global__ void __launch_bounds__(256) resid_norm_kernel(float *x, const float *part, int S, size_t part_stride,
-                                                         const float *g, float *xn, float *cap, int d, float eps) {
+// One block of 1024 threads per token row, four elements per thread and step.
+// x[m] += partial sums; xn[m] = RMSNorm(x[m]) * g (fp32 and, optionally, as two bf16 terms).
+__global__ void __launch_bounds__(1024) resid_norm_kernel(float *x, PartView pv, int has_part, const float *g, float *xn,
+                                                          bf16 *xs, float *cap, int d, float eps) {
     extern __shared__ float row[];  // d floats + 33 scratch
     float *scratch = row + d;
     const int m = blockIdx.x;
     float *xr = x + (size_t)m * d;
     float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float v = xr[i];
-        for (int s = 0; s < S; s++) v += part[(size_t)s * part_stride + (size_t)m * d + i];
-        row[i] = v;
-        if (S > 0) xr[i] = v;
-        if (cap) cap[(size_t)m * d + i] = v;
-        ss += v * v;
+    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+        float4 v = *reinterpret_cast<const float4 *>(xr + i);
+        if (has_part) {
+            const float4 p = part_gather4(pv, m, i);
+            v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+            *reinterpret_cast<float4 *>(xr + i) = v;
+        }
+        *reinterpret_cast<float4 *>(row + i) = v;
+        if (cap) *reinterpret_cast<float4 *>(cap + (size_t)m * d + i) = v;
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
     if (!g) return;
     ss = block_sum(ss, scratch);
     const float rstd = 1.0f / sqrtf(ss / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) xn[(size_t)m * d + i] = row[i] * rstd * g[i];
+    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+        const float4 r4 = *reinterpret_cast<const float4 *>(row + i);
+        const float4 g4 = *reinterpret_cast<const float4 *>(g + i);
+        const float4 v = make_float4(r4.x * rstd * g4.x, r4.y * rstd * g4.y, r4.z * rstd * g4.z, r4.w * rstd * g4.w);
+        *reinterpret_cast<float4 *>(xn + (size_t)m * d + i) = v;
+        if (xs) {
+            store_split(xs, m, d, i, v.x); store_split(xs, m, d, i + 1, v.y);
+            store_split(xs, m, d, i + 2, v.z); store_split(xs, m, d, i + 3, v.w);
+        }
+    }
 }
-void launch_resid_norm(cudaStream_t s, float *x, const float *part, int S, const float *g, float *xn, float *cap,
+void launch_resid_norm(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
                        int M, int d, float eps) {
     size_t smem = (size_t)(d + 33) * sizeof(float);
-    size_t stride = (size_t)M * d;
-    if (!part) S = 0;
-    resid_norm_kernel<<<M, 256, smem, s>>>(x, part, S, stride, g, xn, cap, d, eps);
+    PartView none = {};
+    resid_norm_kernel<<<M, 1024, smem, s>>>(x, pv ? *pv : none, pv != nullptr, g, xn, (bf16 *)xs, cap, d, eps);
 }
 
 // ------------------------------------------------------------------------------------ skinny projection (SIMT)
@@ -169,17 +217,12 @@ int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float 
 // ------------------------------------------------------------------------------------ RoPE + KV append
 // grid (heads, M), block D/2: one thread per rotation pair.
 template <typename AT>
-__global__ void qkv_post_kernel(const float *part, int S, size_t part_stride, int Rw, int pos0, int H, KvGeom kv,
-                                const float2 *rope, float *q, int head_off, int *err) {
+__global__ void qkv_post_kernel(PartView pv, int pos0, int H, KvGeom kv, const float2 *rope, float *q, int head_off,
+                                int *err) {
     const int hh = blockIdx.x + head_off;  // 0..H-1 q, H..H+Hkv-1 k, then v
     const int m = blockIdx.y, i = threadIdx.x, D = kv.D;
     const int col = blockIdx.x * D + 2 * i;
-    float a = 0.f, b = 0.f;
-    for (int s = 0; s < S; s++) {
-        const float *p = part + (size_t)s * part_stride + (size_t)m * Rw + col;
-        a += p[0];
-        b += p[1];
-    }
+    float a = part_gather(pv, m, col), b = part_gather(pv, m, col + 1);
     const int pos = pos0 + m;
     if (hh < H + kv.Hkv) {
         float2 cs = rope[(size_t)pos * (D / 2) + i];
@@ -203,142 +246,191 @@ __global__ void qkv_post_kernel(const float *part, int S, size_t part_stride, in
     dst[0] = from_f<AT>(a);
     dst[1] = from_f<AT>(b);
 }
-void launch_qkv_post(cudaStream_t s, int dtype, const float *part, int S, int M, int pos0, int H,
+void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, int M, int pos0, int H,
                      const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err) {
     const int heads = only_kv ? 2 * kv.Hkv : H + 2 * kv.Hkv;
-    const int Rw = heads * kv.D;
     dim3 grid(heads, M);
-    size_t stride = (size_t)M * Rw;
-    if (dtype == 0) qkv_post_kernel<float><<<grid, kv.D / 2, 0, s>>>(part, S, stride, Rw, pos0, H, kv, rope, q, only_kv ? H : 0, err);
-    else qkv_post_kernel<bf16><<<grid, kv.D / 2, 0, s>>>(part, S, stride, Rw, pos0, H, kv, rope, q, only_kv ? H : 0, err);
+    if (dtype == 0) qkv_post_kernel<float><<<grid, kv.D / 2, 0, s>>>(pv, pos0, H, kv, rope, q, only_kv ? H : 0, err);
+    else qkv_post_kernel<bf16><<<grid, kv.D / 2, 0, s>>>(pv, pos0, H, kv, rope, q, only_kv ? H : 0, err);
 }
 
 // ------------------------------------------------------------------------------------ paged decode attention
-// grid (H, n_split), 256 threads.  Block (h, sp) handles query head h for all M new rows over
-// its share of the cached positions [0, pos0 + M) (split by pages); row m sees positions
-// <= pos0 + m.  Writes un-normalised output, running max and sum per row; the combine kernel
-// merges the splits in index order.
+// grid (H_kv, n_split), 256 threads.  Block (kh, sp) owns up to kAttnPos cached positions of
+// KV head kh (a whole number of pages) and serves every query head of its group and all M new
+// rows from ONE copy of those keys and values: the page blocks ([page_tokens][D], contiguous)
+// are brought into shared memory by bulk asynchronous copies on one mbarrier, so the cache is
+// read from HBM once per KV head.  Row m sees positions <= pos0 + m.  The block writes, per
+// (query head, row), the un-normalised output, the maximum and the sum of its slice; the
+// combine kernel merges the slices in index order.
+constexpr int kAttnPos = 128;     // positions per block
+constexpr int kAttnRows = 32;     // (head, row) pairs processed per batch
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
 template <typename AT, int D>
 __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, KvGeom kv, float *__restrict__ apart,
-                                                   int M, int pos0, int H, int n_split, float scale) {
-    constexpr int CH = 128;        // positions per chunk
-    constexpr int G = 256 / D;     // row groups in the PV phase
-    constexpr int RPG = kMaxRows / G;
-    constexpr int VEC = Vec16<AT>::N;
-    __shared__ __align__(16) float sq[kMaxRows][D];
-    __shared__ float ssc[kMaxRows][CH];
-    __shared__ float s_m[kMaxRows], s_l[kMaxRows], s_c[kMaxRows];
+                                                   int M, int pos0, int H, int pps, int n_split, float scale, int *err) {
+    constexpr int VEC = Vec16<AT>::N;       // elements per 16-byte chunk
+    constexpr int NCH = D / VEC;            // chunks per row
+    extern __shared__ __align__(128) unsigned char attn_smem[];
+    AT *sK = reinterpret_cast<AT *>(attn_smem);
+    AT *sV = sK + kAttnPos * D;
+    float *sq = reinterpret_cast<float *>(sV + kAttnPos * D);   // [kAttnRows][D]
+    float *sS = sq + kAttnRows * D;                              // [kAttnRows][kAttnPos]
+    float *s_m = sS + kAttnRows * kAttnPos;                      // [kAttnRows]
+    float *s_l = s_m + kAttnRows;
+    uint64_t *bar = reinterpret_cast<uint64_t *>(s_l + kAttnRows);
+
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int h = blockIdx.x, sp = blockIdx.y, kh = h / (H / kv.Hkv);
-    const int PT = kv.page_tokens;
+    const int kh = blockIdx.x, sp = blockIdx.y;
+    const int PT = kv.page_tokens, group = H / kv.Hkv;
     const int ctx_len = pos0 + M;
     const int n_pages = (ctx_len + PT - 1) / PT;
-    const int pps = (n_pages + n_split - 1) / n_split;
-    const int lo = sp * pps * PT;
-    const int hi = min(ctx_len, lo + pps * PT);
-    const AT *base = (const AT *)kv.slot_base;
-    const size_t head_stride = (size_t)PT * D;
+    const int page_lo = sp * pps, page_hi = min(n_pages, page_lo + pps);
+    const int lo = page_lo * PT;
+    const int npos = min(ctx_len, page_hi * PT) - lo;   // valid positions of this block
+    const uint32_t blk_bytes = (uint32_t)(PT * D * sizeof(AT));
 
-    for (int idx = tid; idx < kMaxRows * D; idx += 256) {
-        int m = idx / D, e = idx - m * D;
-        sq[m][e] = m < M ? q[(size_t)m * H * D + (size_t)h * D + e] * scale : 0.f;
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(bar)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (tid < kMaxRows) { s_m[tid] = -INFINITY; s_l[tid] = 0.f; s_c[tid] = 1.f; }
-    float o[RPG];
-#pragma unroll
-    for (int r = 0; r < RPG; r++) o[r] = 0.f;
     __syncthreads();
-
-    for (int c0 = lo; c0 < hi; c0 += CH) {
-        {   // phase 1: scores.  thread -> position j, half of the rows
-            const int j = tid & (CH - 1), half = tid / CH;
-            const int pos = c0 + j;
-            const bool valid = pos < hi;
-            float acc[8];
+    if (tid == 0) {
+        const uint32_t total = 2u * blk_bytes * (uint32_t)(page_hi - page_lo);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(total) : "memory");
+        for (int pg = page_lo; pg < page_hi; pg++) {
+            const int page = kv.page_table[pg];
+            const AT *src = (const AT *)kv.slot_base + (((size_t)page * 2) * kv.Hkv + kh) * (size_t)PT * D;
+            const size_t v_off = (size_t)kv.Hkv * PT * D;
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(sK + (size_t)(pg - page_lo) * PT * D)), "l"(src), "r"(blk_bytes), "r"(smem_addr(bar)) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(sV + (size_t)(pg - page_lo) * PT * D)), "l"(src + v_off), "r"(blk_bytes), "r"(smem_addr(bar)) : "memory");
+        }
+    }
+    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
+    bool landed = false;
+    for (int r0 = 0; r0 < rows; r0 += kAttnRows) {
+        const int nb = min(kAttnRows, rows - r0);
+        for (int idx = tid; idx < nb * D; idx += 256) {
+            const int rl = idx / D, e = idx - rl * D;
+            const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
+            sq[rl * D + e] = q[(size_t)m * H * D + (size_t)(kh * group + g) * D + e] * scale;
+        }
+        if (!landed) {
+            bool ok = false;
+            for (uint32_t i = 0; i < (1u << 24) && !ok; i++) {
+                uint32_t p;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(p) : "r"(smem_addr(bar)) : "memory");
+                ok = p != 0;
+                if (!ok) __nanosleep(32);
+            }
+            if (!ok && tid == 0) atomicOr(err, kErrWaitTimeout);
+            landed = true;
+        }
+        __syncthreads();
+        {   // scores: thread -> position j, every second row of the batch
+            const int j = tid & (kAttnPos - 1), rsel = tid >> 7;
+            float acc[kAttnRows / 2];
 #pragma unroll
-            for (int r = 0; r < 8; r++) acc[r] = 0.f;
-            if (valid && half * 8 < M) {
-                const int page = kv.page_table[pos / PT];
-                const AT *kp = base + (((size_t)page * 2 + 0) * kv.Hkv + kh) * head_stride + (size_t)(pos % PT) * D;
-#pragma unroll 4
-                for (int e0 = 0; e0 < D; e0 += VEC) {
+            for (int i = 0; i < kAttnRows / 2; i++) acc[i] = 0.f;
+            if (j < npos) {
+#pragma unroll 2
+                for (int c = 0; c < NCH; c++) {
+                    const int cc = (c + j) % NCH;   // rotate the chunk order: conflict-free shared loads
                     float kvv[VEC];
-                    Vec16<AT>::load(kp + e0, kvv);
+                    if (sizeof(AT) == 2) Vec16<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4 *>(sK + (size_t)j * D + cc * VEC), kvv);
+                    else {
+                        const float4 t = *reinterpret_cast<const float4 *>(sK + (size_t)j * D + cc * VEC);
+                        kvv[0] = t.x; kvv[1] = t.y; kvv[2] = t.z; kvv[3] = t.w;
+                    }
 #pragma unroll
-                    for (int r = 0; r < 8; r++) {
-                        const int m = half * 8 + r;
-                        if (m < M) {
+                    for (int i = 0; i < kAttnRows / 2; i++) {
+                        const int rl = rsel + 2 * i;
+                        if (rl < nb) {
+                            float qv[VEC];
 #pragma unroll
-                            for (int v = 0; v < VEC; v++) acc[r] = fmaf(kvv[v], sq[m][e0 + v], acc[r]);
+                            for (int v = 0; v < VEC; v += 4) {
+                                const float4 t = *reinterpret_cast<const float4 *>(sq + rl * D + cc * VEC + v);
+                                qv[v] = t.x; qv[v + 1] = t.y; qv[v + 2] = t.z; qv[v + 3] = t.w;
+                            }
+#pragma unroll
+                            for (int v = 0; v < VEC; v++) acc[i] = fmaf(kvv[v], qv[v], acc[i]);
                         }
                     }
                 }
             }
 #pragma unroll
-            for (int r = 0; r < 8; r++) {
-                const int m = half * 8 + r;
-                ssc[m][j] = (valid && m < M && pos <= pos0 + m) ? acc[r] : -INFINITY;
+            for (int i = 0; i < kAttnRows / 2; i++) {
+                const int rl = rsel + 2 * i;
+                if (rl < nb) {
+                    const int m = (r0 + rl) % M;
+                    sS[rl * kAttnPos + j] = (j < npos && lo + j <= pos0 + m) ? acc[i] : -INFINITY;
+                }
             }
         }
         __syncthreads();
-        // phase 2: online softmax bookkeeping, warp w handles rows w and w + 8
-        for (int m = warp; m < M; m += 8) {
+        for (int rl = warp; rl < nb; rl += 8) {   // softmax numerators of this slice
             float mx = -INFINITY;
-            for (int j = lane; j < CH; j += 32) mx = fmaxf(mx, ssc[m][j]);
+            for (int j = lane; j < kAttnPos; j += 32) mx = fmaxf(mx, sS[rl * kAttnPos + j]);
             mx = warp_max(mx);
-            const float m_old = s_m[m];
-            const float m_new = fmaxf(m_old, mx);
             float sum = 0.f;
-            for (int j = lane; j < CH; j += 32) {
-                float sv = ssc[m][j];
-                float p = (sv == -INFINITY) ? 0.f : expf(sv - m_new);
-                ssc[m][j] = p;
+            for (int j = lane; j < kAttnPos; j += 32) {
+                const float sv = sS[rl * kAttnPos + j];
+                const float p = (sv == -INFINITY) ? 0.f : expf(sv - mx);
+                sS[rl * kAttnPos + j] = p;
                 sum += p;
             }
             sum = warp_sum(sum);
-            if (lane == 0) {
-                float c = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);
-                s_c[m] = c;
-                s_l[m] = s_l[m] * c + sum;
-                s_m[m] = m_new;
-            }
+            if (lane == 0) { s_m[rl] = mx; s_l[rl] = sum; }
         }
         __syncthreads();
-        {   // phase 3: o = o * c + P V.  thread -> (d, row group)
-            const int dd = tid % D, grp = tid / D;
+        {   // o = P V: thread -> (pair of d, row group)
+            constexpr int HALF = D / 2, NG = 256 / HALF, RPT = kAttnRows / NG;
+            const int d2 = tid % HALF, rg = tid / HALF;
+            float o0[RPT], o1[RPT];
 #pragma unroll
-            for (int r = 0; r < RPG; r++) o[r] *= s_c[grp * RPG + r];
-            const int nj = min(CH, hi - c0);
-            if (grp * RPG < M) {
-                for (int j = 0; j < nj; j++) {
-                    const int pos = c0 + j;
-                    const int page = kv.page_table[pos / PT];
-                    const float v = to_f(base[(((size_t)page * 2 + 1) * kv.Hkv + kh) * head_stride +
-                                              (size_t)(pos % PT) * D + dd]);
+            for (int i = 0; i < RPT; i++) { o0[i] = 0.f; o1[i] = 0.f; }
+            for (int j = 0; j < npos; j++) {
+                float v0, v1;
+                if (sizeof(AT) == 2) {
+                    const uint32_t w = *reinterpret_cast<const uint32_t *>(sV + (size_t)j * D + 2 * d2);
+                    v0 = __uint_as_float(w << 16); v1 = __uint_as_float(w & 0xFFFF0000u);
+                } else {
+                    const float2 t = *reinterpret_cast<const float2 *>(sV + (size_t)j * D + 2 * d2);
+                    v0 = t.x; v1 = t.y;
+                }
 #pragma unroll
-                    for (int r = 0; r < RPG; r++) o[r] = fmaf(ssc[grp * RPG + r][j], v, o[r]);
+                for (int i = 0; i < RPT; i++) {
+                    const int rl = rg + NG * i;
+                    if (rl < nb) {
+                        const float p = sS[rl * kAttnPos + j];
+                        o0[i] = fmaf(p, v0, o0[i]);
+                        o1[i] = fmaf(p, v1, o1[i]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < RPT; i++) {
+                const int rl = rg + NG * i;
+                if (rl < nb) {
+                    const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
+                    float *dst = apart + (((size_t)(kh * group + g) * n_split + sp) * kMaxRows + m) * (D + 2);
+                    dst[2 * d2] = o0[i];
+                    dst[2 * d2 + 1] = o1[i];
+                    if (d2 == 0) { dst[D] = s_m[rl]; dst[D + 1] = s_l[rl]; }
                 }
             }
         }
         __syncthreads();
     }
-    {
-        const int dd = tid % D, grp = tid / D;
-        float *dst = apart + ((size_t)h * n_split + sp) * kMaxRows * (D + 2);
-#pragma unroll
-        for (int r = 0; r < RPG; r++) {
-            const int m = grp * RPG + r;
-            if (m < M) dst[(size_t)m * (D + 2) + dd] = o[r];
-        }
-        if (tid < M) {
-            dst[(size_t)tid * (D + 2) + D] = s_m[tid];
-            dst[(size_t)tid * (D + 2) + D + 1] = s_l[tid];
-        }
-    }
 }
 
 // grid (H, M), block D: merge the splits of one (head, row)
-__global__ void attn_combine_kernel(const float *apart, float *out, int H, int D, int n_split) {
+__global__ void attn_combine_kernel(const float *apart, float *out, bf16 *out_split, int H, int D, int n_split) {
     const int h = blockIdx.x, m = blockIdx.y, dd = threadIdx.x;
     const float *src = apart + (size_t)h * n_split * kMaxRows * (D + 2) + (size_t)m * (D + 2);
     const size_t sstride = (size_t)kMaxRows * (D + 2);
@@ -352,52 +444,72 @@ __global__ void attn_combine_kernel(const float *apart, float *out, int H, int D
         num = fmaf(w, src[s * sstride + dd], num);
         den = fmaf(w, src[s * sstride + D + 1], den);
     }
-    out[(size_t)m * H * D + (size_t)h * D + dd] = den > 0.f ? num / den : 0.f;
+    const float o = den > 0.f ? num / den : 0.f;
+    out[(size_t)m * H * D + (size_t)h * D + dd] = o;
+    if (out_split) store_split(out_split, m, (size_t)H * D, (size_t)h * D + dd, o);
+}
+
+template <typename AT, int D>
+static void attn_launch(cudaStream_t s, const float *q, const KvGeom &kv, float *apart, int M, int pos0, int H, int pps,
+                        int n_split, float scale, int *err) {
+    const size_t smem = (size_t)2 * kAttnPos * D * sizeof(AT) + (size_t)kAttnRows * D * 4 +
+                        (size_t)kAttnRows * kAttnPos * 4 + 2 * kAttnRows * 4 + 16;
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(attn_kernel<AT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        configured = true;
+    }
+    attn_kernel<AT, D><<<dim3(kv.Hkv, n_split), 256, smem, s>>>(q, kv, apart, M, pos0, H, pps, n_split, scale, err);
+}
+
+int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_sm, int max_splits, int *pps_out) {
+    const int n_pages = (ctx_len + page_tokens - 1) / page_tokens;
+    int pps = kAttnPos / page_tokens;                 // most pages one block can hold
+    if (pps < 1) pps = 1;
+    // enough blocks to fill the machine about twice, while slices stay whole pages
+    while (pps > 1 && Hkv * ((n_pages + pps - 1) / pps) < 2 * n_sm) pps--;
+    int n_split = (n_pages + pps - 1) / pps;
+    while (n_split > max_splits) { pps++; n_split = (n_pages + pps - 1) / pps; }
+    *pps_out = pps;
+    return n_split;
 }
 
 void launch_attention(cudaStream_t s, int dtype, const float *q, const KvGeom &kv, float *apart,
-                      float *attn_out, int M, int pos0, int H, int n_split) {
-    dim3 grid(H, n_split);
+                      float *attn_out, void *attn_split, int M, int pos0, int H, int n_sm, int max_splits, int *err) {
+    int pps;
+    const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, n_sm, max_splits, &pps);
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (dtype == 0) {
-        if (kv.D == 64) attn_kernel<float, 64><<<grid, 256, 0, s>>>(q, kv, apart, M, pos0, H, n_split, scale);
-        else attn_kernel<float, 128><<<grid, 256, 0, s>>>(q, kv, apart, M, pos0, H, n_split, scale);
+        if (kv.D == 64) attn_launch<float, 64>(s, q, kv, apart, M, pos0, H, pps, n_split, scale, err);
+        else attn_launch<float, 128>(s, q, kv, apart, M, pos0, H, pps, n_split, scale, err);
     } else {
-        if (kv.D == 64) attn_kernel<bf16, 64><<<grid, 256, 0, s>>>(q, kv, apart, M, pos0, H, n_split, scale);
-        else attn_kernel<bf16, 128><<<grid, 256, 0, s>>>(q, kv, apart, M, pos0, H, n_split, scale);
+        if (kv.D == 64) attn_launch<bf16, 64>(s, q, kv, apart, M, pos0, H, pps, n_split, scale, err);
+        else attn_launch<bf16, 128>(s, q, kv, apart, M, pos0, H, pps, n_split, scale, err);
     }
-    attn_combine_kernel<<<dim3(H, M), kv.D, 0, s>>>(apart, attn_out, H, kv.D, n_split);
+    attn_combine_kernel<<<dim3(H, M), kv.D, 0, s>>>(apart, attn_out, (bf16 *)attn_split, H, kv.D, n_split);
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU, partial sums
-__global__ void swiglu_kernel(const float *part, int S, size_t part_stride, float *h, int F) {
+__global__ void swiglu_kernel(PartView pv, float *h, bf16 *hs, int F) {
     const int m = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= F) return;
-    float g = 0.f, u = 0.f;
-    for (int s = 0; s < S; s++) {
-        const float *p = part + (size_t)s * part_stride + (size_t)m * 2 * F;
-        g += p[i];
-        u += p[F + i];
-    }
-    const float sg = g / (1.0f + expf(-g));
-    h[(size_t)m * F + i] = sg * u;
+    const float g = part_gather(pv, m, i), u = part_gather(pv, m, F + i);
+    const float v = g / (1.0f + expf(-g)) * u;
+    h[(size_t)m * F + i] = v;
+    if (hs) store_split(hs, m, F, i, v);
 }
-void launch_swiglu(cudaStream_t s, const float *part, int S, float *h, int M, int F) {
+void launch_swiglu(cudaStream_t s, const PartView &pv, float *h, void *h_split, int M, int F) {
     dim3 grid((F + 255) / 256, M);
-    size_t stride = (size_t)M * 2 * F;
-    swiglu_kernel<<<grid, 256, 0, s>>>(part, S, stride, h, F);
+    swiglu_kernel<<<grid, 256, 0, s>>>(pv, h, (bf16 *)h_split, F);
 }
 
-__global__ void reduce_partials_kernel(const float *part, int S, size_t stride, float *out, size_t n) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    float v = 0.f;
-    for (int s = 0; s < S; s++) v += part[(size_t)s * stride + i];
-    out[i] = v;
+__global__ void reduce_partials_kernel(PartView pv, float *out, int R) {
+    const int m = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= R) return;
+    out[(size_t)m * R + r] = part_gather(pv, m, r);
 }
-void launch_reduce_partials(cudaStream_t s, const float *part, int S, float *out, int M, int R) {
-    size_t n = (size_t)M * R;
-    reduce_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(part, S, n, out, n);
+void launch_reduce_partials(cudaStream_t s, const PartView &pv, float *out, int M, int R) {
+    reduce_partials_kernel<<<dim3((R + 255) / 256, M), 256, 0, s>>>(pv, out, R);
 }
 
 }  // namespace eesd

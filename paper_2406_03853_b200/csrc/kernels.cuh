@@ -2,6 +2,7 @@
 // and selects the element type of the weights and of the KV cache; the residual stream, the
 // token rows fed to projections, partial sums, attention statistics and logits are fp32.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -17,23 +18,58 @@ struct KvGeom {
     int Hkv, D, page_tokens, n_pages_total;
 };
 
+// Equal split of U = tiles * KB work units (128-row weight tile x 64-wide k block) over G
+// CTAs: CTA c owns units [start(c), start(c+1)); the first `rem` CTAs own one unit more.
+struct StreamK {
+    int U, KB, G, base, rem, max_seg;
+    __host__ __device__ int start(int c) const { return c * base + (c < rem ? c : rem); }
+    __host__ __device__ int owner(int u) const {
+        const int bnd = rem * (base + 1);
+        return u < bnd ? u / (base + 1) : rem + (u - bnd) / base;
+    }
+    __host__ __device__ int first_tile(int c) const { return start(c) / KB; }
+};
+
+// Where a projection left its fp32 partial sums.
+//   mode 0: base[s * split_stride + m * R + r], s < S           (SIMT kernel, S = 1)
+//   mode 1: one [16][128] block per (CTA, segment) of the stream-K tensor-core kernel
+struct PartView {
+    const float *base;
+    int mode, S, R;
+    size_t split_stride;
+    StreamK sk;
+};
+
 void launch_set_ints(cudaStream_t s, int32_t *dst, const IntList16 &vals, int n);
 void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float theta);
 void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
                   int M, int d, int V, int *err);
 // x[m] += sum_s part[s][m] (if part); xn[m] = cast(RMSNorm(x[m]) * g) (if g); cap[m] = x[m] (if cap)
-void launch_resid_norm(cudaStream_t s, float *x, const float *part, int S, const float *g, float *xn, float *cap,
+// `xs` (may be null): the same rows as two bf16 terms, [32][d]: rows 0..15 hi, 16..31 lo
+void launch_resid_norm(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
                        int M, int d, float eps);
 // out[sp][m][r] = sum_{k in split sp} A[m][k] * W[r][k]; returns the number of K splits written
 int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float *out, int M, int R, int K);
 // RoPE + KV append (+ q store).  part rows are [q heads | k heads | v heads] or, when
 // only_kv, [k heads | v heads].
-void launch_qkv_post(cudaStream_t s, int dtype, const float *part, int S, int M, int pos0, int H,
+void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, int M, int pos0, int H,
                      const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err);
+// apart: room for H * max_splits * 16 * (D + 2) floats; page_tokens * D elements per page block
+// must not exceed 128 * D (page_tokens <= 128)
 void launch_attention(cudaStream_t s, int dtype, const float *q, const KvGeom &kv, float *apart,
-                      float *attn_out, int M, int pos0, int H, int n_split);
-void launch_swiglu(cudaStream_t s, const float *part, int S, float *h, int M, int F);
-void launch_reduce_partials(cudaStream_t s, const float *part, int S, float *out, int M, int R);
+                      float *attn_out, void *attn_split, int M, int pos0, int H, int n_sm, int max_splits, int *err);
+void launch_swiglu(cudaStream_t s, const PartView &pv, float *h, void *h_split, int M, int F);
+void launch_reduce_partials(cudaStream_t s, const PartView &pv, float *out, int M, int R);
+
+// tensor-core projection (gemm_tc.cu)
+int tc_init();                                   // once per process; 0 on success
+bool tc_shape_ok(int R, int K);
+bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows);
+StreamK tc_plan(int R, int K, int n_sm);
+size_t tc_partial_floats(const StreamK &sk);
+void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
+                    int M, int *err);
+void launch_split_rows(cudaStream_t s, const float *x, void *xs, int M, int K);
 
 // acceptance / sampling (accept.cu)
 size_t accept_scratch_bytes(int B, int K);

@@ -13,7 +13,7 @@ def oracle_from_spec(spec, max_ctx=256, n_layers=None, device="cpu", seed=synth.
     ex = {k: v.cpu() for k, v in synth.exit_layer_weights(spec, seed, device).items()}
     emb = synth.embedding(spec, seed, device).cpu()
     head = synth.lm_head(spec, seed, device).cpu()
-    s = spec.with_(n_layers=L)
+    s = spec.with_(n_layers=L, n_early=min(spec.n_early, L))
     return oracle.model_from_weights(s, layers, ex, emb, head, max_ctx=max_ctx, kv_bf16=kv_bf16)
 
 
