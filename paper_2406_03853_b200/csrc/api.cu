@@ -27,6 +27,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 int check_config(const eesd_config *c) {
     if (!c) return EESD_ERR_BADARG;
+    if (c->d_model > 1024 * kSsqBlocks || c->n_kv_heads > 1024) return EESD_ERR_UNSUPPORTED;
     if (c->d_model <= 0 || c->n_heads <= 0 || c->n_kv_heads <= 0 || c->ffn_dim <= 0 || c->vocab <= 0 ||
         c->n_layers <= 0 || c->max_ctx <= 1)
         return EESD_ERR_BADARG;
@@ -46,7 +47,7 @@ int check_config(const eesd_config *c) {
 }
 
 struct Workspace {
-    size_t x, xn, q, attn, h, xs[3], part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
+    size_t x, xn, q, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
         accept, total;
 };
 
@@ -75,6 +76,8 @@ Workspace carve(const eesd_config *c) {
     w.xs[X_NORM] = take(2 * R * (size_t)c->d_model * 2);
     w.xs[X_ATTN] = take(2 * R * qd * 2);
     w.xs[X_FFN] = take(2 * R * (size_t)c->ffn_dim * 2);
+    w.ssq = take((size_t)EESD_MAX_ROWS * kSsqBlocks * 4);
+    w.tickets = take(1024 * 4);
     {   // partial sums: SIMT layout [splits][16][maxR], or stream-K blocks of the widest projection
         size_t part_floats = (size_t)kPartSplits * R * maxR;
         const size_t sk_floats = (maxR / 128 + 3 * (size_t)kMaxSm) * R * 128;  // >= G * max_seg blocks
@@ -112,6 +115,8 @@ struct eesd_ctx {
     float *x, *xn, *q, *attn, *h, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
     void *accept_scratch;
     void *xs[3];                 // bf16 hi/lo copies of xn, attn, h
+    float *ssq;                  // RMSNorm partial sums of squares of the rows in xn / xs[X_NORM]
+    unsigned int *tickets;       // arrival counters of the attention merge
     CUtensorMap m_x[3];
     CUtensorMap m_exit_kv, m_lm_head, m_exit_head;
     bool use_tc;
@@ -218,23 +223,39 @@ PartView run_proj(eesd_ctx *c, const void *W, const CUtensorMap *mW, int which, 
     return pv;
 }
 
-// one decoder layer on M rows at positions pos0.. ; on entry xn = RMSNorm(x) * g_attn of this
-// layer; on exit x holds the layer output and, when g_next is given, xn = RMSNorm(x) * g_next.
+RowScale norm_scale(eesd_ctx *c) {
+    RowScale rs;
+    rs.ssq = c->ssq;
+    rs.nblk = (c->cfg.d_model + 1023) / 1024;
+    rs.inv_d = 1.0f / (float)c->cfg.d_model;
+    rs.eps = c->cfg.rms_eps;
+    return rs;
+}
+
+// residual update + the input of the next normalised projection: x += partials; y = x * g
+void run_resid(eesd_ctx *c, const PartView *pv, const float *g, float *cap, int M) {
+    launch_resid(c->stream, c->x, pv, g, c->use_tc ? nullptr : c->xn, c->xs[X_NORM], cap, c->ssq, M, c->cfg.d_model);
+    c->launches++;
+}
+
+// one decoder layer on M rows at positions pos0.. ; on entry y = x * g_attn of this layer (and
+// its sums of squares) are in place; on exit x holds the layer output and y = x * g_next.
 void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const float *g_next, float *cap) {
     const eesd_config &f = c->cfg;
     const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim, d = f.d_model, F = f.ffn_dim;
     cudaStream_t s = c->stream;
-    KvGeom kv = kv_geom(c, slot);
+    const RowScale rs = norm_scale(c), none = {nullptr, 0, 0.f, 0.f};
+    (void)none;
     PartView pv = run_proj(c, w.wqkv, &w.m_qkv, X_NORM, M, qd + 2 * kvd, d);
-    launch_qkv_post(s, f.dtype, pv, M, pos0, f.n_heads, kv, c->rope, c->q, false, c->err);
-    launch_attention(s, f.dtype, c->q, kv, c->apart, c->attn, c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, c->err);
+    launch_attention(s, f.dtype, pv, rs, c->rope, kv_geom(c, slot), c->apart, c->tickets, c->use_tc ? nullptr : c->attn,
+                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, c->err);
     pv = run_proj(c, w.wo, &w.m_o, X_ATTN, M, d, qd);
-    launch_resid_norm(s, c->x, &pv, w.g_ffn, c->xn, c->xs[X_NORM], nullptr, M, d, f.rms_eps);
+    run_resid(c, &pv, w.g_ffn, nullptr, M);
     pv = run_proj(c, w.wgu, &w.m_gu, X_NORM, M, 2 * F, d);
-    launch_swiglu(s, pv, c->h, c->xs[X_FFN], M, F);
+    launch_swiglu(s, pv, rs, c->use_tc ? nullptr : c->h, c->xs[X_FFN], M, F);
     pv = run_proj(c, w.wd, &w.m_d, X_FFN, M, d, F);
-    launch_resid_norm(s, c->x, &pv, g_next, c->xn, c->xs[X_NORM], cap, M, d, f.rms_eps);
-    c->launches += 6;
+    run_resid(c, &pv, g_next, cap, M);
+    c->launches += 2;
 }
 
 float *cap_slot(eesd_ctx *c, int index) {
@@ -248,8 +269,8 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
     cudaStream_t s = c->stream;
     const int L = f.n_layers, d = f.d_model;
     launch_embed(s, f.dtype, d_tok, c->embed, c->x, cap_slot(c, 0), M, d, f.vocab, c->err);
-    launch_resid_norm(s, c->x, nullptr, c->layers[0].g_attn, c->xn, c->xs[X_NORM], nullptr, M, d, f.rms_eps);
-    c->launches += 2;
+    run_resid(c, nullptr, c->layers[0].g_attn, nullptr, M);
+    c->launches += 1;
     for (int l = 0; l < L; l++) {
         const bool exit_here = (l == f.n_early - 1);
         const float *g_after = exit_here ? c->layers[L].g_attn : (l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
@@ -259,15 +280,15 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
             const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim;
             const char *wkv = c->layers[L].wqkv + (size_t)qd * d * c->es;
             PartView pv = run_proj(c, wkv, &c->m_exit_kv, X_NORM, M, 2 * kvd, d);
-            launch_qkv_post(s, f.dtype, pv, M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err);
+            launch_qkv_post(s, f.dtype, pv, norm_scale(c), M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err);
             const float *g_next = l + 1 < L ? c->layers[l + 1].g_attn : c->g_final;
-            launch_resid_norm(s, c->x, nullptr, g_next, c->xn, c->xs[X_NORM], nullptr, M, d, f.rms_eps);
-            c->launches += 2;
+            run_resid(c, nullptr, g_next, nullptr, M);
+            c->launches += 1;
         }
     }
     if (want_logits) {
         PartView pv = run_proj(c, c->lm_head, &c->m_lm_head, X_NORM, M, f.vocab, d);
-        launch_reduce_partials(s, pv, c->logits_p, M, f.vocab);
+        launch_reduce_partials(s, pv, norm_scale(c), c->logits_p, M, f.vocab);
         c->launches += 1;
     }
     return check_launch(c);
@@ -280,7 +301,7 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
     cudaStream_t s = c->stream;
     const int L = f.n_layers, d = f.d_model, N = f.n_early;
     launch_embed(s, f.dtype, c->ints + kRoundTok + i, c->embed, c->x, cap_slot(c, 0), 1, d, f.vocab, c->err);
-    launch_resid_norm(s, c->x, nullptr, c->layers[0].g_attn, c->xn, c->xs[X_NORM], nullptr, 1, d, f.rms_eps);
+    run_resid(c, nullptr, c->layers[0].g_attn, nullptr, 1);
     for (int l = 0; l < N; l++) {
         const float *g_after = l + 1 < N ? c->layers[l + 1].g_attn : c->layers[L].g_attn;
         run_layer(c, c->layers[l], l, 1, pos, g_after, cap_slot(c, l + 1));
@@ -288,9 +309,9 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
     run_layer(c, c->layers[L], L, 1, pos, c->g_exit, cap_slot(c, L + 1));
     float *lq = c->logits_q + (size_t)i * f.vocab;
     PartView pv = run_proj(c, c->exit_head, &c->m_exit_head, X_NORM, 1, f.vocab, d);
-    launch_reduce_partials(s, pv, lq, 1, f.vocab);
+    launch_reduce_partials(s, pv, norm_scale(c), lq, 1, f.vocab);
     launch_sample_rows(s, lq, d_u, 1, f.vocab, f.temperature, c->ints + kRoundTok + i + 1);
-    c->launches += 4;
+    c->launches += 3;
     return check_launch(c);
 }
 
@@ -508,6 +529,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->rope = (float2 *)(ws + w.rope); c->page_table = (int32_t *)(ws + w.page_table);
     c->ints = (int32_t *)(ws + w.ints); c->u_dev = (float *)(ws + w.u_dev); c->u_stage = (float *)(ws + w.u_stage);
     c->err = (int *)(ws + w.err); c->accept_scratch = ws + w.accept;
+    c->ssq = (float *)(ws + w.ssq); c->tickets = (unsigned int *)(ws + w.tickets);
     for (int i = 0; i < 3; i++) c->xs[i] = nullptr;
     c->n_sm = 1;
     {
@@ -565,6 +587,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     }
     memset(c->h_result, 0, 256);
     cudaMemsetAsync(c->err, 0, 16, c->stream);
+    cudaMemsetAsync(c->tickets, 0, 1024 * 4, c->stream);
     cudaMemsetAsync(c->ints, 0, kIntSlots * 4, c->stream);
     cudaMemsetAsync(c->accept_scratch, 0, accept_scratch_bytes(1, EESD_MAX_ROWS), c->stream);
     launch_rope_table(c->stream, c->rope, cfg->max_ctx, cfg->head_dim, cfg->rope_theta);
@@ -876,7 +899,8 @@ int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *
         pv.S = launch_gemm(s, dtype, A, W, part, M, R, K);
         pv.split_stride = (size_t)M * R;
     }
-    launch_reduce_partials(s, pv, out, M, R);
+    const RowScale none = {nullptr, 0, 0.f, 0.f};
+    launch_reduce_partials(s, pv, none, out, M, R);
     return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
 }
 

@@ -77,6 +77,27 @@ __device__ __forceinline__ float block_sum(float v, float *scratch /* >= 33 floa
     return scratch[32];
 }
 
+// Programmatic dependent launch.  pdl_trigger lets the next kernel in the stream be scheduled
+// early; pdl_wait blocks until every kernel this one depends on has completed and its writes
+// are visible.  Both are no-ops for kernels launched without the attribute.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // writes v as two bf16 terms into a [2 * kMaxRows][K] matrix: row m gets hi, row kMaxRows + m gets lo
 __device__ __forceinline__ void store_split(__nv_bfloat16 *xs, int m, size_t K, size_t i, float v) {
     const __nv_bfloat16 hi = __float2bfloat16_rn(v);

@@ -141,6 +141,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
     const int u0 = sk.start(cta), u1 = sk.start(cta + 1);
+    pdl_trigger();
 
     if (tid == 0) {
         for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
@@ -161,9 +162,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (warp == 4) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            int issued = 0;
+            // The weights do not depend on the kernel before this one: fill the ring with weight
+            // tiles at once, and only then wait for the producer of the token rows.
+            const int pre = min(u1 - u0, STAGES);
+            for (int i = 0; i < pre; i++) {
+                const int u = u0 + i, tile = u / sk.KB, kb = u - tile * sk.KB;
+                mbar_expect_tx(&full[i], STAGE_BYTES);
+                tma_load_2d(sW + i * STAGE_W, &tmW, &full[i], kb * BK, tile * BM);
+            }
+            pdl_wait();
+            for (int i = 0; i < pre; i++) {
+                const int u = u0 + i, kb = u % sk.KB;
+                tma_load_2d(sX + i * STAGE_X, &tmX, &full[i], kb * BK, 0);
+            }
+            int issued = pre;
             bool ok = true;
-            for (int u = u0; u < u1 && ok; u++, issued++) {
+            for (int u = u0 + pre; u < u1 && ok; u++, issued++) {
                 const int s = issued % STAGES, round = issued / STAGES;
                 ok = mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag);
                 if (!ok) break;
@@ -214,6 +228,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
     } else {
         // ---------------------------------------------------------------- epilogue (warps 0-3)
+        pdl_wait();   // the partial-sum buffer may still be read by the kernel before this one
         int seg = 0;
         bool ok = true;
         for (int u = u0; u < u1 && ok; seg++) {
@@ -306,7 +321,7 @@ int tc_init() {
 
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
                     int M, int *err) {
-    tc::gemm_tc_kernel<<<sk.G, tc::THREADS, tc::SMEM_BYTES, s>>>(mW, mX, part, sk, M, err);
+    launch_k(tc::gemm_tc_kernel, dim3(sk.G), dim3(tc::THREADS), (size_t)tc::SMEM_BYTES, s, pdl_enabled(), mW, mX, part, sk, M, err);
 }
 
 // fp32 rows -> two bf16 terms: rows 0..15 hold hi = bf16(x), rows 16..31 hold lo = bf16(x - hi)
@@ -314,7 +329,7 @@ __global__ void split_rows_kernel(const float *x, __nv_bfloat16 *xs, int K) {
     const int m = blockIdx.y;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= K) return;
-    const float v = x[(size_t)m * K + i];
+    const float v = x[(size_t)m * K + i];   // launched without early start: x is complete
     const __nv_bfloat16 hi = __float2bfloat16_rn(v);
     xs[(size_t)m * K + i] = hi;
     xs[(size_t)(kMaxRows + m) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));

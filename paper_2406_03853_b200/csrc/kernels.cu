@@ -3,6 +3,8 @@
 // append, paged decode attention with a causal block of new rows, SwiGLU.
 //
 // Every reduction has a fixed combination order, so a pass is bit-reproducible.
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "kernels.cuh"
 
@@ -25,6 +27,13 @@ __device__ __forceinline__ float part_gather(const PartView &pv, int m, int r) {
     return v;
 }
 
+__device__ __forceinline__ float row_rstd(const RowScale &rs, int m) {
+    if (!rs.ssq) return 1.0f;
+    float t = 0.f;
+    for (int b = 0; b < rs.nblk; b++) t += rs.ssq[m * kSsqBlocks + b];
+    return 1.0f / sqrtf(t * rs.inv_d + rs.eps);
+}
+
 // the same for four consecutive outputs r..r+3 (r % 4 == 0, so they share a weight tile)
 __device__ __forceinline__ float4 part_gather4(const PartView &pv, int m, int r) {
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -44,6 +53,12 @@ __device__ __forceinline__ float4 part_gather4(const PartView &pv, int m, int r)
         }
     }
     return v;
+}
+
+bool pdl_enabled() {
+    static int on = -1;
+    if (on < 0) on = getenv("EESD_NO_PDL") ? 0 : 1;
+    return on == 1;
 }
 
 // ------------------------------------------------------------------------------------ small utilities
@@ -73,6 +88,8 @@ void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float 
 template <typename WT>
 __global__ void embed_kernel(const int32_t *tok, const WT *E, float *x, float *cap, int d, int V, int *err) {
     const int m = blockIdx.x;
+    pdl_trigger();
+    pdl_wait();
     int t = tok[m];
     if (t < 0 || t >= V) {
         if (threadIdx.x == 0) atomicOr(err, kErrBadToken);
@@ -87,50 +104,47 @@ __global__ void embed_kernel(const int32_t *tok, const WT *E, float *x, float *c
 }
 void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
                   int M, int d, int V, int *err) {
-    if (dtype == 0) embed_kernel<float><<<M, 256, 0, s>>>(tok, (const float *)E, x, cap, d, V, err);
-    else embed_kernel<bf16><<<M, 256, 0, s>>>(tok, (const bf16 *)E, x, cap, d, V, err);
+    if (dtype == 0) launch_k(embed_kernel<float>, dim3(M), dim3(256), 0, s, pdl_enabled(), tok, (const float *)E, x, cap, d, V, err);
+    else launch_k(embed_kernel<bf16>, dim3(M), dim3(256), 0, s, pdl_enabled(), tok, (const bf16 *)E, x, cap, d, V, err);
 }
 
 // ------------------------------------------------------------------------------------ residual + RMSNorm
-// One block of 1024 threads per token row, four elements per thread and step.
-// x[m] += partial sums; xn[m] = RMSNorm(x[m]) * g (fp32 and, optionally, as two bf16 terms).
-__global__ void __launch_bounds__(1024) resid_norm_kernel(float *x, PartView pv, int has_part, const float *g, float *xn,
-                                                          bf16 *xs, float *cap, int d, float eps) {
-    extern __shared__ float row[];  // d floats + 33 scratch
-    float *scratch = row + d;
-    const int m = blockIdx.x;
-    float *xr = x + (size_t)m * d;
+// grid (ceil(d / 1024), M), 256 threads, four elements per thread.
+// x[m] += partial sums; y = x[m] * g (fp32 and / or two bf16 terms); ssq[m][block] = sum x^2.
+// The RMSNorm scale itself is applied by whoever consumes the projection of y (RowScale).
+__global__ void __launch_bounds__(256) resid_kernel(float *x, PartView pv, int has_part, const float *g, float *xn, bf16 *xs,
+                                                    float *cap, float *ssq, int d) {
+    __shared__ float scratch[33];
+    const int m = blockIdx.y, i = blockIdx.x * 1024 + threadIdx.x * 4;
+    pdl_trigger();
+    pdl_wait();
     float ss = 0.f;
-    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    if (i < d) {
+        float *xr = x + (size_t)m * d;
         float4 v = *reinterpret_cast<const float4 *>(xr + i);
         if (has_part) {
             const float4 p = part_gather4(pv, m, i);
             v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
             *reinterpret_cast<float4 *>(xr + i) = v;
         }
-        *reinterpret_cast<float4 *>(row + i) = v;
         if (cap) *reinterpret_cast<float4 *>(cap + (size_t)m * d + i) = v;
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-    }
-    if (!g) return;
-    ss = block_sum(ss, scratch);
-    const float rstd = 1.0f / sqrtf(ss / (float)d + eps);
-    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
-        const float4 r4 = *reinterpret_cast<const float4 *>(row + i);
+        ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         const float4 g4 = *reinterpret_cast<const float4 *>(g + i);
-        const float4 v = make_float4(r4.x * rstd * g4.x, r4.y * rstd * g4.y, r4.z * rstd * g4.z, r4.w * rstd * g4.w);
-        *reinterpret_cast<float4 *>(xn + (size_t)m * d + i) = v;
+        const float4 y = make_float4(v.x * g4.x, v.y * g4.y, v.z * g4.z, v.w * g4.w);
+        if (xn) *reinterpret_cast<float4 *>(xn + (size_t)m * d + i) = y;
         if (xs) {
-            store_split(xs, m, d, i, v.x); store_split(xs, m, d, i + 1, v.y);
-            store_split(xs, m, d, i + 2, v.z); store_split(xs, m, d, i + 3, v.w);
+            store_split(xs, m, d, i, y.x); store_split(xs, m, d, i + 1, y.y);
+            store_split(xs, m, d, i + 2, y.z); store_split(xs, m, d, i + 3, y.w);
         }
     }
+    ss = block_sum(ss, scratch);
+    if (threadIdx.x == 0) ssq[m * kSsqBlocks + blockIdx.x] = ss;
 }
-void launch_resid_norm(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
-                       int M, int d, float eps) {
-    size_t smem = (size_t)(d + 33) * sizeof(float);
+void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
+                  float *ssq, int M, int d) {
     PartView none = {};
-    resid_norm_kernel<<<M, 1024, smem, s>>>(x, pv ? *pv : none, pv != nullptr, g, xn, (bf16 *)xs, cap, d, eps);
+    launch_k(resid_kernel, dim3((d + 1023) / 1024, M), dim3(256), 0, s, pdl_enabled(), x, pv ? *pv : none,
+             (int)(pv != nullptr), g, xn, (bf16 *)xs, cap, ssq, d);
 }
 
 // ------------------------------------------------------------------------------------ skinny projection (SIMT)
@@ -145,6 +159,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const AT *__restrict__ A
     __shared__ __align__(16) float sA[MT][KC];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r0 = blockIdx.x * 32 + warp * 4;
+    pdl_trigger();
+    pdl_wait();
     float acc[4][MT];
 #pragma unroll
     for (int rr = 0; rr < 4; rr++)
@@ -201,11 +217,12 @@ static void gemm_simt_dispatch(cudaStream_t s, const void *A, const void *W, flo
     dim3 grid((R + 31) / 32);
     const AT *a = (const AT *)A;
     const WT *w = (const WT *)W;
-    if (M <= 1) gemm_simt_kernel<WT, AT, 1><<<grid, 256, 0, s>>>(a, w, out, M, R, K);
-    else if (M <= 2) gemm_simt_kernel<WT, AT, 2><<<grid, 256, 0, s>>>(a, w, out, M, R, K);
-    else if (M <= 4) gemm_simt_kernel<WT, AT, 4><<<grid, 256, 0, s>>>(a, w, out, M, R, K);
-    else if (M <= 8) gemm_simt_kernel<WT, AT, 8><<<grid, 256, 0, s>>>(a, w, out, M, R, K);
-    else gemm_simt_kernel<WT, AT, 16><<<grid, 256, 0, s>>>(a, w, out, M, R, K);
+    const bool pdl = pdl_enabled();
+    if (M <= 1) launch_k(gemm_simt_kernel<WT, AT, 1>, grid, dim3(256), 0, s, pdl, a, w, out, M, R, K);
+    else if (M <= 2) launch_k(gemm_simt_kernel<WT, AT, 2>, grid, dim3(256), 0, s, pdl, a, w, out, M, R, K);
+    else if (M <= 4) launch_k(gemm_simt_kernel<WT, AT, 4>, grid, dim3(256), 0, s, pdl, a, w, out, M, R, K);
+    else if (M <= 8) launch_k(gemm_simt_kernel<WT, AT, 8>, grid, dim3(256), 0, s, pdl, a, w, out, M, R, K);
+    else launch_k(gemm_simt_kernel<WT, AT, 16>, grid, dim3(256), 0, s, pdl, a, w, out, M, R, K);
 }
 
 int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float *out, int M, int R, int K) {
@@ -217,12 +234,15 @@ int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float 
 // ------------------------------------------------------------------------------------ RoPE + KV append
 // grid (heads, M), block D/2: one thread per rotation pair.
 template <typename AT>
-__global__ void qkv_post_kernel(PartView pv, int pos0, int H, KvGeom kv, const float2 *rope, float *q, int head_off,
-                                int *err) {
+__global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeom kv, const float2 *rope, float *q,
+                                int head_off, int *err) {
     const int hh = blockIdx.x + head_off;  // 0..H-1 q, H..H+Hkv-1 k, then v
     const int m = blockIdx.y, i = threadIdx.x, D = kv.D;
     const int col = blockIdx.x * D + 2 * i;
-    float a = part_gather(pv, m, col), b = part_gather(pv, m, col + 1);
+    pdl_trigger();
+    pdl_wait();
+    const float rstd = row_rstd(rs, m);
+    float a = part_gather(pv, m, col) * rstd, b = part_gather(pv, m, col + 1) * rstd;
     const int pos = pos0 + m;
     if (hh < H + kv.Hkv) {
         float2 cs = rope[(size_t)pos * (D / 2) + i];
@@ -246,44 +266,52 @@ __global__ void qkv_post_kernel(PartView pv, int pos0, int H, KvGeom kv, const f
     dst[0] = from_f<AT>(a);
     dst[1] = from_f<AT>(b);
 }
-void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, int M, int pos0, int H,
+void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
                      const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err) {
     const int heads = only_kv ? 2 * kv.Hkv : H + 2 * kv.Hkv;
     dim3 grid(heads, M);
-    if (dtype == 0) qkv_post_kernel<float><<<grid, kv.D / 2, 0, s>>>(pv, pos0, H, kv, rope, q, only_kv ? H : 0, err);
-    else qkv_post_kernel<bf16><<<grid, kv.D / 2, 0, s>>>(pv, pos0, H, kv, rope, q, only_kv ? H : 0, err);
+    if (dtype == 0) launch_k(qkv_post_kernel<float>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, err);
+    else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, err);
 }
 
 // ------------------------------------------------------------------------------------ paged decode attention
-// grid (H_kv, n_split), 256 threads.  Block (kh, sp) owns up to kAttnPos cached positions of
-// KV head kh (a whole number of pages) and serves every query head of its group and all M new
-// rows from ONE copy of those keys and values: the page blocks ([page_tokens][D], contiguous)
-// are brought into shared memory by bulk asynchronous copies on one mbarrier, so the cache is
-// read from HBM once per KV head.  Row m sees positions <= pos0 + m.  The block writes, per
-// (query head, row), the un-normalised output, the maximum and the sum of its slice; the
-// combine kernel merges the slices in index order.
+// One kernel per layer: RoPE + KV append + attention over the paged cache + merge.
+// grid (H_kv, n_split), 256 threads.  Block (kh, sp) owns up to kAttnPos positions of KV head
+// kh (a whole number of pages) and serves every query head of its group and all M new rows
+// from ONE copy of those keys and values: the page blocks ([page_tokens][D], contiguous) are
+// brought into shared memory by bulk asynchronous copies on one mbarrier, so the cache is read
+// from HBM once per KV head.  The new rows' q, k, v come straight from the QKV projection's
+// partial sums (times the RMSNorm scale, rotated); the block whose slice holds a new position
+// places that key/value in its shared-memory tile and appends it to the cache in place.
+// Row m sees positions <= pos0 + m.  Each block writes, per (query head, row), the
+// un-normalised output, maximum and sum of its slice; the block that finishes last for a KV
+// head (an arrival counter, no waiting) merges the slices in index order.
 constexpr int kAttnPos = 128;     // positions per block
-constexpr int kAttnRows = 32;     // (head, row) pairs processed per batch
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-template <typename AT, int D>
-__global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, KvGeom kv, float *__restrict__ apart,
+template <typename AT, int D, int RB>   // RB: (head, row) pairs per batch, 2..32
+__global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, const float2 *__restrict__ rope, KvGeom kv,
+                                                   float *__restrict__ apart, unsigned int *tickets,
+                                                   float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
                                                    int M, int pos0, int H, int pps, int n_split, float scale, int *err) {
     constexpr int VEC = Vec16<AT>::N;       // elements per 16-byte chunk
     constexpr int NCH = D / VEC;            // chunks per row
+    constexpr int RS = RB / 2;              // rows per thread in the score phase
     extern __shared__ __align__(128) unsigned char attn_smem[];
     AT *sK = reinterpret_cast<AT *>(attn_smem);
     AT *sV = sK + kAttnPos * D;
-    float *sq = reinterpret_cast<float *>(sV + kAttnPos * D);   // [kAttnRows][D]
-    float *sS = sq + kAttnRows * D;                              // [kAttnRows][kAttnPos]
-    float *s_m = sS + kAttnRows * kAttnPos;                      // [kAttnRows]
-    float *s_l = s_m + kAttnRows;
-    uint64_t *bar = reinterpret_cast<uint64_t *>(s_l + kAttnRows);
+    float *sq = reinterpret_cast<float *>(sV + kAttnPos * D);   // [RB][D]
+    float *sS = sq + RB * D;                                     // [RB][kAttnPos]
+    float *s_m = sS + RB * kAttnPos;                             // [RB]
+    float *s_l = s_m + RB;
+    float *s_rstd = s_l + RB;                                    // [kMaxRows]
+    uint64_t *bar = reinterpret_cast<uint64_t *>(s_rstd + kMaxRows);
+    __shared__ int s_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
-    const int PT = kv.page_tokens, group = H / kv.Hkv;
+    const int PT = kv.page_tokens, group = H / kv.Hkv, HALF = D / 2;
     const int ctx_len = pos0 + M;
     const int n_pages = (ctx_len + PT - 1) / PT;
     const int page_lo = sp * pps, page_hi = min(n_pages, page_lo + pps);
@@ -291,6 +319,7 @@ __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, 
     const int npos = min(ctx_len, page_hi * PT) - lo;   // valid positions of this block
     const uint32_t blk_bytes = (uint32_t)(PT * D * sizeof(AT));
 
+    pdl_trigger();
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(bar)));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -298,6 +327,7 @@ __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, 
     }
     __syncthreads();
     if (tid == 0) {
+        // cached rows were written by earlier passes: no need to wait for this pass's producers
         const uint32_t total = 2u * blk_bytes * (uint32_t)(page_hi - page_lo);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(total) : "memory");
         for (int pg = page_lo; pg < page_hi; pg++) {
@@ -310,33 +340,62 @@ __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, 
                          ::"r"(smem_addr(sV + (size_t)(pg - page_lo) * PT * D)), "l"(src + v_off), "r"(blk_bytes), "r"(smem_addr(bar)) : "memory");
         }
     }
-    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
-    bool landed = false;
-    for (int r0 = 0; r0 < rows; r0 += kAttnRows) {
-        const int nb = min(kAttnRows, rows - r0);
-        for (int idx = tid; idx < nb * D; idx += 256) {
-            const int rl = idx / D, e = idx - rl * D;
-            const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
-            sq[rl * D + e] = q[(size_t)m * H * D + (size_t)(kh * group + g) * D + e] * scale;
+    pdl_wait();   // from here on the QKV projection's partial sums are read
+    if (tid < M) s_rstd[tid] = row_rstd(rs, tid);
+    {   // wait for the cached slice (bounded)
+        bool ok = false;
+        for (uint32_t i = 0; i < (1u << 24) && !ok; i++) {
+            uint32_t p;
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(p) : "r"(smem_addr(bar)) : "memory");
+            ok = p != 0;
+            if (!ok) __nanosleep(32);
         }
-        if (!landed) {
-            bool ok = false;
-            for (uint32_t i = 0; i < (1u << 24) && !ok; i++) {
-                uint32_t p;
-                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                             : "=r"(p) : "r"(smem_addr(bar)) : "memory");
-                ok = p != 0;
-                if (!ok) __nanosleep(32);
+        if (!ok && tid == 0) atomicOr(err, kErrWaitTimeout);
+    }
+    __syncthreads();
+    {   // new keys / values that fall into this slice: rotate, round, place in the tile, append
+        const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
+        const int n_new = p_last - p_first;
+        for (int idx = tid; idx < n_new * D; idx += 256) {   // idx -> (position, K pair | V pair)
+            const int pn = idx / D, w = idx - pn * D;
+            const int pos = p_first + pn, m = pos - pos0;
+            const int isV = w >= HALF, i = isV ? w - HALF : w;
+            const int col = (H + (isV ? kv.Hkv : 0) + kh) * D + 2 * i;
+            float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
+            if (!isV) {
+                const float2 cs = rope[(size_t)pos * HALF + i];
+                const float ra = a * cs.x - b * cs.y, rb = a * cs.y + b * cs.x;
+                a = ra; b = rb;
             }
-            if (!ok && tid == 0) atomicOr(err, kErrWaitTimeout);
-            landed = true;
+            const AT va = from_f<AT>(a), vb = from_f<AT>(b);
+            AT *tile = (isV ? sV : sK) + (size_t)(pos - lo) * D + 2 * i;
+            tile[0] = va; tile[1] = vb;
+            const int page = kv.page_table[pos / PT];
+            if (page < 0 || page >= kv.n_pages_total) { atomicOr(err, kErrBadPage); continue; }
+            AT *dst = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)PT * D +
+                      (size_t)(pos % PT) * D + 2 * i;
+            dst[0] = va; dst[1] = vb;
+        }
+    }
+    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
+    for (int r0 = 0; r0 < rows; r0 += RB) {
+        const int nb = min(RB, rows - r0);
+        for (int idx = tid; idx < nb * HALF; idx += 256) {   // rotated, pre-scaled queries of the batch
+            const int rl = idx / HALF, i = idx - rl * HALF;
+            const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
+            const int col = (kh * group + g) * D + 2 * i;
+            const float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
+            const float2 cs = rope[(size_t)(pos0 + m) * HALF + i];
+            sq[rl * D + 2 * i] = (a * cs.x - b * cs.y) * scale;
+            sq[rl * D + 2 * i + 1] = (a * cs.y + b * cs.x) * scale;
         }
         __syncthreads();
         {   // scores: thread -> position j, every second row of the batch
             const int j = tid & (kAttnPos - 1), rsel = tid >> 7;
-            float acc[kAttnRows / 2];
+            float acc[RS];
 #pragma unroll
-            for (int i = 0; i < kAttnRows / 2; i++) acc[i] = 0.f;
+            for (int i = 0; i < RS; i++) acc[i] = 0.f;
             if (j < npos) {
 #pragma unroll 2
                 for (int c = 0; c < NCH; c++) {
@@ -348,23 +407,21 @@ __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, 
                         kvv[0] = t.x; kvv[1] = t.y; kvv[2] = t.z; kvv[3] = t.w;
                     }
 #pragma unroll
-                    for (int i = 0; i < kAttnRows / 2; i++) {
-                        const int rl = rsel + 2 * i;
-                        if (rl < nb) {
-                            float qv[VEC];
+                    for (int i = 0; i < RS; i++) {
+                        const int rl = min(rsel + 2 * i, RB - 1);   // rows past nb are computed and dropped
+                        float qv[VEC];
 #pragma unroll
-                            for (int v = 0; v < VEC; v += 4) {
-                                const float4 t = *reinterpret_cast<const float4 *>(sq + rl * D + cc * VEC + v);
-                                qv[v] = t.x; qv[v + 1] = t.y; qv[v + 2] = t.z; qv[v + 3] = t.w;
-                            }
-#pragma unroll
-                            for (int v = 0; v < VEC; v++) acc[i] = fmaf(kvv[v], qv[v], acc[i]);
+                        for (int v = 0; v < VEC; v += 4) {
+                            const float4 t = *reinterpret_cast<const float4 *>(sq + rl * D + cc * VEC + v);
+                            qv[v] = t.x; qv[v + 1] = t.y; qv[v + 2] = t.z; qv[v + 3] = t.w;
                         }
+#pragma unroll
+                        for (int v = 0; v < VEC; v++) acc[i] = fmaf(kvv[v], qv[v], acc[i]);
                     }
                 }
             }
 #pragma unroll
-            for (int i = 0; i < kAttnRows / 2; i++) {
+            for (int i = 0; i < RS; i++) {
                 const int rl = rsel + 2 * i;
                 if (rl < nb) {
                     const int m = (r0 + rl) % M;
@@ -389,7 +446,8 @@ __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, 
         }
         __syncthreads();
         {   // o = P V: thread -> (pair of d, row group)
-            constexpr int HALF = D / 2, NG = 256 / HALF, RPT = kAttnRows / NG;
+            constexpr int NG = 256 / (D / 2);
+            constexpr int RPT = (RB + NG - 1) / NG;
             const int d2 = tid % HALF, rg = tid / HALF;
             float o0[RPT], o1[RPT];
 #pragma unroll
@@ -405,12 +463,10 @@ __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, 
                 }
 #pragma unroll
                 for (int i = 0; i < RPT; i++) {
-                    const int rl = rg + NG * i;
-                    if (rl < nb) {
-                        const float p = sS[rl * kAttnPos + j];
-                        o0[i] = fmaf(p, v0, o0[i]);
-                        o1[i] = fmaf(p, v1, o1[i]);
-                    }
+                    const int rl = min(rg + NG * i, RB - 1);
+                    const float p = sS[rl * kAttnPos + j];
+                    o0[i] = fmaf(p, v0, o0[i]);
+                    o1[i] = fmaf(p, v1, o1[i]);
                 }
             }
 #pragma unroll
@@ -427,39 +483,65 @@ __global__ void __launch_bounds__(256) attn_kernel(const float *__restrict__ q, 
         }
         __syncthreads();
     }
+    // ---- merge: the block that arrives last for this KV head combines all slices
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int prev = atomicAdd(&tickets[kh], 1u);
+        s_last = (prev == (unsigned int)n_split - 1);
+        if (s_last) tickets[kh] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const size_t sstride = (size_t)kMaxRows * (D + 2);
+    for (int idx = tid; idx < rows * D; idx += 256) {
+        const int rho = idx / D, dd = idx - rho * D;
+        const int g = rho / M, m = rho - g * M, h = kh * group + g;
+        const float *src = apart + (size_t)h * n_split * sstride + (size_t)m * (D + 2);
+        float mx = -INFINITY;
+        for (int s2 = 0; s2 < n_split; s2++) mx = fmaxf(mx, __ldcg(src + s2 * sstride + D));
+        float num = 0.f, den = 0.f;
+        for (int s2 = 0; s2 < n_split; s2++) {
+            const float ms = __ldcg(src + s2 * sstride + D);
+            if (ms == -INFINITY) continue;
+            const float w = expf(ms - mx);
+            num = fmaf(w, __ldcg(src + s2 * sstride + dd), num);
+            den = fmaf(w, __ldcg(src + s2 * sstride + D + 1), den);
+        }
+        const float o = den > 0.f ? num / den : 0.f;
+        if (attn_out) attn_out[(size_t)m * H * D + (size_t)h * D + dd] = o;
+        if (attn_split) store_split(attn_split, m, (size_t)H * D, (size_t)h * D + dd, o);
+    }
 }
 
-// grid (H, M), block D: merge the splits of one (head, row)
-__global__ void attn_combine_kernel(const float *apart, float *out, bf16 *out_split, int H, int D, int n_split) {
-    const int h = blockIdx.x, m = blockIdx.y, dd = threadIdx.x;
-    const float *src = apart + (size_t)h * n_split * kMaxRows * (D + 2) + (size_t)m * (D + 2);
-    const size_t sstride = (size_t)kMaxRows * (D + 2);
-    float mx = -INFINITY;
-    for (int s = 0; s < n_split; s++) mx = fmaxf(mx, src[s * sstride + D]);
-    float num = 0.f, den = 0.f;
-    for (int s = 0; s < n_split; s++) {
-        const float ms = src[s * sstride + D];
-        if (ms == -INFINITY) continue;
-        const float w = expf(ms - mx);
-        num = fmaf(w, src[s * sstride + dd], num);
-        den = fmaf(w, src[s * sstride + D + 1], den);
+template <typename AT, int D, int RB>
+static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
+                        float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
+                        int pps, int n_split, float scale, int *err) {
+    const size_t smem = (size_t)2 * kAttnPos * D * sizeof(AT) + (size_t)RB * D * 4 + (size_t)RB * kAttnPos * 4 +
+                        2 * RB * 4 + kMaxRows * 4 + 16;
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(attn_kernel<AT, D, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        configured = true;
     }
-    const float o = den > 0.f ? num / den : 0.f;
-    out[(size_t)m * H * D + (size_t)h * D + dd] = o;
-    if (out_split) store_split(out_split, m, (size_t)H * D, (size_t)h * D + dd, o);
+    launch_k(attn_kernel<AT, D, RB>, dim3(kv.Hkv, n_split), dim3(256), smem, s, pdl_enabled(), pv, rs, rope, kv, apart,
+             tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err);
 }
 
 template <typename AT, int D>
-static void attn_launch(cudaStream_t s, const float *q, const KvGeom &kv, float *apart, int M, int pos0, int H, int pps,
-                        int n_split, float scale, int *err) {
-    const size_t smem = (size_t)2 * kAttnPos * D * sizeof(AT) + (size_t)kAttnRows * D * 4 +
-                        (size_t)kAttnRows * kAttnPos * 4 + 2 * kAttnRows * 4 + 16;
-    static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(attn_kernel<AT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        configured = true;
-    }
-    attn_kernel<AT, D><<<dim3(kv.Hkv, n_split), 256, smem, s>>>(q, kv, apart, M, pos0, H, pps, n_split, scale, err);
+static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
+                          float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
+                          int pps, int n_split, float scale, int *err) {
+    const int rows = (H / kv.Hkv) * M;
+#define EESD_ATTN(RB) attn_launch<AT, D, RB>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err)
+    if (rows <= 2) EESD_ATTN(2);
+    else if (rows <= 4) EESD_ATTN(4);
+    else if (rows <= 8) EESD_ATTN(8);
+    else if (rows <= 16) EESD_ATTN(16);
+    else EESD_ATTN(32);
+#undef EESD_ATTN
 }
 
 int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_sm, int max_splits, int *pps_out) {
@@ -474,42 +556,51 @@ int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_sm, int max_sp
     return n_split;
 }
 
-void launch_attention(cudaStream_t s, int dtype, const float *q, const KvGeom &kv, float *apart,
-                      float *attn_out, void *attn_split, int M, int pos0, int H, int n_sm, int max_splits, int *err) {
+void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
+                      const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
+                      int M, int pos0, int H, int n_sm, int max_splits, int *err) {
     int pps;
     const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, n_sm, max_splits, &pps);
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (dtype == 0) {
-        if (kv.D == 64) attn_launch<float, 64>(s, q, kv, apart, M, pos0, H, pps, n_split, scale, err);
-        else attn_launch<float, 128>(s, q, kv, apart, M, pos0, H, pps, n_split, scale, err);
+        if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);
+        else attn_dispatch<float, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);
     } else {
-        if (kv.D == 64) attn_launch<bf16, 64>(s, q, kv, apart, M, pos0, H, pps, n_split, scale, err);
-        else attn_launch<bf16, 128>(s, q, kv, apart, M, pos0, H, pps, n_split, scale, err);
+        if (kv.D == 64) attn_dispatch<bf16, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);
+        else attn_dispatch<bf16, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);
     }
-    attn_combine_kernel<<<dim3(H, M), kv.D, 0, s>>>(apart, attn_out, (bf16 *)attn_split, H, kv.D, n_split);
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU, partial sums
-__global__ void swiglu_kernel(PartView pv, float *h, bf16 *hs, int F) {
-    const int m = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
+__global__ void swiglu_kernel(PartView pv, RowScale rs, float *h, bf16 *hs, int F) {
+    const int m = blockIdx.y, i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    pdl_trigger();
+    pdl_wait();
     if (i >= F) return;
-    const float g = part_gather(pv, m, i), u = part_gather(pv, m, F + i);
-    const float v = g / (1.0f + expf(-g)) * u;
-    h[(size_t)m * F + i] = v;
-    if (hs) store_split(hs, m, F, i, v);
+    const float rstd = row_rstd(rs, m);
+    const float4 g = part_gather4(pv, m, i), u = part_gather4(pv, m, F + i);
+    const float gg[4] = {g.x * rstd, g.y * rstd, g.z * rstd, g.w * rstd};
+    const float uu[4] = {u.x * rstd, u.y * rstd, u.z * rstd, u.w * rstd};
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        const float v = gg[k] / (1.0f + expf(-gg[k])) * uu[k];
+        if (h) h[(size_t)m * F + i + k] = v;
+        if (hs) store_split(hs, m, F, i + k, v);
+    }
 }
-void launch_swiglu(cudaStream_t s, const PartView &pv, float *h, void *h_split, int M, int F) {
-    dim3 grid((F + 255) / 256, M);
-    swiglu_kernel<<<grid, 256, 0, s>>>(pv, h, (bf16 *)h_split, F);
+void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F) {
+    launch_k(swiglu_kernel, dim3((F / 4 + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, h, (bf16 *)h_split, F);
 }
 
-__global__ void reduce_partials_kernel(PartView pv, float *out, int R) {
+__global__ void reduce_partials_kernel(PartView pv, RowScale rs, float *out, int R) {
     const int m = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
     if (r >= R) return;
-    out[(size_t)m * R + r] = part_gather(pv, m, r);
+    out[(size_t)m * R + r] = part_gather(pv, m, r) * row_rstd(rs, m);
 }
-void launch_reduce_partials(cudaStream_t s, const PartView &pv, float *out, int M, int R) {
-    reduce_partials_kernel<<<dim3((R + 255) / 256, M), 256, 0, s>>>(pv, out, R);
+void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R) {
+    launch_k(reduce_partials_kernel, dim3((R + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, out, R);
 }
 
 }  // namespace eesd

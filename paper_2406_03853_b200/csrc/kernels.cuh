@@ -40,26 +40,45 @@ struct PartView {
     StreamK sk;
 };
 
+// RMSNorm statistics of the rows a projection consumed: the projection runs on x * g, and
+// whoever reads its result multiplies row m by rstd(m) = 1 / sqrt(sum_b ssq[m][b] / d + eps)
+// (the normalisation is a per-row scalar, so it commutes with the projection).
+constexpr int kSsqBlocks = 16;   // partial sums of squares per row (1024 elements each)
+struct RowScale {
+    const float *ssq;   // [16][kSsqBlocks]; null: no scaling
+    int nblk;
+    float inv_d, eps;
+};
+
 void launch_set_ints(cudaStream_t s, int32_t *dst, const IntList16 &vals, int n);
 void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float theta);
 void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
                   int M, int d, int V, int *err);
 // x[m] += sum_s part[s][m] (if part); xn[m] = cast(RMSNorm(x[m]) * g) (if g); cap[m] = x[m] (if cap)
-// `xs` (may be null): the same rows as two bf16 terms, [32][d]: rows 0..15 hi, 16..31 lo
-void launch_resid_norm(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
-                       int M, int d, float eps);
+// x[m] += partial sums (if pv); y = x[m] * g -> xn (fp32, may be null) and xs (two bf16 terms,
+// [32][d]: rows 0..15 hi, 16..31 lo, may be null); ssq[m][b] = sum of squares of block b of x[m];
+// cap[m] = x[m] (if cap)
+void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
+                  float *ssq, int M, int d);
 // out[sp][m][r] = sum_{k in split sp} A[m][k] * W[r][k]; returns the number of K splits written
 int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float *out, int M, int R, int K);
 // RoPE + KV append (+ q store).  part rows are [q heads | k heads | v heads] or, when
 // only_kv, [k heads | v heads].
-void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, int M, int pos0, int H,
+void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
                      const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err);
-// apart: room for H * max_splits * 16 * (D + 2) floats; page_tokens * D elements per page block
-// must not exceed 128 * D (page_tokens <= 128)
-void launch_attention(cudaStream_t s, int dtype, const float *q, const KvGeom &kv, float *apart,
-                      float *attn_out, void *attn_split, int M, int pos0, int H, int n_sm, int max_splits, int *err);
-void launch_swiglu(cudaStream_t s, const PartView &pv, float *h, void *h_split, int M, int F);
-void launch_reduce_partials(cudaStream_t s, const PartView &pv, float *out, int M, int R);
+// Fused attention step of one layer on M new rows: q/k/v of the new rows are taken from the
+// QKV projection's partial sums (scaled by rs, rotated), the new keys/values are appended to
+// the paged cache, every KV head's cached slice is read once, and the slices are merged into
+// attn_out (fp32 [M][H*D], may be null) and attn_split (two bf16 terms, may be null).
+// apart: H * max_splits * 16 * (D + 2) floats; tickets: H_kv zero-initialised counters.
+void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
+                      const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
+                      int M, int pos0, int H, int n_sm, int max_splits, int *err);
+void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F);
+void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R);
+// programmatic dependent launch (kernels start early and wait on-device for their producer):
+// on by default, off when the environment variable EESD_NO_PDL is set
+bool pdl_enabled();
 
 // tensor-core projection (gemm_tc.cu)
 int tc_init();                                   // once per process; 0 on success
