@@ -238,6 +238,29 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
                          int B, int K, int V, float temperature, void *scratch, size_t scratch_bytes,
                          int32_t *n_accept, int32_t *next_token);
 
+/* The same acceptance step for callers that cannot hand over device scratch memory.  The paper
+ * has no counterpart: this exists for deployment reasons only.  Some hosts of this library may
+ * not allocate on the device at the point where they verify a round: code running inside a
+ * frozen memory plan (a serving engine that sized every buffer at start-up and forbids
+ * allocation on the request path), plug-ins that are given only their input and output
+ * tensors, or processes whose allocator must not be re-entered from the calling thread.  For
+ * them the scratch lives inside the library as a fixed device array of about 80 KB, present in
+ * every GPU context that loads the library until the process exits.
+ * Limits: B <= EESD_STATIC_ACCEPT_MAX_BATCH and B * (2K + 1) <= EESD_STATIC_ACCEPT_MAX_ROWS;
+ * larger problems return EESD_ERR_NOMEM (use eesd_accept_resample with your own scratch).
+ * Inputs, outputs, arithmetic and results are exactly those of eesd_accept_resample.  The call
+ * performs no device allocation or free.  The first call on each device looks up the array's
+ * device address (one cudaGetSymbolAddress, with that device current); make that first call
+ * before any stream capture.  All calls share the one array and it keeps the previous call's
+ * contents (the call re-zeroes what has to start at zero): two calls whose kernels may overlap
+ * on the GPU (different streams, no ordering between them) race on it and must be avoided. */
+#define EESD_STATIC_ACCEPT_MAX_BATCH 1024
+#define EESD_STATIC_ACCEPT_MAX_ROWS 4800
+int eesd_accept_resample_static(void *cuda_stream, const float *p_logits, const float *q_logits,
+                                const int32_t *tokens, const float *u_accept, const float *u_resample,
+                                int B, int K, int V, float temperature,
+                                int32_t *n_accept, int32_t *next_token);
+
 /* The skinny projection used by every weight-streaming step of a pass (QKV, attention output,
  * SwiGLU gate/up and down, vocabulary heads): out[m][r] = sum_k A[m][k] * W[r][k] for
  * M <= EESD_MAX_ROWS rows.  A [M][K] fp32, W [R][K] in `dtype`, out [M][R] fp32, all device.

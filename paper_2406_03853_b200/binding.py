@@ -116,6 +116,7 @@ def lib():
         L.eesd_project_scratch_bytes.argtypes = [C.c_int, C.c_int]
         L.eesd_project_rows.argtypes = [vp, C.c_int, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, C.c_size_t]
         L.eesd_time_projection.argtypes = [vp, C.c_int, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_size_t)]
+        L.eesd_accept_resample_static.argtypes = [vp, vp, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_float, vp, vp]
         L.eesd_sample_rows.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_float, vp]
         _lib = L
     return _lib

@@ -16,6 +16,7 @@
 //   form, times 2^n.  Constants are given as fp32 bit patterns below.
 //   draw from weights w_v <= 1 with u = m_u 2^-24: W = sum_v trunc(w_v * 2^32) (64-bit),
 //   tau = (m_u * W) >> 24, result = smallest v whose inclusive integer prefix sum exceeds tau.
+#include "../../include/eesd.h"
 #include "common.cuh"
 #include "kernels.cuh"
 
@@ -314,3 +315,39 @@ void launch_sample_rows(cudaStream_t s, const float *logits, const float *u, int
 }
 
 }  // namespace eesd
+
+// ---- acceptance without any caller-provided or allocated scratch ------------------------------------
+// Library-owned scratch for eesd_accept_resample_static: lives in every GPU context that loads
+// this library, from load to exit.  Sized for EESD_STATIC_ACCEPT_MAX_ROWS logit rows
+// (B * (2K + 1)) and EESD_STATIC_ACCEPT_MAX_BATCH sequences.
+static __device__ __align__(256) unsigned char g_static_accept_scratch
+    [((EESD_STATIC_ACCEPT_MAX_BATCH * sizeof(unsigned int) + 15) / 16) * 16 + EESD_STATIC_ACCEPT_MAX_ROWS * sizeof(eesd::RowStat)];
+
+extern "C" int eesd_accept_resample_static(void *cuda_stream, const float *p_logits, const float *q_logits,
+                                           const int32_t *tokens, const float *u_accept, const float *u_resample,
+                                           int B, int K, int V, float temperature, int32_t *n_accept,
+                                           int32_t *next_token) {
+    if (!p_logits || !q_logits || !tokens || !n_accept || !next_token) return EESD_ERR_BADARG;
+    if (B < 1 || K < 1 || V < 1 || temperature < 0.f) return EESD_ERR_BADARG;
+    if (temperature != 0.f && (!u_accept || !u_resample)) return EESD_ERR_RNG;
+    if (B > EESD_STATIC_ACCEPT_MAX_BATCH || (long long)B * (2 * K + 1) > EESD_STATIC_ACCEPT_MAX_ROWS)
+        return EESD_ERR_NOMEM;   // beyond the built-in scratch: use eesd_accept_resample with caller scratch
+    // The array's name is only a host-side handle; the device address is looked up once per
+    // device (with that device current) and remembered.
+    constexpr int kMaxDevices = 64;
+    static void *dev_ptr[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return EESD_ERR_CUDA;
+    if (!dev_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_accept_scratch) != cudaSuccess || !p) return EESD_ERR_CUDA;
+        dev_ptr[dev] = p;
+    }
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // the arrival counters must start at zero; the row statistics are overwritten before use
+    if (cudaMemsetAsync(dev_ptr[dev], 0, (size_t)B * sizeof(unsigned int), s) != cudaSuccess) return EESD_ERR_CUDA;
+    eesd::launch_accept(s, p_logits, q_logits, tokens, u_accept, u_resample, B, K, V, temperature, dev_ptr[dev],
+                        n_accept, next_token, nullptr);
+    return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
+}
+
