@@ -164,9 +164,11 @@ def time_verify_pass(eng, spec, ctx_len, M, reps=5):
     return statistics.median(ts)
 
 
-def oracle_sample(spec, mean_k, mean_emit, threads_note=True):
-    """CPU oracle on a bounded slice: one decoder layer of this shape on (mean_k + 1) rows
-    against a 512-token cache, and the vocabulary head on one row; scaled to a whole round."""
+def oracle_sample(spec, mean_k, mean_emit, budget_s=12.0):
+    """CPU oracle on a bounded slice: one decoder layer of this shape on (mean_k + 1) rows and
+    on 1 row against a 512-token cache, repeated until about `budget_s` seconds of CPU work
+    have been timed; the medians are scaled to a whole round (all layers, heads by parameter
+    count).  Returns (tokens/s, seconds timed, rows, repetitions)."""
     import oracle
     L1 = spec.with_(n_layers=1, n_early=1, vocab=64)
     lw = {k: v for k, v in synth.layer_weights(spec, 0).items()}
@@ -174,18 +176,25 @@ def oracle_sample(spec, mean_k, mean_emit, threads_note=True):
     m = oracle.model_from_weights(L1, [lw], lw, emb, emb, max_ctx=640)
     rows = max(2, int(round(mean_k)) + 1)
     x = np.asarray(synth.normal_f32(1, 1, rows * spec.d_model).view(rows, spec.d_model), np.float64)
-    t0 = time.time()
-    m.layer_fwd(0, 0, x, 512)
-    t_layer_rows = time.time() - t0
-    t0 = time.time()
-    m.layer_fwd(0, 0, x[:1], 512)
-    t_layer_1 = time.time() - t0
+    m.layer_fwd(0, 0, x[:1], 512)   # touch the weights once, untimed
+    t_rows, t_one, spent, reps = [], [], 0.0, 0
+    while spent < budget_s and reps < 200:
+        t0 = time.time()
+        m.layer_fwd(0, 0, x, 512)
+        t1 = time.time()
+        m.layer_fwd(0, 0, x[:1], 512)
+        t2 = time.time()
+        t_rows.append(t1 - t0)
+        t_one.append(t2 - t1)
+        spent += t2 - t0
+        reps += 1
+    t_layer_rows, t_layer_1 = statistics.median(t_rows), statistics.median(t_one)
     head_rows = spec.vocab * spec.d_model / spec.layer_params  # head cost in units of one layer-row
     per_row = t_layer_rows / rows
     t_verify = spec.n_layers * t_layer_rows + rows * head_rows * per_row
     t_draft = (rows - 1) * ((spec.n_early + 1) * t_layer_1 + head_rows * t_layer_1)
     tok_s = mean_emit / (t_verify + t_draft)
-    return tok_s, t_layer_rows + t_layer_1, rows
+    return tok_s, spent, rows, reps
 
 
 def profile_pass(args, device):
@@ -218,7 +227,7 @@ def run_reference(args):
     vals, ms = [], []
     for i in range(args.warmup + args.steps):
         t0 = time.time()
-        tok_s, _, rows = oracle_sample(spec, 5.0, 3.0)
+        tok_s, _, rows, _ = oracle_sample(spec, 5.0, 3.0)
         if i >= args.warmup:
             vals.append(tok_s)
             ms.append((time.time() - t0) * 1e3)
@@ -370,11 +379,11 @@ def main():
     if not args.no_cpu_baseline and world == 1:
         import oracle
         oracle.build()
-        tok_s, secs, rows = oracle_sample(spec, mean_k, mean_emit)
+        tok_s, secs, rows, reps = oracle_sample(spec, mean_k, mean_emit)
         line["cpu_baseline"] = {
             "value": round(tok_s, 5), "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle",
             "sample": f"one {spec.name}-shaped decoder layer on {rows} rows and on 1 row against a 512-token cache "
-                      f"({secs:.1f} s of CPU work), scaled to a round of mean K={mean_k:.2f} emitting {mean_emit:.2f} "
+                      f"({reps} repetitions, {secs:.1f} s of CPU work, medians), scaled to a round of mean K={mean_k:.2f} emitting {mean_emit:.2f} "
                       f"tokens; extrapolated"}
     print(json.dumps(line))
     eng.close()

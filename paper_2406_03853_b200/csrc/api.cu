@@ -22,6 +22,8 @@ struct LayerW {
 
 // which activation matrix feeds a projection
 enum { X_NORM = 0, X_ATTN = 1, X_FFN = 2 };
+// the distinct projection shapes of a pass (each has its own stream-K plan and block table)
+enum { P_QKV = 0, P_O = 1, P_GU = 2, P_D = 3, P_EXIT_KV = 4, P_HEAD = 5, P_COUNT = 6 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -47,7 +49,7 @@ int check_config(const eesd_config *c) {
 }
 
 struct Workspace {
-    size_t x, xn, q, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
+    size_t x, xn, q, attn, h, xs[3], ssq, tickets, tabs, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
         accept, total;
 };
 
@@ -78,9 +80,10 @@ Workspace carve(const eesd_config *c) {
     w.xs[X_FFN] = take(2 * R * (size_t)c->ffn_dim * 2);
     w.ssq = take((size_t)EESD_MAX_ROWS * kSsqBlocks * 4);
     w.tickets = take(1024 * 4);
+    w.tabs = take((size_t)P_COUNT * (maxR / 128 + 1) * sizeof(int4));
     {   // partial sums: SIMT layout [splits][16][maxR], or stream-K blocks of the widest projection
         size_t part_floats = (size_t)kPartSplits * R * maxR;
-        const size_t sk_floats = (maxR / 128 + 3 * (size_t)kMaxSm) * R * 128;  // >= G * max_seg blocks
+        const size_t sk_floats = (maxR / 128 + (size_t)kMaxSm) * R * 128;  // blocks <= tiles + CTAs
         if (sk_floats > part_floats) part_floats = sk_floats;
         w.part = take(part_floats * 4);
     }
@@ -121,6 +124,7 @@ struct eesd_ctx {
     CUtensorMap m_exit_kv, m_lm_head, m_exit_head;
     bool use_tc;
     int n_sm;
+    StreamK plan[P_COUNT];       // tensor-core path: work split and block table per shape
     float2 *rope;
     int32_t *page_table, *ints;
     int *err;
@@ -205,14 +209,14 @@ void trim_pages(eesd_ctx *c, int n_tokens) {
 
 // One projection: out = X[which] . W^T.  Tensor-core stream-K kernel when the context uses it
 // (bf16, tile-aligned shapes), else the SIMT kernel.  Returns where the partial sums are.
-PartView run_proj(eesd_ctx *c, const void *W, const CUtensorMap *mW, int which, int M, int R, int K) {
+PartView run_proj(eesd_ctx *c, const void *W, const CUtensorMap *mW, int shape, int which, int M, int R, int K) {
     PartView pv = {};
     pv.base = c->part;
     pv.R = R;
     if (c->use_tc) {
         pv.mode = 1;
-        pv.sk = tc_plan(R, K, c->n_sm);
-        launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, pv.sk, M, c->err);
+        pv.tab = c->plan[shape].tab;
+        launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, c->plan[shape], M, c->err);
     } else {
         const float *A = which == X_NORM ? c->xn : which == X_ATTN ? c->attn : c->h;
         pv.mode = 0;
@@ -246,14 +250,14 @@ void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const fl
     cudaStream_t s = c->stream;
     const RowScale rs = norm_scale(c), none = {nullptr, 0, 0.f, 0.f};
     (void)none;
-    PartView pv = run_proj(c, w.wqkv, &w.m_qkv, X_NORM, M, qd + 2 * kvd, d);
+    PartView pv = run_proj(c, w.wqkv, &w.m_qkv, P_QKV, X_NORM, M, qd + 2 * kvd, d);
     launch_attention(s, f.dtype, pv, rs, c->rope, kv_geom(c, slot), c->apart, c->tickets, c->use_tc ? nullptr : c->attn,
                      c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, c->err);
-    pv = run_proj(c, w.wo, &w.m_o, X_ATTN, M, d, qd);
+    pv = run_proj(c, w.wo, &w.m_o, P_O, X_ATTN, M, d, qd);
     run_resid(c, &pv, w.g_ffn, nullptr, M);
-    pv = run_proj(c, w.wgu, &w.m_gu, X_NORM, M, 2 * F, d);
+    pv = run_proj(c, w.wgu, &w.m_gu, P_GU, X_NORM, M, 2 * F, d);
     launch_swiglu(s, pv, rs, c->use_tc ? nullptr : c->h, c->xs[X_FFN], M, F);
-    pv = run_proj(c, w.wd, &w.m_d, X_FFN, M, d, F);
+    pv = run_proj(c, w.wd, &w.m_d, P_D, X_FFN, M, d, F);
     run_resid(c, &pv, g_next, cap, M);
     c->launches += 2;
 }
@@ -279,7 +283,7 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
             // keys / values of the early-exit layer for these rows: they depend on H^N only
             const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim;
             const char *wkv = c->layers[L].wqkv + (size_t)qd * d * c->es;
-            PartView pv = run_proj(c, wkv, &c->m_exit_kv, X_NORM, M, 2 * kvd, d);
+            PartView pv = run_proj(c, wkv, &c->m_exit_kv, P_EXIT_KV, X_NORM, M, 2 * kvd, d);
             launch_qkv_post(s, f.dtype, pv, norm_scale(c), M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err);
             const float *g_next = l + 1 < L ? c->layers[l + 1].g_attn : c->g_final;
             run_resid(c, nullptr, g_next, nullptr, M);
@@ -287,7 +291,7 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
         }
     }
     if (want_logits) {
-        PartView pv = run_proj(c, c->lm_head, &c->m_lm_head, X_NORM, M, f.vocab, d);
+        PartView pv = run_proj(c, c->lm_head, &c->m_lm_head, P_HEAD, X_NORM, M, f.vocab, d);
         launch_reduce_partials(s, pv, norm_scale(c), c->logits_p, M, f.vocab);
         c->launches += 1;
     }
@@ -308,7 +312,7 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
     }
     run_layer(c, c->layers[L], L, 1, pos, c->g_exit, cap_slot(c, L + 1));
     float *lq = c->logits_q + (size_t)i * f.vocab;
-    PartView pv = run_proj(c, c->exit_head, &c->m_exit_head, X_NORM, 1, f.vocab, d);
+    PartView pv = run_proj(c, c->exit_head, &c->m_exit_head, P_HEAD, X_NORM, 1, f.vocab, d);
     launch_reduce_partials(s, pv, norm_scale(c), lq, 1, f.vocab);
     launch_sample_rows(s, lq, d_u, 1, f.vocab, f.temperature, c->ints + kRoundTok + i + 1);
     c->launches += 3;
@@ -567,6 +571,19 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         ok = ok && tc_make_map(&c->m_exit_kv, c->layers[cfg->n_layers].wqkv + (size_t)qd_ * d * 2, 2 * kvd_, d, 128);
         ok = ok && tc_make_map(&c->m_lm_head, c->lm_head, cfg->vocab, d, 128);
         ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128);
+        // work split and block table of every projection shape
+        const int shapes[P_COUNT][2] = {{qd_ + 2 * kvd_, d}, {d, qd_}, {2 * F, d}, {d, F}, {2 * kvd_, d}, {cfg->vocab, d}};
+        size_t maxR = 0;
+        for (auto &sh : shapes) if ((size_t)sh[0] > maxR) maxR = sh[0];
+        std::vector<int4> host_tab;
+        for (int i = 0; i < P_COUNT && ok; i++) {
+            c->plan[i] = tc_plan(shapes[i][0], shapes[i][1], c->n_sm);
+            host_tab.assign(c->plan[i].tiles, make_int4(0, 0, 0, 0));
+            tc_fill_table(c->plan[i], host_tab.data());
+            int4 *dev = (int4 *)(ws + w.tabs) + (size_t)i * (maxR / 128 + 1);
+            ok = cudaMemcpy(dev, host_tab.data(), host_tab.size() * sizeof(int4), cudaMemcpyHostToDevice) == cudaSuccess;
+            c->plan[i].tab = dev;
+        }
         if (!ok) {
             delete c;
             return EESD_ERR_CUDA;
@@ -851,21 +868,23 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
     return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
 }
 
-static size_t project_scratch_layout(int R, int K, size_t *off_xs, size_t *off_part) {
+static size_t project_scratch_layout(int R, int K, size_t *off_xs, size_t *off_tab, size_t *off_part) {
     size_t o = 256;  // error word
     *off_xs = o;
     o = align_up(o + (size_t)2 * EESD_MAX_ROWS * K * 2, 256);
+    *off_tab = o;
+    o = align_up(o + ((size_t)R / 128 + 1) * sizeof(int4), 256);
     *off_part = o;
     size_t floats = (size_t)EESD_MAX_ROWS * R;
-    const size_t sk = ((size_t)R / 128 + 3 * (size_t)kMaxSm) * EESD_MAX_ROWS * 128;
+    const size_t sk = ((size_t)R / 128 + (size_t)kMaxSm) * EESD_MAX_ROWS * 128;
     if (sk > floats) floats = sk;
     return o + floats * 4;
 }
 
 size_t eesd_project_scratch_bytes(int R, int K) {
     if (R < 1 || K < 1) return 0;
-    size_t a, b;
-    return project_scratch_layout(R, K, &a, &b);
+    size_t a, b, t;
+    return project_scratch_layout(R, K, &a, &t, &b);
 }
 
 int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *W, float *out, int M, int R, int K,
@@ -873,8 +892,8 @@ int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *
     if (!A || !W || !out || !scratch) return EESD_ERR_BADARG;
     if (M < 1 || M > EESD_MAX_ROWS || R < 1 || K < 8 || (K % 8)) return EESD_ERR_BADARG;
     if (dtype != EESD_F32 && dtype != EESD_BF16) return EESD_ERR_BADARG;
-    size_t off_xs, off_part;
-    if (scratch_bytes < project_scratch_layout(R, K, &off_xs, &off_part)) return EESD_ERR_NOMEM;
+    size_t off_xs, off_tab, off_part;
+    if (scratch_bytes < project_scratch_layout(R, K, &off_xs, &off_tab, &off_part)) return EESD_ERR_NOMEM;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     char *sc = (char *)scratch;
     float *part = (float *)(sc + off_part);
@@ -889,11 +908,18 @@ int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *
         CUtensorMap mW, mX;
         if (!tc_make_map(&mW, W, R, K, 128) || !tc_make_map(&mX, sc + off_xs, 2 * EESD_MAX_ROWS, K, 2 * EESD_MAX_ROWS))
             return EESD_ERR_CUDA;
+        StreamK sk = tc_plan(R, K, n_sm);
+        std::vector<int4> tab(sk.tiles);
+        tc_fill_table(sk, tab.data());
+        sk.tab = (const int4 *)(sc + off_tab);
         if (cudaMemsetAsync(sc, 0, 16, s) != cudaSuccess) return EESD_ERR_CUDA;
+        // pageable source: the copy is staged before the call returns, so `tab` may go out of scope
+        if (cudaMemcpyAsync(sc + off_tab, tab.data(), tab.size() * sizeof(int4), cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return EESD_ERR_CUDA;
         launch_split_rows(s, A, sc + off_xs, M, K);
         pv.mode = 1;
-        pv.sk = tc_plan(R, K, n_sm);
-        launch_gemm_tc(s, mW, mX, part, pv.sk, M, (int *)sc);
+        pv.tab = sk.tab;
+        launch_gemm_tc(s, mW, mX, part, sk, M, (int *)sc);
     } else {
         pv.mode = 0;
         pv.S = launch_gemm(s, dtype, A, W, part, M, R, K);
@@ -918,7 +944,7 @@ int eesd_time_projection(eesd_ctx *c, int which, int M, float *ms_per_launch, si
             const LayerW &w = c->layers[l];
             const void *W = which == 0 ? w.wqkv : which == 1 ? w.wo : which == 2 ? w.wgu : w.wd;
             const CUtensorMap *m = which == 0 ? &w.m_qkv : which == 1 ? &w.m_o : which == 2 ? &w.m_gu : &w.m_d;
-            run_proj(c, W, m, X, M, R, K);
+            run_proj(c, W, m, which, X, M, R, K);
         }
         if (pass == 1) CU(c, cudaEventRecord(c->ev[1], c->stream));
     }

@@ -16,8 +16,9 @@
 //     the B operand): products are exact, accumulation is fp32, and the result equals an fp32
 //     activation times a bf16 weight to about 2^-17 relative.  The extra columns cost tensor
 //     time only, which this kernel has to spare.
-// Each segment (part of one tile's k range done by one CTA) is written as an fp32 partial;
-// consumers add the partials of a tile in CTA order, so results are bit-reproducible and do
+// Each segment (part of one tile's k range done by one CTA) is written as an fp32 partial
+// block; consumers add the blocks of a tile in CTA order (a small per-tile table says where
+// they are), so results are bit-reproducible and do
 // not depend on M.
 //
 // Every wait is bounded: on expiry the thread raises the error word, the CTA drains its
@@ -72,6 +73,21 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     }
     *abort_flag = 1;
     return false;
+}
+
+// same, with an L2 eviction-priority hint (the weight stream is read once per pass and should
+// not push activations, partial sums and the KV cache out of L2)
+__device__ __forceinline__ void tma_load_2d_hint(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
@@ -164,11 +180,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (lane == 0) {
             // The weights do not depend on the kernel before this one: fill the ring with weight
             // tiles at once, and only then wait for the producer of the token rows.
+            const uint64_t stream_once = policy_evict_first();
             const int pre = min(u1 - u0, STAGES);
             for (int i = 0; i < pre; i++) {
                 const int u = u0 + i, tile = u / sk.KB, kb = u - tile * sk.KB;
                 mbar_expect_tx(&full[i], STAGE_BYTES);
-                tma_load_2d(sW + i * STAGE_W, &tmW, &full[i], kb * BK, tile * BM);
+                tma_load_2d_hint(sW + i * STAGE_W, &tmW, &full[i], kb * BK, tile * BM, stream_once);
             }
             pdl_wait();
             for (int i = 0; i < pre; i++) {
@@ -183,7 +200,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 if (!ok) break;
                 const int tile = u / sk.KB, kb = u - tile * sk.KB;
                 mbar_expect_tx(&full[s], STAGE_BYTES);
-                tma_load_2d(sW + s * STAGE_W, &tmW, &full[s], kb * BK, tile * BM);
+                tma_load_2d_hint(sW + s * STAGE_W, &tmW, &full[s], kb * BK, tile * BM, stream_once);
                 tma_load_2d(sX + s * STAGE_X, &tmX, &full[s], kb * BK, 0);
             }
             if (*abort_flag) {
@@ -244,7 +261,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[b]);
-            float *dst = part + ((size_t)(cta * sk.max_seg + (tile - sk.first_tile(cta))) * kMaxRows) * BM + warp * 32 + lane;
+            const int4 e = sk.tab[tile];   // {first block, blocks, first CTA} of this tile
+            float *dst = part + ((size_t)(e.x + (cta - e.z)) * kMaxRows) * BM + warp * 32 + lane;
 #pragma unroll
             for (int m = 0; m < kMaxRows; m++)
                 if (m < M) dst[(size_t)m * BM] = __uint_as_float(r[m]) + __uint_as_float(r[16 + m]);
@@ -298,15 +316,24 @@ bool tc_shape_ok(int R, int K) { return R > 0 && K > 0 && R % tc::BM == 0 && K %
 StreamK tc_plan(int R, int K, int n_sm) {
     StreamK sk;
     sk.KB = K / tc::BK;
-    sk.U = (R / tc::BM) * sk.KB;
+    sk.tiles = R / tc::BM;
+    sk.U = sk.tiles * sk.KB;
     sk.G = sk.U < n_sm ? sk.U : n_sm;
     sk.base = sk.U / sk.G;
     sk.rem = sk.U % sk.G;
-    sk.max_seg = (sk.base + 1 + sk.KB - 1) / sk.KB + 1;
+    sk.tab = nullptr;
     return sk;
 }
 
-size_t tc_partial_floats(const StreamK &sk) { return (size_t)sk.G * sk.max_seg * kMaxRows * tc::BM; }
+int tc_fill_table(const StreamK &sk, int4 *tab) {
+    int next = 0;
+    for (int t = 0; t < sk.tiles; t++) {
+        const int c0 = sk.owner(t * sk.KB), c1 = sk.owner((t + 1) * sk.KB - 1);
+        tab[t] = make_int4(next, c1 - c0 + 1, c0, 0);
+        next += c1 - c0 + 1;
+    }
+    return next;   // <= tiles + G - 1
+}
 
 int tc_init() {
     static int done = 0;
