@@ -100,8 +100,10 @@ typedef struct eesd_sizes {
 } eesd_sizes;
 
 /* Caller-owned device memory.  kv_pool holds P = floor(kv_bytes / kv_page_bytes) pages laid
- * out [slot 0..L][page 0..P-1][K|V][H_kv][page_tokens][D]; slot L is the early-exit layer's
- * cache.  The workspace must be zero-filled by the caller before eesd_init. */
+ * out [slot 0..L][page 0..P-1][K|V][H_kv] blocks of page_tokens * D elements; slot L is the
+ * early-exit layer's cache.  A value block is [page_tokens][D]; a key block is stored
+ * transposed, [D/2][page_tokens][2] (pairs of adjacent dimensions, one column per token).
+ * The workspace must be zero-filled by the caller before eesd_init. */
 typedef struct eesd_buffers {
     void *weights;   size_t weights_bytes;
     void *kv_pool;   size_t kv_bytes;

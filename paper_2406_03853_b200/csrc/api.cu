@@ -30,6 +30,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int check_config(const eesd_config *c) {
     if (!c) return EESD_ERR_BADARG;
     if (c->d_model > 1024 * kSsqBlocks || c->n_kv_heads > 1024) return EESD_ERR_UNSUPPORTED;
+    if (c->max_ctx > 12288) return EESD_ERR_UNSUPPORTED;   // attention: at most 64 slices of 192 positions
     if (c->d_model <= 0 || c->n_heads <= 0 || c->n_kv_heads <= 0 || c->ffn_dim <= 0 || c->vocab <= 0 ||
         c->n_layers <= 0 || c->max_ctx <= 1)
         return EESD_ERR_BADARG;

@@ -269,11 +269,15 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
         if (i == 0) atomicOr(err, kErrBadPage);
         return;
     }
-    AT *dst = (AT *)kv.slot_base +
-              (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)kv.page_tokens * D +
-              (size_t)(pos % kv.page_tokens) * D + 2 * i;
-    dst[0] = from_f<AT>(a);
-    dst[1] = from_f<AT>(b);
+    AT *blk = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)kv.page_tokens * D;
+    if (isV) {
+        blk[(size_t)(pos % kv.page_tokens) * D + 2 * i] = from_f<AT>(a);
+        blk[(size_t)(pos % kv.page_tokens) * D + 2 * i + 1] = from_f<AT>(b);
+    } else {   // keys are cached transposed per page: pair i of a position at [i][pos % page_tokens]
+        AT *dst = blk + ((size_t)i * kv.page_tokens + (pos % kv.page_tokens)) * 2;
+        dst[0] = from_f<AT>(a);
+        dst[1] = from_f<AT>(b);
+    }
 }
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
                      const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err) {
@@ -285,42 +289,65 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 
 // ------------------------------------------------------------------------------------ paged decode attention
 // One kernel per layer: RoPE + KV append + attention over the paged cache + merge.
-// grid (H_kv, n_split), 256 threads.  Block (kh, sp) owns up to kAttnPos positions of KV head
-// kh (a whole number of pages) and serves every query head of its group and all M new rows
-// from ONE copy of those keys and values: the page blocks ([page_tokens][D], contiguous) are
-// brought into shared memory by bulk asynchronous copies on one mbarrier, so the cache is read
-// from HBM once per KV head.  The new rows' q, k, v come straight from the QKV projection's
-// partial sums (times the RMSNorm scale, rotated); the block whose slice holds a new position
-// places that key/value in its shared-memory tile and appends it to the cache in place.
+// grid (H_kv, n_split), 256 threads.  Block (kh, sp) owns `cap` cached positions of KV head kh
+// (a whole number of pages) and serves every query head of its group and all M new rows from
+// ONE copy of those keys and values: the page blocks are brought into shared memory by bulk
+// asynchronous copies on one mbarrier, so the cache is read from HBM once per KV head.
+// Keys are cached transposed per page ([D/2][page_tokens] pairs), so that in the score phase
+// consecutive lanes read consecutive positions of one pair of dimensions (no bank conflicts)
+// while the query values are broadcast; values are cached [page_tokens][D].
+// The new rows' q, k, v come straight from the QKV projection's partial sums (times the RMSNorm
+// scale, rotated); they are gathered while the cached slice is still arriving.  The block whose
+// slice holds a new position places that key/value in its tile and appends it to the cache.
 // Row m sees positions <= pos0 + m.  Each block writes, per (query head, row), the
 // un-normalised output, maximum and sum of its slice; the block that finishes last for a KV
 // head (an arrival counter, no waiting) merges the slices in index order.
-constexpr int kAttnPos = 128;     // positions per block
+constexpr int kAttnPos = 192;     // most positions per block
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-template <typename AT, int D, int RB>   // RB: (head, row) pairs per batch, 2..32
+// a pair of adjacent head dimensions of one key
+template <typename AT> struct KPair;
+template <> struct KPair<bf16> {
+    typedef uint32_t T;
+    __device__ __forceinline__ static T make(bf16 a, bf16 b) {
+        return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
+    }
+    __device__ __forceinline__ static void get(T w, float &a, float &b) {
+        a = __uint_as_float(w << 16);
+        b = __uint_as_float(w & 0xFFFF0000u);
+    }
+};
+template <> struct KPair<float> {
+    typedef float2 T;
+    __device__ __forceinline__ static T make(float a, float b) { return make_float2(a, b); }
+    __device__ __forceinline__ static void get(T w, float &a, float &b) { a = w.x; b = w.y; }
+};
+
+template <typename AT, int D, int RB>   // RB: (head, row) pairs per batch: 8, 16 or 32
 __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, const float2 *__restrict__ rope, KvGeom kv,
                                                    float *__restrict__ apart, unsigned int *tickets,
                                                    float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
                                                    int M, int pos0, int H, int pps, int n_split, float scale, int *err) {
-    constexpr int VEC = Vec16<AT>::N;       // elements per 16-byte chunk
-    constexpr int NCH = D / VEC;            // chunks per row
-    constexpr int RS = RB / 2;              // rows per thread in the score phase
+    typedef typename KPair<AT>::T KP;
+    constexpr int HALF = D / 2;
+    constexpr int DPL = D / 32;             // output dimensions per lane in the PV phase
     extern __shared__ __align__(128) unsigned char attn_smem[];
-    AT *sK = reinterpret_cast<AT *>(attn_smem);
-    AT *sV = sK + kAttnPos * D;
-    float *sq = reinterpret_cast<float *>(sV + kAttnPos * D);   // [RB][D]
-    float *sS = sq + RB * D;                                     // [RB][kAttnPos]
-    float *s_m = sS + RB * kAttnPos;                             // [RB]
+    const int PT = kv.page_tokens, group = H / kv.Hkv;
+    const int cap = pps * PT;               // positions this block's tiles hold
+    KP *sK = reinterpret_cast<KP *>(attn_smem);                  // [pps][D/2][PT] pairs
+    AT *sV = reinterpret_cast<AT *>(sK + (size_t)cap * HALF);   // [cap][D]
+    float2 *sq = reinterpret_cast<float2 *>(sV + (size_t)cap * D);   // [RB][D/2] rotated, scaled queries
+    float *sS = reinterpret_cast<float *>(sq + RB * HALF);       // [RB][cap]
+    float *s_m = sS + (size_t)RB * cap;                          // [RB]
     float *s_l = s_m + RB;
     float *s_rstd = s_l + RB;                                    // [kMaxRows]
     uint64_t *bar = reinterpret_cast<uint64_t *>(s_rstd + kMaxRows);
+    float *wgt = reinterpret_cast<float *>(bar + 2);             // [rows][n_split] merge weights
     __shared__ int s_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
-    const int PT = kv.page_tokens, group = H / kv.Hkv, HALF = D / 2;
     const int ctx_len = pos0 + M;
     const int n_pages = (ctx_len + PT - 1) / PT;
     const int page_lo = sp * pps, page_hi = min(n_pages, page_lo + pps);
@@ -335,23 +362,64 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-    if (tid == 0) {
-        // cached rows were written by earlier passes: no need to wait for this pass's producers
-        const uint32_t total = 2u * blk_bytes * (uint32_t)(page_hi - page_lo);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(total) : "memory");
-        for (int pg = page_lo; pg < page_hi; pg++) {
+    if (warp == 0) {
+        // cached rows were written by earlier passes: no need to wait for this pass's producers.
+        // One lane per page, so the page-table reads are in flight together.
+        if (lane == 0) {
+            const uint32_t total = 2u * blk_bytes * (uint32_t)(page_hi - page_lo);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(total) : "memory");
+        }
+        __syncwarp();
+        for (int pg = page_lo + lane; pg < page_hi; pg += 32) {
             const int page = kv.page_table[pg];
             const AT *src = (const AT *)kv.slot_base + (((size_t)page * 2) * kv.Hkv + kh) * (size_t)PT * D;
             const size_t v_off = (size_t)kv.Hkv * PT * D;
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(smem_addr(sK + (size_t)(pg - page_lo) * PT * D)), "l"(src), "r"(blk_bytes), "r"(smem_addr(bar)) : "memory");
+                         ::"r"(smem_addr(sK + (size_t)(pg - page_lo) * PT * HALF)), "l"(src), "r"(blk_bytes), "r"(smem_addr(bar)) : "memory");
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                          ::"r"(smem_addr(sV + (size_t)(pg - page_lo) * PT * D)), "l"(src + v_off), "r"(blk_bytes), "r"(smem_addr(bar)) : "memory");
         }
     }
     pdl_wait();   // from here on the QKV projection's partial sums are read
     if (tid < M) s_rstd[tid] = row_rstd(rs, tid);
-    {   // wait for the cached slice (bounded)
+    __syncthreads();
+    // new keys / values that fall into this slice: rotate and round now (while the cached slice
+    // is still arriving); they go into the tile and the cache once the slice has landed
+    constexpr int kNewPerThread = kMaxRows * D / 256;
+    const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
+    const int n_new = max(0, p_last - p_first) * D;
+    AT new_a[kNewPerThread], new_b[kNewPerThread];
+#pragma unroll
+    for (int it = 0; it < kNewPerThread; it++) {
+        const int idx = tid + it * 256;   // -> (position, K pair | V pair)
+        if (idx < n_new) {
+            const int pn = idx / D, w = idx - pn * D;
+            const int pos = p_first + pn, m = pos - pos0;
+            const int isV = w >= HALF, i = isV ? w - HALF : w;
+            const int col = (H + (isV ? kv.Hkv : 0) + kh) * D + 2 * i;
+            float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
+            if (!isV) {
+                const float2 cs = rope[(size_t)pos * HALF + i];
+                const float ra = a * cs.x - b * cs.y, rb = a * cs.y + b * cs.x;
+                a = ra; b = rb;
+            }
+            new_a[it] = from_f<AT>(a);
+            new_b[it] = from_f<AT>(b);
+        }
+    }
+    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
+    auto load_queries = [&](int r0, int nb) {   // rotated, pre-scaled queries of a batch
+        for (int idx = tid; idx < nb * HALF; idx += 256) {
+            const int rl = idx / HALF, i = idx - rl * HALF;
+            const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
+            const int col = (kh * group + g) * D + 2 * i;
+            const float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
+            const float2 cs = rope[(size_t)(pos0 + m) * HALF + i];
+            sq[rl * HALF + i] = make_float2((a * cs.x - b * cs.y) * scale, (a * cs.y + b * cs.x) * scale);
+        }
+    };
+    load_queries(0, min(RB, rows));
+    if (warp == 0) {   // wait for the cached slice (bounded); the other warps park at the barrier below
         bool ok = false;
         for (uint32_t i = 0; i < (1u << 24) && !ok; i++) {
             uint32_t p;
@@ -363,130 +431,131 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
         if (!ok && tid == 0) atomicOr(err, kErrWaitTimeout);
     }
     __syncthreads();
-    {   // new keys / values that fall into this slice: rotate, round, place in the tile, append
-        const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
-        const int n_new = p_last - p_first;
-        for (int idx = tid; idx < n_new * D; idx += 256) {   // idx -> (position, K pair | V pair)
+#pragma unroll
+    for (int it = 0; it < kNewPerThread; it++) {
+        const int idx = tid + it * 256;
+        if (idx < n_new) {
             const int pn = idx / D, w = idx - pn * D;
-            const int pos = p_first + pn, m = pos - pos0;
+            const int pos = p_first + pn, j = pos - lo;
             const int isV = w >= HALF, i = isV ? w - HALF : w;
-            const int col = (H + (isV ? kv.Hkv : 0) + kh) * D + 2 * i;
-            float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
-            if (!isV) {
-                const float2 cs = rope[(size_t)pos * HALF + i];
-                const float ra = a * cs.x - b * cs.y, rb = a * cs.y + b * cs.x;
-                a = ra; b = rb;
-            }
-            const AT va = from_f<AT>(a), vb = from_f<AT>(b);
-            AT *tile = (isV ? sV : sK) + (size_t)(pos - lo) * D + 2 * i;
-            tile[0] = va; tile[1] = vb;
             const int page = kv.page_table[pos / PT];
             if (page < 0 || page >= kv.n_pages_total) { atomicOr(err, kErrBadPage); continue; }
-            AT *dst = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)PT * D +
-                      (size_t)(pos % PT) * D + 2 * i;
-            dst[0] = va; dst[1] = vb;
+            AT *blk = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)PT * D;
+            if (isV) {
+                AT *tile = sV + (size_t)j * D + 2 * i;
+                tile[0] = new_a[it]; tile[1] = new_b[it];
+                blk[(size_t)(pos % PT) * D + 2 * i] = new_a[it];
+                blk[(size_t)(pos % PT) * D + 2 * i + 1] = new_b[it];
+            } else {   // keys: pair i of position pos at [i][pos % PT] of the page block
+                const KP w2 = KPair<AT>::make(new_a[it], new_b[it]);
+                sK[(size_t)(j / PT) * PT * HALF + (size_t)i * PT + (j % PT)] = w2;
+                reinterpret_cast<KP *>(blk)[(size_t)i * PT + (pos % PT)] = w2;
+            }
         }
     }
-    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
+    __syncthreads();
+
     for (int r0 = 0; r0 < rows; r0 += RB) {
         const int nb = min(RB, rows - r0);
-        for (int idx = tid; idx < nb * HALF; idx += 256) {   // rotated, pre-scaled queries of the batch
-            const int rl = idx / HALF, i = idx - rl * HALF;
-            const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
-            const int col = (kh * group + g) * D + 2 * i;
-            const float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
-            const float2 cs = rope[(size_t)(pos0 + m) * HALF + i];
-            sq[rl * D + 2 * i] = (a * cs.x - b * cs.y) * scale;
-            sq[rl * D + 2 * i + 1] = (a * cs.y + b * cs.x) * scale;
+        if (r0 > 0) {
+            load_queries(r0, nb);
+            __syncthreads();
         }
-        __syncthreads();
-        {   // scores: thread -> position j, every second row of the batch
-            const int j = tid & (kAttnPos - 1), rsel = tid >> 7;
-            float acc[RS];
+        {   // scores.  Work item = (16 consecutive positions, 8 rows); lane = position + 16 * (dimension pair parity)
+            const int t = lane & 15, eh = lane >> 4;
+            const int n_task = (npos + 15) / 16, n_rc = (nb + 7) / 8;
+            for (int item = warp; item < n_task * n_rc; item += 8) {
+                const int task = item % n_task, rc = item / n_task;
+                const int j = task * 16 + t;
+                const int jj = min(j, npos - 1);   // lanes past the slice recompute its last position
+                const KP *kp = sK + (size_t)(jj / PT) * PT * HALF + (jj % PT);
+                const float2 *qp = sq + (size_t)rc * 8 * HALF;
+                float acc[8];
 #pragma unroll
-            for (int i = 0; i < RS; i++) acc[i] = 0.f;
-            if (j < npos) {
-#pragma unroll 2
-                for (int c = 0; c < NCH; c++) {
-                    const int cc = (c + j) % NCH;   // rotate the chunk order: conflict-free shared loads
-                    float kvv[VEC];
-                    if (sizeof(AT) == 2) Vec16<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4 *>(sK + (size_t)j * D + cc * VEC), kvv);
-                    else {
-                        const float4 t = *reinterpret_cast<const float4 *>(sK + (size_t)j * D + cc * VEC);
-                        kvv[0] = t.x; kvv[1] = t.y; kvv[2] = t.z; kvv[3] = t.w;
+                for (int i = 0; i < 8; i++) acc[i] = 0.f;
+#pragma unroll 4
+                for (int e2 = eh; e2 < HALF; e2 += 2) {
+                    float ka, kb;
+                    KPair<AT>::get(kp[(size_t)e2 * PT], ka, kb);
+#pragma unroll
+                    for (int i = 0; i < 8; i++) {
+                        const float2 qv = qp[i * HALF + e2];   // rows past nb hold stale values: results dropped
+                        acc[i] = fmaf(ka, qv.x, acc[i]);
+                        acc[i] = fmaf(kb, qv.y, acc[i]);
                     }
+                }
 #pragma unroll
-                    for (int i = 0; i < RS; i++) {
-                        const int rl = min(rsel + 2 * i, RB - 1);   // rows past nb are computed and dropped
-                        float qv[VEC];
+                for (int i = 0; i < 8; i++) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 16);
+                if (eh == 0 && j < cap) {
 #pragma unroll
-                        for (int v = 0; v < VEC; v += 4) {
-                            const float4 t = *reinterpret_cast<const float4 *>(sq + rl * D + cc * VEC + v);
-                            qv[v] = t.x; qv[v + 1] = t.y; qv[v + 2] = t.z; qv[v + 3] = t.w;
+                    for (int i = 0; i < 8; i++) {
+                        const int rl = rc * 8 + i;
+                        if (rl < nb) {
+                            const int m = (r0 + rl) % M;
+                            sS[(size_t)rl * cap + j] = (j < npos && lo + j <= pos0 + m) ? acc[i] : -INFINITY;
                         }
-#pragma unroll
-                        for (int v = 0; v < VEC; v++) acc[i] = fmaf(kvv[v], qv[v], acc[i]);
                     }
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < RS; i++) {
-                const int rl = rsel + 2 * i;
-                if (rl < nb) {
-                    const int m = (r0 + rl) % M;
-                    sS[rl * kAttnPos + j] = (j < npos && lo + j <= pos0 + m) ? acc[i] : -INFINITY;
                 }
             }
         }
         __syncthreads();
+        const int npos16 = ((npos + 15) / 16) * 16 < cap ? ((npos + 15) / 16) * 16 : cap;   // entries the score phase wrote
         for (int rl = warp; rl < nb; rl += 8) {   // softmax numerators of this slice
             float mx = -INFINITY;
-            for (int j = lane; j < kAttnPos; j += 32) mx = fmaxf(mx, sS[rl * kAttnPos + j]);
+            for (int j = lane; j < npos16; j += 32) mx = fmaxf(mx, sS[(size_t)rl * cap + j]);
             mx = warp_max(mx);
             float sum = 0.f;
-            for (int j = lane; j < kAttnPos; j += 32) {
-                const float sv = sS[rl * kAttnPos + j];
+            for (int j = lane; j < npos16; j += 32) {
+                const float sv = sS[(size_t)rl * cap + j];
                 const float p = (sv == -INFINITY) ? 0.f : expf(sv - mx);
-                sS[rl * kAttnPos + j] = p;
+                sS[(size_t)rl * cap + j] = p;
                 sum += p;
             }
             sum = warp_sum(sum);
             if (lane == 0) { s_m[rl] = mx; s_l[rl] = sum; }
         }
         __syncthreads();
-        {   // o = P V: thread -> (pair of d, row group)
-            constexpr int NG = 256 / (D / 2);
-            constexpr int RPT = (RB + NG - 1) / NG;
-            const int d2 = tid % HALF, rg = tid / HALF;
-            float o0[RPT], o1[RPT];
+        {   // o = P V.  Warp w owns rows w, w + 8, ... of the batch; lane owns DPL output dimensions
+            constexpr int RPW = RB / 8;
+            float o[RPW][DPL];
 #pragma unroll
-            for (int i = 0; i < RPT; i++) { o0[i] = 0.f; o1[i] = 0.f; }
-            for (int j = 0; j < npos; j++) {
-                float v0, v1;
-                if (sizeof(AT) == 2) {
-                    const uint32_t w = *reinterpret_cast<const uint32_t *>(sV + (size_t)j * D + 2 * d2);
-                    v0 = __uint_as_float(w << 16); v1 = __uint_as_float(w & 0xFFFF0000u);
-                } else {
-                    const float2 t = *reinterpret_cast<const float2 *>(sV + (size_t)j * D + 2 * d2);
-                    v0 = t.x; v1 = t.y;
-                }
+            for (int i = 0; i < RPW; i++)
 #pragma unroll
-                for (int i = 0; i < RPT; i++) {
-                    const int rl = min(rg + NG * i, RB - 1);
-                    const float p = sS[rl * kAttnPos + j];
-                    o0[i] = fmaf(p, v0, o0[i]);
-                    o1[i] = fmaf(p, v1, o1[i]);
+                for (int e = 0; e < DPL; e++) o[i][e] = 0.f;
+            if (warp < nb) {
+                for (int j = 0; j < npos; j++) {
+                    float v[DPL];
+                    if (sizeof(AT) == 2) {
+                        if (DPL == 4) {
+                            const uint2 w = *reinterpret_cast<const uint2 *>(sV + (size_t)j * D + lane * 4);
+                            v[0] = __uint_as_float(w.x << 16); v[1] = __uint_as_float(w.x & 0xFFFF0000u);
+                            v[2 % DPL] = __uint_as_float(w.y << 16); v[3 % DPL] = __uint_as_float(w.y & 0xFFFF0000u);
+                        } else {
+                            const uint32_t w = *reinterpret_cast<const uint32_t *>(sV + (size_t)j * D + lane * 2);
+                            v[0] = __uint_as_float(w << 16); v[1] = __uint_as_float(w & 0xFFFF0000u);
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < DPL; e++) v[e] = to_f(sV[(size_t)j * D + lane * DPL + e]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < RPW; i++) {
+                        const int rl = min(warp + 8 * i, RB - 1);
+                        const float p = sS[(size_t)rl * cap + j];
+#pragma unroll
+                        for (int e = 0; e < DPL; e++) o[i][e] = fmaf(p, v[e], o[i][e]);
+                    }
                 }
             }
 #pragma unroll
-            for (int i = 0; i < RPT; i++) {
-                const int rl = rg + NG * i;
+            for (int i = 0; i < RPW; i++) {
+                const int rl = warp + 8 * i;
                 if (rl < nb) {
                     const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
                     float *dst = apart + (((size_t)(kh * group + g) * n_split + sp) * kMaxRows + m) * (D + 2);
-                    dst[2 * d2] = o0[i];
-                    dst[2 * d2 + 1] = o1[i];
-                    if (d2 == 0) { dst[D] = s_m[rl]; dst[D + 1] = s_l[rl]; }
+#pragma unroll
+                    for (int e = 0; e < DPL; e++) dst[lane * DPL + e] = o[i][e];
+                    if (lane == 0) { dst[D] = s_m[rl]; dst[D + 1] = s_l[rl]; }
                 }
             }
         }
@@ -504,36 +573,60 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     if (!s_last) return;
     __threadfence();
     const size_t sstride = (size_t)kMaxRows * (D + 2);
-    for (int idx = tid; idx < rows * D; idx += 256) {
-        const int rho = idx / D, dd = idx - rho * D;
+    for (int rho = warp; rho < rows; rho += 8) {   // normalised weight of every (pair, slice)
         const int g = rho / M, m = rho - g * M, h = kh * group + g;
         const float *src = apart + (size_t)h * n_split * sstride + (size_t)m * (D + 2);
         float mx = -INFINITY;
-        for (int s2 = 0; s2 < n_split; s2++) mx = fmaxf(mx, __ldcg(src + s2 * sstride + D));
-        float num = 0.f, den = 0.f;
-        for (int s2 = 0; s2 < n_split; s2++) {
+        for (int s2 = lane; s2 < n_split; s2 += 32) mx = fmaxf(mx, __ldcg(src + s2 * sstride + D));
+        mx = warp_max(mx);
+        float den = 0.f;   // each lane's slices first, then a fixed butterfly over the lanes
+        for (int s2 = lane; s2 < n_split; s2 += 32) {
             const float ms = __ldcg(src + s2 * sstride + D);
-            if (ms == -INFINITY) continue;
-            const float w = expf(ms - mx);
-            num = fmaf(w, __ldcg(src + s2 * sstride + dd), num);
+            const float w = (ms == -INFINITY) ? 0.f : expf(ms - mx);
+            wgt[rho * n_split + s2] = w;
             den = fmaf(w, __ldcg(src + s2 * sstride + D + 1), den);
         }
-        const float o = den > 0.f ? num / den : 0.f;
+        den = warp_sum(den);
+        const float inv = den > 0.f ? 1.0f / den : 0.f;
+        for (int s2 = lane; s2 < n_split; s2 += 32) wgt[rho * n_split + s2] *= inv;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < rows * D; idx += 256) {
+        const int rho = idx / D, dd = idx - rho * D;
+        const int g = rho / M, m = rho - g * M, h = kh * group + g;
+        const float *src = apart + (size_t)h * n_split * sstride + (size_t)m * (D + 2) + dd;
+        const float *wr = wgt + rho * n_split;
+        float o = 0.f;
+        int s2 = 0;
+        for (; s2 + 4 <= n_split; s2 += 4) {   // four independent loads in flight
+            const float a0 = __ldcg(src + (s2 + 0) * sstride), a1 = __ldcg(src + (s2 + 1) * sstride);
+            const float a2 = __ldcg(src + (s2 + 2) * sstride), a3 = __ldcg(src + (s2 + 3) * sstride);
+            o = fmaf(wr[s2], a0, o);
+            o = fmaf(wr[s2 + 1], a1, o);
+            o = fmaf(wr[s2 + 2], a2, o);
+            o = fmaf(wr[s2 + 3], a3, o);
+        }
+        for (; s2 < n_split; s2++) o = fmaf(wr[s2], __ldcg(src + s2 * sstride), o);
         if (attn_out) attn_out[(size_t)m * H * D + (size_t)h * D + dd] = o;
         if (attn_split) store_split(attn_split, m, (size_t)H * D, (size_t)h * D + dd, o);
     }
+}
+
+static size_t attn_smem_bytes(int es, int D, int RB, int cap, int rows, int n_split) {
+    return (size_t)2 * cap * D * es + (size_t)RB * D * 4 + (size_t)RB * cap * 4 + 2 * RB * 4 + kMaxRows * 4 + 16 +
+           (size_t)rows * n_split * 4 + 16;
 }
 
 template <typename AT, int D, int RB>
 static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                         float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
                         int pps, int n_split, float scale, int *err) {
-    const size_t smem = (size_t)2 * kAttnPos * D * sizeof(AT) + (size_t)RB * D * 4 + (size_t)RB * kAttnPos * 4 +
-                        2 * RB * 4 + kMaxRows * 4 + 16;
-    static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(attn_kernel<AT, D, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        configured = true;
+    const int rows = (H / kv.Hkv) * M;
+    const size_t smem = attn_smem_bytes((int)sizeof(AT), D, RB, pps * kv.page_tokens, rows, n_split);
+    static size_t configured = 0;   // largest dynamic shared memory size enabled so far
+    if (smem > configured) {
+        cudaFuncSetAttribute(attn_kernel<AT, D, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
+        configured = 227 * 1024 - 1024;
     }
     launch_k(attn_kernel<AT, D, RB>, dim3(kv.Hkv, n_split), dim3(256), smem, s, pdl_enabled(), pv, rs, rope, kv, apart,
              tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err);
@@ -545,22 +638,25 @@ static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs
                           int pps, int n_split, float scale, int *err) {
     const int rows = (H / kv.Hkv) * M;
 #define EESD_ATTN(RB) attn_launch<AT, D, RB>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err)
-    if (rows <= 2) EESD_ATTN(2);
-    else if (rows <= 4) EESD_ATTN(4);
-    else if (rows <= 8) EESD_ATTN(8);
+    if (rows <= 8) EESD_ATTN(8);
     else if (rows <= 16) EESD_ATTN(16);
     else EESD_ATTN(32);
 #undef EESD_ATTN
 }
 
+// slices of the cached context: pages per block and number of blocks per KV head
 int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_sm, int max_splits, int *pps_out) {
     const int n_pages = (ctx_len + page_tokens - 1) / page_tokens;
-    int pps = kAttnPos / page_tokens;                 // most pages one block can hold
+    const int cap = kAttnPos / page_tokens > 0 ? kAttnPos / page_tokens : 1;   // pages one block can hold
+    // one wave: about two blocks per SM in flight, so aim for H_kv * n_split <= 2 * n_sm
+    int want = 2 * n_sm / Hkv;
+    if (want < 1) want = 1;
+    if (want > max_splits) want = max_splits;
+    int pps = (n_pages + want - 1) / want;
+    if (pps > cap) pps = cap;            // longer contexts: more slices than one wave holds
     if (pps < 1) pps = 1;
-    // enough blocks to fill the machine about twice, while slices stay whole pages
-    while (pps > 1 && Hkv * ((n_pages + pps - 1) / pps) < 2 * n_sm) pps--;
     int n_split = (n_pages + pps - 1) / pps;
-    while (n_split > max_splits) { pps++; n_split = (n_pages + pps - 1) / pps; }
+    while (n_split > max_splits && pps < cap) { pps++; n_split = (n_pages + pps - 1) / pps; }
     *pps_out = pps;
     return n_split;
 }

@@ -13,7 +13,8 @@ struct IntList16 { int32_t v[16]; };
 
 // geometry of one paged KV cache slot
 struct KvGeom {
-    void *slot_base;            // first byte of the slot: [page][K|V][H_kv][page_tokens][D]
+    void *slot_base;            // first byte of the slot: [page][K|V][H_kv] blocks of page_tokens * D
+                                // elements; K block [D/2][page_tokens][2], V block [page_tokens][D]
     const int32_t *page_table;  // logical page -> physical page
     int Hkv, D, page_tokens, n_pages_total;
 };
