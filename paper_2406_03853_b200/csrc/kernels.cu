@@ -303,6 +303,7 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 // un-normalised output, maximum and sum of its slice; the block that finishes last for a KV
 // head (an arrival counter, no waiting) merges the slices in index order.
 constexpr int kAttnPos = 192;     // most positions per block
+constexpr int kMaxSlices = 64;    // most slices per head (layout of the per-slice maxima and sums)
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -337,13 +338,22 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     const int cap = pps * PT;               // positions this block's tiles hold
     KP *sK = reinterpret_cast<KP *>(attn_smem);                  // [pps][D/2][PT] pairs
     AT *sV = reinterpret_cast<AT *>(sK + (size_t)cap * HALF);   // [cap][D]
-    float2 *sq = reinterpret_cast<float2 *>(sV + (size_t)cap * D);   // [RB][D/2] rotated, scaled queries
-    float *sS = reinterpret_cast<float *>(sq + RB * HALF);       // [RB][cap]
-    float *s_m = sS + (size_t)RB * cap;                          // [RB]
+    // rotated, scaled queries: fp32 pairs [RB][D/2] (fp32 cache), or two bf16 terms per pair,
+    // [2][RBP][QS] words (bf16 cache, tensor-core path; QS is padded against bank conflicts)
+    constexpr bool kTC = sizeof(AT) == 2;
+    constexpr int RBP = RB < 16 ? 16 : RB, QS = HALF + 4;
+    constexpr int SQ_WORDS = kTC ? 2 * RBP * QS : 2 * RB * HALF;
+    float2 *sq = reinterpret_cast<float2 *>(sV + (size_t)cap * D);
+    uint32_t *sqh = reinterpret_cast<uint32_t *>(sq), *sql = sqh + RBP * QS;
+    const int ss = cap + 12;                                     // row stride of the score matrix
+    float *sS = reinterpret_cast<float *>(sq) + SQ_WORDS;        // [RB][ss]
+    float *s_m = sS + (size_t)RB * ss;                           // [RB]
     float *s_l = s_m + RB;
     float *s_rstd = s_l + RB;                                    // [kMaxRows]
     uint64_t *bar = reinterpret_cast<uint64_t *>(s_rstd + kMaxRows);
     float *wgt = reinterpret_cast<float *>(bar + 2);             // [rows][n_split] merge weights
+    // per-slice (maximum, sum) pairs live behind the outputs: [H][16][kMaxSlices]
+    float2 *ml = reinterpret_cast<float2 *>(apart + (size_t)H * kMaxSlices * kMaxRows * D);
     __shared__ int s_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -415,7 +425,15 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const int col = (kh * group + g) * D + 2 * i;
             const float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
             const float2 cs = rope[(size_t)(pos0 + m) * HALF + i];
-            sq[rl * HALF + i] = make_float2((a * cs.x - b * cs.y) * scale, (a * cs.y + b * cs.x) * scale);
+            const float qa = (a * cs.x - b * cs.y) * scale, qb = (a * cs.y + b * cs.x) * scale;
+            if (kTC) {
+                const bf16 ha = __float2bfloat16_rn(qa), hb = __float2bfloat16_rn(qb);
+                sqh[rl * QS + i] = KPair<bf16>::make(ha, hb);
+                sql[rl * QS + i] = KPair<bf16>::make(__float2bfloat16_rn(qa - __bfloat162float(ha)),
+                                                     __float2bfloat16_rn(qb - __bfloat162float(hb)));
+            } else {
+                sq[rl * HALF + i] = make_float2(qa, qb);
+            }
         }
     };
     load_queries(0, min(RB, rows));
@@ -453,6 +471,11 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             }
         }
     }
+    const int npos_k = min(cap, ((npos + 15) / 16) * 16);   // positions the PV products run over
+    if (kTC) {   // value rows past the slice hold whatever the page held: make them zeros
+        for (int idx = tid; idx < (npos_k - npos) * (D / 8); idx += 256)
+            reinterpret_cast<uint4 *>(sV + (size_t)npos * D)[idx] = make_uint4(0u, 0u, 0u, 0u);
+    }
     __syncthreads();
 
     for (int r0 = 0; r0 < rows; r0 += RB) {
@@ -461,7 +484,51 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             load_queries(r0, nb);
             __syncthreads();
         }
-        {   // scores.  Work item = (16 consecutive positions, 8 rows); lane = position + 16 * (dimension pair parity)
+        if constexpr (kTC) {
+            // scores on the tensor cores: S = Q K^T as m16n8k16 products, Q = hi + lo (two bf16
+            // terms, exact products, fp32 accumulation).  The transposed key tile yields the
+            // B fragments as plain 32-bit loads: pair (2t, 2t+1) of position n0 + g.
+            const int g = lane >> 2, t = lane & 3;
+            const int n_tiles = (npos + 7) / 8;
+            for (int mt = 0; mt * 16 < nb; mt++) {
+                uint32_t ah[D / 16][4], al[D / 16][4];
+                const int ra = (mt * 16 + g) * QS, rb2 = (mt * 16 + g + 8) * QS;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ks++) {
+                    ah[ks][0] = sqh[ra + ks * 8 + t];      ah[ks][1] = sqh[rb2 + ks * 8 + t];
+                    ah[ks][2] = sqh[ra + ks * 8 + t + 4];  ah[ks][3] = sqh[rb2 + ks * 8 + t + 4];
+                    al[ks][0] = sql[ra + ks * 8 + t];      al[ks][1] = sql[rb2 + ks * 8 + t];
+                    al[ks][2] = sql[ra + ks * 8 + t + 4];  al[ks][3] = sql[rb2 + ks * 8 + t + 4];
+                }
+                for (int nt = warp; nt < n_tiles; nt += 8) {
+                    const int n0 = nt * 8;
+                    const uint32_t *kp = reinterpret_cast<const uint32_t *>(sK) + (size_t)(n0 / PT) * PT * HALF + (n0 % PT) + g;
+                    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ks++) {
+                        const uint32_t b0 = kp[(size_t)(ks * 8 + t) * PT], b1 = kp[(size_t)(ks * 8 + t + 4) * PT];
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                                     : "r"(ah[ks][0]), "r"(ah[ks][1]), "r"(ah[ks][2]), "r"(ah[ks][3]), "r"(b0), "r"(b1));
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                                     : "r"(al[ks][0]), "r"(al[ks][1]), "r"(al[ks][2]), "r"(al[ks][3]), "r"(b0), "r"(b1));
+                    }
+#pragma unroll
+                    for (int hf = 0; hf < 2; hf++) {
+                        const int rl = mt * 16 + g + 8 * hf;
+                        if (rl < nb) {
+                            const int m = (r0 + rl) % M;
+#pragma unroll
+                            for (int q2 = 0; q2 < 2; q2++) {
+                                const int j = n0 + 2 * t + q2;
+                                sS[(size_t)rl * ss + j] = (j < npos && lo + j <= pos0 + m) ? c[hf * 2 + q2] : -INFINITY;
+                            }
+                        }
+                    }
+                }
+            }
+        } else {   // scores.  Work item = (16 consecutive positions, 8 rows); lane = position + 16 * (dimension pair parity)
             const int t = lane & 15, eh = lane >> 4;
             const int n_task = (npos + 15) / 16, n_rc = (nb + 7) / 8;
             for (int item = warp; item < n_task * n_rc; item += 8) {
@@ -492,30 +559,84 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                         const int rl = rc * 8 + i;
                         if (rl < nb) {
                             const int m = (r0 + rl) % M;
-                            sS[(size_t)rl * cap + j] = (j < npos && lo + j <= pos0 + m) ? acc[i] : -INFINITY;
+                            sS[(size_t)rl * ss + j] = (j < npos && lo + j <= pos0 + m) ? acc[i] : -INFINITY;
                         }
                     }
                 }
             }
         }
         __syncthreads();
-        const int npos16 = ((npos + 15) / 16) * 16 < cap ? ((npos + 15) / 16) * 16 : cap;   // entries the score phase wrote
+        const int nposw = kTC ? ((npos + 7) / 8) * 8 : min(cap, ((npos + 15) / 16) * 16);   // entries the score phase wrote
+        const int npos16 = max(nposw, npos_k);   // the tensor-core PV reads weights (zeros) up to npos_k
         for (int rl = warp; rl < nb; rl += 8) {   // softmax numerators of this slice
             float mx = -INFINITY;
-            for (int j = lane; j < npos16; j += 32) mx = fmaxf(mx, sS[(size_t)rl * cap + j]);
+            for (int j = lane; j < nposw; j += 32) mx = fmaxf(mx, sS[(size_t)rl * ss + j]);
             mx = warp_max(mx);
             float sum = 0.f;
             for (int j = lane; j < npos16; j += 32) {
-                const float sv = sS[(size_t)rl * cap + j];
+                const float sv = j < nposw ? sS[(size_t)rl * ss + j] : -INFINITY;
                 const float p = (sv == -INFINITY) ? 0.f : expf(sv - mx);
-                sS[(size_t)rl * cap + j] = p;
+                sS[(size_t)rl * ss + j] = p;
                 sum += p;
             }
             sum = warp_sum(sum);
             if (lane == 0) { s_m[rl] = mx; s_l[rl] = sum; }
         }
         __syncthreads();
-        {   // o = P V.  Warp w owns rows w, w + 8, ... of the batch; lane owns DPL output dimensions
+        if constexpr (kTC) {
+            // o = P V on the tensor cores: P = hi + lo (two bf16 terms), V fragments by transposing
+            // matrix loads from the row-major value tile.  Warp w owns output dimensions 8w.. and
+            // 8(w+8)..; accumulators stay in registers over all positions.
+            const int g = lane >> 2, t = lane & 3;
+            for (int mt = 0; mt * 16 < nb; mt++) {
+                float c[D / 64][4];
+#pragma unroll
+                for (int x = 0; x < D / 64; x++) { c[x][0] = c[x][1] = c[x][2] = c[x][3] = 0.f; }
+                const float *pa = sS + (size_t)(mt * 16 + g) * ss, *pb = sS + (size_t)min(mt * 16 + g + 8, RB - 1) * ss;
+                for (int k0 = 0; k0 < npos_k; k0 += 16) {
+                    const float2 f0 = *reinterpret_cast<const float2 *>(pa + k0 + 2 * t);
+                    const float2 f1 = *reinterpret_cast<const float2 *>(pb + k0 + 2 * t);
+                    const float2 f2 = *reinterpret_cast<const float2 *>(pa + k0 + 2 * t + 8);
+                    const float2 f3 = *reinterpret_cast<const float2 *>(pb + k0 + 2 * t + 8);
+                    uint32_t ah[4], al[4];
+                    const float2 ff[4] = {f0, f1, f2, f3};
+#pragma unroll
+                    for (int x = 0; x < 4; x++) {
+                        const bf16 ha = __float2bfloat16_rn(ff[x].x), hb = __float2bfloat16_rn(ff[x].y);
+                        ah[x] = KPair<bf16>::make(ha, hb);
+                        al[x] = KPair<bf16>::make(__float2bfloat16_rn(ff[x].x - __bfloat162float(ha)),
+                                                  __float2bfloat16_rn(ff[x].y - __bfloat162float(hb)));
+                    }
+#pragma unroll
+                    for (int x = 0; x < D / 64; x++) {
+                        const int d0 = (warp + 8 * x) * 8;
+                        uint32_t b0, b1;
+                        const uint32_t addr = smem_addr(sV + (size_t)(k0 + (lane & 15)) * D + d0);
+                        asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+f"(c[x][0]), "+f"(c[x][1]), "+f"(c[x][2]), "+f"(c[x][3])
+                                     : "r"(ah[0]), "r"(ah[1]), "r"(ah[2]), "r"(ah[3]), "r"(b0), "r"(b1));
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+f"(c[x][0]), "+f"(c[x][1]), "+f"(c[x][2]), "+f"(c[x][3])
+                                     : "r"(al[0]), "r"(al[1]), "r"(al[2]), "r"(al[3]), "r"(b0), "r"(b1));
+                    }
+                }
+#pragma unroll
+                for (int hf = 0; hf < 2; hf++) {
+                    const int rl = mt * 16 + g + 8 * hf;
+                    if (rl < nb) {
+                        const int gq = (r0 + rl) / M, m = (r0 + rl) - gq * M, h = kh * group + gq;
+                        float *dst = apart + (((size_t)h * n_split + sp) * kMaxRows + m) * D;
+#pragma unroll
+                        for (int x = 0; x < D / 64; x++) {
+                            const int d0 = (warp + 8 * x) * 8;
+                            *reinterpret_cast<float2 *>(dst + d0 + 2 * t) = make_float2(c[x][hf * 2], c[x][hf * 2 + 1]);
+                        }
+                        if (warp == 0 && t == 0) ml[((size_t)h * kMaxRows + m) * kMaxSlices + sp] = make_float2(s_m[rl], s_l[rl]);
+                    }
+                }
+            }
+        } else {   // o = P V.  Warp w owns rows w, w + 8, ... of the batch; lane owns DPL output dimensions
             constexpr int RPW = RB / 8;
             float o[RPW][DPL];
 #pragma unroll
@@ -541,7 +662,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
 #pragma unroll
                     for (int i = 0; i < RPW; i++) {
                         const int rl = min(warp + 8 * i, RB - 1);
-                        const float p = sS[(size_t)rl * cap + j];
+                        const float p = sS[(size_t)rl * ss + j];
 #pragma unroll
                         for (int e = 0; e < DPL; e++) o[i][e] = fmaf(p, v[e], o[i][e]);
                     }
@@ -552,10 +673,11 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                 const int rl = warp + 8 * i;
                 if (rl < nb) {
                     const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
-                    float *dst = apart + (((size_t)(kh * group + g) * n_split + sp) * kMaxRows + m) * (D + 2);
+                    const int h = kh * group + g;
+                    float *dst = apart + (((size_t)h * n_split + sp) * kMaxRows + m) * D;
 #pragma unroll
                     for (int e = 0; e < DPL; e++) dst[lane * DPL + e] = o[i][e];
-                    if (lane == 0) { dst[D] = s_m[rl]; dst[D + 1] = s_l[rl]; }
+                    if (lane == 0) ml[((size_t)h * kMaxRows + m) * kMaxSlices + sp] = make_float2(s_m[rl], s_l[rl]);
                 }
             }
         }
@@ -572,48 +694,43 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    const size_t sstride = (size_t)kMaxRows * (D + 2);
-    for (int rho = warp; rho < rows; rho += 8) {   // normalised weight of every (pair, slice)
+    const size_t sstride = (size_t)kMaxRows * D;
+    for (int rho = warp; rho < rows; rho += 8) {   // normalised weight of every (pair, slice): one round trip
         const int g = rho / M, m = rho - g * M, h = kh * group + g;
-        const float *src = apart + (size_t)h * n_split * sstride + (size_t)m * (D + 2);
-        float mx = -INFINITY;
-        for (int s2 = lane; s2 < n_split; s2 += 32) mx = fmaxf(mx, __ldcg(src + s2 * sstride + D));
-        mx = warp_max(mx);
-        float den = 0.f;   // each lane's slices first, then a fixed butterfly over the lanes
-        for (int s2 = lane; s2 < n_split; s2 += 32) {
-            const float ms = __ldcg(src + s2 * sstride + D);
-            const float w = (ms == -INFINITY) ? 0.f : expf(ms - mx);
-            wgt[rho * n_split + s2] = w;
-            den = fmaf(w, __ldcg(src + s2 * sstride + D + 1), den);
-        }
-        den = warp_sum(den);
+        const float2 *src = ml + ((size_t)h * kMaxRows + m) * kMaxSlices;
+        const float2 none = make_float2(-INFINITY, 0.f);
+        const float2 v0 = lane < n_split ? __ldcg(src + lane) : none;
+        const float2 v1 = lane + 32 < n_split ? __ldcg(src + lane + 32) : none;
+        const float mx = warp_max(fmaxf(v0.x, v1.x));
+        const float w0 = (v0.x == -INFINITY) ? 0.f : expf(v0.x - mx), w1 = (v1.x == -INFINITY) ? 0.f : expf(v1.x - mx);
+        const float den = warp_sum(fmaf(w0, v0.y, w1 * v1.y));   // fixed butterfly over the lanes
         const float inv = den > 0.f ? 1.0f / den : 0.f;
-        for (int s2 = lane; s2 < n_split; s2 += 32) wgt[rho * n_split + s2] *= inv;
+        if (lane < n_split) wgt[rho * n_split + lane] = w0 * inv;
+        if (lane + 32 < n_split) wgt[rho * n_split + lane + 32] = w1 * inv;
     }
     __syncthreads();
     for (int idx = tid; idx < rows * D; idx += 256) {
         const int rho = idx / D, dd = idx - rho * D;
         const int g = rho / M, m = rho - g * M, h = kh * group + g;
-        const float *src = apart + (size_t)h * n_split * sstride + (size_t)m * (D + 2) + dd;
+        const float *src = apart + ((size_t)h * n_split * kMaxRows + m) * D + dd;
         const float *wr = wgt + rho * n_split;
         float o = 0.f;
-        int s2 = 0;
-        for (; s2 + 4 <= n_split; s2 += 4) {   // four independent loads in flight
-            const float a0 = __ldcg(src + (s2 + 0) * sstride), a1 = __ldcg(src + (s2 + 1) * sstride);
-            const float a2 = __ldcg(src + (s2 + 2) * sstride), a3 = __ldcg(src + (s2 + 3) * sstride);
-            o = fmaf(wr[s2], a0, o);
-            o = fmaf(wr[s2 + 1], a1, o);
-            o = fmaf(wr[s2 + 2], a2, o);
-            o = fmaf(wr[s2 + 3], a3, o);
+        for (int s2 = 0; s2 < n_split; s2 += 8) {   // eight independent loads in flight, added in slice order
+            float a[8];
+#pragma unroll
+            for (int u = 0; u < 8; u++) a[u] = __ldcg(src + (size_t)min(s2 + u, n_split - 1) * sstride);
+#pragma unroll
+            for (int u = 0; u < 8; u++) o = fmaf(s2 + u < n_split ? wr[s2 + u] : 0.f, a[u], o);
         }
-        for (; s2 < n_split; s2++) o = fmaf(wr[s2], __ldcg(src + s2 * sstride), o);
         if (attn_out) attn_out[(size_t)m * H * D + (size_t)h * D + dd] = o;
         if (attn_split) store_split(attn_split, m, (size_t)H * D, (size_t)h * D + dd, o);
     }
 }
 
 static size_t attn_smem_bytes(int es, int D, int RB, int cap, int rows, int n_split) {
-    return (size_t)2 * cap * D * es + (size_t)RB * D * 4 + (size_t)RB * cap * 4 + 2 * RB * 4 + kMaxRows * 4 + 16 +
+    const int rbp = RB < 16 ? 16 : RB;
+    const size_t sq_words = es == 2 ? (size_t)2 * rbp * (D / 2 + 4) : (size_t)RB * D;
+    return (size_t)2 * cap * D * es + sq_words * 4 + (size_t)RB * (cap + 12) * 4 + 2 * RB * 4 + kMaxRows * 4 + 16 +
            (size_t)rows * n_split * 4 + 16;
 }
 
@@ -655,8 +772,9 @@ int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_sm, int max_sp
     int pps = (n_pages + want - 1) / want;
     if (pps > cap) pps = cap;            // longer contexts: more slices than one wave holds
     if (pps < 1) pps = 1;
+    if ((pps * page_tokens) % 16) pps++;   // tiles hold a multiple of 16 positions
     int n_split = (n_pages + pps - 1) / pps;
-    while (n_split > max_splits && pps < cap) { pps++; n_split = (n_pages + pps - 1) / pps; }
+    while (n_split > max_splits && pps < cap) { pps += (page_tokens < 16 ? 2 : 1); n_split = (n_pages + pps - 1) / pps; }
     *pps_out = pps;
     return n_split;
 }
