@@ -125,7 +125,7 @@ struct eesd_ctx {
     CUtensorMap m_exit_kv, m_lm_head, m_exit_head;
     bool use_tc;
     int n_sm;
-    StreamK plan[P_COUNT];       // tensor-core path: work split and block table per shape
+    StreamK plan[P_COUNT];       // tensor-core path: work split per shape
     float2 *rope;
     int32_t *page_table, *ints;
     int *err;
@@ -216,7 +216,7 @@ PartView run_proj(eesd_ctx *c, const void *W, const CUtensorMap *mW, int shape, 
     pv.R = R;
     if (c->use_tc) {
         pv.mode = 1;
-        pv.tab = c->plan[shape].tab;
+        pv.sk = c->plan[shape];
         launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, c->plan[shape], M, c->err);
     } else {
         const float *A = which == X_NORM ? c->xn : which == X_ATTN ? c->attn : c->h;
@@ -572,19 +572,9 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         ok = ok && tc_make_map(&c->m_exit_kv, c->layers[cfg->n_layers].wqkv + (size_t)qd_ * d * 2, 2 * kvd_, d, 128);
         ok = ok && tc_make_map(&c->m_lm_head, c->lm_head, cfg->vocab, d, 128);
         ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128);
-        // work split and block table of every projection shape
+        // work split of every projection shape
         const int shapes[P_COUNT][2] = {{qd_ + 2 * kvd_, d}, {d, qd_}, {2 * F, d}, {d, F}, {2 * kvd_, d}, {cfg->vocab, d}};
-        size_t maxR = 0;
-        for (auto &sh : shapes) if ((size_t)sh[0] > maxR) maxR = sh[0];
-        std::vector<int4> host_tab;
-        for (int i = 0; i < P_COUNT && ok; i++) {
-            c->plan[i] = tc_plan(shapes[i][0], shapes[i][1], c->n_sm);
-            host_tab.assign(c->plan[i].tiles, make_int4(0, 0, 0, 0));
-            tc_fill_table(c->plan[i], host_tab.data());
-            int4 *dev = (int4 *)(ws + w.tabs) + (size_t)i * (maxR / 128 + 1);
-            ok = cudaMemcpy(dev, host_tab.data(), host_tab.size() * sizeof(int4), cudaMemcpyHostToDevice) == cudaSuccess;
-            c->plan[i].tab = dev;
-        }
+        for (int i = 0; i < P_COUNT; i++) c->plan[i] = tc_plan(shapes[i][0], shapes[i][1], c->n_sm);
         if (!ok) {
             delete c;
             return EESD_ERR_CUDA;
@@ -909,17 +899,11 @@ int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *
         CUtensorMap mW, mX;
         if (!tc_make_map(&mW, W, R, K, 128) || !tc_make_map(&mX, sc + off_xs, 2 * EESD_MAX_ROWS, K, 2 * EESD_MAX_ROWS))
             return EESD_ERR_CUDA;
-        StreamK sk = tc_plan(R, K, n_sm);
-        std::vector<int4> tab(sk.tiles);
-        tc_fill_table(sk, tab.data());
-        sk.tab = (const int4 *)(sc + off_tab);
+        const StreamK sk = tc_plan(R, K, n_sm);
         if (cudaMemsetAsync(sc, 0, 16, s) != cudaSuccess) return EESD_ERR_CUDA;
-        // pageable source: the copy is staged before the call returns, so `tab` may go out of scope
-        if (cudaMemcpyAsync(sc + off_tab, tab.data(), tab.size() * sizeof(int4), cudaMemcpyHostToDevice, s) != cudaSuccess)
-            return EESD_ERR_CUDA;
         launch_split_rows(s, A, sc + off_xs, M, K);
         pv.mode = 1;
-        pv.tab = sk.tab;
+        pv.sk = sk;
         launch_gemm_tc(s, mW, mX, part, sk, M, (int *)sc);
     } else {
         pv.mode = 0;

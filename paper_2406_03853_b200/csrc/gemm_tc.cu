@@ -17,8 +17,7 @@
 //     activation times a bf16 weight to about 2^-17 relative.  The extra columns cost tensor
 //     time only, which this kernel has to spare.
 // Each segment (part of one tile's k range done by one CTA) is written as an fp32 partial
-// block; consumers add the blocks of a tile in CTA order (a small per-tile table says where
-// they are), so results are bit-reproducible and do
+// block (numbered cta + tile); consumers add the blocks of a tile in CTA order, so results are bit-reproducible and do
 // not depend on M.
 //
 // Every wait is bounded: on expiry the thread raises the error word, the CTA drains its
@@ -261,8 +260,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[b]);
-            const int4 e = sk.tab[tile];   // {first block, blocks, first CTA} of this tile
-            float *dst = part + ((size_t)(e.x + (cta - e.z)) * kMaxRows) * BM + warp * 32 + lane;
+            float *dst = part + ((size_t)(cta + tile) * kMaxRows) * BM + warp * 32 + lane;
 #pragma unroll
             for (int m = 0; m < kMaxRows; m++)
                 if (m < M) dst[(size_t)m * BM] = __uint_as_float(r[m]) + __uint_as_float(r[16 + m]);
@@ -321,18 +319,7 @@ StreamK tc_plan(int R, int K, int n_sm) {
     sk.G = sk.U < n_sm ? sk.U : n_sm;
     sk.base = sk.U / sk.G;
     sk.rem = sk.U % sk.G;
-    sk.tab = nullptr;
     return sk;
-}
-
-int tc_fill_table(const StreamK &sk, int4 *tab) {
-    int next = 0;
-    for (int t = 0; t < sk.tiles; t++) {
-        const int c0 = sk.owner(t * sk.KB), c1 = sk.owner((t + 1) * sk.KB - 1);
-        tab[t] = make_int4(next, c1 - c0 + 1, c0, 0);
-        next += c1 - c0 + 1;
-    }
-    return next;   // <= tiles + G - 1
 }
 
 int tc_init() {

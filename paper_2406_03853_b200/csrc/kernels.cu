@@ -18,15 +18,16 @@ __device__ __forceinline__ float part_gather(const PartView &pv, int m, int r) {
     if (pv.mode == 0) {
         for (int s = 0; s < pv.S; s++) v += pv.base[(size_t)s * pv.split_stride + (size_t)m * pv.R + r];
     } else {
-        const int4 e = __ldg(pv.tab + (r >> 7));
-        const float *p = pv.base + ((size_t)e.x * kMaxRows + m) * 128 + (r & 127);
+        const int t = r >> 7;
+        const int c0 = pv.sk.owner(t * pv.sk.KB), n = pv.sk.owner((t + 1) * pv.sk.KB - 1) - c0 + 1;
+        const float *p = pv.base + ((size_t)(c0 + t) * kMaxRows + m) * 128 + (r & 127);
         int i = 0;
-        for (; i + 2 <= e.y; i += 2) {   // two loads in flight, added in block order
+        for (; i + 2 <= n; i += 2) {   // two loads in flight, added in block order
             const float a = __ldcg(p + (size_t)i * kMaxRows * 128), b = __ldcg(p + (size_t)(i + 1) * kMaxRows * 128);
             v += a;
             v += b;
         }
-        if (i < e.y) v += __ldcg(p + (size_t)i * kMaxRows * 128);
+        if (i < n) v += __ldcg(p + (size_t)i * kMaxRows * 128);
     }
     return v;
 }
@@ -47,16 +48,17 @@ __device__ __forceinline__ float4 part_gather4(const PartView &pv, int m, int r)
             v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
         }
     } else {
-        const int4 e = __ldg(pv.tab + (r >> 7));
-        const float *p = pv.base + ((size_t)e.x * kMaxRows + m) * 128 + (r & 127);
+        const int t = r >> 7;
+        const int c0 = pv.sk.owner(t * pv.sk.KB), n = pv.sk.owner((t + 1) * pv.sk.KB - 1) - c0 + 1;
+        const float *p = pv.base + ((size_t)(c0 + t) * kMaxRows + m) * 128 + (r & 127);
         int i = 0;
-        for (; i + 2 <= e.y; i += 2) {
+        for (; i + 2 <= n; i += 2) {
             const float4 a = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)i * kMaxRows * 128));
             const float4 b = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)(i + 1) * kMaxRows * 128));
             v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
             v.x += b.x; v.y += b.y; v.z += b.z; v.w += b.w;
         }
-        if (i < e.y) {
+        if (i < n) {
             const float4 a = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)i * kMaxRows * 128));
             v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
         }

@@ -21,11 +21,12 @@ struct KvGeom {
 
 // Equal split of U = tiles * KB work units (128-row weight tile x 64-wide k block) over G
 // CTAs: CTA c owns units [start(c), start(c+1)); the first `rem` CTAs own one unit more.
-// Each (CTA, tile) segment writes one [16][128] fp32 block of partial sums; the blocks of a tile
-// are numbered consecutively in CTA order: tab[tile] = {first block, number of blocks, first CTA}.
+// Each (CTA, tile) segment writes one [16][128] fp32 block of partial sums, block number
+// cta + tile: unique, because the CTA ranges are disjoint and ordered (if CTA c reaches tile
+// t + 1, CTA c + 1 starts no earlier than tile t + 1), and at most G + tiles - 1.  A tile's
+// blocks are those of CTAs owner(first unit) .. owner(last unit), consecutive numbers.
 struct StreamK {
     int U, KB, G, base, rem, tiles;
-    const int4 *tab;   // device, `tiles` entries
     __host__ __device__ int start(int c) const { return c * base + (c < rem ? c : rem); }
     __host__ __device__ int owner(int u) const {
         const int bnd = rem * (base + 1);
@@ -35,12 +36,12 @@ struct StreamK {
 
 // Where a projection left its fp32 partial sums.
 //   mode 0: base[s * split_stride + m * R + r], s < S           (SIMT kernel, S = 1)
-//   mode 1: blocks of the stream-K tensor-core kernel, located through tab
+//   mode 1: blocks of the stream-K tensor-core kernel (numbered cta + tile, see StreamK)
 struct PartView {
     const float *base;
     int mode, S, R;
     size_t split_stride;
-    const int4 *tab;
+    StreamK sk;
 };
 
 // RMSNorm statistics of the rows a projection consumed: the projection runs on x * g, and
@@ -87,8 +88,7 @@ bool pdl_enabled();
 int tc_init();                                   // once per process; 0 on success
 bool tc_shape_ok(int R, int K);
 bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows);
-StreamK tc_plan(int R, int K, int n_sm);              // tab left null
-int tc_fill_table(const StreamK &sk, int4 *host_tab);  // host table of sk.tiles entries; returns the block count
+StreamK tc_plan(int R, int K, int n_sm);
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
                     int M, int *err);
 void launch_split_rows(cudaStream_t s, const float *x, void *xs, int M, int K);
