@@ -94,11 +94,11 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_engine(wl, temperature, controller, device, n_layers=0):
+def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None):
     from paper_2406_03853_b200 import Engine
     from paper_2406_03853_b200 import binding as b
     spec_name, n_prompt, max_new, damp, _ = WORKLOADS[wl]
-    spec = synth.SPECS[spec_name].with_(damp=damp)
+    spec = synth.SPECS[spec_name].with_(damp=damp if alpha is None else alpha)
     if n_layers:
         spec = spec.with_(n_layers=n_layers, n_early=min(spec.n_early, n_layers))
     max_ctx = max(n_prompt + max_new + 16, 1024 + 32)
@@ -252,6 +252,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="13b-eesd", choices=sorted(WORKLOADS))
     ap.add_argument("--temperature", type=float, default=0.0)
+    ap.add_argument("--alpha", type=float, default=None,
+                    help="scale of the upper layers' output projections (draft/target agreement): 0.05 high, "
+                         "0.2 medium (default), 0.5 low acceptance")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-pass", type=int, default=0, metavar="M",
                     help="only run verify passes of M rows (and draft steps) inside a cudaProfilerStart/Stop "
@@ -277,7 +280,8 @@ def main():
     from paper_2406_03853_b200 import binding as b
     if args.profile_pass:
         return profile_pass(args, device)
-    eng, spec, n_prompt, max_new = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device)
+    from paper_2406_03853_b200 import report
+    eng, spec, n_prompt, max_new = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha)
     prompt = synth.prompt_tokens(synth.SEED, n_prompt, spec.vocab).numpy()
     u = {k: v.numpy() for k, v in synth.generate_uniforms(eng.cfg.max_ctx, 1 << 20).items()}
 
@@ -309,11 +313,8 @@ def main():
     clk = clocks.stop()
     barrier()
     launches = eng.launch_count() - launches0
-    t = torch.tensor([dec_ms], dtype=torch.float64, device=device)
-    if dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dec_ms = float(t.item())
-    value = world * args.steps * max_new / (dec_ms / 1e3)
+    # independent replicas: the job's time is the slowest rank's, its work the sum over ranks
+    dec_ms, _, value = report.aggregate_replicas(dec_ms, args.steps * max_new, dist, device)
 
     # ---- e2e: eesd_generate with host buffers (prefill and all copies inside the timed region)
     e2e_ms = 0.0
@@ -324,11 +325,7 @@ def main():
         e1.record()
         torch.cuda.synchronize()
         e2e_ms += e0.elapsed_time(e1)
-    t = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
-    if dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item())
-    e2e_value = world * args.steps * max_new / (e2e_ms / 1e3)
+    e2e_ms, _, e2e_value = report.aggregate_replicas(e2e_ms, args.steps * max_new, dist, device)
     greedy = args.temperature == 0.0
     h2d = n_prompt * 4 + (0 if greedy else 3 * eng.cfg.max_ctx * 4)
     d2h = sum(12 + 4 * k for k, _, _ in trace2)
@@ -345,14 +342,19 @@ def main():
     kv_len = WORKLOADS[args.workload][4]
     bv, bd = pass_bytes(spec, kv_len)
     vp = {}
-    for M in (1, M_typ, 16):
+    for M in sorted({1, M_typ, 6, 11, 16}):   # 6 and 11: K = 5 (the paper's best fixed K for 13B) and K = k_cap
         ms = time_verify_pass(eng, spec, kv_len, M)
         vp[f"M{M}"] = {"ms": round(ms, 4), "gbs": round(bv / (ms * 1e-3) / 1e9, 1),
                        "frac_of_measured_copy": round(bv / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
                        "frac_of_8tbs": round(bv / (ms * 1e-3) / 1e9 / 8000.0, 4)}
     s0 = stats[-1]
-    v_d = s0["accepted"] / max(1, s0["drafted"])
-    r_d = s0["accepted"] / max(1, s0["emitted"])
+    qual = report.run_quality(s0["drafted"], s0["accepted"], s0["emitted"])
+    v_d, r_d = qual["v_d"], qual["r_d"]
+    # the paper's cost model (its appendix on the harmonic mean) with the measured draft-step and
+    # verify-pass times: what speed-up over one-token-per-pass decoding these v_d, r_d predict
+    t_d = s0["ms_draft"] / max(1, s0["drafted"])
+    t_t = vp["M1"]["ms"]
+    model_speedup = report.modelled_speedup(v_d, r_d, t_d / t_t) if v_d > 0 else None
     line = {
         "metric": "eesd_decode_tokens_per_s", "value": round(value, 3), "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dec_ms / args.steps, 3),
@@ -372,7 +374,10 @@ def main():
         "verify_pass": {"kv_len": kv_len, "bytes": bv, **vp},
         "draft_step_bytes": bd,
         "round_stats": {"rounds": s0["rounds"], "mean_k": round(mean_k, 3), "v_d": round(v_d, 4), "r_d": round(r_d, 4),
-                        "hm": round(2 * v_d * r_d / max(1e-9, v_d + r_d), 4),
+                        "hm": round(qual["hm"], 2),
+                        "ms_per_draft_step": round(t_d, 4), "autoregressive_tokens_per_s": round(1e3 / t_t, 2),
+                        "speedup_vs_autoregressive": round(value / world / (1e3 / t_t), 4),
+                        "speedup_by_cost_model": None if model_speedup is None else round(model_speedup, 4),
                         "ms_draft": round(s0["ms_draft"], 3), "ms_verify": round(s0["ms_verify"], 3),
                         "ms_prefill_e2e": round(st2.ms_prefill, 3)},
     }

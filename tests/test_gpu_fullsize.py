@@ -1,0 +1,60 @@
+"""Full-size properties on the LLaMA-2-13B-shaped model (all 40 layers, the launch
+configuration the benchmark times), where the CPU oracle cannot follow in seconds:
+
+* losslessness: greedy EESD emits the target model's own greedy sequence, so the tokens must
+  not depend on the draft lengths (K = 1, 4, 10 and a Thompson-sampling run);
+* sampled outputs against the oracle: the embedding row and the first decoder layer of a
+  verify pass, checked on the rows the oracle computes from the same weights.
+"""
+import numpy as np
+import pytest
+import torch
+
+import eesd_synth as synth
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def engine13b():
+    import bench
+    from paper_2406_03853_b200 import binding as b
+    eng, spec, _, _ = bench.build_engine("13b-eesd", 0.0, b.CTRL_FIXED_K, torch.device("cuda:0"))
+    yield eng, spec
+    eng.close()
+
+
+def test_greedy_tokens_do_not_depend_on_draft_length(engine13b):
+    eng, spec = engine13b
+    prompt = synth.prompt_tokens(synth.SEED, 200, spec.vocab).numpy()
+    outs, accepted = [], []
+    for ks in ([1] * 64, [4] * 64, [10] * 64, [3, 7, 1, 10, 2, 5] * 12):
+        out, trace, st = eng.generate(prompt, 40, k_schedule=ks)
+        outs.append(out)
+        accepted.append(st.accepted)
+        assert st.emitted == 40 and all(0 <= a <= k for k, a, _ in trace)
+    for o in outs[1:]:
+        np.testing.assert_array_equal(o, outs[0])
+    assert max(accepted) > 0   # drafts are really accepted somewhere, so the equality is not vacuous
+
+
+def test_first_layer_of_a_full_size_pass_matches_oracle(engine13b):
+    eng, spec = engine13b
+    from tests.helpers import oracle_from_spec
+    m = oracle_from_spec(spec, max_ctx=64, n_layers=1, device="cuda")
+    prompt = synth.prompt_tokens(11, 9, spec.vocab).numpy()
+    m.target_rows(prompt[:-1], 0, want_logits=False)
+    eng.prefill(prompt)
+    cap = eng.capture_hidden(True)
+    rows = np.concatenate([prompt[-1:], synth.prompt_tokens(12, 5, spec.vocab).numpy()]).astype(np.int32)
+    eng.verify_only(rows)
+    torch.cuda.synchronize()
+    hid, _ = m.target_rows(rows, len(prompt) - 1, want_hidden=True, want_logits=False)
+    got = cap[:2, :len(rows)].cpu().numpy()
+    assert np.abs(got[0] - hid[0]).max() == 0.0          # embedding rows: exact
+    assert np.abs(got[1] - hid[1]).max() < 2e-2          # after layer 1, bf16 tolerance
+    eng.capture_hidden(False)
+    # the pass left finite logits of the right shape behind
+    lg = eng.logits(0, len(rows))
+    assert torch.isfinite(lg).all() and lg.shape == (len(rows), spec.vocab)
