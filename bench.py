@@ -36,7 +36,7 @@ import eesd_synth as synth
 
 WORKLOADS = {
     # name: (spec, prompt length, generated tokens, damp alpha, kv cache length for the verify-pass leg)
-    "13b-eesd": ("13b", 512, 256, 0.2, 1024),
+    "13b-eesd": ("13b", 512, 256, 0.05, 1024),   # alpha 0.05: acceptance statistics of the paper's 13B rows
     "70b-eesd": ("70b", 1024, 256, 0.2, 1024),
     "tiny-eesd": ("tiny", 32, 64, 0.1, 64),
 }
