@@ -101,8 +101,10 @@ typedef struct eesd_sizes {
 
 /* Caller-owned device memory.  kv_pool holds P = floor(kv_bytes / kv_page_bytes) pages laid
  * out [slot 0..L][page 0..P-1][K|V][H_kv] blocks of page_tokens * D elements; slot L is the
- * early-exit layer's cache.  A value block is [page_tokens][D]; a key block is stored
- * transposed, [D/2][page_tokens][2] (pairs of adjacent dimensions, one column per token).
+ * early-exit layer's cache.  A key block is stored transposed, [D/2][page_tokens][2] (pairs of
+ * adjacent dimensions, one column per token); a value block is [page_tokens][D] with the 16-byte
+ * chunks of token t's row permuted (chunk c sits at c ^ (t & 7)).  Both are internal formats:
+ * the library writes and reads the pool itself.
  * The workspace must be zero-filled by the caller before eesd_init. */
 typedef struct eesd_buffers {
     void *weights;   size_t weights_bytes;

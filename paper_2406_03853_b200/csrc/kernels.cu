@@ -243,6 +243,7 @@ int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float 
 }
 
 // ------------------------------------------------------------------------------------ RoPE + KV append
+template <typename AT> __device__ __forceinline__ int v_elem(int pos, int e);
 // grid (heads, M), block D/2: one thread per rotation pair.
 template <typename AT>
 __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeom kv, const float2 *rope, float *q,
@@ -273,8 +274,9 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
     }
     AT *blk = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)kv.page_tokens * D;
     if (isV) {
-        blk[(size_t)(pos % kv.page_tokens) * D + 2 * i] = from_f<AT>(a);
-        blk[(size_t)(pos % kv.page_tokens) * D + 2 * i + 1] = from_f<AT>(b);
+        AT *dst = blk + (size_t)(pos % kv.page_tokens) * D + v_elem<AT>(pos, 2 * i);
+        dst[0] = from_f<AT>(a);
+        dst[1] = from_f<AT>(b);
     } else {   // keys are cached transposed per page: pair i of a position at [i][pos % page_tokens]
         AT *dst = blk + ((size_t)i * kv.page_tokens + (pos % kv.page_tokens)) * 2;
         dst[0] = from_f<AT>(a);
@@ -327,7 +329,16 @@ template <> struct KPair<float> {
     __device__ __forceinline__ static void get(T w, float &a, float &b) { a = w.x; b = w.y; }
 };
 
-template <typename AT, int D, int RB>   // RB: (head, row) pairs per batch: 8, 16 or 32
+// Values are cached [page_tokens][D] with the 16-byte chunks of a token's row permuted by the
+// low three bits of its position (chunk c of token t sits at c ^ (t & 7)): eight consecutive
+// tokens then hold any given chunk in eight different bank groups, so the transposing matrix
+// loads of the PV product are conflict-free.  Index of element e of a row at position pos:
+template <typename AT> __device__ __forceinline__ int v_elem(int pos, int e) {
+    constexpr int CPV = 16 / (int)sizeof(AT);
+    return (((e / CPV) ^ (pos & 7)) * CPV) + (e % CPV);
+}
+
+template <typename AT, int D, int RB>   // RB: (head, row) pairs per block: 8, 16 or 32
 __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, const float2 *__restrict__ rope, KvGeom kv,
                                                    float *__restrict__ apart, unsigned int *tickets,
                                                    float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
@@ -353,13 +364,14 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     float *s_l = s_m + RB;
     float *s_rstd = s_l + RB;                                    // [kMaxRows]
     uint64_t *bar = reinterpret_cast<uint64_t *>(s_rstd + kMaxRows);
-    float *wgt = reinterpret_cast<float *>(bar + 2);             // [rows][n_split] merge weights
+    float *wgt = reinterpret_cast<float *>(bar + 2);             // [RB][n_split] merge weights
     // per-slice (maximum, sum) pairs live behind the outputs: [H][16][kMaxSlices]
     float2 *ml = reinterpret_cast<float2 *>(apart + (size_t)H * kMaxSlices * kMaxRows * D);
     __shared__ int s_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
+    const int r0 = blockIdx.z * RB;          // first (head, row) pair of this block's batch
     const int ctx_len = pos0 + M;
     const int n_pages = (ctx_len + PT - 1) / PT;
     const int page_lo = sp * pps, page_hi = min(n_pages, page_lo + pps);
@@ -393,23 +405,51 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
         }
     }
     pdl_wait();   // from here on the QKV projection's partial sums are read
+    // One round of global loads: the RMSNorm statistics (threads 0..M-1) and the raw partial
+    // sums of this block's queries and of the new keys / values that fall into its slice; they
+    // are scaled, rotated and rounded after the barrier, while the cached slice is still arriving.
     if (tid < M) s_rstd[tid] = row_rstd(rs, tid);
-    __syncthreads();
-    // new keys / values that fall into this slice: rotate and round now (while the cached slice
-    // is still arriving); they go into the tile and the cache once the slice has landed
     constexpr int kNewPerThread = kMaxRows * D / 256;
     const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
     const int n_new = max(0, p_last - p_first) * D;
-    AT new_a[kNewPerThread], new_b[kNewPerThread];
+    float raw_a[kNewPerThread], raw_b[kNewPerThread];
 #pragma unroll
     for (int it = 0; it < kNewPerThread; it++) {
         const int idx = tid + it * 256;   // -> (position, K pair | V pair)
         if (idx < n_new) {
             const int pn = idx / D, w = idx - pn * D;
-            const int pos = p_first + pn, m = pos - pos0;
+            const int m = p_first + pn - pos0;
             const int isV = w >= HALF, i = isV ? w - HALF : w;
             const int col = (H + (isV ? kv.Hkv : 0) + kh) * D + 2 * i;
-            float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
+            raw_a[it] = part_gather(pv, m, col);
+            raw_b[it] = part_gather(pv, m, col + 1);
+        }
+    }
+    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
+    const int nb = min(RB, rows - r0);
+    constexpr int kQPerThread = RB * HALF / 256;
+    float qraw_a[kQPerThread], qraw_b[kQPerThread];
+#pragma unroll
+    for (int it = 0; it < kQPerThread; it++) {
+        const int idx = tid + it * 256;
+        if (idx < nb * HALF) {
+            const int rl = idx / HALF, i = idx - rl * HALF;
+            const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
+            const int col = (kh * group + g) * D + 2 * i;
+            qraw_a[it] = part_gather(pv, m, col);
+            qraw_b[it] = part_gather(pv, m, col + 1);
+        }
+    }
+    __syncthreads();
+    AT new_a[kNewPerThread], new_b[kNewPerThread];
+#pragma unroll
+    for (int it = 0; it < kNewPerThread; it++) {
+        const int idx = tid + it * 256;
+        if (idx < n_new) {
+            const int pn = idx / D, w = idx - pn * D;
+            const int pos = p_first + pn, m = pos - pos0;
+            const int isV = w >= HALF, i = isV ? w - HALF : w;
+            float a = raw_a[it] * s_rstd[m], b = raw_b[it] * s_rstd[m];
             if (!isV) {
                 const float2 cs = rope[(size_t)pos * HALF + i];
                 const float ra = a * cs.x - b * cs.y, rb = a * cs.y + b * cs.x;
@@ -419,13 +459,14 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             new_b[it] = from_f<AT>(b);
         }
     }
-    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
-    auto load_queries = [&](int r0, int nb) {   // rotated, pre-scaled queries of a batch
-        for (int idx = tid; idx < nb * HALF; idx += 256) {
+    {   // rotated, pre-scaled queries of this block's batch
+#pragma unroll
+        for (int it = 0; it < kQPerThread; it++) {
+            const int idx = tid + it * 256;
+            if (idx >= nb * HALF) continue;
             const int rl = idx / HALF, i = idx - rl * HALF;
-            const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
-            const int col = (kh * group + g) * D + 2 * i;
-            const float a = part_gather(pv, m, col) * s_rstd[m], b = part_gather(pv, m, col + 1) * s_rstd[m];
+            const int m = (r0 + rl) % M;
+            const float a = qraw_a[it] * s_rstd[m], b = qraw_b[it] * s_rstd[m];
             const float2 cs = rope[(size_t)(pos0 + m) * HALF + i];
             const float qa = (a * cs.x - b * cs.y) * scale, qb = (a * cs.y + b * cs.x) * scale;
             if (kTC) {
@@ -437,8 +478,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                 sq[rl * HALF + i] = make_float2(qa, qb);
             }
         }
-    };
-    load_queries(0, min(RB, rows));
+    }
     if (warp == 0) {   // wait for the cached slice (bounded); the other warps park at the barrier below
         bool ok = false;
         for (uint32_t i = 0; i < (1u << 24) && !ok; i++) {
@@ -461,15 +501,19 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const int page = kv.page_table[pos / PT];
             if (page < 0 || page >= kv.n_pages_total) { atomicOr(err, kErrBadPage); continue; }
             AT *blk = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)PT * D;
+            const bool append = blockIdx.z == 0;   // every batch needs the row in its tile; one block writes the cache
             if (isV) {
-                AT *tile = sV + (size_t)j * D + 2 * i;
+                const int e = v_elem<AT>(pos, 2 * i);
+                AT *tile = sV + (size_t)j * D + e;
                 tile[0] = new_a[it]; tile[1] = new_b[it];
-                blk[(size_t)(pos % PT) * D + 2 * i] = new_a[it];
-                blk[(size_t)(pos % PT) * D + 2 * i + 1] = new_b[it];
+                if (append) {
+                    blk[(size_t)(pos % PT) * D + e] = new_a[it];
+                    blk[(size_t)(pos % PT) * D + e + 1] = new_b[it];
+                }
             } else {   // keys: pair i of position pos at [i][pos % PT] of the page block
                 const KP w2 = KPair<AT>::make(new_a[it], new_b[it]);
                 sK[(size_t)(j / PT) * PT * HALF + (size_t)i * PT + (j % PT)] = w2;
-                reinterpret_cast<KP *>(blk)[(size_t)i * PT + (pos % PT)] = w2;
+                if (append) reinterpret_cast<KP *>(blk)[(size_t)i * PT + (pos % PT)] = w2;
             }
         }
     }
@@ -480,12 +524,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     }
     __syncthreads();
 
-    for (int r0 = 0; r0 < rows; r0 += RB) {
-        const int nb = min(RB, rows - r0);
-        if (r0 > 0) {
-            load_queries(r0, nb);
-            __syncthreads();
-        }
+    {
         if constexpr (kTC) {
             // scores on the tensor cores: S = Q K^T as m16n8k16 products, Q = hi + lo (two bf16
             // terms, exact products, fp32 accumulation).  The transposed key tile yields the
@@ -613,7 +652,8 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                     for (int x = 0; x < D / 64; x++) {
                         const int d0 = (warp + 8 * x) * 8;
                         uint32_t b0, b1;
-                        const uint32_t addr = smem_addr(sV + (size_t)(k0 + (lane & 15)) * D + d0);
+                        const int jr = k0 + (lane & 15);
+                        const uint32_t addr = smem_addr(sV + (size_t)jr * D + v_elem<AT>(jr, d0));
                         asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
                         asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                                      : "+f"(c[x][0]), "+f"(c[x][1]), "+f"(c[x][2]), "+f"(c[x][3])
@@ -648,19 +688,8 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             if (warp < nb) {
                 for (int j = 0; j < npos; j++) {
                     float v[DPL];
-                    if (sizeof(AT) == 2) {
-                        if (DPL == 4) {
-                            const uint2 w = *reinterpret_cast<const uint2 *>(sV + (size_t)j * D + lane * 4);
-                            v[0] = __uint_as_float(w.x << 16); v[1] = __uint_as_float(w.x & 0xFFFF0000u);
-                            v[2 % DPL] = __uint_as_float(w.y << 16); v[3 % DPL] = __uint_as_float(w.y & 0xFFFF0000u);
-                        } else {
-                            const uint32_t w = *reinterpret_cast<const uint32_t *>(sV + (size_t)j * D + lane * 2);
-                            v[0] = __uint_as_float(w << 16); v[1] = __uint_as_float(w & 0xFFFF0000u);
-                        }
-                    } else {
 #pragma unroll
-                        for (int e = 0; e < DPL; e++) v[e] = to_f(sV[(size_t)j * D + lane * DPL + e]);
-                    }
+                    for (int e = 0; e < DPL; e++) v[e] = to_f(sV[(size_t)j * D + v_elem<AT>(j, lane * DPL + e)]);
 #pragma unroll
                     for (int i = 0; i < RPW; i++) {
                         const int rl = min(warp + 8 * i, RB - 1);
@@ -689,15 +718,17 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const unsigned int prev = atomicAdd(&tickets[kh], 1u);
+        unsigned int *tk = tickets + kh * gridDim.z + blockIdx.z;   // one counter per (KV head, batch)
+        const unsigned int prev = atomicAdd(tk, 1u);
         s_last = (prev == (unsigned int)n_split - 1);
-        if (s_last) tickets[kh] = 0;
+        if (s_last) *tk = 0;
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
     const size_t sstride = (size_t)kMaxRows * D;
-    for (int rho = warp; rho < rows; rho += 8) {   // normalised weight of every (pair, slice): one round trip
+    for (int rl = warp; rl < nb; rl += 8) {   // normalised weight of every (pair, slice): one round trip
+        const int rho = r0 + rl;
         const int g = rho / M, m = rho - g * M, h = kh * group + g;
         const float2 *src = ml + ((size_t)h * kMaxRows + m) * kMaxSlices;
         const float2 none = make_float2(-INFINITY, 0.f);
@@ -707,15 +738,15 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
         const float w0 = (v0.x == -INFINITY) ? 0.f : expf(v0.x - mx), w1 = (v1.x == -INFINITY) ? 0.f : expf(v1.x - mx);
         const float den = warp_sum(fmaf(w0, v0.y, w1 * v1.y));   // fixed butterfly over the lanes
         const float inv = den > 0.f ? 1.0f / den : 0.f;
-        if (lane < n_split) wgt[rho * n_split + lane] = w0 * inv;
-        if (lane + 32 < n_split) wgt[rho * n_split + lane + 32] = w1 * inv;
+        if (lane < n_split) wgt[rl * n_split + lane] = w0 * inv;
+        if (lane + 32 < n_split) wgt[rl * n_split + lane + 32] = w1 * inv;
     }
     __syncthreads();
-    for (int idx = tid; idx < rows * D; idx += 256) {
-        const int rho = idx / D, dd = idx - rho * D;
+    for (int idx = tid; idx < nb * D; idx += 256) {
+        const int rl = idx / D, dd = idx - rl * D, rho = r0 + rl;
         const int g = rho / M, m = rho - g * M, h = kh * group + g;
         const float *src = apart + ((size_t)h * n_split * kMaxRows + m) * D + dd;
-        const float *wr = wgt + rho * n_split;
+        const float *wr = wgt + rl * n_split;
         float o = 0.f;
         for (int s2 = 0; s2 < n_split; s2 += 8) {   // eight independent loads in flight, added in slice order
             float a[8];
@@ -733,7 +764,7 @@ static size_t attn_smem_bytes(int es, int D, int RB, int cap, int rows, int n_sp
     const int rbp = RB < 16 ? 16 : RB;
     const size_t sq_words = es == 2 ? (size_t)2 * rbp * (D / 2 + 4) : (size_t)RB * D;
     return (size_t)2 * cap * D * es + sq_words * 4 + (size_t)RB * (cap + 12) * 4 + 2 * RB * 4 + kMaxRows * 4 + 16 +
-           (size_t)rows * n_split * 4 + 16;
+           (size_t)RB * n_split * 4 + 16;
 }
 
 template <typename AT, int D, int RB>
@@ -747,7 +778,7 @@ static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, 
         cudaFuncSetAttribute(attn_kernel<AT, D, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
         configured = 227 * 1024 - 1024;
     }
-    launch_k(attn_kernel<AT, D, RB>, dim3(kv.Hkv, n_split), dim3(256), smem, s, pdl_enabled(), pv, rs, rope, kv, apart,
+    launch_k(attn_kernel<AT, D, RB>, dim3(kv.Hkv, n_split, (rows + RB - 1) / RB), dim3(256), smem, s, pdl_enabled(), pv, rs, rope, kv, apart,
              tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err);
 }
 
@@ -764,11 +795,11 @@ static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs
 }
 
 // slices of the cached context: pages per block and number of blocks per KV head
-int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_sm, int max_splits, int *pps_out) {
+int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out) {
     const int n_pages = (ctx_len + page_tokens - 1) / page_tokens;
     const int cap = kAttnPos / page_tokens > 0 ? kAttnPos / page_tokens : 1;   // pages one block can hold
     // one wave: about two blocks per SM in flight, so aim for H_kv * n_split <= 2 * n_sm
-    int want = 2 * n_sm / Hkv;
+    int want = 2 * n_sm / (Hkv * n_batches);
     if (want < 1) want = 1;
     if (want > max_splits) want = max_splits;
     int pps = (n_pages + want - 1) / want;
@@ -785,7 +816,8 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
                       int M, int pos0, int H, int n_sm, int max_splits, int *err) {
     int pps;
-    const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, n_sm, max_splits, &pps);
+    const int rows = (H / kv.Hkv) * M, rb = rows <= 8 ? 8 : rows <= 16 ? 16 : 32;
+    const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb, n_sm, max_splits, &pps);
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (dtype == 0) {
         if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);

@@ -14,7 +14,8 @@ struct IntList16 { int32_t v[16]; };
 // geometry of one paged KV cache slot
 struct KvGeom {
     void *slot_base;            // first byte of the slot: [page][K|V][H_kv] blocks of page_tokens * D
-                                // elements; K block [D/2][page_tokens][2], V block [page_tokens][D]
+                                // elements; K block [D/2][page_tokens][2], V block [page_tokens][D] with the 16-byte
+                                // chunks of token t's row permuted (chunk c at c ^ (t & 7))
     const int32_t *page_table;  // logical page -> physical page
     int Hkv, D, page_tokens, n_pages_total;
 };
@@ -74,7 +75,8 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 // QKV projection's partial sums (scaled by rs, rotated), the new keys/values are appended to
 // the paged cache, every KV head's cached slice is read once, and the slices are merged into
 // attn_out (fp32 [M][H*D], may be null) and attn_split (two bf16 terms, may be null).
-// apart: H * max_splits * 16 * (D + 2) floats; tickets: H_kv zero-initialised counters.
+// apart: H * max_splits * 16 * (D + 2) floats; tickets: zero-initialised counters, one per
+// (KV head, batch of 32 (head, row) pairs): at most H_kv * 4.
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
                       int M, int pos0, int H, int n_sm, int max_splits, int *err);
