@@ -12,58 +12,53 @@ namespace eesd {
 
 typedef __nv_bfloat16 bf16;
 
-// sum of the partial results of output element (m, r), in a fixed order
-__device__ __forceinline__ float part_gather(const PartView &pv, int m, int r) {
-    float v = 0.f;
+// Sum of the partial results of output elements (m, r .. r + N - 1), N = 1, 2 or 4 (r % N == 0,
+// so they share a weight tile), in a fixed order.  All loads of up to four blocks are issued
+// before the first add, so a gather costs one round trip to L2, not one per block.
+template <int N> struct PartVec;
+template <> struct PartVec<1> { typedef float T; };
+template <> struct PartVec<2> { typedef float2 T; };
+template <> struct PartVec<4> { typedef float4 T; };
+__device__ __forceinline__ void vadd(float &a, float b) { a += b; }
+__device__ __forceinline__ void vadd(float2 &a, float2 b) { a.x += b.x; a.y += b.y; }
+__device__ __forceinline__ void vadd(float4 &a, float4 b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+
+template <int N>
+__device__ __forceinline__ typename PartVec<N>::T part_gather_n(const PartView &pv, int m, int r) {
+    typedef typename PartVec<N>::T V;
+    V v = V();
     if (pv.mode == 0) {
-        for (int s = 0; s < pv.S; s++) v += pv.base[(size_t)s * pv.split_stride + (size_t)m * pv.R + r];
+        for (int s = 0; s < pv.S; s++)
+            vadd(v, *reinterpret_cast<const V *>(pv.base + (size_t)s * pv.split_stride + (size_t)m * pv.R + r));
     } else {
         const int t = r >> 7;
         const int c0 = pv.sk.owner(t * pv.sk.KB), n = pv.sk.owner((t + 1) * pv.sk.KB - 1) - c0 + 1;
-        const float *p = pv.base + ((size_t)(c0 + t) * kMaxRows + m) * 128 + (r & 127);
-        int i = 0;
-        for (; i + 2 <= n; i += 2) {   // two loads in flight, added in block order
-            const float a = __ldcg(p + (size_t)i * kMaxRows * 128), b = __ldcg(p + (size_t)(i + 1) * kMaxRows * 128);
-            v += a;
-            v += b;
-        }
-        if (i < n) v += __ldcg(p + (size_t)i * kMaxRows * 128);
+        constexpr size_t BS = (size_t)kMaxRows * 128;   // floats per block
+        const V *p = reinterpret_cast<const V *>(pv.base + ((size_t)(c0 + t) * kMaxRows + m) * 128 + (r & 127));
+        const V *p1 = reinterpret_cast<const V *>(reinterpret_cast<const float *>(p) + BS);
+        const V *p2 = reinterpret_cast<const V *>(reinterpret_cast<const float *>(p) + 2 * BS);
+        const V *p3 = reinterpret_cast<const V *>(reinterpret_cast<const float *>(p) + 3 * BS);
+        const V a0 = __ldcg(p);
+        const V a1 = n > 1 ? __ldcg(p1) : V();
+        const V a2 = n > 2 ? __ldcg(p2) : V();
+        const V a3 = n > 3 ? __ldcg(p3) : V();
+        v = a0;
+        vadd(v, a1);
+        vadd(v, a2);
+        vadd(v, a3);
+        for (int i = 4; i < n; i++)
+            vadd(v, __ldcg(reinterpret_cast<const V *>(reinterpret_cast<const float *>(p) + (size_t)i * BS)));
     }
     return v;
 }
+__device__ __forceinline__ float part_gather(const PartView &pv, int m, int r) { return part_gather_n<1>(pv, m, r); }
+__device__ __forceinline__ float4 part_gather4(const PartView &pv, int m, int r) { return part_gather_n<4>(pv, m, r); }
 
 __device__ __forceinline__ float row_rstd(const RowScale &rs, int m) {
     if (!rs.ssq) return 1.0f;
     float t = 0.f;
     for (int b = 0; b < rs.nblk; b++) t += rs.ssq[m * kSsqBlocks + b];
     return 1.0f / sqrtf(t * rs.inv_d + rs.eps);
-}
-
-// the same for four consecutive outputs r..r+3 (r % 4 == 0, so they share a weight tile)
-__device__ __forceinline__ float4 part_gather4(const PartView &pv, int m, int r) {
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (pv.mode == 0) {
-        for (int s = 0; s < pv.S; s++) {
-            const float4 t = *reinterpret_cast<const float4 *>(pv.base + (size_t)s * pv.split_stride + (size_t)m * pv.R + r);
-            v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
-        }
-    } else {
-        const int t = r >> 7;
-        const int c0 = pv.sk.owner(t * pv.sk.KB), n = pv.sk.owner((t + 1) * pv.sk.KB - 1) - c0 + 1;
-        const float *p = pv.base + ((size_t)(c0 + t) * kMaxRows + m) * 128 + (r & 127);
-        int i = 0;
-        for (; i + 2 <= n; i += 2) {
-            const float4 a = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)i * kMaxRows * 128));
-            const float4 b = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)(i + 1) * kMaxRows * 128));
-            v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
-            v.x += b.x; v.y += b.y; v.z += b.z; v.w += b.w;
-        }
-        if (i < n) {
-            const float4 a = __ldcg(reinterpret_cast<const float4 *>(p + (size_t)i * kMaxRows * 128));
-            v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
-        }
-    }
-    return v;
 }
 
 bool pdl_enabled() {
@@ -254,7 +249,8 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
     pdl_trigger();
     pdl_wait();
     const float rstd = row_rstd(rs, m);
-    float a = part_gather(pv, m, col) * rstd, b = part_gather(pv, m, col + 1) * rstd;
+    const float2 pr = part_gather_n<2>(pv, m, col);
+    float a = pr.x * rstd, b = pr.y * rstd;
     const int pos = pos0 + m;
     if (hh < H + kv.Hkv) {
         float2 cs = rope[(size_t)pos * (D / 2) + i];
@@ -413,16 +409,19 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
     const int n_new = max(0, p_last - p_first) * D;
     float raw_a[kNewPerThread], raw_b[kNewPerThread];
+    int new_page[kNewPerThread];
 #pragma unroll
     for (int it = 0; it < kNewPerThread; it++) {
         const int idx = tid + it * 256;   // -> (position, K pair | V pair)
         if (idx < n_new) {
             const int pn = idx / D, w = idx - pn * D;
             const int m = p_first + pn - pos0;
+            new_page[it] = kv.page_table[(p_first + pn) / PT];
             const int isV = w >= HALF, i = isV ? w - HALF : w;
             const int col = (H + (isV ? kv.Hkv : 0) + kh) * D + 2 * i;
-            raw_a[it] = part_gather(pv, m, col);
-            raw_b[it] = part_gather(pv, m, col + 1);
+            const float2 pr = part_gather_n<2>(pv, m, col);
+            raw_a[it] = pr.x;
+            raw_b[it] = pr.y;
         }
     }
     const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
@@ -436,8 +435,9 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const int rl = idx / HALF, i = idx - rl * HALF;
             const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
             const int col = (kh * group + g) * D + 2 * i;
-            qraw_a[it] = part_gather(pv, m, col);
-            qraw_b[it] = part_gather(pv, m, col + 1);
+            const float2 pr = part_gather_n<2>(pv, m, col);
+            qraw_a[it] = pr.x;
+            qraw_b[it] = pr.y;
         }
     }
     __syncthreads();
@@ -498,7 +498,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const int pn = idx / D, w = idx - pn * D;
             const int pos = p_first + pn, j = pos - lo;
             const int isV = w >= HALF, i = isV ? w - HALF : w;
-            const int page = kv.page_table[pos / PT];
+            const int page = new_page[it];
             if (page < 0 || page >= kv.n_pages_total) { atomicOr(err, kErrBadPage); continue; }
             AT *blk = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)PT * D;
             const bool append = blockIdx.z == 0;   // every batch needs the row in its tile; one block writes the cache
