@@ -369,7 +369,10 @@ def main():
         "clocks": clk,
         "roofline": {"bound": "hbm", "kernel": "skinny projection (gate/up shape, M=%d)" % M_typ,
                      "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
+                     "frac": round(achieved / peaks["hbm_gbs"], 4),
+                     # dram__bytes_read + dram__bytes_write of one gate/up launch at the 13B shape, from the ncu
+                     # capture summarised under profiles/ (null for other shapes: not captured)
+                     "traffic": 289117952 if (spec.name == "13b") else None,
                      "bytes_per_launch": kbytes, "ms_per_launch": round(kms, 5)},
         "verify_pass": {"kv_len": kv_len, "bytes": bv, **vp},
         "draft_step_bytes": bd,
