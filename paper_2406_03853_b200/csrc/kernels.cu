@@ -51,6 +51,27 @@ __device__ __forceinline__ typename PartVec<N>::T part_gather_n(const PartView &
     }
     return v;
 }
+// same for the stream-K layout when the tile's {first block, block count} is already known
+template <int N>
+__device__ __forceinline__ typename PartVec<N>::T part_gather_blocks(const PartView &pv, int2 tb, int m, int r) {
+    typedef typename PartVec<N>::T V;
+    constexpr size_t BS = (size_t)kMaxRows * 128;
+    const float *p = pv.base + ((size_t)tb.x * kMaxRows + m) * 128 + (r & 127);
+    const V a0 = __ldcg(reinterpret_cast<const V *>(p));
+    const V a1 = tb.y > 1 ? __ldcg(reinterpret_cast<const V *>(p + BS)) : V();
+    const V a2 = tb.y > 2 ? __ldcg(reinterpret_cast<const V *>(p + 2 * BS)) : V();
+    const V a3 = tb.y > 3 ? __ldcg(reinterpret_cast<const V *>(p + 3 * BS)) : V();
+    V v = a0;
+    vadd(v, a1);
+    vadd(v, a2);
+    vadd(v, a3);
+    for (int i = 4; i < tb.y; i++) vadd(v, __ldcg(reinterpret_cast<const V *>(p + (size_t)i * BS)));
+    return v;
+}
+__device__ __forceinline__ int2 tile_blocks(const StreamK &sk, int t) {
+    const int c0 = sk.owner(t * sk.KB);
+    return make_int2(c0 + t, sk.owner((t + 1) * sk.KB - 1) - c0 + 1);
+}
 __device__ __forceinline__ float part_gather(const PartView &pv, int m, int r) { return part_gather_n<1>(pv, m, r); }
 __device__ __forceinline__ float4 part_gather4(const PartView &pv, int m, int r) { return part_gather_n<4>(pv, m, r); }
 
@@ -400,6 +421,21 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                          ::"r"(smem_addr(sV + (size_t)(pg - page_lo) * PT * D)), "l"(src + v_off), "r"(blk_bytes), "r"(smem_addr(bar)) : "memory");
         }
     }
+    // where the partial sums this block needs live (block numbers of the query tiles of its
+    // batch and of its key and value tile): integer arithmetic only, done before the wait
+    __shared__ int2 s_tb[40];
+    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
+    const int nb = min(RB, rows - r0);
+    const int tq0 = ((kh * group + r0 / M) * D) >> 7, tq1 = ((kh * group + (r0 + nb - 1) / M) * D + D - 1) >> 7;
+    const int nq = tq1 - tq0 + 1, tk = ((H + kh) * D) >> 7, tv = ((H + kv.Hkv + kh) * D) >> 7;
+    if (pv.mode == 1 && tid < nq + 2 && tid < 40)
+        s_tb[tid] = tile_blocks(pv.sk, tid < nq ? tq0 + tid : (tid == nq ? tk : tv));
+    __syncthreads();
+    auto gather_pair = [&](int m, int col) -> float2 {
+        if (pv.mode == 0) return part_gather_n<2>(pv, m, col);
+        const int t = col >> 7;
+        return part_gather_blocks<2>(pv, s_tb[t == tk ? nq : (t == tv ? nq + 1 : t - tq0)], m, col);
+    };
     pdl_wait();   // from here on the QKV projection's partial sums are read
     // One round of global loads: the RMSNorm statistics (threads 0..M-1) and the raw partial
     // sums of this block's queries and of the new keys / values that fall into its slice; they
@@ -419,13 +455,11 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             new_page[it] = kv.page_table[(p_first + pn) / PT];
             const int isV = w >= HALF, i = isV ? w - HALF : w;
             const int col = (H + (isV ? kv.Hkv : 0) + kh) * D + 2 * i;
-            const float2 pr = part_gather_n<2>(pv, m, col);
+            const float2 pr = gather_pair(m, col);
             raw_a[it] = pr.x;
             raw_b[it] = pr.y;
         }
     }
-    const int rows = group * M;   // (head in group, new row) pairs; rho = g * M + m
-    const int nb = min(RB, rows - r0);
     constexpr int kQPerThread = RB * HALF / 256;
     float qraw_a[kQPerThread], qraw_b[kQPerThread];
 #pragma unroll
@@ -435,7 +469,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const int rl = idx / HALF, i = idx - rl * HALF;
             const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
             const int col = (kh * group + g) * D + 2 * i;
-            const float2 pr = part_gather_n<2>(pv, m, col);
+            const float2 pr = gather_pair(m, col);
             qraw_a[it] = pr.x;
             qraw_b[it] = pr.y;
         }
