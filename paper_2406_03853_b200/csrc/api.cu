@@ -50,7 +50,7 @@ int check_config(const eesd_config *c) {
 }
 
 struct Workspace {
-    size_t x, xn, q, attn, h, xs[3], ssq, tickets, tabs, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
+    size_t x, xn, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
         accept, total;
 };
 
@@ -61,7 +61,6 @@ constexpr int kMaxSm = 256;      // upper bound on CTAs of the persistent projec
 
 Workspace carve(const eesd_config *c) {
     Workspace w;
-    const size_t es = c->dtype == EESD_F32 ? 4 : 2;
     const size_t R = EESD_MAX_ROWS;
     const size_t qd = (size_t)c->n_heads * c->head_dim, kvd = (size_t)c->n_kv_heads * c->head_dim;
     size_t maxR = qd + 2 * kvd;
@@ -72,7 +71,6 @@ Workspace carve(const eesd_config *c) {
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     w.x = take(R * c->d_model * 4);
     w.xn = take(R * c->d_model * 4);
-    w.q = take(R * qd * 4);
     w.attn = take(R * qd * 4);
     w.h = take(R * (size_t)c->ffn_dim * 4);
     // the same three activation matrices as two bf16 terms, [32][K] (tensor-core path)
@@ -81,7 +79,6 @@ Workspace carve(const eesd_config *c) {
     w.xs[X_FFN] = take(2 * R * (size_t)c->ffn_dim * 2);
     w.ssq = take((size_t)EESD_MAX_ROWS * kSsqBlocks * 4);
     w.tickets = take(1024 * 4);
-    w.tabs = take((size_t)P_COUNT * (maxR / 128 + 1) * sizeof(int4));
     {   // partial sums: SIMT layout [splits][16][maxR], or stream-K blocks of the widest projection
         size_t part_floats = (size_t)kPartSplits * R * maxR;
         const size_t sk_floats = (maxR / 128 + (size_t)kMaxSm) * R * 128;  // blocks <= tiles + CTAs
@@ -116,7 +113,7 @@ struct eesd_ctx {
     cudaStream_t stream;
     size_t es;
     // device pointers
-    float *x, *xn, *q, *attn, *h, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
+    float *x, *xn, *attn, *h, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
     void *accept_scratch;
     void *xs[3];                 // bf16 hi/lo copies of xn, attn, h
     float *ssq;                  // RMSNorm partial sums of squares of the rows in xn / xs[X_NORM]
@@ -249,8 +246,7 @@ void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const fl
     const eesd_config &f = c->cfg;
     const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim, d = f.d_model, F = f.ffn_dim;
     cudaStream_t s = c->stream;
-    const RowScale rs = norm_scale(c), none = {nullptr, 0, 0.f, 0.f};
-    (void)none;
+    const RowScale rs = norm_scale(c);
     PartView pv = run_proj(c, w.wqkv, &w.m_qkv, P_QKV, X_NORM, M, qd + 2 * kvd, d);
     launch_attention(s, f.dtype, pv, rs, c->rope, kv_geom(c, slot), c->apart, c->tickets, c->use_tc ? nullptr : c->attn,
                      c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, c->err);
@@ -528,7 +524,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->slot_bytes = (size_t)c->n_pages_total * 2 * cfg->n_kv_heads * cfg->page_tokens * cfg->head_dim * c->es;
     Workspace w = carve(cfg);
     char *ws = (char *)b->workspace;
-    c->x = (float *)(ws + w.x); c->xn = (float *)(ws + w.xn); c->q = (float *)(ws + w.q); c->attn = (float *)(ws + w.attn);
+    c->x = (float *)(ws + w.x); c->xn = (float *)(ws + w.xn); c->attn = (float *)(ws + w.attn);
     c->h = (float *)(ws + w.h); c->part = (float *)(ws + w.part); c->apart = (float *)(ws + w.apart);
     c->logits_p = (float *)(ws + w.logits_p); c->logits_q = (float *)(ws + w.logits_q);
     c->rope = (float2 *)(ws + w.rope); c->page_table = (int32_t *)(ws + w.page_table);

@@ -1,0 +1,130 @@
+"""GPU edge cases against the oracle: shortest and longest rounds, page boundaries, context
+limits, grouped-query and wide-head variants, bf16 models on both projection paths, the step
+API with explicit uniforms, and launch without programmatic dependent launch."""
+import os
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+import eesd_synth as synth
+import oracle
+from tests.helpers import engine_from_spec, oracle_from_spec
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_one_token_prompt_one_new_token_and_longest_round():
+    spec = synth.TINY
+    eng = engine_from_spec(spec, max_ctx=96, k_cap=15, fixed_k=15, page_tokens=8)
+    m = oracle_from_spec(spec, 96)
+    out, trace, st = eng.generate(np.array([7], np.int32), 1)
+    ref, rtrace, _ = m.generate(np.array([7], np.int32), 1, k_cap=15, fixed_k=15)
+    np.testing.assert_array_equal(out, ref)
+    assert trace == rtrace and trace[0][0] == 15          # a 15-token draft, 16-row verify pass
+    prompt = synth.prompt_tokens(2, 9, spec.vocab).numpy()
+    out, trace, _ = eng.generate(prompt, 40)
+    ref, rtrace, _ = oracle_from_spec(spec, 96).generate(prompt, 40, k_cap=15, fixed_k=15)
+    np.testing.assert_array_equal(out, ref)
+    assert trace == rtrace
+    eng.close()
+
+
+def test_context_limit_is_an_error_not_a_fault():
+    from paper_2406_03853_b200 import EesdError
+    spec = synth.TINY
+    eng = engine_from_spec(spec, max_ctx=48, k_cap=10, fixed_k=4, page_tokens=8)
+    prompt = synth.prompt_tokens(3, 30, spec.vocab).numpy()
+    with pytest.raises(EesdError) as e:
+        eng.generate(prompt, 30)                           # 30 + 30 + 1 > max_ctx
+    assert e.value.status == -5
+    out, _, _ = eng.generate(prompt, 17)                   # exactly fits: 30 + 17 + 1 = 48
+    ref, _, _ = oracle_from_spec(spec, 48).generate(prompt, 17, fixed_k=4)
+    np.testing.assert_array_equal(out, ref)
+    eng.prefill(prompt)
+    eng.draft(10)
+    with pytest.raises(EesdError):
+        eng.draft(1)                                       # beyond k_cap within one round
+    eng.close()
+    with pytest.raises(EesdError):
+        engine_from_spec(spec, max_ctx=64, kv_pages=3)     # page pool smaller than max_ctx needs
+
+
+@pytest.mark.parametrize("variant", ["gqa", "wide_head", "bf16_simt", "bf16_tensor_core"])
+def test_model_variants_match_oracle(variant):
+    base = synth.TINY
+    spec = {
+        "gqa": base.with_(n_kv_heads=2),
+        "wide_head": base.with_(n_heads=2, n_kv_heads=1, head_dim=128),
+        "bf16_simt": base.with_(dtype="bf16"),                       # 2F = 1376 is not a multiple of 128
+        "bf16_tensor_core": base.with_(dtype="bf16", ffn_dim=640),   # every projection tile-aligned
+    }[variant]
+    eng = engine_from_spec(spec, max_ctx=96, k_cap=10, fixed_k=3, page_tokens=16)
+    m = oracle_from_spec(spec, 96)
+    prompt = synth.prompt_tokens(4, 37, spec.vocab).numpy()
+    m.target_rows(prompt[:-1], 0, want_logits=False)
+    eng.prefill(prompt)
+    cap = eng.capture_hidden(True)
+    rows = np.concatenate([prompt[-1:], synth.prompt_tokens(5, 6, spec.vocab).numpy()]).astype(np.int32)
+    eng.verify_only(rows)
+    torch.cuda.synchronize()
+    hid, lg = m.target_rows(rows, 36, want_hidden=True)
+    tol = 2e-5 if spec.dtype == "f32" else 2e-2
+    assert np.abs(cap[:spec.n_layers + 1, :7].cpu().numpy() - hid).max() < tol
+    assert np.abs(eng.logits(0, 7).cpu().numpy() - lg).max() < tol
+    eng.capture_hidden(False)
+    if spec.dtype == "f32":
+        out, trace, _ = eng.generate(prompt, 24)
+        ref, rtrace, _ = oracle_from_spec(spec, 96).generate(prompt, 24, fixed_k=3)
+        np.testing.assert_array_equal(out, ref)
+        assert trace == rtrace
+    eng.close()
+
+
+def test_step_api_with_explicit_uniforms_equals_oracle_rounds():
+    spec = synth.TINY
+    eng = engine_from_spec(spec, max_ctx=128, k_cap=10, temperature=1.0, page_tokens=8)
+    m = oracle_from_spec(spec, 128)
+    prompt = synth.prompt_tokens(6, 15, spec.vocab).numpy()   # ends one short of a page boundary
+    eng.prefill(prompt)
+    m.target_rows(prompt[:-1], 0, want_logits=False)
+    ctx = list(prompt)
+    for rnd, K in enumerate([3, 1, 10, 2, 6]):
+        ud = synth.uniforms(100 + rnd, 1, K).numpy()
+        ua = synth.uniforms(100 + rnd, 2, K).numpy()
+        ur = float(synth.uniforms(100 + rnd, 3, 1).numpy()[0])
+        toks = np.concatenate([eng.draft(K - K // 2, ud[:K - K // 2]), eng.draft(K // 2, ud[K - K // 2:])]) if K > 1 \
+            else eng.draft(1, ud)                              # drafting may be interleaved call by call
+        T = len(ctx)
+        xs, ql = [ctx[-1]], []
+        for i in range(K):
+            lgq = m.draft_row(xs[-1], T - 1 + i)
+            ql.append(lgq)
+            xs.append(oracle.sample_logits(lgq, 1.0, float(ud[i])))
+        np.testing.assert_array_equal(toks, xs[1:])
+        n_acc, y = eng.verify_accept(ua, ur)
+        _, pl = m.target_rows(np.array(xs, np.int32), T - 1)
+        assert (n_acc, y) == oracle.accept_resample(pl, np.stack(ql), xs[1:], ua, ur, 1.0)
+        ctx += xs[1:1 + n_acc] + [y]
+        n_tok, pages = eng.context_len()
+        assert n_tok == len(ctx) and pages == (n_tok - 1 + 7) // 8
+    eng.close()
+
+
+def test_same_tokens_without_programmatic_dependent_launch():
+    code = ("import sys; sys.path.insert(0, %r); import numpy as np, eesd_synth as synth;"
+            "from tests.helpers import engine_from_spec;"
+            "spec = synth.TINY.with_(dtype='bf16', ffn_dim=640);"
+            "eng = engine_from_spec(spec, max_ctx=96, fixed_k=4);"
+            "out, _, _ = eng.generate(synth.prompt_tokens(8, 20, 1024).numpy(), 32);"
+            "print(' '.join(map(str, out)))") % ROOT
+    outs = []
+    for env_extra in ({}, {"EESD_NO_PDL": "1"}):
+        env = dict(os.environ, **env_extra)
+        r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env, timeout=600)
+        assert r.returncode == 0, r.stderr[-2000:]
+        outs.append(r.stdout.strip().splitlines()[-1])
+    assert outs[0] == outs[1] and len(outs[0].split()) == 32
