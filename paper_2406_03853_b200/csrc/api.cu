@@ -51,13 +51,28 @@ int check_config(const eesd_config *c) {
 
 struct Workspace {
     size_t x, xn, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
-        accept, total;
+        accept, wx, wout, wxs[3], wssq, wtok, total;
 };
 
 constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
 constexpr int kAttnSplits = 64;  // most KV slices per head in attention
 constexpr int kIntSlots = 64;    // small device integer area
 constexpr int kMaxSm = 256;      // upper bound on CTAs of the persistent projection kernel
+constexpr int kPrefillRows = 512; // most prompt rows per pass of the wide (prompt) path
+
+bool tc_shapes_ok(const eesd_config *c) {
+    const int qd = c->n_heads * c->head_dim, kvd = c->n_kv_heads * c->head_dim;
+    return c->dtype == EESD_BF16 && tc_shape_ok(qd + 2 * kvd, c->d_model) && tc_shape_ok(c->d_model, qd) &&
+           tc_shape_ok(2 * c->ffn_dim, c->d_model) && tc_shape_ok(c->d_model, c->ffn_dim) &&
+           tc_shape_ok(2 * kvd, c->d_model) && tc_shape_ok(c->vocab, c->d_model);
+}
+
+// rows the wide path's buffers hold (a multiple of 128); 0 when the model cannot use it
+int prefill_rows(const eesd_config *c) {
+    if (!tc_shapes_ok(c)) return 0;
+    const int need = (c->max_ctx - 1 + 127) / 128 * 128;
+    return need < kPrefillRows ? need : kPrefillRows;
+}
 
 Workspace carve(const eesd_config *c) {
     Workspace w;
@@ -95,6 +110,21 @@ Workspace carve(const eesd_config *c) {
     w.u_stage = take(64 * 4);
     w.err = take(16);
     w.accept = take(accept_scratch_bytes(1, EESD_MAX_ROWS));
+    w.wx = w.wout = w.wssq = w.wtok = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
+    if (const size_t P = (size_t)prefill_rows(c)) {
+        // prompt path: residual stream, one projection result, the three activation matrices as
+        // two bf16 terms ([chunk of 16][hi | lo][16][K]), RMSNorm statistics, token ids
+        size_t wideR = qd + 2 * kvd;
+        if ((size_t)2 * c->ffn_dim > wideR) wideR = (size_t)2 * c->ffn_dim;
+        if ((size_t)c->d_model > wideR) wideR = c->d_model;
+        w.wx = take(P * c->d_model * 4);
+        w.wout = take(P * wideR * 4);
+        w.wxs[X_NORM] = take(2 * P * (size_t)c->d_model * 2);
+        w.wxs[X_ATTN] = take(2 * P * qd * 2);
+        w.wxs[X_FFN] = take(2 * P * (size_t)c->ffn_dim * 2);
+        w.wssq = take(P * kSsqBlocks * 4);
+        w.wtok = take(P * 4);
+    }
     w.total = o;
     return w;
 }
@@ -119,6 +149,12 @@ struct eesd_ctx {
     float *ssq;                  // RMSNorm partial sums of squares of the rows in xn / xs[X_NORM]
     unsigned int *tickets;       // arrival counters of the attention merge
     CUtensorMap m_x[3];
+    // prompt (wide) path: up to wide_rows prompt rows per pass
+    int wide_rows;
+    float *wx, *wout, *wssq;
+    void *wxs[3];
+    int32_t *wtok;
+    CUtensorMap m_wx[3];
     CUtensorMap m_exit_kv, m_lm_head, m_exit_head;
     bool use_tc;
     int n_sm;
@@ -249,7 +285,7 @@ void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const fl
     const RowScale rs = norm_scale(c);
     PartView pv = run_proj(c, w.wqkv, &w.m_qkv, P_QKV, X_NORM, M, qd + 2 * kvd, d);
     launch_attention(s, f.dtype, pv, rs, c->rope, kv_geom(c, slot), c->apart, c->tickets, c->use_tc ? nullptr : c->attn,
-                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, c->err);
+                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, true, c->err);
     pv = run_proj(c, w.wo, &w.m_o, P_O, X_ATTN, M, d, qd);
     run_resid(c, &pv, w.g_ffn, nullptr, M);
     pv = run_proj(c, w.wgu, &w.m_gu, P_GU, X_NORM, M, 2 * F, d);
@@ -291,6 +327,65 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
         PartView pv = run_proj(c, c->lm_head, &c->m_lm_head, P_HEAD, X_NORM, M, f.vocab, d);
         launch_reduce_partials(s, pv, norm_scale(c), c->logits_p, M, f.vocab);
         c->launches += 1;
+    }
+    return check_launch(c);
+}
+
+// Prompt pass (wide path): the target model on Mtot <= wide_rows prompt rows at positions
+// p0.., no logits.  Projections run on the wide tensor-core kernel (weights cross HBM once
+// per pass); attention runs chunk by chunk (16 rows), each chunk appending its keys / values
+// before the next one reads them; the exit layer's keys / values follow layer N.
+int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
+    const eesd_config &f = c->cfg;
+    cudaStream_t s = c->stream;
+    const int L = f.n_layers, d = f.d_model, F = f.ffn_dim, H = f.n_heads;
+    const int qd = H * f.head_dim, kvd = f.n_kv_heads * f.head_dim;
+    CU(c, cudaMemcpyAsync(c->wtok, prompt_host + p0, (size_t)Mtot * 4, cudaMemcpyHostToDevice, s));
+    RowScale rs = norm_scale(c);
+    rs.ssq = c->wssq;
+    auto proj = [&](const CUtensorMap &mW, int which, int R, int K) {
+        launch_gemm_wide(s, mW, c->m_wx[which], c->wout, R, K, Mtot, c->n_sm, c->err);
+        c->launches++;
+        PartView pv = {};
+        pv.base = c->wout; pv.mode = 0; pv.S = 1; pv.R = R; pv.split_stride = 0;
+        return pv;
+    };
+    auto resid = [&](const PartView *pv, const float *g) {
+        launch_resid(s, c->wx, pv, g, nullptr, c->wxs[X_NORM], nullptr, c->wssq, Mtot, d);
+        c->launches++;
+    };
+    launch_embed(s, f.dtype, c->wtok, c->embed, c->wx, nullptr, Mtot, d, f.vocab, c->err);
+    c->launches++;
+    resid(nullptr, c->layers[0].g_attn);
+    for (int l = 0; l < L; l++) {
+        const LayerW &w = c->layers[l];
+        const bool exit_here = (l == f.n_early - 1);
+        const float *g_after = exit_here ? c->layers[L].g_attn : (l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
+        PartView pv = proj(w.m_qkv, X_NORM, qd + 2 * kvd, d);
+        for (int c0 = 0; c0 < Mtot; c0 += EESD_MAX_ROWS) {
+            const int m = Mtot - c0 < EESD_MAX_ROWS ? Mtot - c0 : EESD_MAX_ROWS;
+            PartView cpv = pv;
+            cpv.base = pv.base + (size_t)c0 * pv.R;
+            RowScale crs = rs;
+            crs.ssq = rs.ssq + (size_t)c0 * kSsqBlocks;
+            char *dst = (char *)c->wxs[X_ATTN] + (size_t)(c0 / EESD_MAX_ROWS) * 2 * EESD_MAX_ROWS * qd * 2;
+            launch_attention(s, f.dtype, cpv, crs, c->rope, kv_geom(c, l), c->apart, c->tickets, nullptr, dst, m, p0 + c0, H,
+                             c->n_sm, kAttnSplits, c0 == 0, c->err);
+            c->launches++;
+        }
+        pv = proj(w.m_o, X_ATTN, d, qd);
+        resid(&pv, w.g_ffn);
+        pv = proj(w.m_gu, X_NORM, 2 * F, d);
+        launch_swiglu(s, pv, rs, nullptr, c->wxs[X_FFN], Mtot, F);
+        c->launches++;
+        pv = proj(w.m_d, X_FFN, d, F);
+        resid(&pv, g_after);
+        if (exit_here) {
+            pv = proj(c->m_exit_kv, X_NORM, 2 * kvd, d);
+            launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, L), c->rope, nullptr, true, c->err);
+            c->launches++;
+            resid(nullptr, l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
+        }
     }
     return check_launch(c);
 }
@@ -368,7 +463,16 @@ int prefill_impl(eesd_ctx *c, const int32_t *prompt, int n_prompt) {
     reset_sequence(c);
     int st = ensure_pages(c, n_prompt);
     if (st) return st;
-    for (int p = 0; p < n_prompt - 1; p += EESD_MAX_ROWS) {
+    int p = 0;
+    // long prompts: wide passes (hidden-state capture holds 16 rows per layer, so it keeps the row-chunk path)
+    while (c->wide_rows > 0 && !c->capture && n_prompt - 1 - p > EESD_MAX_ROWS) {
+        int M = n_prompt - 1 - p;
+        if (M > c->wide_rows) M = c->wide_rows;
+        st = run_prompt_pass(c, prompt, p, M);
+        if (st) return st;
+        p += M;
+    }
+    for (; p < n_prompt - 1; p += EESD_MAX_ROWS) {
         int M = n_prompt - 1 - p;
         if (M > EESD_MAX_ROWS) M = EESD_MAX_ROWS;
         st = set_device_ints(c, kRowTok, prompt + p, M);
@@ -540,9 +644,8 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         if (c->n_sm > kMaxSm) c->n_sm = kMaxSm;
     }
     const int qd_ = cfg->n_heads * cfg->head_dim, kvd_ = cfg->n_kv_heads * cfg->head_dim;
-    c->use_tc = cfg->dtype == EESD_BF16 && tc_shape_ok(qd_ + 2 * kvd_, cfg->d_model) && tc_shape_ok(cfg->d_model, qd_) &&
-                tc_shape_ok(2 * cfg->ffn_dim, cfg->d_model) && tc_shape_ok(cfg->d_model, cfg->ffn_dim) &&
-                tc_shape_ok(2 * kvd_, cfg->d_model) && tc_shape_ok(cfg->vocab, cfg->d_model) && tc_init() == 0;
+    c->use_tc = tc_shapes_ok(cfg) && tc_init() == 0;
+    c->wide_rows = c->use_tc ? prefill_rows(cfg) : 0;
     const char *wb = (const char *)b->weights;
     c->layers.resize(cfg->n_layers + 1);
     for (int l = 0; l <= cfg->n_layers; l++) {
@@ -568,6 +671,15 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         ok = ok && tc_make_map(&c->m_exit_kv, c->layers[cfg->n_layers].wqkv + (size_t)qd_ * d * 2, 2 * kvd_, d, 128);
         ok = ok && tc_make_map(&c->m_lm_head, c->lm_head, cfg->vocab, d, 128);
         ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128);
+        if (c->wide_rows) {
+            c->wx = (float *)(ws + w.wx); c->wout = (float *)(ws + w.wout); c->wssq = (float *)(ws + w.wssq);
+            c->wtok = (int32_t *)(ws + w.wtok);
+            const int ks[3] = {d, qd_, F};
+            for (int i = 0; i < 3; i++) {
+                c->wxs[i] = ws + w.wxs[i];
+                ok = ok && tc_make_map_rows(&c->m_wx[i], c->wxs[i], ks[i], c->wide_rows / EESD_MAX_ROWS);
+            }
+        }
         // work split of every projection shape
         const int shapes[P_COUNT][2] = {{qd_ + 2 * kvd_, d}, {d, qd_}, {2 * F, d}, {d, F}, {2 * kvd_, d}, {cfg->vocab, d}};
         for (int i = 0; i < P_COUNT; i++) c->plan[i] = tc_plan(shapes[i][0], shapes[i][1], c->n_sm);

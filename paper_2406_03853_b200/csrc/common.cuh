@@ -98,11 +98,14 @@ inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
     cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-// writes v as two bf16 terms into a [2 * kMaxRows][K] matrix: row m gets hi, row kMaxRows + m gets lo
+// writes v as two bf16 terms into a [chunk][hi | lo][kMaxRows][K] matrix: token row m belongs to
+// chunk m / kMaxRows; its hi term goes to row m % kMaxRows of the chunk's first half, its lo
+// term to the same row of the second half (one chunk, [2 * kMaxRows][K], in a decode pass)
 __device__ __forceinline__ void store_split(__nv_bfloat16 *xs, int m, size_t K, size_t i, float v) {
     const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-    xs[(size_t)m * K + i] = hi;
-    xs[(size_t)(kMaxRows + m) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    const size_t row = (size_t)(m / kMaxRows) * (2 * kMaxRows) + (size_t)(m % kMaxRows);
+    xs[row * K + i] = hi;
+    xs[(row + kMaxRows) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
 }  // namespace eesd

@@ -39,6 +39,10 @@ constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 2
 constexpr int THREADS = 192;  // warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA issuer
 constexpr uint32_t TMEM_COLS = 64;   // two 128 x 32 fp32 accumulators
 constexpr uint32_t SPIN_LIMIT = 1u << 25;  // polls of a barrier before a wait gives up (about a second)
+// The tensor core adds into its fp32 accumulator with truncation, so a long chain of MMAs
+// drifts towards zero.  Chains are therefore cut after KSEG k blocks (4 * KSEG MMAs): the
+// epilogue warps drain the accumulator and carry the sum in registers with IEEE fp32 adds.
+constexpr int KSEG = 16;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -215,55 +219,66 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     } else if (warp == 5) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            int it = 0, seg = 0;
+            int it = 0, sub = 0;   // sub: accumulator chains started so far (buffer = sub & 1)
             bool ok = true;
-            for (int u = u0; u < u1 && ok; seg++) {
+            for (int u = u0; u < u1 && ok;) {
                 const int tile = u / sk.KB;
                 const int u_end = min(u1, (tile + 1) * sk.KB);
-                const int b = seg & 1, use = seg >> 1;
-                ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_addr = tmem_base + (uint32_t)(b * BN);
-                for (int uu = u; uu < u_end; uu++, it++) {
-                    const int s = it % STAGES, round = it / STAGES;
-                    ok = mbar_wait(&full[s], round & 1, abort_flag);
+                for (int c0 = u; c0 < u_end && ok; c0 += KSEG, sub++) {
+                    const int c1 = min(u_end, c0 + KSEG);
+                    const int b = sub & 1, use = sub >> 1;
+                    ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t da = smem_desc(smem_u32(sW + s * STAGE_W));
-                    const uint64_t db = smem_desc(smem_u32(sX + s * STAGE_X));
+                    const uint32_t d_addr = tmem_base + (uint32_t)(b * BN);
+                    for (int uu = c0; uu < c1; uu++, it++) {
+                        const int s = it % STAGES, round = it / STAGES;
+                        ok = mbar_wait(&full[s], round & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t da = smem_desc(smem_u32(sW + s * STAGE_W));
+                        const uint64_t db = smem_desc(smem_u32(sX + s * STAGE_X));
 #pragma unroll
-                    for (int j = 0; j < BK / 16; j++)
-                        mma_bf16(d_addr, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), (uu > u || j > 0) ? 1u : 0u);
-                    mma_commit(&empty[s]);   // the stage may be refilled once these MMAs have read it
+                        for (int j = 0; j < BK / 16; j++)
+                            mma_bf16(d_addr, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), (uu > c0 || j > 0) ? 1u : 0u);
+                        mma_commit(&empty[s]);   // the stage may be refilled once these MMAs have read it
+                    }
+                    if (!ok) break;
+                    mma_commit(&acc_full[b]);    // chain complete
                 }
-                if (!ok) break;
-                mma_commit(&acc_full[b]);    // accumulator complete
                 u = u_end;
             }
         }
     } else {
         // ---------------------------------------------------------------- epilogue (warps 0-3)
         pdl_wait();   // the partial-sum buffer may still be read by the kernel before this one
-        int seg = 0;
+        int sub = 0;
         bool ok = true;
-        for (int u = u0; u < u1 && ok; seg++) {
+        for (int u = u0; u < u1 && ok;) {
             const int tile = u / sk.KB;
             const int u_end = min(u1, (tile + 1) * sk.KB);
-            const int b = seg & 1, use = seg >> 1;
-            ok = mbar_wait(&acc_full[b], use & 1, abort_flag, 64);
-            ok = __all_sync(0xffffffffu, ok);
+            float acc[kMaxRows];
+#pragma unroll
+            for (int m = 0; m < kMaxRows; m++) acc[m] = 0.f;
+            for (int c0 = u; c0 < u_end; c0 += KSEG, sub++) {
+                const int b = sub & 1, use = sub >> 1;
+                ok = mbar_wait(&acc_full[b], use & 1, abort_flag, 64);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * BN), r);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[b]);
+#pragma unroll
+                for (int m = 0; m < kMaxRows; m++) acc[m] += __uint_as_float(r[m]) + __uint_as_float(r[16 + m]);
+            }
             if (!ok) break;
-            tc_fence_after();
-            uint32_t r[32];
-            tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * BN), r);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[b]);
             float *dst = part + ((size_t)(cta + tile) * kMaxRows) * BM + warp * 32 + lane;
 #pragma unroll
             for (int m = 0; m < kMaxRows; m++)
-                if (m < M) dst[(size_t)m * BM] = __uint_as_float(r[m]) + __uint_as_float(r[16 + m]);
+                if (m < M) dst[(size_t)m * BM] = acc[m];
             u = u_end;
         }
     }
@@ -273,6 +288,187 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (warp == 5) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// Wide variant for prompt processing: up to 128 token rows per tile (256 operand columns: hi
+// and lo terms), the whole k range per tile, result written directly as out[m][r] (fp32).
+//
+//   * tile = (128-row weight tile, 128-row token panel); tiles are dealt round-robin with the
+//     panels of one weight tile adjacent, so CTAs running side by side share it through L2 and
+//     the weights cross HBM once per pass over all panels;
+//   * 4-stage ring of (16 KB weight tile + 32 KB token tile); the token tile is two boxes of a
+//     4-D map over the [chunk][hi|lo][16][K] activation layout (8 chunks of 16 rows each);
+//   * tcgen05.mma M = 128, N = 256, K = 16; two accumulators of 256 columns fill the tensor memory.
+constexpr int WN = 256, WROWS = 128;               // operand columns / token rows per panel
+constexpr int WSTAGES = 4;
+constexpr int WSTAGE_X = WN * BK * 2, WSTAGE_BYTES = STAGE_W + WSTAGE_X;
+constexpr int WSMEM_BYTES = WSTAGES * WSTAGE_BYTES + 1024 + 256;
+constexpr uint32_t WTMEM_COLS = 512;
+constexpr uint32_t IDESC_W = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(WN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y, int z, int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
+__device__ __forceinline__ void mma_bf16_wide(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC_W), "r"(accumulate)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+                 float *__restrict__ out, int R, int KB, int Mtot, int panels, int *err) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *sbase = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sW = sbase;
+    uint8_t *sX = sbase + WSTAGES * STAGE_W;
+    uint64_t *full = (uint64_t *)(sbase + WSTAGES * WSTAGE_BYTES);
+    uint64_t *empty = full + WSTAGES;
+    uint64_t *acc_full = empty + WSTAGES;   // [2]
+    uint64_t *acc_empty = acc_full + 2;     // [2]
+    uint32_t *tmem_slot = (uint32_t *)(acc_empty + 2);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_tiles = (R / BM) * panels;
+    const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // tiles cta, cta + G, ...
+    const int n_units = my_tiles * KB;
+    pdl_trigger();
+
+    if (tid == 0) {
+        for (int i = 0; i < WSTAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < 2; i++) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(WTMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 4) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            // unit i of this CTA -> (tile, k block)
+            auto w_load = [&](int i, int s) {
+                const int t = (int)blockIdx.x + (i / KB) * (int)gridDim.x, kb = i % KB;
+                mbar_expect_tx(&full[s], WSTAGE_BYTES);
+                tma_load_2d(sW + s * STAGE_W, &tmW, &full[s], kb * BK, (t / panels) * BM);
+            };
+            auto x_load = [&](int i, int s) {
+                const int t = (int)blockIdx.x + (i / KB) * (int)gridDim.x, kb = i % KB, chunk0 = (t % panels) * (WROWS / 16);
+                tma_load_4d(sX + s * WSTAGE_X, &tmX, &full[s], kb * BK, 0, 0, chunk0);
+                tma_load_4d(sX + s * WSTAGE_X + WSTAGE_X / 2, &tmX, &full[s], kb * BK, 0, 1, chunk0);
+            };
+            const int pre = min(n_units, WSTAGES);
+            for (int i = 0; i < pre; i++) w_load(i, i);   // weights do not depend on the previous kernel
+            pdl_wait();
+            for (int i = 0; i < pre; i++) x_load(i, i);
+            int issued = pre;
+            for (; issued < n_units; issued++) {
+                const int s = issued % WSTAGES, round = issued / WSTAGES;
+                if (!mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag)) break;
+                w_load(issued, s);
+                x_load(issued, s);
+            }
+            if (*abort_flag) {
+                const int first = issued > WSTAGES ? issued - WSTAGES : 0;
+                for (int i = first; i < issued; i++) {
+                    uint64_t *b = &full[i % WSTAGES];
+                    const uint32_t par = (uint32_t)((i / WSTAGES) & 1);
+                    for (uint32_t t = 0; t < SPIN_LIMIT && !mbar_try(b, par); t++) {}
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            int it = 0, sub = 0;
+            bool ok = true;
+            for (int seg = 0; seg < my_tiles && ok; seg++) {
+                for (int c0 = 0; c0 < KB && ok; c0 += KSEG, sub++) {
+                    const int c1 = min(KB, c0 + KSEG);
+                    const int b = sub & 1, use = sub >> 1;
+                    ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t d_addr = tmem_base + (uint32_t)(b * WN);
+                    for (int kb = c0; kb < c1; kb++, it++) {
+                        const int s = it % WSTAGES, round = it / WSTAGES;
+                        ok = mbar_wait(&full[s], round & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t da = smem_desc(smem_u32(sW + s * STAGE_W));
+                        const uint64_t db = smem_desc(smem_u32(sX + s * WSTAGE_X));
+#pragma unroll
+                        for (int j = 0; j < BK / 16; j++)
+                            mma_bf16_wide(d_addr, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), (kb > c0 || j > 0) ? 1u : 0u);
+                        mma_commit(&empty[s]);
+                    }
+                    if (!ok) break;
+                    mma_commit(&acc_full[b]);
+                }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (warps 0-3)
+        pdl_wait();   // the output buffer may still be read by the kernel before this one
+        bool ok = true;
+        int sub = 0;
+        for (int seg = 0; seg < my_tiles && ok; seg++) {
+            const int t = (int)blockIdx.x + seg * (int)gridDim.x, wt = t / panels, pn = t % panels;
+            float acc[WROWS];   // this thread's weight row against the panel's 128 token rows
+#pragma unroll
+            for (int i = 0; i < WROWS; i++) acc[i] = 0.f;
+            for (int c0 = 0; c0 < KB; c0 += KSEG, sub++) {
+                const int b = sub & 1, use = sub >> 1;
+                ok = mbar_wait(&acc_full[b], use & 1, abort_flag, 64);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * WN);
+#pragma unroll
+                for (int j = 0; j < WROWS / 32; j++) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + (uint32_t)(WROWS + j * 32), v);   // lo terms first: the smaller addend
+#pragma unroll
+                    for (int i = 0; i < 32; i++) acc[j * 32 + i] += __uint_as_float(v[i]);
+                    tmem_ld32(taddr + (uint32_t)(j * 32), v);
+#pragma unroll
+                    for (int i = 0; i < 32; i++) acc[j * 32 + i] += __uint_as_float(v[i]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[b]);
+            }
+            if (!ok) break;
+            float *dst = out + (size_t)(pn * WROWS) * R + (size_t)wt * BM + warp * 32 + lane;
+            const int rows_left = Mtot - pn * WROWS;
+#pragma unroll
+            for (int i = 0; i < WROWS; i++)
+                if (i < rows_left) dst[(size_t)i * R] = acc[i];
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && *abort_flag) atomicOr(err, kErrWaitTimeout);
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(WTMEM_COLS) : "memory");
     }
 }
 
@@ -309,6 +505,21 @@ bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box
     return r == CUDA_SUCCESS;
 }
 
+// 4-D map over token rows kept as [chunk][hi | lo][16][K] bf16; box = 64 k x 16 rows x 1 x 8 chunks
+bool tc_make_map_rows(CUtensorMap *out, const void *base, int K, int chunks) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    if (((uintptr_t)base & 15) || (K % 8)) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)K, 16, 2, (cuuint64_t)chunks};
+    cuuint64_t strides[3] = {(cuuint64_t)K * 2, (cuuint64_t)K * 2 * 16, (cuuint64_t)K * 2 * 32};
+    cuuint32_t box[4] = {(cuuint32_t)tc::BK, 16, 1, (cuuint32_t)(tc::WROWS / 16)};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides,
+                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool tc_shape_ok(int R, int K) { return R > 0 && K > 0 && R % tc::BM == 0 && K % tc::BK == 0; }
 
 StreamK tc_plan(int R, int K, int n_sm) {
@@ -327,6 +538,8 @@ int tc_init() {
     if (!done) {
         if (cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess)
             return -1;
+        if (cudaFuncSetAttribute(tc::gemm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::WSMEM_BYTES) != cudaSuccess)
+            return -1;
         if (!encode_fn()) return -1;
         done = 1;
     }
@@ -336,6 +549,14 @@ int tc_init() {
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
                     int M, int *err) {
     launch_k(tc::gemm_tc_kernel, dim3(sk.G), dim3(tc::THREADS), (size_t)tc::SMEM_BYTES, s, pdl_enabled(), mW, mX, part, sk, M, err);
+}
+
+void launch_gemm_wide(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *out, int R, int K, int Mtot,
+                      int n_sm, int *err) {
+    const int panels = (Mtot + tc::WROWS - 1) / tc::WROWS;
+    const int tiles = (R / tc::BM) * panels;
+    launch_k(tc::gemm_wide_kernel, dim3(tiles < n_sm ? tiles : n_sm), dim3(tc::THREADS), (size_t)tc::WSMEM_BYTES, s, pdl_enabled(),
+             mW, mX, out, R, K / tc::BK, Mtot, panels, err);
 }
 
 // fp32 rows -> two bf16 terms: rows 0..15 hold hi = bf16(x), rows 16..31 hold lo = bf16(x - hi)

@@ -804,7 +804,7 @@ static size_t attn_smem_bytes(int es, int D, int RB, int cap, int rows, int n_sp
 template <typename AT, int D, int RB>
 static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                         float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                        int pps, int n_split, float scale, int *err) {
+                        int pps, int n_split, float scale, bool early, int *err) {
     const int rows = (H / kv.Hkv) * M;
     const size_t smem = attn_smem_bytes((int)sizeof(AT), D, RB, pps * kv.page_tokens, rows, n_split);
     static size_t configured = 0;   // largest dynamic shared memory size enabled so far
@@ -812,16 +812,16 @@ static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, 
         cudaFuncSetAttribute(attn_kernel<AT, D, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
         configured = 227 * 1024 - 1024;
     }
-    launch_k(attn_kernel<AT, D, RB>, dim3(kv.Hkv, n_split, (rows + RB - 1) / RB), dim3(256), smem, s, pdl_enabled(), pv, rs, rope, kv, apart,
+    launch_k(attn_kernel<AT, D, RB>, dim3(kv.Hkv, n_split, (rows + RB - 1) / RB), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv, apart,
              tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err);
 }
 
 template <typename AT, int D>
 static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                           float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                          int pps, int n_split, float scale, int *err) {
+                          int pps, int n_split, float scale, bool early, int *err) {
     const int rows = (H / kv.Hkv) * M;
-#define EESD_ATTN(RB) attn_launch<AT, D, RB>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err)
+#define EESD_ATTN(RB) attn_launch<AT, D, RB>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err)
     if (rows <= 8) EESD_ATTN(8);
     else if (rows <= 16) EESD_ATTN(16);
     else EESD_ATTN(32);
@@ -848,17 +848,17 @@ int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n
 
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
-                      int M, int pos0, int H, int n_sm, int max_splits, int *err) {
+                      int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err) {
     int pps;
     const int rows = (H / kv.Hkv) * M, rb = rows <= 8 ? 8 : rows <= 16 ? 16 : 32;
     const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb, n_sm, max_splits, &pps);
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (dtype == 0) {
-        if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);
-        else attn_dispatch<float, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);
+        if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err);
+        else attn_dispatch<float, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err);
     } else {
-        if (kv.D == 64) attn_dispatch<bf16, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);
-        else attn_dispatch<bf16, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, err);
+        if (kv.D == 64) attn_dispatch<bf16, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err);
+        else attn_dispatch<bf16, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err);
     }
 }
 

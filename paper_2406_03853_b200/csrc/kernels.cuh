@@ -77,9 +77,11 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 // attn_out (fp32 [M][H*D], may be null) and attn_split (two bf16 terms, may be null).
 // apart: H * max_splits * 16 * (D + 2) floats; tickets: zero-initialised counters, one per
 // (KV head, batch of 32 (head, row) pairs): at most H_kv * 4.
+// early: the kernel may start (and read cached rows) while the kernel before it still runs;
+// must be false when that kernel appends rows to the same cache slot.
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
-                      int M, int pos0, int H, int n_sm, int max_splits, int *err);
+                      int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err);
 void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F);
 void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R);
 // programmatic dependent launch (kernels start early and wait on-device for their producer):
@@ -93,6 +95,11 @@ bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box
 StreamK tc_plan(int R, int K, int n_sm);
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
                     int M, int *err);
+// wide projection for prompt processing: out[m][r] (fp32, row stride R) for m < Mtot rows kept
+// as [chunk of 16][hi | lo][16][K] bf16 (mX from tc_make_map_rows); R % 128 == 0, K % 64 == 0
+bool tc_make_map_rows(CUtensorMap *out, const void *base, int K, int chunks);
+void launch_gemm_wide(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *out, int R, int K, int Mtot,
+                      int n_sm, int *err);
 void launch_split_rows(cudaStream_t s, const float *x, void *xs, int M, int K);
 
 // acceptance / sampling (accept.cu)

@@ -128,3 +128,36 @@ def test_same_tokens_without_programmatic_dependent_launch():
         assert r.returncode == 0, r.stderr[-2000:]
         outs.append(r.stdout.strip().splitlines()[-1])
     assert outs[0] == outs[1] and len(outs[0].split()) == 32
+
+
+def test_wide_prompt_pass_matches_row_chunks_and_oracle():
+    """Prompts longer than 16 rows go through the wide projection kernel (128-row panels); the
+    cache it leaves must equal, up to summation order, the one built 16 rows at a time, and the
+    next pass must match the oracle."""
+    spec = synth.TINY.with_(dtype="bf16", ffn_dim=640, n_layers=3)
+    n_prompt = 300                                            # 299 rows: two full panels and a ragged one
+    prompt = synth.prompt_tokens(9, n_prompt, spec.vocab).numpy()
+    wide = engine_from_spec(spec, max_ctx=384, k_cap=10, fixed_k=3, page_tokens=16)
+    rows = engine_from_spec(spec, max_ctx=384, k_cap=10, fixed_k=3, page_tokens=16)
+    rows.capture_hidden(True)                                 # capture keeps the 16-row path
+    n0 = wide.launch_count()
+    wide.prefill(prompt)
+    n_wide = wide.launch_count() - n0
+    n0 = rows.launch_count()
+    rows.prefill(prompt)
+    assert n_wide < (rows.launch_count() - n0) // 2
+    torch.cuda.synchronize()
+    a = wide.kv_pool.view(torch.bfloat16).float()
+    b = rows.kv_pool.view(torch.bfloat16).float()
+    assert (a != 0).sum() == (b != 0).sum() > 0
+    assert (a - b).abs().max().item() < 2e-2
+    assert ((a - b).abs() > 1e-3).float().mean().item() < 1e-3   # bf16 rounding flips only
+    m = oracle_from_spec(spec, 384)
+    m.target_rows(prompt[:-1], 0, want_logits=False)
+    new = np.concatenate([prompt[-1:], synth.prompt_tokens(10, 4, spec.vocab).numpy()]).astype(np.int32)
+    _, lg = m.target_rows(new, n_prompt - 1)
+    for eng in (wide, rows):
+        eng.verify_only(new)
+        torch.cuda.synchronize()
+        assert np.abs(eng.logits(0, 5).cpu().numpy() - lg).max() < 2e-2
+    wide.close(); rows.close()
