@@ -325,6 +325,7 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 // head (an arrival counter, no waiting) merges the slices in index order.
 constexpr int kAttnPos = 192;     // most positions per block
 constexpr int kMaxSlices = 64;    // most slices per head (layout of the per-slice maxima and sums)
+constexpr int kRows16 = 24;       // up to this many (head, row) pairs per KV head: batches of 16, beyond: of 32
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -761,36 +762,56 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     if (!s_last) return;
     __threadfence();
     const size_t sstride = (size_t)kMaxRows * D;
-    for (int rl = warp; rl < nb; rl += 8) {   // normalised weight of every (pair, slice): one round trip
-        const int rho = r0 + rl;
-        const int g = rho / M, m = rho - g * M, h = kh * group + g;
-        const float2 *src = ml + ((size_t)h * kMaxRows + m) * kMaxSlices;
+    {   // normalised weight of every (pair, slice); a warp's rows are loaded together: one round trip
+        constexpr int RPW = RB / 8;
         const float2 none = make_float2(-INFINITY, 0.f);
-        const float2 v0 = lane < n_split ? __ldcg(src + lane) : none;
-        const float2 v1 = lane + 32 < n_split ? __ldcg(src + lane + 32) : none;
-        const float mx = warp_max(fmaxf(v0.x, v1.x));
-        const float w0 = (v0.x == -INFINITY) ? 0.f : expf(v0.x - mx), w1 = (v1.x == -INFINITY) ? 0.f : expf(v1.x - mx);
-        const float den = warp_sum(fmaf(w0, v0.y, w1 * v1.y));   // fixed butterfly over the lanes
-        const float inv = den > 0.f ? 1.0f / den : 0.f;
-        if (lane < n_split) wgt[rl * n_split + lane] = w0 * inv;
-        if (lane + 32 < n_split) wgt[rl * n_split + lane + 32] = w1 * inv;
+        float2 v0[RPW], v1[RPW];
+#pragma unroll
+        for (int i = 0; i < RPW; i++) {
+            const int rl = warp + 8 * i, rho = r0 + min(rl, nb - 1);
+            const int g = rho / M, m = rho - g * M, h = kh * group + g;
+            const float2 *src = ml + ((size_t)h * kMaxRows + m) * kMaxSlices;
+            v0[i] = (rl < nb && lane < n_split) ? __ldcg(src + lane) : none;
+            v1[i] = (rl < nb && lane + 32 < n_split) ? __ldcg(src + lane + 32) : none;
+        }
+#pragma unroll
+        for (int i = 0; i < RPW; i++) {
+            const int rl = warp + 8 * i;
+            const float mx = warp_max(fmaxf(v0[i].x, v1[i].x));
+            const float w0 = (v0[i].x == -INFINITY) ? 0.f : expf(v0[i].x - mx), w1 = (v1[i].x == -INFINITY) ? 0.f : expf(v1[i].x - mx);
+            const float den = warp_sum(fmaf(w0, v0[i].y, w1 * v1[i].y));   // fixed butterfly over the lanes
+            const float inv = den > 0.f ? 1.0f / den : 0.f;
+            if (rl < nb) {
+                if (lane < n_split) wgt[rl * n_split + lane] = w0 * inv;
+                if (lane + 32 < n_split) wgt[rl * n_split + lane + 32] = w1 * inv;
+            }
+        }
     }
     __syncthreads();
-    for (int idx = tid; idx < nb * D; idx += 256) {
-        const int rl = idx / D, dd = idx - rl * D, rho = r0 + rl;
+    for (int idx = tid; idx < nb * (D / 4); idx += 256) {   // four output dimensions per item
+        const int rl = idx / (D / 4), dd = (idx - rl * (D / 4)) * 4, rho = r0 + rl;
         const int g = rho / M, m = rho - g * M, h = kh * group + g;
         const float *src = apart + ((size_t)h * n_split * kMaxRows + m) * D + dd;
         const float *wr = wgt + rl * n_split;
-        float o = 0.f;
-        for (int s2 = 0; s2 < n_split; s2 += 8) {   // eight independent loads in flight, added in slice order
-            float a[8];
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s2 = 0; s2 < n_split; s2 += 16) {   // sixteen slices in flight, added in slice order
+            float4 a[16];
 #pragma unroll
-            for (int u = 0; u < 8; u++) a[u] = __ldcg(src + (size_t)min(s2 + u, n_split - 1) * sstride);
+            for (int u = 0; u < 16; u++)
+                a[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)min(s2 + u, n_split - 1) * sstride));
 #pragma unroll
-            for (int u = 0; u < 8; u++) o = fmaf(s2 + u < n_split ? wr[s2 + u] : 0.f, a[u], o);
+            for (int u = 0; u < 16; u++) {
+                const float w = s2 + u < n_split ? wr[s2 + u] : 0.f;
+                o.x = fmaf(w, a[u].x, o.x); o.y = fmaf(w, a[u].y, o.y);
+                o.z = fmaf(w, a[u].z, o.z); o.w = fmaf(w, a[u].w, o.w);
+            }
         }
-        if (attn_out) attn_out[(size_t)m * H * D + (size_t)h * D + dd] = o;
-        if (attn_split) store_split(attn_split, m, (size_t)H * D, (size_t)h * D + dd, o);
+        const size_t col = (size_t)h * D + dd;
+        if (attn_out) *reinterpret_cast<float4 *>(attn_out + (size_t)m * H * D + col) = o;
+        if (attn_split) {
+            store_split(attn_split, m, (size_t)H * D, col, o.x); store_split(attn_split, m, (size_t)H * D, col + 1, o.y);
+            store_split(attn_split, m, (size_t)H * D, col + 2, o.z); store_split(attn_split, m, (size_t)H * D, col + 3, o.w);
+        }
     }
 }
 
@@ -823,7 +844,7 @@ static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs
     const int rows = (H / kv.Hkv) * M;
 #define EESD_ATTN(RB) attn_launch<AT, D, RB>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err)
     if (rows <= 8) EESD_ATTN(8);
-    else if (rows <= 16) EESD_ATTN(16);
+    else if (rows <= kRows16) EESD_ATTN(16);
     else EESD_ATTN(32);
 #undef EESD_ATTN
 }
@@ -832,7 +853,8 @@ static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs
 int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out) {
     const int n_pages = (ctx_len + page_tokens - 1) / page_tokens;
     const int cap = kAttnPos / page_tokens > 0 ? kAttnPos / page_tokens : 1;   // pages one block can hold
-    // one wave: about two blocks per SM in flight, so aim for H_kv * n_split <= 2 * n_sm
+    // one wave: about two blocks per SM in flight, so aim for H_kv * n_split <= 2 * n_sm (measured:
+    // half and 1.5x as many slices are both slower at 6 to 16 rows)
     int want = 2 * n_sm / (Hkv * n_batches);
     if (want < 1) want = 1;
     if (want > max_splits) want = max_splits;
@@ -850,7 +872,7 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
                       int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err) {
     int pps;
-    const int rows = (H / kv.Hkv) * M, rb = rows <= 8 ? 8 : rows <= 16 ? 16 : 32;
+    const int rows = (H / kv.Hkv) * M, rb = rows <= 8 ? 8 : rows <= kRows16 ? 16 : 32;
     const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb, n_sm, max_splits, &pps);
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (dtype == 0) {
