@@ -356,7 +356,9 @@ template <typename AT> __device__ __forceinline__ int v_elem(int pos, int e) {
     return (((e / CPV) ^ (pos & 7)) * CPV) + (e % CPV);
 }
 
-template <typename AT, int D, int RB>   // RB: (head, row) pairs per block: 8, 16 or 32
+// RB: (head, row) pairs per block: 8, 16 or 32; NM: most new rows (M <= NM), which sizes the
+// unrolled handling of the new keys / values (a one-row pass runs an eighth of the code)
+template <typename AT, int D, int RB, int NM>
 __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, const float2 *__restrict__ rope, KvGeom kv,
                                                    float *__restrict__ apart, unsigned int *tickets,
                                                    float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
@@ -437,14 +439,30 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
         const int t = col >> 7;
         return part_gather_blocks<2>(pv, s_tb[t == tk ? nq : (t == tv ? nq + 1 : t - tq0)], m, col);
     };
+    // rotation factors of the new keys and of this block's queries: a constant table, fetched
+    // before the wait so that they are not one more round trip behind the partial sums
+    constexpr int kNewPerThread = (NM * D + 255) / 256;
+    constexpr int kQPerThread = RB * HALF / 256;
+    const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
+    const int n_new = max(0, p_last - p_first) * D;
+    float2 cs_new[kNewPerThread], cs_q[kQPerThread];
+#pragma unroll
+    for (int it = 0; it < kNewPerThread; it++) {
+        const int idx = tid + it * 256;
+        const int pn = idx / D, w = idx - pn * D;
+        cs_new[it] = (idx < n_new && w < HALF) ? rope[(size_t)(p_first + pn) * HALF + w] : make_float2(1.f, 0.f);
+    }
+#pragma unroll
+    for (int it = 0; it < kQPerThread; it++) {
+        const int idx = tid + it * 256;
+        const int rl = idx / HALF, i = idx - rl * HALF;
+        cs_q[it] = idx < nb * HALF ? rope[(size_t)(pos0 + (r0 + rl) % M) * HALF + i] : make_float2(1.f, 0.f);
+    }
     pdl_wait();   // from here on the QKV projection's partial sums are read
     // One round of global loads: the RMSNorm statistics (threads 0..M-1) and the raw partial
     // sums of this block's queries and of the new keys / values that fall into its slice; they
     // are scaled, rotated and rounded after the barrier, while the cached slice is still arriving.
     if (tid < M) s_rstd[tid] = row_rstd(rs, tid);
-    constexpr int kNewPerThread = kMaxRows * D / 256;
-    const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
-    const int n_new = max(0, p_last - p_first) * D;
     float raw_a[kNewPerThread], raw_b[kNewPerThread];
     int new_page[kNewPerThread];
 #pragma unroll
@@ -461,7 +479,6 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             raw_b[it] = pr.y;
         }
     }
-    constexpr int kQPerThread = RB * HALF / 256;
     float qraw_a[kQPerThread], qraw_b[kQPerThread];
 #pragma unroll
     for (int it = 0; it < kQPerThread; it++) {
@@ -486,7 +503,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const int isV = w >= HALF, i = isV ? w - HALF : w;
             float a = raw_a[it] * s_rstd[m], b = raw_b[it] * s_rstd[m];
             if (!isV) {
-                const float2 cs = rope[(size_t)pos * HALF + i];
+                const float2 cs = cs_new[it];
                 const float ra = a * cs.x - b * cs.y, rb = a * cs.y + b * cs.x;
                 a = ra; b = rb;
             }
@@ -502,7 +519,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const int rl = idx / HALF, i = idx - rl * HALF;
             const int m = (r0 + rl) % M;
             const float a = qraw_a[it] * s_rstd[m], b = qraw_b[it] * s_rstd[m];
-            const float2 cs = rope[(size_t)(pos0 + m) * HALF + i];
+            const float2 cs = cs_q[it];
             const float qa = (a * cs.x - b * cs.y) * scale, qb = (a * cs.y + b * cs.x) * scale;
             if (kTC) {
                 const bf16 ha = __float2bfloat16_rn(qa), hb = __float2bfloat16_rn(qb);
@@ -822,7 +839,7 @@ static size_t attn_smem_bytes(int es, int D, int RB, int cap, int rows, int n_sp
            (size_t)RB * n_split * 4 + 16;
 }
 
-template <typename AT, int D, int RB>
+template <typename AT, int D, int RB, int NM>
 static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                         float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
                         int pps, int n_split, float scale, bool early, int *err) {
@@ -830,10 +847,10 @@ static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, 
     const size_t smem = attn_smem_bytes((int)sizeof(AT), D, RB, pps * kv.page_tokens, rows, n_split);
     static size_t configured = 0;   // largest dynamic shared memory size enabled so far
     if (smem > configured) {
-        cudaFuncSetAttribute(attn_kernel<AT, D, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
+        cudaFuncSetAttribute(attn_kernel<AT, D, RB, NM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
         configured = 227 * 1024 - 1024;
     }
-    launch_k(attn_kernel<AT, D, RB>, dim3(kv.Hkv, n_split, (rows + RB - 1) / RB), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv, apart,
+    launch_k(attn_kernel<AT, D, RB, NM>, dim3(kv.Hkv, n_split, (rows + RB - 1) / RB), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv, apart,
              tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err);
 }
 
@@ -842,10 +859,18 @@ static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs
                           float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
                           int pps, int n_split, float scale, bool early, int *err) {
     const int rows = (H / kv.Hkv) * M;
-#define EESD_ATTN(RB) attn_launch<AT, D, RB>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err)
-    if (rows <= 8) EESD_ATTN(8);
-    else if (rows <= kRows16) EESD_ATTN(16);
-    else EESD_ATTN(32);
+#define EESD_ATTN(RB, NM) attn_launch<AT, D, RB, NM>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err)
+    if (rows <= 8) {
+        if (M == 1) EESD_ATTN(8, 1);
+        else if (M <= 4) EESD_ATTN(8, 4);
+        else EESD_ATTN(8, 8);
+    } else if (rows <= kRows16) {
+        if (M <= 4) EESD_ATTN(16, 4);
+        else EESD_ATTN(16, 16);
+    } else {
+        if (M <= 4) EESD_ATTN(32, 4);
+        else EESD_ATTN(32, 16);
+    }
 #undef EESD_ATTN
 }
 
