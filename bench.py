@@ -215,6 +215,24 @@ def profile_pass(args, device):
     eng.close()
 
 
+def profile_prefill(args, device):
+    """One prompt pass (eesd_prefill) between cudaProfilerStart/Stop (for the ncu recipes)."""
+    from paper_2406_03853_b200 import binding as b
+    eng, spec, n_prompt, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, args.layers)
+    prompt = synth.prompt_tokens(synth.SEED, n_prompt, spec.vocab).numpy()
+    eng.prefill(prompt)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()
+    e0.record()
+    eng.prefill(prompt)
+    e1.record()
+    torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
+    print("profiled: prefill of %d tokens, %s, %d layers, %.3f ms" % (n_prompt, spec.name, spec.n_layers, e0.elapsed_time(e1)))
+    eng.close()
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle as it stands, timed on the host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -259,6 +277,8 @@ def main():
     ap.add_argument("--profile-pass", type=int, default=0, metavar="M",
                     help="only run verify passes of M rows (and draft steps) inside a cudaProfilerStart/Stop "
                          "bracket, for ncu --profile-from-start off")
+    ap.add_argument("--profile-prefill", action="store_true",
+                    help="only run one prompt pass inside a cudaProfilerStart/Stop region (for ncu)")
     ap.add_argument("--layers", type=int, default=0, help="with --profile-pass: keep only this many layers")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -280,6 +300,8 @@ def main():
     from paper_2406_03853_b200 import binding as b
     if args.profile_pass:
         return profile_pass(args, device)
+    if args.profile_prefill:
+        return profile_prefill(args, device)
     from paper_2406_03853_b200 import report
     eng, spec, n_prompt, max_new = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha)
     # acceptance along one greedy trajectory of a random-init model is noisy, so every step
@@ -378,7 +400,7 @@ def main():
                      "frac": round(achieved / peaks["hbm_gbs"], 4),
                      # dram__bytes_read + dram__bytes_write of one gate/up launch at the 13B shape, from the ncu
                      # capture summarised under profiles/ (null for other shapes: not captured)
-                     "traffic": 289117952 if (spec.name == "13b") else None,
+                     "traffic": 288015872 if (spec.name == "13b") else None,
                      "bytes_per_launch": kbytes, "ms_per_launch": round(kms, 5)},
         "verify_pass": {"kv_len": kv_len, "bytes": bv, **vp},
         "draft_step_bytes": bd,
