@@ -94,11 +94,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None):
+def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None):
     from paper_2406_03853_b200 import Engine
     from paper_2406_03853_b200 import binding as b
     spec_name, n_prompt, max_new, damp, _ = WORKLOADS[wl]
     spec = synth.SPECS[spec_name].with_(damp=damp if alpha is None else alpha)
+    if n_early:
+        spec = spec.with_(n_early=n_early)
     if n_layers:
         spec = spec.with_(n_layers=n_layers, n_early=min(spec.n_early, n_layers))
     max_ctx = max(n_prompt + max_new + 16, 1024 + 32)
@@ -233,6 +235,55 @@ def profile_prefill(args, device):
     eng.close()
 
 
+def run_sweep(args, device):
+    """Method sweeps on the synthetic model (one JSON line per setting, rank 0 only, not the
+    contract line): `--sweep k` decodes with every fixed draft length K = 1..10 and with the
+    Beta-TS controller (the paper's fixed-K curve against Thompson sampling); `--sweep n` rebuilds
+    the model with the early exit after N = 1, 2, 3, 5, 8, 10 layers (the paper's N sweep; in the
+    synthetic model the layers after N are the damped ones, so acceptance changes with N by
+    construction).  Each setting decodes `--steps` different seeded prompts."""
+    from paper_2406_03853_b200 import binding as b
+    from paper_2406_03853_b200 import report
+    spec_name, n_prompt, max_new, damp, kv_len = WORKLOADS[args.workload]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def measure(eng, spec, label, k_schedule):
+        u = {k: v.numpy() for k, v in synth.generate_uniforms(eng.cfg.max_ctx, 1 << 20).items()}
+        tot = {"drafted": 0, "accepted": 0, "emitted": 0, "rounds": 0}
+        ms = 0.0
+        for i in range(args.steps):
+            eng.prefill(synth.prompt_tokens(synth.SEED + i, n_prompt, spec.vocab).numpy())
+            torch.cuda.synchronize()
+            e0.record()
+            _, _, st = eng.decode(max_new, k_schedule=k_schedule, uniforms=u)
+            e1.record()
+            torch.cuda.synchronize()
+            ms += e0.elapsed_time(e1)
+            for k in tot:
+                tot[k] += st.as_dict()[k]
+        q = report.run_quality(tot["drafted"], tot["accepted"], tot["emitted"])
+        t1 = time_verify_pass(eng, spec, kv_len, 1)
+        tps = args.steps * max_new / (ms / 1e3)
+        print(json.dumps({"sweep": args.sweep, "setting": label, "workload": args.workload, "tokens_per_s": round(tps, 2),
+                          "speedup_vs_autoregressive": round(tps / (1e3 / t1), 4), "mean_k": round(tot["drafted"] / max(1, tot["rounds"]), 3),
+                          "v_d": round(q["v_d"], 4), "r_d": round(q["r_d"], 4), "hm": round(q["hm"], 2),
+                          "early_layers": spec.n_early, "damp_alpha": spec.damp, "steps": args.steps}), flush=True)
+
+    if args.sweep == "k":
+        eng, spec, _, _ = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha)
+        for K in range(1, 11):
+            measure(eng, spec, f"fixed K={K}", [K] * max_new)
+        measure(eng, spec, "beta-ts", None)
+        eng.close()
+    else:
+        for N in (1, 2, 3, 5, 8, 10):
+            eng, spec, _, _ = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha, n_early=N)
+            measure(eng, spec, f"N={N}", None)
+            eng.close()
+            del eng
+            torch.cuda.empty_cache()
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle as it stands, timed on the host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -277,6 +328,8 @@ def main():
     ap.add_argument("--profile-pass", type=int, default=0, metavar="M",
                     help="only run verify passes of M rows (and draft steps) inside a cudaProfilerStart/Stop "
                          "bracket, for ncu --profile-from-start off")
+    ap.add_argument("--sweep", choices=["k", "n"], default=None,
+                    help="method sweep instead of the benchmark line: fixed K = 1..10 against Beta-TS, or the exit depth N")
     ap.add_argument("--profile-prefill", action="store_true",
                     help="only run one prompt pass inside a cudaProfilerStart/Stop region (for ncu)")
     ap.add_argument("--layers", type=int, default=0, help="with --profile-pass: keep only this many layers")
@@ -302,6 +355,8 @@ def main():
         return profile_pass(args, device)
     if args.profile_prefill:
         return profile_prefill(args, device)
+    if args.sweep:
+        return run_sweep(args, device) if rank == 0 else None
     from paper_2406_03853_b200 import report
     eng, spec, n_prompt, max_new = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha)
     # acceptance along one greedy trajectory of a random-init model is noisy, so every step
