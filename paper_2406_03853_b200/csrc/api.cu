@@ -51,7 +51,7 @@ int check_config(const eesd_config *c) {
 
 struct Workspace {
     size_t x, xn, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
-        accept, wx, wout, wxs[3], wssq, wtok, total;
+        accept, wx, wout, wxs[3], wssq, wtok, wapart, total;
 };
 
 constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
@@ -74,6 +74,10 @@ int prefill_rows(const eesd_config *c) {
     return need < kPrefillRows ? need : kPrefillRows;
 }
 
+// arrival counters of the attention merge: one per (KV head, batch) in a decode pass, one per
+// (16-row chunk, KV head, batch) in a prompt pass
+size_t ticket_count(const eesd_config *c) { return 1024 + (size_t)(kPrefillRows / EESD_MAX_ROWS) * c->n_heads; }
+
 Workspace carve(const eesd_config *c) {
     Workspace w;
     const size_t R = EESD_MAX_ROWS;
@@ -93,7 +97,7 @@ Workspace carve(const eesd_config *c) {
     w.xs[X_ATTN] = take(2 * R * qd * 2);
     w.xs[X_FFN] = take(2 * R * (size_t)c->ffn_dim * 2);
     w.ssq = take((size_t)EESD_MAX_ROWS * kSsqBlocks * 4);
-    w.tickets = take(1024 * 4);
+    w.tickets = take(ticket_count(c) * 4);
     {   // partial sums: SIMT layout [splits][16][maxR], or stream-K blocks of the widest projection
         size_t part_floats = (size_t)kPartSplits * R * maxR;
         const size_t sk_floats = (maxR / 128 + (size_t)kMaxSm) * R * 128;  // blocks <= tiles + CTAs
@@ -110,7 +114,7 @@ Workspace carve(const eesd_config *c) {
     w.u_stage = take(64 * 4);
     w.err = take(16);
     w.accept = take(accept_scratch_bytes(1, EESD_MAX_ROWS));
-    w.wx = w.wout = w.wssq = w.wtok = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
+    w.wx = w.wout = w.wssq = w.wtok = w.wapart = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
     if (const size_t P = (size_t)prefill_rows(c)) {
         // prompt path: residual stream, one projection result, the three activation matrices as
         // two bf16 terms ([chunk of 16][hi | lo][16][K]), RMSNorm statistics, token ids
@@ -124,6 +128,7 @@ Workspace carve(const eesd_config *c) {
         w.wxs[X_FFN] = take(2 * P * (size_t)c->ffn_dim * 2);
         w.wssq = take(P * kSsqBlocks * 4);
         w.wtok = take(P * 4);
+        w.wapart = take(attention_prompt_scratch_floats(c->max_ctx, c->page_tokens, c->n_heads, c->head_dim, (int)P) * 4);
     }
     w.total = o;
     return w;
@@ -151,7 +156,7 @@ struct eesd_ctx {
     CUtensorMap m_x[3];
     // prompt (wide) path: up to wide_rows prompt rows per pass
     int wide_rows;
-    float *wx, *wout, *wssq;
+    float *wx, *wout, *wssq, *wapart;
     void *wxs[3];
     int32_t *wtok;
     CUtensorMap m_wx[3];
@@ -333,8 +338,8 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
 
 // Prompt pass (wide path): the target model on Mtot <= wide_rows prompt rows at positions
 // p0.., no logits.  Projections run on the wide tensor-core kernel (weights cross HBM once
-// per pass); attention runs chunk by chunk (16 rows), each chunk appending its keys / values
-// before the next one reads them; the exit layer's keys / values follow layer N.
+// per pass); the rows' keys / values are appended first, then all 16-row chunks attend to the
+// cache in one launch; the exit layer's keys / values follow layer N.
 int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
     const eesd_config &f = c->cfg;
     cudaStream_t s = c->stream;
@@ -362,17 +367,10 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
         const bool exit_here = (l == f.n_early - 1);
         const float *g_after = exit_here ? c->layers[L].g_attn : (l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
         PartView pv = proj(w.m_qkv, X_NORM, qd + 2 * kvd, d);
-        for (int c0 = 0; c0 < Mtot; c0 += EESD_MAX_ROWS) {
-            const int m = Mtot - c0 < EESD_MAX_ROWS ? Mtot - c0 : EESD_MAX_ROWS;
-            PartView cpv = pv;
-            cpv.base = pv.base + (size_t)c0 * pv.R;
-            RowScale crs = rs;
-            crs.ssq = rs.ssq + (size_t)c0 * kSsqBlocks;
-            char *dst = (char *)c->wxs[X_ATTN] + (size_t)(c0 / EESD_MAX_ROWS) * 2 * EESD_MAX_ROWS * qd * 2;
-            launch_attention(s, f.dtype, cpv, crs, c->rope, kv_geom(c, l), c->apart, c->tickets, nullptr, dst, m, p0 + c0, H,
-                             c->n_sm, kAttnSplits, c0 == 0, c->err);
-            c->launches++;
-        }
+        // keys / values of all rows into the cache first, then every 16-row chunk attends in one launch
+        launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, l), c->rope, nullptr, true, c->err, qd);
+        launch_attention_prompt(s, f.dtype, pv, rs, c->rope, kv_geom(c, l), c->wapart, c->tickets, c->wxs[X_ATTN], Mtot, p0, H, c->err);
+        c->launches += 2;
         pv = proj(w.m_o, X_ATTN, d, qd);
         resid(&pv, w.g_ffn);
         pv = proj(w.m_gu, X_NORM, 2 * F, d);
@@ -673,7 +671,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128);
         if (c->wide_rows) {
             c->wx = (float *)(ws + w.wx); c->wout = (float *)(ws + w.wout); c->wssq = (float *)(ws + w.wssq);
-            c->wtok = (int32_t *)(ws + w.wtok);
+            c->wtok = (int32_t *)(ws + w.wtok); c->wapart = (float *)(ws + w.wapart);
             const int ks[3] = {d, qd_, F};
             for (int i = 0; i < 3; i++) {
                 c->wxs[i] = ws + w.wxs[i];
@@ -703,7 +701,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     }
     memset(c->h_result, 0, 256);
     cudaMemsetAsync(c->err, 0, 16, c->stream);
-    cudaMemsetAsync(c->tickets, 0, 1024 * 4, c->stream);
+    cudaMemsetAsync(c->tickets, 0, ticket_count(cfg) * 4, c->stream);
     cudaMemsetAsync(c->ints, 0, kIntSlots * 4, c->stream);
     cudaMemsetAsync(c->accept_scratch, 0, accept_scratch_bytes(1, EESD_MAX_ROWS), c->stream);
     launch_rope_table(c->stream, c->rope, cfg->max_ctx, cfg->head_dim, cfg->rope_theta);

@@ -263,10 +263,10 @@ template <typename AT> __device__ __forceinline__ int v_elem(int pos, int e);
 // grid (heads, M), block D/2: one thread per rotation pair.
 template <typename AT>
 __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeom kv, const float2 *rope, float *q,
-                                int head_off, int *err) {
+                                int head_off, int col_off, int *err) {
     const int hh = blockIdx.x + head_off;  // 0..H-1 q, H..H+Hkv-1 k, then v
     const int m = blockIdx.y, i = threadIdx.x, D = kv.D;
-    const int col = blockIdx.x * D + 2 * i;
+    const int col = col_off + blockIdx.x * D + 2 * i;
     pdl_trigger();
     pdl_wait();
     const float rstd = row_rstd(rs, m);
@@ -301,11 +301,11 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
     }
 }
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
-                     const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err) {
+                     const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0) {
     const int heads = only_kv ? 2 * kv.Hkv : H + 2 * kv.Hkv;
     dim3 grid(heads, M);
-    if (dtype == 0) launch_k(qkv_post_kernel<float>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, err);
-    else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, err);
+    if (dtype == 0) launch_k(qkv_post_kernel<float>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err);
+    else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err);
 }
 
 // ------------------------------------------------------------------------------------ paged decode attention
@@ -362,7 +362,8 @@ template <typename AT, int D, int RB, int NM>
 __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, const float2 *__restrict__ rope, KvGeom kv,
                                                    float *__restrict__ apart, unsigned int *tickets,
                                                    float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
-                                                   int M, int pos0, int H, int pps, int n_split, float scale, int *err) {
+                                                   int M, int pos0, int H, int pps, int n_split, float scale, int *err,
+                                                   int Mtot, int nbat, size_t ml_off) {
     typedef typename KPair<AT>::T KP;
     constexpr int HALF = D / 2;
     constexpr int DPL = D / 32;             // output dimensions per lane in the PV phase
@@ -385,13 +386,29 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     float *s_rstd = s_l + RB;                                    // [kMaxRows]
     uint64_t *bar = reinterpret_cast<uint64_t *>(s_rstd + kMaxRows);
     float *wgt = reinterpret_cast<float *>(bar + 2);             // [RB][n_split] merge weights
-    // per-slice (maximum, sum) pairs live behind the outputs: [H][16][kMaxSlices]
-    float2 *ml = reinterpret_cast<float2 *>(apart + (size_t)H * kMaxSlices * kMaxRows * D);
     __shared__ int s_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
-    const int r0 = blockIdx.z * RB;          // first (head, row) pair of this block's batch
+    // Prompt mode (Mtot > 0): grid z also runs over the 16-row chunks of Mtot prompt rows whose
+    // keys and values are in the cache already; chunk c is an independent problem (rows
+    // pos0 + 16 c .., its own scratch, counters and slice count) and nothing is appended.
+    const int chunk = blockIdx.z / nbat, bz = blockIdx.z - chunk * nbat;
+    const bool cached_rows = Mtot > 0;
+    if (cached_rows) {
+        M = min(kMaxRows, Mtot - chunk * kMaxRows);
+        pos0 += chunk * kMaxRows;
+        n_split = ((pos0 + M + PT - 1) / PT + pps - 1) / pps;
+        if (sp >= n_split || group * M <= bz * RB) return;   // a short last chunk fills fewer slices and batches
+        pv.base += (size_t)chunk * kMaxRows * pv.R;
+        rs.ssq += (size_t)chunk * kMaxRows * kSsqBlocks;
+        if (attn_out) attn_out += (size_t)chunk * kMaxRows * H * D;
+        if (attn_split) attn_split += (size_t)chunk * 2 * kMaxRows * H * D;
+        apart += (size_t)chunk * (ml_off + (size_t)H * kMaxRows * kMaxSlices * 2);
+    }
+    // per-slice (maximum, sum) pairs live behind the outputs: [H][16][kMaxSlices]
+    float2 *ml = reinterpret_cast<float2 *>(apart + ml_off);
+    const int r0 = bz * RB;                  // first (head, row) pair of this block's batch
     const int ctx_len = pos0 + M;
     const int n_pages = (ctx_len + PT - 1) / PT;
     const int page_lo = sp * pps, page_hi = min(n_pages, page_lo + pps);
@@ -444,7 +461,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     constexpr int kNewPerThread = (NM * D + 255) / 256;
     constexpr int kQPerThread = RB * HALF / 256;
     const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
-    const int n_new = max(0, p_last - p_first) * D;
+    const int n_new = cached_rows ? 0 : max(0, p_last - p_first) * D;
     float2 cs_new[kNewPerThread], cs_q[kQPerThread];
 #pragma unroll
     for (int it = 0; it < kNewPerThread; it++) {
@@ -770,7 +787,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        unsigned int *tk = tickets + kh * gridDim.z + blockIdx.z;   // one counter per (KV head, batch)
+        unsigned int *tk = tickets + ((size_t)chunk * gridDim.x + kh) * nbat + bz;   // one counter per (chunk, KV head, batch)
         const unsigned int prev = atomicAdd(tk, 1u);
         s_last = (prev == (unsigned int)n_split - 1);
         if (s_last) *tk = 0;
@@ -842,24 +859,26 @@ static size_t attn_smem_bytes(int es, int D, int RB, int cap, int rows, int n_sp
 template <typename AT, int D, int RB, int NM>
 static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                         float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                        int pps, int n_split, float scale, bool early, int *err) {
-    const int rows = (H / kv.Hkv) * M;
+                        int pps, int n_split, float scale, bool early, int *err, int Mtot) {
+    const int rows = (H / kv.Hkv) * M, nbat = (rows + RB - 1) / RB;
+    const int chunks = Mtot > 0 ? (Mtot + kMaxRows - 1) / kMaxRows : 1;
+    const size_t ml_off = (size_t)H * (Mtot > 0 ? n_split : kMaxSlices) * kMaxRows * D;
     const size_t smem = attn_smem_bytes((int)sizeof(AT), D, RB, pps * kv.page_tokens, rows, n_split);
     static size_t configured = 0;   // largest dynamic shared memory size enabled so far
     if (smem > configured) {
         cudaFuncSetAttribute(attn_kernel<AT, D, RB, NM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
         configured = 227 * 1024 - 1024;
     }
-    launch_k(attn_kernel<AT, D, RB, NM>, dim3(kv.Hkv, n_split, (rows + RB - 1) / RB), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv, apart,
-             tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err);
+    launch_k(attn_kernel<AT, D, RB, NM>, dim3(kv.Hkv, n_split, chunks * nbat), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv,
+             apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, Mtot, nbat, ml_off);
 }
 
 template <typename AT, int D>
 static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                           float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                          int pps, int n_split, float scale, bool early, int *err) {
+                          int pps, int n_split, float scale, bool early, int *err, int Mtot) {
     const int rows = (H / kv.Hkv) * M;
-#define EESD_ATTN(RB, NM) attn_launch<AT, D, RB, NM>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err)
+#define EESD_ATTN(RB, NM) attn_launch<AT, D, RB, NM>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot)
     if (rows <= 8) {
         if (M == 1) EESD_ATTN(8, 1);
         else if (M <= 4) EESD_ATTN(8, 4);
@@ -893,20 +912,49 @@ int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n
     return n_split;
 }
 
+static void attention_any(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
+                          const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
+                          int M, int pos0, int H, int pps, int n_split, bool early, int *err, int Mtot) {
+    const float scale = 1.0f / sqrtf((float)kv.D);
+    if (dtype == 0) {
+        if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot);
+        else attn_dispatch<float, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot);
+    } else {
+        if (kv.D == 64) attn_dispatch<bf16, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot);
+        else attn_dispatch<bf16, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot);
+    }
+}
+
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
                       int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err) {
     int pps;
     const int rows = (H / kv.Hkv) * M, rb = rows <= 8 ? 8 : rows <= kRows16 ? 16 : 32;
     const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb, n_sm, max_splits, &pps);
-    const float scale = 1.0f / sqrtf((float)kv.D);
-    if (dtype == 0) {
-        if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err);
-        else attn_dispatch<float, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err);
-    } else {
-        if (kv.D == 64) attn_dispatch<bf16, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err);
-        else attn_dispatch<bf16, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err);
-    }
+    attention_any(s, dtype, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, 0);
+}
+
+// Prompt attention: Mtot rows at positions pos0.. whose keys / values are in the cache already
+// (launch_qkv_post), all 16-row chunks in one launch.  Slices are as long as a block can hold.
+static int prompt_pps(int page_tokens) {
+    int pps = kAttnPos / page_tokens > 0 ? kAttnPos / page_tokens : 1;
+    if ((pps * page_tokens) % 16) pps++;
+    return pps;
+}
+int attention_prompt_splits(int ctx_len, int page_tokens) {
+    const int pps = prompt_pps(page_tokens), n_pages = (ctx_len + page_tokens - 1) / page_tokens;
+    return (n_pages + pps - 1) / pps;
+}
+size_t attention_prompt_scratch_floats(int ctx_len, int page_tokens, int H, int D, int rows) {
+    const size_t chunks = (rows + kMaxRows - 1) / kMaxRows;
+    const size_t per_chunk = (size_t)H * attention_prompt_splits(ctx_len, page_tokens) * kMaxRows * D + (size_t)H * kMaxRows * kMaxSlices * 2;
+    return chunks * per_chunk;
+}
+void launch_attention_prompt(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
+                             const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
+                             int Mtot, int pos0, int H, int *err) {
+    const int pps = prompt_pps(kv.page_tokens), n_split = attention_prompt_splits(pos0 + Mtot, kv.page_tokens);
+    attention_any(s, dtype, pv, rs, rope, kv, apart, tickets, nullptr, attn_split, kMaxRows, pos0, H, pps, n_split, false, err, Mtot);
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU, partial sums

@@ -68,9 +68,9 @@ void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, 
 // out[sp][m][r] = sum_{k in split sp} A[m][k] * W[r][k]; returns the number of K splits written
 int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float *out, int M, int R, int K);
 // RoPE + KV append (+ q store).  part rows are [q heads | k heads | v heads] or, when
-// only_kv, [k heads | v heads].
+// only_kv, [k heads | v heads] starting at column kv_col0 of the projection result.
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
-                     const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err);
+                     const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0 = 0);
 // Fused attention step of one layer on M new rows: q/k/v of the new rows are taken from the
 // QKV projection's partial sums (scaled by rs, rotated), the new keys/values are appended to
 // the paged cache, every KV head's cached slice is read once, and the slices are merged into
@@ -82,6 +82,15 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
                       int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err);
+// Prompt attention: all 16-row chunks of Mtot rows in one launch; the rows' keys / values must be
+// in the cache already (launch_qkv_post with only_kv on the QKV result) and pv must be a plain
+// [Mtot][R] result (mode 0).  apart: attention_prompt_scratch_floats(...) floats; tickets: zeroed
+// counters, one per (chunk, KV head, batch).  attn_split: [chunk][hi | lo][16][H * D] bf16.
+int attention_prompt_splits(int ctx_len, int page_tokens);
+size_t attention_prompt_scratch_floats(int ctx_len, int page_tokens, int H, int D, int rows);
+void launch_attention_prompt(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
+                             const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
+                             int Mtot, int pos0, int H, int *err);
 void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F);
 void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R);
 // programmatic dependent launch (kernels start early and wait on-device for their producer):
