@@ -166,6 +166,36 @@ def time_verify_pass(eng, spec, ctx_len, M, reps=5):
     return statistics.median(ts)
 
 
+def time_accept_kernel(device, batches=(1, 8, 64), ks=(4, 16), vocab=32000, reps=20):
+    """The fused softmax / accept / resample kernel on the accept-sweep inputs (vocab 32000,
+    sigma 1, delta 1, temperature 1).  Algorithmic bytes: every p and q logit read once, plus the
+    rejected (or bonus) row pair read again for the residual draw: (2K + 3) V 4 bytes per sequence
+    at most.  Inputs exceed L2 only at batch 64 x K 16 (262 MB); the smaller cases are timed from
+    L2, are latency bound, and their figure includes the host's launch overhead (one call, one
+    memset and one kernel, between the two events)."""
+    from paper_2406_03853_b200 import binding as b
+    out = {}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for B in batches:
+        for K in ks:
+            p, q, ua, ur, ud = synth.accept_case(0, B, K, vocab, 1.0, 1.0, device=device)
+            toks = b.sample_rows(q.view(B * K, vocab), ud.view(-1), 1.0).view(B, K)
+            for _ in range(3):
+                b.accept_resample(p, q, toks, ua, ur, 1.0)
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(reps):
+                e0.record()
+                b.accept_resample(p, q, toks, ua, ur, 1.0)
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            ms = statistics.median(ts)
+            nbytes = B * (2 * K + 3) * vocab * 4
+            out[f"B{B}_K{K}"] = {"us": round(ms * 1e3, 2), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1)}
+    return out
+
+
 def oracle_sample(spec, mean_k, mean_emit, budget_s=12.0):
     """CPU oracle on a bounded slice: one decoder layer of this shape on (mean_k + 1) rows and
     on 1 row against a 512-token cache, repeated until about `budget_s` seconds of CPU work
@@ -459,6 +489,7 @@ def main():
                      "bytes_per_launch": kbytes, "ms_per_launch": round(kms, 5)},
         "verify_pass": {"kv_len": kv_len, "bytes": bv, **vp},
         "draft_step_bytes": bd,
+        "accept_kernel": time_accept_kernel(device),
         "round_stats": {"rounds_per_step": round(s0["rounds"] / args.steps, 1), "mean_k": round(mean_k, 3), "v_d": round(v_d, 4), "r_d": round(r_d, 4),
                         "hm": round(qual["hm"], 2),
                         "ms_per_draft_step": round(t_d, 4), "autoregressive_tokens_per_s": round(1e3 / t_t, 2),

@@ -42,7 +42,11 @@ __device__ __forceinline__ float exp_c(float t) {
     return __fmul_rn(p, __int_as_float(((int)n + 127) << 23));
 }
 
-__device__ __forceinline__ float expo(float l, float m, float T) { return exp_c(__fdiv_rn(__fsub_rn(l, m), T)); }
+// (x / 1 is x exactly, so the division is skipped at T = 1 without changing a bit)
+__device__ __forceinline__ float expo(float l, float m, float T) {
+    const float d = __fsub_rn(l, m);
+    return exp_c(T == 1.0f ? d : __fdiv_rn(d, T));
+}
 __device__ __forceinline__ unsigned long long fix40(float e) { return __float2ull_rz(__fmul_rn(e, 1099511627776.0f)); }
 __device__ __forceinline__ unsigned long long fix32(float w) { return __float2ull_rz(__fmul_rn(w, 4294967296.0f)); }
 __device__ __forceinline__ float z_to_float(unsigned long long Z) {
@@ -148,8 +152,45 @@ struct AccSmem {
     int found;
 };
 
-// max / argmax / integer normaliser of one row
+// max / argmax / integer normaliser of one row.  Rows of up to kRegRow logits (16-byte aligned,
+// V % 4 == 0) are read from memory ONCE, eight 16-byte loads per thread all in flight, and both
+// passes (maximum, then the integer normaliser) run from registers; other rows take two passes
+// over memory.  Every sum is an exact integer sum, so the result does not depend on the path.
+constexpr int kRegVec = 8;                              // float4 per thread held in registers
+constexpr int kRegRow = kAccThreads * kRegVec * 4;      // 32768 logits
 __device__ RowStat row_stat(const float *l, int V, float T, bool need_z, AccSmem &sm) {
+    RowStat st;
+    if (V <= kRegRow && (V & 3) == 0 && ((uintptr_t)l & 15) == 0) {
+        const int nv = V >> 2;
+        float4 x[kRegVec];
+#pragma unroll
+        for (int k = 0; k < kRegVec; k++) {
+            const int i = threadIdx.x + k * kAccThreads;
+            x[k] = i < nv ? __ldcs(reinterpret_cast<const float4 *>(l) + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        }
+        float v = -INFINITY;
+        int idx = 0x7fffffff;
+#pragma unroll
+        for (int k = 0; k < kRegVec; k++) {   // ascending index within the thread: strict > keeps the lowest
+            const int i4 = (threadIdx.x + k * kAccThreads) * 4;
+            if (x[k].x > v) { v = x[k].x; idx = i4; }
+            if (x[k].y > v) { v = x[k].y; idx = i4 + 1; }
+            if (x[k].z > v) { v = x[k].z; idx = i4 + 2; }
+            if (x[k].w > v) { v = x[k].w; idx = i4 + 3; }
+        }
+        block_argmax(v, idx, sm.sv, sm.si);
+        st.m = v; st.arg = idx; st.Z = 0;
+        if (need_z) {
+            unsigned long long z = 0;
+#pragma unroll
+            for (int k = 0; k < kRegVec; k++) {
+                if (threadIdx.x + k * kAccThreads < nv)
+                    z += fix40(expo(x[k].x, v, T)) + fix40(expo(x[k].y, v, T)) + fix40(expo(x[k].z, v, T)) + fix40(expo(x[k].w, v, T));
+            }
+            st.Z = block_sum_u64(z, sm.s64);
+        }
+        return st;
+    }
     float v = -INFINITY;
     int idx = 0x7fffffff;
     for (int i = threadIdx.x; i < V; i += blockDim.x) {
@@ -157,7 +198,6 @@ __device__ RowStat row_stat(const float *l, int V, float T, bool need_z, AccSmem
         if (x > v) { v = x; idx = i; }
     }
     block_argmax(v, idx, sm.sv, sm.si);
-    RowStat st;
     st.m = v; st.arg = idx; st.Z = 0;
     if (need_z) {
         unsigned long long z = 0;
@@ -181,25 +221,49 @@ __device__ __forceinline__ float weight_of(int v, const float *lp, const RowStat
     return r > 0.0f ? r : 0.0f;
 }
 
-// inverse-CDF draw over the whole block; returns -1 when every weight truncates to zero
+// inverse-CDF draw over the whole block; returns -1 when every weight truncates to zero.
+// Warp w owns the contiguous entries [w * chunk, (w + 1) * chunk) and walks them 32 at a time
+// (lane = entry within the group: coalesced reads); the warp that holds tau walks its chunk
+// once more with an inclusive scan per group to find the entry.
 __device__ int block_draw(const float *lp, const RowStat &sp, const float *lq, const RowStat &sq, float T,
                           int V, float u, AccSmem &sm) {
-    const int seg = (V + blockDim.x - 1) / blockDim.x;
-    const int lo = min(V, (int)threadIdx.x * seg), hi = min(V, lo + seg);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    const int chunk = ((V + nwarp - 1) / nwarp + 31) & ~31;   // a multiple of 32 entries per warp
+    const int lo = min(V, warp * chunk), hi = min(V, lo + chunk);
     unsigned long long mine = 0;
-    for (int v = lo; v < hi; v++) mine += fix32(weight_of(v, lp, sp, lq, sq, T));
-    unsigned long long W;
-    const unsigned long long off = block_excl_scan_u64(mine, sm.s64, &W);
+    for (int v = lo + lane; v < hi; v += 32) mine += fix32(weight_of(v, lp, sp, lq, sq, T));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);   // the warp's total, in every lane
+    __syncthreads();
+    if (lane == 0) sm.s64[warp] = mine;
     if (threadIdx.x == 0) sm.found = -1;
     __syncthreads();
+    unsigned long long off = 0, W = 0;
+    for (int w = 0; w < nwarp; w++) {   // 32 values from shared memory: exclusive prefix and total
+        const unsigned long long t = sm.s64[w];
+        if (w < warp) off += t;
+        W += t;
+    }
     if (W != 0) {
         const unsigned long long mu = __float2ull_rz(__fmul_rn(u, 16777216.0f));
         const unsigned long long tau = (mu * W) >> 24;
-        if (off <= tau && tau < off + mine) {
+        if (off <= tau && tau < off + mine) {   // warp-uniform
             unsigned long long acc = off;
-            for (int v = lo; v < hi; v++) {
-                acc += fix32(weight_of(v, lp, sp, lq, sq, T));
-                if (acc > tau) { sm.found = v; break; }
+            for (int base = lo; base < hi; base += 32) {
+                const int v = base + lane;
+                const unsigned long long w = v < hi ? fix32(weight_of(v, lp, sp, lq, sq, T)) : 0ull;
+                unsigned long long inc = w;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc += t;
+                }
+                const unsigned int hit = __ballot_sync(0xffffffffu, acc + inc > tau);
+                if (hit) {
+                    if (lane == 0) sm.found = base + __ffs(hit) - 1;   // smallest entry whose inclusive prefix exceeds tau
+                    break;
+                }
+                acc += __shfl_sync(0xffffffffu, inc, 31);
             }
         }
     }
@@ -245,9 +309,25 @@ __global__ void __launch_bounds__(kAccThreads) accept_kernel(const float *p_logi
     __threadfence();
 
     const int32_t *x = tokens + (size_t)b * K;
+    __shared__ int s_ok[EESD_MAX_ROWS];
+    if ((int)threadIdx.x < K && K <= EESD_MAX_ROWS) {   // one test per thread: their loads are in flight together
+        const int j = threadIdx.x, t = x[j];
+        bool ok;
+        if (greedy) {
+            ok = t == ld_stat(&st[j]).arg;
+        } else {
+            const float p = prob_of(pl[(size_t)j * V + t], ld_stat(&st[j]), T);
+            const float q = prob_of(ql[(size_t)j * V + t], ld_stat(&st[K + 1 + j]), T);
+            ok = __fmul_rn(u_acc[(size_t)b * K + j], q) < p;
+        }
+        s_ok[j] = ok;
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
         int j = 0;
-        if (greedy) {
+        if (K <= EESD_MAX_ROWS) {
+            while (j < K && s_ok[j]) j++;
+        } else if (greedy) {
             while (j < K && x[j] == ld_stat(&st[j]).arg) j++;
         } else {
             for (; j < K; j++) {
