@@ -130,15 +130,22 @@ def test_same_tokens_without_programmatic_dependent_launch():
     assert outs[0] == outs[1] and len(outs[0].split()) == 32
 
 
-def test_wide_prompt_pass_matches_row_chunks_and_oracle():
-    """Prompts longer than 16 rows go through the wide projection kernel (128-row panels); the
-    cache it leaves must equal, up to summation order, the one built 16 rows at a time, and the
-    next pass must match the oracle."""
-    spec = synth.TINY.with_(dtype="bf16", ffn_dim=640, n_layers=3)
-    n_prompt = 300                                            # 299 rows: two full panels and a ragged one
+@pytest.mark.parametrize("variant,n_prompt,max_ctx", [("mha", 300, 384), ("gqa8", 150, 256), ("wide_head", 200, 256),
+                                                        ("two_passes", 700, 768)])
+def test_wide_prompt_pass_matches_row_chunks_and_oracle(variant, n_prompt, max_ctx):
+    """Prompts longer than 16 rows go through the wide projection kernel (128-row panels) and
+    the prompt mode of the attention kernel (all 16-row chunks in one launch); the cache they
+    leave must equal, up to summation order, the one built 16 rows at a time, and the next pass
+    must match the oracle.  Variants: ragged panels, 8 query heads per KV head (four row batches
+    per chunk), 128-wide heads, and a prompt of more than 512 rows (a second pass that starts at
+    a non-zero position and attends over several slices)."""
+    base = synth.TINY.with_(dtype="bf16", ffn_dim=640, n_layers=3)
+    spec = {"mha": base, "two_passes": base.with_(n_layers=2),
+            "gqa8": base.with_(n_heads=8, n_kv_heads=1, head_dim=64),
+            "wide_head": base.with_(n_heads=2, n_kv_heads=1, head_dim=128)}[variant]
     prompt = synth.prompt_tokens(9, n_prompt, spec.vocab).numpy()
-    wide = engine_from_spec(spec, max_ctx=384, k_cap=10, fixed_k=3, page_tokens=16)
-    rows = engine_from_spec(spec, max_ctx=384, k_cap=10, fixed_k=3, page_tokens=16)
+    wide = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, page_tokens=16)
+    rows = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, page_tokens=16)
     rows.capture_hidden(True)                                 # capture keeps the 16-row path
     n0 = wide.launch_count()
     wide.prefill(prompt)
@@ -152,7 +159,7 @@ def test_wide_prompt_pass_matches_row_chunks_and_oracle():
     assert (a != 0).sum() == (b != 0).sum() > 0
     assert (a - b).abs().max().item() < 2e-2
     assert ((a - b).abs() > 1e-3).float().mean().item() < 1e-3   # bf16 rounding flips only
-    m = oracle_from_spec(spec, 384)
+    m = oracle_from_spec(spec, max_ctx)
     m.target_rows(prompt[:-1], 0, want_logits=False)
     new = np.concatenate([prompt[-1:], synth.prompt_tokens(10, 4, spec.vocab).numpy()]).astype(np.int32)
     _, lg = m.target_rows(new, n_prompt - 1)
