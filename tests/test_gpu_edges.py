@@ -168,3 +168,26 @@ def test_wide_prompt_pass_matches_row_chunks_and_oracle(variant, n_prompt, max_c
         torch.cuda.synchronize()
         assert np.abs(eng.logits(0, 5).cpu().numpy() - lg).max() < 2e-2
     wide.close(); rows.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_long_context_many_slices(dtype):
+    """Contexts far beyond one block's slice: the fp32 model (8-token pages, prompt fed 16 rows at
+    a time) reaches 63 slices per head in the verify pass (both halves of the 64-entry merge);
+    the bf16 model feeds a 2000-token prompt through four wide passes whose attention chunks
+    see 1 to 11 slices."""
+    if dtype == "f32":
+        spec, n_prompt, max_ctx, pt, tol = synth.TINY.with_(n_layers=2), 4000, 4096, 8, 2e-4
+    else:
+        spec, n_prompt, max_ctx, pt, tol = synth.TINY.with_(dtype="bf16", ffn_dim=640, n_layers=2), 2000, 2048, 16, 2e-2
+    eng = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, page_tokens=pt)
+    m = oracle_from_spec(spec, max_ctx)
+    prompt = synth.prompt_tokens(13, n_prompt, spec.vocab).numpy()
+    eng.prefill(prompt)
+    m.target_rows(prompt[:-1], 0, want_logits=False)
+    new = np.concatenate([prompt[-1:], synth.prompt_tokens(14, 8, spec.vocab).numpy()]).astype(np.int32)
+    eng.verify_only(new)
+    torch.cuda.synchronize()
+    _, lg = m.target_rows(new, n_prompt - 1)
+    assert np.abs(eng.logits(0, 9).cpu().numpy() - lg).max() < tol
+    eng.close()

@@ -58,3 +58,39 @@ def test_first_layer_of_a_full_size_pass_matches_oracle(engine13b):
     # the pass left finite logits of the right shape behind
     lg = eng.logits(0, len(rows))
     assert torch.isfinite(lg).all() and lg.shape == (len(rows), spec.vocab)
+
+
+def test_stochastic_rounds_at_13b_layer_shapes_follow_the_rule_on_the_gpus_own_logits():
+    """Temperature 1 on bf16 weights: token streams may leave the fp64 oracle's after a draw near
+    a boundary, so the stochastic path is checked on what stays exact and on statistics.  Every
+    round, the q logits the draft steps left and the p logits the verify pass left are read
+    back; the oracle's sampler must choose the same draft tokens from those q logits, the
+    oracle's accept / resample rule must take the same decision on those (p, q, uniforms),
+    bit for bit; and over all rounds the first draft token is accepted as often as the closed
+    form sum_v min(p(v), q(v)) says (4 sigma)."""
+    import bench
+    from paper_2406_03853_b200 import binding as b
+    eng, spec, _, _ = bench.build_engine("13b-eesd", 1.0, b.CTRL_FIXED_K, torch.device("cuda:0"), n_layers=8)
+    prompt = synth.prompt_tokens(21, 40, spec.vocab).numpy()
+    eng.prefill(prompt)
+    K, rounds = 3, 60
+    expect, var, hits = 0.0, 0.0, 0
+    for r in range(rounds):
+        ud = synth.uniforms(500 + r, 1, K).numpy()
+        ua = synth.uniforms(500 + r, 2, K).numpy()
+        ur = float(synth.uniforms(500 + r, 3, 1).numpy()[0])
+        toks = eng.draft(K, ud)
+        torch.cuda.synchronize()
+        ql = eng.logits(1, K).clone()
+        for i in range(K):
+            assert oracle.sample_logits(ql[i].cpu().numpy(), 1.0, float(ud[i])) == toks[i]
+        n_acc, y = eng.verify_accept(ua, ur)
+        pl = eng.logits(0, K + 1).clone()
+        assert (n_acc, y) == oracle.accept_resample(pl.cpu().numpy(), ql.cpu().numpy(), toks, ua, ur, 1.0)
+        a1 = torch.minimum(torch.softmax(pl[0].double(), 0), torch.softmax(ql[0].double(), 0)).sum().item()
+        expect += a1
+        var += a1 * (1.0 - a1)
+        hits += int(n_acc >= 1)
+    assert abs(hits - expect) < 4.0 * np.sqrt(var) + 1.0, (hits, expect, var)
+    assert 0.05 * rounds < expect < 0.999 * rounds          # neither a degenerate draft nor a copy of the target
+    eng.close()
