@@ -223,3 +223,16 @@ def generate_uniforms(max_ctx: int, n_ctrl: int, seed: int = SEED, device="cpu")
         "u_resample": uniforms(seed, STREAM_RESAMPLE, max_ctx, device),
         "u_ctrl": uniforms(seed, STREAM_CTRL, n_ctrl, device),
     }
+
+
+STREAM_CALI = 7
+
+
+def cali_weights(spec: ModelSpec, seed: int = SEED, device="cpu") -> Dict[str, torch.Tensor]:
+    """Random-init weights of the calibration predictor (trained ones are not available): ten
+    d x d matrices W^1..W^10 in the model's dtype and the 2 x 2d matrix W_p in fp32, N(0, 0.02^2)
+    and N(0, 0.05^2)."""
+    d = spec.d_model
+    w = torch.stack([weight_tensor(seed, 4000 + i, d, d, 1.0, _torch_dtype(spec), device) for i in range(10)])
+    wp = (normal_f32(seed, STREAM_CALI, 4 * d, device) * 0.05).view(2, 2 * d)
+    return {"w": w, "wp": wp}

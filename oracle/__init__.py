@@ -36,7 +36,9 @@ class _GenCfg(C.Structure):
                 ("controller", C.c_int), ("fixed_k", C.c_int), ("alpha0", C.c_long), ("beta0", C.c_long),
                 ("ts_rule", C.c_int), ("k_schedule", C.POINTER(C.c_int)), ("n_schedule", C.c_int),
                 ("u_draft", C.POINTER(C.c_float)), ("u_accept", C.POINTER(C.c_float)),
-                ("u_resample", C.POINTER(C.c_float)), ("u_ctrl", C.POINTER(C.c_float)), ("n_ctrl", C.c_long)]
+                ("u_resample", C.POINTER(C.c_float)), ("u_ctrl", C.POINTER(C.c_float)), ("n_ctrl", C.c_long),
+                ("cali_w", C.POINTER(C.c_float)), ("cali_wp", C.POINTER(C.c_float)),
+                ("sigma_m", C.c_double), ("sigma_s", C.c_double), ("theta_hat0", C.c_double)]
 
 
 class _Round(C.Structure):
@@ -168,6 +170,42 @@ def ts_update(alpha: int, beta: int, q_v: int, n_draft: int, rule: int = 0):
     return a.value, b.value
 
 
+# Thompson sampling with calibration (Sec. 3.3, Eq. 5-8, Algorithm 3)
+def cali_theta_m(Wi, Wp, hT, hD) -> float:
+    Wi, Wp = _f32(Wi), _f32(Wp)
+    hT, hD = np.ascontiguousarray(hT, np.float64), np.ascontiguousarray(hD, np.float64)
+    d = hT.shape[0]
+    assert Wi.shape == (d, d) and Wp.shape == (2, 2 * d) and hD.shape == (d,)
+    f = lib().orc_cali_theta_m
+    f.restype, f.argtypes = C.c_double, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int]
+    return f(_p(Wi), _p(Wp), _p(hT), _p(hD), d)
+
+
+def cali_posterior(theta_m: float, theta_hat: float, n: int, sigma_m: float, sigma_s: float):
+    """Eq. 6-7: returns (mu, variance)."""
+    mu, var = C.c_double(), C.c_double()
+    f = lib().orc_cali_posterior
+    f.argtypes = [C.c_double, C.c_double, C.c_long, C.c_double, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    f(theta_m, theta_hat, n, sigma_m, sigma_s, C.byref(mu), C.byref(var))
+    return mu.value, var.value
+
+
+def cali_theta_hat(prev: float, trials_prev: int, r: int, n: int) -> float:
+    f = lib().orc_cali_theta_hat
+    f.restype, f.argtypes = C.c_double, [C.c_double, C.c_long, C.c_int, C.c_int]
+    return f(prev, trials_prev, r, n)
+
+
+def cali_continue(mu: float, var: float, u, cursor: int):
+    """Returns (chi, theta, new_cursor)."""
+    u = _f32(u)
+    cur, th = C.c_long(cursor), C.c_double()
+    f = lib().orc_cali_continue
+    f.restype, f.argtypes = C.c_int, [C.c_double, C.c_double, C.c_void_p, C.c_long, C.POINTER(C.c_long), C.POINTER(C.c_double)]
+    chi = f(mu, var, _p(u), u.shape[0], C.byref(cur), C.byref(th))
+    return chi, th.value, cur.value
+
+
 # ----------------------------------------------------------------------------- model
 class OracleModel:
     """The target + draft model over fp32 copies of the given weights.
@@ -233,8 +271,10 @@ class OracleModel:
         return (lg, hid) if want_hidden else lg
 
     def generate(self, prompt, max_new: int, *, k_cap=10, temperature=0.0, controller=0, fixed_k=4,
-                 alpha0=1, beta0=1, ts_rule=0, k_schedule=None, uniforms=None):
-        """Algorithm 1.  Returns (tokens[max_new], trace[(k, n_acc, y)], (alpha, beta))."""
+                 alpha0=1, beta0=1, ts_rule=0, k_schedule=None, uniforms=None, cali=None):
+        """Algorithm 1.  Returns (tokens[max_new], trace[(k, n_acc, y)], (alpha, beta)).
+        controller 2 (TS with calibration) takes cali = dict(w [10, d, d], wp [2, 2d], sigma_m,
+        sigma_s, theta_hat0)."""
         prompt = np.ascontiguousarray(prompt, dtype=np.int32)
         g = _GenCfg()
         g.max_new, g.k_cap, g.temperature, g.controller, g.fixed_k = max_new, k_cap, temperature, controller, fixed_k
@@ -250,6 +290,12 @@ class OracleModel:
                 keep.append(a)
                 setattr(g, name, a.ctypes.data_as(C.POINTER(C.c_float)))
             g.n_ctrl = len(keep[-1])
+        if cali is not None:
+            cw, cp = _f32(cali["w"]), _f32(cali["wp"])
+            assert cw.shape == (10, self.d, self.d) and cp.shape == (2, 2 * self.d)
+            keep += [cw, cp]
+            g.cali_w, g.cali_wp = cw.ctypes.data_as(C.POINTER(C.c_float)), cp.ctypes.data_as(C.POINTER(C.c_float))
+            g.sigma_m, g.sigma_s, g.theta_hat0 = cali["sigma_m"], cali["sigma_s"], cali["theta_hat0"]
         out = np.empty(max_new, np.int32)
         cap = max_new + 1
         trace = (_Round * cap)()

@@ -398,11 +398,63 @@ void orc_ts_update(long *alpha, long *beta, int q_v, int n_draft, int rule) {
 }
 
 /* ------------------------------------------------------------------ generation (Algorithm 1) */
+/* ------------------------------------------------------------------ Thompson sampling with calibration
+ * (Sec. 3.3 "TS with Calibration", Eq. 5-8, Algorithm 3).  Readings where the text leaves a choice:
+ *  - Eq. 5 applies "Sigmoid" to the output of a TWO-row W_p trained with cross-entropy: theta_M is
+ *    read as the class-1 probability of the 2-class softmax, 1 / (1 + exp(l_0 - l_1)).
+ *  - H_t^(T): the target's residual stream after its last layer (before the final norm) at the
+ *    last position the target has processed; H_{t+i}^(D): the draft model's residual stream after
+ *    the early-exit layer (before its norm) at the current draft step.
+ *  - W^i: i is the number of the draft step within the round (1-based), capped at 10.
+ *  - theta_hat: Eq. 8 read literally (with |Q_v| counting the token the target supplies) adds the
+ *    same amount to numerator and denominator and can only rise towards 1; the text calls it the
+ *    observed sample mean of chi, so it is kept as exactly that: with r successes in n verified
+ *    drafts of a round (the r, n of Eq. 3-4), theta_hat <- (theta_hat * (N + 1) + r) / (N + n + 1),
+ *    N = verified drafts so far, the initial theta_hat_0 weighing as one observation (the "+1"
+ *    of Eq. 8). */
+double orc_cali_theta_m(const float *Wi /* [d][d] */, const float *Wp /* [2][2d] */, const double *hT,
+                        const double *hD, int d) {
+    double *v = (double *)malloc(sizeof(double) * d);
+    matvec(Wi, hT, d, d, v);
+    double l[2];
+    for (int c = 0; c < 2; c++) {
+        double s = 0.0;
+        for (int k = 0; k < d; k++) s += (double)Wp[(size_t)c * 2 * d + k] * v[k];
+        for (int k = 0; k < d; k++) s += (double)Wp[(size_t)c * 2 * d + d + k] * hD[k];
+        l[c] = s;
+    }
+    free(v);
+    return 1.0 / (1.0 + exp(l[0] - l[1]));
+}
+
+/* Eq. 6 and Eq. 7: posterior of mu after n verifications */
+void orc_cali_posterior(double theta_m, double theta_hat, long n, double sigma_m, double sigma_s, double *mu, double *var) {
+    const double sm2 = sigma_m * sigma_m, ss2 = sigma_s * sigma_s;
+    const double den = (double)n * sm2 + ss2;
+    *mu = ss2 / den * theta_m + (double)n * sm2 / den * theta_hat;
+    *var = sm2 * ss2 / (ss2 + (double)n * sm2);
+}
+
+double orc_cali_theta_hat(double prev, long trials_prev, int r, int n) {
+    return (prev * (double)(trials_prev + 1) + (double)r) / (double)(trials_prev + n + 1);
+}
+
+/* theta ~ N(mu, var) by the Box-Muller transform of two uniforms, chi ~ Bernoulli(theta) from a
+ * third (theta outside [0, 1] acts as 0 or 1).  Returns chi, or -1 when the stream is exhausted. */
+int orc_cali_continue(double mu, double var, const float *u, long n_u, long *cursor, double *theta_out) {
+    if (*cursor + 3 > n_u) return -1;
+    const double r = sqrt(2.0 * neg_log_u(u[(*cursor)++]));
+    const double z = r * cos(6.283185307179586476925286766559 * (double)u[(*cursor)++]);
+    const double theta = mu + sqrt(var) * z;
+    if (theta_out) *theta_out = theta;
+    return (double)u[(*cursor)++] < theta ? 1 : 0;
+}
+
 typedef struct {
     int max_new;
     int k_cap;          /* upper bound on drafted tokens per round */
     float temperature;  /* 0 = greedy */
-    int controller;     /* 0: K from k_schedule[round] (or fixed_k), 1: Beta-TS */
+    int controller;     /* 0: K from k_schedule[round] (or fixed_k), 1: Beta-TS, 2: TS with calibration */
     int fixed_k;
     long alpha0, beta0;
     int ts_rule;
@@ -411,6 +463,10 @@ typedef struct {
         u_draft / u_accept by the position the drafted token takes, u_resample by the position
         of the round's first drafted token */
     const float *u_ctrl; long n_ctrl;             /* consumed in order */
+    /* TS with calibration: predictor weights W^1..W^10 ([10][d][d]) and W_p ([2][2d]), the
+     * hyper-parameters sigma_M, sigma_S and the initial sample mean theta_hat_0 */
+    const float *cali_w, *cali_wp;
+    double sigma_m, sigma_s, theta_hat0;
 } orc_gen_cfg;
 
 typedef struct { int k, n_acc, y; } orc_round;
@@ -426,7 +482,18 @@ int orc_generate(orc_model *m, const int32_t *prompt, int n_prompt, const orc_ge
     int32_t *ctx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_prompt + g->max_new + K_cap + 2));
     memcpy(ctx, prompt, sizeof(int32_t) * n_prompt);
     int T = n_prompt;
-    if (n_prompt > 1) orc_target_rows(m, prompt, n_prompt - 1, 0, NULL, NULL);
+    const int cali = g->controller == 2;
+    const int d = c->d;
+    double *hT = (double *)calloc((size_t)d, sizeof(double));   /* H^(T): zeros until the target has run */
+    double *hD = (double *)malloc(sizeof(double) * d);
+    double *hid = NULL;
+    if (cali) hid = (double *)malloc(sizeof(double) * (size_t)(c->L + 1) * (n_prompt > K_cap + 1 ? n_prompt : K_cap + 1) * d);
+    if (n_prompt > 1) {
+        orc_target_rows(m, prompt, n_prompt - 1, 0, hid, NULL);
+        if (cali) memcpy(hT, hid + ((size_t)c->L * (n_prompt - 1) + (n_prompt - 2)) * d, sizeof(double) * d);
+    }
+    double theta_hat = g->theta_hat0;
+    long n_verify = 0, trials = 0;
     float *ql = (float *)malloc(sizeof(float) * (size_t)K_cap * V);
     float *pl = (float *)malloc(sizeof(float) * (size_t)(K_cap + 1) * V);
     int32_t *xs = (int32_t *)malloc(sizeof(int32_t) * (K_cap + 1));
@@ -444,18 +511,25 @@ int orc_generate(orc_model *m, const int32_t *prompt, int n_prompt, const orc_ge
         int K = 0;
         while (1) {
             int pos = T - 1 + K; /* position of the token fed to the draft model */
-            orc_draft_row(m, xs[K], pos, ql + (size_t)K * V, NULL);
+            orc_draft_row(m, xs[K], pos, ql + (size_t)K * V, cali ? hD : NULL);
             xs[K + 1] = orc_sample_logits(ql + (size_t)K * V, V, g->temperature, g->u_draft ? g->u_draft[pos + 1] : 0.0f);
             K++;
             if (K >= K_cap || T + K >= c->max_ctx - 1) break;
             if (g->controller == 0) { if (K >= k_force) break; }
-            else {
+            else if (cali) {
+                const int wi = (K < 10 ? K : 10) - 1;   /* K drafts done: this was draft step K */
+                const double th_m = orc_cali_theta_m(g->cali_w + (size_t)wi * d * d, g->cali_wp, hT, hD, d);
+                double mu, var;
+                orc_cali_posterior(th_m, theta_hat, n_verify, g->sigma_m, g->sigma_s, &mu, &var);
+                int chi = orc_cali_continue(mu, var, g->u_ctrl, g->n_ctrl, &cur, NULL);
+                if (chi <= 0) break;
+            } else {
                 int chi = orc_ts_continue(alpha, beta, g->u_ctrl, g->n_ctrl, &cur, NULL);
                 if (chi <= 0) break;
             }
         }
         /* verify: K+1 rows x_0..x_K at positions T-1..T-1+K */
-        orc_target_rows(m, xs, K + 1, T - 1, NULL, pl);
+        orc_target_rows(m, xs, K + 1, T - 1, hid, pl);
         int n_acc, y;
         orc_accept_resample(pl, ql, xs + 1, g->u_accept ? g->u_accept + T : NULL,
                             g->u_resample ? g->u_resample[T] : 0.0f, K, V, g->temperature, &n_acc, &y);
@@ -465,11 +539,20 @@ int orc_generate(orc_model *m, const int32_t *prompt, int n_prompt, const orc_ge
         T += n_acc + 1;
         t += n_acc + 1;
         orc_ts_update(&alpha, &beta, n_acc + 1, K, g->ts_rule);
+        if (cali) {
+            /* the row whose logits gave the next token is row n_acc of this pass */
+            memcpy(hT, hid + ((size_t)c->L * (K + 1) + n_acc) * d, sizeof(double) * d);
+            long a0 = 0, b0 = 0;
+            orc_ts_update(&a0, &b0, n_acc + 1, K, g->ts_rule);   /* r and n - r of this round (Eq. 3-4) */
+            theta_hat = orc_cali_theta_hat(theta_hat, trials, (int)a0, (int)(a0 + b0));
+            trials += a0 + b0;
+            n_verify++;
+        }
         rounds++;
     }
     memcpy(out, ctx + n_prompt, sizeof(int32_t) * g->max_new);
     if (alpha_out) *alpha_out = alpha;
     if (beta_out) *beta_out = beta;
-    free(ctx); free(ql); free(pl); free(xs);
+    free(ctx); free(ql); free(pl); free(xs); free(hT); free(hD); free(hid);
     return rounds;
 }
