@@ -94,7 +94,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None):
+def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None, cali=False):
     from paper_2406_03853_b200 import Engine
     from paper_2406_03853_b200 import binding as b
     spec_name, n_prompt, max_new, damp, _ = WORKLOADS[wl]
@@ -107,7 +107,7 @@ def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_
     cfg = b.make_config(d_model=spec.d_model, n_heads=spec.n_heads, n_kv_heads=spec.n_kv_heads, head_dim=spec.head_dim,
                         ffn_dim=spec.ffn_dim, vocab=spec.vocab, n_layers=spec.n_layers, n_early=spec.n_early,
                         dtype=spec.dtype, tie_exit_head=spec.tie_exit_head, max_ctx=max_ctx, k_cap=10,
-                        temperature=temperature, controller=controller, fixed_k=5, page_tokens=16)
+                        temperature=temperature, controller=b.CTRL_CALI_TS if cali else controller, fixed_k=5, page_tokens=16)
     eng = Engine(cfg, device=device)
     # synthetic weights, generated on the device by the shared seeded generator
     for l in range(spec.n_layers):
@@ -125,6 +125,10 @@ def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_
         g["exit_head"].copy_(head)
     g["g_final"].fill_(1.0)
     g["g_exit"].fill_(1.0)
+    if cali:   # random-init predictor (trained weights are not available): times the mechanism only
+        cw = synth.cali_weights(spec, synth.SEED, device)
+        g["cali_w"].copy_(cw["w"])
+        g["cali_wp"].copy_(cw["wp"])
     torch.cuda.synchronize(device)
     return eng, spec, n_prompt, max_new
 
@@ -358,6 +362,8 @@ def main():
     ap.add_argument("--profile-pass", type=int, default=0, metavar="M",
                     help="only run verify passes of M rows (and draft steps) inside a cudaProfilerStart/Stop "
                          "bracket, for ncu --profile-from-start off")
+    ap.add_argument("--controller", choices=["beta", "cali"], default="beta",
+                    help="draft-length controller: Beta-TS (default) or TS with calibration (random-init predictor)")
     ap.add_argument("--sweep", choices=["k", "n"], default=None,
                     help="method sweep instead of the benchmark line: fixed K = 1..10 against Beta-TS, or the exit depth N")
     ap.add_argument("--profile-prefill", action="store_true",
@@ -388,7 +394,8 @@ def main():
     if args.sweep:
         return run_sweep(args, device) if rank == 0 else None
     from paper_2406_03853_b200 import report
-    eng, spec, n_prompt, max_new = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha)
+    eng, spec, n_prompt, max_new = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha,
+                                                cali=args.controller == "cali")
     # acceptance along one greedy trajectory of a random-init model is noisy, so every step
     # decodes a different seeded prompt (the same ones on every run; ranks take disjoint seeds)
     prompts = [synth.prompt_tokens(synth.SEED + 1000 * rank + i, n_prompt, spec.vocab).numpy()
@@ -472,7 +479,8 @@ def main():
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dec_ms / args.steps, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": spec.dtype, "data": "synthetic",
         "config": {"workload": args.workload, "shape": spec.name, "prompt_tokens": n_prompt, "new_tokens": max_new,
-                   "batch": 1, "early_layers": spec.n_early, "damp_alpha": spec.damp, "controller": "beta_ts",
+                   "batch": 1, "early_layers": spec.n_early, "damp_alpha": spec.damp,
+                   "controller": "beta_ts" if args.controller == "beta" else "cali_ts (random-init predictor)",
                    "k_cap": 10, "temperature": args.temperature, "parallelism": f"replicas x{world}",
                    "prompts": "a different seeded prompt every step",
                    "l2_policy": "inputs larger than L2 (each pass streams every weight once)"},

@@ -45,7 +45,7 @@ enum {
 };
 
 enum { EESD_F32 = 0, EESD_BF16 = 1 };
-enum { EESD_CTRL_FIXED_K = 0, EESD_CTRL_BETA_TS = 1 };
+enum { EESD_CTRL_FIXED_K = 0, EESD_CTRL_BETA_TS = 1, EESD_CTRL_CALI_TS = 2 };
 enum { EESD_TS_RULE_PAPER = 0, EESD_TS_RULE_SINGLE_FAILURE = 1 };
 
 #define EESD_MAX_ROWS 16 /* most token rows one pass processes (k_cap + 1 <= 16) */
@@ -68,11 +68,15 @@ typedef struct eesd_config {
     int32_t max_ctx;      /* most tokens a sequence may hold (prompt + generated + drafts)      */
     int32_t k_cap;        /* most draft tokens per round, 1 <= k_cap <= EESD_MAX_ROWS - 1       */
     float temperature;    /* 0: greedy (draft top-1, accept while equal to target top-1)        */
-    int32_t controller;   /* EESD_CTRL_FIXED_K or EESD_CTRL_BETA_TS                             */
+    int32_t controller;   /* EESD_CTRL_FIXED_K, EESD_CTRL_BETA_TS or EESD_CTRL_CALI_TS                */
     int32_t fixed_k;      /* draft length for EESD_CTRL_FIXED_K                                 */
     int32_t alpha0;       /* Beta prior (Algorithm 2, initialisation); positive integers        */
     int32_t beta0;
     int32_t ts_update_rule; /* EESD_TS_RULE_PAPER: r = |Q_v|-1, n = min(|Q_v|+1, |Q_d|)          */
+    /* EESD_CTRL_CALI_TS only (Sec. 3.3 "TS with Calibration", Algorithm 3): the assumed error of
+     * the model's prediction, the assumed deviation of a round's sample mean, and the initial
+     * observed mean theta_hat_0; sigmas must be positive */
+    float cali_sigma_m, cali_sigma_s, cali_theta0;
 } eesd_config;
 
 /* Byte offsets inside the weight buffer.  A decoder layer holds, in this order:
@@ -89,6 +93,8 @@ typedef struct eesd_layout {
     size_t exit_layer;   /* one decoder layer                                                   */
     size_t exit_norm;    /* f32[d], the RMSNorm before the exit head                            */
     size_t exit_head;    /* [V][d]; equals lm_head when tie_exit_head                           */
+    size_t cali_w;       /* EESD_CTRL_CALI_TS only (else 0): W^1..W^10 of Eq. 5, [10][d][d]           */
+    size_t cali_wp;      /* EESD_CTRL_CALI_TS only (else 0): W_p of Eq. 5, f32 [2][2d]                */
     size_t total_bytes;
 } eesd_layout;
 
@@ -205,6 +211,30 @@ int eesd_decode(eesd_ctx *ctx, int max_new, const int32_t *k_schedule, int n_sch
 int eesd_context_len(const eesd_ctx *ctx, int *n_tokens, int *pages_in_use);
 /* Posterior parameters of the controller. */
 int eesd_posterior(const eesd_ctx *ctx, int64_t *alpha, int64_t *beta);
+
+/* Thompson sampling with calibration (Sec. 3.3, Eq. 5-8, Algorithm 3; EESD_CTRL_CALI_TS).
+ * eesd_generate / eesd_decode then run the draft loop step by step: after every draft step
+ * the device evaluates the predictor of Eq. 5,
+ *     theta_M = softmax(W_p [W^i H^(T) ; H^(D)])[1],   i = min(draft step, 10),
+ * with H^(T) the target's residual stream after its last layer at the last position it has
+ * processed (the row whose logits produced the pending token; zeros before any pass) and H^(D)
+ * the draft model's residual stream after the early-exit layer of that step; the host reads the
+ * one float back (a stream synchronisation per draft step, which this controller cannot avoid),
+ * forms the posterior of Eq. 6-7 from theta_M, the observed mean theta_hat and the number of
+ * verifications n, draws theta ~ N(mu, sigma^2) (Box-Muller on two controller uniforms) and
+ * chi ~ Bernoulli(theta) (a third).  After a verification theta_hat <- (theta_hat (N + 1) + r) /
+ * (N + n_r + 1) with r successes in n_r verified drafts (those of Eq. 3-4) and N the verified
+ * drafts before: the observed sample mean, theta_hat_0 counting as one observation.
+ *
+ * eesd_cali_predict: theta_M for the latest draft step of the round being drafted (for callers
+ * driving eesd_draft / eesd_verify_accept themselves); host pointer; synchronises the stream.
+ * STATE unless the controller is EESD_CTRL_CALI_TS and at least one step has been drafted.
+ * eesd_cali_state: theta_hat, verifications so far, verified drafts so far.
+ * eesd_cali_posterior: Eq. 6-7 on the host (no context needed); BADARG for non-positive sigmas. */
+int eesd_cali_predict(eesd_ctx *ctx, float *theta_m);
+int eesd_cali_state(const eesd_ctx *ctx, double *theta_hat, int64_t *n_verify, int64_t *n_trials);
+int eesd_cali_posterior(double theta_m, double theta_hat, int64_t n, double sigma_m, double sigma_s,
+                        double *mu, double *variance);
 
 /* Declares that the KV cache already holds n_ctx - 1 valid rows (whatever bytes the pool
  * contains) and that `pending` is the pending token: allocates pages, sets the length.  Used to

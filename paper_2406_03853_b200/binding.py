@@ -19,7 +19,7 @@ _LIB_PATH = os.path.join(_HERE, "libeesd.so")
 _lib = None
 
 F32, BF16 = 0, 1
-CTRL_FIXED_K, CTRL_BETA_TS = 0, 1
+CTRL_FIXED_K, CTRL_BETA_TS, CTRL_CALI_TS = 0, 1, 2
 MAX_ROWS = 16
 
 
@@ -36,13 +36,15 @@ class Config(C.Structure):
                 ("dtype", C.c_int32), ("tie_exit_head", C.c_int32), ("rms_eps", C.c_float), ("rope_theta", C.c_float),
                 ("page_tokens", C.c_int32), ("max_ctx", C.c_int32), ("k_cap", C.c_int32), ("temperature", C.c_float),
                 ("controller", C.c_int32), ("fixed_k", C.c_int32), ("alpha0", C.c_int32), ("beta0", C.c_int32),
-                ("ts_update_rule", C.c_int32)]
+                ("ts_update_rule", C.c_int32), ("cali_sigma_m", C.c_float), ("cali_sigma_s", C.c_float),
+                ("cali_theta0", C.c_float)]
 
 
 class Layout(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in
                 ("embed", "layer0", "layer_stride", "off_g_attn", "off_wqkv", "off_wo", "off_g_ffn", "off_wgu",
-                 "off_wd", "final_norm", "lm_head", "exit_layer", "exit_norm", "exit_head", "total_bytes")]
+                 "off_wd", "final_norm", "lm_head", "exit_layer", "exit_norm", "exit_head", "cali_w", "cali_wp",
+                 "total_bytes")]
 
 
 class Sizes(C.Structure):
@@ -103,6 +105,10 @@ def lib():
                                   C.POINTER(C.c_int)]
         L.eesd_context_len.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.eesd_posterior.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.eesd_cali_predict.argtypes = [vp, C.POINTER(C.c_float)]
+        L.eesd_cali_state.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.eesd_cali_posterior.argtypes = [C.c_double, C.c_double, C.c_int64, C.c_double, C.c_double,
+                                          C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.eesd_assume_context.argtypes = [vp, C.c_int, C.c_int32]
         L.eesd_verify_only.argtypes = [vp, vp, C.c_int]
         L.eesd_logits.argtypes = [vp, C.c_int, C.POINTER(vp)]
@@ -143,11 +149,12 @@ def _np_f32(a) -> np.ndarray:
 
 def make_config(*, d_model, n_heads, n_kv_heads, head_dim, ffn_dim, vocab, n_layers, n_early, dtype,
                 tie_exit_head=False, rms_eps=1e-5, rope_theta=10000.0, page_tokens=16, max_ctx=2048, k_cap=10,
-                temperature=0.0, controller=CTRL_FIXED_K, fixed_k=4, alpha0=1, beta0=1, ts_update_rule=0) -> Config:
+                temperature=0.0, controller=CTRL_FIXED_K, fixed_k=4, alpha0=1, beta0=1, ts_update_rule=0,
+                cali_sigma_m=0.2, cali_sigma_s=0.5, cali_theta0=0.5) -> Config:
     dt = {"f32": F32, "bf16": BF16}.get(dtype, dtype)
     return Config(d_model, n_heads, n_kv_heads, head_dim, ffn_dim, vocab, n_layers, n_early, dt, int(tie_exit_head),
                   rms_eps, rope_theta, page_tokens, max_ctx, k_cap, temperature, controller, fixed_k, alpha0, beta0,
-                  ts_update_rule)
+                  ts_update_rule, cali_sigma_m, cali_sigma_s, cali_theta0)
 
 
 class Engine:
@@ -214,13 +221,28 @@ class Engine:
 
     def global_views(self) -> Dict[str, torch.Tensor]:
         c, lay = self.cfg, self.layout
-        return {
+        v = {
             "embed": self._view(lay.embed, (c.vocab, c.d_model), self.wdtype),
             "g_final": self._view(lay.final_norm, (c.d_model,), torch.float32),
             "lm_head": self._view(lay.lm_head, (c.vocab, c.d_model), self.wdtype),
             "g_exit": self._view(lay.exit_norm, (c.d_model,), torch.float32),
             "exit_head": self._view(lay.exit_head, (c.vocab, c.d_model), self.wdtype),
         }
+        if c.controller == CTRL_CALI_TS:   # predictor of the calibrated controller: W^1..W^10 and W_p
+            v["cali_w"] = self._view(lay.cali_w, (10, c.d_model, c.d_model), self.wdtype)
+            v["cali_wp"] = self._view(lay.cali_wp, (2, 2 * c.d_model), torch.float32)
+        return v
+
+    # ---- Thompson sampling with calibration
+    def cali_predict(self) -> float:
+        th = C.c_float()
+        self._check(lib().eesd_cali_predict(self.h, C.byref(th)), "eesd_cali_predict")
+        return th.value
+
+    def cali_state(self):
+        th, n, tr = C.c_double(), C.c_int64(), C.c_int64()
+        self._check(lib().eesd_cali_state(self.h, C.byref(th), C.byref(n), C.byref(tr)), "eesd_cali_state")
+        return th.value, n.value, tr.value
 
     # ---- the five calls
     def reset(self):
@@ -354,6 +376,16 @@ def accept_resample(p_logits: torch.Tensor, q_logits: torch.Tensor, tokens: torc
     if st:
         raise EesdError(st, "eesd_accept_resample")
     return n, y
+
+
+def cali_posterior(theta_m: float, theta_hat: float, n: int, sigma_m: float, sigma_s: float):
+    """eesd_cali_posterior (Eq. 6-7, host arithmetic): returns (mu, variance)."""
+    mu, var = C.c_double(), C.c_double()
+    st = lib().eesd_cali_posterior(C.c_double(theta_m), C.c_double(theta_hat), C.c_int64(n), C.c_double(sigma_m),
+                                   C.c_double(sigma_s), C.byref(mu), C.byref(var))
+    if st:
+        raise EesdError(st, "eesd_cali_posterior")
+    return mu.value, var.value
 
 
 def sample_rows(logits: torch.Tensor, u: Optional[torch.Tensor], temperature: float) -> torch.Tensor:

@@ -21,9 +21,9 @@ struct LayerW {
 };
 
 // which activation matrix feeds a projection
-enum { X_NORM = 0, X_ATTN = 1, X_FFN = 2 };
+enum { X_NORM = 0, X_ATTN = 1, X_FFN = 2, X_CALI = 3 };   // X_CALI: H^(T) of the calibration predictor
 // the distinct projection shapes of a pass (each has its own stream-K plan and block table)
-enum { P_QKV = 0, P_O = 1, P_GU = 2, P_D = 3, P_EXIT_KV = 4, P_HEAD = 5, P_COUNT = 6 };
+enum { P_QKV = 0, P_O = 1, P_GU = 2, P_D = 3, P_EXIT_KV = 4, P_HEAD = 5, P_CALI = 6, P_COUNT = 7 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -42,7 +42,9 @@ int check_config(const eesd_config *c) {
     if (c->page_tokens < 8 || c->page_tokens > 128 || (c->page_tokens & (c->page_tokens - 1))) return EESD_ERR_BADARG;
     if (c->k_cap < 1 || c->k_cap > EESD_MAX_ROWS - 1) return EESD_ERR_BADARG;
     if (c->temperature < 0.f) return EESD_ERR_BADARG;
-    if (c->controller != EESD_CTRL_FIXED_K && c->controller != EESD_CTRL_BETA_TS) return EESD_ERR_BADARG;
+    if (c->controller != EESD_CTRL_FIXED_K && c->controller != EESD_CTRL_BETA_TS && c->controller != EESD_CTRL_CALI_TS)
+        return EESD_ERR_BADARG;
+    if (c->controller == EESD_CTRL_CALI_TS && (!(c->cali_sigma_m > 0.f) || !(c->cali_sigma_s > 0.f))) return EESD_ERR_BADARG;
     if (c->controller == EESD_CTRL_FIXED_K && c->fixed_k < 1) return EESD_ERR_BADARG;
     if (c->alpha0 < 1 || c->beta0 < 1) return EESD_ERR_BADARG;
     if (c->rms_eps < 0.f || c->rope_theta <= 1.f) return EESD_ERR_BADARG;
@@ -51,7 +53,7 @@ int check_config(const eesd_config *c) {
 
 struct Workspace {
     size_t x, xn, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
-        accept, wx, wout, wxs[3], wssq, wtok, wapart, total;
+        accept, wx, wout, wxs[3], wssq, wtok, wapart, hT, xs_cali, theta, total;
 };
 
 constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
@@ -114,6 +116,9 @@ Workspace carve(const eesd_config *c) {
     w.u_stage = take(64 * 4);
     w.err = take(16);
     w.accept = take(accept_scratch_bytes(1, EESD_MAX_ROWS));
+    w.hT = take((size_t)c->d_model * 4);
+    w.xs_cali = take(2 * R * (size_t)c->d_model * 2);
+    w.theta = take(16);
     w.wx = w.wout = w.wssq = w.wtok = w.wapart = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
     if (const size_t P = (size_t)prefill_rows(c)) {
         // prompt path: residual stream, one projection result, the three activation matrices as
@@ -150,10 +155,17 @@ struct eesd_ctx {
     // device pointers
     float *x, *xn, *attn, *h, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
     void *accept_scratch;
-    void *xs[3];                 // bf16 hi/lo copies of xn, attn, h
+    void *xs[4];                 // bf16 hi/lo copies of xn, attn, h, and of H^(T) (calibration predictor)
     float *ssq;                  // RMSNorm partial sums of squares of the rows in xn / xs[X_NORM]
     unsigned int *tickets;       // arrival counters of the attention merge
-    CUtensorMap m_x[3];
+    CUtensorMap m_x[4];
+    // Thompson sampling with calibration
+    float *hT, *theta_dev;       // H^(T) (fp32 [d]) and the predictor's output
+    const char *cali_w;          // W^1..W^10
+    const float *cali_wp;
+    CUtensorMap m_cali[10];
+    double theta_hat;
+    int64_t n_verify, n_trials;
     // prompt (wide) path: up to wide_rows prompt rows per pass
     int wide_rows;
     float *wx, *wout, *wssq, *wapart;
@@ -257,7 +269,7 @@ PartView run_proj(eesd_ctx *c, const void *W, const CUtensorMap *mW, int shape, 
         pv.sk = c->plan[shape];
         launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, c->plan[shape], M, c->err);
     } else {
-        const float *A = which == X_NORM ? c->xn : which == X_ATTN ? c->attn : c->h;
+        const float *A = which == X_NORM ? c->xn : which == X_ATTN ? c->attn : which == X_FFN ? c->h : c->hT;
         pv.mode = 0;
         pv.S = launch_gemm(c->stream, c->cfg.dtype, A, W, c->part, M, R, K);
         pv.split_stride = (size_t)M * R;
@@ -442,6 +454,41 @@ void ts_update(eesd_ctx *c, int q_v, int n_draft) {
     if (n < r) n = r;
     c->alpha += r;
     c->beta += n - r;
+    // TS with calibration: observed mean of chi over the verified drafts (theta_hat_0 counts as one)
+    c->theta_hat = (c->theta_hat * (double)(c->n_trials + 1) + (double)r) / (double)(c->n_trials + n + 1);
+    c->n_trials += n;
+    c->n_verify++;
+}
+
+bool cali_on(const eesd_ctx *c) { return c->cfg.controller == EESD_CTRL_CALI_TS; }
+
+// H^(T): row `row` (or the row whose index sits in device memory) of a residual-stream matrix
+void save_target_state(eesd_ctx *c, const float *x, int row, const int32_t *row_dev) {
+    launch_copy_row(c->stream, x, row, row_dev, c->hT, c->use_tc ? c->xs[X_CALI] : nullptr, c->cfg.d_model);
+    c->launches++;
+}
+
+// theta_M of Eq. 5 for draft step `step` (1-based) of the round; the draft step's residual
+// stream after the early-exit layer is row 0 of x
+int run_cali_predict(eesd_ctx *c, int step) {
+    const int d = c->cfg.d_model, wi = (step < 10 ? step : 10) - 1;
+    const char *W = c->cali_w + (size_t)wi * d * d * c->es;
+    PartView pv = run_proj(c, W, &c->m_cali[wi], P_CALI, X_CALI, 1, d, d);
+    launch_cali_theta(c->stream, pv, c->cali_wp, c->x, d, c->theta_dev);
+    c->launches++;
+    return check_launch(c);
+}
+
+// posterior of Eq. 6-7, theta ~ N(mu, var) by Box-Muller, chi ~ Bernoulli(theta)
+int cali_continue(eesd_ctx *c, float theta_m, const eesd_uniforms *u, int64_t *cursor) {
+    if (!u || !u->u_ctrl || *cursor + 3 > u->n_ctrl) return EESD_ERR_RNG;
+    double mu, var;
+    eesd_cali_posterior(theta_m, c->theta_hat, c->n_verify, c->cfg.cali_sigma_m, c->cfg.cali_sigma_s, &mu, &var);
+    auto nl = [](float v) { return -log(v > 0.0f ? (double)v : 2.98023223876953125e-08); };
+    const double r = sqrt(2.0 * nl(u->u_ctrl[(*cursor)++]));
+    const double z = r * cos(6.283185307179586476925286766559 * (double)u->u_ctrl[(*cursor)++]);
+    const double theta = mu + sqrt(var) * z;
+    return (double)u->u_ctrl[(*cursor)++] < theta ? 1 : 0;
 }
 
 void reset_sequence(eesd_ctx *c) {
@@ -451,6 +498,9 @@ void reset_sequence(eesd_ctx *c) {
     c->round_k = 0;
     c->alpha = c->cfg.alpha0;
     c->beta = c->cfg.beta0;
+    c->theta_hat = c->cfg.cali_theta0;
+    c->n_verify = 0;
+    c->n_trials = 0;
 }
 
 int prefill_impl(eesd_ctx *c, const int32_t *prompt, int n_prompt) {
@@ -469,6 +519,7 @@ int prefill_impl(eesd_ctx *c, const int32_t *prompt, int n_prompt) {
         st = run_prompt_pass(c, prompt, p, M);
         if (st) return st;
         p += M;
+        if (cali_on(c) && p == n_prompt - 1) save_target_state(c, c->wx, M - 1, nullptr);
     }
     for (; p < n_prompt - 1; p += EESD_MAX_ROWS) {
         int M = n_prompt - 1 - p;
@@ -477,6 +528,11 @@ int prefill_impl(eesd_ctx *c, const int32_t *prompt, int n_prompt) {
         if (st) return st;
         st = run_target(c, c->ints + kRowTok, M, p, false);
         if (st) return st;
+        if (cali_on(c) && p + M == n_prompt - 1) save_target_state(c, c->x, M - 1, nullptr);
+    }
+    if (cali_on(c) && n_prompt == 1) {   // the target has processed nothing yet: H^(T) = 0
+        CU(c, cudaMemsetAsync(c->hT, 0, (size_t)c->cfg.d_model * 4, c->stream));
+        if (c->use_tc) CU(c, cudaMemsetAsync(c->xs[X_CALI], 0, (size_t)2 * EESD_MAX_ROWS * c->cfg.d_model * 2, c->stream));
     }
     st = set_device_ints(c, kRoundTok, prompt + n_prompt - 1, 1);
     if (st) return st;
@@ -512,6 +568,7 @@ int verify_impl(eesd_ctx *c, const float *d_u_acc, const float *d_u_res) {
     launch_accept(c->stream, c->logits_p, c->logits_q, c->ints + kRoundTok + 1, d_u_acc, d_u_res, 1, K, f.vocab,
                   f.temperature, c->accept_scratch, c->ints + kResult, c->ints + kResult + 1, c->ints + kRoundTok);
     c->launches++;
+    if (cali_on(c)) save_target_state(c, c->x, 0, c->ints + kResult);   // the row that gave the next token
     st = check_launch(c);
     if (st) return st;
     CU(c, cudaMemcpyAsync(c->h_result, c->ints + kResult, 8, cudaMemcpyDeviceToHost, c->stream));
@@ -585,6 +642,11 @@ int eesd_weight_layout(const eesd_config *c, eesd_layout *out) {
     o += out->layer_stride;
     out->exit_norm = take(d * 4);
     out->exit_head = c->tie_exit_head ? out->lm_head : take(V * d * es);
+    out->cali_w = out->cali_wp = 0;
+    if (c->controller == EESD_CTRL_CALI_TS) {
+        out->cali_w = take(10 * d * d * es);
+        out->cali_wp = take(4 * d * 4);
+    }
     out->total_bytes = o;
     return EESD_OK;
 }
@@ -633,7 +695,9 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->ints = (int32_t *)(ws + w.ints); c->u_dev = (float *)(ws + w.u_dev); c->u_stage = (float *)(ws + w.u_stage);
     c->err = (int *)(ws + w.err); c->accept_scratch = ws + w.accept;
     c->ssq = (float *)(ws + w.ssq); c->tickets = (unsigned int *)(ws + w.tickets);
-    for (int i = 0; i < 3; i++) c->xs[i] = nullptr;
+    for (int i = 0; i < 4; i++) c->xs[i] = nullptr;
+    c->hT = (float *)(ws + w.hT); c->theta_dev = (float *)(ws + w.theta);
+    c->cali_w = nullptr; c->cali_wp = nullptr;
     c->n_sm = 1;
     {
         int dev = 0;
@@ -653,10 +717,16 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         lw.g_ffn = (const float *)(base + lay.off_g_ffn); lw.wgu = base + lay.off_wgu; lw.wd = base + lay.off_wd;
     }
     c->embed = wb + lay.embed; c->lm_head = wb + lay.lm_head; c->exit_head = wb + lay.exit_head;
+    if (cfg->controller == EESD_CTRL_CALI_TS) { c->cali_w = wb + lay.cali_w; c->cali_wp = (const float *)(wb + lay.cali_wp); }
     if (c->use_tc) {
         const int d = cfg->d_model, F = cfg->ffn_dim, R2 = 2 * EESD_MAX_ROWS;
         bool ok = true;
         for (int i = 0; i < 3; i++) c->xs[i] = ws + w.xs[i];
+        c->xs[X_CALI] = ws + w.xs_cali;
+        if (c->cali_w && tc_shape_ok(d, d)) {
+            ok = ok && tc_make_map(&c->m_x[X_CALI], c->xs[X_CALI], R2, d, R2);
+            for (int i = 0; i < 10; i++) ok = ok && tc_make_map(&c->m_cali[i], c->cali_w + (size_t)i * d * d * 2, d, d, 128);
+        }
         ok = ok && tc_make_map(&c->m_x[X_NORM], c->xs[X_NORM], R2, d, R2);
         ok = ok && tc_make_map(&c->m_x[X_ATTN], c->xs[X_ATTN], R2, qd_, R2);
         ok = ok && tc_make_map(&c->m_x[X_FFN], c->xs[X_FFN], R2, F, R2);
@@ -679,7 +749,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
             }
         }
         // work split of every projection shape
-        const int shapes[P_COUNT][2] = {{qd_ + 2 * kvd_, d}, {d, qd_}, {2 * F, d}, {d, F}, {2 * kvd_, d}, {cfg->vocab, d}};
+        const int shapes[P_COUNT][2] = {{qd_ + 2 * kvd_, d}, {d, qd_}, {2 * F, d}, {d, F}, {2 * kvd_, d}, {cfg->vocab, d}, {d, d}};
         for (int i = 0; i < P_COUNT; i++) c->plan[i] = tc_plan(shapes[i][0], shapes[i][1], c->n_sm);
         if (!ok) {
             delete c;
@@ -776,7 +846,12 @@ int eesd_verify_accept(eesd_ctx *c, const float *u_accept, float u_resample, int
     if (st) return st;
     CU(c, cudaMemcpyAsync(drafts, c->ints + kRoundTok + 1, (size_t)K * 4, cudaMemcpyDeviceToHost, c->stream));
     CU(c, cudaStreamSynchronize(c->stream));
-    return finish_round(c, drafts, n_accept, next_token);
+    int a = 0;
+    st = finish_round(c, drafts, &a, next_token);
+    if (st) return st;
+    if (n_accept) *n_accept = a;
+    ts_update(c, a + 1, K);   // the controllers' posteriors follow the observed rounds in the step API too
+    return EESD_OK;
 }
 
 // rounds of {draft, verify, accept, posterior update} from the current context until max_new
@@ -787,7 +862,7 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
     const eesd_config &f = c->cfg;
     const bool greedy = f.temperature == 0.f;
     if (!greedy && (!u || !u->u_draft || !u->u_accept || !u->u_resample)) return EESD_ERR_RNG;
-    if (f.controller == EESD_CTRL_BETA_TS && (!u || !u->u_ctrl)) return EESD_ERR_RNG;
+    if (f.controller != EESD_CTRL_FIXED_K && (!u || !u->u_ctrl)) return EESD_ERR_RNG;
     const int n0 = (int)c->tokens.size();
     if (n0 + max_new + 1 > f.max_ctx) return EESD_ERR_CTX_FULL;
     float *d_ud = c->u_dev, *d_ua = c->u_dev + f.max_ctx, *d_ur = c->u_dev + 2 * (size_t)f.max_ctx;
@@ -809,8 +884,12 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
         if (f.max_ctx - 1 - T < cap) cap = f.max_ctx - 1 - T;
         if (cap < 1) return EESD_ERR_CTX_FULL;
         int K;
+        // TS with calibration needs the predictor's output after every draft step: such rounds
+        // are drafted step by step, with a synchronisation per step (Algorithm 3)
+        const bool stepwise = f.controller == EESD_CTRL_CALI_TS && !(k_schedule && rounds < n_schedule);
         if (k_schedule && rounds < n_schedule) K = k_schedule[rounds];
         else if (f.controller == EESD_CTRL_FIXED_K) K = f.fixed_k;
+        else if (stepwise) K = 1;
         else {
             K = 1;
             while (K < cap) {
@@ -823,8 +902,24 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
         if (K < 1) K = 1;
         if (K > cap) K = cap;
         CU(c, cudaEventRecord(c->ev[2], c->stream));
-        st = draft_impl(c, K, greedy ? nullptr : d_ud + T, 1);
-        if (st) return st;
+        if (!stepwise) {
+            st = draft_impl(c, K, greedy ? nullptr : d_ud + T, 1);
+            if (st) return st;
+        } else {
+            for (K = 0;;) {
+                st = draft_impl(c, 1, greedy ? nullptr : d_ud + T + K, 1);
+                if (st) return st;
+                if (++K >= cap) break;
+                st = run_cali_predict(c, K);
+                if (st) return st;
+                float *h_theta = (float *)(c->h_result + 32);
+                CU(c, cudaMemcpyAsync(h_theta, c->theta_dev, 4, cudaMemcpyDeviceToHost, c->stream));
+                CU(c, cudaStreamSynchronize(c->stream));
+                const int chi = cali_continue(c, *h_theta, u, &cursor);
+                if (chi < 0) return chi;
+                if (!chi) break;
+            }
+        }
         CU(c, cudaEventRecord(c->ev[3], c->stream));
         st = verify_impl(c, d_ua + T, d_ur + T);
         if (st) return st;
@@ -883,6 +978,35 @@ int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new,
     float ms_p = 0.f;
     cudaEventElapsedTime(&ms_p, c->ev[0], c->ev[1]);
     return decode_impl(c, max_new, k_schedule, n_schedule, u, out, stats, trace, trace_cap, n_rounds, launches0, ms_p);
+}
+
+int eesd_cali_posterior(double theta_m, double theta_hat, int64_t n, double sigma_m, double sigma_s, double *mu,
+                        double *variance) {
+    if (!mu || !variance || !(sigma_m > 0.0) || !(sigma_s > 0.0) || n < 0) return EESD_ERR_BADARG;
+    const double sm2 = sigma_m * sigma_m, ss2 = sigma_s * sigma_s, den = (double)n * sm2 + ss2;
+    *mu = ss2 / den * theta_m + (double)n * sm2 / den * theta_hat;   // Eq. 6
+    *variance = sm2 * ss2 / den;                                      // Eq. 7
+    return EESD_OK;
+}
+
+int eesd_cali_state(const eesd_ctx *c, double *theta_hat, int64_t *n_verify, int64_t *n_trials) {
+    if (!c) return EESD_ERR_BADARG;
+    if (theta_hat) *theta_hat = c->theta_hat;
+    if (n_verify) *n_verify = c->n_verify;
+    if (n_trials) *n_trials = c->n_trials;
+    return EESD_OK;
+}
+
+int eesd_cali_predict(eesd_ctx *c, float *theta_m) {
+    if (!c || !theta_m) return EESD_ERR_BADARG;
+    if (!cali_on(c) || !c->prefilled || c->round_k < 1) return EESD_ERR_STATE;
+    int st = run_cali_predict(c, c->round_k);
+    if (st) return st;
+    float *h = (float *)(c->h_result + 32);
+    CU(c, cudaMemcpyAsync(h, c->theta_dev, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    *theta_m = *h;
+    return EESD_OK;
 }
 
 int eesd_context_len(const eesd_ctx *c, int *n_tokens, int *pages_in_use) {

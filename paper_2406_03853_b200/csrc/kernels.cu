@@ -978,6 +978,42 @@ void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float
     launch_k(swiglu_kernel, dim3((F / 4 + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, h, (bf16 *)h_split, F);
 }
 
+// ------------------------------------------------------------------------------------ calibration predictor (Eq. 5)
+__global__ void copy_row_kernel(const float *x, int row, const int32_t *row_dev, float *hT, bf16 *xs, int d) {
+    pdl_trigger();
+    pdl_wait();
+    const int r = row_dev ? *row_dev : row;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < d; i += gridDim.x * blockDim.x) {
+        const float v = x[(size_t)r * d + i];
+        hT[i] = v;
+        if (xs) store_split(xs, 0, d, i, v);
+    }
+}
+void launch_copy_row(cudaStream_t s, const float *x, int row, const int32_t *row_dev, float *hT, void *xs, int d) {
+    launch_k(copy_row_kernel, dim3((d + 255) / 256), dim3(256), 0, s, pdl_enabled(), x, row, row_dev, hT, (bf16 *)xs, d);
+}
+
+// one block: l_c = sum_k Wp[c][k] v[k] + sum_k Wp[c][d + k] hD[k]; theta = 1 / (1 + exp(l_0 - l_1))
+__global__ void __launch_bounds__(256) cali_theta_kernel(PartView pv, const float *Wp, const float *hD, int d, float *theta) {
+    __shared__ float scratch[33];
+    pdl_trigger();
+    pdl_wait();
+    float l0 = 0.f, l1 = 0.f;
+    for (int k = threadIdx.x; k < d; k += blockDim.x) {
+        const float v = part_gather(pv, 0, k), h = hD[k];
+        l0 = fmaf(Wp[k], v, l0);
+        l0 = fmaf(Wp[d + k], h, l0);
+        l1 = fmaf(Wp[2 * d + k], v, l1);
+        l1 = fmaf(Wp[3 * d + k], h, l1);
+    }
+    l0 = block_sum(l0, scratch);
+    l1 = block_sum(l1, scratch);
+    if (threadIdx.x == 0) *theta = 1.0f / (1.0f + expf(l0 - l1));
+}
+void launch_cali_theta(cudaStream_t s, const PartView &pv, const float *Wp, const float *hD, int d, float *theta) {
+    launch_k(cali_theta_kernel, dim3(1), dim3(256), 0, s, pdl_enabled(), pv, Wp, hD, d, theta);
+}
+
 __global__ void reduce_partials_kernel(PartView pv, RowScale rs, float *out, int R) {
     const int m = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;
     pdl_trigger();

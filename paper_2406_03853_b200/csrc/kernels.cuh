@@ -91,6 +91,11 @@ size_t attention_prompt_scratch_floats(int ctx_len, int page_tokens, int H, int 
 void launch_attention_prompt(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                              const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
                              int Mtot, int pos0, int H, int *err);
+// H^(T) of the calibration predictor: row `row` (or row *row_dev when row_dev is given) of x[.][d]
+// is copied to hT (fp32) and, if xs is given, written as two bf16 terms into a one-chunk [32][d] matrix
+void launch_copy_row(cudaStream_t s, const float *x, int row, const int32_t *row_dev, float *hT, void *xs, int d);
+// theta_M = softmax(Wp [v ; hD])[1] with v = the d partial results of W^i H^(T) (Eq. 5)
+void launch_cali_theta(cudaStream_t s, const PartView &pv, const float *Wp, const float *hD, int d, float *theta);
 void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F);
 void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R);
 // programmatic dependent launch (kernels start early and wait on-device for their producer):
