@@ -44,7 +44,7 @@ class Layout(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in
                 ("embed", "layer0", "layer_stride", "off_g_attn", "off_wqkv", "off_wo", "off_g_ffn", "off_wgu",
                  "off_wd", "final_norm", "lm_head", "exit_layer", "exit_norm", "exit_head", "cali_w", "cali_wp",
-                 "total_bytes")]
+                 "total_bytes", "tiled")]
 
 
 class Sizes(C.Structure):
@@ -157,6 +157,27 @@ def make_config(*, d_model, n_heads, n_kv_heads, head_dim, ffn_dim, vocab, n_lay
                   ts_update_rule, cali_sigma_m, cali_sigma_s, cali_theta0)
 
 
+class TiledMatrix:
+    """A weight matrix [R, K] (or a stack [n, R, K]) stored tile-major in the weight buffer:
+    [R/128][K/64] tiles of [128][64] elements (eesd_layout.tiled).  `copy_` takes the matrix in
+    its usual [.., R, K] form and places every element in its tile; `dense()` reads it back."""
+
+    def __init__(self, flat: torch.Tensor, shape: Sequence[int]):
+        *lead, R, K = shape
+        assert R % 128 == 0 and K % 64 == 0
+        self.shape = tuple(shape)
+        n = len(lead)
+        # storage order [.., R/128, K/64, 128, 64]; seen as [.., R/128, 128, K/64, 64]
+        self._v = flat.view(*lead, R // 128, K // 64, 128, 64).permute(*range(n), n, n + 2, n + 1, n + 3)
+
+    def copy_(self, t: torch.Tensor):
+        self._v.copy_(t.reshape(self._v.shape))
+        return self
+
+    def dense(self) -> torch.Tensor:
+        return self._v.reshape(self.shape)
+
+
 class Engine:
     """One EESD context over torch-allocated device buffers (eesd_init .. eesd_destroy)."""
 
@@ -205,6 +226,14 @@ class Engine:
         n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
         return self.weights[off:off + n].view(dtype).view(*shape)
 
+    def _matrix(self, off: int, shape: Sequence[int]):
+        """A projection matrix of the weight buffer: a plain tensor view when the layout is
+        row-major, a TiledMatrix (same `copy_`) when it is tile-major."""
+        if not self.layout.tiled:
+            return self._view(off, shape, self.wdtype)
+        n = int(np.prod(shape)) * torch.empty((), dtype=self.wdtype).element_size()
+        return TiledMatrix(self.weights[off:off + n].view(self.wdtype), shape)
+
     def layer_views(self, l: int) -> Dict[str, torch.Tensor]:
         """Tensors aliasing target layer l (l == n_layers: the early-exit layer)."""
         c, lay = self.cfg, self.layout
@@ -212,11 +241,11 @@ class Engine:
         qd, kvd = c.n_heads * c.head_dim, c.n_kv_heads * c.head_dim
         return {
             "g_attn": self._view(base + lay.off_g_attn, (c.d_model,), torch.float32),
-            "wqkv": self._view(base + lay.off_wqkv, (qd + 2 * kvd, c.d_model), self.wdtype),
-            "wo": self._view(base + lay.off_wo, (c.d_model, qd), self.wdtype),
+            "wqkv": self._matrix(base + lay.off_wqkv, (qd + 2 * kvd, c.d_model)),
+            "wo": self._matrix(base + lay.off_wo, (c.d_model, qd)),
             "g_ffn": self._view(base + lay.off_g_ffn, (c.d_model,), torch.float32),
-            "wgu": self._view(base + lay.off_wgu, (2 * c.ffn_dim, c.d_model), self.wdtype),
-            "wd": self._view(base + lay.off_wd, (c.d_model, c.ffn_dim), self.wdtype),
+            "wgu": self._matrix(base + lay.off_wgu, (2 * c.ffn_dim, c.d_model)),
+            "wd": self._matrix(base + lay.off_wd, (c.d_model, c.ffn_dim)),
         }
 
     def global_views(self) -> Dict[str, torch.Tensor]:
@@ -224,12 +253,12 @@ class Engine:
         v = {
             "embed": self._view(lay.embed, (c.vocab, c.d_model), self.wdtype),
             "g_final": self._view(lay.final_norm, (c.d_model,), torch.float32),
-            "lm_head": self._view(lay.lm_head, (c.vocab, c.d_model), self.wdtype),
+            "lm_head": self._matrix(lay.lm_head, (c.vocab, c.d_model)),
             "g_exit": self._view(lay.exit_norm, (c.d_model,), torch.float32),
-            "exit_head": self._view(lay.exit_head, (c.vocab, c.d_model), self.wdtype),
+            "exit_head": self._matrix(lay.exit_head, (c.vocab, c.d_model)),
         }
         if c.controller == CTRL_CALI_TS:   # predictor of the calibrated controller: W^1..W^10 and W_p
-            v["cali_w"] = self._view(lay.cali_w, (10, c.d_model, c.d_model), self.wdtype)
+            v["cali_w"] = self._matrix(lay.cali_w, (10, c.d_model, c.d_model))
             v["cali_wp"] = self._view(lay.cali_wp, (2, 2 * c.d_model), torch.float32)
         return v
 

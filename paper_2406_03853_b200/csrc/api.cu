@@ -64,7 +64,7 @@ constexpr int kPrefillRows = 512; // most prompt rows per pass of the wide (prom
 
 bool tc_shapes_ok(const eesd_config *c) {
     const int qd = c->n_heads * c->head_dim, kvd = c->n_kv_heads * c->head_dim;
-    return c->dtype == EESD_BF16 && tc_shape_ok(qd + 2 * kvd, c->d_model) && tc_shape_ok(c->d_model, qd) &&
+    return c->dtype == EESD_BF16 && qd % 128 == 0 && tc_shape_ok(qd + 2 * kvd, c->d_model) && tc_shape_ok(c->d_model, qd) &&
            tc_shape_ok(2 * c->ffn_dim, c->d_model) && tc_shape_ok(c->d_model, c->ffn_dim) &&
            tc_shape_ok(2 * kvd, c->d_model) && tc_shape_ok(c->vocab, c->d_model);
 }
@@ -267,7 +267,7 @@ PartView run_proj(eesd_ctx *c, const void *W, const CUtensorMap *mW, int shape, 
     if (c->use_tc) {
         pv.mode = 1;
         pv.sk = c->plan[shape];
-        launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, c->plan[shape], M, c->err);
+        launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, c->plan[shape], M, true, c->err);
     } else {
         const float *A = which == X_NORM ? c->xn : which == X_ATTN ? c->attn : which == X_FFN ? c->h : c->hT;
         pv.mode = 0;
@@ -361,7 +361,7 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
     RowScale rs = norm_scale(c);
     rs.ssq = c->wssq;
     auto proj = [&](const CUtensorMap &mW, int which, int R, int K) {
-        launch_gemm_wide(s, mW, c->m_wx[which], c->wout, R, K, Mtot, c->n_sm, c->err);
+        launch_gemm_wide(s, mW, c->m_wx[which], c->wout, R, K, Mtot, c->n_sm, true, c->err);
         c->launches++;
         PartView pv = {};
         pv.base = c->wout; pv.mode = 0; pv.S = 1; pv.R = R; pv.split_stride = 0;
@@ -648,6 +648,7 @@ int eesd_weight_layout(const eesd_config *c, eesd_layout *out) {
         out->cali_wp = take(4 * d * 4);
     }
     out->total_bytes = o;
+    out->tiled = tc_shapes_ok(c) ? 1 : 0;
     return EESD_OK;
 }
 
@@ -707,6 +708,10 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     }
     const int qd_ = cfg->n_heads * cfg->head_dim, kvd_ = cfg->n_kv_heads * cfg->head_dim;
     c->use_tc = tc_shapes_ok(cfg) && tc_init() == 0;
+    if (lay.tiled && !c->use_tc) {   // tile-major weights are only read by the tensor-core kernels
+        delete c;
+        return EESD_ERR_UNSUPPORTED;
+    }
     c->wide_rows = c->use_tc ? prefill_rows(cfg) : 0;
     const char *wb = (const char *)b->weights;
     c->layers.resize(cfg->n_layers + 1);
@@ -725,20 +730,20 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         c->xs[X_CALI] = ws + w.xs_cali;
         if (c->cali_w && tc_shape_ok(d, d)) {
             ok = ok && tc_make_map(&c->m_x[X_CALI], c->xs[X_CALI], R2, d, R2);
-            for (int i = 0; i < 10; i++) ok = ok && tc_make_map(&c->m_cali[i], c->cali_w + (size_t)i * d * d * 2, d, d, 128);
+            for (int i = 0; i < 10; i++) ok = ok && tc_make_map(&c->m_cali[i], c->cali_w + (size_t)i * d * d * 2, d, d, 128, true);
         }
         ok = ok && tc_make_map(&c->m_x[X_NORM], c->xs[X_NORM], R2, d, R2);
         ok = ok && tc_make_map(&c->m_x[X_ATTN], c->xs[X_ATTN], R2, qd_, R2);
         ok = ok && tc_make_map(&c->m_x[X_FFN], c->xs[X_FFN], R2, F, R2);
         for (auto &lw : c->layers) {
-            ok = ok && tc_make_map(&lw.m_qkv, lw.wqkv, qd_ + 2 * kvd_, d, 128);
-            ok = ok && tc_make_map(&lw.m_o, lw.wo, d, qd_, 128);
-            ok = ok && tc_make_map(&lw.m_gu, lw.wgu, 2 * F, d, 128);
-            ok = ok && tc_make_map(&lw.m_d, lw.wd, d, F, 128);
+            ok = ok && tc_make_map(&lw.m_qkv, lw.wqkv, qd_ + 2 * kvd_, d, 128, true);
+            ok = ok && tc_make_map(&lw.m_o, lw.wo, d, qd_, 128, true);
+            ok = ok && tc_make_map(&lw.m_gu, lw.wgu, 2 * F, d, 128, true);
+            ok = ok && tc_make_map(&lw.m_d, lw.wd, d, F, 128, true);
         }
-        ok = ok && tc_make_map(&c->m_exit_kv, c->layers[cfg->n_layers].wqkv + (size_t)qd_ * d * 2, 2 * kvd_, d, 128);
-        ok = ok && tc_make_map(&c->m_lm_head, c->lm_head, cfg->vocab, d, 128);
-        ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128);
+        ok = ok && tc_make_map(&c->m_exit_kv, c->layers[cfg->n_layers].wqkv + (size_t)qd_ * d * 2, 2 * kvd_, d, 128, true);
+        ok = ok && tc_make_map(&c->m_lm_head, c->lm_head, cfg->vocab, d, 128, true);
+        ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128, true);
         if (c->wide_rows) {
             c->wx = (float *)(ws + w.wx); c->wout = (float *)(ws + w.wout); c->wssq = (float *)(ws + w.wssq);
             c->wtok = (int32_t *)(ws + w.wtok); c->wapart = (float *)(ws + w.wapart);
@@ -1134,7 +1139,7 @@ int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *
         launch_split_rows(s, A, sc + off_xs, M, K);
         pv.mode = 1;
         pv.sk = sk;
-        launch_gemm_tc(s, mW, mX, part, sk, M, (int *)sc);
+        launch_gemm_tc(s, mW, mX, part, sk, M, false, (int *)sc);
     } else {
         pv.mode = 0;
         pv.S = launch_gemm(s, dtype, A, W, part, M, R, K);

@@ -145,7 +145,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *r) {
 
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-               float *__restrict__ part, StreamK sk, int M, int *err) {
+               float *__restrict__ part, StreamK sk, int M, int tiled, int *err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sbase = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sW = sbase;
@@ -188,7 +188,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             for (int i = 0; i < pre; i++) {
                 const int u = u0 + i, tile = u / sk.KB, kb = u - tile * sk.KB;
                 mbar_expect_tx(&full[i], STAGE_BYTES);
-                tma_load_2d_hint(sW + i * STAGE_W, &tmW, &full[i], kb * BK, tile * BM, stream_once);
+                tma_load_2d_hint(sW + i * STAGE_W, &tmW, &full[i], tiled ? 0 : kb * BK, tiled ? (tile * sk.KB + kb) * BM : tile * BM, stream_once);
             }
             pdl_wait();
             for (int i = 0; i < pre; i++) {
@@ -203,7 +203,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 if (!ok) break;
                 const int tile = u / sk.KB, kb = u - tile * sk.KB;
                 mbar_expect_tx(&full[s], STAGE_BYTES);
-                tma_load_2d_hint(sW + s * STAGE_W, &tmW, &full[s], kb * BK, tile * BM, stream_once);
+                tma_load_2d_hint(sW + s * STAGE_W, &tmW, &full[s], tiled ? 0 : kb * BK, tiled ? (tile * sk.KB + kb) * BM : tile * BM, stream_once);
                 tma_load_2d(sX + s * STAGE_X, &tmX, &full[s], kb * BK, 0);
             }
             if (*abort_flag) {
@@ -326,7 +326,7 @@ __device__ __forceinline__ void mma_bf16_wide(uint32_t tmem_d, uint64_t da, uint
 
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                 float *__restrict__ out, int R, int KB, int Mtot, int panels, int *err) {
+                 float *__restrict__ out, int R, int KB, int Mtot, int panels, int tiled, int *err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sbase = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sW = sbase;
@@ -367,7 +367,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
             auto w_load = [&](int i, int s) {
                 const int t = (int)blockIdx.x + (i / KB) * (int)gridDim.x, kb = i % KB;
                 mbar_expect_tx(&full[s], WSTAGE_BYTES);
-                tma_load_2d(sW + s * STAGE_W, &tmW, &full[s], kb * BK, (t / panels) * BM);
+                tma_load_2d(sW + s * STAGE_W, &tmW, &full[s], tiled ? 0 : kb * BK, tiled ? ((t / panels) * KB + kb) * BM : (t / panels) * BM);
             };
             auto x_load = [&](int i, int s) {
                 const int t = (int)blockIdx.x + (i / KB) * (int)gridDim.x, kb = i % KB, chunk0 = (t % panels) * (WROWS / 16);
@@ -491,12 +491,15 @@ static EncodeFn encode_fn() {
     return fn;
 }
 
-bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows) {
+bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows, bool tiled) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
     if (((uintptr_t)base & 15) || (cols % 8)) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    // tile-major storage: [rows / 128][cols / 64] tiles of [128][64], each 16 KB contiguous; seen
+    // by the copy engine as rows * cols / 64 rows of 64 elements, one box = one tile
+    if (tiled && (box_rows != tc::BM || rows % tc::BM || cols % tc::BK)) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)(tiled ? tc::BK : cols), (cuuint64_t)(tiled ? (size_t)rows * cols / tc::BK : rows)};
+    cuuint64_t strides[1] = {(cuuint64_t)(tiled ? tc::BK : cols) * 2};
     cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
@@ -547,16 +550,17 @@ int tc_init() {
 }
 
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
-                    int M, int *err) {
-    launch_k(tc::gemm_tc_kernel, dim3(sk.G), dim3(tc::THREADS), (size_t)tc::SMEM_BYTES, s, pdl_enabled(), mW, mX, part, sk, M, err);
+                    int M, bool tiled, int *err) {
+    launch_k(tc::gemm_tc_kernel, dim3(sk.G), dim3(tc::THREADS), (size_t)tc::SMEM_BYTES, s, pdl_enabled(), mW, mX, part, sk, M,
+             (int)tiled, err);
 }
 
 void launch_gemm_wide(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *out, int R, int K, int Mtot,
-                      int n_sm, int *err) {
+                      int n_sm, bool tiled, int *err) {
     const int panels = (Mtot + tc::WROWS - 1) / tc::WROWS;
     const int tiles = (R / tc::BM) * panels;
     launch_k(tc::gemm_wide_kernel, dim3(tiles < n_sm ? tiles : n_sm), dim3(tc::THREADS), (size_t)tc::WSMEM_BYTES, s, pdl_enabled(),
-             mW, mX, out, R, K / tc::BK, Mtot, panels, err);
+             mW, mX, out, R, K / tc::BK, Mtot, panels, (int)tiled, err);
 }
 
 // fp32 rows -> two bf16 terms: rows 0..15 hold hi = bf16(x), rows 16..31 hold lo = bf16(x - hi)

@@ -105,15 +105,16 @@ bool pdl_enabled();
 // tensor-core projection (gemm_tc.cu)
 int tc_init();                                   // once per process; 0 on success
 bool tc_shape_ok(int R, int K);
-bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows);
+// tiled: the matrix is stored tile-major, [rows / 128][cols / 64] tiles of [128][64] (box_rows must be 128)
+bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows, bool tiled = false);
 StreamK tc_plan(int R, int K, int n_sm);
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
-                    int M, int *err);
+                    int M, bool tiled, int *err);
 // wide projection for prompt processing: out[m][r] (fp32, row stride R) for m < Mtot rows kept
 // as [chunk of 16][hi | lo][16][K] bf16 (mX from tc_make_map_rows); R % 128 == 0, K % 64 == 0
 bool tc_make_map_rows(CUtensorMap *out, const void *base, int K, int chunks);
 void launch_gemm_wide(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *out, int R, int K, int Mtot,
-                      int n_sm, int *err);
+                      int n_sm, bool tiled, int *err);
 void launch_split_rows(cudaStream_t s, const float *x, void *xs, int M, int K);
 
 // acceptance / sampling (accept.cu)

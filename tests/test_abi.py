@@ -41,6 +41,14 @@ def test_layout_sizes_and_config_checks(L):
         assert sz.kv_page_bytes == (spec.n_layers + 1) * 2 * spec.kv_dim * 16 * es
         assert sz.min_pages == 96
         assert (lay.exit_head == lay.lm_head) == spec.tie_exit_head
+        assert lay.tiled == (0 if spec.dtype == "f32" else 1)      # bf16 models with tile-aligned shapes: tile-major matrices
+        assert lay.cali_w == 0 and lay.cali_wp == 0
+        cfg.controller, cfg.cali_sigma_m, cfg.cali_sigma_s = b.CTRL_CALI_TS, 0.2, 0.5
+        lay2 = b.Layout()
+        assert L.eesd_weight_layout(C.byref(cfg), C.byref(lay2)) == 0
+        assert lay2.cali_w >= lay.total_bytes and lay2.total_bytes - lay.total_bytes >= (10 * spec.d_model ** 2) * es + 16 * spec.d_model
+        cfg.cali_sigma_s = 0.0
+        assert L.eesd_weight_layout(C.byref(cfg), C.byref(lay2)) == -1
     bad = config_from_spec(synth.TINY)
     bad.n_kv_heads = 3
     assert L.eesd_weight_layout(C.byref(bad), C.byref(lay)) == -1
@@ -51,6 +59,20 @@ def test_layout_sizes_and_config_checks(L):
     assert L.eesd_required_bytes(C.byref(bad), C.byref(sz)) == -1
     assert L.eesd_strerror(-5).decode().startswith("context")
     assert L.eesd_prefill(None, None, 0) == -1 and L.eesd_generate(None, None, 0, 0, None, 0, None, None, None, None, 0, None) == -1
+
+
+def test_tile_major_matrix_places_elements_where_the_header_says():
+    import torch
+    from paper_2406_03853_b200 import binding as b
+    R, K = 256, 192
+    flat = torch.zeros(2 * R * K)
+    t = torch.arange(2 * R * K, dtype=torch.float32).view(2, R, K)
+    m = b.TiledMatrix(flat, (2, R, K))
+    m.copy_(t)
+    for n, r, k in ((0, 0, 0), (0, 5, 70), (1, 129, 63), (1, 255, 191), (0, 128, 64)):
+        pos = n * R * K + ((r // 128 * (K // 64) + k // 64) * 128 + r % 128) * 64 + k % 64
+        assert flat[pos].item() == t[n, r, k].item()
+    assert torch.equal(m.dense(), t)
 
 
 def test_binding_refuses_to_run_without_cuda():
