@@ -53,7 +53,7 @@ int check_config(const eesd_config *c) {
 
 struct Workspace {
     size_t x, xn, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
-        accept, wx, wout, wxs[3], wssq, wtok, wapart, hT, xs_cali, theta, total;
+        accept, wx, wout, wout_floats, wxs[3], wssq, wtok, wapart, hT, xs_cali, theta, total;
 };
 
 constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
@@ -119,7 +119,7 @@ Workspace carve(const eesd_config *c) {
     w.hT = take((size_t)c->d_model * 4);
     w.xs_cali = take(2 * R * (size_t)c->d_model * 2);
     w.theta = take(16);
-    w.wx = w.wout = w.wssq = w.wtok = w.wapart = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
+    w.wx = w.wout = w.wout_floats = w.wssq = w.wtok = w.wapart = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
     if (const size_t P = (size_t)prefill_rows(c)) {
         // prompt path: residual stream, one projection result, the three activation matrices as
         // two bf16 terms ([chunk of 16][hi | lo][16][K]), RMSNorm statistics, token ids
@@ -128,6 +128,7 @@ Workspace carve(const eesd_config *c) {
         if ((size_t)c->d_model > wideR) wideR = c->d_model;
         w.wx = take(P * c->d_model * 4);
         w.wout = take(P * wideR * 4);
+        w.wout_floats = P * wideR;
         w.wxs[X_NORM] = take(2 * P * (size_t)c->d_model * 2);
         w.wxs[X_ATTN] = take(2 * P * qd * 2);
         w.wxs[X_FFN] = take(2 * P * (size_t)c->ffn_dim * 2);
@@ -169,6 +170,7 @@ struct eesd_ctx {
     // prompt (wide) path: up to wide_rows prompt rows per pass
     int wide_rows;
     float *wx, *wout, *wssq, *wapart;
+    size_t wout_floats;          // room in wout
     void *wxs[3];
     int32_t *wtok;
     CUtensorMap m_wx[3];
@@ -361,10 +363,12 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
     RowScale rs = norm_scale(c);
     rs.ssq = c->wssq;
     auto proj = [&](const CUtensorMap &mW, int which, int R, int K) {
-        launch_gemm_wide(s, mW, c->m_wx[which], c->wout, R, K, Mtot, c->n_sm, true, c->err);
+        // narrow results (O, down, exit keys/values) leave SMs idle in the last wave: split their k range
+        const int S = gemm_wide_splits(R, K, Mtot, c->n_sm, (int)(c->wout_floats / ((size_t)c->wide_rows * R)));
+        launch_gemm_wide(s, mW, c->m_wx[which], c->wout, R, K, Mtot, c->n_sm, true, S, c->err);
         c->launches++;
         PartView pv = {};
-        pv.base = c->wout; pv.mode = 0; pv.S = 1; pv.R = R; pv.split_stride = 0;
+        pv.base = c->wout; pv.mode = 0; pv.S = S; pv.R = R; pv.split_stride = (size_t)Mtot * R;
         return pv;
     };
     auto resid = [&](const PartView *pv, const float *g) {
@@ -745,7 +749,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         ok = ok && tc_make_map(&c->m_lm_head, c->lm_head, cfg->vocab, d, 128, true);
         ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128, true);
         if (c->wide_rows) {
-            c->wx = (float *)(ws + w.wx); c->wout = (float *)(ws + w.wout); c->wssq = (float *)(ws + w.wssq);
+            c->wx = (float *)(ws + w.wx); c->wout = (float *)(ws + w.wout); c->wout_floats = w.wout_floats; c->wssq = (float *)(ws + w.wssq);
             c->wtok = (int32_t *)(ws + w.wtok); c->wapart = (float *)(ws + w.wapart);
             const int ks[3] = {d, qd_, F};
             for (int i = 0; i < 3; i++) {

@@ -326,7 +326,7 @@ __device__ __forceinline__ void mma_bf16_wide(uint32_t tmem_d, uint64_t da, uint
 
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                 float *__restrict__ out, int R, int KB, int Mtot, int panels, int tiled, int *err) {
+                 float *__restrict__ out, int R, int KB, int Mtot, int panels, int tiled, int S, size_t split_stride, int *err) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sbase = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sW = sbase;
@@ -339,9 +339,12 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_tiles = (R / BM) * panels;
-    const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // tiles cta, cta + G, ...
-    const int n_units = my_tiles * KB;
+    // work item = (tile, k split): item t covers k blocks [ks * KBs, (ks + 1) * KBs) of tile t / S and
+    // writes its sums to out + ks * split_stride (the consumers add the S results)
+    const int KBs = KB / S;
+    const int n_tiles = (R / BM) * panels * S;
+    const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // items cta, cta + G, ...
+    const int n_units = my_tiles * KBs;
     pdl_trigger();
 
     if (tid == 0) {
@@ -365,12 +368,13 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
         if (lane == 0) {
             // unit i of this CTA -> (tile, k block)
             auto w_load = [&](int i, int s) {
-                const int t = (int)blockIdx.x + (i / KB) * (int)gridDim.x, kb = i % KB;
+                const int it = (int)blockIdx.x + (i / KBs) * (int)gridDim.x, t = it / S, kb = (it % S) * KBs + i % KBs;
                 mbar_expect_tx(&full[s], WSTAGE_BYTES);
                 tma_load_2d(sW + s * STAGE_W, &tmW, &full[s], tiled ? 0 : kb * BK, tiled ? ((t / panels) * KB + kb) * BM : (t / panels) * BM);
             };
             auto x_load = [&](int i, int s) {
-                const int t = (int)blockIdx.x + (i / KB) * (int)gridDim.x, kb = i % KB, chunk0 = (t % panels) * (WROWS / 16);
+                const int it = (int)blockIdx.x + (i / KBs) * (int)gridDim.x, t = it / S, kb = (it % S) * KBs + i % KBs;
+                const int chunk0 = (t % panels) * (WROWS / 16);
                 tma_load_4d(sX + s * WSTAGE_X, &tmX, &full[s], kb * BK, 0, 0, chunk0);
                 tma_load_4d(sX + s * WSTAGE_X + WSTAGE_X / 2, &tmX, &full[s], kb * BK, 0, 1, chunk0);
             };
@@ -400,8 +404,8 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
             int it = 0, sub = 0;
             bool ok = true;
             for (int seg = 0; seg < my_tiles && ok; seg++) {
-                for (int c0 = 0; c0 < KB && ok; c0 += KSEG, sub++) {
-                    const int c1 = min(KB, c0 + KSEG);
+                for (int c0 = 0; c0 < KBs && ok; c0 += KSEG, sub++) {
+                    const int c1 = min(KBs, c0 + KSEG);
                     const int b = sub & 1, use = sub >> 1;
                     ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag);
                     if (!ok) break;
@@ -430,11 +434,11 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
         bool ok = true;
         int sub = 0;
         for (int seg = 0; seg < my_tiles && ok; seg++) {
-            const int t = (int)blockIdx.x + seg * (int)gridDim.x, wt = t / panels, pn = t % panels;
+            const int it = (int)blockIdx.x + seg * (int)gridDim.x, t = it / S, ks = it % S, wt = t / panels, pn = t % panels;
             float acc[WROWS];   // this thread's weight row against the panel's 128 token rows
 #pragma unroll
             for (int i = 0; i < WROWS; i++) acc[i] = 0.f;
-            for (int c0 = 0; c0 < KB; c0 += KSEG, sub++) {
+            for (int c0 = 0; c0 < KBs; c0 += KSEG, sub++) {
                 const int b = sub & 1, use = sub >> 1;
                 ok = mbar_wait(&acc_full[b], use & 1, abort_flag, 64);
                 ok = __all_sync(0xffffffffu, ok);
@@ -456,7 +460,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                 if (lane == 0) mbar_arrive(&acc_empty[b]);
             }
             if (!ok) break;
-            float *dst = out + (size_t)(pn * WROWS) * R + (size_t)wt * BM + warp * 32 + lane;
+            float *dst = out + (size_t)ks * split_stride + (size_t)(pn * WROWS) * R + (size_t)wt * BM + warp * 32 + lane;
             const int rows_left = Mtot - pn * WROWS;
 #pragma unroll
             for (int i = 0; i < WROWS; i++)
@@ -555,12 +559,25 @@ void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX
              (int)tiled, err);
 }
 
+int gemm_wide_splits(int R, int K, int Mtot, int n_sm, int max_splits) {
+    const int panels = (Mtot + tc::WROWS - 1) / tc::WROWS, tiles = (R / tc::BM) * panels, KB = K / tc::BK;
+    int best = 1;
+    double cost = 1e30;
+    for (int S = 1; S <= max_splits && S <= 4; S++) {
+        if (KB % S) continue;
+        const int G = tiles * S < n_sm ? tiles * S : n_sm;
+        const double c = (double)((tiles * S + G - 1) / G) / S + 0.02 * (S - 1);   // waves of 1/S of a tile, a little for each extra result
+        if (c < cost - 1e-9) { cost = c; best = S; }
+    }
+    return best;
+}
+
 void launch_gemm_wide(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *out, int R, int K, int Mtot,
-                      int n_sm, bool tiled, int *err) {
+                      int n_sm, bool tiled, int splits, int *err) {
     const int panels = (Mtot + tc::WROWS - 1) / tc::WROWS;
-    const int tiles = (R / tc::BM) * panels;
+    const int tiles = (R / tc::BM) * panels * splits;
     launch_k(tc::gemm_wide_kernel, dim3(tiles < n_sm ? tiles : n_sm), dim3(tc::THREADS), (size_t)tc::WSMEM_BYTES, s, pdl_enabled(),
-             mW, mX, out, R, K / tc::BK, Mtot, panels, (int)tiled, err);
+             mW, mX, out, R, K / tc::BK, Mtot, panels, (int)tiled, splits, (size_t)Mtot * R, err);
 }
 
 // fp32 rows -> two bf16 terms: rows 0..15 hold hi = bf16(x), rows 16..31 hold lo = bf16(x - hi)

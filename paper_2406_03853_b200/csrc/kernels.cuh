@@ -113,8 +113,11 @@ void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX
 // wide projection for prompt processing: out[m][r] (fp32, row stride R) for m < Mtot rows kept
 // as [chunk of 16][hi | lo][16][K] bf16 (mX from tc_make_map_rows); R % 128 == 0, K % 64 == 0
 bool tc_make_map_rows(CUtensorMap *out, const void *base, int K, int chunks);
+// splits > 1: the k range is cut into `splits` parts whose results land Mtot * R floats apart (PartView
+// mode 0 with S = splits); gemm_wide_splits picks the count that fills the SMs best (at most max_splits)
+int gemm_wide_splits(int R, int K, int Mtot, int n_sm, int max_splits);
 void launch_gemm_wide(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *out, int R, int K, int Mtot,
-                      int n_sm, bool tiled, int *err);
+                      int n_sm, bool tiled, int splits, int *err);
 void launch_split_rows(cudaStream_t s, const float *x, void *xs, int M, int K);
 
 // acceptance / sampling (accept.cu)
