@@ -1,6 +1,7 @@
 // Host-callable launchers of the EESD model kernels.  `dtype` is EESD_F32 (0) or EESD_BF16 (1)
-// and selects the element type of the weights and of the KV cache; the residual stream, the
-// token rows fed to projections, partial sums, attention statistics and logits are fp32.
+// and selects the element type of the weights and of the KV cache; the residual stream, partial
+// sums, attention statistics and logits are fp32; the token rows fed to the tensor-core
+// projections are fp32 values carried as two bf16 terms.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -59,10 +60,9 @@ void launch_set_ints(cudaStream_t s, int32_t *dst, const IntList16 &vals, int n)
 void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float theta);
 void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
                   int M, int d, int V, int *err);
-// x[m] += sum_s part[s][m] (if part); xn[m] = cast(RMSNorm(x[m]) * g) (if g); cap[m] = x[m] (if cap)
 // x[m] += partial sums (if pv); y = x[m] * g -> xn (fp32, may be null) and xs (two bf16 terms,
-// [32][d]: rows 0..15 hi, 16..31 lo, may be null); ssq[m][b] = sum of squares of block b of x[m];
-// cap[m] = x[m] (if cap)
+// [chunk of 16 rows][hi | lo][16][d], may be null); ssq[m][b] = sum of squares of block b (1024
+// columns) of x[m]; cap[m] = x[m] (if cap).  The RMSNorm scale itself is applied by the consumers.
 void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
                   float *ssq, int M, int d);
 // out[sp][m][r] = sum_{k in split sp} A[m][k] * W[r][k]; returns the number of K splits written
