@@ -461,9 +461,9 @@ def main():
     kv_len = WORKLOADS[args.workload][4]
     bv, bd = pass_bytes(spec, kv_len)
     vp = {}
-    for M in sorted({1, M_typ, 6, 11, 16}):   # 6 and 11: K = 5 (the paper's best fixed K for 13B) and K = k_cap
+    for M in sorted({1, 2, 4, 8, 16, M_typ, 6, 11}):   # 6 and 11: K = 5 (the paper's best fixed K for 13B) and K = k_cap
         ms = time_verify_pass(eng, spec, kv_len, M)
-        vp[f"M{M}"] = {"ms": round(ms, 4), "gbs": round(bv / (ms * 1e-3) / 1e9, 1),
+        vp[f"M{M}"] = {"ms": round(ms, 4), "ms_per_layer": round(ms / spec.n_layers, 5), "gbs": round(bv / (ms * 1e-3) / 1e9, 1),
                        "frac_of_measured_copy": round(bv / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
                        "frac_of_8tbs": round(bv / (ms * 1e-3) / 1e9 / 8000.0, 4)}
     s0 = {k: sum(st[k] for st in stats) for k in ("drafted", "accepted", "emitted", "rounds", "ms_draft", "ms_verify")}
