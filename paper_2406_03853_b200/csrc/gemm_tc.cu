@@ -7,7 +7,7 @@
 //   * persistent grid (one CTA per SM), work = (128-row weight tile, 64-wide k block) units
 //     dealt out as one contiguous, equal range per CTA ("stream-K"), so every SM streams the
 //     same number of bytes whatever R and K are;
-//   * a 10-stage TMA ring (16 KB weight tile + 4 KB token tile per stage, 128-byte swizzle)
+//   * an 8-stage TMA ring (16 KB weight tile + 4 KB token tile per stage, 128-byte swizzle)
 //     fed by one producer thread; nothing but mbarriers between HBM and the tensor core;
 //   * tcgen05.mma with the weight tile as the 128-row A operand and the token rows as the
 //     32-column B operand; fp32 accumulators in tensor memory, two buffers so the epilogue of
@@ -32,7 +32,7 @@ namespace eesd {
 namespace tc {
 
 constexpr int BM = 128, BK = 64, BN = 32;
-constexpr int STAGES = 10;
+constexpr int STAGES = 8;   // with tile-major weights 7 to 9 stages time alike, 10 and more are slower (measured)
 constexpr int STAGE_W = BM * BK * 2, STAGE_X = BN * BK * 2;
 constexpr int STAGE_BYTES = STAGE_W + STAGE_X;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
