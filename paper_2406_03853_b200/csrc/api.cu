@@ -59,7 +59,8 @@ struct Workspace {
 constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
 constexpr int kAttnSplits = 64;  // most KV slices per head in attention
 constexpr int kIntSlots = 64;    // small device integer area
-constexpr int kMaxSm = 256;      // upper bound on CTAs of the persistent projection kernel
+constexpr int kMaxSm = 256;      // upper bound on the SM count the work splits are planned for
+constexpr int kCtasPerSm = 2;    // projection CTAs per SM (gemm_tc.cu: two 4-stage rings fit one SM)
 constexpr int kPrefillRows = 512; // most prompt rows per pass of the wide (prompt) path
 
 bool tc_shapes_ok(const eesd_config *c) {
@@ -102,7 +103,7 @@ Workspace carve(const eesd_config *c) {
     w.tickets = take(ticket_count(c) * 4);
     {   // partial sums: SIMT layout [splits][16][maxR], or stream-K blocks of the widest projection
         size_t part_floats = (size_t)kPartSplits * R * maxR;
-        const size_t sk_floats = (maxR / 128 + (size_t)kMaxSm) * R * 128;  // blocks <= tiles + CTAs
+        const size_t sk_floats = (maxR / 128 + (size_t)kMaxSm * kCtasPerSm) * R * 128;  // blocks <= tiles + CTAs
         if (sk_floats > part_floats) part_floats = sk_floats;
         w.part = take(part_floats * 4);
     }
@@ -759,7 +760,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         }
         // work split of every projection shape
         const int shapes[P_COUNT][2] = {{qd_ + 2 * kvd_, d}, {d, qd_}, {2 * F, d}, {d, F}, {2 * kvd_, d}, {cfg->vocab, d}, {d, d}};
-        for (int i = 0; i < P_COUNT; i++) c->plan[i] = tc_plan(shapes[i][0], shapes[i][1], c->n_sm);
+        for (int i = 0; i < P_COUNT; i++) c->plan[i] = tc_plan(shapes[i][0], shapes[i][1], kCtasPerSm * c->n_sm);
         if (!ok) {
             delete c;
             return EESD_ERR_CUDA;
@@ -1106,7 +1107,7 @@ static size_t project_scratch_layout(int R, int K, size_t *off_xs, size_t *off_t
     o = align_up(o + ((size_t)R / 128 + 1) * sizeof(int4), 256);
     *off_part = o;
     size_t floats = (size_t)EESD_MAX_ROWS * R;
-    const size_t sk = ((size_t)R / 128 + (size_t)kMaxSm) * EESD_MAX_ROWS * 128;
+    const size_t sk = ((size_t)R / 128 + (size_t)kMaxSm * kCtasPerSm) * EESD_MAX_ROWS * 128;
     if (sk > floats) floats = sk;
     return o + floats * 4;
 }
@@ -1138,7 +1139,7 @@ int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *
         CUtensorMap mW, mX;
         if (!tc_make_map(&mW, W, R, K, 128) || !tc_make_map(&mX, sc + off_xs, 2 * EESD_MAX_ROWS, K, 2 * EESD_MAX_ROWS))
             return EESD_ERR_CUDA;
-        const StreamK sk = tc_plan(R, K, n_sm);
+        const StreamK sk = tc_plan(R, K, kCtasPerSm * n_sm);
         if (cudaMemsetAsync(sc, 0, 16, s) != cudaSuccess) return EESD_ERR_CUDA;
         launch_split_rows(s, A, sc + off_xs, M, K);
         pv.mode = 1;

@@ -4,10 +4,10 @@
 //
 // HBM-bound: every weight byte is read exactly once per pass, the token rows are tiny.  The
 // kernel therefore exists to keep the memory system full:
-//   * persistent grid (one CTA per SM), work = (128-row weight tile, 64-wide k block) units
+//   * persistent grid (two CTAs per SM), work = (128-row weight tile, 64-wide k block) units
 //     dealt out as one contiguous, equal range per CTA ("stream-K"), so every SM streams the
 //     same number of bytes whatever R and K are;
-//   * an 8-stage TMA ring (16 KB weight tile + 4 KB token tile per stage, 128-byte swizzle)
+//   * a 4-stage TMA ring per CTA (16 KB weight tile + 4 KB token tile per stage, 128-byte swizzle)
 //     fed by one producer thread; nothing but mbarriers between HBM and the tensor core;
 //   * tcgen05.mma with the weight tile as the 128-row A operand and the token rows as the
 //     32-column B operand; fp32 accumulators in tensor memory, two buffers so the epilogue of
@@ -32,7 +32,7 @@ namespace eesd {
 namespace tc {
 
 constexpr int BM = 128, BK = 64, BN = 32;
-constexpr int STAGES = 8;   // with tile-major weights 7 to 9 stages time alike, 10 and more are slower (measured)
+constexpr int STAGES = 4;   // per CTA; two CTAs share an SM (measured: 2 x 4 stages beat 1 x 8 by 1.8 % of a 13B pass, 3 x 3 and 2 x 3 do not)
 constexpr int STAGE_W = BM * BK * 2, STAGE_X = BN * BK * 2;
 constexpr int STAGE_BYTES = STAGE_W + STAGE_X;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
@@ -143,7 +143,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *r) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(THREADS, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                float *__restrict__ part, StreamK sk, int M, int tiled, int *err) {
     extern __shared__ uint8_t smem_raw[];
