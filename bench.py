@@ -493,7 +493,7 @@ def main():
                      "frac": round(achieved / peaks["hbm_gbs"], 4),
                      # dram__bytes_read + dram__bytes_write of one gate/up launch at the 13B shape, from the ncu
                      # capture summarised under profiles/ (null for other shapes: not captured)
-                     "traffic": 287219712 if (spec.name == "13b") else None,
+                     "traffic": 287024384 if (spec.name == "13b") else None,
                      "bytes_per_launch": kbytes, "ms_per_launch": round(kms, 5)},
         "verify_pass": {"kv_len": kv_len, "bytes": bv, **vp},
         "draft_step_bytes": bd,
