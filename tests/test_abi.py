@@ -26,6 +26,19 @@ def test_every_declared_symbol_is_exported(L):
         assert hasattr(L, n), n
 
 
+def test_header_is_plain_c(tmp_path):
+    import shutil
+    import subprocess
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "eesd.h"\nint main(void) { eesd_config c; (void)c; return EESD_OK; }\n')
+    gcc = shutil.which("gcc")
+    if not gcc:
+        pytest.skip("no C compiler")
+    r = subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(ROOT, "include"), "-fsyntax-only", str(src)],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+
+
 def test_layout_sizes_and_config_checks(L):
     from paper_2406_03853_b200 import binding as b
     import eesd_synth as synth
