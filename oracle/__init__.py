@@ -305,6 +305,55 @@ class OracleModel:
         return out, [(trace[i].k, trace[i].n_acc, trace[i].y) for i in range(n)], (a.value, b.value)
 
 
+    def generate_tree(self, prompt, max_new: int, *, width: int, fixed_k=4, k_schedule=None):
+        """Greedy EESD with tree verification (the tree-attention appendix: several draft
+        candidates per position, only the one equal to the target's top-1 token is kept).
+
+        The paper fixes no tree shape.  Reading taken here: the draft model's greedy chain
+        x_1..x_K, plus at every depth i the next `width - 1` best tokens of the same draft
+        distribution as leaves (ranked by logit, lower token id first among equals).  The target's
+        top-1 token after the accepted path so far is compared with the children at the next
+        depth: the chain token continues the walk, a leaf ends it (the target's top-1 after the
+        path ending in that leaf is the round's last token), neither ends it with the target's
+        own token.  Each "top-1 after a path" is taken by its definition: the target run on that
+        path.  Returns (tokens[max_new], trace[(k, n_acc, y)], leaves accepted); n_acc counts
+        accepted draft tokens, an accepted leaf included."""
+        ctx = [int(t) for t in prompt]
+        if len(ctx) > 1:
+            self.target_rows(np.array(ctx[:-1], np.int32), 0, want_logits=False)
+        n0, trace, leaves, rounds = len(ctx), [], 0, 0
+        while len(ctx) - n0 < max_new:
+            T = len(ctx)
+            K = int(k_schedule[rounds]) if k_schedule is not None and rounds < len(k_schedule) else fixed_k
+            K = max(1, min(K, (self.max_ctx - T) // width))
+            xs, sib = [ctx[-1]], []
+            for i in range(K):
+                lg = self.draft_row(xs[i], T - 1 + i)
+                order = np.argsort(-lg.astype(np.float64), kind="stable")[:width]   # equal logits: lower id first
+                xs.append(int(order[0]))
+                sib.append([int(v) for v in order[1:]])
+            _, pl = self.target_rows(np.array(xs, np.int32), T - 1)
+            top = [int(row.argmax()) for row in pl]   # target's token after the chain prefix x_0..x_i
+            accepted, y = xs[1:K + 1], top[K]
+            for i in range(1, K + 1):
+                want = top[i - 1]
+                if want == xs[i]:
+                    continue
+                if want in sib[i - 1]:
+                    # the path x_0..x_{i-1}, leaf: run the target on the leaf at its position (this
+                    # also leaves the leaf's keys / values there, in every layer and the exit layer)
+                    _, ps = self.target_rows(np.array([want], np.int32), T - 1 + i)
+                    accepted, y = xs[1:i] + [want], int(ps[0].argmax())
+                    leaves += 1
+                else:
+                    accepted, y = xs[1:i], want
+                break
+            ctx += accepted + [y]
+            trace.append((K, len(accepted), y))
+            rounds += 1
+        return np.array(ctx[n0:n0 + max_new], np.int32), trace, leaves
+
+
 def bf16_round(x: float) -> float:
     return float(lib().orc_bf16_round(float(x)))
 
