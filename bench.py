@@ -94,7 +94,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None, cali=False):
+def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None, cali=False, tree_width=0):
     from paper_2406_03853_b200 import Engine
     from paper_2406_03853_b200 import binding as b
     spec_name, n_prompt, max_new, damp, _ = WORKLOADS[wl]
@@ -106,8 +106,10 @@ def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_
     max_ctx = max(n_prompt + max_new + 16, 1024 + 32)
     cfg = b.make_config(d_model=spec.d_model, n_heads=spec.n_heads, n_kv_heads=spec.n_kv_heads, head_dim=spec.head_dim,
                         ffn_dim=spec.ffn_dim, vocab=spec.vocab, n_layers=spec.n_layers, n_early=spec.n_early,
-                        dtype=spec.dtype, tie_exit_head=spec.tie_exit_head, max_ctx=max_ctx, k_cap=10,
-                        temperature=temperature, controller=b.CTRL_CALI_TS if cali else controller, fixed_k=5, page_tokens=16)
+                        dtype=spec.dtype, tie_exit_head=spec.tie_exit_head, max_ctx=max_ctx,
+                        k_cap=10 if tree_width < 2 else 15 // tree_width,
+                        temperature=temperature, controller=b.CTRL_CALI_TS if cali else controller, fixed_k=5, page_tokens=16,
+                        tree_width=tree_width)
     eng = Engine(cfg, device=device)
     # synthetic weights, generated on the device by the shared seeded generator
     for l in range(spec.n_layers):
@@ -275,7 +277,9 @@ def run_sweep(args, device):
     Beta-TS controller (the paper's fixed-K curve against Thompson sampling); `--sweep n` rebuilds
     the model with the early exit after N = 1, 2, 3, 5, 8, 10 layers (the paper's N sweep; in the
     synthetic model the layers after N are the damped ones, so acceptance changes with N by
-    construction).  Each setting decodes `--steps` different seeded prompts."""
+    construction); `--sweep tree` decodes greedily with tree verification of width 1 (the chain),
+    2 and 3 at fixed draft lengths (the paper's table on tree attention: more candidates per
+    position, one verification pass).  Each setting decodes `--steps` different seeded prompts."""
     from paper_2406_03853_b200 import binding as b
     from paper_2406_03853_b200 import report
     spec_name, n_prompt, max_new, damp, kv_len = WORKLOADS[args.workload]
@@ -284,7 +288,7 @@ def run_sweep(args, device):
     def measure(eng, spec, label, k_schedule):
         u = {k: v.numpy() for k, v in synth.generate_uniforms(eng.cfg.max_ctx, 1 << 20).items()}
         tot = {"drafted": 0, "accepted": 0, "emitted": 0, "rounds": 0}
-        ms = 0.0
+        ms, leaves = 0.0, 0
         for i in range(args.steps):
             eng.prefill(synth.prompt_tokens(synth.SEED + i, n_prompt, spec.vocab).numpy())
             torch.cuda.synchronize()
@@ -295,12 +299,14 @@ def run_sweep(args, device):
             ms += e0.elapsed_time(e1)
             for k in tot:
                 tot[k] += st.as_dict()[k]
+            leaves += st.leaves_kept
         q = report.run_quality(tot["drafted"], tot["accepted"], tot["emitted"])
         t1 = time_verify_pass(eng, spec, kv_len, 1)
         tps = args.steps * max_new / (ms / 1e3)
         print(json.dumps({"sweep": args.sweep, "setting": label, "workload": args.workload, "tokens_per_s": round(tps, 2),
                           "speedup_vs_autoregressive": round(tps / (1e3 / t1), 4), "mean_k": round(tot["drafted"] / max(1, tot["rounds"]), 3),
                           "v_d": round(q["v_d"], 4), "r_d": round(q["r_d"], 4), "hm": round(q["hm"], 2),
+                          "leaves_kept_per_round": round(leaves / max(1, tot["rounds"]), 4),
                           "early_layers": spec.n_early, "damp_alpha": spec.damp, "steps": args.steps}), flush=True)
 
     if args.sweep == "k":
@@ -309,6 +315,14 @@ def run_sweep(args, device):
             measure(eng, spec, f"fixed K={K}", [K] * max_new)
         measure(eng, spec, "beta-ts", None)
         eng.close()
+    elif args.sweep == "tree":
+        for W in (1, 2, 3):
+            eng, spec, _, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, alpha=args.alpha, tree_width=W)
+            for K in (2, 3, 4, 5):
+                measure(eng, spec, f"width {W}, fixed K={K} ({1 + K * max(W, 1)} rows per pass)", [K] * max_new)
+            eng.close()
+            del eng
+            torch.cuda.empty_cache()
     else:
         for N in (1, 2, 3, 5, 8, 10):
             eng, spec, _, _ = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha, n_early=N)
@@ -364,7 +378,7 @@ def main():
                          "bracket, for ncu --profile-from-start off")
     ap.add_argument("--controller", choices=["beta", "cali"], default="beta",
                     help="draft-length controller: Beta-TS (default) or TS with calibration (random-init predictor)")
-    ap.add_argument("--sweep", choices=["k", "n"], default=None,
+    ap.add_argument("--sweep", choices=["k", "n", "tree"], default=None,
                     help="method sweep instead of the benchmark line: fixed K = 1..10 against Beta-TS, or the exit depth N")
     ap.add_argument("--profile-prefill", action="store_true",
                     help="only run one prompt pass inside a cudaProfilerStart/Stop region (for ncu)")

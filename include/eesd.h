@@ -77,6 +77,18 @@ typedef struct eesd_config {
      * the model's prediction, the assumed deviation of a round's sample mean, and the initial
      * observed mean theta_hat_0; sigmas must be positive */
     float cali_sigma_m, cali_sigma_s, cali_theta0;
+    /* Tree verification (appendix "Implement Tree Attention": several draft candidates per
+     * position, only the one equal to the target's top-1 token is kept).  0 or 1: off.  2..4:
+     * beside the draft's greedy chain x_1..x_K, the tree_width - 1 next-best tokens of each draft
+     * step (by logit, lower id first among equals) enter the verification pass as leaves of that
+     * depth; a leaf sees the cache, the chain before its depth and itself.  The target's top-1
+     * after the accepted path is compared with the candidates of the next depth: the chain token
+     * continues, a leaf is kept and ends the round (next token = the target's top-1 after that
+     * leaf), neither ends the round with the target's token.  The paper fixes no tree shape: this
+     * one is a choice.  Needs temperature 0, a controller other than EESD_CTRL_CALI_TS and
+     * 1 + k_cap * tree_width <= EESD_MAX_ROWS (else UNSUPPORTED / BADARG); a round of K drafts
+     * uses 1 + K * tree_width cache rows past the context before it is cut back. */
+    int32_t tree_width;
 } eesd_config;
 
 /* Byte offsets inside the weight buffer.  A decoder layer holds, in this order:
@@ -144,6 +156,7 @@ typedef struct eesd_stats {
     double ms_prefill, ms_draft, ms_verify, ms_total; /* device time, CUDA events               */
     int64_t kernel_launches;
     int64_t alpha, beta;                               /* posterior after the last round         */
+    int64_t leaves_kept;                               /* tree verification: rounds that kept a leaf */
 } eesd_stats;
 
 typedef struct eesd_ctx eesd_ctx;
@@ -216,6 +229,10 @@ int eesd_decode(eesd_ctx *ctx, int max_new, const int32_t *k_schedule, int n_sch
 
 /* Context length in tokens (including the pending one), and KV pages in use. */
 int eesd_context_len(const eesd_ctx *ctx, int *n_tokens, int *pages_in_use);
+/* Tokens first .. first + n - 1 of the context (prompt, accepted tokens, pending token) into
+ * out (host).  With tree verification this is how the step API shows which candidate a round
+ * kept.  BADARG if the range passes the end of the context. */
+int eesd_context_tokens(const eesd_ctx *ctx, int first, int n, int32_t *out);
 /* Posterior parameters of the controller. */
 int eesd_posterior(const eesd_ctx *ctx, int64_t *alpha, int64_t *beta);
 

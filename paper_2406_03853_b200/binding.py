@@ -37,7 +37,7 @@ class Config(C.Structure):
                 ("page_tokens", C.c_int32), ("max_ctx", C.c_int32), ("k_cap", C.c_int32), ("temperature", C.c_float),
                 ("controller", C.c_int32), ("fixed_k", C.c_int32), ("alpha0", C.c_int32), ("beta0", C.c_int32),
                 ("ts_update_rule", C.c_int32), ("cali_sigma_m", C.c_float), ("cali_sigma_s", C.c_float),
-                ("cali_theta0", C.c_float)]
+                ("cali_theta0", C.c_float), ("tree_width", C.c_int32)]
 
 
 class Layout(C.Structure):
@@ -69,7 +69,8 @@ class Round(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("rounds", C.c_int64), ("drafted", C.c_int64), ("accepted", C.c_int64), ("emitted", C.c_int64),
                 ("ms_prefill", C.c_double), ("ms_draft", C.c_double), ("ms_verify", C.c_double),
-                ("ms_total", C.c_double), ("kernel_launches", C.c_int64), ("alpha", C.c_int64), ("beta", C.c_int64)]
+                ("ms_total", C.c_double), ("kernel_launches", C.c_int64), ("alpha", C.c_int64), ("beta", C.c_int64),
+                ("leaves_kept", C.c_int64)]
 
     def as_dict(self) -> Dict:
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -104,6 +105,7 @@ def lib():
         L.eesd_decode.argtypes = [vp, C.c_int, vp, C.c_int, C.POINTER(Uniforms), vp, C.POINTER(Stats), vp, C.c_int,
                                   C.POINTER(C.c_int)]
         L.eesd_context_len.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        L.eesd_context_tokens.argtypes = [vp, C.c_int, C.c_int, vp]
         L.eesd_posterior.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.eesd_cali_predict.argtypes = [vp, C.POINTER(C.c_float)]
         L.eesd_cali_state.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
@@ -150,11 +152,11 @@ def _np_f32(a) -> np.ndarray:
 def make_config(*, d_model, n_heads, n_kv_heads, head_dim, ffn_dim, vocab, n_layers, n_early, dtype,
                 tie_exit_head=False, rms_eps=1e-5, rope_theta=10000.0, page_tokens=16, max_ctx=2048, k_cap=10,
                 temperature=0.0, controller=CTRL_FIXED_K, fixed_k=4, alpha0=1, beta0=1, ts_update_rule=0,
-                cali_sigma_m=0.2, cali_sigma_s=0.5, cali_theta0=0.5) -> Config:
+                cali_sigma_m=0.2, cali_sigma_s=0.5, cali_theta0=0.5, tree_width=0) -> Config:
     dt = {"f32": F32, "bf16": BF16}.get(dtype, dtype)
     return Config(d_model, n_heads, n_kv_heads, head_dim, ffn_dim, vocab, n_layers, n_early, dt, int(tie_exit_head),
                   rms_eps, rope_theta, page_tokens, max_ctx, k_cap, temperature, controller, fixed_k, alpha0, beta0,
-                  ts_update_rule, cali_sigma_m, cali_sigma_s, cali_theta0)
+                  ts_update_rule, cali_sigma_m, cali_sigma_s, cali_theta0, tree_width)
 
 
 class TiledMatrix:
@@ -342,6 +344,13 @@ class Engine:
         n, p = C.c_int(), C.c_int()
         self._check(lib().eesd_context_len(self.h, C.byref(n), C.byref(p)), "eesd_context_len")
         return n.value, p.value
+
+    def context_tokens(self, first: int = 0, n: Optional[int] = None) -> np.ndarray:
+        if n is None:
+            n = self.context_len()[0] - first
+        out = np.empty(n, np.int32)
+        self._check(lib().eesd_context_tokens(self.h, first, n, out.ctypes.data), "eesd_context_tokens")
+        return out
 
     def posterior(self):
         a, b = C.c_int64(), C.c_int64()

@@ -48,6 +48,11 @@ int check_config(const eesd_config *c) {
     if (c->controller == EESD_CTRL_FIXED_K && c->fixed_k < 1) return EESD_ERR_BADARG;
     if (c->alpha0 < 1 || c->beta0 < 1) return EESD_ERR_BADARG;
     if (c->rms_eps < 0.f || c->rope_theta <= 1.f) return EESD_ERR_BADARG;
+    if (c->tree_width < 0 || c->tree_width > 4) return EESD_ERR_BADARG;
+    if (c->tree_width > 1) {   // tree verification: greedy only, 1 + k_cap * width rows in one pass
+        if (c->temperature != 0.f || c->controller == EESD_CTRL_CALI_TS) return EESD_ERR_UNSUPPORTED;
+        if (1 + c->k_cap * c->tree_width > EESD_MAX_ROWS) return EESD_ERR_BADARG;
+    }
     return EESD_OK;
 }
 
@@ -58,7 +63,7 @@ struct Workspace {
 
 constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
 constexpr int kAttnSplits = 64;  // most KV slices per head in attention
-constexpr int kIntSlots = 64;    // small device integer area
+constexpr int kIntSlots = 128;   // small device integer area
 constexpr int kMaxSm = 256;      // upper bound on the SM count the work splits are planned for
 constexpr int kCtasPerSm = 2;    // projection CTAs per SM (gemm_tc.cu: two 4-stage rings fit one SM)
 constexpr int kPrefillRows = 512; // most prompt rows per pass of the wide (prompt) path
@@ -144,7 +149,9 @@ Workspace carve(const eesd_config *c) {
 // offsets inside the device integer area
 constexpr int kRoundTok = 0;   // [17]: pending token, then the round's draft tokens
 constexpr int kRowTok = 20;    // [16]: token rows of a prefill chunk / verify_only
-constexpr int kResult = 40;    // [2]: n_accept, next token
+constexpr int kResult = 40;    // [3]: n_accept, next token, row of the kept leaf (tree verification) or -1
+constexpr int kLeafTok = 64;   // [15]: tree verification: leaves of depth 1, depth 2, ... (width - 1 each)
+constexpr int kTreeTop = 80;   // [16]: tree verification: the target's top-1 token of every row
 
 }  // namespace
 
@@ -195,6 +202,10 @@ struct eesd_ctx {
     int round_k;
     int64_t alpha, beta;
     int64_t launches;
+    // tree verification: geometry of the pass being enqueued (null: a chain), leaves kept so far
+    const TreeRows *tree_cur;
+    TreeRows tree_rows;
+    int64_t leaves_kept;
     int32_t *h_result;  // pinned: [0] n_accept, [1] next token, [2] error word, [8..23] draft tokens
     cudaEvent_t ev[5];  // prefill start / end, draft start, verify start, round end
     char cuda_err[256];
@@ -230,6 +241,8 @@ KvGeom kv_geom(eesd_ctx *c, int slot) {
     g.n_pages_total = (int)c->n_pages_total;
     return g;
 }
+
+bool tree_on(const eesd_ctx *c) { return c->cfg.tree_width > 1; }
 
 // make sure pages exist for `n_tokens` cache rows; pushes new table entries to the device
 int ensure_pages(eesd_ctx *c, int n_tokens) {
@@ -305,7 +318,7 @@ void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const fl
     const RowScale rs = norm_scale(c);
     PartView pv = run_proj(c, w.wqkv, &w.m_qkv, P_QKV, X_NORM, M, qd + 2 * kvd, d);
     launch_attention(s, f.dtype, pv, rs, c->rope, kv_geom(c, slot), c->apart, c->tickets, c->use_tc ? nullptr : c->attn,
-                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, true, c->err);
+                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, true, c->err, c->tree_cur);
     pv = run_proj(c, w.wo, &w.m_o, P_O, X_ATTN, M, d, qd);
     run_resid(c, &pv, w.g_ffn, nullptr, M);
     pv = run_proj(c, w.wgu, &w.m_gu, P_GU, X_NORM, M, 2 * F, d);
@@ -337,7 +350,8 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
             const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim;
             const char *wkv = c->layers[L].wqkv + (size_t)qd * d * c->es;
             PartView pv = run_proj(c, wkv, &c->m_exit_kv, P_EXIT_KV, X_NORM, M, 2 * kvd, d);
-            launch_qkv_post(s, f.dtype, pv, norm_scale(c), M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err);
+            launch_qkv_post(s, f.dtype, pv, norm_scale(c), M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err, 0,
+                            c->tree_cur);
             const float *g_next = l + 1 < L ? c->layers[l + 1].g_attn : c->g_final;
             run_resid(c, nullptr, g_next, nullptr, M);
             c->launches += 1;
@@ -423,8 +437,15 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
     launch_reduce_partials(s, pv, norm_scale(c), lq, 1, f.vocab);
     launch_sample_rows(s, lq, d_u, 1, f.vocab, f.temperature, c->ints + kRoundTok + i + 1);
     c->launches += 3;
+    if (tree_on(c)) {   // the next-best candidates of this step become leaves of depth i + 1
+        launch_next_best(s, lq, f.vocab, f.tree_width, c->ints + kLeafTok + i * (f.tree_width - 1));
+        c->launches++;
+    }
     return check_launch(c);
 }
+
+// rows of a tree verification pass after K draft steps: chain rows 0..K, then the leaves by depth
+int tree_pass_rows(const eesd_ctx *c, int K) { return 1 + K * c->cfg.tree_width; }
 
 int set_device_ints(eesd_ctx *c, int slot, const int32_t *vals, int n) {
     IntList16 l;
@@ -551,6 +572,7 @@ int draft_impl(eesd_ctx *c, int k, const float *d_u, int u_stride) {
     const int T = (int)c->tokens.size();
     if (c->round_k + k > c->cfg.k_cap) return EESD_ERR_CTX_FULL;
     if (T + c->round_k + k > c->cfg.max_ctx - 1) return EESD_ERR_CTX_FULL;
+    if (tree_on(c) && T - 1 + tree_pass_rows(c, c->round_k + k) > c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
     int st = ensure_pages(c, T + c->round_k + k);
     if (st) return st;
     for (int j = 0; j < k; j++) {
@@ -562,10 +584,47 @@ int draft_impl(eesd_ctx *c, int k, const float *d_u, int u_stride) {
     return EESD_OK;
 }
 
+// Tree verification (greedy): one pass over the chain x_0..x_K and the width - 1 next-best
+// candidates of every depth as leaves; leaf j of depth i is row K + 1 + (i - 1)(width - 1) + j,
+// rotated as position T - 1 + i, and sees the cache, chain rows 0..i-1 and itself.  The target's
+// top-1 token of every row decides the walk; a kept leaf's keys / values then move from the
+// position of its row to the position of its depth in every layer and in the exit layer.
+int verify_tree_impl(eesd_ctx *c) {
+    const eesd_config &f = c->cfg;
+    const int T = (int)c->tokens.size(), K = c->round_k, W = f.tree_width, M = tree_pass_rows(c, K);
+    if (T - 1 + M > f.max_ctx) return EESD_ERR_CTX_FULL;
+    int st = ensure_pages(c, T - 1 + M);
+    if (st) return st;
+    TreeRows &tr = c->tree_rows;
+    tr = chain_rows();
+    for (int i = 1; i <= K; i++)
+        for (int j = 0; j < W - 1; j++) {
+            const int m = K + 1 + (i - 1) * (W - 1) + j;
+            tr.depth[m] = (uint8_t)i;
+            tr.vis[m] = (uint16_t)(((1u << i) - 1u) | (1u << m));
+        }
+    launch_tree_rows(c->stream, c->ints + kRoundTok, c->ints + kLeafTok, K, W, c->ints + kRowTok);
+    c->tree_cur = &tr;
+    st = run_target(c, c->ints + kRowTok, M, T - 1, true);
+    c->tree_cur = nullptr;
+    if (st) return st;
+    launch_sample_rows(c->stream, c->logits_p, nullptr, M, f.vocab, 0.f, c->ints + kTreeTop);
+    launch_tree_walk(c->stream, c->ints + kTreeTop, c->ints + kRoundTok, c->ints + kLeafTok, K, W, c->ints + kResult);
+    launch_kv_move(c->stream, f.dtype, kv_geom(c, 0), c->slot_bytes, f.n_layers + 1, T - 1, c->ints + kResult, c->err);
+    c->launches += 4;
+    st = check_launch(c);
+    if (st) return st;
+    CU(c, cudaMemcpyAsync(c->h_result, c->ints + kResult, 8, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaMemcpyAsync(c->h_result + 2, c->err, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaMemcpyAsync(c->h_result + 3, c->ints + kResult + 2, 4, cudaMemcpyDeviceToHost, c->stream));
+    return EESD_OK;
+}
+
 // verify pass + acceptance; leaves (n_accept, next token, error word) in h_result after a sync
 int verify_impl(eesd_ctx *c, const float *d_u_acc, const float *d_u_res) {
     const eesd_config &f = c->cfg;
     const int T = (int)c->tokens.size(), K = c->round_k;
+    if (tree_on(c)) return verify_tree_impl(c);
     int st = ensure_pages(c, T + K);
     if (st) return st;
     st = run_target(c, c->ints + kRoundTok, K + 1, T - 1, true);
@@ -592,6 +651,7 @@ int finish_round(eesd_ctx *c, const int32_t *draft_tokens_host, int *n_accept, i
     }
     for (int i = 0; i < a; i++) c->tokens.push_back(draft_tokens_host[i]);
     c->tokens.push_back(y);
+    if (tree_on(c) && c->h_result[3] >= 0) c->leaves_kept++;
     c->round_k = 0;
     trim_pages(c, (int)c->tokens.size() - 1);  // rows of rejected tokens are dropped
     if (n_accept) *n_accept = a;
@@ -690,6 +750,8 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->cuda_err[0] = 0;
     c->capture = nullptr;
     c->launches = 0;
+    c->tree_cur = nullptr;
+    c->leaves_kept = 0;
     c->n_pages_total = pages > 0x7fffffff ? 0x7fffffff : pages;
     c->slot_bytes = (size_t)c->n_pages_total * 2 * cfg->n_kv_heads * cfg->page_tokens * cfg->head_dim * c->es;
     Workspace w = carve(cfg);
@@ -884,6 +946,7 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
     eesd_stats sacc;
     memset(&sacc, 0, sizeof(sacc));
     int64_t cursor = 0;
+    const int64_t leaves0 = c->leaves_kept;
     int t = 0, rounds = 0, st;
     int32_t *drafts = c->h_result + 8;
     while (t < max_new) {
@@ -892,6 +955,7 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
         // so they are taken before the round is enqueued (Algorithm 2, draft loop)
         int cap = f.k_cap;
         if (f.max_ctx - 1 - T < cap) cap = f.max_ctx - 1 - T;
+        if (tree_on(c) && (f.max_ctx - T) / f.tree_width < cap) cap = (f.max_ctx - T) / f.tree_width;
         if (cap < 1) return EESD_ERR_CTX_FULL;
         int K;
         // TS with calibration needs the predictor's output after every draft step: such rounds
@@ -962,6 +1026,7 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
         sacc.kernel_launches = c->launches - launches0;
         sacc.alpha = c->alpha;
         sacc.beta = c->beta;
+        sacc.leaves_kept = c->leaves_kept - leaves0;
         *stats = sacc;
     }
     return EESD_OK;
@@ -1023,6 +1088,12 @@ int eesd_context_len(const eesd_ctx *c, int *n_tokens, int *pages_in_use) {
     if (!c) return EESD_ERR_BADARG;
     if (n_tokens) *n_tokens = (int)c->tokens.size();
     if (pages_in_use) *pages_in_use = (int)c->page_of.size();
+    return EESD_OK;
+}
+
+int eesd_context_tokens(const eesd_ctx *c, int first, int n, int32_t *out) {
+    if (!c || !out || first < 0 || n < 0 || (size_t)first + (size_t)n > c->tokens.size()) return EESD_ERR_BADARG;
+    for (int i = 0; i < n; i++) out[i] = c->tokens[(size_t)first + i];
     return EESD_OK;
 }
 

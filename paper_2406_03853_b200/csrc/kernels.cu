@@ -194,7 +194,7 @@ template <typename AT> __device__ __forceinline__ int v_elem(int pos, int e);
 // grid (heads, M), block D/2: one thread per rotation pair.
 template <typename AT>
 __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeom kv, const float2 *rope, float *q,
-                                int head_off, int col_off, int *err) {
+                                int head_off, int col_off, int *err, TreeRows tr, int tree_on) {
     const int hh = blockIdx.x + head_off;  // 0..H-1 q, H..H+Hkv-1 k, then v
     const int m = blockIdx.y, i = threadIdx.x, D = kv.D;
     const int col = col_off + blockIdx.x * D + 2 * i;
@@ -203,9 +203,9 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
     const float rstd = row_rstd(rs, m);
     const float2 pr = part_gather_n<2>(pv, m, col);
     float a = pr.x * rstd, b = pr.y * rstd;
-    const int pos = pos0 + m;
+    const int pos = pos0 + m;   // where the row is stored; a tree row is rotated as its depth's position
     if (hh < H + kv.Hkv) {
-        float2 cs = rope[(size_t)pos * (D / 2) + i];
+        float2 cs = rope[(size_t)(tree_on ? pos0 + tr.depth[m & 15] : pos) * (D / 2) + i];
         float ra = a * cs.x - b * cs.y, rb = a * cs.y + b * cs.x;
         a = ra; b = rb;
     }
@@ -232,11 +232,14 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
     }
 }
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
-                     const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0) {
+                     const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0,
+                     const TreeRows *tree) {
     const int heads = only_kv ? 2 * kv.Hkv : H + 2 * kv.Hkv;
     dim3 grid(heads, M);
-    if (dtype == 0) launch_k(qkv_post_kernel<float>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err);
-    else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err);
+    const TreeRows tr = tree ? *tree : chain_rows();
+    const int tree_on = tree && M <= 16 ? 1 : 0;
+    if (dtype == 0) launch_k(qkv_post_kernel<float>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on);
+    else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on);
 }
 
 // ------------------------------------------------------------------------------------ paged decode attention
@@ -294,7 +297,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                                                    float *__restrict__ apart, unsigned int *tickets,
                                                    float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
                                                    int M, int pos0, int H, int pps, int n_split, float scale, int *err,
-                                                   int Mtot, int nbat, size_t ml_off) {
+                                                   int Mtot, int nbat, size_t ml_off, TreeRows tr) {
     typedef typename KPair<AT>::T KP;
     constexpr int HALF = D / 2;
     constexpr int DPL = D / 32;             // output dimensions per lane in the PV phase
@@ -318,6 +321,9 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     uint64_t *bar = reinterpret_cast<uint64_t *>(s_rstd + kMaxRows);
     float *wgt = reinterpret_cast<float *>(bar + 2);             // [RB][n_split] merge weights
     __shared__ int s_last;
+    // which new rows a row sees and the position it is rotated as (a chain unless the pass verifies a tree)
+    __shared__ uint16_t s_vis[kMaxRows];
+    __shared__ uint8_t s_dep[kMaxRows];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
@@ -348,6 +354,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     const uint32_t blk_bytes = (uint32_t)(PT * D * sizeof(AT));
 
     pdl_trigger();
+    if (tid >= 32 && tid < 32 + kMaxRows) { s_vis[tid - 32] = tr.vis[tid - 32]; s_dep[tid - 32] = tr.depth[tid - 32]; }
     if (tid == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(bar)));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -398,13 +405,13 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     for (int it = 0; it < kNewPerThread; it++) {
         const int idx = tid + it * 256;
         const int pn = idx / D, w = idx - pn * D;
-        cs_new[it] = (idx < n_new && w < HALF) ? rope[(size_t)(p_first + pn) * HALF + w] : make_float2(1.f, 0.f);
+        cs_new[it] = (idx < n_new && w < HALF) ? rope[(size_t)(pos0 + s_dep[p_first + pn - pos0]) * HALF + w] : make_float2(1.f, 0.f);
     }
 #pragma unroll
     for (int it = 0; it < kQPerThread; it++) {
         const int idx = tid + it * 256;
         const int rl = idx / HALF, i = idx - rl * HALF;
-        cs_q[it] = idx < nb * HALF ? rope[(size_t)(pos0 + (r0 + rl) % M) * HALF + i] : make_float2(1.f, 0.f);
+        cs_q[it] = idx < nb * HALF ? rope[(size_t)(pos0 + s_dep[(r0 + rl) % M]) * HALF + i] : make_float2(1.f, 0.f);
     }
     pdl_wait();   // from here on the QKV projection's partial sums are read
     // One round of global loads: the RMSNorm statistics (threads 0..M-1) and the raw partial
@@ -563,7 +570,8 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
 #pragma unroll
                             for (int q2 = 0; q2 < 2; q2++) {
                                 const int j = n0 + 2 * t + q2;
-                                sS[(size_t)rl * ss + j] = (j < npos && lo + j <= pos0 + m) ? c[hf * 2 + q2] : -INFINITY;
+                                const int jn = lo + j - pos0;   // >= 0: a new row
+                                sS[(size_t)rl * ss + j] = (j < npos && (jn < 0 || ((s_vis[m] >> jn) & 1))) ? c[hf * 2 + q2] : -INFINITY;
                             }
                         }
                     }
@@ -600,7 +608,8 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                         const int rl = rc * 8 + i;
                         if (rl < nb) {
                             const int m = (r0 + rl) % M;
-                            sS[(size_t)rl * ss + j] = (j < npos && lo + j <= pos0 + m) ? acc[i] : -INFINITY;
+                            const int jn = lo + j - pos0;
+                            sS[(size_t)rl * ss + j] = (j < npos && (jn < 0 || ((s_vis[m] >> jn) & 1))) ? acc[i] : -INFINITY;
                         }
                     }
                 }
@@ -790,7 +799,7 @@ static size_t attn_smem_bytes(int es, int D, int RB, int cap, int rows, int n_sp
 template <typename AT, int D, int RB, int NM>
 static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                         float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                        int pps, int n_split, float scale, bool early, int *err, int Mtot) {
+                        int pps, int n_split, float scale, bool early, int *err, int Mtot, const TreeRows &tr) {
     const int rows = (H / kv.Hkv) * M, nbat = (rows + RB - 1) / RB;
     const int chunks = Mtot > 0 ? (Mtot + kMaxRows - 1) / kMaxRows : 1;
     const size_t ml_off = (size_t)H * (Mtot > 0 ? n_split : kMaxSlices) * kMaxRows * D;
@@ -801,15 +810,15 @@ static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, 
         configured = 227 * 1024 - 1024;
     }
     launch_k(attn_kernel<AT, D, RB, NM>, dim3(kv.Hkv, n_split, chunks * nbat), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv,
-             apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, Mtot, nbat, ml_off);
+             apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, Mtot, nbat, ml_off, tr);
 }
 
 template <typename AT, int D>
 static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                           float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                          int pps, int n_split, float scale, bool early, int *err, int Mtot) {
+                          int pps, int n_split, float scale, bool early, int *err, int Mtot, const TreeRows &tr) {
     const int rows = (H / kv.Hkv) * M;
-#define EESD_ATTN(RB, NM) attn_launch<AT, D, RB, NM>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot)
+#define EESD_ATTN(RB, NM) attn_launch<AT, D, RB, NM>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr)
     if (rows <= 8) {
         if (M == 1) EESD_ATTN(8, 1);
         else if (M <= 4) EESD_ATTN(8, 4);
@@ -845,24 +854,25 @@ int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n
 
 static void attention_any(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                           const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
-                          int M, int pos0, int H, int pps, int n_split, bool early, int *err, int Mtot) {
+                          int M, int pos0, int H, int pps, int n_split, bool early, int *err, int Mtot, const TreeRows &tr) {
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (dtype == 0) {
-        if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot);
-        else attn_dispatch<float, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot);
+        if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr);
+        else attn_dispatch<float, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr);
     } else {
-        if (kv.D == 64) attn_dispatch<bf16, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot);
-        else attn_dispatch<bf16, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot);
+        if (kv.D == 64) attn_dispatch<bf16, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr);
+        else attn_dispatch<bf16, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr);
     }
 }
 
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
-                      int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err) {
+                      int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err, const TreeRows *tree) {
     int pps;
     const int rows = (H / kv.Hkv) * M, rb = rows <= 8 ? 8 : rows <= kRows16 ? 16 : 32;
     const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb, n_sm, max_splits, &pps);
-    attention_any(s, dtype, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, 0);
+    attention_any(s, dtype, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, 0,
+                  tree ? *tree : chain_rows());
 }
 
 // Prompt attention: Mtot rows at positions pos0.. whose keys / values are in the cache already
@@ -885,7 +895,8 @@ void launch_attention_prompt(cudaStream_t s, int dtype, const PartView &pv, cons
                              const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
                              int Mtot, int pos0, int H, int *err) {
     const int pps = prompt_pps(kv.page_tokens), n_split = attention_prompt_splits(pos0 + Mtot, kv.page_tokens);
-    attention_any(s, dtype, pv, rs, rope, kv, apart, tickets, nullptr, attn_split, kMaxRows, pos0, H, pps, n_split, false, err, Mtot);
+    attention_any(s, dtype, pv, rs, rope, kv, apart, tickets, nullptr, attn_split, kMaxRows, pos0, H, pps, n_split, false, err, Mtot,
+                  chain_rows());
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU, partial sums
@@ -907,6 +918,130 @@ __global__ void swiglu_kernel(PartView pv, RowScale rs, float *h, bf16 *hs, int 
 }
 void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F) {
     launch_k(swiglu_kernel, dim3((F / 4 + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, h, (bf16 *)h_split, F);
+}
+
+// ------------------------------------------------------------------------------------ tree verification helpers
+// Tokens ranked 2..width of one logit row, ranked by logit with the lower id first among equals
+// (rank 1 is the greedy draft token).  One block; every rank is one pass over the row that keeps
+// the best element ranked after the previous pick.
+__global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict__ logits, int V, int width, int32_t *out) {
+    __shared__ float s_v[32];
+    __shared__ int s_i[32];
+    __shared__ float s_pv;
+    __shared__ int s_pi;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    float pv = INFINITY;
+    int pi = -1;
+    auto better = [](float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); };
+    for (int r = 0; r < width; r++) {
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int i = threadIdx.x; i < V; i += blockDim.x) {
+            const float v = logits[i];
+            const bool after = v < pv || (v == pv && i > pi);
+            if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) { s_v[warp] = bv; s_i[warp] = bi; }
+        __syncthreads();
+        if (warp == 0) {
+            bv = lane < nw ? s_v[lane] : -INFINITY;
+            bi = lane < nw ? s_i[lane] : 0x7fffffff;
+#pragma unroll
+            for (int o = 16; o; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+            }
+            if (lane == 0) {
+                s_pv = bv;
+                s_pi = bi;
+                if (r >= 1) out[r - 1] = bi;
+            }
+        }
+        __syncthreads();
+        pv = s_pv;
+        pi = s_pi;
+        __syncthreads();
+    }
+}
+void launch_next_best(cudaStream_t s, const float *logits, int V, int width, int32_t *out) {
+    next_best_kernel<<<1, 1024, 0, s>>>(logits, V, width, out);
+}
+
+__global__ void tree_rows_kernel(const int32_t *chain, const int32_t *leaf, int K, int width, int32_t *rows) {
+    const int t = threadIdx.x, M = 1 + K * width;
+    if (t < M) rows[t] = t <= K ? chain[t] : leaf[t - K - 1];
+}
+void launch_tree_rows(cudaStream_t s, const int32_t *src_chain, const int32_t *src_leaf, int K, int width, int32_t *rows) {
+    tree_rows_kernel<<<1, 32, 0, s>>>(src_chain, src_leaf, K, width, rows);
+}
+
+// Row i (1 <= i <= K) holds chain token x_i, row K + 1 + (i - 1)(width - 1) + j leaf j of depth i.
+// top[m] is the target's top-1 token after the path that ends in row m.
+__global__ void tree_walk_kernel(const int32_t *top, int32_t *chain, const int32_t *leaf, int K, int width, int32_t *result) {
+    if (threadIdx.x != 0) return;
+    int a = K, y = top[K], row = -1;
+    for (int i = 1; i <= K; i++) {
+        const int want = top[i - 1];
+        if (want == chain[i]) continue;
+        a = i - 1;
+        y = want;
+        for (int j = 0; j < width - 1; j++) {
+            const int li = (i - 1) * (width - 1) + j;
+            if (leaf[li] == want) {
+                row = K + 1 + li;
+                a = i;
+                y = top[row];
+                chain[i] = want;
+                break;
+            }
+        }
+        break;
+    }
+    result[0] = a;
+    result[1] = y;
+    result[2] = row;
+    chain[0] = y;
+}
+void launch_tree_walk(cudaStream_t s, const int32_t *top, int32_t *chain, const int32_t *leaf, int K, int width,
+                      int32_t *result) {
+    tree_walk_kernel<<<1, 32, 0, s>>>(top, chain, leaf, K, width, result);
+}
+
+// A kept leaf's keys / values move from the position its row was stored at to the position of
+// its depth.  grid (H_kv, slots), D / 2 threads: one rotation pair of the key, two value elements.
+template <typename AT>
+__global__ void kv_move_kernel(KvGeom kv, size_t slot_bytes, int pos0, const int32_t *result, int *err) {
+    const int row = result[2];
+    if (row < 0) return;
+    const int src = pos0 + row, dst = pos0 + result[0];
+    const int kh = blockIdx.x, i = threadIdx.x, D = kv.D, PT = kv.page_tokens;
+    const int ps = kv.page_table[src / PT], pd = kv.page_table[dst / PT];
+    if (ps < 0 || ps >= kv.n_pages_total || pd < 0 || pd >= kv.n_pages_total) {
+        if (i == 0) atomicOr(err, kErrBadPage);
+        return;
+    }
+    AT *base = (AT *)((char *)kv.slot_base + (size_t)blockIdx.y * slot_bytes);
+    const size_t blk = (size_t)PT * D;
+    const AT *ks = base + (((size_t)ps * 2) * kv.Hkv + kh) * blk, *vs = base + (((size_t)ps * 2 + 1) * kv.Hkv + kh) * blk;
+    AT *kd = base + (((size_t)pd * 2) * kv.Hkv + kh) * blk, *vd = base + (((size_t)pd * 2 + 1) * kv.Hkv + kh) * blk;
+    const int sj = src % PT, dj = dst % PT;
+#pragma unroll
+    for (int e = 0; e < 2; e++) {
+        kd[((size_t)i * PT + dj) * 2 + e] = ks[((size_t)i * PT + sj) * 2 + e];
+        vd[(size_t)dj * D + v_elem<AT>(dst, 2 * i + e)] = vs[(size_t)sj * D + v_elem<AT>(src, 2 * i + e)];
+    }
+}
+void launch_kv_move(cudaStream_t s, int dtype, const KvGeom &kv0, size_t slot_bytes, int slots, int pos0,
+                    const int32_t *result, int *err) {
+    if (dtype == 0) kv_move_kernel<float><<<dim3(kv0.Hkv, slots), kv0.D / 2, 0, s>>>(kv0, slot_bytes, pos0, result, err);
+    else kv_move_kernel<bf16><<<dim3(kv0.Hkv, slots), kv0.D / 2, 0, s>>>(kv0, slot_bytes, pos0, result, err);
 }
 
 // ------------------------------------------------------------------------------------ calibration predictor (Eq. 5)

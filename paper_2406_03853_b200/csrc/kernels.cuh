@@ -56,6 +56,20 @@ struct RowScale {
     float inv_d, eps;
 };
 
+// Rows of a verification pass that form a tree instead of a chain (several draft candidates
+// per position).  Row m is stored at cache position pos0 + m, is rotated as position
+// pos0 + depth[m], and sees every position before pos0 plus the rows whose bit is set in vis[m]
+// (its ancestors and itself).  A chain is depth[m] = m, vis[m] = bits 0..m.
+struct TreeRows {
+    uint16_t vis[16];
+    uint8_t depth[16];
+};
+inline TreeRows chain_rows() {
+    TreeRows t;
+    for (int m = 0; m < 16; m++) { t.vis[m] = (uint16_t)((2u << m) - 1u); t.depth[m] = (uint8_t)m; }
+    return t;
+}
+
 void launch_set_ints(cudaStream_t s, int32_t *dst, const IntList16 &vals, int n);
 void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float theta);
 void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
@@ -69,8 +83,10 @@ void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, 
 int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float *out, int M, int R, int K);
 // RoPE + KV append (+ q store).  part rows are [q heads | k heads | v heads] or, when
 // only_kv, [k heads | v heads] starting at column kv_col0 of the projection result.
+// tree (optional, M <= 16): row m is rotated as position pos0 + depth[m] and stored at pos0 + m.
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
-                     const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0 = 0);
+                     const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0 = 0,
+                     const TreeRows *tree = nullptr);
 // Fused attention step of one layer on M new rows: q/k/v of the new rows are taken from the
 // QKV projection's partial sums (scaled by rs, rotated), the new keys/values are appended to
 // the paged cache, every KV head's cached slice is read once, and the slices are merged into
@@ -81,7 +97,8 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 // must be false when that kernel appends rows to the same cache slot.
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
-                      int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err);
+                      int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err,
+                      const TreeRows *tree = nullptr);
 // Prompt attention: all 16-row chunks of Mtot rows in one launch; the rows' keys / values must be
 // in the cache already (launch_qkv_post with only_kv on the QKV result) and pv must be a plain
 // [Mtot][R] result (mode 0).  apart: attention_prompt_scratch_floats(...) floats; tickets: zeroed
@@ -96,6 +113,22 @@ void launch_attention_prompt(cudaStream_t s, int dtype, const PartView &pv, cons
 void launch_copy_row(cudaStream_t s, const float *x, int row, const int32_t *row_dev, float *hT, void *xs, int d);
 // theta_M = softmax(Wp [v ; hD])[1] with v = the d partial results of W^i H^(T) (Eq. 5)
 void launch_cali_theta(cudaStream_t s, const PartView &pv, const float *Wp, const float *hD, int d, float *theta);
+// Tree verification helpers.  launch_next_best: tokens ranked 2..width of one logit row (by
+// logit, lower id first among equals) -> out[width - 1].  launch_tree_rows: the pass's token rows
+// = chain tokens src_chain[0..K], then the leaves src_leaf[0..K * (width - 1)).
+// launch_tree_walk: given the target's top-1 token of every row, walks the tree (chain token
+// continues, a leaf ends the round, neither ends it with the target's token); writes
+// result[0] = accepted draft tokens, result[1] = the round's last token, result[2] = row of the
+// kept leaf or -1; the kept leaf's token replaces the chain token at its depth in chain[],
+// and chain[0] becomes the round's last token (the next round's pending token).
+// launch_kv_move: when result[2] >= 0, copies the keys / values stored at position
+// pos0 + result[2] to position pos0 + result[0] in `slots` cache slots of slot_bytes each.
+void launch_next_best(cudaStream_t s, const float *logits, int V, int width, int32_t *out);
+void launch_tree_rows(cudaStream_t s, const int32_t *src_chain, const int32_t *src_leaf, int K, int width, int32_t *rows);
+void launch_tree_walk(cudaStream_t s, const int32_t *top, int32_t *chain, const int32_t *leaf, int K, int width,
+                      int32_t *result);
+void launch_kv_move(cudaStream_t s, int dtype, const KvGeom &kv0, size_t slot_bytes, int slots, int pos0,
+                    const int32_t *result, int *err);
 void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F);
 void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R);
 // programmatic dependent launch (kernels start early and wait on-device for their producer):
