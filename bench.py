@@ -373,6 +373,7 @@ def main():
                     help="scale of the upper layers' output projections (draft/target agreement): 0.05 high, "
                          "0.2 medium (default), 0.5 low acceptance")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-tree", action="store_true", help="skip the tree-verification leg of the default run")
     ap.add_argument("--profile-pass", type=int, default=0, metavar="M",
                     help="only run verify passes of M rows (and draft steps) inside a cudaProfilerStart/Stop "
                          "bracket, for ncu --profile-from-start off")
@@ -529,8 +530,35 @@ def main():
             "sample": f"one {spec.name}-shaped decoder layer on {rows} rows and on 1 row against a 512-token cache "
                       f"({reps} repetitions, {secs:.1f} s of CPU work, medians), scaled to a round of mean K={mean_k:.2f} emitting {mean_emit:.2f} "
                       f"tokens; extrapolated"}
-    print(json.dumps(line))
     eng.close()
+    del eng
+    if world == 1 and greedy and args.controller == "beta" and not args.no_tree:
+        # tree verification (the paper's tree-attention table) on the same prompts: width 2, three
+        # draft steps per round (7 rows per pass), against the chain at the same draft length
+        torch.cuda.empty_cache()
+        tv = {}
+        for W in (1, 2):
+            eng_t, _, _, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, alpha=args.alpha, tree_width=W)
+            ms_t, tot = 0.0, {"drafted": 0, "accepted": 0, "rounds": 0, "leaves_kept": 0}
+            for i in range(args.steps):
+                eng_t.prefill(prompts[i])
+                torch.cuda.synchronize()
+                e0.record()
+                _, _, st_t = eng_t.decode(max_new, k_schedule=[3] * max_new)
+                e1.record()
+                torch.cuda.synchronize()
+                ms_t += e0.elapsed_time(e1)
+                for k in tot:
+                    tot[k] += st_t.as_dict()[k]
+            tv["chain_k3" if W == 1 else "width2_k3"] = {
+                "tokens_per_s": round(args.steps * max_new / (ms_t * 1e-3), 2),
+                "v_d": round(tot["accepted"] / max(1, tot["drafted"]), 4),
+                "leaves_kept_per_round": round(tot["leaves_kept"] / max(1, tot["rounds"]), 4)}
+            eng_t.close()
+            del eng_t
+            torch.cuda.empty_cache()
+        line["tree_verification"] = tv
+    print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
 
