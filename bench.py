@@ -253,6 +253,28 @@ def profile_pass(args, device):
     eng.close()
 
 
+def profile_tree_round(args, device):
+    """One greedy round with tree verification (K = 3 draft steps, width --profile-tree, so
+    1 + 3 width rows in the verify pass) against a 1024-token cache, between
+    cudaProfilerStart/Stop (for the ncu recipes)."""
+    from paper_2406_03853_b200 import binding as b
+    W = args.profile_tree
+    eng, spec, _, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, args.layers, tree_width=W)
+    kv_len = WORKLOADS[args.workload][4]
+    eng.assume_context(kv_len, 17)
+    eng.draft(3)
+    eng.verify_accept()
+    torch.cuda.synchronize()
+    torch.cuda.profiler.start()
+    eng.draft(3)
+    a, y = eng.verify_accept()
+    torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
+    print("profiled: 1 round of 3 draft steps + tree verify pass of %d rows (width %d), %s, %d layers; accepted %d"
+          % (1 + 3 * W, W, spec.name, spec.n_layers, a))
+    eng.close()
+
+
 def profile_prefill(args, device):
     """One prompt pass (eesd_prefill) between cudaProfilerStart/Stop (for the ncu recipes)."""
     from paper_2406_03853_b200 import binding as b
@@ -383,6 +405,8 @@ def main():
                     help="method sweep instead of the benchmark line: fixed K = 1..10 against Beta-TS, or the exit depth N")
     ap.add_argument("--profile-prefill", action="store_true",
                     help="only run one prompt pass inside a cudaProfilerStart/Stop region (for ncu)")
+    ap.add_argument("--profile-tree", type=int, default=0, metavar="W",
+                    help="only run one round with tree verification of width W inside a cudaProfilerStart/Stop bracket")
     ap.add_argument("--layers", type=int, default=0, help="with --profile-pass: keep only this many layers")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -406,6 +430,8 @@ def main():
         return profile_pass(args, device)
     if args.profile_prefill:
         return profile_prefill(args, device)
+    if args.profile_tree:
+        return profile_tree_round(args, device)
     if args.sweep:
         return run_sweep(args, device) if rank == 0 else None
     from paper_2406_03853_b200 import report

@@ -934,7 +934,8 @@ void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float
 // ------------------------------------------------------------------------------------ tree verification helpers
 // Tokens ranked 2..width of one logit row, ranked by logit with the lower id first among equals
 // (rank 1 is the greedy draft token).  One block; every rank is one pass over the row that keeps
-// the best element ranked after the previous pick.
+// the best element ranked after the previous pick.  Rows of up to 32768 logits are read once
+// into registers (all loads in flight together: the kernel is one block and latency bound).
 __global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict__ logits, int V, int width, int32_t *out) {
     __shared__ float s_v[32];
     __shared__ int s_i[32];
@@ -944,13 +945,33 @@ __global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict
     float pv = INFINITY;
     int pi = -1;
     auto better = [](float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); };
+    constexpr int kPer = 32;
+    const bool in_regs = V <= kPer * (int)blockDim.x;
+    float reg[kPer];
+    if (in_regs) {
+#pragma unroll
+        for (int j = 0; j < kPer; j++) {
+            const int i = threadIdx.x + j * blockDim.x;
+            reg[j] = i < V ? logits[i] : NAN;   // NaN compares false: never picked
+        }
+    }
     for (int r = 0; r < width; r++) {
         float bv = -INFINITY;
         int bi = 0x7fffffff;
-        for (int i = threadIdx.x; i < V; i += blockDim.x) {
-            const float v = logits[i];
-            const bool after = v < pv || (v == pv && i > pi);
-            if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
+        if (in_regs) {
+#pragma unroll
+            for (int j = 0; j < kPer; j++) {
+                const int i = threadIdx.x + j * blockDim.x;
+                const float v = reg[j];
+                const bool after = v < pv || (v == pv && i > pi);
+                if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
+            }
+        } else {
+            for (int i = threadIdx.x; i < V; i += blockDim.x) {
+                const float v = logits[i];
+                const bool after = v < pv || (v == pv && i > pi);
+                if (after && better(v, i, bv, bi)) { bv = v; bi = i; }
+            }
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) {

@@ -131,3 +131,19 @@ def test_tree_pass_13b_layer_shape():
     worst, kept = _rounds_through_the_step_api(spec, 2, width=3, k=5, n_prompt=21, n_rounds=2, max_ctx=96)
     print(f"tree pass, 13B layer shape (2 layers): worst logit distance {worst:.3e}")
     assert worst < TOL
+
+
+def test_tree_generation_under_the_beta_controller():
+    # draft lengths chosen by Thompson sampling; the oracle's round is driven by the lengths the engine took
+    from paper_2406_03853_b200 import binding as b
+    spec = synth.TINY
+    prompt = synth.prompt_tokens(synth.SEED + 21, 28, spec.vocab).numpy()
+    u = {k: v.numpy() for k, v in synth.generate_uniforms(160, 100000).items()}
+    eng = engine_from_spec(spec, max_ctx=160, k_cap=7, tree_width=2, controller=b.CTRL_BETA_TS)
+    out, trace, st = eng.generate(prompt, 48, uniforms=u)
+    ks = [k for k, _, _ in trace]
+    assert len(set(ks)) > 1 and max(ks) <= 7
+    ref, rtrace, rleaves = oracle_from_spec(spec, 160).generate_tree(prompt, 48, width=2, k_schedule=ks)
+    np.testing.assert_array_equal(out, ref)
+    assert trace == rtrace and st.leaves_kept == rleaves
+    eng.close()
