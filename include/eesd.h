@@ -87,7 +87,9 @@ typedef struct eesd_config {
      * leaf), neither ends the round with the target's token.  The paper fixes no tree shape: this
      * one is a choice.  Needs temperature 0, a controller other than EESD_CTRL_CALI_TS and
      * 1 + k_cap * tree_width <= EESD_MAX_ROWS (else UNSUPPORTED / BADARG); a round of K drafts
-     * uses 1 + K * tree_width cache rows past the context before it is cut back. */
+     * uses 1 + K * tree_width cache rows past the context before it is cut back, so
+     * eesd_generate / eesd_decode want n_prompt + max_new + tree_width <= max_ctx (CTX_FULL
+     * otherwise) and shorten the last rounds' drafts to what fits. */
     int32_t tree_width;
 } eesd_config;
 

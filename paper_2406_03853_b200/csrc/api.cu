@@ -937,6 +937,8 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
     if (f.controller != EESD_CTRL_FIXED_K && (!u || !u->u_ctrl)) return EESD_ERR_RNG;
     const int n0 = (int)c->tokens.size();
     if (n0 + max_new + 1 > f.max_ctx) return EESD_ERR_CTX_FULL;
+    // tree verification stores its leaves past the chain: leave room for the shortest round (one draft step)
+    if (tree_on(c) && n0 + max_new + f.tree_width > f.max_ctx) return EESD_ERR_CTX_FULL;
     float *d_ud = c->u_dev, *d_ua = c->u_dev + f.max_ctx, *d_ur = c->u_dev + 2 * (size_t)f.max_ctx;
     if (!greedy) {
         CU(c, cudaMemcpyAsync(d_ud, u->u_draft, (size_t)f.max_ctx * 4, cudaMemcpyHostToDevice, c->stream));

@@ -147,3 +147,19 @@ def test_tree_generation_under_the_beta_controller():
     np.testing.assert_array_equal(out, ref)
     assert trace == rtrace and st.leaves_kept == rleaves
     eng.close()
+
+
+def test_tree_generation_up_to_the_context_limit():
+    # the last rounds draft fewer tokens so that the tree rows still fit; one token more is refused up front
+    from paper_2406_03853_b200 import EesdError
+    spec = synth.TINY
+    prompt = synth.prompt_tokens(synth.SEED + 5, 30, spec.vocab).numpy()
+    ref, rtrace, rleaves = oracle_from_spec(spec, 64).generate_tree(prompt, 31, width=3, fixed_k=5)
+    eng = engine_from_spec(spec, max_ctx=64, fixed_k=5, k_cap=5, tree_width=3)
+    out, trace, st = eng.generate(prompt, 31)
+    np.testing.assert_array_equal(out, ref)
+    assert trace == rtrace and st.leaves_kept == rleaves
+    assert trace[-1][0] < 5   # shortened at the end
+    with pytest.raises(EesdError):
+        eng.generate(prompt, 32)
+    eng.close()
