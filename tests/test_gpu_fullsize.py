@@ -94,3 +94,25 @@ def test_stochastic_rounds_at_13b_layer_shapes_follow_the_rule_on_the_gpus_own_l
     assert abs(hits - expect) < 4.0 * np.sqrt(var) + 1.0, (hits, expect, var)
     assert 0.05 * rounds < expect < 0.999 * rounds          # neither a degenerate draft nor a copy of the target
     eng.close()
+
+
+def test_tree_verification_at_full_size_emits_the_same_greedy_tokens(engine13b):
+    """Losslessness of tree verification at the benchmark's size: whatever candidates a pass
+    holds, the output is the target's own greedy sequence, so a tree run (two and three
+    candidates per position, 7 to 16 rows per pass) must emit the chain run's tokens; and it
+    must keep leaves, or the equality would say nothing."""
+    import bench
+    from paper_2406_03853_b200 import binding as b
+    eng, spec = engine13b
+    prompt = synth.prompt_tokens(synth.SEED, 200, spec.vocab).numpy()
+    ref, _, st_chain = eng.generate(prompt, 40, k_schedule=[3] * 64)
+    for width, ks in ((2, [3] * 64), (3, [5, 1, 4, 2, 3] * 13)):
+        eng_t, _, _, _ = bench.build_engine("13b-eesd", 0.0, b.CTRL_FIXED_K, torch.device("cuda:0"), tree_width=width)
+        out, trace, st = eng_t.generate(prompt, 40, k_schedule=ks)
+        eng_t.close()
+        del eng_t
+        torch.cuda.empty_cache()
+        np.testing.assert_array_equal(out, ref)
+        assert st.leaves_kept > 0 and all(0 <= a <= k for k, a, _ in trace)
+        if width == 2:
+            assert st.rounds <= st_chain.rounds   # same draft length, more candidates: never more rounds here
