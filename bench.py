@@ -339,9 +339,10 @@ def run_sweep(args, device):
         eng.close()
     elif args.sweep == "tree":
         for W in (1, 2, 3):
-            eng, spec, _, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, alpha=args.alpha, tree_width=W)
+            eng, spec, _, _ = build_engine(args.workload, 0.0, b.CTRL_BETA_TS, device, alpha=args.alpha, tree_width=W)
             for K in (2, 3, 4, 5):
                 measure(eng, spec, f"width {W}, fixed K={K} ({1 + K * max(W, 1)} rows per pass)", [K] * max_new)
+            measure(eng, spec, f"width {W}, beta-ts (K cap {eng.cfg.k_cap})", None)
             eng.close()
             del eng
             torch.cuda.empty_cache()
