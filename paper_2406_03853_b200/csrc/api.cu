@@ -435,12 +435,11 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
     float *lq = c->logits_q + (size_t)i * f.vocab;
     PartView pv = run_proj(c, c->exit_head, &c->m_exit_head, P_HEAD, X_NORM, 1, f.vocab, d);
     launch_reduce_partials(s, pv, norm_scale(c), lq, 1, f.vocab);
-    launch_sample_rows(s, lq, d_u, 1, f.vocab, f.temperature, c->ints + kRoundTok + i + 1);
+    if (tree_on(c))   // greedy token and, in the same kernel, the next-best candidates: leaves of depth i + 1
+        launch_next_best(s, lq, f.vocab, f.tree_width, c->ints + kRoundTok + i + 1, c->ints + kLeafTok + i * (f.tree_width - 1));
+    else
+        launch_sample_rows(s, lq, d_u, 1, f.vocab, f.temperature, c->ints + kRoundTok + i + 1);
     c->launches += 3;
-    if (tree_on(c)) {   // the next-best candidates of this step become leaves of depth i + 1
-        launch_next_best(s, lq, f.vocab, f.tree_width, c->ints + kLeafTok + i * (f.tree_width - 1));
-        c->launches++;
-    }
     return check_launch(c);
 }
 

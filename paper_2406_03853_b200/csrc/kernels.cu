@@ -932,11 +932,12 @@ void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float
 }
 
 // ------------------------------------------------------------------------------------ tree verification helpers
-// Tokens ranked 2..width of one logit row, ranked by logit with the lower id first among equals
-// (rank 1 is the greedy draft token).  One block; every rank is one pass over the row that keeps
+// Tokens ranked 1..width of one logit row, ranked by logit with the lower id first among equals
+// (rank 1, the greedy draft token, goes to *first when given; ranks 2.. to out).  One block; every rank is one pass over the row that keeps
 // the best element ranked after the previous pick.  Rows of up to 32768 logits are read once
 // into registers (all loads in flight together: the kernel is one block and latency bound).
-__global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict__ logits, int V, int width, int32_t *out) {
+__global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict__ logits, int V, int width, int32_t *first,
+                                                         int32_t *out) {
     __shared__ float s_v[32];
     __shared__ int s_i[32];
     __shared__ float s_pv;
@@ -994,6 +995,7 @@ __global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict
                 s_pv = bv;
                 s_pi = bi;
                 if (r >= 1) out[r - 1] = bi;
+                else if (first) *first = bi;
             }
         }
         __syncthreads();
@@ -1002,8 +1004,8 @@ __global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict
         __syncthreads();
     }
 }
-void launch_next_best(cudaStream_t s, const float *logits, int V, int width, int32_t *out) {
-    next_best_kernel<<<1, 1024, 0, s>>>(logits, V, width, out);
+void launch_next_best(cudaStream_t s, const float *logits, int V, int width, int32_t *first, int32_t *out) {
+    next_best_kernel<<<1, 1024, 0, s>>>(logits, V, width, first, out);
 }
 
 __global__ void tree_rows_kernel(const int32_t *chain, const int32_t *leaf, int K, int width, int32_t *rows) {

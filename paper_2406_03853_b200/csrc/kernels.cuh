@@ -113,8 +113,8 @@ void launch_attention_prompt(cudaStream_t s, int dtype, const PartView &pv, cons
 void launch_copy_row(cudaStream_t s, const float *x, int row, const int32_t *row_dev, float *hT, void *xs, int d);
 // theta_M = softmax(Wp [v ; hD])[1] with v = the d partial results of W^i H^(T) (Eq. 5)
 void launch_cali_theta(cudaStream_t s, const PartView &pv, const float *Wp, const float *hD, int d, float *theta);
-// Tree verification helpers.  launch_next_best: tokens ranked 2..width of one logit row (by
-// logit, lower id first among equals) -> out[width - 1].  launch_tree_rows: the pass's token rows
+// Tree verification helpers.  launch_next_best: tokens ranked 1..width of one logit row (by
+// logit, lower id first among equals): rank 1 -> *first (optional), ranks 2.. -> out[width - 1].  launch_tree_rows: the pass's token rows
 // = chain tokens src_chain[0..K], then the leaves src_leaf[0..K * (width - 1)).
 // launch_tree_walk: given the target's top-1 token of every row, walks the tree (chain token
 // continues, a leaf ends the round, neither ends it with the target's token); writes
@@ -123,7 +123,7 @@ void launch_cali_theta(cudaStream_t s, const PartView &pv, const float *Wp, cons
 // and chain[0] becomes the round's last token (the next round's pending token).
 // launch_kv_move: when result[2] >= 0, copies the keys / values stored at position
 // pos0 + result[2] to position pos0 + result[0] in `slots` cache slots of slot_bytes each.
-void launch_next_best(cudaStream_t s, const float *logits, int V, int width, int32_t *out);
+void launch_next_best(cudaStream_t s, const float *logits, int V, int width, int32_t *first, int32_t *out);
 void launch_tree_rows(cudaStream_t s, const int32_t *src_chain, const int32_t *src_leaf, int K, int width, int32_t *rows);
 void launch_tree_walk(cudaStream_t s, const int32_t *top, int32_t *chain, const int32_t *leaf, int K, int width,
                       int32_t *result);
