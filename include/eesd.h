@@ -205,7 +205,12 @@ int eesd_draft(eesd_ctx *ctx, int k, const float *u_draft, int32_t *out_tokens);
  * u_resample.  Greedy: accept while x_i = argmax p_i, next token = argmax of the first
  * disagreeing row.  KV rows of rejected tokens are rolled back (pages past the end freed).
  * Afterwards the context holds the accepted tokens plus next_token, which is pending.
- * u_accept: host array of K values (may be NULL when greedy).  Errors: STATE (nothing drafted). */
+ * u_accept: host array of K values (may be NULL when greedy).  Errors: STATE (nothing drafted).
+ * With tree verification (eesd_config.tree_width > 1) the pass also holds the draft steps'
+ * next-best tokens as leaves; n_accept then counts a kept leaf as an accepted draft, and the
+ * token accepted at that depth is the leaf, not the one eesd_draft returned:
+ * eesd_context_tokens shows what the context gained.  Errors: CTX_FULL when the tree rows do
+ * not fit below max_ctx. */
 int eesd_verify_accept(eesd_ctx *ctx, const float *u_accept, float u_resample,
                        int *n_accept, int32_t *next_token);
 
