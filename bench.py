@@ -563,7 +563,7 @@ def main():
         # tree verification (the paper's tree-attention table) on the same prompts: width 2, three
         # draft steps per round (7 rows per pass), against the chain at the same draft length
         torch.cuda.empty_cache()
-        tv = {}
+        tv, outs = {}, {}
         for W in (1, 2):
             eng_t, _, _, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, alpha=args.alpha, tree_width=W)
             ms_t, tot = 0.0, {"drafted": 0, "accepted": 0, "rounds": 0, "leaves_kept": 0}
@@ -571,7 +571,8 @@ def main():
                 eng_t.prefill(prompts[i])
                 torch.cuda.synchronize()
                 e0.record()
-                _, _, st_t = eng_t.decode(max_new, k_schedule=[3] * max_new)
+                out_t, _, st_t = eng_t.decode(max_new, k_schedule=[3] * max_new)
+                outs.setdefault(W, []).append(out_t.copy())
                 e1.record()
                 torch.cuda.synchronize()
                 ms_t += e0.elapsed_time(e1)
@@ -584,6 +585,8 @@ def main():
             eng_t.close()
             del eng_t
             torch.cuda.empty_cache()
+        # greedy decoding is lossless either way: both runs must have emitted the same tokens
+        tv["same_tokens_as_chain"] = all((a == c).all() for a, c in zip(outs[2], outs[1]))
         line["tree_verification"] = tv
     print(json.dumps(line))
     if dist:
