@@ -206,7 +206,7 @@ struct eesd_ctx {
     const TreeRows *tree_cur;
     TreeRows tree_rows;
     int64_t leaves_kept;
-    int32_t *h_result;  // pinned: [0] n_accept, [1] next token, [2] error word, [8..23] draft tokens
+    int32_t *h_result;  // pinned: [0] n_accept, [1] next token, [2] error word, [3] row of the kept leaf or -1, [8..23] draft tokens
     cudaEvent_t ev[5];  // prefill start / end, draft start, verify start, round end
     char cuda_err[256];
 };
