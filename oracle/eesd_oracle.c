@@ -392,7 +392,6 @@ int orc_ts_continue(long alpha, long beta, const float *u, long n_u, long *curso
 void orc_ts_update(long *alpha, long *beta, int q_v, int n_draft, int rule) {
     long r = q_v - 1;
     long n = rule == 0 ? (q_v + 1 < n_draft ? q_v + 1 : n_draft) : (q_v < n_draft ? q_v : n_draft);
-    if (n < r) n = r;
     *alpha += r;
     *beta += n - r;
 }

@@ -197,8 +197,7 @@ def test_bf16_storage_rounding_matches_library_conversion_and_only_touches_the_c
     got = np.array([oracle.bf16_round(x) for x in xs])
     ref = torch.tensor(xs, dtype=torch.float32).to(torch.bfloat16).double().numpy()  # round-to-nearest-even
     np.testing.assert_array_equal(got, ref)
-    # with one cached position attention returns v exactly, so the layer output moves by exactly
-    # Wo (bf16(v) - v); with more positions a bf16 cache stays within bf16 rounding of the fp64 one
+    # the storage rounding moves a layer's output: not a no-op on these inputs
     spec = synth.TINY.with_(n_layers=1, n_early=1)
     lw = synth.layer_weights(spec, 0)
     emb, head = synth.embedding(spec), synth.lm_head(spec)
@@ -208,3 +207,127 @@ def test_bf16_storage_rounding_matches_library_conversion_and_only_touches_the_c
     ya, yb = a.layer_fwd(0, 0, x0, 0), b.layer_fwd(0, 0, x0, 0)
     d = np.abs(ya - yb).max()
     assert 0 < d < 2.0 ** -7 * np.abs(ya).max()
+
+
+def _bf16(a):
+    """bfloat16 storage of fp64 values through the library conversion (fp64 -> fp32 -> bf16, nearest even)."""
+    import torch
+    return torch.tensor(np.asarray(a, np.float64), dtype=torch.float32).to(torch.bfloat16).double().numpy()
+
+
+def test_bf16_cache_one_position_moves_the_output_by_exactly_wo_times_the_value_rounding():
+    # One cached position: the softmax weight is 1 whatever the key is, so attention returns the
+    # cached value itself.  With W_down = 0 the layer is x + Wo v, hence
+    #   layer(bf16 cache) - layer(fp64 cache) = Wo (bf16(v) - v),   v = Wv RMSNorm(x)
+    # exactly (a rounding of the value only; rounding anything else, or not rounding, breaks it).
+    spec = synth.TINY.with_(n_layers=1, n_early=1, n_kv_heads=2)
+    lw = synth.layer_weights(spec, 0)
+    lw = dict(lw, wd=np.zeros_like(lw["wd"].numpy()))
+    emb, head = synth.embedding(spec), synth.lm_head(spec)
+    a = oracle.model_from_weights(spec, [lw], lw, emb, head, max_ctx=8, kv_bf16=False)
+    b = oracle.model_from_weights(spec, [lw], lw, emb, head, max_ctx=8, kv_bf16=True)
+    x0 = a.embed([5]) * 30.0
+    H, Hkv, D = spec.n_heads, spec.n_kv_heads, spec.head_dim
+    n = x0[0] / np.sqrt((x0[0] ** 2).mean() + spec.rms_eps)
+    v = lw["wqkv"][(H + Hkv) * D:].double().numpy() @ n                     # [Hkv * D]
+    dv = np.repeat((_bf16(v) - v).reshape(Hkv, D), H // Hkv, axis=0).reshape(H * D)   # every query head reads its group's value
+    assert np.abs(dv).max() > 1e-6
+    want = lw["wo"].double().numpy() @ dv
+    got = b.layer_fwd(0, 0, x0, 0)[0] - a.layer_fwd(0, 0, x0, 0)[0]
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+
+
+def _dense_layer_bf16_cache(x, lw, spec, where="after", theta=10000.0, eps=1e-5):
+    """The dense causal formulation of a decoder layer with keys and values stored as bfloat16:
+    keys rounded AFTER the rotation (what sits in a cache of rotated keys), values as projected.
+    `where` = "before" rounds the keys before the rotation, "values_only" leaves the keys alone:
+    the two misplacements the pin below must tell apart from the right one."""
+    T, d = x.shape
+    H, Hkv, D, F = spec.n_heads, spec.n_kv_heads, spec.head_dim, spec.ffn_dim
+    w = {k: (v.double().numpy() if hasattr(v, "double") else np.asarray(v, np.float64)) for k, v in lw.items()}
+
+    def norm(a, g):
+        return a / np.sqrt((a * a).mean(-1, keepdims=True) + eps) * g
+
+    def rot(a):
+        i = np.arange(D // 2)
+        ang = np.arange(T)[:, None] * theta ** (-2.0 * i / D)[None, :]
+        c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+        out = np.empty_like(a)
+        out[..., 0::2] = a[..., 0::2] * c - a[..., 1::2] * s
+        out[..., 1::2] = a[..., 0::2] * s + a[..., 1::2] * c
+        return out
+
+    n = norm(x, w["g_attn"])
+    qkv = n @ w["wqkv"].T
+    q = rot(qkv[:, :H * D].reshape(T, H, D))
+    k = qkv[:, H * D:(H + Hkv) * D].reshape(T, Hkv, D)
+    k = {"after": lambda: _bf16(rot(k)), "before": lambda: rot(_bf16(k)), "values_only": lambda: rot(k)}[where]()
+    v = _bf16(qkv[:, (H + Hkv) * D:].reshape(T, Hkv, D))
+    k, v = np.repeat(k, H // Hkv, axis=1), np.repeat(v, H // Hkv, axis=1)
+    sc = np.einsum("thd,shd->hts", q, k) / math.sqrt(D)
+    sc = np.where(np.tril(np.ones((T, T), bool))[None], sc, -np.inf)
+    p = np.exp(sc - sc.max(-1, keepdims=True))
+    p /= p.sum(-1, keepdims=True)
+    att = np.einsum("hts,shd->thd", p, v).reshape(T, H * D)
+    x = x + att @ w["wo"].T
+    n = norm(x, w["g_ffn"])
+    gu = n @ w["wgu"].T
+    g, u = gu[:, :F], gu[:, F:]
+    return x + (g / (1 + np.exp(-g)) * u) @ w["wd"].T
+
+
+def test_bf16_cache_rounds_rotated_keys_and_values_where_they_enter_the_cache():
+    # The whole layer with a bf16 cache against the dense formulation above, on 24 positions and a
+    # grouped-query layer: keys are rounded after the rotation, values as projected, queries and all
+    # arithmetic stay fp64.  The two plausible misplacements differ from the oracle by far more than
+    # the agreement asked of the right one.
+    spec = synth.TINY.with_(n_layers=1, n_early=1, n_kv_heads=2)
+    lw = synth.layer_weights(spec, 0)
+    emb, head = synth.embedding(spec), synth.lm_head(spec)
+    m = oracle.model_from_weights(spec, [lw], lw, emb, head, max_ctx=32, kv_bf16=True)
+    x0 = m.embed(synth.prompt_tokens(7, 24, spec.vocab).numpy()) * 30.0
+    got = m.layer_fwd(0, 0, x0, 0)
+    np.testing.assert_allclose(got, _dense_layer_bf16_cache(x0, lw, spec, "after"), rtol=0, atol=1e-10)
+    for wrong in ("before", "values_only"):
+        assert np.abs(got - _dense_layer_bf16_cache(x0, lw, spec, wrong)).max() > 1e-6
+    # cached across calls the same values come back: 16 rows, then 8 single rows
+    m2 = oracle.model_from_weights(spec, [lw], lw, emb, head, max_ctx=32, kv_bf16=True)
+    parts = [m2.layer_fwd(0, 0, x0[:16], 0)] + [m2.layer_fwd(0, 0, x0[i:i + 1], i) for i in range(16, 24)]
+    np.testing.assert_allclose(np.concatenate(parts), got, rtol=0, atol=1e-12)
+
+
+def test_bf16_cache_two_position_hand_case_key_rounded_after_rotation():
+    # D = 2, one head, two positions, hand numbers.  Raw key at position 1: (1 + 2^-8, 1).  bf16 keeps
+    # 8 significant bits, so rounding BEFORE the rotation turns it into (1, 1) (tie to even); rotated
+    # by 1 radian first it is (cos1 - sin1 - 2^-8 sin1 ..., ...) and rounds to other values.  The
+    # score difference s_1 - s_0 of the row at position 1 is read off the layer output through
+    # values (1, 0) and (0, 1): output - x = (w_0, w_1), w = softmax(s).
+    import types
+    D = 2
+    c1, s1 = math.cos(1.0), math.sin(1.0)
+    spec = types.SimpleNamespace(d_model=2, n_heads=1, n_kv_heads=1, head_dim=2, ffn_dim=2, vocab=2, n_early=1,
+                                 rms_eps=0.0, rope_theta=10000.0, dtype="bf16")
+    # rows of x are chosen so that RMSNorm (gain 1, eps 0) returns them: mean square 1
+    x = np.array([[1.0, 1.0], [1.0, -1.0]])
+    a, b = 1.0 + 2.0 ** -8, 1.0
+    # n_0 = (1, 1), n_1 = (1, -1): solve Wk n_0 = (1, 0) (position 0 is not rotated), Wk n_1 = (a, b)
+    wk = np.array([[(1 + a) / 2, (1 - a) / 2], [b / 2, -b / 2]])
+    wv = np.array([[0.5, 0.5], [0.5, -0.5]])   # v_0 = (1, 0), v_1 = (0, 1): exact in bf16
+    wq = np.array([[1.0, 0.0], [0.0, 1.0]])
+    lw = dict(g_attn=np.ones(2, np.float32), g_ffn=np.ones(2, np.float32), wqkv=np.concatenate([wq, wk, wv]).astype(np.float32),
+              wo=np.eye(2, dtype=np.float32), wgu=np.zeros((4, 2), np.float32), wd=np.zeros((2, 2), np.float32))
+    assert (lw["wqkv"].astype(np.float64) == np.concatenate([wq, wk, wv])).all()   # the weights are exact in fp32
+    emb = np.zeros((2, 2), np.float32)
+    m = oracle.model_from_weights(spec, [lw], lw, emb, emb, max_ctx=4, kv_bf16=True)
+    y = m.layer_fwd(0, 0, x, 0)
+    w = y[1] - x[1]
+    got = math.log(w[1] / w[0])                      # s_1 - s_0
+    q1 = np.array([c1 + s1, s1 - c1])                # (1, -1) rotated by 1 radian
+    k0 = np.array([1.0, 0.0])
+    k1_after = _bf16(np.array([a * c1 - b * s1, a * s1 + b * c1]))
+    k1_before = np.array([1.0 * c1 - 1.0 * s1, 1.0 * s1 + 1.0 * c1])   # bf16(a) = 1
+    want = (q1 @ k1_after - q1 @ k0) / math.sqrt(D)
+    wrong = (q1 @ k1_before - q1 @ k0) / math.sqrt(D)
+    assert abs(want - wrong) > 1e-4                  # the case tells the two placements apart
+    assert abs(got - want) < 1e-12
