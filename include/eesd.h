@@ -20,7 +20,9 @@
  *     acceptance entry points take a batch of independent sequences.
  *   - all work is enqueued on the CUDA stream given at eesd_init(); calls that return
  *     host-visible results synchronise that stream before returning.
- *   - a context is not thread-safe; use one per host thread / stream.
+ *   - a context is not thread-safe; use one per host thread / stream.  Contexts on different
+ *     host threads may be created and used concurrently (one-time set-up inside the library is
+ *     guarded).
  */
 #ifndef EESD_H
 #define EESD_H
@@ -267,6 +269,23 @@ int eesd_cali_state(const eesd_ctx *ctx, double *theta_hat, int64_t *n_verify, i
 int eesd_cali_posterior(double theta_m, double theta_hat, int64_t n, double sigma_m, double sigma_s,
                         double *mu, double *variance);
 
+/* The host-side controller arithmetic, exported so that it can be checked on its own (no context,
+ * no device).  These are the functions eesd_generate / eesd_decode / eesd_verify_accept call.
+ * eesd_ts_decide (Algorithm 2, draft loop): theta ~ Beta(alpha, beta), chi ~ Bernoulli(theta), from
+ * alpha + beta + 1 uniforms u[*cursor ...] (host): theta = X / (X + Y), X = sum of -ln u over the
+ * first alpha of them, Y over the next beta, chi = [next uniform < theta]; a zero uniform counts
+ * as 2^-25.  Returns chi (0 or 1) and advances *cursor; RNG when fewer than alpha + beta + 1
+ * uniforms are left (cursor unchanged), BADARG for non-positive parameters.  theta_out may be NULL.
+ * eesd_ts_posterior_update (Eq. 3-4; Algorithm 2, update steps) after a round that drafted
+ * n_draft = |Q_d| tokens and added q_v = |Q_v| tokens (accepted drafts + the target's own):
+ * r = q_v - 1, n = min(q_v + 1, n_draft) (EESD_TS_RULE_PAPER) or min(q_v, n_draft)
+ * (EESD_TS_RULE_SINGLE_FAILURE); alpha += r, beta += n - r.  BADARG unless 1 <= q_v <= n_draft + 1.
+ * eesd_cali_decide (Algorithm 3, draft loop): theta = mu + sqrt(variance) * sqrt(-2 ln u_0) *
+ * cos(2 pi u_1), chi = [u_2 < theta], three uniforms from u[*cursor ...]. */
+int eesd_ts_decide(int64_t alpha, int64_t beta, const float *u, int64_t n_u, int64_t *cursor, double *theta_out);
+int eesd_ts_posterior_update(int64_t *alpha, int64_t *beta, int q_v, int n_draft, int rule);
+int eesd_cali_decide(double mu, double variance, const float *u, int64_t n_u, int64_t *cursor, double *theta_out);
+
 /* Declares that the KV cache already holds n_ctx - 1 valid rows (whatever bytes the pool
  * contains) and that `pending` is the pending token: allocates pages, sets the length.  Used to
  * time a verify pass against a cache of a chosen length without running a prefill. */
@@ -295,8 +314,10 @@ int eesd_launch_count(const eesd_ctx *ctx, int64_t *n);
  * sequences (the acceptance step of eesd_verify_accept).  All pointers are device pointers:
  * p_logits [B][K+1][V] f32, q_logits [B][K][V] f32, tokens [B][K] i32 (the drafted x_i),
  * u_accept [B][K], u_resample [B]; outputs n_accept [B], next_token [B] (i32).  scratch: 16-byte
- * aligned, at least eesd_accept_scratch_bytes(B, K) bytes, contents irrelevant (the call clears
- * what it needs).  Asynchronous on `cuda_stream`.  Errors: BADARG, NOMEM (scratch), RNG. */
+ * aligned (BADARG otherwise), at least eesd_accept_scratch_bytes(B, K) bytes, contents irrelevant
+ * (the call clears what it needs).  A drafted token id outside [0, V) is rejected at its position
+ * (it cannot have been drawn from q); no logit is read for it.  Asynchronous on `cuda_stream`.
+ * Errors: BADARG, NOMEM (scratch), RNG. */
 size_t eesd_accept_scratch_bytes(int B, int K);
 int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *q_logits,
                          const int32_t *tokens, const float *u_accept, const float *u_resample,
@@ -315,8 +336,9 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
  * larger problems return EESD_ERR_NOMEM (use eesd_accept_resample with your own scratch).
  * Inputs, outputs, arithmetic and results are exactly those of eesd_accept_resample.  The call
  * performs no device allocation or free.  The first call on each device looks up the array's
- * device address (one cudaGetSymbolAddress, with that device current); make that first call
- * before any stream capture.  All calls share the one array and it keeps the previous call's
+ * device address (one cudaGetSymbolAddress, with that device current; the address is kept for
+ * the life of that device's primary context, so do not reset the device while the library is in
+ * use); make that first call before any stream capture.  All calls share the one array and it keeps the previous call's
  * contents (the call re-zeroes what has to start at zero): two calls whose kernels may overlap
  * on the GPU (different streams, no ordering between them) race on it and must be avoided. */
 #define EESD_STATIC_ACCEPT_MAX_BATCH 1024

@@ -111,6 +111,10 @@ def lib():
         L.eesd_cali_state.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.eesd_cali_posterior.argtypes = [C.c_double, C.c_double, C.c_int64, C.c_double, C.c_double,
                                           C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        i64p, f64p = C.POINTER(C.c_int64), C.POINTER(C.c_double)
+        L.eesd_ts_decide.argtypes = [C.c_int64, C.c_int64, vp, C.c_int64, i64p, f64p]
+        L.eesd_ts_posterior_update.argtypes = [i64p, i64p, C.c_int, C.c_int, C.c_int]
+        L.eesd_cali_decide.argtypes = [C.c_double, C.c_double, vp, C.c_int64, i64p, f64p]
         L.eesd_assume_context.argtypes = [vp, C.c_int, C.c_int32]
         L.eesd_verify_only.argtypes = [vp, vp, C.c_int]
         L.eesd_logits.argtypes = [vp, C.c_int, C.POINTER(vp)]
@@ -424,6 +428,36 @@ def cali_posterior(theta_m: float, theta_hat: float, n: int, sigma_m: float, sig
     if st:
         raise EesdError(st, "eesd_cali_posterior")
     return mu.value, var.value
+
+
+def ts_decide(alpha: int, beta: int, u, cursor: int = 0):
+    """eesd_ts_decide (host arithmetic): returns (chi, theta, new cursor)."""
+    u = _np_f32(u)
+    cur, th = C.c_int64(cursor), C.c_double()
+    chi = lib().eesd_ts_decide(alpha, beta, u.ctypes.data_as(C.c_void_p), len(u), C.byref(cur), C.byref(th))
+    if chi < 0:
+        raise EesdError(chi, "eesd_ts_decide")
+    return chi, th.value, cur.value
+
+
+def ts_posterior_update(alpha: int, beta: int, q_v: int, n_draft: int, rule: int = 0):
+    """eesd_ts_posterior_update (host arithmetic, Eq. 3-4): returns the new (alpha, beta)."""
+    a, b = C.c_int64(alpha), C.c_int64(beta)
+    st = lib().eesd_ts_posterior_update(C.byref(a), C.byref(b), q_v, n_draft, rule)
+    if st:
+        raise EesdError(st, "eesd_ts_posterior_update")
+    return a.value, b.value
+
+
+def cali_decide(mu: float, variance: float, u, cursor: int = 0):
+    """eesd_cali_decide (host arithmetic): returns (chi, theta, new cursor)."""
+    u = _np_f32(u)
+    cur, th = C.c_int64(cursor), C.c_double()
+    chi = lib().eesd_cali_decide(C.c_double(mu), C.c_double(variance), u.ctypes.data_as(C.c_void_p), len(u),
+                                 C.byref(cur), C.byref(th))
+    if chi < 0:
+        raise EesdError(chi, "eesd_cali_decide")
+    return chi, th.value, cur.value
 
 
 def sample_rows(logits: torch.Tensor, u: Optional[torch.Tensor], temperature: float) -> torch.Tensor:

@@ -16,6 +16,8 @@
 //   form, times 2^n.  Constants are given as fp32 bit patterns below.
 //   draw from weights w_v <= 1 with u = m_u 2^-24: W = sum_v trunc(w_v * 2^32) (64-bit),
 //   tau = (m_u * W) >> 24, result = smallest v whose inclusive integer prefix sum exceeds tau.
+#include <atomic>
+
 #include "../../include/eesd.h"
 #include "common.cuh"
 #include "kernels.cuh"
@@ -313,7 +315,9 @@ __global__ void __launch_bounds__(kAccThreads) accept_kernel(const float *p_logi
     if ((int)threadIdx.x < K && K <= EESD_MAX_ROWS) {   // one test per thread: their loads are in flight together
         const int j = threadIdx.x, t = x[j];
         bool ok;
-        if (greedy) {
+        if (t < 0 || t >= V) {   // not a token of this vocabulary: rejected where it stands, no address is formed
+            ok = false;
+        } else if (greedy) {
             ok = t == ld_stat(&st[j]).arg;
         } else {
             const float p = prob_of(pl[(size_t)j * V + t], ld_stat(&st[j]), T);
@@ -332,6 +336,7 @@ __global__ void __launch_bounds__(kAccThreads) accept_kernel(const float *p_logi
         } else {
             for (; j < K; j++) {
                 const int t = x[j];
+                if (t < 0 || t >= V) break;
                 const float p = prob_of(pl[(size_t)j * V + t], ld_stat(&st[j]), T);
                 const float q = prob_of(ql[(size_t)j * V + t], ld_stat(&st[K + 1 + j]), T);
                 if (!(__fmul_rn(u_acc[(size_t)b * K + j], q) < p)) break;
@@ -414,19 +419,21 @@ extern "C" int eesd_accept_resample_static(void *cuda_stream, const float *p_log
         return EESD_ERR_NOMEM;   // beyond the built-in scratch: use eesd_accept_resample with caller scratch
     // The array's name is only a host-side handle; the device address is looked up once per
     // device (with that device current) and remembered.
+    // Threads may race to fill a slot: they store the same address (atomically), so any order is
+    // fine.  The address belongs to the device's primary context and holds for its lifetime.
     constexpr int kMaxDevices = 64;
-    static void *dev_ptr[kMaxDevices] = {};
+    static std::atomic<void *> dev_ptr[kMaxDevices];
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return EESD_ERR_CUDA;
-    if (!dev_ptr[dev]) {
-        void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_accept_scratch) != cudaSuccess || !p) return EESD_ERR_CUDA;
-        dev_ptr[dev] = p;
+    void *scratch = dev_ptr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        if (cudaGetSymbolAddress(&scratch, g_static_accept_scratch) != cudaSuccess || !scratch) return EESD_ERR_CUDA;
+        dev_ptr[dev].store(scratch, std::memory_order_release);
     }
     cudaStream_t s = (cudaStream_t)cuda_stream;
     // the arrival counters must start at zero; the row statistics are overwritten before use
-    if (cudaMemsetAsync(dev_ptr[dev], 0, (size_t)B * sizeof(unsigned int), s) != cudaSuccess) return EESD_ERR_CUDA;
-    eesd::launch_accept(s, p_logits, q_logits, tokens, u_accept, u_resample, B, K, V, temperature, dev_ptr[dev],
+    if (cudaMemsetAsync(scratch, 0, (size_t)B * sizeof(unsigned int), s) != cudaSuccess) return EESD_ERR_CUDA;
+    eesd::launch_accept(s, p_logits, q_logits, tokens, u_accept, u_resample, B, K, V, temperature, scratch,
                         n_accept, next_token, nullptr);
     return cudaGetLastError() == cudaSuccess ? EESD_OK : EESD_ERR_CUDA;
 }

@@ -459,26 +459,17 @@ int read_error_word(eesd_ctx *c) {
     return c->h_result[2] ? EESD_ERR_DEVICE : EESD_OK;
 }
 
-// theta ~ Beta(alpha, beta) through two Gamma sums of -ln u, chi ~ Bernoulli(theta)
+// Controller decisions and posterior updates are pure host functions of the C ABI
+// (eesd_ts_decide, eesd_ts_posterior_update, eesd_cali_decide below); the context only keeps the state.
 int ts_continue(eesd_ctx *c, const eesd_uniforms *u, int64_t *cursor) {
     if (!u || !u->u_ctrl) return EESD_ERR_RNG;
-    if (*cursor + c->alpha + c->beta + 1 > u->n_ctrl) return EESD_ERR_RNG;
-    auto nl = [](float v) { return -log(v > 0.0f ? (double)v : 2.98023223876953125e-08); };
-    double X = 0.0, Y = 0.0;
-    for (int64_t i = 0; i < c->alpha; i++) X += nl(u->u_ctrl[(*cursor)++]);
-    for (int64_t i = 0; i < c->beta; i++) Y += nl(u->u_ctrl[(*cursor)++]);
-    const double theta = X / (X + Y);
-    return (double)u->u_ctrl[(*cursor)++] < theta ? 1 : 0;
+    return eesd_ts_decide(c->alpha, c->beta, u->u_ctrl, u->n_ctrl, cursor, nullptr);
 }
 
-// Eq. 3-4 with r = |Q_v| - 1 and n = min(|Q_v| + 1, |Q_d|) (Algorithm 2, update steps)
 void ts_update(eesd_ctx *c, int q_v, int n_draft) {
-    const int64_t r = q_v - 1;
-    int64_t n = c->cfg.ts_update_rule == EESD_TS_RULE_PAPER ? (q_v + 1 < n_draft ? q_v + 1 : n_draft)
-                                                            : (q_v < n_draft ? q_v : n_draft);
-    if (n < r) n = r;
-    c->alpha += r;
-    c->beta += n - r;
+    const int64_t a0 = c->alpha, b0 = c->beta;
+    eesd_ts_posterior_update(&c->alpha, &c->beta, q_v, n_draft, c->cfg.ts_update_rule);
+    const int64_t r = c->alpha - a0, n = r + (c->beta - b0);
     // TS with calibration: observed mean of chi over the verified drafts (theta_hat_0 counts as one)
     c->theta_hat = (c->theta_hat * (double)(c->n_trials + 1) + (double)r) / (double)(c->n_trials + n + 1);
     c->n_trials += n;
@@ -504,16 +495,12 @@ int run_cali_predict(eesd_ctx *c, int step) {
     return check_launch(c);
 }
 
-// posterior of Eq. 6-7, theta ~ N(mu, var) by Box-Muller, chi ~ Bernoulli(theta)
+// posterior of Eq. 6-7, then the draw of Algorithm 3
 int cali_continue(eesd_ctx *c, float theta_m, const eesd_uniforms *u, int64_t *cursor) {
-    if (!u || !u->u_ctrl || *cursor + 3 > u->n_ctrl) return EESD_ERR_RNG;
+    if (!u || !u->u_ctrl) return EESD_ERR_RNG;
     double mu, var;
     eesd_cali_posterior(theta_m, c->theta_hat, c->n_verify, c->cfg.cali_sigma_m, c->cfg.cali_sigma_s, &mu, &var);
-    auto nl = [](float v) { return -log(v > 0.0f ? (double)v : 2.98023223876953125e-08); };
-    const double r = sqrt(2.0 * nl(u->u_ctrl[(*cursor)++]));
-    const double z = r * cos(6.283185307179586476925286766559 * (double)u->u_ctrl[(*cursor)++]);
-    const double theta = mu + sqrt(var) * z;
-    return (double)u->u_ctrl[(*cursor)++] < theta ? 1 : 0;
+    return eesd_cali_decide(mu, var, u->u_ctrl, u->n_ctrl, cursor, nullptr);
 }
 
 void reset_sequence(eesd_ctx *c) {
@@ -1056,6 +1043,48 @@ int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new,
     return decode_impl(c, max_new, k_schedule, n_schedule, u, out, stats, trace, trace_cap, n_rounds, launches0, ms_p);
 }
 
+// -ln u of a controller uniform; a zero uniform counts as half the grid step, 2^-25
+static double minus_log_uniform(float u) { return -log(u > 0.0f ? (double)u : 0x1p-25); }
+
+int eesd_ts_decide(int64_t alpha, int64_t beta, const float *u, int64_t n_u, int64_t *cursor, double *theta_out) {
+    if (!u || !cursor || alpha < 1 || beta < 1 || *cursor < 0) return EESD_ERR_BADARG;
+    if (*cursor + alpha + beta + 1 > n_u) return EESD_ERR_RNG;
+    // Beta(alpha, beta) with integer parameters: Gamma(alpha, 1) / (Gamma(alpha, 1) + Gamma(beta, 1)),
+    // each Gamma with an integer shape a sum of that many unit exponentials
+    const float *p = u + *cursor;
+    double ga = 0.0, gb = 0.0;
+    for (int64_t i = 0; i < alpha; i++) ga += minus_log_uniform(p[i]);
+    for (int64_t i = 0; i < beta; i++) gb += minus_log_uniform(p[alpha + i]);
+    const double theta = ga / (ga + gb);
+    const int chi = (double)p[alpha + beta] < theta;
+    *cursor += alpha + beta + 1;
+    if (theta_out) *theta_out = theta;
+    return chi;
+}
+
+int eesd_ts_posterior_update(int64_t *alpha, int64_t *beta, int q_v, int n_draft, int rule) {
+    if (!alpha || !beta || q_v < 1 || n_draft < 1 || q_v > n_draft + 1) return EESD_ERR_BADARG;
+    if (rule != EESD_TS_RULE_PAPER && rule != EESD_TS_RULE_SINGLE_FAILURE) return EESD_ERR_BADARG;
+    const int64_t r = q_v - 1;                                             // accepted drafts: successes
+    const int64_t tried = rule == EESD_TS_RULE_PAPER ? q_v + 1 : q_v;      // |Q_v| + 1 as printed, or |Q_v|
+    const int64_t n = tried < n_draft ? tried : n_draft;                   // never below r, because r <= |Q_d|
+    *alpha += r;          // Eq. 3
+    *beta += n - r;       // Eq. 4
+    return EESD_OK;
+}
+
+int eesd_cali_decide(double mu, double variance, const float *u, int64_t n_u, int64_t *cursor, double *theta_out) {
+    if (!u || !cursor || !(variance >= 0.0) || *cursor < 0) return EESD_ERR_BADARG;
+    if (*cursor + 3 > n_u) return EESD_ERR_RNG;
+    const float *p = u + *cursor;
+    // Box-Muller: a standard normal from two uniforms
+    const double z = sqrt(2.0 * minus_log_uniform(p[0])) * cos(6.283185307179586476925286766559 * (double)p[1]);
+    const double theta = mu + sqrt(variance) * z;
+    *cursor += 3;
+    if (theta_out) *theta_out = theta;
+    return (double)p[2] < theta ? 1 : 0;
+}
+
 int eesd_cali_posterior(double theta_m, double theta_hat, int64_t n, double sigma_m, double sigma_s, double *mu,
                         double *variance) {
     if (!mu || !variance || !(sigma_m > 0.0) || !(sigma_s > 0.0) || n < 0) return EESD_ERR_BADARG;
@@ -1162,6 +1191,7 @@ int eesd_accept_resample(void *cuda_stream, const float *p_logits, const float *
     if (B < 1 || K < 1 || V < 1 || temperature < 0.f) return EESD_ERR_BADARG;
     if (temperature != 0.f && (!u_accept || !u_resample)) return EESD_ERR_RNG;
     if ((long long)B * (2 * K + 1) > 0x7fffffffLL) return EESD_ERR_UNSUPPORTED;
+    if ((uintptr_t)scratch & 15) return EESD_ERR_BADARG;   // the row statistics are read with 16-byte loads
     const size_t need = accept_scratch_bytes(B, K);
     if (scratch_bytes < need) return EESD_ERR_NOMEM;
     cudaStream_t s = (cudaStream_t)cuda_stream;

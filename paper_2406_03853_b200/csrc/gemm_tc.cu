@@ -484,14 +484,15 @@ typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, voi
                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeFn encode_fn() {
-    static EncodeFn fn = nullptr;
-    if (!fn) {
+    // looked up once; the initialisation of a function-local static is thread-safe
+    static const EncodeFn fn = [] {
         void *p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = (EncodeFn)p;
-    }
+            return (EncodeFn)p;
+        return (EncodeFn) nullptr;
+    }();
     return fn;
 }
 
@@ -541,16 +542,15 @@ StreamK tc_plan(int R, int K, int n_sm) {
 }
 
 int tc_init() {
-    static int done = 0;
-    if (!done) {
+    // once per process, whichever host thread comes first (thread-safe static initialisation)
+    static const int rc = [] {
         if (cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES) != cudaSuccess)
             return -1;
         if (cudaFuncSetAttribute(tc::gemm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::WSMEM_BYTES) != cudaSuccess)
             return -1;
-        if (!encode_fn()) return -1;
-        done = 1;
-    }
-    return 0;
+        return encode_fn() ? 0 : -1;
+    }();
+    return rc;
 }
 
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,

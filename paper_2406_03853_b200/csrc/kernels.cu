@@ -14,9 +14,8 @@ namespace eesd {
 typedef __nv_bfloat16 bf16;
 
 bool pdl_enabled() {
-    static int on = -1;
-    if (on < 0) on = getenv("EESD_NO_PDL") ? 0 : 1;
-    return on == 1;
+    static const bool on = getenv("EESD_NO_PDL") == nullptr;   // read once (thread-safe static initialisation)
+    return on;
 }
 
 // ------------------------------------------------------------------------------------ small utilities
@@ -809,11 +808,10 @@ static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, 
     const int chunks = Mtot > 0 ? (Mtot + kMaxRows - 1) / kMaxRows : 1;
     const size_t ml_off = (size_t)H * (Mtot > 0 ? n_split : kMaxSlices) * kMaxRows * D;
     const size_t smem = attn_smem_bytes((int)sizeof(AT), D, RB, pps * kv.page_tokens, rows, n_split);
-    static size_t configured = 0;   // largest dynamic shared memory size enabled so far
-    if (smem > configured) {
+    // once per instantiation (thread-safe static initialisation)
+    static const cudaError_t configured =
         cudaFuncSetAttribute(attn_kernel<AT, D, RB, NM, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
-        configured = 227 * 1024 - 1024;
-    }
+    (void)configured;
     launch_k(attn_kernel<AT, D, RB, NM, TR>, dim3(kv.Hkv, n_split, chunks * nbat), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv,
              apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, Mtot, nbat, ml_off, tr);
 }
