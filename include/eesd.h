@@ -67,7 +67,8 @@ typedef struct eesd_config {
     float rms_eps;        /* RMSNorm epsilon                                                    */
     float rope_theta;     /* rotary base; pairs (2i, 2i+1) turn by pos * theta^(-2i/D)          */
     int32_t page_tokens;  /* tokens per KV page (power of two, 8..128)                          */
-    int32_t max_ctx;      /* most tokens a sequence may hold (prompt + generated + drafts)      */
+    int32_t max_ctx;      /* most tokens a sequence may hold (prompt + generated + drafts);
+                             at most 12288, and 8192 for an fp32 cache with 128-token pages         */
     int32_t k_cap;        /* most draft tokens per round, 1 <= k_cap <= EESD_MAX_ROWS - 1       */
     float temperature;    /* 0: greedy (draft top-1, accept while equal to target top-1)        */
     int32_t controller;   /* EESD_CTRL_FIXED_K, EESD_CTRL_BETA_TS or EESD_CTRL_CALI_TS                */
@@ -130,11 +131,13 @@ typedef struct eesd_sizes {
 
 /* Caller-owned device memory.  kv_pool holds P = floor(kv_bytes / kv_page_bytes) pages laid
  * out [slot 0..L][page 0..P-1][K|V][H_kv] blocks of page_tokens * D elements; slot L is the
- * early-exit layer's cache.  A key block is stored transposed, [D/2][page_tokens][2] (pairs of
- * adjacent dimensions, one column per token); a value block is [page_tokens][D] with the 16-byte
- * chunks of token t's row permuted (chunk c sits at c ^ (t & 7)).  Both are internal formats:
- * the library writes and reads the pool itself.
- * The workspace must be zero-filled by the caller before eesd_init. */
+ * early-exit layer's cache.  The element order inside a block is an internal format (the library
+ * writes and reads the pool itself): for a bf16 cache both blocks are grids of 8 x 8 element
+ * groups, [token/8][D/8][8][8], keys with a group's 8 tokens as rows, values with its 8 dimensions
+ * as rows, which is the form the tensor cores take an operand in; for an fp32 cache keys are
+ * [D/2][page_tokens][2] and values [page_tokens][D] with 16-byte chunks permuted by the token.
+ * The workspace must be zero-filled by the caller before eesd_init; eesd_init zero-fills the KV
+ * pool itself (the attention kernel relies on the pool never holding a non-finite value). */
 typedef struct eesd_buffers {
     void *weights;   size_t weights_bytes;
     void *kv_pool;   size_t kv_bytes;
@@ -306,6 +309,26 @@ int eesd_logits(const eesd_ctx *ctx, int which, const float **device_ptr);
  * (index l + 1) and, in draft steps, after the early-exit layer (index L + 1) as
  * [index][row][d] fp32. */
 int eesd_capture_hidden(eesd_ctx *ctx, float *device_buf, size_t bytes);
+
+/* Bound of the waits inside the kernels.  Every wait of a kernel on data in flight (a bulk copy
+ * into shared memory, a tensor-core operation) polls at most `polls` times (about a second's worth
+ * by default; 0xffffffff restores the default); a wait that runs out makes its thread block raise
+ * the context's error word, skip the rest of its work, let the copies it has already requested land
+ * and return, and the call that reads results next returns EESD_ERR_DEVICE.  polls = 0 makes the
+ * first wait of every block give up at once: no result is produced, nothing is left in flight, and
+ * the error path can be exercised without stalling anything.
+ * eesd_clear_device_error: zeroes the error word and the counters a failed pass may have left half
+ * counted, and forgets the sequence (as eesd_reset); the context is usable again afterwards. */
+int eesd_set_wait_limit(eesd_ctx *ctx, uint32_t polls);
+int eesd_clear_device_error(eesd_ctx *ctx);
+
+/* How the attention kernel of a pass would cut a context of ctx_len tokens (host arithmetic, no
+ * device needed): pages per thread block and thread blocks ("slices") per KV head, for `pairs`
+ * (query head, new row) pairs per KV head on a device of n_sm multiprocessors.  A slice count
+ * above 64 cannot be merged; configurations that could need one are refused by eesd_init
+ * (UNSUPPORTED), and this call returns UNSUPPORTED for such a ctx_len. */
+int eesd_attention_plan(int dtype, int ctx_len, int page_tokens, int n_kv_heads, int pairs, int n_sm,
+                        int *pages_per_block, int *n_slices);
 
 /* Kernel launches issued by this context since creation. */
 int eesd_launch_count(const eesd_ctx *ctx, int64_t *n);

@@ -120,6 +120,9 @@ def lib():
         L.eesd_logits.argtypes = [vp, C.c_int, C.POINTER(vp)]
         L.eesd_capture_hidden.argtypes = [vp, vp, C.c_size_t]
         L.eesd_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
+        L.eesd_set_wait_limit.argtypes = [vp, C.c_uint32]
+        L.eesd_clear_device_error.argtypes = [vp]
+        L.eesd_attention_plan.argtypes = [C.c_int] * 6 + [C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.eesd_accept_scratch_bytes.restype = C.c_size_t
         L.eesd_accept_scratch_bytes.argtypes = [C.c_int, C.c_int]
         L.eesd_accept_resample.argtypes = [vp, vp, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_float, vp,
@@ -394,6 +397,13 @@ class Engine:
         self._check(lib().eesd_time_projection(self.h, which, M, C.byref(ms), C.byref(nb)), "eesd_time_projection")
         return ms.value, nb.value
 
+    def set_wait_limit(self, polls: Optional[int]):
+        """eesd_set_wait_limit; None restores the default bound."""
+        self._check(lib().eesd_set_wait_limit(self.h, 0xffffffff if polls is None else polls), "eesd_set_wait_limit")
+
+    def clear_device_error(self):
+        self._check(lib().eesd_clear_device_error(self.h), "eesd_clear_device_error")
+
     def launch_count(self) -> int:
         n = C.c_int64()
         self._check(lib().eesd_launch_count(self.h, C.byref(n)), "eesd_launch_count")
@@ -458,6 +468,15 @@ def cali_decide(mu: float, variance: float, u, cursor: int = 0):
     if chi < 0:
         raise EesdError(chi, "eesd_cali_decide")
     return chi, th.value, cur.value
+
+
+def attention_plan(dtype: int, ctx_len: int, page_tokens: int, n_kv_heads: int, pairs: int, n_sm: int = 148):
+    """eesd_attention_plan (host arithmetic): returns (pages per block, slices per KV head)."""
+    pps, ns = C.c_int(), C.c_int()
+    st = lib().eesd_attention_plan(dtype, ctx_len, page_tokens, n_kv_heads, pairs, n_sm, C.byref(pps), C.byref(ns))
+    if st:
+        raise EesdError(st, "eesd_attention_plan")
+    return pps.value, ns.value
 
 
 def sample_rows(logits: torch.Tensor, u: Optional[torch.Tensor], temperature: float) -> torch.Tensor:

@@ -30,7 +30,6 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int check_config(const eesd_config *c) {
     if (!c) return EESD_ERR_BADARG;
     if (c->d_model > 1024 * kSsqBlocks || c->n_kv_heads > 1024) return EESD_ERR_UNSUPPORTED;
-    if (c->max_ctx > 12288) return EESD_ERR_UNSUPPORTED;   // attention: at most 64 slices of 192 positions
     if (c->d_model <= 0 || c->n_heads <= 0 || c->n_kv_heads <= 0 || c->ffn_dim <= 0 || c->vocab <= 0 ||
         c->n_layers <= 0 || c->max_ctx <= 1)
         return EESD_ERR_BADARG;
@@ -40,6 +39,8 @@ int check_config(const eesd_config *c) {
     if (c->head_dim != 64 && c->head_dim != 128) return EESD_ERR_UNSUPPORTED;
     if (c->d_model % 8 || c->ffn_dim % 8 || (c->n_heads * c->head_dim) % 8) return EESD_ERR_UNSUPPORTED;
     if (c->page_tokens < 8 || c->page_tokens > 128 || (c->page_tokens & (c->page_tokens - 1))) return EESD_ERR_BADARG;
+    // attention: at most 64 slices per head, each as long as one block can hold
+    if (c->max_ctx > 12288 || c->max_ctx > attention_max_ctx(c->dtype, c->page_tokens)) return EESD_ERR_UNSUPPORTED;
     if (c->k_cap < 1 || c->k_cap > EESD_MAX_ROWS - 1) return EESD_ERR_BADARG;
     if (c->temperature < 0.f) return EESD_ERR_BADARG;
     if (c->controller != EESD_CTRL_FIXED_K && c->controller != EESD_CTRL_BETA_TS && c->controller != EESD_CTRL_CALI_TS)
@@ -67,6 +68,7 @@ constexpr int kIntSlots = 128;   // small device integer area
 constexpr int kMaxSm = 256;      // upper bound on the SM count the work splits are planned for
 constexpr int kCtasPerSm = 2;    // projection CTAs per SM (gemm_tc.cu: two 4-stage rings fit one SM)
 constexpr int kPrefillRows = 512; // most prompt rows per pass of the wide (prompt) path
+constexpr uint32_t kDefaultWaitPolls = 1u << 25;   // polls before a wait inside a kernel gives up (about a second)
 
 bool tc_shapes_ok(const eesd_config *c) {
     const int qd = c->n_heads * c->head_dim, kvd = c->n_kv_heads * c->head_dim;
@@ -184,6 +186,7 @@ struct eesd_ctx {
     CUtensorMap m_wx[3];
     CUtensorMap m_exit_kv, m_lm_head, m_exit_head;
     bool use_tc;
+    uint32_t wait_polls;         // bound of the waits inside the kernels (eesd_set_wait_limit)
     int n_sm;
     StreamK plan[P_COUNT];       // tensor-core path: work split per shape
     float2 *rope;
@@ -283,7 +286,7 @@ PartView run_proj(eesd_ctx *c, const void *W, const CUtensorMap *mW, int shape, 
     if (c->use_tc) {
         pv.mode = 1;
         pv.sk = c->plan[shape];
-        launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, c->plan[shape], M, true, c->err);
+        launch_gemm_tc(c->stream, *mW, c->m_x[which], c->part, c->plan[shape], M, true, c->err, c->wait_polls);
     } else {
         const float *A = which == X_NORM ? c->xn : which == X_ATTN ? c->attn : which == X_FFN ? c->h : c->hT;
         pv.mode = 0;
@@ -318,7 +321,7 @@ void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const fl
     const RowScale rs = norm_scale(c);
     PartView pv = run_proj(c, w.wqkv, &w.m_qkv, P_QKV, X_NORM, M, qd + 2 * kvd, d);
     launch_attention(s, f.dtype, pv, rs, c->rope, kv_geom(c, slot), c->apart, c->tickets, c->use_tc ? nullptr : c->attn,
-                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, true, c->err, c->tree_cur);
+                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, true, c->err, c->tree_cur, c->wait_polls);
     pv = run_proj(c, w.wo, &w.m_o, P_O, X_ATTN, M, d, qd);
     run_resid(c, &pv, w.g_ffn, nullptr, M);
     pv = run_proj(c, w.wgu, &w.m_gu, P_GU, X_NORM, M, 2 * F, d);
@@ -380,7 +383,7 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
     auto proj = [&](const CUtensorMap &mW, int which, int R, int K) {
         // narrow results (O, down, exit keys/values) leave SMs idle in the last wave: split their k range
         const int S = gemm_wide_splits(R, K, Mtot, c->n_sm, (int)(c->wout_floats / ((size_t)c->wide_rows * R)));
-        launch_gemm_wide(s, mW, c->m_wx[which], c->wout, R, K, Mtot, c->n_sm, true, S, c->err);
+        launch_gemm_wide(s, mW, c->m_wx[which], c->wout, R, K, Mtot, c->n_sm, true, S, c->err, c->wait_polls);
         c->launches++;
         PartView pv = {};
         pv.base = c->wout; pv.mode = 0; pv.S = S; pv.R = R; pv.split_stride = (size_t)Mtot * R;
@@ -400,7 +403,7 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
         PartView pv = proj(w.m_qkv, X_NORM, qd + 2 * kvd, d);
         // keys / values of all rows into the cache first, then every 16-row chunk attends in one launch
         launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, l), c->rope, nullptr, true, c->err, qd);
-        launch_attention_prompt(s, f.dtype, pv, rs, c->rope, kv_geom(c, l), c->wapart, c->tickets, c->wxs[X_ATTN], Mtot, p0, H, c->err);
+        launch_attention_prompt(s, pv, rs, c->rope, kv_geom(c, l), c->wapart, c->tickets, c->wxs[X_ATTN], Mtot, p0, H, c->err, c->wait_polls);
         c->launches += 2;
         pv = proj(w.m_o, X_ATTN, d, qd);
         resid(&pv, w.g_ffn);
@@ -738,6 +741,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->launches = 0;
     c->tree_cur = nullptr;
     c->leaves_kept = 0;
+    c->wait_polls = kDefaultWaitPolls;
     c->n_pages_total = pages > 0x7fffffff ? 0x7fffffff : pages;
     c->slot_bytes = (size_t)c->n_pages_total * 2 * cfg->n_kv_heads * cfg->page_tokens * cfg->head_dim * c->es;
     Workspace w = carve(cfg);
@@ -832,6 +836,10 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     cudaMemsetAsync(c->tickets, 0, ticket_count(cfg) * 4, c->stream);
     cudaMemsetAsync(c->ints, 0, kIntSlots * 4, c->stream);
     cudaMemsetAsync(c->accept_scratch, 0, accept_scratch_bytes(1, EESD_MAX_ROWS), c->stream);
+    // The tensor-core attention multiplies cached values past the end of a slice by weights that are
+    // exactly zero; that is only harmless while every value the pool ever holds is finite, so the pool
+    // starts as zeros (afterwards only this library writes it).
+    cudaMemsetAsync(b->kv_pool, 0, (size_t)(cfg->n_layers + 1) * c->slot_bytes, c->stream);
     launch_rope_table(c->stream, c->rope, cfg->max_ctx, cfg->head_dim, cfg->rope_theta);
     c->launches++;
     st = check_launch(c);
@@ -1114,6 +1122,39 @@ int eesd_cali_predict(eesd_ctx *c, float *theta_m) {
     return EESD_OK;
 }
 
+int eesd_set_wait_limit(eesd_ctx *c, uint32_t polls) {
+    if (!c) return EESD_ERR_BADARG;
+    c->wait_polls = polls == 0xffffffffu ? kDefaultWaitPolls : polls;
+    return EESD_OK;
+}
+
+int eesd_clear_device_error(eesd_ctx *c) {
+    if (!c) return EESD_ERR_BADARG;
+    // kernels that gave up may have left the merge counters of the attention kernel half counted
+    CU(c, cudaMemsetAsync(c->err, 0, 16, c->stream));
+    CU(c, cudaMemsetAsync(c->tickets, 0, ticket_count(&c->cfg) * 4, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    c->h_result[2] = 0;
+    reset_sequence(c);
+    return EESD_OK;
+}
+
+int eesd_attention_plan(int dtype, int ctx_len, int page_tokens, int n_kv_heads, int pairs, int n_sm, int *pages_per_block,
+                        int *n_slices) {
+    if ((dtype != EESD_F32 && dtype != EESD_BF16) || ctx_len < 1 || n_kv_heads < 1 || pairs < 1 || n_sm < 1 || !pages_per_block || !n_slices)
+        return EESD_ERR_BADARG;
+    if (page_tokens < 8 || page_tokens > 128 || (page_tokens & (page_tokens - 1))) return EESD_ERR_BADARG;
+    if (ctx_len > attention_max_ctx(dtype, page_tokens)) return EESD_ERR_UNSUPPORTED;
+    if (dtype == EESD_BF16) {
+        const int nc = attention_tc_columns(pairs);
+        *n_slices = attention_tc_splits(ctx_len, page_tokens, n_kv_heads, (pairs + nc - 1) / nc, n_sm, kAttnSplits, pages_per_block);
+    } else {
+        const int rb = pairs <= 8 ? 8 : pairs <= 24 ? 16 : 32;
+        *n_slices = attention_splits(ctx_len, page_tokens, n_kv_heads, (pairs + rb - 1) / rb, n_sm, kAttnSplits, pages_per_block);
+    }
+    return EESD_OK;
+}
+
 int eesd_context_len(const eesd_ctx *c, int *n_tokens, int *pages_in_use) {
     if (!c) return EESD_ERR_BADARG;
     if (n_tokens) *n_tokens = (int)c->tokens.size();
@@ -1246,7 +1287,7 @@ int eesd_project_rows(void *cuda_stream, int dtype, const float *A, const void *
         launch_split_rows(s, A, sc + off_xs, M, K);
         pv.mode = 1;
         pv.sk = sk;
-        launch_gemm_tc(s, mW, mX, part, sk, M, false, (int *)sc);
+        launch_gemm_tc(s, mW, mX, part, sk, M, false, (int *)sc, kDefaultWaitPolls);
     } else {
         pv.mode = 0;
         pv.S = launch_gemm(s, dtype, A, W, part, M, R, K);

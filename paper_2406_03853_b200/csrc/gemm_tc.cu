@@ -26,6 +26,7 @@
 
 #include "common.cuh"
 #include "kernels.cuh"
+#include "tc_ptx.cuh"
 
 namespace eesd {
 
@@ -38,114 +39,17 @@ constexpr int STAGE_BYTES = STAGE_W + STAGE_X;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr int THREADS = 192;  // warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA issuer
 constexpr uint32_t TMEM_COLS = 64;   // two 128 x 32 fp32 accumulators
-constexpr uint32_t SPIN_LIMIT = 1u << 25;  // polls of a barrier before a wait gives up (about a second)
 // The tensor core adds into its fp32 accumulator with truncation, so a long chain of MMAs
 // drifts towards zero.  Chains are therefore cut after KSEG k blocks (4 * KSEG MMAs): the
 // epilogue warps drain the accumulator and carry the sum in registers with IEEE fp32 adds.
 constexpr int KSEG = 16;
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// bounded wait; false (and the abort flag set) when the limit is reached or another role gave up
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
-                                          uint32_t sleep_ns = 0) {
-    for (uint32_t i = 0; i < SPIN_LIMIT; i++) {
-        if (mbar_try(bar, parity)) return true;   // non-blocking poll
-        if (sleep_ns) __nanosleep(sleep_ns);
-        if ((i & 1023u) == 1023u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    return false;
-}
-
-// same, with an L2 eviction-priority hint (the weight stream is read once per pass and should
-// not push activations, partial sums and the KV cache out of L2)
-__device__ __forceinline__ void tma_load_2d_hint(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y,
-                                                 uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
-        ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
-        : "memory");
-}
-__device__ __forceinline__ uint64_t policy_evict_first() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
-        : "memory");
-}
-
-// shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row
-// groups 1024 bytes apart
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                          // leading byte offset (unused with swizzle)
-    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                          // descriptor version for this architecture
-    d |= (uint64_t)2 << 61;                          // 128-byte swizzle
-    return d;
-}
-
 // instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 32
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-
-__device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint64_t *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
+constexpr uint32_t IDESC = idesc_bf16(BN);
 
 __global__ void __launch_bounds__(THREADS, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-               float *__restrict__ part, StreamK sk, int M, int tiled, int *err) {
+               float *__restrict__ part, StreamK sk, int M, int tiled, int *err, uint32_t spin) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sbase = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sW = sbase;
@@ -160,18 +64,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
     const int u0 = sk.start(cta), u1 = sk.start(cta + 1);
+    int issued = 0;   // producer thread: stages requested so far
     pdl_trigger();
 
     if (tid == 0) {
         for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
         for (int i = 0; i < 2; i++) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
         *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_init_fence();
     }
     if (warp == 5) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc(tmem_slot, TMEM_COLS);
     }
     tc_fence_before();
     __syncthreads();
@@ -195,25 +98,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 const int u = u0 + i, kb = u % sk.KB;
                 tma_load_2d(sX + i * STAGE_X, &tmX, &full[i], kb * BK, 0);
             }
-            int issued = pre;
+            issued = pre;
             bool ok = true;
             for (int u = u0 + pre; u < u1 && ok; u++, issued++) {
                 const int s = issued % STAGES, round = issued / STAGES;
-                ok = mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag);
+                ok = mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag, spin);
                 if (!ok) break;
                 const int tile = u / sk.KB, kb = u - tile * sk.KB;
                 mbar_expect_tx(&full[s], STAGE_BYTES);
                 tma_load_2d_hint(sW + s * STAGE_W, &tmW, &full[s], tiled ? 0 : kb * BK, tiled ? (tile * sk.KB + kb) * BM : tile * BM, stream_once);
                 tma_load_2d(sX + s * STAGE_X, &tmX, &full[s], kb * BK, 0);
-            }
-            if (*abort_flag) {
-                // let every copy still in flight land before the CTA's shared memory is released
-                const int first = issued > STAGES ? issued - STAGES : 0;
-                for (int i = first; i < issued; i++) {
-                    uint64_t *b = &full[i % STAGES];
-                    const uint32_t par = (uint32_t)((i / STAGES) & 1);
-                    for (uint32_t t = 0; t < SPIN_LIMIT && !mbar_try(b, par); t++) {}
-                }
             }
         }
     } else if (warp == 5) {
@@ -227,20 +121,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 for (int c0 = u; c0 < u_end && ok; c0 += KSEG, sub++) {
                     const int c1 = min(u_end, c0 + KSEG);
                     const int b = sub & 1, use = sub >> 1;
-                    ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag);
+                    ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag, spin);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t d_addr = tmem_base + (uint32_t)(b * BN);
                     for (int uu = c0; uu < c1; uu++, it++) {
                         const int s = it % STAGES, round = it / STAGES;
-                        ok = mbar_wait(&full[s], round & 1, abort_flag);
+                        ok = mbar_wait(&full[s], round & 1, abort_flag, spin);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint64_t da = smem_desc(smem_u32(sW + s * STAGE_W));
-                        const uint64_t db = smem_desc(smem_u32(sX + s * STAGE_X));
+                        const uint64_t da = smem_desc_sw128(smem_u32(sW + s * STAGE_W));
+                        const uint64_t db = smem_desc_sw128(smem_u32(sX + s * STAGE_X));
 #pragma unroll
                         for (int j = 0; j < BK / 16; j++)
-                            mma_bf16(d_addr, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), (uu > c0 || j > 0) ? 1u : 0u);
+                            mma_bf16(d_addr, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), IDESC, (uu > c0 || j > 0) ? 1u : 0u);
                         mma_commit(&empty[s]);   // the stage may be refilled once these MMAs have read it
                     }
                     if (!ok) break;
@@ -262,7 +156,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             for (int m = 0; m < kMaxRows; m++) acc[m] = 0.f;
             for (int c0 = u; c0 < u_end; c0 += KSEG, sub++) {
                 const int b = sub & 1, use = sub >> 1;
-                ok = mbar_wait(&acc_full[b], use & 1, abort_flag, 64);
+                ok = mbar_wait(&acc_full[b], use & 1, abort_flag, spin, 64);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -284,10 +178,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
-    if (tid == 0 && *abort_flag) atomicOr(err, kErrWaitTimeout);
+    if (*abort_flag) {   // some wait gave up (every role has stopped by now)
+        if (tid == 0) atomicOr(err, kErrWaitTimeout);
+        // let every copy still in flight land before the CTA's shared memory is released
+        if (warp == 4 && lane == 0)
+            for (int i = issued > STAGES ? issued - STAGES : 0; i < issued; i++) mbar_drain(&full[i % STAGES], (uint32_t)((i / STAGES) & 1));
+    }
     if (warp == 5) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -307,26 +206,11 @@ constexpr int WSTAGES = 4;
 constexpr int WSTAGE_X = WN * BK * 2, WSTAGE_BYTES = STAGE_W + WSTAGE_X;
 constexpr int WSMEM_BYTES = WSTAGES * WSTAGE_BYTES + 1024 + 256;
 constexpr uint32_t WTMEM_COLS = 512;
-constexpr uint32_t IDESC_W = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(WN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-
-__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y, int z, int w) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
-        : "memory");
-}
-__device__ __forceinline__ void mma_bf16_wide(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC_W), "r"(accumulate)
-        : "memory");
-}
+constexpr uint32_t IDESC_W = idesc_bf16(WN);
 
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                 float *__restrict__ out, int R, int KB, int Mtot, int panels, int tiled, int S, size_t split_stride, int *err) {
+                 float *__restrict__ out, int R, int KB, int Mtot, int panels, int tiled, int S, size_t split_stride, int *err, uint32_t spin) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sbase = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sW = sbase;
@@ -345,18 +229,17 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     const int n_tiles = (R / BM) * panels * S;
     const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // items cta, cta + G, ...
     const int n_units = my_tiles * KBs;
+    int issued = 0;   // producer thread: stages requested so far
     pdl_trigger();
 
     if (tid == 0) {
         for (int i = 0; i < WSTAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
         for (int i = 0; i < 2; i++) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
         *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_init_fence();
     }
     if (warp == 5) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(WTMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc(tmem_slot, WTMEM_COLS);
     }
     tc_fence_before();
     __syncthreads();
@@ -382,20 +265,12 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
             for (int i = 0; i < pre; i++) w_load(i, i);   // weights do not depend on the previous kernel
             pdl_wait();
             for (int i = 0; i < pre; i++) x_load(i, i);
-            int issued = pre;
+            issued = pre;
             for (; issued < n_units; issued++) {
                 const int s = issued % WSTAGES, round = issued / WSTAGES;
-                if (!mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag)) break;
+                if (!mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag, spin)) break;
                 w_load(issued, s);
                 x_load(issued, s);
-            }
-            if (*abort_flag) {
-                const int first = issued > WSTAGES ? issued - WSTAGES : 0;
-                for (int i = first; i < issued; i++) {
-                    uint64_t *b = &full[i % WSTAGES];
-                    const uint32_t par = (uint32_t)((i / WSTAGES) & 1);
-                    for (uint32_t t = 0; t < SPIN_LIMIT && !mbar_try(b, par); t++) {}
-                }
             }
         }
     } else if (warp == 5) {
@@ -407,20 +282,20 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                 for (int c0 = 0; c0 < KBs && ok; c0 += KSEG, sub++) {
                     const int c1 = min(KBs, c0 + KSEG);
                     const int b = sub & 1, use = sub >> 1;
-                    ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag);
+                    ok = mbar_wait(&acc_empty[b], (use & 1) ^ 1, abort_flag, spin);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t d_addr = tmem_base + (uint32_t)(b * WN);
                     for (int kb = c0; kb < c1; kb++, it++) {
                         const int s = it % WSTAGES, round = it / WSTAGES;
-                        ok = mbar_wait(&full[s], round & 1, abort_flag);
+                        ok = mbar_wait(&full[s], round & 1, abort_flag, spin);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint64_t da = smem_desc(smem_u32(sW + s * STAGE_W));
-                        const uint64_t db = smem_desc(smem_u32(sX + s * WSTAGE_X));
+                        const uint64_t da = smem_desc_sw128(smem_u32(sW + s * STAGE_W));
+                        const uint64_t db = smem_desc_sw128(smem_u32(sX + s * WSTAGE_X));
 #pragma unroll
                         for (int j = 0; j < BK / 16; j++)
-                            mma_bf16_wide(d_addr, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), (kb > c0 || j > 0) ? 1u : 0u);
+                            mma_bf16(d_addr, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), IDESC_W, (kb > c0 || j > 0) ? 1u : 0u);
                         mma_commit(&empty[s]);
                     }
                     if (!ok) break;
@@ -440,7 +315,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
             for (int i = 0; i < WROWS; i++) acc[i] = 0.f;
             for (int c0 = 0; c0 < KBs; c0 += KSEG, sub++) {
                 const int b = sub & 1, use = sub >> 1;
-                ok = mbar_wait(&acc_full[b], use & 1, abort_flag, 64);
+                ok = mbar_wait(&acc_full[b], use & 1, abort_flag, spin, 64);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -469,10 +344,14 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
-    if (tid == 0 && *abort_flag) atomicOr(err, kErrWaitTimeout);
+    if (*abort_flag) {
+        if (tid == 0) atomicOr(err, kErrWaitTimeout);
+        if (warp == 4 && lane == 0)
+            for (int i = issued > WSTAGES ? issued - WSTAGES : 0; i < issued; i++) mbar_drain(&full[i % WSTAGES], (uint32_t)((i / WSTAGES) & 1));
+    }
     if (warp == 5) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(WTMEM_COLS) : "memory");
+        tmem_dealloc(tmem_base, WTMEM_COLS);
     }
 }
 
@@ -554,9 +433,9 @@ int tc_init() {
 }
 
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
-                    int M, bool tiled, int *err) {
+                    int M, bool tiled, int *err, uint32_t wait_polls) {
     launch_k(tc::gemm_tc_kernel, dim3(sk.G), dim3(tc::THREADS), (size_t)tc::SMEM_BYTES, s, pdl_enabled(), mW, mX, part, sk, M,
-             (int)tiled, err);
+             (int)tiled, err, wait_polls);
 }
 
 int gemm_wide_splits(int R, int K, int Mtot, int n_sm, int max_splits) {
@@ -573,11 +452,11 @@ int gemm_wide_splits(int R, int K, int Mtot, int n_sm, int max_splits) {
 }
 
 void launch_gemm_wide(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *out, int R, int K, int Mtot,
-                      int n_sm, bool tiled, int splits, int *err) {
+                      int n_sm, bool tiled, int splits, int *err, uint32_t wait_polls) {
     const int panels = (Mtot + tc::WROWS - 1) / tc::WROWS;
     const int tiles = (R / tc::BM) * panels * splits;
     launch_k(tc::gemm_wide_kernel, dim3(tiles < n_sm ? tiles : n_sm), dim3(tc::THREADS), (size_t)tc::WSMEM_BYTES, s, pdl_enabled(),
-             mW, mX, out, R, K / tc::BK, Mtot, panels, (int)tiled, splits, (size_t)Mtot * R, err);
+             mW, mX, out, R, K / tc::BK, Mtot, panels, (int)tiled, splits, (size_t)Mtot * R, err, wait_polls);
 }
 
 // fp32 rows -> two bf16 terms: rows 0..15 hold hi = bf16(x), rows 16..31 hold lo = bf16(x - hi)

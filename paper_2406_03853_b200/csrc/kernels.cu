@@ -7,7 +7,9 @@
 
 #include "common.cuh"
 #include "kernels.cuh"
+#include "kv_layout.cuh"
 #include "partials.cuh"
+#include "tc_ptx.cuh"
 
 namespace eesd {
 
@@ -189,7 +191,6 @@ int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float 
 }
 
 // ------------------------------------------------------------------------------------ RoPE + KV append
-template <typename AT> __device__ __forceinline__ int v_elem(int pos, int e);
 // grid (heads, M), block D/2: one thread per rotation pair.
 template <typename AT>
 __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeom kv, const float2 *rope, float *q,
@@ -220,14 +221,13 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
         return;
     }
     AT *blk = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)kv.page_tokens * D;
+    const int p = pos % kv.page_tokens;   // element order inside a block: kv_layout.cuh
     if (isV) {
-        AT *dst = blk + (size_t)(pos % kv.page_tokens) * D + v_elem<AT>(pos, 2 * i);
-        dst[0] = from_f<AT>(a);
-        dst[1] = from_f<AT>(b);
-    } else {   // keys are cached transposed per page: pair i of a position at [i][pos % page_tokens]
-        AT *dst = blk + ((size_t)i * kv.page_tokens + (pos % kv.page_tokens)) * 2;
-        dst[0] = from_f<AT>(a);
-        dst[1] = from_f<AT>(b);
+        blk[v_index<AT>(pos, p, 2 * i, kv.page_tokens, D)] = from_f<AT>(a);
+        blk[v_index<AT>(pos, p, 2 * i + 1, kv.page_tokens, D)] = from_f<AT>(b);
+    } else {
+        blk[k_index<AT>(p, 2 * i, kv.page_tokens, D)] = from_f<AT>(a);
+        blk[k_index<AT>(p, 2 * i + 1, kv.page_tokens, D)] = from_f<AT>(b);
     }
 }
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
@@ -241,7 +241,8 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
     else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on);
 }
 
-// ------------------------------------------------------------------------------------ paged decode attention
+// ------------------------------------------------------------------------------------ paged decode attention, fp32 cache
+// (models with bf16 weights and cache run the tensor-core kernel of attn_tc.cu instead)
 // One kernel per layer: RoPE + KV append + attention over the paged cache + merge.
 // grid (H_kv, n_split), 256 threads.  Block (kh, sp) owns `cap` cached positions of KV head kh
 // (a whole number of pages) and serves every query head of its group and all M new rows from
@@ -262,45 +263,19 @@ constexpr int kRows16 = 24;       // up to this many (head, row) pairs per KV he
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// a pair of adjacent head dimensions of one key
-template <typename AT> struct KPair;
-template <> struct KPair<bf16> {
-    typedef uint32_t T;
-    __device__ __forceinline__ static T make(bf16 a, bf16 b) {
-        return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
-    }
-    __device__ __forceinline__ static void get(T w, float &a, float &b) {
-        a = __uint_as_float(w << 16);
-        b = __uint_as_float(w & 0xFFFF0000u);
-    }
-};
-template <> struct KPair<float> {
-    typedef float2 T;
-    __device__ __forceinline__ static T make(float a, float b) { return make_float2(a, b); }
-    __device__ __forceinline__ static void get(T w, float &a, float &b) { a = w.x; b = w.y; }
-};
-
-// Values are cached [page_tokens][D] with the 16-byte chunks of a token's row permuted by the
-// low three bits of its position (chunk c of token t sits at c ^ (t & 7)): eight consecutive
-// tokens then hold any given chunk in eight different bank groups, so the transposing matrix
-// loads of the PV product are conflict-free.  Index of element e of a row at position pos:
-template <typename AT> __device__ __forceinline__ int v_elem(int pos, int e) {
-    constexpr int CPV = 16 / (int)sizeof(AT);
-    return (((e / CPV) ^ (pos & 7)) * CPV) + (e % CPV);
-}
-
 // RB: (head, row) pairs per block: 8, 16 or 32; NM: most new rows (M <= NM), which sizes the
 // unrolled handling of the new keys / values (a one-row pass runs an eighth of the code); TR: the
 // new rows form a tree (per-row depth and visibility mask) instead of a chain.  The chain code is
 // kept as its own instantiation: with the mask lookups compiled in, an ordinary 13B pass of 1 / 16
 // rows measured 4.90 / 5.49 ms against 4.88 / 5.44 ms.
-template <typename AT, int D, int RB, int NM, bool TR>
+template <int D, int RB, int NM, bool TR>
 __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, const float2 *__restrict__ rope, KvGeom kv,
                                                    float *__restrict__ apart, unsigned int *tickets,
                                                    float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
                                                    int M, int pos0, int H, int pps, int n_split, float scale, int *err,
-                                                   int Mtot, int nbat, size_t ml_off, TreeRows tr) {
-    typedef typename KPair<AT>::T KP;
+                                                   int Mtot, int nbat, size_t ml_off, TreeRows tr, uint32_t spin) {
+    typedef float AT;
+    typedef float2 KP;   // a pair of adjacent head dimensions of one key
     constexpr int HALF = D / 2;
     constexpr int DPL = D / 32;             // output dimensions per lane in the PV phase
     extern __shared__ __align__(128) unsigned char attn_smem[];
@@ -308,13 +283,9 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     const int cap = pps * PT;               // positions this block's tiles hold
     KP *sK = reinterpret_cast<KP *>(attn_smem);                  // [pps][D/2][PT] pairs
     AT *sV = reinterpret_cast<AT *>(sK + (size_t)cap * HALF);   // [cap][D]
-    // rotated, scaled queries: fp32 pairs [RB][D/2] (fp32 cache), or two bf16 terms per pair,
-    // [2][RBP][QS] words (bf16 cache, tensor-core path; QS is padded against bank conflicts)
-    constexpr bool kTC = sizeof(AT) == 2;
-    constexpr int RBP = RB < 16 ? 16 : RB, QS = HALF + 4;
-    constexpr int SQ_WORDS = kTC ? 2 * RBP * QS : 2 * RB * HALF;
+    // rotated, scaled queries: fp32 pairs [RB][D/2]
+    constexpr int SQ_WORDS = 2 * RB * HALF;
     float2 *sq = reinterpret_cast<float2 *>(sV + (size_t)cap * D);
-    uint32_t *sqh = reinterpret_cast<uint32_t *>(sq), *sql = sqh + RBP * QS;
     const int ss = cap + 12;                                     // row stride of the score matrix
     float *sS = reinterpret_cast<float *>(sq) + SQ_WORDS;        // [RB][ss]
     float *s_m = sS + (size_t)RB * ss;                           // [RB]
@@ -322,7 +293,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     float *s_rstd = s_l + RB;                                    // [kMaxRows]
     uint64_t *bar = reinterpret_cast<uint64_t *>(s_rstd + kMaxRows);
     float *wgt = reinterpret_cast<float *>(bar + 2);             // [RB][n_split] merge weights
-    __shared__ int s_last;
+    __shared__ int s_last, s_abort;
     // which new rows a row sees and the position it is rotated as (a chain unless the pass verifies a tree)
     __shared__ uint16_t s_vis[kMaxRows];
     __shared__ uint8_t s_dep[kMaxRows];
@@ -358,9 +329,9 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     pdl_trigger();
     if (TR && tid >= 32 && tid < 32 + kMaxRows) { s_vis[tid - 32] = tr.vis[tid - 32]; s_dep[tid - 32] = tr.depth[tid - 32]; }
     if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(bar)));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        s_abort = 0;
+        tc::mbar_init(bar, 1);
+        tc::mbar_init_fence();
     }
     __syncthreads();
     if (warp == 0) {
@@ -478,28 +449,22 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const float a = qraw_a[it] * s_rstd[m], b = qraw_b[it] * s_rstd[m];
             const float2 cs = cs_q[it];
             const float qa = (a * cs.x - b * cs.y) * scale, qb = (a * cs.y + b * cs.x) * scale;
-            if (kTC) {
-                const bf16 ha = __float2bfloat16_rn(qa), hb = __float2bfloat16_rn(qb);
-                sqh[rl * QS + i] = KPair<bf16>::make(ha, hb);
-                sql[rl * QS + i] = KPair<bf16>::make(__float2bfloat16_rn(qa - __bfloat162float(ha)),
-                                                     __float2bfloat16_rn(qb - __bfloat162float(hb)));
-            } else {
-                sq[rl * HALF + i] = make_float2(qa, qb);
-            }
+            sq[rl * HALF + i] = make_float2(qa, qb);
         }
     }
     if (warp == 0) {   // wait for the cached slice (bounded); the other warps park at the barrier below
         bool ok = false;
-        for (uint32_t i = 0; i < (1u << 24) && !ok; i++) {
-            uint32_t p;
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                         : "=r"(p) : "r"(smem_addr(bar)) : "memory");
-            ok = p != 0;
+        for (uint32_t i = 0; i < spin && !ok; i++) {
+            ok = tc::mbar_try(bar, 0);
             if (!ok) __nanosleep(32);
         }
-        if (!ok && tid == 0) atomicOr(err, kErrWaitTimeout);
+        if (!ok && tid == 0) { s_abort = 1; atomicOr(err, kErrWaitTimeout); }
     }
     __syncthreads();
+    if (s_abort) {   // the wait gave up: nothing of the slice is used; its copies must still land before the block ends
+        if (tid == 0) tc::mbar_drain(bar, 0);
+        return;
+    }
 #pragma unroll
     for (int it = 0; it < kNewPerThread; it++) {
         const int idx = tid + it * 256;
@@ -520,67 +485,16 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                     blk[(size_t)(pos % PT) * D + e + 1] = new_b[it];
                 }
             } else {   // keys: pair i of position pos at [i][pos % PT] of the page block
-                const KP w2 = KPair<AT>::make(new_a[it], new_b[it]);
+                const KP w2 = make_float2(new_a[it], new_b[it]);
                 sK[(size_t)(j / PT) * PT * HALF + (size_t)i * PT + (j % PT)] = w2;
                 if (append) reinterpret_cast<KP *>(blk)[(size_t)i * PT + (pos % PT)] = w2;
             }
         }
     }
-    const int npos_k = min(cap, ((npos + 15) / 16) * 16);   // positions the PV products run over
-    if (kTC) {   // value rows past the slice hold whatever the page held: make them zeros
-        for (int idx = tid; idx < (npos_k - npos) * (D / 8); idx += 256)
-            reinterpret_cast<uint4 *>(sV + (size_t)npos * D)[idx] = make_uint4(0u, 0u, 0u, 0u);
-    }
     __syncthreads();
 
     {
-        if constexpr (kTC) {
-            // scores on the tensor cores: S = Q K^T as m16n8k16 products, Q = hi + lo (two bf16
-            // terms, exact products, fp32 accumulation).  The transposed key tile yields the
-            // B fragments as plain 32-bit loads: pair (2t, 2t+1) of position n0 + g.
-            const int g = lane >> 2, t = lane & 3;
-            const int n_tiles = (npos + 7) / 8;
-            for (int mt = 0; mt * 16 < nb; mt++) {
-                uint32_t ah[D / 16][4], al[D / 16][4];
-                const int ra = (mt * 16 + g) * QS, rb2 = (mt * 16 + g + 8) * QS;
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ks++) {
-                    ah[ks][0] = sqh[ra + ks * 8 + t];      ah[ks][1] = sqh[rb2 + ks * 8 + t];
-                    ah[ks][2] = sqh[ra + ks * 8 + t + 4];  ah[ks][3] = sqh[rb2 + ks * 8 + t + 4];
-                    al[ks][0] = sql[ra + ks * 8 + t];      al[ks][1] = sql[rb2 + ks * 8 + t];
-                    al[ks][2] = sql[ra + ks * 8 + t + 4];  al[ks][3] = sql[rb2 + ks * 8 + t + 4];
-                }
-                for (int nt = warp; nt < n_tiles; nt += 8) {
-                    const int n0 = nt * 8;
-                    const uint32_t *kp = reinterpret_cast<const uint32_t *>(sK) + (size_t)(n0 / PT) * PT * HALF + (n0 % PT) + g;
-                    float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ks++) {
-                        const uint32_t b0 = kp[(size_t)(ks * 8 + t) * PT], b1 = kp[(size_t)(ks * 8 + t + 4) * PT];
-                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                                     : "r"(ah[ks][0]), "r"(ah[ks][1]), "r"(ah[ks][2]), "r"(ah[ks][3]), "r"(b0), "r"(b1));
-                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                                     : "r"(al[ks][0]), "r"(al[ks][1]), "r"(al[ks][2]), "r"(al[ks][3]), "r"(b0), "r"(b1));
-                    }
-#pragma unroll
-                    for (int hf = 0; hf < 2; hf++) {
-                        const int rl = mt * 16 + g + 8 * hf;
-                        if (rl < nb) {
-                            const int m = (r0 + rl) % M;
-#pragma unroll
-                            for (int q2 = 0; q2 < 2; q2++) {
-                                const int j = n0 + 2 * t + q2;
-                                const int jn = lo + j - pos0;   // >= 0: a new row
-                                const bool seen = TR ? (jn < 0 || ((s_vis[m] >> jn) & 1)) : (jn <= m);
-                                sS[(size_t)rl * ss + j] = (j < npos && seen) ? c[hf * 2 + q2] : -INFINITY;
-                            }
-                        }
-                    }
-                }
-            }
-        } else {   // scores.  Work item = (16 consecutive positions, 8 rows); lane = position + 16 * (dimension pair parity)
+        {   // scores.  Work item = (16 consecutive positions, 8 rows); lane = position + 16 * (dimension pair parity)
             const int t = lane & 15, eh = lane >> 4;
             const int n_task = (npos + 15) / 16, n_rc = (nb + 7) / 8;
             for (int item = warp; item < n_task * n_rc; item += 8) {
@@ -594,8 +508,8 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                 for (int i = 0; i < 8; i++) acc[i] = 0.f;
 #pragma unroll 4
                 for (int e2 = eh; e2 < HALF; e2 += 2) {
-                    float ka, kb;
-                    KPair<AT>::get(kp[(size_t)e2 * PT], ka, kb);
+                    const KP kk = kp[(size_t)e2 * PT];
+                    const float ka = kk.x, kb = kk.y;
 #pragma unroll
                     for (int i = 0; i < 8; i++) {
                         const float2 qv = qp[i * HALF + e2];   // rows past nb hold stale values: results dropped
@@ -620,8 +534,8 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             }
         }
         __syncthreads();
-        const int nposw = kTC ? ((npos + 7) / 8) * 8 : min(cap, ((npos + 15) / 16) * 16);   // entries the score phase wrote
-        const int npos16 = max(nposw, npos_k);   // the tensor-core PV reads weights (zeros) up to npos_k
+        const int nposw = min(cap, ((npos + 15) / 16) * 16);   // entries the score phase wrote
+        const int npos16 = nposw;
         for (int rl = warp; rl < nb; rl += 8) {   // softmax numerators of this slice
             float mx = -INFINITY;
             for (int j = lane; j < nposw; j += 32) mx = fmaxf(mx, sS[(size_t)rl * ss + j]);
@@ -637,61 +551,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             if (lane == 0) { s_m[rl] = mx; s_l[rl] = sum; }
         }
         __syncthreads();
-        if constexpr (kTC) {
-            // o = P V on the tensor cores: P = hi + lo (two bf16 terms), V fragments by transposing
-            // matrix loads from the row-major value tile.  Warp w owns output dimensions 8w.. and
-            // 8(w+8)..; accumulators stay in registers over all positions.
-            const int g = lane >> 2, t = lane & 3;
-            for (int mt = 0; mt * 16 < nb; mt++) {
-                float c[D / 64][4];
-#pragma unroll
-                for (int x = 0; x < D / 64; x++) { c[x][0] = c[x][1] = c[x][2] = c[x][3] = 0.f; }
-                const float *pa = sS + (size_t)(mt * 16 + g) * ss, *pb = sS + (size_t)min(mt * 16 + g + 8, RB - 1) * ss;
-                for (int k0 = 0; k0 < npos_k; k0 += 16) {
-                    const float2 f0 = *reinterpret_cast<const float2 *>(pa + k0 + 2 * t);
-                    const float2 f1 = *reinterpret_cast<const float2 *>(pb + k0 + 2 * t);
-                    const float2 f2 = *reinterpret_cast<const float2 *>(pa + k0 + 2 * t + 8);
-                    const float2 f3 = *reinterpret_cast<const float2 *>(pb + k0 + 2 * t + 8);
-                    uint32_t ah[4], al[4];
-                    const float2 ff[4] = {f0, f1, f2, f3};
-#pragma unroll
-                    for (int x = 0; x < 4; x++) {
-                        const bf16 ha = __float2bfloat16_rn(ff[x].x), hb = __float2bfloat16_rn(ff[x].y);
-                        ah[x] = KPair<bf16>::make(ha, hb);
-                        al[x] = KPair<bf16>::make(__float2bfloat16_rn(ff[x].x - __bfloat162float(ha)),
-                                                  __float2bfloat16_rn(ff[x].y - __bfloat162float(hb)));
-                    }
-#pragma unroll
-                    for (int x = 0; x < D / 64; x++) {
-                        const int d0 = (warp + 8 * x) * 8;
-                        uint32_t b0, b1;
-                        const int jr = k0 + (lane & 15);
-                        const uint32_t addr = smem_addr(sV + (size_t)jr * D + v_elem<AT>(jr, d0));
-                        asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
-                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                     : "+f"(c[x][0]), "+f"(c[x][1]), "+f"(c[x][2]), "+f"(c[x][3])
-                                     : "r"(ah[0]), "r"(ah[1]), "r"(ah[2]), "r"(ah[3]), "r"(b0), "r"(b1));
-                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                     : "+f"(c[x][0]), "+f"(c[x][1]), "+f"(c[x][2]), "+f"(c[x][3])
-                                     : "r"(al[0]), "r"(al[1]), "r"(al[2]), "r"(al[3]), "r"(b0), "r"(b1));
-                    }
-                }
-#pragma unroll
-                for (int hf = 0; hf < 2; hf++) {
-                    const int rl = mt * 16 + g + 8 * hf;
-                    if (rl < nb) {
-                        const int gq = (r0 + rl) / M, m = (r0 + rl) - gq * M, h = kh * group + gq;
-                        float *dst = apart + (((size_t)h * n_split + sp) * kMaxRows + m) * D;
-#pragma unroll
-                        for (int x = 0; x < D / 64; x++) {
-                            const int d0 = (warp + 8 * x) * 8;
-                            *reinterpret_cast<float2 *>(dst + d0 + 2 * t) = make_float2(c[x][hf * 2], c[x][hf * 2 + 1]);
-                        }
-                        if (warp == 0 && t == 0) ml[((size_t)h * kMaxRows + m) * kMaxSlices + sp] = make_float2(s_m[rl], s_l[rl]);
-                    }
-                }
-            }
-        } else {   // o = P V.  Warp w owns rows w, w + 8, ... of the batch; lane owns DPL output dimensions
+        {   // o = P V.  Warp w owns rows w, w + 8, ... of the batch; lane owns DPL output dimensions
             constexpr int RPW = RB / 8;
             float o[RPW][DPL];
 #pragma unroll
@@ -793,37 +653,34 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     }
 }
 
-static size_t attn_smem_bytes(int es, int D, int RB, int cap, int rows, int n_split) {
-    const int rbp = RB < 16 ? 16 : RB;
-    const size_t sq_words = es == 2 ? (size_t)2 * rbp * (D / 2 + 4) : (size_t)RB * D;
-    return (size_t)2 * cap * D * es + sq_words * 4 + (size_t)RB * (cap + 12) * 4 + 2 * RB * 4 + kMaxRows * 4 + 16 +
+static size_t attn_smem_bytes(int D, int RB, int cap, int n_split) {
+    return (size_t)2 * cap * D * 4 + (size_t)RB * D * 4 + (size_t)RB * (cap + 12) * 4 + 2 * RB * 4 + kMaxRows * 4 + 16 +
            (size_t)RB * n_split * 4 + 16;
 }
 
-template <typename AT, int D, int RB, int NM, bool TR>
+template <int D, int RB, int NM, bool TR>
 static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                         float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                        int pps, int n_split, float scale, bool early, int *err, int Mtot, const TreeRows &tr) {
+                        int pps, int n_split, float scale, bool early, int *err, const TreeRows &tr, uint32_t wait_polls) {
     const int rows = (H / kv.Hkv) * M, nbat = (rows + RB - 1) / RB;
-    const int chunks = Mtot > 0 ? (Mtot + kMaxRows - 1) / kMaxRows : 1;
-    const size_t ml_off = (size_t)H * (Mtot > 0 ? n_split : kMaxSlices) * kMaxRows * D;
-    const size_t smem = attn_smem_bytes((int)sizeof(AT), D, RB, pps * kv.page_tokens, rows, n_split);
+    const size_t ml_off = (size_t)H * kMaxSlices * kMaxRows * D;
+    const size_t smem = attn_smem_bytes(D, RB, pps * kv.page_tokens, n_split);
     // once per instantiation (thread-safe static initialisation)
     static const cudaError_t configured =
-        cudaFuncSetAttribute(attn_kernel<AT, D, RB, NM, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
+        cudaFuncSetAttribute(attn_kernel<D, RB, NM, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
     (void)configured;
-    launch_k(attn_kernel<AT, D, RB, NM, TR>, dim3(kv.Hkv, n_split, chunks * nbat), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv,
-             apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, Mtot, nbat, ml_off, tr);
+    launch_k(attn_kernel<D, RB, NM, TR>, dim3(kv.Hkv, n_split, nbat), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv,
+             apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, 0, nbat, ml_off, tr, wait_polls);
 }
 
-template <typename AT, int D>
+template <int D>
 static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                           float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                          int pps, int n_split, float scale, bool early, int *err, int Mtot, const TreeRows *tree) {
+                          int pps, int n_split, float scale, bool early, int *err, const TreeRows *tree, uint32_t wait_polls) {
     const int rows = (H / kv.Hkv) * M;
     const TreeRows tr = tree ? *tree : chain_rows();
-#define EESD_ATTN(RB, NM) attn_launch<AT, D, RB, NM, false>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr)
-#define EESD_ATTN_TREE(RB, NM) attn_launch<AT, D, RB, NM, true>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr)
+#define EESD_ATTN(RB, NM) attn_launch<D, RB, NM, false>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls)
+#define EESD_ATTN_TREE(RB, NM) attn_launch<D, RB, NM, true>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls)
     if (tree) {   // tree passes: one instantiation per batch size
         if (rows <= 8) EESD_ATTN_TREE(8, 8);
         else if (rows <= kRows16) EESD_ATTN_TREE(16, 16);
@@ -843,7 +700,7 @@ static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs
 #undef EESD_ATTN_TREE
 }
 
-// slices of the cached context: pages per block and number of blocks per KV head
+// slices of the cached context (fp32 kernel): pages per block and number of blocks per KV head
 int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out) {
     const int n_pages = (ctx_len + page_tokens - 1) / page_tokens;
     const int cap = kAttnPos / page_tokens > 0 ? kAttnPos / page_tokens : 1;   // pages one block can hold
@@ -856,43 +713,43 @@ int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n
     if (pps > cap) pps = cap;            // longer contexts: more slices than one wave holds
     if (pps < 1) pps = 1;
     if ((pps * page_tokens) % 16) pps++;   // tiles hold a multiple of 16 positions
-    int n_split = (n_pages + pps - 1) / pps;
-    while (n_split > max_splits && pps < cap) { pps += (page_tokens < 16 ? 2 : 1); n_split = (n_pages + pps - 1) / pps; }
     *pps_out = pps;
-    return n_split;
+    return (n_pages + pps - 1) / pps;
 }
 
-static void attention_any(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
-                          const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
-                          int M, int pos0, int H, int pps, int n_split, bool early, int *err, int Mtot, const TreeRows *tr) {
-    const float scale = 1.0f / sqrtf((float)kv.D);
-    if (dtype == 0) {
-        if (kv.D == 64) attn_dispatch<float, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr);
-        else attn_dispatch<float, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr);
-    } else {
-        if (kv.D == 64) attn_dispatch<bf16, 64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr);
-        else attn_dispatch<bf16, 128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr);
-    }
+// most context tokens the attention kernels can serve: at most kMaxSlices slices per head, each as
+// long as one block can hold (fp32 cache: 192 positions, or one page of 128; bf16 cache: 256)
+int attention_max_ctx(int dtype, int page_tokens) {
+    if (dtype != 0) return kMaxSlices * 256;
+    int pps = kAttnPos / page_tokens > 0 ? kAttnPos / page_tokens : 1;
+    if ((pps * page_tokens) % 16) pps++;
+    return kMaxSlices * pps * page_tokens;
 }
 
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
-                      int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err, const TreeRows *tree) {
+                      int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err, const TreeRows *tree,
+                      uint32_t wait_polls) {
     int pps;
-    const int rows = (H / kv.Hkv) * M, rb = rows <= 8 ? 8 : rows <= kRows16 ? 16 : 32;
+    const int rows = (H / kv.Hkv) * M;
+    if (dtype != 0) {   // bf16 cache: tensor-core kernel
+        const int nc = attention_tc_columns(rows);
+        const int n_split = attention_tc_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + nc - 1) / nc, n_sm, max_splits, &pps);
+        launch_attention_tc(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, 0, tree,
+                            wait_polls);
+        return;
+    }
+    const int rb = rows <= 8 ? 8 : rows <= kRows16 ? 16 : 32;
     const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb, n_sm, max_splits, &pps);
-    attention_any(s, dtype, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, 0, tree);
+    const float scale = 1.0f / sqrtf((float)kv.D);
+    if (kv.D == 64) attn_dispatch<64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls);
+    else attn_dispatch<128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls);
 }
 
-// Prompt attention: Mtot rows at positions pos0.. whose keys / values are in the cache already
-// (launch_qkv_post), all 16-row chunks in one launch.  Slices are as long as a block can hold.
-static int prompt_pps(int page_tokens) {
-    int pps = kAttnPos / page_tokens > 0 ? kAttnPos / page_tokens : 1;
-    if ((pps * page_tokens) % 16) pps++;
-    return pps;
-}
+// Prompt attention (bf16 models): Mtot rows at positions pos0.. whose keys / values are in the cache
+// already (launch_qkv_post), all 16-row chunks in one launch.  Slices are as long as a block can hold.
 int attention_prompt_splits(int ctx_len, int page_tokens) {
-    const int pps = prompt_pps(page_tokens), n_pages = (ctx_len + page_tokens - 1) / page_tokens;
+    const int pps = attention_tc_prompt_pps(page_tokens), n_pages = (ctx_len + page_tokens - 1) / page_tokens;
     return (n_pages + pps - 1) / pps;
 }
 size_t attention_prompt_scratch_floats(int ctx_len, int page_tokens, int H, int D, int rows) {
@@ -900,12 +757,12 @@ size_t attention_prompt_scratch_floats(int ctx_len, int page_tokens, int H, int 
     const size_t per_chunk = (size_t)H * attention_prompt_splits(ctx_len, page_tokens) * kMaxRows * D + (size_t)H * kMaxRows * kMaxSlices * 2;
     return chunks * per_chunk;
 }
-void launch_attention_prompt(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
+void launch_attention_prompt(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope,
                              const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
-                             int Mtot, int pos0, int H, int *err) {
-    const int pps = prompt_pps(kv.page_tokens), n_split = attention_prompt_splits(pos0 + Mtot, kv.page_tokens);
-    attention_any(s, dtype, pv, rs, rope, kv, apart, tickets, nullptr, attn_split, kMaxRows, pos0, H, pps, n_split, false, err, Mtot,
-                  nullptr);
+                             int Mtot, int pos0, int H, int *err, uint32_t wait_polls) {
+    const int pps = attention_tc_prompt_pps(kv.page_tokens), n_split = attention_prompt_splits(pos0 + Mtot, kv.page_tokens);
+    launch_attention_tc(s, pv, rs, rope, kv, apart, tickets, nullptr, attn_split, kMaxRows, pos0, H, pps, n_split, false, err, Mtot,
+                        nullptr, wait_polls);
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU, partial sums
@@ -1066,8 +923,8 @@ __global__ void kv_move_kernel(KvGeom kv, size_t slot_bytes, int pos0, const int
     const int sj = src % PT, dj = dst % PT;
 #pragma unroll
     for (int e = 0; e < 2; e++) {
-        kd[((size_t)i * PT + dj) * 2 + e] = ks[((size_t)i * PT + sj) * 2 + e];
-        vd[(size_t)dj * D + v_elem<AT>(dst, 2 * i + e)] = vs[(size_t)sj * D + v_elem<AT>(src, 2 * i + e)];
+        kd[k_index<AT>(dj, 2 * i + e, PT, D)] = ks[k_index<AT>(sj, 2 * i + e, PT, D)];
+        vd[v_index<AT>(dst, dj, 2 * i + e, PT, D)] = vs[v_index<AT>(src, sj, 2 * i + e, PT, D)];
     }
 }
 void launch_kv_move(cudaStream_t s, int dtype, const KvGeom &kv0, size_t slot_bytes, int slots, int pos0,

@@ -15,8 +15,7 @@ struct IntList16 { int32_t v[16]; };
 // geometry of one paged KV cache slot
 struct KvGeom {
     void *slot_base;            // first byte of the slot: [page][K|V][H_kv] blocks of page_tokens * D
-                                // elements; K block [D/2][page_tokens][2], V block [page_tokens][D] with the 16-byte
-                                // chunks of token t's row permuted (chunk c at c ^ (t & 7))
+                                // elements; element order inside a block: kv_layout.cuh
     const int32_t *page_table;  // logical page -> physical page
     int Hkv, D, page_tokens, n_pages_total;
 };
@@ -98,16 +97,27 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
                       int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err,
-                      const TreeRows *tree = nullptr);
+                      const TreeRows *tree, uint32_t wait_polls);
+// most context tokens the attention kernel of `dtype` can serve with pages of page_tokens
+int attention_max_ctx(int dtype, int page_tokens);
+// tensor-core attention (attn_tc.cu; bf16 cache): columns ((head, row) pairs) per block for `rows` pairs per KV head,
+// slices of the context, pages per block in prompt mode, and the launcher (Mtot > 0: prompt mode)
+int attention_tc_columns(int rows);
+int attention_tc_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out);
+int attention_tc_prompt_pps(int page_tokens);
+void launch_attention_tc(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv, float *apart,
+                         unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H, int pps, int n_split,
+                         bool early, int *err, int Mtot, const TreeRows *tree, uint32_t wait_polls);
 // Prompt attention: all 16-row chunks of Mtot rows in one launch; the rows' keys / values must be
 // in the cache already (launch_qkv_post with only_kv on the QKV result) and pv must be a plain
 // [Mtot][R] result (mode 0).  apart: attention_prompt_scratch_floats(...) floats; tickets: zeroed
 // counters, one per (chunk, KV head, batch).  attn_split: [chunk][hi | lo][16][H * D] bf16.
+int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out);
 int attention_prompt_splits(int ctx_len, int page_tokens);
 size_t attention_prompt_scratch_floats(int ctx_len, int page_tokens, int H, int D, int rows);
-void launch_attention_prompt(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
+void launch_attention_prompt(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope,
                              const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
-                             int Mtot, int pos0, int H, int *err);
+                             int Mtot, int pos0, int H, int *err, uint32_t wait_polls);
 // H^(T) of the calibration predictor: row `row` (or row *row_dev when row_dev is given) of x[.][d]
 // is copied to hT (fp32) and, if xs is given, written as two bf16 terms into a one-chunk [32][d] matrix
 void launch_copy_row(cudaStream_t s, const float *x, int row, const int32_t *row_dev, float *hT, void *xs, int d);
@@ -141,8 +151,9 @@ bool tc_shape_ok(int R, int K);
 // tiled: the matrix is stored tile-major, [rows / 128][cols / 64] tiles of [128][64] (box_rows must be 128)
 bool tc_make_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows, bool tiled = false);
 StreamK tc_plan(int R, int K, int n_sm);
+// wait_polls: polls after which a wait inside the kernel gives up and raises the error word
 void launch_gemm_tc(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *part, const StreamK &sk,
-                    int M, bool tiled, int *err);
+                    int M, bool tiled, int *err, uint32_t wait_polls);
 // wide projection for prompt processing: out[m][r] (fp32, row stride R) for m < Mtot rows kept
 // as [chunk of 16][hi | lo][16][K] bf16 (mX from tc_make_map_rows); R % 128 == 0, K % 64 == 0
 bool tc_make_map_rows(CUtensorMap *out, const void *base, int K, int chunks);
@@ -150,7 +161,7 @@ bool tc_make_map_rows(CUtensorMap *out, const void *base, int K, int chunks);
 // mode 0 with S = splits); gemm_wide_splits picks the count that fills the SMs best (at most max_splits)
 int gemm_wide_splits(int R, int K, int Mtot, int n_sm, int max_splits);
 void launch_gemm_wide(cudaStream_t s, const CUtensorMap &mW, const CUtensorMap &mX, float *out, int R, int K, int Mtot,
-                      int n_sm, bool tiled, int splits, int *err);
+                      int n_sm, bool tiled, int splits, int *err, uint32_t wait_polls);
 void launch_split_rows(cudaStream_t s, const float *x, void *xs, int M, int K);
 
 // acceptance / sampling (accept.cu)

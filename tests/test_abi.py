@@ -97,3 +97,33 @@ def test_binding_refuses_to_run_without_cuda():
     import eesd_synth as synth
     with pytest.raises(RuntimeError):
         eesd.Engine(config_from_spec(synth.TINY))
+
+
+def test_attention_plan_never_needs_more_slices_than_can_be_merged(L):
+    # every allowed page size, every context length up to what the configuration check admits, the
+    # fewest and the most (head, row) pairs: at most 64 slices per head, slices of a whole number of
+    # 16-position steps, every page covered, and a block never holds more than its kernel can
+    from paper_2406_03853_b200 import binding as b
+    for dtype, block_cap in ((b.F32, 192), (b.BF16, 256)):
+        for pt in (8, 16, 32, 64, 128):
+            limit = 12288
+            pps, ns = C.c_int(), C.c_int()
+            while L.eesd_attention_plan(dtype, limit, pt, 8, 1, 148, C.byref(pps), C.byref(ns)) != 0:
+                limit -= pt
+            assert limit >= 8192
+            assert L.eesd_attention_plan(dtype, limit + 1, pt, 8, 1, 148, C.byref(pps), C.byref(ns)) == -8 or limit == 12288
+            for ctx in list(range(1, 600)) + list(range(600, limit + 1, 97)) + [limit]:
+                for hkv, pairs in ((1, 1), (8, 8), (40, 16), (8, 128), (1024, 1)):
+                    pp, n = b.attention_plan(dtype, ctx, pt, hkv, pairs)
+                    assert 1 <= n <= 64 and pp >= 1
+                    assert (pp * pt) % 16 == 0
+                    assert pp * pt <= max(block_cap, pt) + (8 if pt == 8 else 0)
+                    assert pp * n >= (ctx + pt - 1) // pt > pp * (n - 1)
+    # a configuration whose context could need more than 64 slices is refused
+    from tests.helpers import config_from_spec
+    import eesd_synth as synth
+    cfg = config_from_spec(synth.TINY, max_ctx=8192 + 128, page_tokens=128)
+    sz = b.Sizes()
+    assert L.eesd_required_bytes(C.byref(cfg), C.byref(sz)) == -8
+    cfg = config_from_spec(synth.TINY, max_ctx=8192, page_tokens=128)
+    assert L.eesd_required_bytes(C.byref(cfg), C.byref(sz)) == 0

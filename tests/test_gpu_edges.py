@@ -191,3 +191,30 @@ def test_long_context_many_slices(dtype):
     _, lg = m.target_rows(new, n_prompt - 1)
     assert np.abs(eng.logits(0, 9).cpu().numpy() - lg).max() < tol
     eng.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(dtype):
+    # With the bound of the in-kernel waits at zero, the first wait of every thread block (attention:
+    # its cache slice; projection: the first ring stage / accumulator) gives up before any tensor-core
+    # operation is issued; the blocks let the copies they had requested land and return.  The call
+    # must report a device error (not hang, not fault), and after clearing it the same context must
+    # produce the oracle's tokens again.  Nothing is stalled on the GPU to get here.
+    from paper_2406_03853_b200 import EesdError
+    spec = synth.TINY if dtype == "f32" else synth.TINY.with_(dtype="bf16", ffn_dim=640)
+    eng = engine_from_spec(spec, max_ctx=96, fixed_k=3)
+    prompt = synth.prompt_tokens(21, 12, spec.vocab).numpy()
+    out0, trace0, _ = eng.generate(prompt, 16)
+    eng.set_wait_limit(0)
+    with pytest.raises(EesdError) as e:
+        eng.generate(prompt, 16)
+    assert e.value.status == -7                             # EESD_ERR_DEVICE
+    eng.set_wait_limit(None)
+    eng.clear_device_error()
+    out1, trace1, _ = eng.generate(prompt, 16)
+    np.testing.assert_array_equal(out1, out0)
+    assert trace1 == trace0
+    if dtype == "f32":
+        ref, rtrace, _ = oracle_from_spec(spec, 96).generate(prompt, 16, fixed_k=3)
+        np.testing.assert_array_equal(out1, ref)
+    eng.close()
