@@ -52,6 +52,40 @@ __device__ __forceinline__ int f2ord(float f) {
 }
 __device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
+// 2^x by the special-function unit (2^-inf = 0)
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Sums of N = 16 or 32 per-lane values v[c] over the 32 lanes of a warp, all columns at once: each
+// step halves the columns a lane carries (lanes with the step's bit set keep the upper half and
+// hand over the lower one), so the whole reduction takes N shuffles instead of 5 N.  Returns the
+// sum of column `lane` (N = 32) or `lane / 2` (N = 16, both lanes of a pair hold it).  The order
+// of the additions is fixed.
+template <int N>
+__device__ __forceinline__ float column_sums(float (&v)[N], int lane) {
+    int n = N;
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        if (n == 1) {   // N = 16, last step: the pair's two halves of one column
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], s);
+        } else {
+            const bool up = (lane & s) != 0;
+            n >>= 1;
+#pragma unroll
+            for (int i = 0; i < N / 2; i++) {
+                if (i < n) {
+                    const float send = up ? v[i] : v[i + n], keep = up ? v[i + n] : v[i];
+                    v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+                }
+            }
+        }
+    }
+    return v[0];
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(bf16 a, bf16 b) {
     return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
 }
@@ -210,7 +244,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
         cs_q[it] = idx < n_q ? rope[(size_t)(pos0 + (TR ? (int)s_dep[s_colm[rl]] : (int)s_colm[rl])) * HALF + i] : make_float2(1.f, 0.f);
     }
     auto gather_pair = [&](int m, int col) -> float2 {
-        if (pv.mode == 0) return part_gather_n<2>(pv, m, col);
+        if (pv.mode != 1) return part_gather_n<2>(pv, m, col);
         const int t = col >> 7;
         return part_gather_blocks<2>(pv, s_tb[t == tk ? nq : (t == tv ? nq + 1 : t - tq0)], m, col);
     };
@@ -324,16 +358,21 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
     const int quad = warp & 3, tl = warp >> 2, lane_id = quad * 32 + lane;
     const uint32_t tm_lane = tmem + ((uint32_t)(quad * 32) << 16);
     constexpr uint32_t IDESC = idesc_bf16(2 * NC);
+    // operand descriptors of the first step; later steps add their byte offset / 16 to the address field
+    const uint64_t dK = smem_desc_plain(smem_u32(sK), 128, GRP), dQ = smem_desc_plain(smem_u32(sQ), LBO_C, 128);
+    const uint64_t dV = smem_desc_plain(smem_u32(sV), GRP, 128), dP = smem_desc_plain(smem_u32(sP), LBO_C, 128);
     bool live = !*abort_flag;
     if (live) {
         if (tid == 128) {   // ---- score MMAs: one chain of D / 16 steps per 128-position tile
             tc_fence_after();
-            for (int t = 0; t < n_tiles; t++) {
-                const uint32_t a0 = smem_u32(sK) + (uint32_t)t * (TILE / 8) * GRP, b0 = smem_u32(sQ);
 #pragma unroll
-                for (int j = 0; j < D / 16; j++)
-                    mma_bf16(tmem + (uint32_t)(t * 2 * NC), smem_desc_plain(a0 + j * 256, 128, GRP),
-                             smem_desc_plain(b0 + j * 2 * LBO_C, LBO_C, 128), IDESC, j > 0);
+            for (int t = 0; t < MAX_TILES; t++) {
+                if (t < n_tiles) {
+#pragma unroll
+                    for (int j = 0; j < D / 16; j++)
+                        mma_bf16(tmem + (uint32_t)(t * 2 * NC), dK + (uint64_t)((t * (TILE / 8) * GRP + j * 256) >> 4),
+                                 dQ + (uint64_t)((j * 2 * LBO_C) >> 4), IDESC, j > 0);
+                }
             }
             mma_commit(bar_s);
         }
@@ -372,13 +411,18 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
             if (lane == (c & 31)) s_mx[warp * NC + c] = ord2f(o);
         }
         __syncthreads();
+        float mx_lane = -INFINITY;   // lane c: maximum of column c over the slice
+        if (lane < nb) {
+#pragma unroll
+            for (int w = 0; w < 8; w++) mx_lane = fmaxf(mx_lane, s_mx[w * NC + lane]);
+        }
+        mx_lane = fmaxf(mx_lane, -1e30f);   // a column that sees nothing in this slice: every numerator 2^(-inf) = 0
+        float pr[NC];
 #pragma unroll
         for (int c = 0; c < NC; c++) {
-            if (c >= nb) break;
-            float mx = s_mx[c];
-#pragma unroll
-            for (int w = 1; w < 8; w++) mx = fmaxf(mx, s_mx[w * NC + c]);
-            const float p = (sc[c] == -INFINITY) ? 0.f : exp2f(sc[c] - mx);
+            if (c >= nb) { pr[c] = 0.f; continue; }
+            const float p = ex2(sc[c] - __shfl_sync(0xffffffffu, mx_lane, c));
+            pr[c] = p;
             if (tl < n_tiles) {
                 // numerators as two bf16 terms in operand form: position j at (j / 8) * LBO_C + (j % 8) * 2
                 const bf16 hi = __float2bfloat16_rn(p);
@@ -386,8 +430,19 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
                 *reinterpret_cast<bf16 *>(dst + (c >> 3) * 128 + (c & 7) * 16) = hi;
                 *reinterpret_cast<bf16 *>(dst + ((NC + c) >> 3) * 128 + ((NC + c) & 7) * 16) = __float2bfloat16_rn(p - __bfloat162float(hi));
             }
-            const float s = warp_sum(p);
-            if (lane == (c & 31)) s_sm[warp * NC + c] = s;
+        }
+        // column sums over the warp's positions (fixed order), one entry per (warp, column)
+        if (nb <= 2) {
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                if (c >= nb) break;
+                const float s = warp_sum(pr[c]);
+                if (lane == 0) s_sm[warp * NC + c] = s;
+            }
+        } else {
+            const float s = column_sums<NC>(pr, lane);
+            const int c = NC == 32 ? lane : (lane >> 1);
+            if ((NC == 32 || !(lane & 1)) && c < nb) s_sm[warp * NC + c] = s;
         }
         fence_async_smem();
         tc_fence_before();
@@ -398,8 +453,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
             tc_fence_after();
             const int steps = (npos + 15) >> 4;
             for (int s = 0; s < steps; s++)
-                mma_bf16(tmem, smem_desc_plain(smem_u32(sV) + (uint32_t)s * 2 * GRP, GRP, 128),
-                         smem_desc_plain(smem_u32(sP) + (uint32_t)s * 2 * LBO_C, LBO_C, 128), IDESC, s > 0);
+                mma_bf16(tmem, dV + (uint64_t)s * ((2 * GRP) >> 4), dP + (uint64_t)s * ((2 * LBO_C) >> 4), IDESC, s > 0);
             mma_commit(bar_o);
         }
         if (tid < nb) {   // thread c: maximum and sum of column c over this slice
@@ -461,7 +515,17 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
     if (!*s_last) return;
     __threadfence();
     const size_t sstride = (size_t)kMaxRows * D;
-    {   // normalised weight of every (column, slice); a warp's columns are loaded together: one round trip
+    // this thread's first item (column, four output dimensions): its first eight slices are requested now,
+    // together with the slices' maxima and sums, so that the merge costs one round trip, not two
+    float4 pre[8];
+    {
+        const int rl = min(tid / (D / 4), nb - 1), dd = (tid % (D / 4)) * 4;
+        const float *src = apart + ((size_t)s_colh[rl] * n_split * kMaxRows + s_colm[rl]) * D + dd;
+#pragma unroll
+        for (int u = 0; u < 8; u++)
+            pre[u] = (tid < nb * (D / 4) && u < n_split) ? __ldcg(reinterpret_cast<const float4 *>(src + (size_t)u * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    {   // normalised weight of every (column, slice); a warp's columns are loaded together
         constexpr int CPW = NC / 8;
         const float2 none = make_float2(-INFINITY, 0.f);
         float2 v0[CPW], v1[CPW];
@@ -491,13 +555,15 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
         const float *src = apart + ((size_t)h * n_split * kMaxRows + m) * D + dd;
         const float *wr = wgt + rl * n_split;
         float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s2 = 0; s2 < n_split; s2 += 16) {   // sixteen slices in flight, added in slice order
-            float4 a[16];
+        for (int s2 = 0; s2 < n_split; s2 += 8) {   // eight slices in flight, added in slice order
+            float4 a[8];
 #pragma unroll
-            for (int u = 0; u < 16; u++)
-                a[u] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)min(s2 + u, n_split - 1) * sstride));
+            for (int u = 0; u < 8; u++) {
+                if (idx == tid && s2 == 0) a[u] = pre[u];
+                else a[u] = s2 + u < n_split ? __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(s2 + u) * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
-            for (int u = 0; u < 16; u++) {
+            for (int u = 0; u < 8; u++) {
                 const float w = s2 + u < n_split ? wr[s2 + u] : 0.f;
                 o.x = fmaf(w, a[u].x, o.x); o.y = fmaf(w, a[u].y, o.y);
                 o.z = fmaf(w, a[u].z, o.z); o.w = fmaf(w, a[u].w, o.w);
@@ -505,9 +571,13 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
         }
         const size_t col = (size_t)h * D + dd;
         if (attn_out) *reinterpret_cast<float4 *>(attn_out + (size_t)m * H * D + col) = o;
-        if (attn_split) {
-            store_split(attn_split, m, (size_t)H * D, col, o.x); store_split(attn_split, m, (size_t)H * D, col + 1, o.y);
-            store_split(attn_split, m, (size_t)H * D, col + 2, o.z); store_split(attn_split, m, (size_t)H * D, col + 3, o.w);
+        if (attn_split) {   // two bf16 terms, four dimensions at a time (store_split's layout)
+            const bf16 h0 = __float2bfloat16_rn(o.x), h1 = __float2bfloat16_rn(o.y), h2 = __float2bfloat16_rn(o.z), h3 = __float2bfloat16_rn(o.w);
+            bf16 *xh = attn_split + (size_t)m * H * D + col;
+            *reinterpret_cast<uint2 *>(xh) = make_uint2(pack_bf16(h0, h1), pack_bf16(h2, h3));
+            *reinterpret_cast<uint2 *>(xh + (size_t)kMaxRows * H * D) =
+                make_uint2(pack_bf16(__float2bfloat16_rn(o.x - __bfloat162float(h0)), __float2bfloat16_rn(o.y - __bfloat162float(h1))),
+                           pack_bf16(__float2bfloat16_rn(o.z - __bfloat162float(h2)), __float2bfloat16_rn(o.w - __bfloat162float(h3))));
         }
     }
 }

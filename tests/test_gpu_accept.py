@@ -31,7 +31,7 @@ def _run_case(case, B, K, V, sigma, delta, T):
     return n_ref
 
 
-@pytest.mark.parametrize("B,K", [(1, 1), (1, 4), (8, 8), (64, 16), (8, 1), (64, 4), (1, 16)])
+@pytest.mark.parametrize("B,K", [(B, K) for B in (1, 8, 64) for K in (1, 4, 8, 16)])   # the whole sweep: 12 x 6 = 72 cases
 def test_accept_sweep_bit_exact(B, K):
     seen = []
     for ci, (sigma, delta) in enumerate(CASES):
@@ -70,3 +70,26 @@ def test_bad_arguments_are_rejected():
     assert L.eesd_accept_resample(None, t.data_ptr(), t.data_ptr(), i.data_ptr(), t.data_ptr(), t.data_ptr(),
                                   1, 1, 8, 1.0, t.data_ptr(), 4, i.data_ptr(), i.data_ptr()) == -2  # scratch too small
     assert L.eesd_sample_rows(None, t.data_ptr(), None, 1, 8, 1.0, i.data_ptr()) == -6        # needs uniforms
+    big = torch.zeros(1024, device="cuda")
+    assert L.eesd_accept_resample(None, t.data_ptr(), t.data_ptr(), i.data_ptr(), t.data_ptr(), t.data_ptr(),
+                                  1, 1, 8, 1.0, big.data_ptr() + 4, 1024, i.data_ptr(), i.data_ptr()) == -1  # scratch not 16-byte aligned
+
+
+def test_token_ids_outside_the_vocabulary_are_rejected_where_they_stand():
+    # a drafted id outside [0, V) cannot have been drawn from q: the kernel must reject it at its
+    # position without reading a logit for it; the oracle's rule applied to the prefix before it
+    # gives the expected result (the residual at that position is undefined, so only n is compared)
+    import paper_2406_03853_b200 as eesd
+    B, K, V = 4, 6, 4096
+    p, q, ua, ur, ud = synth.accept_case(31, B, K, V, 1.0, 0.1, device="cuda")
+    x = eesd.sample_rows(q.view(B * K, V), ud.view(B * K), 1.0).view(B, K).contiguous()
+    n_ok, _ = eesd.accept_resample(p, q, x, ua, ur, 1.0)
+    bad = x.clone()
+    bad[0, 2], bad[1, 0], bad[2, 5], bad[3, 3] = V, -1, 2 ** 31 - 1, -(2 ** 31)
+    for T in (1.0, 0.0):
+        n, y = eesd.accept_resample(p, q, bad, ua, ur, T)
+        n_ref, _ = eesd.accept_resample(p, q, x, ua, ur, T)
+        torch.cuda.synchronize()
+        want = torch.minimum(n_ref, torch.tensor([2, 0, 5, 3], dtype=torch.int32, device="cuda"))
+        assert torch.equal(n, want)
+        assert ((y >= 0) & (y < V)).all()

@@ -61,8 +61,13 @@ def _slice_parity(spec, n_layers, n_prompt, M, max_ctx=96):
     m64.target_rows(prompt[:-1], 0, want_logits=False)
     hid64, lg64 = m64.target_rows(rows, n_prompt - 1, want_hidden=True)
     e64 = np.abs(got - hid64).max()
-    print(f"{spec.name}: vs fp64-cache oracle: hidden {e64:.3e}, logits {np.abs(eng.logits(0, M).cpu().numpy() - lg64).max():.3e}")
+    storage_h, storage_l = np.abs(hid - hid64).max(), np.abs(lg - lg64).max()
+    print(f"{spec.name}: vs fp64-cache oracle: hidden {e64:.3e}, logits {np.abs(eng.logits(0, M).cpu().numpy() - lg64).max():.3e}; "
+          f"storage alone (bf16-cache oracle against fp64-cache oracle): hidden {storage_h:.3e}, logits {storage_l:.3e}")
     assert e64 < 2.0 ** -7 * np.abs(hid64).max()
+    # the tolerance is stated against the oracle with the SAME storage format: against an unrounded cache
+    # the engine may be as far as the storage rounding itself moves the oracle, plus that tolerance
+    assert e64 <= storage_h + TOL
     # the draft model on the same slice: one draft step against the oracle's draft row
     eng.prefill(prompt)
     eng.draft(1)
@@ -80,3 +85,86 @@ def test_13b_shape_slice_hidden_and_logits():
 
 def test_70b_shape_slice_hidden_and_logits():
     _slice_parity(synth.LLAMA2_70B, n_layers=1, n_prompt=19, M=6)
+
+
+def _long_cache_parity(spec, n_layers, n_prompt, Ms, seed=synth.SEED + 3):
+    """A real prefill of n_prompt tokens in the engine (wide prompt passes) and in the oracle, then verify
+    passes of M rows for every M in Ms against ONE oracle pass of max(Ms) rows (rows are causal, so
+    its first M rows are the oracle's answer for a pass of M rows), hidden states per layer and
+    logits; then one draft step.  This is the cache length and the launch configuration the
+    benchmark's verify-pass leg times: every attention slice of the pass is in play."""
+    max_ctx = n_prompt + 32
+    eng = engine_from_spec(spec, n_layers=n_layers, max_ctx=max_ctx, k_cap=15)
+    m = oracle_from_spec(spec, max_ctx=max_ctx, n_layers=n_layers, device="cuda")
+    prompt = synth.prompt_tokens(seed, n_prompt, spec.vocab).numpy()
+    m.target_rows(prompt[:-1], 0, want_logits=False)
+    eng.prefill(prompt)
+    cap = eng.capture_hidden(True)
+    Mx = max(Ms)
+    rows = np.concatenate([prompt[-1:], synth.prompt_tokens(seed + 1, Mx - 1, spec.vocab).numpy()]).astype(np.int32)
+    hid, lg = m.target_rows(rows, n_prompt - 1, want_hidden=True)
+    for M in Ms:
+        eng.verify_only(rows[:M])
+        torch.cuda.synchronize()
+        got = cap[:n_layers + 1, :M].cpu().numpy()
+        err_h = np.abs(got - hid[:, :M]).max(axis=(1, 2))
+        err_l = np.abs(eng.logits(0, M).cpu().numpy() - lg[:M]).max()
+        print(f"{spec.name}, cache {n_prompt - 1}, {M} rows: hidden max-abs err per layer {err_h}, logits {err_l:.3e}")
+        assert err_h.max() < TOL and err_l < TOL
+    eng.capture_hidden(False)
+    eng.prefill(prompt)
+    eng.draft(1)
+    torch.cuda.synchronize()
+    err_q = np.abs(eng.logits(1, 1).cpu().numpy()[0] - m.draft_row(int(prompt[-1]), n_prompt - 1)).max()
+    print(f"{spec.name}, cache {n_prompt - 1}: draft logits err {err_q:.3e}")
+    assert err_q < TOL
+    eng.close()
+
+
+def test_13b_shape_1024_token_cache_verify_passes():
+    _long_cache_parity(synth.LLAMA2_13B, n_layers=2, n_prompt=1024, Ms=(1, 6, 16))
+
+
+def test_70b_shape_1024_token_cache_verify_passes():
+    # 8 query heads per KV head: 6 rows are 48 (head, row) pairs, two column batches per KV head
+    _long_cache_parity(synth.LLAMA2_70B, n_layers=1, n_prompt=1024, Ms=(1, 6))
+
+
+def test_13b_shape_error_growth_over_eight_layers():
+    # A deeper slice (8 layers, the first five undamped, short cache): the per-layer distance to the
+    # oracle on record.  Logits stay within the stated 2e-2.  Hidden states of magnitude 30 do not, and
+    # cannot for any fp32 implementation: with keys and values STORED as bf16 the function itself jumps
+    # where a value sits on a rounding boundary.  The size of those jumps is measured here on the
+    # oracle alone (its own output when the embedding moves by about one fp32 unit in the last place),
+    # and the engine is asked to stay within the stated tolerance plus three times that distance.
+    import oracle
+    spec, L, n_prompt, M = synth.LLAMA2_13B, 8, 21, 6
+    eng = engine_from_spec(spec, n_layers=L, max_ctx=64, k_cap=15)
+    layers = [{k: v.cpu() for k, v in synth.layer_weights(spec, l, synth.SEED, "cuda").items()} for l in range(L)]
+    ex = {k: v.cpu() for k, v in synth.exit_layer_weights(spec, synth.SEED, "cuda").items()}
+    emb, head = synth.embedding(spec, synth.SEED, "cuda").cpu().float(), synth.lm_head(spec, synth.SEED, "cuda").cpu()
+    s = spec.with_(n_layers=L, n_early=min(spec.n_early, L))
+    prompt = synth.prompt_tokens(synth.SEED + 9, n_prompt, spec.vocab).numpy()
+    rows = np.concatenate([prompt[-1:], synth.prompt_tokens(77, M - 1, spec.vocab).numpy()]).astype(np.int32)
+    noise = 1 + (torch.rand(emb.shape, generator=torch.Generator().manual_seed(1)) - 0.5) * 2.0 ** -22
+    runs = []
+    for e in (emb, emb * noise):
+        m = oracle.model_from_weights(s, layers, ex, e, head, max_ctx=64, kv_bf16=True)
+        m.target_rows(prompt[:-1], 0, want_logits=False)
+        runs.append(m.target_rows(rows, n_prompt - 1, want_hidden=True))
+    (hid, lg), (hid_n, lg_n) = runs
+    jump_h, jump_l = np.abs(hid - hid_n).max(axis=(1, 2)), np.abs(lg - lg_n).max()
+    eng.prefill(prompt)
+    cap = eng.capture_hidden(True)
+    eng.verify_only(rows)
+    torch.cuda.synchronize()
+    err_h = np.abs(cap[:L + 1, :M].cpu().numpy() - hid).max(axis=(1, 2))
+    err_l = np.abs(eng.logits(0, M).cpu().numpy() - lg).max()
+    np.set_printoptions(linewidth=250)
+    print(f"13b, {L} layers: engine vs oracle, hidden max-abs after the embedding and after each layer {np.array2string(err_h, precision=4)}; "
+          f"oracle vs oracle with the embedding moved by one fp32 ulp {np.array2string(jump_h, precision=4)}; "
+          f"|hidden| {np.array2string(np.abs(hid).max(axis=(1, 2)), precision=1)}; logits: engine {err_l:.3e}, oracle jump {jump_l:.3e}")
+    assert err_l < TOL
+    assert (err_h < TOL + 3 * jump_h).all()
+    assert err_h[:3].max() < TOL          # the shallow part holds the plain tolerance
+    eng.close()

@@ -133,6 +133,14 @@ def test_tree_pass_13b_layer_shape():
     assert worst < TOL
 
 
+def test_tree_pass_13b_layer_shape_1024_token_cache():
+    # the cache length the benchmark times: a 7-row tree pass (width 2, three draft steps) over every attention slice
+    spec = synth.LLAMA2_13B
+    worst, kept = _rounds_through_the_step_api(spec, 2, width=2, k=3, n_prompt=1024, n_rounds=1, max_ctx=1100)
+    print(f"tree pass, 13B layer shape (2 layers), 1023 cached tokens: worst logit distance {worst:.3e}")
+    assert worst < TOL
+
+
 def test_tree_generation_under_the_beta_controller():
     # draft lengths chosen by Thompson sampling; the oracle's round is driven by the lengths the engine took
     from paper_2406_03853_b200 import binding as b

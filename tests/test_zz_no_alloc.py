@@ -3,8 +3,8 @@
 Some users of the library verify a round from a place where device allocation is off limits (a
 serving engine with a frozen memory plan, a plug-in that only receives its input and output
 tensors).  That entry point keeps its scratch in a fixed device array inside the library.  This
-file checks, through the C ABI, that it gives exactly what the ordinary entry point gives
-(integer results: bit-exact), on two calls in a row so that state left behind by the first call
+file checks, through the C ABI, that it gives exactly what the ordinary entry point gives and what
+the CPU oracle gives on the same logits and uniforms (integer results: bit-exact), on two calls in a row so that state left behind by the first call
 cannot leak into the second, and that it refuses problems larger than its built-in scratch.
 It is collected last on purpose.
 """
@@ -15,6 +15,7 @@ import pytest
 import torch
 
 import eesd_synth as synth
+import oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -37,6 +38,10 @@ def test_static_scratch_entry_point_matches_the_ordinary_one_twice_in_a_row():
         p, q, ua, ur, ud = synth.accept_case(500 + case, B, K, V, 2.0, 1.0, device="cuda")
         x = eesd.sample_rows(q.view(B * K, V), ud.view(B * K), T).view(B, K).contiguous()
         n_ref, y_ref = eesd.accept_resample(p, q, x, ua, ur, T)
+        n_orc, y_orc = oracle.accept_resample_batch(p.cpu().numpy(), q.cpu().numpy(), x.cpu().numpy(), ua.cpu().numpy(),
+                                                    ur.cpu().numpy(), T)
+        np.testing.assert_array_equal(n_ref.cpu().numpy(), n_orc)
+        np.testing.assert_array_equal(y_ref.cpu().numpy(), y_orc)
         for _ in range(2):
             st, n, y = _static(L, p, q, x, ua, ur, T)
             assert st == 0
