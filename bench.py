@@ -42,6 +42,20 @@ WORKLOADS = {
 }
 
 
+def profiled_traffic(spec_name):
+    """DRAM bytes (read + write) of one launch of the dominant kernel from the ncu capture summarised
+    under profiles/ (a line `dram_bytes_per_launch <shape> <bytes>`); None when no capture of this shape
+    is on file."""
+    path = os.path.join(ROOT, "profiles", "gemm_tc_gate_up_dram_traffic.txt")
+    if not os.path.exists(path):
+        return None, None
+    for line in open(path):
+        f = line.split()
+        if len(f) >= 3 and f[0] == "dram_bytes_per_launch" and f[1] == spec_name:
+            return int(f[2]), "profiles/gemm_tc_gate_up_dram_traffic.txt"
+    return None, None
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -202,37 +216,84 @@ def time_accept_kernel(device, batches=(1, 8, 64), ks=(4, 16), vocab=32000, reps
     return out
 
 
-def oracle_sample(spec, mean_k, mean_emit, budget_s=12.0):
-    """CPU oracle on a bounded slice: one decoder layer of this shape on (mean_k + 1) rows and
-    on 1 row against a 512-token cache, repeated until about `budget_s` seconds of CPU work
-    have been timed; the medians are scaled to a whole round (all layers, heads by parameter
-    count).  Returns (tokens/s, seconds timed, rows, repetitions)."""
-    import oracle
-    L1 = spec.with_(n_layers=1, n_early=1, vocab=64)
-    lw = {k: v for k, v in synth.layer_weights(spec, 0).items()}
-    emb = np.zeros((64, spec.d_model), np.float32)
-    m = oracle.model_from_weights(L1, [lw], lw, emb, emb, max_ctx=640)
-    rows = max(2, int(round(mean_k)) + 1)
+# The round both CPU legs (cpu_baseline of the default run, --impl reference) are scaled to: K drafted
+# tokens and EMIT emitted tokens per round, the rounded means of the default workload under Beta-TS
+# (mean K 2.5, 2.2 tokens per round).  Fixed so that both legs describe the same work.
+ORACLE_ROUND_K, ORACLE_ROUND_EMIT = 3, 2.2
+
+
+def _omp_threads(n=None):
+    """Sets (n given) or reads the OpenMP thread count of the process the oracle runs in."""
+    import ctypes
+    try:
+        gomp = ctypes.CDLL("libgomp.so.1")
+    except OSError:
+        return os.cpu_count() or 1
+    if n is not None:
+        gomp.omp_set_num_threads(int(n))
+    return int(gomp.omp_get_max_threads())
+
+
+_SLICES = {}
+
+
+def _oracle_slice(spec):
+    """The oracle's model for the timed slice (built once per process): one layer, the real head."""
+    if spec.name not in _SLICES:
+        import oracle
+        L1 = spec.with_(n_layers=1, n_early=1)
+        lw = {k: v for k, v in synth.layer_weights(spec, 0).items()}
+        emb = np.zeros((spec.vocab, spec.d_model), np.float32)
+        _SLICES[spec.name] = oracle.model_from_weights(L1, [lw], lw, emb, synth.lm_head(spec), max_ctx=640)
+    return _SLICES[spec.name]
+
+
+def oracle_sample(spec, budget_s=12.0):
+    """CPU oracle on a bounded slice of the workload: ONE decoder layer of this shape and the real
+    vocabulary head (full vocabulary), on ORACLE_ROUND_K + 1 rows (a verify pass) and on 1 row (a draft
+    step) against a 512-token cache, repeated until about `budget_s` seconds of CPU work have been
+    timed with all OpenMP threads, then once more single-threaded.  The medians are scaled to a whole
+    round by the layer counts (all layers + head for the verify pass; early layers + exit layer + exit
+    head per draft step).  Returns a dict with tokens/s (all threads and one thread) and what was timed."""
+    m = _oracle_slice(spec)
+    rows = ORACLE_ROUND_K + 1
     x = np.asarray(synth.normal_f32(1, 1, rows * spec.d_model).view(rows, spec.d_model), np.float64)
     m.layer_fwd(0, 0, x[:1], 512)   # touch the weights once, untimed
-    t_rows, t_one, spent, reps = [], [], 0.0, 0
-    while spent < budget_s and reps < 200:
+    m.head(x[:1])
+
+    def one():
         t0 = time.time()
         m.layer_fwd(0, 0, x, 512)
         t1 = time.time()
         m.layer_fwd(0, 0, x[:1], 512)
         t2 = time.time()
-        t_rows.append(t1 - t0)
-        t_one.append(t2 - t1)
-        spent += t2 - t0
-        reps += 1
-    t_layer_rows, t_layer_1 = statistics.median(t_rows), statistics.median(t_one)
-    head_rows = spec.vocab * spec.d_model / spec.layer_params  # head cost in units of one layer-row
-    per_row = t_layer_rows / rows
-    t_verify = spec.n_layers * t_layer_rows + rows * head_rows * per_row
-    t_draft = (rows - 1) * ((spec.n_early + 1) * t_layer_1 + head_rows * t_layer_1)
-    tok_s = mean_emit / (t_verify + t_draft)
-    return tok_s, spent, rows, reps
+        m.head(x)
+        t3 = time.time()
+        m.head(x[:1])
+        t4 = time.time()
+        return t1 - t0, t2 - t1, t3 - t2, t4 - t3
+
+    def tokens_per_s(t):
+        t_layer_rows, t_layer_1, t_head_rows, t_head_1 = t
+        t_verify = spec.n_layers * t_layer_rows + t_head_rows
+        t_draft = ORACLE_ROUND_K * ((spec.n_early + 1) * t_layer_1 + t_head_1)
+        return ORACLE_ROUND_EMIT / (t_verify + t_draft)
+
+    threads = _omp_threads()
+    samples, spent = [], 0.0
+    while spent < budget_s and len(samples) < 200:
+        samples.append(one())
+        spent += sum(samples[-1])
+    med = tuple(statistics.median(c) for c in zip(*samples))
+    _omp_threads(1)
+    single = one()
+    _omp_threads(threads)
+    return {"tokens_per_s": tokens_per_s(med), "tokens_per_s_one_thread": tokens_per_s(single), "threads": threads,
+            "seconds_timed": spent + sum(single), "repetitions": len(samples), "rows": rows,
+            "sample": (f"one {spec.name}-shaped decoder layer and the {spec.vocab}-entry vocabulary head on {rows} rows and on 1 row "
+                       f"against a 512-token cache ({len(samples)} repetitions with {threads} OpenMP threads, medians; once with 1 thread), "
+                       f"scaled by layer count to a round of K={ORACLE_ROUND_K} drafts emitting {ORACLE_ROUND_EMIT} tokens "
+                       f"({spec.n_layers} layers + head per verify pass, {spec.n_early + 1} layers + head per draft step); extrapolated over layers")}
 
 
 def profile_pass(args, device):
@@ -355,6 +416,57 @@ def run_sweep(args, device):
             torch.cuda.empty_cache()
 
 
+def leg_70b(device, peaks, steps=2, new_tokens=64):
+    """The LLaMA-2-70B-shaped configuration (80 layers, 64 / 8 heads, about 140 GB of bf16 weights, early
+    exit after 10 layers, damping 0.2, 1024-token prompt) on the same GPU: verify passes of 1, 6 and 16
+    rows against a 1024-token cache, and a short decode (`steps` prompts x `new_tokens` tokens, Beta-TS)."""
+    from paper_2406_03853_b200 import binding as b
+    from paper_2406_03853_b200 import report
+    t0 = time.time()
+    torch.cuda.empty_cache()
+    eng, spec, n_prompt, _ = build_engine("70b-eesd", 0.0, b.CTRL_BETA_TS, device)
+    t_build = time.time() - t0
+    kv_len = WORKLOADS["70b-eesd"][4]
+    bv, bd = pass_bytes(spec, kv_len)
+    out = {"weights_gb": round(eng.sizes.weights_bytes / 1e9, 1), "verify_pass": {"kv_len": kv_len, "bytes": bv}, "draft_step_bytes": bd}
+    for M in (1, 6, 16):
+        ms = time_verify_pass(eng, spec, kv_len, M)
+        out["verify_pass"][f"M{M}"] = {"ms": round(ms, 4), "gbs": round(bv / (ms * 1e-3) / 1e9, 1),
+                                       "frac_of_measured_copy": round(bv / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                                       "frac_of_8tbs": round(bv / (ms * 1e-3) / 1e9 / 8000.0, 4)}
+    u = {k: v.numpy() for k, v in synth.generate_uniforms(eng.cfg.max_ctx, 1 << 20).items()}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ms_dec, ms_e2e, tot = 0.0, 0.0, {"drafted": 0, "accepted": 0, "emitted": 0, "rounds": 0, "ms_draft": 0.0}
+    for i in range(steps):
+        prompt = synth.prompt_tokens(synth.SEED + i, n_prompt, spec.vocab).numpy()
+        eng.prefill(prompt)
+        torch.cuda.synchronize()
+        e0.record()
+        _, _, st = eng.decode(new_tokens, uniforms=u)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_dec += e0.elapsed_time(e1)
+        for k in tot:
+            tot[k] += st.as_dict()[k]
+        e0.record()
+        eng.generate(prompt, new_tokens, uniforms=u)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_e2e += e0.elapsed_time(e1)
+    q = report.run_quality(tot["drafted"], tot["accepted"], tot["emitted"])
+    out["decode"] = {"tokens_per_s": round(steps * new_tokens / (ms_dec * 1e-3), 2), "prompts": steps, "new_tokens": new_tokens,
+                     "prompt_tokens": n_prompt, "e2e_tokens_per_s": round(steps * new_tokens / (ms_e2e * 1e-3), 2),
+                     "autoregressive_tokens_per_s": round(1e3 / out["verify_pass"]["M1"]["ms"], 2),
+                     "ms_per_draft_step": round(tot["ms_draft"] / max(1, tot["drafted"]), 4),
+                     "mean_k": round(tot["drafted"] / max(1, tot["rounds"]), 3), "v_d": round(q["v_d"], 4), "r_d": round(q["r_d"], 4),
+                     "early_layers": spec.n_early, "damp_alpha": spec.damp}
+    eng.close()
+    del eng
+    torch.cuda.empty_cache()
+    out["seconds"] = {"build": round(t_build, 1), "whole_leg": round(time.time() - t0, 1)}
+    return out
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle as it stands, timed on the host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -364,23 +476,20 @@ def run_reference(args):
     oracle.build()
     spec_name, n_prompt, max_new, damp, _ = WORKLOADS[args.workload]
     spec = synth.SPECS[spec_name].with_(damp=damp)
-    vals, ms = [], []
+    vals, ms, last = [], [], None
     for i in range(args.warmup + args.steps):
         t0 = time.time()
-        tok_s, _, rows, _ = oracle_sample(spec, 5.0, 3.0)
+        last = oracle_sample(spec, budget_s=8.0)
         if i >= args.warmup:
-            vals.append(tok_s)
+            vals.append(last["tokens_per_s"])
             ms.append((time.time() - t0) * 1e3)
     v = statistics.median(vals)
-    sample = (f"one {spec.name}-shaped decoder layer on {rows} rows + on 1 row against a 512-token cache, scaled to "
-              f"a round of K=5 drafts emitting 3 tokens ({spec.n_layers} layers verify, {spec.n_early + 1} layers per "
-              f"draft step, vocabulary heads by parameter count); extrapolated, not a full-model run")
-    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
     print(json.dumps({"impl": "reference", "metric": "eesd_decode_tokens_per_s", "value": v, "unit": "tokens/s",
                       "n_gpus": 0, "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.median(ms),
                       "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-                      "config": {"workload": args.workload},
-                      "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+                      "config": {"workload": args.workload, "round_model": {"k": ORACLE_ROUND_K, "tokens_per_round": ORACLE_ROUND_EMIT}},
+                      "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": last["threads"], "kind": "oracle",
+                                       "value_one_thread": last["tokens_per_s_one_thread"], "sample": last["sample"]},
                       "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
@@ -397,6 +506,8 @@ def main():
                          "0.2 medium (default), 0.5 low acceptance")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-tree", action="store_true", help="skip the tree-verification leg of the default run")
+    ap.add_argument("--no-70b", action="store_true",
+                    help="skip the LLaMA-2-70B-shaped leg of the default run (verify passes and a short decode; about a minute)")
     ap.add_argument("--profile-pass", type=int, default=0, metavar="M",
                     help="only run verify passes of M rows (and draft steps) inside a cudaProfilerStart/Stop "
                          "bracket, for ncu --profile-from-start off")
@@ -508,7 +619,9 @@ def main():
         vp[f"M{M}"] = {"ms": round(ms, 4), "ms_per_layer": round(ms / spec.n_layers, 5), "gbs": round(bv / (ms * 1e-3) / 1e9, 1),
                        "frac_of_measured_copy": round(bv / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
                        "frac_of_8tbs": round(bv / (ms * 1e-3) / 1e9 / 8000.0, 4)}
-    s0 = {k: sum(st[k] for st in stats) for k in ("drafted", "accepted", "emitted", "rounds", "ms_draft", "ms_verify")}
+    traffic, traffic_src = profiled_traffic(spec.name)
+    s0 = {k: sum(st[k] for st in stats) for k in ("drafted", "accepted", "emitted", "rounds", "ms_draft", "ms_verify", "ms_sampling",
+                                                  "ms_other", "ms_total")}
     qual = report.run_quality(s0["drafted"], s0["accepted"], s0["emitted"])
     v_d, r_d = qual["v_d"], qual["r_d"]
     # the paper's cost model (its appendix on the harmonic mean) with the measured draft-step and
@@ -533,10 +646,12 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "skinny projection (gate/up shape, M=%d)" % M_typ,
                      "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": round(achieved / peaks["hbm_gbs"], 4),
-                     # dram__bytes_read + dram__bytes_write of one gate/up launch at the 13B shape, from the ncu
-                     # capture summarised under profiles/ (null for other shapes: not captured)
-                     "traffic": 287024384 if (spec.name == "13b") else None,
+                     "frac_of_8tbs": round(achieved / 8000.0, 4),
+                     "note": "the denominator is a COPY rate (read + write); a read-only weight stream can exceed it, so a "
+                             "fraction above 1 is not headroom.  The figure the target is set on is verify_pass_frac_of_8tbs",
+                     "traffic": traffic, "traffic_source": traffic_src,
                      "bytes_per_launch": kbytes, "ms_per_launch": round(kms, 5)},
+        "verify_pass_frac_of_8tbs": {spec.name: {k: v["frac_of_8tbs"] for k, v in vp.items() if k in ("M1", "M6", "M16")}},
         "verify_pass": {"kv_len": kv_len, "bytes": bv, **vp},
         "draft_step_bytes": bd,
         "accept_kernel": time_accept_kernel(device),
@@ -545,18 +660,20 @@ def main():
                         "ms_per_draft_step": round(t_d, 4), "autoregressive_tokens_per_s": round(1e3 / t_t, 2),
                         "speedup_vs_autoregressive": round(value / world / (1e3 / t_t), 4),
                         "speedup_by_cost_model": None if model_speedup is None else round(model_speedup, 4),
+                        # the paper's time-breakdown buckets, per decoded sequence (decode loop only: no prompt pass)
                         "ms_draft": round(s0["ms_draft"] / args.steps, 3), "ms_verify": round(s0["ms_verify"] / args.steps, 3),
+                        "ms_sampling": round(s0["ms_sampling"] / args.steps, 3), "ms_other": round(s0["ms_other"] / args.steps, 3),
+                        "ms_wall": round(s0["ms_total"] / args.steps, 3),
                         "ms_prefill_e2e": round(st2.ms_prefill, 3)},
     }
     if not args.no_cpu_baseline and world == 1:
         import oracle
         oracle.build()
-        tok_s, secs, rows, reps = oracle_sample(spec, mean_k, mean_emit)
+        o = oracle_sample(spec)
         line["cpu_baseline"] = {
-            "value": round(tok_s, 5), "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle",
-            "sample": f"one {spec.name}-shaped decoder layer on {rows} rows and on 1 row against a 512-token cache "
-                      f"({reps} repetitions, {secs:.1f} s of CPU work, medians), scaled to a round of mean K={mean_k:.2f} emitting {mean_emit:.2f} "
-                      f"tokens; extrapolated"}
+            "value": round(o["tokens_per_s"], 5), "unit": "tokens/s", "cores": o["threads"], "kind": "oracle",
+            "value_one_thread": round(o["tokens_per_s_one_thread"], 5), "seconds_timed": round(o["seconds_timed"], 1),
+            "round_model": {"k": ORACLE_ROUND_K, "tokens_per_round": ORACLE_ROUND_EMIT}, "sample": o["sample"]}
     eng.close()
     del eng
     if world == 1 and greedy and args.controller == "beta" and not args.no_tree:
@@ -588,6 +705,10 @@ def main():
         # greedy decoding is lossless either way: both runs must have emitted the same tokens
         tv["same_tokens_as_chain"] = all((a == c).all() for a, c in zip(outs[2], outs[1]))
         line["tree_verification"] = tv
+    if world == 1 and greedy and args.controller == "beta" and not args.no_70b and args.workload == "13b-eesd":
+        line["shape_70b"] = leg_70b(device, peaks)
+        line["verify_pass_frac_of_8tbs"]["70b"] = {k: v["frac_of_8tbs"] for k, v in line["shape_70b"]["verify_pass"].items()
+                                                   if k.startswith("M")}
     print(json.dumps(line))
     if dist:
         dist.destroy_process_group()

@@ -156,14 +156,25 @@ typedef struct eesd_uniforms {
 
 typedef struct eesd_round { int32_t k, n_accept, next_token; } eesd_round;
 
-/* Counters of one eesd_generate call.  v_d = accepted / drafted and r_d = accepted / emitted
- * are the paper's acceptance rate and draft proportion (metrics paragraph of Sec. 4.1). */
+/* Counters of one eesd_generate / eesd_decode call.  v_d = accepted / drafted and r_d = accepted /
+ * emitted are the paper's acceptance rate and draft proportion (metrics paragraph of Sec. 4.1).
+ * Times follow the buckets of the paper's time-breakdown table (drafting, verification, sampling,
+ * others), with the prompt pass kept apart:
+ *   ms_prefill   device time of the prompt pass (CUDA events; 0 for eesd_decode)
+ *   ms_draft     device time of the draft steps (draft model + token choice)
+ *   ms_verify    device time of the verification passes, without their acceptance step
+ *   ms_sampling  the acceptance step (device: fused softmax / accept / resample kernel, or the tree
+ *                walk), the calibrated controller's predictor steps (device), and the controller's
+ *                draws on the host (host clock)
+ *   ms_other     what is left of ms_total: synchronisation gaps, copies, host bookkeeping
+ *   ms_total     wall time of the call on the host clock; the five above add up to it */
 typedef struct eesd_stats {
     int64_t rounds, drafted, accepted, emitted;
-    double ms_prefill, ms_draft, ms_verify, ms_total; /* device time, CUDA events               */
+    double ms_prefill, ms_draft, ms_verify, ms_total;
     int64_t kernel_launches;
     int64_t alpha, beta;                               /* posterior after the last round         */
     int64_t leaves_kept;                               /* tree verification: rounds that kept a leaf */
+    double ms_sampling, ms_other;
 } eesd_stats;
 
 typedef struct eesd_ctx eesd_ctx;

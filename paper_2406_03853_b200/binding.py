@@ -70,7 +70,7 @@ class Stats(C.Structure):
     _fields_ = [("rounds", C.c_int64), ("drafted", C.c_int64), ("accepted", C.c_int64), ("emitted", C.c_int64),
                 ("ms_prefill", C.c_double), ("ms_draft", C.c_double), ("ms_verify", C.c_double),
                 ("ms_total", C.c_double), ("kernel_launches", C.c_int64), ("alpha", C.c_int64), ("beta", C.c_int64),
-                ("leaves_kept", C.c_int64)]
+                ("leaves_kept", C.c_int64), ("ms_sampling", C.c_double), ("ms_other", C.c_double)]
 
     def as_dict(self) -> Dict:
         return {n: getattr(self, n) for n, _ in self._fields_}

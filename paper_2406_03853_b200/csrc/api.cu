@@ -4,6 +4,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <chrono>
 #include <new>
 #include <vector>
 
@@ -210,7 +211,7 @@ struct eesd_ctx {
     TreeRows tree_rows;
     int64_t leaves_kept;
     int32_t *h_result;  // pinned: [0] n_accept, [1] next token, [2] error word, [3] row of the kept leaf or -1, [8..23] draft tokens
-    cudaEvent_t ev[5];  // prefill start / end, draft start, verify start, round end
+    cudaEvent_t ev[7];  // prefill start / end, draft start, verify start, round end, start / end of an acceptance or predictor step
     char cuda_err[256];
 };
 
@@ -597,9 +598,11 @@ int verify_tree_impl(eesd_ctx *c) {
     st = run_target(c, c->ints + kRowTok, M, T - 1, true);
     c->tree_cur = nullptr;
     if (st) return st;
+    CU(c, cudaEventRecord(c->ev[5], c->stream));
     launch_sample_rows(c->stream, c->logits_p, nullptr, M, f.vocab, 0.f, c->ints + kTreeTop);
     launch_tree_walk(c->stream, c->ints + kTreeTop, c->ints + kRoundTok, c->ints + kLeafTok, K, W, c->ints + kResult);
     launch_kv_move(c->stream, f.dtype, kv_geom(c, 0), c->slot_bytes, f.n_layers + 1, T - 1, c->ints + kResult, c->err);
+    CU(c, cudaEventRecord(c->ev[6], c->stream));
     c->launches += 4;
     st = check_launch(c);
     if (st) return st;
@@ -618,8 +621,10 @@ int verify_impl(eesd_ctx *c, const float *d_u_acc, const float *d_u_res) {
     if (st) return st;
     st = run_target(c, c->ints + kRoundTok, K + 1, T - 1, true);
     if (st) return st;
+    CU(c, cudaEventRecord(c->ev[5], c->stream));
     launch_accept(c->stream, c->logits_p, c->logits_q, c->ints + kRoundTok + 1, d_u_acc, d_u_res, 1, K, f.vocab,
                   f.temperature, c->accept_scratch, c->ints + kResult, c->ints + kResult + 1, c->ints + kRoundTok);
+    CU(c, cudaEventRecord(c->ev[6], c->stream));
     c->launches++;
     if (cali_on(c)) save_target_state(c, c->x, 0, c->ints + kResult);   // the row that gave the next token
     st = check_launch(c);
@@ -826,7 +831,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->h_result = nullptr;
     for (auto &e : c->ev) e = nullptr;
     cudaError_t e = cudaHostAlloc((void **)&c->h_result, 256, cudaHostAllocDefault);
-    for (int i = 0; i < 5 && e == cudaSuccess; i++) e = cudaEventCreate(&c->ev[i]);
+    for (int i = 0; i < 7 && e == cudaSuccess; i++) e = cudaEventCreate(&c->ev[i]);
     if (e != cudaSuccess) {
         eesd_destroy(c);
         return EESD_ERR_CUDA;
@@ -922,9 +927,12 @@ int eesd_verify_accept(eesd_ctx *c, const float *u_accept, float u_resample, int
 
 // rounds of {draft, verify, accept, posterior update} from the current context until max_new
 // tokens exist (Algorithm 1, outer loop)
+typedef std::chrono::steady_clock host_clock;
+static double ms_since(host_clock::time_point t0) { return std::chrono::duration<double, std::milli>(host_clock::now() - t0).count(); }
+
 static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int n_schedule, const eesd_uniforms *u,
                        int32_t *out, eesd_stats *stats, eesd_round *trace, int trace_cap, int *n_rounds,
-                       int64_t launches0, float ms_prefill) {
+                       int64_t launches0, float ms_prefill, host_clock::time_point wall0) {
     const eesd_config &f = c->cfg;
     const bool greedy = f.temperature == 0.f;
     if (!greedy && (!u || !u->u_draft || !u->u_accept || !u->u_resample)) return EESD_ERR_RNG;
@@ -954,6 +962,7 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
         if (tree_on(c) && (f.max_ctx - T) / f.tree_width < cap) cap = (f.max_ctx - T) / f.tree_width;
         if (cap < 1) return EESD_ERR_CTX_FULL;
         int K;
+        const host_clock::time_point ctrl0 = host_clock::now();
         // TS with calibration needs the predictor's output after every draft step: such rounds
         // are drafted step by step, with a synchronisation per step (Algorithm 3)
         const bool stepwise = f.controller == EESD_CTRL_CALI_TS && !(k_schedule && rounds < n_schedule);
@@ -971,6 +980,8 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
         }
         if (K < 1) K = 1;
         if (K > cap) K = cap;
+        sacc.ms_sampling += ms_since(ctrl0);   // the controller's draws on the host
+        float ms_pred = 0.f;                   // device time of this round's predictor steps (calibrated controller)
         CU(c, cudaEventRecord(c->ev[2], c->stream));
         if (!stepwise) {
             st = draft_impl(c, K, greedy ? nullptr : d_ud + T, 1);
@@ -980,12 +991,19 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
                 st = draft_impl(c, 1, greedy ? nullptr : d_ud + T + K, 1);
                 if (st) return st;
                 if (++K >= cap) break;
+                CU(c, cudaEventRecord(c->ev[5], c->stream));
                 st = run_cali_predict(c, K);
                 if (st) return st;
                 float *h_theta = (float *)(c->h_result + 32);
                 CU(c, cudaMemcpyAsync(h_theta, c->theta_dev, 4, cudaMemcpyDeviceToHost, c->stream));
+                CU(c, cudaEventRecord(c->ev[6], c->stream));
                 CU(c, cudaStreamSynchronize(c->stream));
+                float ms_one = 0.f;
+                cudaEventElapsedTime(&ms_one, c->ev[5], c->ev[6]);
+                ms_pred += ms_one;
+                const host_clock::time_point draw0 = host_clock::now();
                 const int chi = cali_continue(c, *h_theta, u, &cursor);
+                sacc.ms_sampling += ms_since(draw0);
                 if (chi < 0) return chi;
                 if (!chi) break;
             }
@@ -1000,11 +1018,13 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
         int32_t y;
         st = finish_round(c, drafts, &a, &y);
         if (st) return st;
-        float ms_d = 0.f, ms_v = 0.f;
+        float ms_d = 0.f, ms_v = 0.f, ms_a = 0.f;
         cudaEventElapsedTime(&ms_d, c->ev[2], c->ev[3]);
         cudaEventElapsedTime(&ms_v, c->ev[3], c->ev[4]);
-        sacc.ms_draft += ms_d;
-        sacc.ms_verify += ms_v;
+        cudaEventElapsedTime(&ms_a, c->ev[5], c->ev[6]);   // the acceptance step inside the verification
+        sacc.ms_draft += ms_d - ms_pred;
+        sacc.ms_verify += ms_v - ms_a;
+        sacc.ms_sampling += ms_a + ms_pred;
         sacc.drafted += K;
         sacc.accepted += a < max_new - t ? a : max_new - t;
         ts_update(c, a + 1, K);
@@ -1018,7 +1038,8 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
         sacc.rounds = rounds;
         sacc.emitted = max_new;
         sacc.ms_prefill = ms_prefill;
-        sacc.ms_total = sacc.ms_prefill + sacc.ms_draft + sacc.ms_verify;
+        sacc.ms_total = ms_since(wall0);
+        sacc.ms_other = sacc.ms_total - (sacc.ms_prefill + sacc.ms_draft + sacc.ms_verify + sacc.ms_sampling);
         sacc.kernel_launches = c->launches - launches0;
         sacc.alpha = c->alpha;
         sacc.beta = c->beta;
@@ -1032,7 +1053,7 @@ int eesd_decode(eesd_ctx *c, int max_new, const int32_t *k_schedule, int n_sched
                 int32_t *out, eesd_stats *stats, eesd_round *trace, int trace_cap, int *n_rounds) {
     if (!c || !out || max_new < 1) return EESD_ERR_BADARG;
     if (!c->prefilled || c->round_k != 0) return EESD_ERR_STATE;
-    return decode_impl(c, max_new, k_schedule, n_schedule, u, out, stats, trace, trace_cap, n_rounds, c->launches, 0.f);
+    return decode_impl(c, max_new, k_schedule, n_schedule, u, out, stats, trace, trace_cap, n_rounds, c->launches, 0.f, host_clock::now());
 }
 
 int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new, const int32_t *k_schedule,
@@ -1041,6 +1062,7 @@ int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new,
     if (!c || !out || max_new < 1) return EESD_ERR_BADARG;
     if (n_prompt + max_new + 1 > c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
     const int64_t launches0 = c->launches;
+    const host_clock::time_point wall0 = host_clock::now();
     CU(c, cudaEventRecord(c->ev[0], c->stream));
     int st = prefill_impl(c, prompt, n_prompt);
     if (st) return st;
@@ -1048,7 +1070,7 @@ int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new,
     CU(c, cudaEventSynchronize(c->ev[1]));
     float ms_p = 0.f;
     cudaEventElapsedTime(&ms_p, c->ev[0], c->ev[1]);
-    return decode_impl(c, max_new, k_schedule, n_schedule, u, out, stats, trace, trace_cap, n_rounds, launches0, ms_p);
+    return decode_impl(c, max_new, k_schedule, n_schedule, u, out, stats, trace, trace_cap, n_rounds, launches0, ms_p, wall0);
 }
 
 // -ln u of a controller uniform; a zero uniform counts as half the grid step, 2^-25

@@ -45,3 +45,14 @@ def aggregate_replicas(local_ms: float, local_units: float, dist=None, device: O
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(u, op=dist.ReduceOp.SUM)
     return float(t.item()), float(u.item()), float(u.item()) / (float(t.item()) / 1e3)
+
+
+def time_breakdown(stats: Dict[str, float]) -> Dict[str, float]:
+    """The four buckets of the paper's time-breakdown table (drafting, verification, sampling,
+    others) from an eesd_stats record, in seconds, plus the prompt pass and their sum, which is
+    the call's wall time (the table's rows add up to the per-instance inference time)."""
+    b = {"drafting": stats["ms_draft"] / 1e3, "verification": stats["ms_verify"] / 1e3,
+         "sampling": stats["ms_sampling"] / 1e3, "others": stats["ms_other"] / 1e3,
+         "prefill": stats["ms_prefill"] / 1e3}
+    b["total"] = sum(b.values())
+    return b

@@ -112,3 +112,42 @@ def test_reproducible_and_independent_of_page_size():
         eng.close()
     for o in outs[1:]:
         np.testing.assert_array_equal(o, outs[0])
+
+
+@pytest.mark.parametrize("mode", ["beta", "cali", "tree"])
+def test_time_buckets_add_up_to_the_wall_time_of_the_call(mode):
+    # the paper's time-breakdown table: drafting + verification + sampling + others = inference time.
+    # The library's buckets (plus the prompt pass) must add up to the wall time it reports, and that
+    # wall time must be the one a caller measures around the call.
+    import time
+    from paper_2406_03853_b200 import binding as b
+    from paper_2406_03853_b200 import report
+    spec = synth.TINY
+    kw = dict(max_ctx=256, k_cap=7)
+    if mode == "beta":
+        kw.update(controller=b.CTRL_BETA_TS, temperature=1.0)
+    elif mode == "cali":
+        kw.update(controller=b.CTRL_CALI_TS, cali_sigma_m=0.3, cali_sigma_s=0.5, cali_theta0=0.5)
+    else:
+        kw.update(tree_width=2, fixed_k=3)
+    eng = engine_from_spec(spec, **kw)
+    if mode == "cali":
+        cw = synth.cali_weights(spec, synth.SEED, "cuda")
+        g = eng.global_views()
+        g["cali_w"].copy_(cw["w"])
+        g["cali_wp"].copy_(cw["wp"])
+    prompt = synth.prompt_tokens(synth.SEED + 2, 40, spec.vocab).numpy()
+    u = {k: v.numpy() for k, v in synth.generate_uniforms(256, 200000).items()}
+    eng.generate(prompt, 32, uniforms=u)       # warm-up
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    _, _, st = eng.generate(prompt, 160, uniforms=u)
+    wall = (time.perf_counter() - t0) * 1e3
+    s = st.as_dict()
+    parts = report.time_breakdown(s)
+    assert abs(parts["total"] * 1e3 - s["ms_total"]) < 1e-6 * s["ms_total"]
+    assert s["ms_total"] <= wall and wall - s["ms_total"] < 0.01 * wall + 0.5     # the binding adds well under 1 % + 0.5 ms
+    for k in ("ms_draft", "ms_verify", "ms_sampling", "ms_other", "ms_prefill"):
+        assert s[k] > 0.0, k
+    assert s["ms_sampling"] < s["ms_verify"] + s["ms_draft"]
+    eng.close()

@@ -75,3 +75,17 @@ def test_replica_aggregation_two_gloo_ranks():
     for _, ms, units, rate in res:
         assert ms == 200.0 and units == 512.0 and rate == pytest.approx(512.0 / 0.2)  # slowest rank sets the time
     assert report.aggregate_replicas(50.0, 10.0) == (50.0, 10.0, 200.0)
+
+
+def test_time_breakdown_has_the_papers_four_buckets_and_adds_up():
+    # the same bookkeeping as the time-breakdown table: its four buckets add up to the inference time
+    from paper_2406_03853_b200 import report
+    for line in open(os.path.join(GOLD, "time_breakdown_table8.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = line.split()
+        d, v, s, o, total = (float(x) for x in f[2:7])
+        b = report.time_breakdown({"ms_draft": d * 1e3, "ms_verify": v * 1e3, "ms_sampling": s * 1e3, "ms_other": o * 1e3,
+                                   "ms_prefill": 0.0})
+        assert set(b) == {"drafting", "verification", "sampling", "others", "prefill", "total"}
+        assert abs(b["total"] - total) < 0.006          # the table prints three decimals, the total two
