@@ -190,9 +190,11 @@ def lm_head(spec: ModelSpec, seed: int = SEED, device="cpu") -> torch.Tensor:
     return weight_tensor(seed, TID_LM_HEAD, spec.vocab, spec.d_model, 1.0, _torch_dtype(spec), device)
 
 
-def exit_layer_weights(spec: ModelSpec, seed: int = SEED, device="cpu") -> Dict[str, torch.Tensor]:
-    """The early-exit layer: a copy of the last target layer."""
-    return layer_weights(spec, spec.n_layers - 1, seed, device)
+def exit_layer_weights(spec: ModelSpec, seed: int = SEED, device="cpu", index: int = 0, count: int = 1) -> Dict[str, torch.Tensor]:
+    """The early-exit layer: a copy of the last target layer.  With `count` exit layers (the paper's
+    experiment on their number) exit layer `index` is a copy of target layer L - count + index: the
+    last `count` target layers in their order."""
+    return layer_weights(spec, spec.n_layers - count + index, seed, device)
 
 
 def accept_case(case: int, batch: int, k: int, vocab: int, sigma: float, delta: float,

@@ -28,7 +28,7 @@ def build(force: bool = False) -> str:
 
 class _Cfg(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("d", "H", "Hkv", "D", "F", "V", "L", "N", "max_ctx")] + \
-               [("eps", C.c_double), ("theta", C.c_double), ("kv_bf16", C.c_int)]
+               [("eps", C.c_double), ("theta", C.c_double), ("kv_bf16", C.c_int), ("E", C.c_int)]
 
 
 class _GenCfg(C.Structure):
@@ -211,18 +211,21 @@ class OracleModel:
     """The target + draft model over fp32 copies of the given weights.
 
     layers: list of L dicts with g_attn, wqkv, wo, g_ffn, wgu ([2F, d], gate rows first), wd;
-    exit_layer: one such dict.  Weights may be torch tensors of any float dtype: their values
-    are widened to fp32 unchanged.
+    exit_layer: one such dict, or a list of them (a draft model with several early-exit layers,
+    stacked in that order).  Weights may be torch tensors of any float dtype: their values are
+    widened to fp32 unchanged.
     """
 
     def __init__(self, *, d, H, Hkv, D, F, V, N, max_ctx, layers: Sequence[Dict], exit_layer: Dict,
                  embed, g_final, lm_head, g_exit, exit_head, eps=1e-5, theta=10000.0, kv_bf16=False):
         self.L = len(layers)
-        self.cfg = _Cfg(d, H, Hkv, D, F, V, self.L, N, max_ctx, eps, theta, int(kv_bf16))
+        exit_layers = list(exit_layer) if isinstance(exit_layer, (list, tuple)) else [exit_layer]
+        self.E = len(exit_layers)
+        self.cfg = _Cfg(d, H, Hkv, D, F, V, self.L, N, max_ctx, eps, theta, int(kv_bf16), self.E)
         self.d, self.V, self.F, self.N, self.max_ctx = d, V, F, N, max_ctx
         self._keep = []
         self.h = C.c_void_p(lib().orc_model_new(C.byref(self.cfg)))
-        for i, lw in enumerate(list(layers) + [exit_layer]):
+        for i, lw in enumerate(list(layers) + exit_layers):
             wgu = _f32(lw["wgu"])
             arrs = [_f32(lw["g_attn"]), _f32(lw["wqkv"]), _f32(lw["wo"]), _f32(lw["g_ffn"]),
                     np.ascontiguousarray(wgu[:F]), np.ascontiguousarray(wgu[F:]), _f32(lw["wd"])]

@@ -32,6 +32,9 @@ typedef struct {
     double eps, theta;
     int kv_bf16; /* 1: cached keys/values are stored rounded to bfloat16 (the storage format of
                     the bf16 configurations); arithmetic on them stays fp64 */
+    int E;       /* early-exit layers of the draft model (the experiment on the number of exit layers;
+                    Eq. 1 has one): a stack of E decoder layers on H^N, each with its own weights and
+                    cache slot; 0 reads as 1 */
 } orc_cfg;
 
 typedef struct {
@@ -41,16 +44,17 @@ typedef struct {
 typedef struct {
     orc_cfg c;
     const float *embed, *g_final, *lm_head, *g_exit, *exit_head;
-    orc_layer *layers; /* L target layers; index L is the early-exit layer */
-    double *kc, *vc;   /* [(L+1)][max_ctx][Hkv*D] rotated keys / values */
+    orc_layer *layers; /* L target layers; indices L .. L+E-1 are the early-exit layers */
+    double *kc, *vc;   /* [(L+E)][max_ctx][Hkv*D] rotated keys / values */
 } orc_model;
 
 /* ------------------------------------------------------------------ model plumbing */
 orc_model *orc_model_new(const orc_cfg *c) {
     orc_model *m = (orc_model *)calloc(1, sizeof(orc_model));
     m->c = *c;
-    m->layers = (orc_layer *)calloc((size_t)c->L + 1, sizeof(orc_layer));
-    size_t n = (size_t)(c->L + 1) * c->max_ctx * c->Hkv * c->D;
+    if (m->c.E < 1) m->c.E = 1;
+    m->layers = (orc_layer *)calloc((size_t)c->L + m->c.E, sizeof(orc_layer));
+    size_t n = (size_t)(c->L + m->c.E) * c->max_ctx * c->Hkv * c->D;
     m->kc = (double *)calloc(n, sizeof(double));
     m->vc = (double *)calloc(n, sizeof(double));
     return m;
@@ -212,9 +216,12 @@ void orc_head(const orc_model *m, const double *x, int M, const float *g, const 
 }
 
 /* Target model on M rows (tokens at positions pos0..): all L layers, KV rows written for
- * every layer, and the exit layer's k,v written for the same positions from H^N (they depend
- * on nothing else).  hidden (optional) receives the residual stream after the embedding and
- * after every layer: [(L+1)][M][d].  logits (optional) [M][V]. */
+ * every layer, and the exit layers' k,v written for the same positions: those of the first exit
+ * layer depend on H^N only; with E > 1 exit layers, those of exit layer e depend on the output of
+ * exit layer e-1, so exit layers 1..E-1 run in full on a copy of H^N (the target's own residual
+ * stream is not touched) and the last one contributes its key / value projection only.  hidden
+ * (optional) receives the residual stream after the embedding and after every target layer:
+ * [(L+1)][M][d].  logits (optional) [M][V]. */
 void orc_target_rows(orc_model *m, const int32_t *tok, int M, int pos0, double *hidden, float *logits) {
     const orc_cfg *c = &m->c;
     size_t md = (size_t)M * c->d;
@@ -224,20 +231,26 @@ void orc_target_rows(orc_model *m, const int32_t *tok, int M, int pos0, double *
     for (int l = 0; l < c->L; l++) {
         orc_layer_fwd(m, l, l, x, M, pos0);
         if (hidden) memcpy(hidden + (size_t)(l + 1) * md, x, sizeof(double) * md);
-        if (l == c->N - 1) project_qkv(m, &m->layers[c->L], c->L, x, M, pos0, NULL);
+        if (l == c->N - 1) {
+            double *xe = (double *)malloc(sizeof(double) * md);
+            memcpy(xe, x, sizeof(double) * md);
+            for (int e = 0; e < c->E - 1; e++) orc_layer_fwd(m, c->L + e, c->L + e, xe, M, pos0);
+            project_qkv(m, &m->layers[c->L + c->E - 1], c->L + c->E - 1, xe, M, pos0, NULL);
+            free(xe);
+        }
     }
     if (logits) orc_head(m, x, M, m->g_final, m->lm_head, logits);
     free(x);
 }
 
 /* Draft model (Eq. 1) on ONE row: first N layers (sharing the target's KV cache), the
- * early-exit layer with its own weights and KV slot, RMSNorm, exit head W. */
+ * early-exit layer(s) with their own weights and KV slots, RMSNorm, exit head W. */
 void orc_draft_row(orc_model *m, int32_t tok, int pos, float *logits, double *hidden_exit /* [d] or NULL */) {
     const orc_cfg *c = &m->c;
     double *x = (double *)malloc(sizeof(double) * c->d);
     orc_embed(m, &tok, 1, x);
     for (int l = 0; l < c->N; l++) orc_layer_fwd(m, l, l, x, 1, pos);
-    orc_layer_fwd(m, c->L, c->L, x, 1, pos);
+    for (int e = 0; e < c->E; e++) orc_layer_fwd(m, c->L + e, c->L + e, x, 1, pos);
     if (hidden_exit) memcpy(hidden_exit, x, sizeof(double) * c->d);
     orc_head(m, x, 1, m->g_exit, m->exit_head, logits);
     free(x);

@@ -5,12 +5,12 @@ import eesd_synth as synth
 import oracle
 
 
-def oracle_from_spec(spec, max_ctx=256, n_layers=None, device="cpu", seed=synth.SEED, kv_bf16=None):
+def oracle_from_spec(spec, max_ctx=256, n_layers=None, device="cpu", seed=synth.SEED, kv_bf16=None, n_exit=1):
     """Oracle model with the synthetic weights of `spec` (optionally only the first n_layers;
-    the exit layer is then still the copy of the spec's last layer)."""
+    the exit layers are then still the copies of the spec's last layers)."""
     L = spec.n_layers if n_layers is None else n_layers
     layers = [{k: v.cpu() for k, v in synth.layer_weights(spec, l, seed, device).items()} for l in range(L)]
-    ex = {k: v.cpu() for k, v in synth.exit_layer_weights(spec, seed, device).items()}
+    ex = [{k: v.cpu() for k, v in synth.exit_layer_weights(spec, seed, device, e, n_exit).items()} for e in range(n_exit)]
     emb = synth.embedding(spec, seed, device).cpu()
     head = synth.lm_head(spec, seed, device).cpu()
     s = spec.with_(n_layers=L, n_early=min(spec.n_early, L))

@@ -124,3 +124,57 @@ def test_controller_posterior_in_generation_matches_trace():
         aa, bb = oracle.ts_update(aa, bb, n_acc + 1, k, 0)
     assert (a, b) == (aa, bb)
     assert len({k for k, _, _ in trace}) > 1  # the controller really varies the draft length
+
+
+# ---------------------------------------------------------------- several early-exit layers
+def test_one_exit_layer_given_as_a_list_is_the_same_model_bit_for_bit():
+    spec = synth.TINY
+    prompt = synth.prompt_tokens(synth.SEED + 3, 20, spec.vocab).numpy()
+    a, b = oracle_from_spec(spec, 96), oracle_from_spec(spec, 96, n_exit=1)
+    out_a, tr_a, _ = a.generate(prompt, 24, fixed_k=4)
+    out_b, tr_b, _ = b.generate(prompt, 24, fixed_k=4)
+    np.testing.assert_array_equal(out_a, out_b)
+    assert tr_a == tr_b
+    np.testing.assert_array_equal(a.draft_row(5, 60), b.draft_row(5, 60))
+
+
+@pytest.mark.parametrize("n_exit", [2, 3])
+def test_draft_row_with_several_exit_layers_is_the_stack_of_layers_on_the_early_hidden_state(n_exit):
+    # Eq. 1 with a stack of exit layers: p = softmax(W^T RMSNorm(T^e_E(...T^e_1(H^N)))).  The cached
+    # draft row after a target pass over the prefix must equal the stack composed from the layer
+    # primitive on the WHOLE prefix (which also checks that the target pass left every exit layer's
+    # keys / values for the prefix: exit layer e sees the output of exit layer e - 1 there).
+    spec = synth.TINY
+    toks = synth.prompt_tokens(5, 9, spec.vocab).numpy()
+    m = oracle_from_spec(spec, 64, n_exit=n_exit)
+    m.target_rows(toks[:-1], 0, want_logits=False)
+    lg, hid = m.draft_row(toks[-1], 8, want_hidden=True)
+    m2 = oracle_from_spec(spec, 64, n_exit=n_exit)
+    x = m2.embed(toks)
+    for l in range(spec.n_early):
+        x = m2.layer_fwd(l, l, x, 0)
+    for e in range(n_exit):
+        x = m2.layer_fwd(spec.n_layers + e, spec.n_layers + e, x, 0)
+    np.testing.assert_allclose(hid, x[-1], atol=1e-12)
+    np.testing.assert_allclose(lg, m2.head(x[-1:], exit_head=True)[0], atol=1e-6)
+    # the exit layers are copies of the last target layers, in order; and a second exit layer changes the draft
+    for e in range(n_exit):
+        a, b = synth.exit_layer_weights(spec, index=e, count=n_exit), synth.layer_weights(spec, spec.n_layers - n_exit + e)
+        assert all((a[k] == b[k]).all() for k in a)
+    m1 = oracle_from_spec(spec, 64)
+    m1.target_rows(toks[:-1], 0, want_logits=False)
+    assert np.abs(m1.draft_row(toks[-1], 8) - lg).max() > 1e-4
+    # the target's own output does not depend on how many exit layers hang off layer N
+    _, t1 = m1.target_rows(toks, 0)
+    _, t2 = oracle_from_spec(spec, 64, n_exit=n_exit).target_rows(toks, 0)
+    np.testing.assert_array_equal(t1, t2)
+
+
+def test_greedy_eesd_with_two_exit_layers_still_equals_vanilla_autoregressive():
+    spec = synth.TINY
+    prompt = synth.prompt_tokens(synth.SEED, 32, spec.vocab).numpy()
+    ref = _autoregressive_greedy(oracle_from_spec(spec, 160), prompt, 32)
+    for kw in (dict(fixed_k=4), dict(k_schedule=[1, 7, 2, 10, 3, 5] * 6)):
+        out, trace, _ = oracle_from_spec(spec, 160, n_exit=2).generate(prompt, 32, **kw)
+        np.testing.assert_array_equal(out, ref)
+    assert sum(a for _, a, _ in trace) > 5
