@@ -108,7 +108,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None, cali=False, tree_width=0):
+def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None, cali=False, tree_width=0, n_exit=1):
     from paper_2406_03853_b200 import Engine
     from paper_2406_03853_b200 import binding as b
     spec_name, n_prompt, max_new, damp, _ = WORKLOADS[wl]
@@ -123,16 +123,17 @@ def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_
                         dtype=spec.dtype, tie_exit_head=spec.tie_exit_head, max_ctx=max_ctx,
                         k_cap=10 if tree_width < 2 else 15 // tree_width,
                         temperature=temperature, controller=b.CTRL_CALI_TS if cali else controller, fixed_k=5, page_tokens=16,
-                        tree_width=tree_width)
+                        tree_width=tree_width, n_exit_layers=n_exit)
     eng = Engine(cfg, device=device)
     # synthetic weights, generated on the device by the shared seeded generator
     for l in range(spec.n_layers):
         v = eng.layer_views(l)
         for k, t in synth.layer_weights(spec, l, synth.SEED, device).items():
             v[k].copy_(t)
-    v = eng.layer_views(spec.n_layers)
-    for k, t in synth.exit_layer_weights(spec, synth.SEED, device).items():
-        v[k].copy_(t)
+    for e in range(n_exit):
+        v = eng.layer_views(spec.n_layers + e)
+        for k, t in synth.exit_layer_weights(spec, synth.SEED, device, e, n_exit).items():
+            v[k].copy_(t)
     g = eng.global_views()
     g["embed"].copy_(synth.embedding(spec, synth.SEED, device))
     head = synth.lm_head(spec, synth.SEED, device)
@@ -407,6 +408,14 @@ def run_sweep(args, device):
             eng.close()
             del eng
             torch.cuda.empty_cache()
+    elif args.sweep == "exit":
+        # the paper's experiment on the number of early-exit layers: a deeper draft head accepts more and costs more
+        for E in (1, 2, 3):
+            eng, spec, _, _ = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha, n_exit=E)
+            measure(eng, spec, f"{E} exit layer(s)", None)
+            eng.close()
+            del eng
+            torch.cuda.empty_cache()
     else:
         for N in (1, 2, 3, 5, 8, 10):
             eng, spec, _, _ = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha, n_early=N)
@@ -513,8 +522,9 @@ def main():
                          "bracket, for ncu --profile-from-start off")
     ap.add_argument("--controller", choices=["beta", "cali"], default="beta",
                     help="draft-length controller: Beta-TS (default) or TS with calibration (random-init predictor)")
-    ap.add_argument("--sweep", choices=["k", "n", "tree"], default=None,
-                    help="method sweep instead of the benchmark line: fixed K = 1..10 against Beta-TS, or the exit depth N")
+    ap.add_argument("--sweep", choices=["k", "n", "tree", "exit"], default=None,
+                    help="method sweep instead of the benchmark line: fixed K = 1..10 against Beta-TS, the exit depth N, "
+                         "tree verification widths, or the number of early-exit layers")
     ap.add_argument("--profile-prefill", action="store_true",
                     help="only run one prompt pass inside a cudaProfilerStart/Stop region (for ncu)")
     ap.add_argument("--profile-tree", type=int, default=0, metavar="W",

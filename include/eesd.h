@@ -94,6 +94,12 @@ typedef struct eesd_config {
      * eesd_generate / eesd_decode want n_prompt + max_new + tree_width <= max_ctx (CTX_FULL
      * otherwise) and shorten the last rounds' drafts to what fits. */
     int32_t tree_width;
+    /* Early-exit layers of the draft model (the paper's experiment on the number of exit layers; its
+     * method and Eq. 1 use one).  0 or 1: one.  2..4: a stack of that many decoder layers on H^N, stored
+     * one after the other from eesd_layout.exit_layer on, each with its own cache slot; prefill and
+     * verification then also run all exit layers but the last on their rows (exit layer e needs the
+     * output of exit layer e - 1 to form its keys / values), so each costs that many more layers. */
+    int32_t n_exit_layers;
 } eesd_config;
 
 /* Byte offsets inside the weight buffer.  A decoder layer holds, in this order:
@@ -113,7 +119,7 @@ typedef struct eesd_layout {
     size_t off_g_attn, off_wqkv, off_wo, off_g_ffn, off_wgu, off_wd; /* within a layer          */
     size_t final_norm;   /* f32[d]                                                              */
     size_t lm_head;      /* [V][d]                                                              */
-    size_t exit_layer;   /* one decoder layer                                                   */
+    size_t exit_layer;   /* the early-exit layer(s): n_exit_layers decoder layers, layer_stride apart */
     size_t exit_norm;    /* f32[d], the RMSNorm before the exit head                            */
     size_t exit_head;    /* [V][d]; equals lm_head when tie_exit_head                           */
     size_t cali_w;       /* EESD_CTRL_CALI_TS only (else 0): W^1..W^10 of Eq. 5, [10][d][d]           */
@@ -124,14 +130,14 @@ typedef struct eesd_layout {
 
 typedef struct eesd_sizes {
     size_t weights_bytes;
-    size_t kv_page_bytes;   /* bytes of ONE page across all L+1 cache slots                     */
+    size_t kv_page_bytes;   /* bytes of ONE page across all L + n_exit_layers cache slots       */
     int64_t min_pages;      /* pages needed to hold max_ctx tokens                              */
     size_t workspace_bytes;
 } eesd_sizes;
 
 /* Caller-owned device memory.  kv_pool holds P = floor(kv_bytes / kv_page_bytes) pages laid
- * out [slot 0..L][page 0..P-1][K|V][H_kv] blocks of page_tokens * D elements; slot L is the
- * early-exit layer's cache.  The element order inside a block is an internal format (the library
+ * out [slot 0..L+E-1][page 0..P-1][K|V][H_kv] blocks of page_tokens * D elements; slots L.. are the
+ * caches of the E early-exit layers.  The element order inside a block is an internal format (the library
  * writes and reads the pool itself): for a bf16 cache both blocks are grids of 8 x 8 element
  * groups, [token/8][D/8][8][8], keys with a group's 8 tokens as rows, values with its 8 dimensions
  * as rows, which is the form the tensor cores take an operand in; for an fp32 cache keys are

@@ -37,7 +37,7 @@ class Config(C.Structure):
                 ("page_tokens", C.c_int32), ("max_ctx", C.c_int32), ("k_cap", C.c_int32), ("temperature", C.c_float),
                 ("controller", C.c_int32), ("fixed_k", C.c_int32), ("alpha0", C.c_int32), ("beta0", C.c_int32),
                 ("ts_update_rule", C.c_int32), ("cali_sigma_m", C.c_float), ("cali_sigma_s", C.c_float),
-                ("cali_theta0", C.c_float), ("tree_width", C.c_int32)]
+                ("cali_theta0", C.c_float), ("tree_width", C.c_int32), ("n_exit_layers", C.c_int32)]
 
 
 class Layout(C.Structure):
@@ -159,11 +159,11 @@ def _np_f32(a) -> np.ndarray:
 def make_config(*, d_model, n_heads, n_kv_heads, head_dim, ffn_dim, vocab, n_layers, n_early, dtype,
                 tie_exit_head=False, rms_eps=1e-5, rope_theta=10000.0, page_tokens=16, max_ctx=2048, k_cap=10,
                 temperature=0.0, controller=CTRL_FIXED_K, fixed_k=4, alpha0=1, beta0=1, ts_update_rule=0,
-                cali_sigma_m=0.2, cali_sigma_s=0.5, cali_theta0=0.5, tree_width=0) -> Config:
+                cali_sigma_m=0.2, cali_sigma_s=0.5, cali_theta0=0.5, tree_width=0, n_exit_layers=1) -> Config:
     dt = {"f32": F32, "bf16": BF16}.get(dtype, dtype)
     return Config(d_model, n_heads, n_kv_heads, head_dim, ffn_dim, vocab, n_layers, n_early, dt, int(tie_exit_head),
                   rms_eps, rope_theta, page_tokens, max_ctx, k_cap, temperature, controller, fixed_k, alpha0, beta0,
-                  ts_update_rule, cali_sigma_m, cali_sigma_s, cali_theta0, tree_width)
+                  ts_update_rule, cali_sigma_m, cali_sigma_s, cali_theta0, tree_width, n_exit_layers)
 
 
 class TiledMatrix:
@@ -244,9 +244,9 @@ class Engine:
         return TiledMatrix(self.weights[off:off + n].view(self.wdtype), shape)
 
     def layer_views(self, l: int) -> Dict[str, torch.Tensor]:
-        """Tensors aliasing target layer l (l == n_layers: the early-exit layer)."""
+        """Tensors aliasing target layer l (l >= n_layers: early-exit layer l - n_layers)."""
         c, lay = self.cfg, self.layout
-        base = lay.exit_layer if l == c.n_layers else lay.layer0 + l * lay.layer_stride
+        base = lay.exit_layer + (l - c.n_layers) * lay.layer_stride if l >= c.n_layers else lay.layer0 + l * lay.layer_stride
         qd, kvd = c.n_heads * c.head_dim, c.n_kv_heads * c.head_dim
         return {
             "g_attn": self._view(base + lay.off_g_attn, (c.d_model,), torch.float32),

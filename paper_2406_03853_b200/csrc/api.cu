@@ -50,6 +50,7 @@ int check_config(const eesd_config *c) {
     if (c->controller == EESD_CTRL_FIXED_K && c->fixed_k < 1) return EESD_ERR_BADARG;
     if (c->alpha0 < 1 || c->beta0 < 1) return EESD_ERR_BADARG;
     if (c->rms_eps < 0.f || c->rope_theta <= 1.f) return EESD_ERR_BADARG;
+    if (c->n_exit_layers < 0 || c->n_exit_layers > 4) return EESD_ERR_BADARG;
     if (c->tree_width < 0 || c->tree_width > 4) return EESD_ERR_BADARG;
     if (c->tree_width > 1) {   // tree verification: greedy only, 1 + k_cap * width rows in one pass
         if (c->temperature != 0.f || c->controller == EESD_CTRL_CALI_TS) return EESD_ERR_UNSUPPORTED;
@@ -59,8 +60,8 @@ int check_config(const eesd_config *c) {
 }
 
 struct Workspace {
-    size_t x, xn, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
-        accept, wx, wout, wout_floats, wxs[3], wssq, wtok, wapart, hT, xs_cali, theta, total;
+    size_t x, x_save, xn, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
+        accept, wx, wx_save, wout, wout_floats, wxs[3], wssq, wtok, wapart, hT, xs_cali, theta, total;
 };
 
 constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
@@ -70,6 +71,9 @@ constexpr int kMaxSm = 256;      // upper bound on the SM count the work splits 
 constexpr int kCtasPerSm = 2;    // projection CTAs per SM (gemm_tc.cu: two 4-stage rings fit one SM)
 constexpr int kPrefillRows = 512; // most prompt rows per pass of the wide (prompt) path
 constexpr uint32_t kDefaultWaitPolls = 1u << 25;   // polls before a wait inside a kernel gives up (about a second)
+
+// early-exit layers of the draft model (0 in the configuration reads as 1, the paper's setting)
+int n_exit(const eesd_config *c) { return c->n_exit_layers < 1 ? 1 : c->n_exit_layers; }
 
 bool tc_shapes_ok(const eesd_config *c) {
     const int qd = c->n_heads * c->head_dim, kvd = c->n_kv_heads * c->head_dim;
@@ -100,6 +104,7 @@ Workspace carve(const eesd_config *c) {
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     w.x = take(R * c->d_model * 4);
+    w.x_save = take(n_exit(c) > 1 ? R * c->d_model * 4 : 0);   // the target's rows while the exit layers before the last run on a copy
     w.xn = take(R * c->d_model * 4);
     w.attn = take(R * qd * 4);
     w.h = take(R * (size_t)c->ffn_dim * 4);
@@ -128,7 +133,7 @@ Workspace carve(const eesd_config *c) {
     w.hT = take((size_t)c->d_model * 4);
     w.xs_cali = take(2 * R * (size_t)c->d_model * 2);
     w.theta = take(16);
-    w.wx = w.wout = w.wout_floats = w.wssq = w.wtok = w.wapart = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
+    w.wx = w.wx_save = w.wout = w.wout_floats = w.wssq = w.wtok = w.wapart = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
     if (const size_t P = (size_t)prefill_rows(c)) {
         // prompt path: residual stream, one projection result, the three activation matrices as
         // two bf16 terms ([chunk of 16][hi | lo][16][K]), RMSNorm statistics, token ids
@@ -136,6 +141,7 @@ Workspace carve(const eesd_config *c) {
         if ((size_t)2 * c->ffn_dim > wideR) wideR = (size_t)2 * c->ffn_dim;
         if ((size_t)c->d_model > wideR) wideR = c->d_model;
         w.wx = take(P * c->d_model * 4);
+        w.wx_save = take(n_exit(c) > 1 ? P * c->d_model * 4 : 0);
         w.wout = take(P * wideR * 4);
         w.wout_floats = P * wideR;
         w.wxs[X_NORM] = take(2 * P * (size_t)c->d_model * 2);
@@ -165,7 +171,7 @@ struct eesd_ctx {
     cudaStream_t stream;
     size_t es;
     // device pointers
-    float *x, *xn, *attn, *h, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
+    float *x, *x_save, *xn, *attn, *h, *part, *apart, *logits_p, *logits_q, *u_dev, *u_stage, *capture;
     void *accept_scratch;
     void *xs[4];                 // bf16 hi/lo copies of xn, attn, h, and of H^(T) (calibration predictor)
     float *ssq;                  // RMSNorm partial sums of squares of the rows in xn / xs[X_NORM]
@@ -180,7 +186,7 @@ struct eesd_ctx {
     int64_t n_verify, n_trials;
     // prompt (wide) path: up to wide_rows prompt rows per pass
     int wide_rows;
-    float *wx, *wout, *wssq, *wapart;
+    float *wx, *wx_save, *wout, *wssq, *wapart;
     size_t wout_floats;          // room in wout
     void *wxs[3];
     int32_t *wtok;
@@ -193,7 +199,8 @@ struct eesd_ctx {
     float2 *rope;
     int32_t *page_table, *ints;
     int *err;
-    std::vector<LayerW> layers;  // L target layers + exit layer at index L
+    std::vector<LayerW> layers;  // L target layers, then the early-exit layers (indices L .. L + E - 1; cache slots likewise)
+    int E;                       // early-exit layers
     const void *embed, *lm_head, *exit_head;
     const float *g_final, *g_exit;
     // KV pool
@@ -350,12 +357,18 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
         const float *g_after = exit_here ? c->layers[L].g_attn : (l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
         run_layer(c, c->layers[l], l, M, pos0, g_after, cap_slot(c, l + 1));
         if (exit_here) {
-            // keys / values of the early-exit layer for these rows: they depend on H^N only
-            const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim;
-            const char *wkv = c->layers[L].wqkv + (size_t)qd * d * c->es;
+            // Keys / values of the early-exit layers for these rows.  Those of the first exit layer depend on H^N
+            // only; with several exit layers, layer e sees the output of layer e - 1, so all but the last run in
+            // full on these rows (the target's own rows are set aside meanwhile) and the last one contributes
+            // its key / value projection.
+            const int qd = f.n_heads * f.head_dim, kvd = f.n_kv_heads * f.head_dim, E = c->E;
+            if (E > 1) CU(c, cudaMemcpyAsync(c->x_save, c->x, (size_t)M * d * 4, cudaMemcpyDeviceToDevice, s));
+            for (int e = 0; e + 1 < E; e++) run_layer(c, c->layers[L + e], L + e, M, pos0, c->layers[L + e + 1].g_attn, nullptr);
+            const char *wkv = c->layers[L + E - 1].wqkv + (size_t)qd * d * c->es;
             PartView pv = run_proj(c, wkv, &c->m_exit_kv, P_EXIT_KV, X_NORM, M, 2 * kvd, d);
-            launch_qkv_post(s, f.dtype, pv, norm_scale(c), M, pos0, f.n_heads, kv_geom(c, L), c->rope, nullptr, true, c->err, 0,
+            launch_qkv_post(s, f.dtype, pv, norm_scale(c), M, pos0, f.n_heads, kv_geom(c, L + E - 1), c->rope, nullptr, true, c->err, 0,
                             c->tree_cur);
+            if (E > 1) CU(c, cudaMemcpyAsync(c->x, c->x_save, (size_t)M * d * 4, cudaMemcpyDeviceToDevice, s));
             const float *g_next = l + 1 < L ? c->layers[l + 1].g_attn : c->g_final;
             run_resid(c, nullptr, g_next, nullptr, M);
             c->launches += 1;
@@ -397,14 +410,11 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
     launch_embed(s, f.dtype, c->wtok, c->embed, c->wx, nullptr, Mtot, d, f.vocab, c->err);
     c->launches++;
     resid(nullptr, c->layers[0].g_attn);
-    for (int l = 0; l < L; l++) {
-        const LayerW &w = c->layers[l];
-        const bool exit_here = (l == f.n_early - 1);
-        const float *g_after = exit_here ? c->layers[L].g_attn : (l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
+    auto layer = [&](const LayerW &w, int slot, const float *g_after) {
         PartView pv = proj(w.m_qkv, X_NORM, qd + 2 * kvd, d);
         // keys / values of all rows into the cache first, then every 16-row chunk attends in one launch
-        launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, l), c->rope, nullptr, true, c->err, qd);
-        launch_attention_prompt(s, pv, rs, c->rope, kv_geom(c, l), c->wapart, c->tickets, c->wxs[X_ATTN], Mtot, p0, H, c->err, c->wait_polls);
+        launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, slot), c->rope, nullptr, true, c->err, qd);
+        launch_attention_prompt(s, pv, rs, c->rope, kv_geom(c, slot), c->wapart, c->tickets, c->wxs[X_ATTN], Mtot, p0, H, c->err, c->wait_polls);
         c->launches += 2;
         pv = proj(w.m_o, X_ATTN, d, qd);
         resid(&pv, w.g_ffn);
@@ -413,10 +423,18 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
         c->launches++;
         pv = proj(w.m_d, X_FFN, d, F);
         resid(&pv, g_after);
-        if (exit_here) {
-            pv = proj(c->m_exit_kv, X_NORM, 2 * kvd, d);
-            launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, L), c->rope, nullptr, true, c->err);
+    };
+    for (int l = 0; l < L; l++) {
+        const bool exit_here = (l == f.n_early - 1);
+        layer(c->layers[l], l, exit_here ? c->layers[L].g_attn : (l + 1 < L ? c->layers[l + 1].g_attn : c->g_final));
+        if (exit_here) {   // the exit layers' keys / values of the prompt rows (as in a verification pass)
+            const int E = c->E;
+            if (E > 1) CU(c, cudaMemcpyAsync(c->wx_save, c->wx, (size_t)Mtot * d * 4, cudaMemcpyDeviceToDevice, s));
+            for (int e = 0; e + 1 < E; e++) layer(c->layers[L + e], L + e, c->layers[L + e + 1].g_attn);
+            PartView pv = proj(c->m_exit_kv, X_NORM, 2 * kvd, d);
+            launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, L + E - 1), c->rope, nullptr, true, c->err);
             c->launches++;
+            if (E > 1) CU(c, cudaMemcpyAsync(c->wx, c->wx_save, (size_t)Mtot * d * 4, cudaMemcpyDeviceToDevice, s));
             resid(nullptr, l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
         }
     }
@@ -435,7 +453,9 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
         const float *g_after = l + 1 < N ? c->layers[l + 1].g_attn : c->layers[L].g_attn;
         run_layer(c, c->layers[l], l, 1, pos, g_after, cap_slot(c, l + 1));
     }
-    run_layer(c, c->layers[L], L, 1, pos, c->g_exit, cap_slot(c, L + 1));
+    for (int e = 0; e < c->E; e++)   // the early-exit layer(s), each on its own cache slot
+        run_layer(c, c->layers[L + e], L + e, 1, pos, e + 1 < c->E ? c->layers[L + e + 1].g_attn : c->g_exit,
+                  e + 1 < c->E ? nullptr : cap_slot(c, L + 1));
     float *lq = c->logits_q + (size_t)i * f.vocab;
     PartView pv = run_proj(c, c->exit_head, &c->m_exit_head, P_HEAD, X_NORM, 1, f.vocab, d);
     launch_reduce_partials(s, pv, norm_scale(c), lq, 1, f.vocab);
@@ -601,7 +621,7 @@ int verify_tree_impl(eesd_ctx *c) {
     CU(c, cudaEventRecord(c->ev[5], c->stream));
     launch_sample_rows(c->stream, c->logits_p, nullptr, M, f.vocab, 0.f, c->ints + kTreeTop);
     launch_tree_walk(c->stream, c->ints + kTreeTop, c->ints + kRoundTok, c->ints + kLeafTok, K, W, c->ints + kResult);
-    launch_kv_move(c->stream, f.dtype, kv_geom(c, 0), c->slot_bytes, f.n_layers + 1, T - 1, c->ints + kResult, c->err);
+    launch_kv_move(c->stream, f.dtype, kv_geom(c, 0), c->slot_bytes, f.n_layers + c->E, T - 1, c->ints + kResult, c->err);
     CU(c, cudaEventRecord(c->ev[6], c->stream));
     c->launches += 4;
     st = check_launch(c);
@@ -698,7 +718,7 @@ int eesd_weight_layout(const eesd_config *c, eesd_layout *out) {
     out->final_norm = take(d * 4);
     out->lm_head = take(V * d * es);
     out->exit_layer = o;
-    o += out->layer_stride;
+    o += out->layer_stride * (size_t)n_exit(c);
     out->exit_norm = take(d * 4);
     out->exit_head = c->tie_exit_head ? out->lm_head : take(V * d * es);
     out->cali_w = out->cali_wp = 0;
@@ -718,7 +738,7 @@ int eesd_required_bytes(const eesd_config *c, eesd_sizes *out) {
     if (!out) return EESD_ERR_BADARG;
     const size_t es = c->dtype == EESD_F32 ? 4 : 2;
     out->weights_bytes = lay.total_bytes;
-    out->kv_page_bytes = (size_t)(c->n_layers + 1) * 2 * c->n_kv_heads * c->page_tokens * c->head_dim * es;
+    out->kv_page_bytes = (size_t)(c->n_layers + n_exit(c)) * 2 * c->n_kv_heads * c->page_tokens * c->head_dim * es;
     out->min_pages = (c->max_ctx + c->page_tokens - 1) / c->page_tokens;
     out->workspace_bytes = carve(c).total;
     return EESD_OK;
@@ -751,7 +771,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->slot_bytes = (size_t)c->n_pages_total * 2 * cfg->n_kv_heads * cfg->page_tokens * cfg->head_dim * c->es;
     Workspace w = carve(cfg);
     char *ws = (char *)b->workspace;
-    c->x = (float *)(ws + w.x); c->xn = (float *)(ws + w.xn); c->attn = (float *)(ws + w.attn);
+    c->x = (float *)(ws + w.x); c->x_save = (float *)(ws + w.x_save); c->xn = (float *)(ws + w.xn); c->attn = (float *)(ws + w.attn);
     c->h = (float *)(ws + w.h); c->part = (float *)(ws + w.part); c->apart = (float *)(ws + w.apart);
     c->logits_p = (float *)(ws + w.logits_p); c->logits_q = (float *)(ws + w.logits_q);
     c->rope = (float2 *)(ws + w.rope); c->page_table = (int32_t *)(ws + w.page_table);
@@ -776,9 +796,11 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     }
     c->wide_rows = c->use_tc ? prefill_rows(cfg) : 0;
     const char *wb = (const char *)b->weights;
-    c->layers.resize(cfg->n_layers + 1);
-    for (int l = 0; l <= cfg->n_layers; l++) {
-        const char *base = wb + (l < cfg->n_layers ? lay.layer0 + (size_t)l * lay.layer_stride : lay.exit_layer);
+    c->E = n_exit(cfg);
+    c->layers.resize(cfg->n_layers + c->E);
+    for (int l = 0; l < cfg->n_layers + c->E; l++) {
+        const char *base = wb + (l < cfg->n_layers ? lay.layer0 + (size_t)l * lay.layer_stride
+                                                    : lay.exit_layer + (size_t)(l - cfg->n_layers) * lay.layer_stride);
         LayerW &lw = c->layers[l];
         lw.g_attn = (const float *)(base + lay.off_g_attn); lw.wqkv = base + lay.off_wqkv; lw.wo = base + lay.off_wo;
         lw.g_ffn = (const float *)(base + lay.off_g_ffn); lw.wgu = base + lay.off_wgu; lw.wd = base + lay.off_wd;
@@ -803,11 +825,11 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
             ok = ok && tc_make_map(&lw.m_gu, lw.wgu, 2 * F, d, 128, true);
             ok = ok && tc_make_map(&lw.m_d, lw.wd, d, F, 128, true);
         }
-        ok = ok && tc_make_map(&c->m_exit_kv, c->layers[cfg->n_layers].wqkv + (size_t)qd_ * d * 2, 2 * kvd_, d, 128, true);
+        ok = ok && tc_make_map(&c->m_exit_kv, c->layers[cfg->n_layers + c->E - 1].wqkv + (size_t)qd_ * d * 2, 2 * kvd_, d, 128, true);
         ok = ok && tc_make_map(&c->m_lm_head, c->lm_head, cfg->vocab, d, 128, true);
         ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128, true);
         if (c->wide_rows) {
-            c->wx = (float *)(ws + w.wx); c->wout = (float *)(ws + w.wout); c->wout_floats = w.wout_floats; c->wssq = (float *)(ws + w.wssq);
+            c->wx = (float *)(ws + w.wx); c->wx_save = (float *)(ws + w.wx_save); c->wout = (float *)(ws + w.wout); c->wout_floats = w.wout_floats; c->wssq = (float *)(ws + w.wssq);
             c->wtok = (int32_t *)(ws + w.wtok); c->wapart = (float *)(ws + w.wapart);
             const int ks[3] = {d, qd_, F};
             for (int i = 0; i < 3; i++) {
@@ -844,7 +866,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     // The tensor-core attention multiplies cached values past the end of a slice by weights that are
     // exactly zero; that is only harmless while every value the pool ever holds is finite, so the pool
     // starts as zeros (afterwards only this library writes it).
-    cudaMemsetAsync(b->kv_pool, 0, (size_t)(cfg->n_layers + 1) * c->slot_bytes, c->stream);
+    cudaMemsetAsync(b->kv_pool, 0, (size_t)(cfg->n_layers + c->E) * c->slot_bytes, c->stream);
     launch_rope_table(c->stream, c->rope, cfg->max_ctx, cfg->head_dim, cfg->rope_theta);
     c->launches++;
     st = check_launch(c);

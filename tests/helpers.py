@@ -42,9 +42,11 @@ def fill_engine(engine, spec, seed=synth.SEED):
         views = engine.layer_views(l)
         for k, v in synth.layer_weights(spec, l, seed, dev).items():
             views[k].copy_(v)
-    views = engine.layer_views(L)
-    for k, v in synth.exit_layer_weights(spec, seed, dev).items():
-        views[k].copy_(v)
+    E = max(1, engine.cfg.n_exit_layers)
+    for e in range(E):
+        views = engine.layer_views(L + e)
+        for k, v in synth.exit_layer_weights(spec, seed, dev, e, E).items():
+            views[k].copy_(v)
     g = engine.global_views()
     g["embed"].copy_(synth.embedding(spec, seed, dev))
     head = synth.lm_head(spec, seed, dev)

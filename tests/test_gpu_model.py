@@ -151,3 +151,38 @@ def test_time_buckets_add_up_to_the_wall_time_of_the_call(mode):
         assert s[k] > 0.0, k
     assert s["ms_sampling"] < s["ms_verify"] + s["ms_draft"]
     eng.close()
+
+
+@pytest.mark.parametrize("variant", ["fp32", "bf16"])
+def test_two_and_three_exit_layers_match_the_oracle(variant):
+    # the paper's experiment on the number of early-exit layers: the draft model is the first N layers plus a
+    # stack of exit layers, each with its own cache slot that prefill, verification and draft steps keep in step
+    base = synth.TINY if variant == "fp32" else synth.TINY.with_(dtype="bf16", ffn_dim=640)
+    for E in (2, 3):
+        eng = engine_from_spec(base, max_ctx=160, fixed_k=4, n_exit_layers=E)
+        m = oracle_from_spec(base, 160, n_exit=E)
+        prompt = synth.prompt_tokens(synth.SEED + E, 37, base.vocab).numpy()
+        if variant == "fp32":
+            out, trace, _ = eng.generate(prompt, 40, k_schedule=[4, 1, 7, 2, 5] * 8)
+            ref, rtrace, _ = m.generate(prompt, 40, k_schedule=[4, 1, 7, 2, 5] * 8)
+            np.testing.assert_array_equal(out, ref)
+            assert trace == rtrace and sum(a for _, a, _ in trace) > 5
+        else:
+            # prompt pass (wide kernels), a verify pass, then draft steps whose exit caches were filled by both
+            eng.prefill(prompt)
+            m.target_rows(prompt[:-1], 0, want_logits=False)
+            rows = np.concatenate([prompt[-1:], synth.prompt_tokens(5, 5, base.vocab).numpy()]).astype(np.int32)
+            eng.verify_only(rows)
+            torch.cuda.synchronize()
+            _, lg = m.target_rows(rows, 36)
+            assert np.abs(eng.logits(0, 6).cpu().numpy() - lg).max() < 2e-2
+            eng.prefill(prompt)
+            toks = eng.draft(3)
+            torch.cuda.synchronize()
+            ql = eng.logits(1, 3).cpu().numpy()
+            x = int(prompt[-1])
+            for i in range(3):
+                ref_q = m.draft_row(x, 36 + i)
+                assert np.abs(ql[i] - ref_q).max() < 2e-2
+                x = int(toks[i])
+        eng.close()
