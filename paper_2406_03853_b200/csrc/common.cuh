@@ -12,6 +12,7 @@ constexpr int kMaxRows = 16;  // most token rows per pass
 constexpr int kErrBadToken = 1;
 constexpr int kErrWaitTimeout = 2;
 constexpr int kErrBadPage = 4;
+constexpr int kErrPlan = 8;   // a launcher was asked for more attention slices than can be merged (the configuration check prevents it)
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }

@@ -200,8 +200,8 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
     const int col = col_off + blockIdx.x * D + 2 * i;
     pdl_trigger();
     pdl_wait();
-    const float rstd = row_rstd(rs, m);
     const float2 pr = part_gather_n<2>(pv, m, col);
+    const float rstd = row_rstd(rs, m);
     float a = pr.x * rstd, b = pr.y * rstd;
     const int pos = pos0 + m;   // where the row is stored; a tree row is rotated as its depth's position
     if (hh < H + kv.Hkv) {
@@ -732,15 +732,23 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
                       uint32_t wait_polls) {
     int pps;
     const int rows = (H / kv.Hkv) * M;
+    auto refuse = [&](int n_split) {   // more slices than the merge can take: report, launch nothing
+        if (n_split <= kMaxSlices && n_split <= max_splits) return false;
+        const int e = kErrPlan;
+        cudaMemcpyAsync(err, &e, sizeof(e), cudaMemcpyHostToDevice, s);
+        return true;
+    };
     if (dtype != 0) {   // bf16 cache: tensor-core kernel
         const int nc = attention_tc_columns(rows);
         const int n_split = attention_tc_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + nc - 1) / nc, n_sm, max_splits, &pps);
+        if (refuse(n_split)) return;
         launch_attention_tc(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, 0, tree,
                             wait_polls);
         return;
     }
     const int rb = rows <= 8 ? 8 : rows <= kRows16 ? 16 : 32;
     const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb, n_sm, max_splits, &pps);
+    if (refuse(n_split)) return;
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (kv.D == 64) attn_dispatch<64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls);
     else attn_dispatch<128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls);
@@ -761,6 +769,11 @@ void launch_attention_prompt(cudaStream_t s, const PartView &pv, const RowScale 
                              const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
                              int Mtot, int pos0, int H, int *err, uint32_t wait_polls) {
     const int pps = attention_tc_prompt_pps(kv.page_tokens), n_split = attention_prompt_splits(pos0 + Mtot, kv.page_tokens);
+    if (n_split > kMaxSlices) {
+        const int e = kErrPlan;
+        cudaMemcpyAsync(err, &e, sizeof(e), cudaMemcpyHostToDevice, s);
+        return;
+    }
     launch_attention_tc(s, pv, rs, rope, kv, apart, tickets, nullptr, attn_split, kMaxRows, pos0, H, pps, n_split, false, err, Mtot,
                         nullptr, wait_polls);
 }
@@ -771,8 +784,8 @@ __global__ void swiglu_kernel(PartView pv, RowScale rs, float *h, bf16 *hs, int 
     pdl_trigger();
     pdl_wait();
     if (i >= F) return;
+    const float4 g = part_gather4(pv, m, i), u = part_gather4(pv, m, F + i);   // requested first: the longest loads
     const float rstd = row_rstd(rs, m);
-    const float4 g = part_gather4(pv, m, i), u = part_gather4(pv, m, F + i);
     const float gg[4] = {g.x * rstd, g.y * rstd, g.z * rstd, g.w * rstd};
     const float uu[4] = {u.x * rstd, u.y * rstd, u.z * rstd, u.w * rstd};
 #pragma unroll
