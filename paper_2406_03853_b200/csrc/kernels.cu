@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                                                    float *__restrict__ apart, unsigned int *tickets,
                                                    float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
                                                    int M, int pos0, int H, int pps, int n_split, float scale, int *err,
-                                                   int Mtot, int nbat, size_t ml_off, TreeRows tr, uint32_t spin) {
+                                                   int nbat, size_t ml_off, TreeRows tr, uint32_t spin) {
     typedef float AT;
     typedef float2 KP;   // a pair of adjacent head dimensions of one key
     constexpr int HALF = D / 2;
@@ -300,22 +300,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
-    // Prompt mode (Mtot > 0): grid z also runs over the 16-row chunks of Mtot prompt rows whose
-    // keys and values are in the cache already; chunk c is an independent problem (rows
-    // pos0 + 16 c .., its own scratch, counters and slice count) and nothing is appended.
-    const int chunk = blockIdx.z / nbat, bz = blockIdx.z - chunk * nbat;
-    const bool cached_rows = Mtot > 0;
-    if (cached_rows) {
-        M = min(kMaxRows, Mtot - chunk * kMaxRows);
-        pos0 += chunk * kMaxRows;
-        n_split = ((pos0 + M + PT - 1) / PT + pps - 1) / pps;
-        if (sp >= n_split || group * M <= bz * RB) return;   // a short last chunk fills fewer slices and batches
-        pv.base += (size_t)chunk * kMaxRows * pv.R;
-        rs.ssq += (size_t)chunk * kMaxRows * kSsqBlocks;
-        if (attn_out) attn_out += (size_t)chunk * kMaxRows * H * D;
-        if (attn_split) attn_split += (size_t)chunk * 2 * kMaxRows * H * D;
-        apart += (size_t)chunk * (ml_off + (size_t)H * kMaxRows * kMaxSlices * 2);
-    }
+    const int bz = blockIdx.z;   // batch of (head, row) pairs
     // per-slice (maximum, sum) pairs live behind the outputs: [H][16][kMaxSlices]
     float2 *ml = reinterpret_cast<float2 *>(apart + ml_off);
     const int r0 = bz * RB;                  // first (head, row) pair of this block's batch
@@ -372,7 +357,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     constexpr int kNewPerThread = (NM * D + 255) / 256;
     constexpr int kQPerThread = RB * HALF / 256;
     const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
-    const int n_new = cached_rows ? 0 : max(0, p_last - p_first) * D;
+    const int n_new = max(0, p_last - p_first) * D;
     float2 cs_new[kNewPerThread], cs_q[kQPerThread];
 #pragma unroll
     for (int it = 0; it < kNewPerThread; it++) {
@@ -591,7 +576,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        unsigned int *tk = tickets + ((size_t)chunk * gridDim.x + kh) * nbat + bz;   // one counter per (chunk, KV head, batch)
+        unsigned int *tk = tickets + (size_t)kh * nbat + bz;   // one counter per (KV head, batch)
         const unsigned int prev = atomicAdd(tk, 1u);
         s_last = (prev == (unsigned int)n_split - 1);
         if (s_last) *tk = 0;
@@ -670,7 +655,7 @@ static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, 
         cudaFuncSetAttribute(attn_kernel<D, RB, NM, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
     (void)configured;
     launch_k(attn_kernel<D, RB, NM, TR>, dim3(kv.Hkv, n_split, nbat), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv,
-             apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, 0, nbat, ml_off, tr, wait_polls);
+             apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, nbat, ml_off, tr, wait_polls);
 }
 
 template <int D>
