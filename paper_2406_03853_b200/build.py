@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libeesd.so")
-SOURCES = ["api.cu", "kernels.cu", "accept.cu", "gemm_tc.cu", "attn_tc.cu"]
+SOURCES = ["api.cu", "kernels.cu", "accept.cu", "gemm_tc.cu", "attn_tc.cu", "attn_prompt.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-Xcompiler", "-fPIC"]
 
 

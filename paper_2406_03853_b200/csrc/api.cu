@@ -61,7 +61,7 @@ int check_config(const eesd_config *c) {
 
 struct Workspace {
     size_t x, x_save, xn, attn, h, xs[3], ssq, tickets, part, apart, logits_p, logits_q, rope, page_table, ints, u_dev, u_stage, err,
-        accept, wx, wx_save, wout, wout_floats, wxs[3], wssq, wtok, wapart, hT, xs_cali, theta, total;
+        accept, wx, wx_save, wout, wout_floats, wxs[3], wssq, wtok, hT, xs_cali, theta, total;
 };
 
 constexpr int kPartSplits = 1;   // room for K-split partial sums of one projection
@@ -89,9 +89,8 @@ int prefill_rows(const eesd_config *c) {
     return need < kPrefillRows ? need : kPrefillRows;
 }
 
-// arrival counters of the attention merge: one per (KV head, batch) in a decode pass, one per
-// (16-row chunk, KV head, batch) in a prompt pass
-size_t ticket_count(const eesd_config *c) { return 1024 + (size_t)(kPrefillRows / EESD_MAX_ROWS) * c->n_heads; }
+// arrival counters of the attention merge: one per (KV head, batch of (head, row) pairs)
+size_t ticket_count(const eesd_config *c) { return 1024 + (size_t)c->n_heads; }
 
 Workspace carve(const eesd_config *c) {
     Workspace w;
@@ -133,7 +132,7 @@ Workspace carve(const eesd_config *c) {
     w.hT = take((size_t)c->d_model * 4);
     w.xs_cali = take(2 * R * (size_t)c->d_model * 2);
     w.theta = take(16);
-    w.wx = w.wx_save = w.wout = w.wout_floats = w.wssq = w.wtok = w.wapart = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
+    w.wx = w.wx_save = w.wout = w.wout_floats = w.wssq = w.wtok = w.wxs[0] = w.wxs[1] = w.wxs[2] = 0;
     if (const size_t P = (size_t)prefill_rows(c)) {
         // prompt path: residual stream, one projection result, the three activation matrices as
         // two bf16 terms ([chunk of 16][hi | lo][16][K]), RMSNorm statistics, token ids
@@ -149,7 +148,6 @@ Workspace carve(const eesd_config *c) {
         w.wxs[X_FFN] = take(2 * P * (size_t)c->ffn_dim * 2);
         w.wssq = take(P * kSsqBlocks * 4);
         w.wtok = take(P * 4);
-        w.wapart = take(attention_prompt_scratch_floats(c->max_ctx, c->page_tokens, c->n_heads, c->head_dim, (int)P) * 4);
     }
     w.total = o;
     return w;
@@ -186,7 +184,7 @@ struct eesd_ctx {
     int64_t n_verify, n_trials;
     // prompt (wide) path: up to wide_rows prompt rows per pass
     int wide_rows;
-    float *wx, *wx_save, *wout, *wssq, *wapart;
+    float *wx, *wx_save, *wout, *wssq;
     size_t wout_floats;          // room in wout
     void *wxs[3];
     int32_t *wtok;
@@ -384,8 +382,8 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
 
 // Prompt pass (wide path): the target model on Mtot <= wide_rows prompt rows at positions
 // p0.., no logits.  Projections run on the wide tensor-core kernel (weights cross HBM once
-// per pass); the rows' keys / values are appended first, then all 16-row chunks attend to the
-// cache in one launch; the exit layer's keys / values follow layer N.
+// per pass); the rows' keys / values are appended first, then the rows attend to the cache 128 at a
+// time (causal tensor-core attention); the exit layer's keys / values follow layer N.
 int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
     const eesd_config &f = c->cfg;
     cudaStream_t s = c->stream;
@@ -412,9 +410,9 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
     resid(nullptr, c->layers[0].g_attn);
     auto layer = [&](const LayerW &w, int slot, const float *g_after) {
         PartView pv = proj(w.m_qkv, X_NORM, qd + 2 * kvd, d);
-        // keys / values of all rows into the cache first, then every 16-row chunk attends in one launch
+        // keys / values of all rows into the cache first, then the causal attention of all rows
         launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, slot), c->rope, nullptr, true, c->err, qd);
-        launch_attention_prompt(s, pv, rs, c->rope, kv_geom(c, slot), c->wapart, c->tickets, c->wxs[X_ATTN], Mtot, p0, H, c->err, c->wait_polls);
+        launch_attention_prompt(s, pv, rs, c->rope, kv_geom(c, slot), c->wxs[X_ATTN], Mtot, p0, H, c->err, c->wait_polls);
         c->launches += 2;
         pv = proj(w.m_o, X_ATTN, d, qd);
         resid(&pv, w.g_ffn);
@@ -830,7 +828,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
         ok = ok && tc_make_map(&c->m_exit_head, c->exit_head, cfg->vocab, d, 128, true);
         if (c->wide_rows) {
             c->wx = (float *)(ws + w.wx); c->wx_save = (float *)(ws + w.wx_save); c->wout = (float *)(ws + w.wout); c->wout_floats = w.wout_floats; c->wssq = (float *)(ws + w.wssq);
-            c->wtok = (int32_t *)(ws + w.wtok); c->wapart = (float *)(ws + w.wapart);
+            c->wtok = (int32_t *)(ws + w.wtok);
             const int ks[3] = {d, qd_, F};
             for (int i = 0; i < 3; i++) {
                 c->wxs[i] = ws + w.wxs[i];

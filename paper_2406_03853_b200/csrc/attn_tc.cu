@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
                                                           float *__restrict__ apart, unsigned int *tickets,
                                                           float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
                                                           int M, int pos0, int H, int pps, int n_split, float scale2, int *err,
-                                                          int Mtot, int nbat, size_t ml_off, TreeRows tr, uint32_t spin) {
+                                                          TreeRows tr, uint32_t spin) {
     constexpr int HALF = D / 2;
     constexpr uint32_t LBO_C = Opnd<NC>::LBO;          // query / numerator operands
     constexpr uint32_t GRP = (D / 8) * 128;            // bytes of one 8-position group of a key / value tile
@@ -153,23 +153,9 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
-    // Prompt mode (Mtot > 0): grid z also runs over the 16-row chunks of Mtot prompt rows whose
-    // keys and values are in the cache already; chunk c is an independent problem (rows
-    // pos0 + 16 c .., its own scratch, counters and slice count) and nothing is appended.
-    const int chunk = blockIdx.z / nbat, bz = blockIdx.z - chunk * nbat;
-    const bool cached_rows = Mtot > 0;
-    if (cached_rows) {
-        M = min(kMaxRows, Mtot - chunk * kMaxRows);
-        pos0 += chunk * kMaxRows;
-        n_split = (((pos0 + M + PT - 1) >> ptl) + pps - 1) / pps;
-        if (sp >= n_split || group * M <= bz * NC) return;   // a short last chunk fills fewer slices and batches
-        pv.base += (size_t)chunk * kMaxRows * pv.R;
-        rs.ssq += (size_t)chunk * kMaxRows * kSsqBlocks;
-        if (attn_out) attn_out += (size_t)chunk * kMaxRows * H * D;
-        if (attn_split) attn_split += (size_t)chunk * 2 * kMaxRows * H * D;
-        apart += (size_t)chunk * (ml_off + (size_t)H * kMaxRows * kMaxSlices * 2);
-    }
-    float2 *ml = reinterpret_cast<float2 *>(apart + ml_off);   // per-slice (maximum, sum): [H][16][kMaxSlices]
+    const int bz = blockIdx.z;
+    // per-slice (maximum, sum) pairs live behind the outputs: [H][16][kMaxSlices]
+    float2 *ml = reinterpret_cast<float2 *>(apart + (size_t)H * kMaxSlices * kMaxRows * D);
     const int r0 = bz * NC;                  // first column ((head, row) pair) of this block's batch
     const int nb = min(NC, group * M - r0);  // columns in use; pair rho = r0 + c = g * M + m
     const int ctx_len = pos0 + M;
@@ -221,7 +207,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
         s_tb[tid - 160] = tile_blocks(pv.sk, tid - 160 < nq ? tq0 + tid - 160 : (tid - 160 == nq ? tk : tv));
     // new rows that fall into this slice: (position, key pair | value pair) items
     const int p_first = max(lo, pos0), p_last = min(lo + npos, ctx_len);   // [p_first, p_last)
-    const int n_new = cached_rows ? 0 : max(0, p_last - p_first) * D;
+    const int n_new = max(0, p_last - p_first) * D;
     const int n_q = nb * HALF;
     constexpr int kNewMax = (kMaxRows * D + THREADS - 1) / THREADS;
     constexpr int kQMax = (NC * HALF + THREADS - 1) / THREADS;
@@ -506,7 +492,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
     }
     // ---- merge: the block that arrives last for this (KV head, batch) combines all slices
     if (tid == 0) {
-        unsigned int *tkt = tickets + ((size_t)chunk * gridDim.x + kh) * nbat + bz;   // one counter per (chunk, KV head, batch)
+        unsigned int *tkt = tickets + (size_t)kh * gridDim.z + bz;   // one counter per (KV head, batch)
         const unsigned int prev = atomicAdd(tkt, 1u);
         *s_last = (prev == (unsigned int)n_split - 1);
         if (*s_last) *tkt = 0;
@@ -585,18 +571,15 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
 template <int D, int NC, bool TR>
 static void launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv, float *apart,
                    unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H, int pps, int n_split,
-                   float scale, bool early, int *err, int Mtot, const TreeRows &tr, uint32_t wait_polls) {
+                   float scale, bool early, int *err, const TreeRows &tr, uint32_t wait_polls) {
     const int rows = (H / kv.Hkv) * M, nbat = (rows + NC - 1) / NC;
-    const int chunks = Mtot > 0 ? (Mtot + kMaxRows - 1) / kMaxRows : 1;
-    const size_t ml_off = (size_t)H * (Mtot > 0 ? n_split : kMaxSlices) * kMaxRows * D;
     const Smem lay = carve(pps * kv.page_tokens, D, NC, n_split);
     // once per instantiation (thread-safe static initialisation)
     static const cudaError_t configured =
         cudaFuncSetAttribute(attn_tc_kernel<D, NC, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
     (void)configured;
-    launch_k(attn_tc_kernel<D, NC, TR>, dim3(kv.Hkv, n_split, chunks * nbat), dim3(THREADS), (size_t)lay.total, s, early && pdl_enabled(),
-             pv, rs, rope, kv, apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, Mtot, nbat, ml_off,
-             tr, wait_polls);
+    launch_k(attn_tc_kernel<D, NC, TR>, dim3(kv.Hkv, n_split, nbat), dim3(THREADS), (size_t)lay.total, s, early && pdl_enabled(),
+             pv, rs, rope, kv, apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, tr, wait_polls);
 }
 
 }  // namespace at
@@ -620,18 +603,15 @@ int attention_tc_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, in
     return (n_pages + pps - 1) / pps;
 }
 
-// pages per block in prompt mode: as long as a block can hold
-int attention_tc_prompt_pps(int page_tokens) { return at::MAX_TILES * at::TILE / page_tokens; }
-
 void launch_attention_tc(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv, float *apart,
                          unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H, int pps, int n_split,
-                         bool early, int *err, int Mtot, const TreeRows *tree, uint32_t wait_polls) {
+                         bool early, int *err, const TreeRows *tree, uint32_t wait_polls) {
     // queries are scaled by 1 / sqrt(D) and by log2 e: the softmax numerators are powers of two
     const float scale = 1.4426950408889634f / sqrtf((float)kv.D);
     const int rows = (H / kv.Hkv) * M;
     const TreeRows tr = tree ? *tree : chain_rows();
     const bool wide = attention_tc_columns(rows) == 32;
-#define EESD_AT(D, NC, TR) at::launch<D, NC, TR>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, Mtot, tr, wait_polls)
+#define EESD_AT(D, NC, TR) at::launch<D, NC, TR>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls)
     if (kv.D == 64) {
         if (tree) { if (wide) EESD_AT(64, 32, true); else EESD_AT(64, 16, true); }
         else { if (wide) EESD_AT(64, 32, false); else EESD_AT(64, 16, false); }

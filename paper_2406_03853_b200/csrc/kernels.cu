@@ -727,7 +727,7 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
         const int nc = attention_tc_columns(rows);
         const int n_split = attention_tc_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + nc - 1) / nc, n_sm, max_splits, &pps);
         if (refuse(n_split)) return;
-        launch_attention_tc(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, 0, tree,
+        launch_attention_tc(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, tree,
                             wait_polls);
         return;
     }
@@ -737,30 +737,6 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
     const float scale = 1.0f / sqrtf((float)kv.D);
     if (kv.D == 64) attn_dispatch<64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls);
     else attn_dispatch<128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls);
-}
-
-// Prompt attention (bf16 models): Mtot rows at positions pos0.. whose keys / values are in the cache
-// already (launch_qkv_post), all 16-row chunks in one launch.  Slices are as long as a block can hold.
-int attention_prompt_splits(int ctx_len, int page_tokens) {
-    const int pps = attention_tc_prompt_pps(page_tokens), n_pages = (ctx_len + page_tokens - 1) / page_tokens;
-    return (n_pages + pps - 1) / pps;
-}
-size_t attention_prompt_scratch_floats(int ctx_len, int page_tokens, int H, int D, int rows) {
-    const size_t chunks = (rows + kMaxRows - 1) / kMaxRows;
-    const size_t per_chunk = (size_t)H * attention_prompt_splits(ctx_len, page_tokens) * kMaxRows * D + (size_t)H * kMaxRows * kMaxSlices * 2;
-    return chunks * per_chunk;
-}
-void launch_attention_prompt(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope,
-                             const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
-                             int Mtot, int pos0, int H, int *err, uint32_t wait_polls) {
-    const int pps = attention_tc_prompt_pps(kv.page_tokens), n_split = attention_prompt_splits(pos0 + Mtot, kv.page_tokens);
-    if (n_split > kMaxSlices) {
-        const int e = kErrPlan;
-        cudaMemcpyAsync(err, &e, sizeof(e), cudaMemcpyHostToDevice, s);
-        return;
-    }
-    launch_attention_tc(s, pv, rs, rope, kv, apart, tickets, nullptr, attn_split, kMaxRows, pos0, H, pps, n_split, false, err, Mtot,
-                        nullptr, wait_polls);
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU, partial sums

@@ -101,23 +101,18 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
 // most context tokens the attention kernel of `dtype` can serve with pages of page_tokens
 int attention_max_ctx(int dtype, int page_tokens);
 // tensor-core attention (attn_tc.cu; bf16 cache): columns ((head, row) pairs) per block for `rows` pairs per KV head,
-// slices of the context, pages per block in prompt mode, and the launcher (Mtot > 0: prompt mode)
+// slices of the context, and the launcher
 int attention_tc_columns(int rows);
 int attention_tc_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out);
-int attention_tc_prompt_pps(int page_tokens);
 void launch_attention_tc(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv, float *apart,
                          unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H, int pps, int n_split,
-                         bool early, int *err, int Mtot, const TreeRows *tree, uint32_t wait_polls);
-// Prompt attention: all 16-row chunks of Mtot rows in one launch; the rows' keys / values must be
-// in the cache already (launch_qkv_post with only_kv on the QKV result) and pv must be a plain
-// [Mtot][R] result (mode 0).  apart: attention_prompt_scratch_floats(...) floats; tickets: zeroed
-// counters, one per (chunk, KV head, batch).  attn_split: [chunk][hi | lo][16][H * D] bf16.
+                         bool early, int *err, const TreeRows *tree, uint32_t wait_polls);
 int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out);
-int attention_prompt_splits(int ctx_len, int page_tokens);
-size_t attention_prompt_scratch_floats(int ctx_len, int page_tokens, int H, int D, int rows);
-void launch_attention_prompt(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope,
-                             const KvGeom &kv, float *apart, unsigned int *tickets, void *attn_split,
-                             int Mtot, int pos0, int H, int *err, uint32_t wait_polls);
+// Causal prompt attention (attn_prompt.cu; bf16 cache, D = 64 or 128): Mtot rows at positions pos0.., 128 rows per
+// block; the rows' keys / values must be in the cache already (launch_qkv_post with only_kv on the QKV
+// result) and pv must be a plain [Mtot][R] result (mode 0).  attn_split: [chunk][hi | lo][16][H * D] bf16.
+void launch_attention_prompt(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
+                             void *attn_split, int Mtot, int pos0, int H, int *err, uint32_t wait_polls);
 // H^(T) of the calibration predictor: row `row` (or row *row_dev when row_dev is given) of x[.][d]
 // is copied to hT (fp32) and, if xs is given, written as two bf16 terms into a one-chunk [32][d] matrix
 void launch_copy_row(cudaStream_t s, const float *x, int row, const int32_t *row_dev, float *hT, void *xs, int d);

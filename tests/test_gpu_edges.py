@@ -130,22 +130,25 @@ def test_same_tokens_without_programmatic_dependent_launch():
     assert outs[0] == outs[1] and len(outs[0].split()) == 32
 
 
-@pytest.mark.parametrize("variant,n_prompt,max_ctx", [("mha", 300, 384), ("gqa8", 150, 256), ("wide_head", 200, 256),
-                                                        ("two_passes", 700, 768)])
-def test_wide_prompt_pass_matches_row_chunks_and_oracle(variant, n_prompt, max_ctx):
+@pytest.mark.parametrize("variant,n_prompt,max_ctx,pt", [("mha", 300, 384, 16), ("gqa8", 150, 256, 16), ("wide_head", 200, 256, 16),
+                                                           ("two_passes", 700, 768, 16), ("mha", 131, 256, 8), ("mha", 258, 384, 128),
+                                                           ("wide_head", 700, 768, 128), ("wide_head", 530, 640, 8),
+                                                           ("gqa8", 66, 128, 32)])
+def test_wide_prompt_pass_matches_row_chunks_and_oracle(variant, n_prompt, max_ctx, pt):
     """Prompts longer than 16 rows go through the wide projection kernel (128-row panels) and
-    the prompt mode of the attention kernel (all 16-row chunks in one launch); the cache they
-    leave must equal, up to summation order, the one built 16 rows at a time, and the next pass
-    must match the oracle.  Variants: ragged panels, 8 query heads per KV head (four row batches
-    per chunk), 128-wide heads, and a prompt of more than 512 rows (a second pass that starts at
-    a non-zero position and attends over several slices)."""
+    the causal prompt attention kernel (128 query rows per block, streaming over 128-position
+    tiles); the cache they leave must equal, up to summation order, the one built 16 rows at a
+    time, and the next pass must match the oracle.  Variants: ragged panels and row tiles (a last
+    tile of 1, 2 or 17 rows), 8 query heads per KV head, 128-wide heads, every page size from 8
+    to 128 tokens, and prompts of more than 512 rows (a second pass that starts at a non-zero
+    position, whose first row tile already sees four full tiles)."""
     base = synth.TINY.with_(dtype="bf16", ffn_dim=640, n_layers=3)
     spec = {"mha": base, "two_passes": base.with_(n_layers=2),
             "gqa8": base.with_(n_heads=8, n_kv_heads=1, head_dim=64),
             "wide_head": base.with_(n_heads=2, n_kv_heads=1, head_dim=128)}[variant]
     prompt = synth.prompt_tokens(9, n_prompt, spec.vocab).numpy()
-    wide = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, page_tokens=16)
-    rows = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, page_tokens=16)
+    wide = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, page_tokens=pt)
+    rows = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, page_tokens=pt)
     rows.capture_hidden(True)                                 # capture keeps the 16-row path
     n0 = wide.launch_count()
     wide.prefill(prompt)
@@ -193,8 +196,8 @@ def test_long_context_many_slices(dtype):
     eng.close()
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(dtype):
+@pytest.mark.parametrize("dtype,n_prompt", [("f32", 12), ("bf16", 12), ("bf16", 150)])
+def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(dtype, n_prompt):
     # With the bound of the in-kernel waits at zero, the first wait of every thread block (attention:
     # its cache slice; projection: the first ring stage / accumulator) gives up before any tensor-core
     # operation is issued; the blocks let the copies they had requested land and return.  The call
@@ -202,8 +205,8 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(dtype):
     # produce the oracle's tokens again.  Nothing is stalled on the GPU to get here.
     from paper_2406_03853_b200 import EesdError
     spec = synth.TINY if dtype == "f32" else synth.TINY.with_(dtype="bf16", ffn_dim=640)
-    eng = engine_from_spec(spec, max_ctx=96, fixed_k=3)
-    prompt = synth.prompt_tokens(21, 12, spec.vocab).numpy()
+    eng = engine_from_spec(spec, max_ctx=96 if n_prompt < 64 else 192, fixed_k=3)
+    prompt = synth.prompt_tokens(21, n_prompt, spec.vocab).numpy()   # 150 tokens: the prompt pass's wide kernels give up too
     out0, trace0, _ = eng.generate(prompt, 16)
     eng.set_wait_limit(0)
     with pytest.raises(EesdError) as e:
