@@ -418,6 +418,8 @@ def run_sweep(args, device):
             torch.cuda.empty_cache()
     else:
         for N in (1, 2, 3, 5, 8, 10):
+            if N >= synth.SPECS[spec_name].n_layers:   # the exit must leave at least one layer to skip
+                continue
             eng, spec, _, _ = build_engine(args.workload, args.temperature, b.CTRL_BETA_TS, device, alpha=args.alpha, n_early=N)
             measure(eng, spec, f"N={N}", None)
             eng.close()
