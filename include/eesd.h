@@ -339,6 +339,44 @@ int eesd_capture_hidden(eesd_ctx *ctx, float *device_buf, size_t bytes);
 int eesd_set_wait_limit(eesd_ctx *ctx, uint32_t polls);
 int eesd_clear_device_error(eesd_ctx *ctx);
 
+/* ---- batch mode: several sequences decoded together -------------------------------------------
+ * An extension: the paper decodes one sequence at a time (its experiments run at batch 1).  The
+ * rows of a pass (at most EESD_MAX_ROWS) are shared by up to EESD_MAX_BATCH sequences, each with
+ * its own KV pages (one pool), positions and tokens; every weight crosses HBM once per pass for
+ * all of them.  A round drafts the same number K of tokens for every sequence that still owes
+ * tokens (n * (K + 1) <= EESD_MAX_ROWS rows in its verification pass): K comes from the schedule
+ * or from eesd_config.fixed_k; the controllers' per-sequence stopping rule (Algorithms 2-3) has
+ * no batch counterpart and is not consulted.  Per sequence the result is what single-sequence
+ * decoding with the same draft lengths and the same uniforms gives (Algorithm 1: drafting,
+ * verification and acceptance of a sequence never look at another sequence).
+ * bf16 models only (UNSUPPORTED otherwise, and with tree verification).  While batch mode is on,
+ * the single-sequence calls that start or feed a sequence return STATE. */
+#define EESD_MAX_BATCH 8
+/* Enters batch mode with n_seq empty sequences (1..EESD_MAX_BATCH), or leaves it (n_seq = 0); either
+ * way every sequence is forgotten and all KV pages are free afterwards. */
+int eesd_batch_begin(eesd_ctx *ctx, int n_seq);
+/* eesd_prefill for sequence `seq` of the batch (same arguments and errors). */
+int eesd_batch_prefill(eesd_ctx *ctx, int seq, const int32_t *prompt, int n_prompt);
+/* Rounds of {K draft steps on one row per sequence, one verification pass of K + 1 rows per sequence,
+ * acceptance of all sequences in one kernel launch} until every sequence has max_new new tokens; a
+ * sequence that has them leaves the rounds.  k_schedule[r] (host, may be NULL) is the draft length of
+ * round r < n_schedule, then fixed_k; either is cut to what the pass rows, k_cap and the contexts allow.
+ * u: one eesd_uniforms per sequence (host; may be NULL when greedy; u_ctrl unused).
+ * out: host, [n_seq][max_new].  stats: sums over the sequences (rounds = rounds of the batch).
+ * trace (may be NULL): [n_seq][trace_cap]; n_rounds (may be NULL): [n_seq] rounds each sequence took part in.
+ * Errors: BADARG, STATE (batch mode off or a sequence without prompt), RNG, CTX_FULL, DEVICE. */
+int eesd_batch_decode(eesd_ctx *ctx, int max_new, const int32_t *k_schedule, int n_schedule,
+                      const eesd_uniforms *u, int32_t *out, eesd_stats *stats, eesd_round *trace,
+                      int trace_cap, int *n_rounds);
+/* Context length (pending token included) and KV pages of one sequence of the batch. */
+int eesd_batch_context_len(const eesd_ctx *ctx, int seq, int *n_tokens, int *pages_in_use);
+/* Test and measurement hooks, the batch forms of eesd_verify_only / eesd_assume_context: one pass of the
+ * target model over m rows per sequence (tokens: host, [n_seq][m], n_seq * m <= EESD_MAX_ROWS) at the end
+ * of each sequence's context, logits of row b * m + i in eesd_logits(.., 0, ..); and a sequence declared
+ * to hold n_ctx tokens whose cache rows are whatever the pool holds. */
+int eesd_batch_verify_only(eesd_ctx *ctx, const int32_t *tokens, int m);
+int eesd_batch_assume_context(eesd_ctx *ctx, int seq, int n_ctx, int32_t pending);
+
 /* How the attention kernel of a pass would cut a context of ctx_len tokens (host arithmetic, no
  * device needed): pages per thread block and thread blocks ("slices") per KV head, for `pairs`
  * (query head, new row) pairs per KV head on a device of n_sm multiprocessors.  A slice count

@@ -118,6 +118,12 @@ def lib():
         L.eesd_assume_context.argtypes = [vp, C.c_int, C.c_int32]
         L.eesd_verify_only.argtypes = [vp, vp, C.c_int]
         L.eesd_logits.argtypes = [vp, C.c_int, C.POINTER(vp)]
+        L.eesd_batch_begin.argtypes = [vp, C.c_int]
+        L.eesd_batch_prefill.argtypes = [vp, C.c_int, vp, C.c_int]
+        L.eesd_batch_decode.argtypes = [vp, C.c_int, vp, C.c_int, vp, vp, C.POINTER(Stats), vp, C.c_int, vp]
+        L.eesd_batch_context_len.argtypes = [vp, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        L.eesd_batch_verify_only.argtypes = [vp, vp, C.c_int]
+        L.eesd_batch_assume_context.argtypes = [vp, C.c_int, C.c_int, C.c_int32]
         L.eesd_capture_hidden.argtypes = [vp, vp, C.c_size_t]
         L.eesd_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
         L.eesd_set_wait_limit.argtypes = [vp, C.c_uint32]
@@ -370,6 +376,52 @@ class Engine:
     def verify_only(self, tokens):
         t = _np_i32(tokens)
         self._check(lib().eesd_verify_only(self.h, t.ctypes.data, len(t)), "eesd_verify_only")
+
+    # ---- batch mode: several sequences decoded together
+    def batch_begin(self, n_seq: int):
+        """eesd_batch_begin: n_seq empty sequences (0 leaves batch mode)."""
+        self._check(lib().eesd_batch_begin(self.h, n_seq), "eesd_batch_begin")
+        self._n_seq = n_seq
+
+    def batch_prefill(self, seq: int, prompt):
+        p = _np_i32(prompt)
+        self._check(lib().eesd_batch_prefill(self.h, seq, p.ctypes.data, len(p)), "eesd_batch_prefill")
+
+    def batch_context_len(self, seq: int):
+        n, p = C.c_int(), C.c_int()
+        self._check(lib().eesd_batch_context_len(self.h, seq, C.byref(n), C.byref(p)), "eesd_batch_context_len")
+        return n.value, p.value
+
+    def batch_assume_context(self, seq: int, n_ctx: int, pending: int = 0):
+        self._check(lib().eesd_batch_assume_context(self.h, seq, n_ctx, pending), "eesd_batch_assume_context")
+
+    def batch_verify_only(self, tokens):
+        """tokens: [n_seq, m] rows per sequence; logits of row b * m + i are row b * m + i of logits(0, n_seq * m)."""
+        t = np.ascontiguousarray(np.asarray(tokens, np.int32))
+        self._check(lib().eesd_batch_verify_only(self.h, t.ctypes.data, t.shape[1]), "eesd_batch_verify_only")
+
+    def batch_decode(self, max_new: int, k_schedule=None, uniforms=None):
+        """eesd_batch_decode.  uniforms: one dict per sequence (or None when greedy).  Returns
+        (tokens[n_seq, max_new], per-sequence traces [(k, n_accept, next_token)], Stats)."""
+        B = self._n_seq
+        out = np.empty((B, max_new), np.int32)
+        ks = None if k_schedule is None else _np_i32(k_schedule)
+        keep, U = [], None
+        if uniforms is not None:
+            U = (Uniforms * B)()
+            for b in range(B):
+                Ub, kb = self._uniforms(uniforms[b])
+                keep.append(kb)
+                U[b] = Ub
+        cap = max_new + 1
+        trace = (Round * (cap * B))()
+        st, nr = Stats(), (C.c_int * B)()
+        self._check(lib().eesd_batch_decode(self.h, max_new, None if ks is None else ks.ctypes.data, 0 if ks is None else len(ks),
+                                            None if U is None else C.cast(U, C.c_void_p), out.ctypes.data, C.byref(st),
+                                            C.cast(trace, C.c_void_p), cap, C.cast(nr, C.c_void_p)), "eesd_batch_decode")
+        traces = [[(trace[b * cap + i].k, trace[b * cap + i].n_accept, trace[b * cap + i].next_token) for i in range(nr[b])]
+                  for b in range(B)]
+        return out, traces, st
 
     def logits(self, which: int, rows: int) -> torch.Tensor:
         """fp32 [rows, V] tensor aliasing the context's logits (0: verify pass, 1: draft steps)."""

@@ -285,7 +285,7 @@ __global__ void __launch_bounds__(kAccThreads) accept_kernel(const float *p_logi
                                                              const int32_t *tokens, const float *u_acc,
                                                              const float *u_res, int K, int V, float T,
                                                              RowStat *stats, unsigned int *counters,
-                                                             int32_t *n_acc, int32_t *y, int32_t *pending_out) {
+                                                             int32_t *n_acc, int32_t *y, int32_t *pending_out, int tok_stride) {
     __shared__ AccSmem sm;
     __shared__ int s_last, s_j;
     const int rows = 2 * K + 1;
@@ -310,7 +310,7 @@ __global__ void __launch_bounds__(kAccThreads) accept_kernel(const float *p_logi
     if (!s_last) return;
     __threadfence();
 
-    const int32_t *x = tokens + (size_t)b * K;
+    const int32_t *x = tokens + (size_t)b * tok_stride;   // the sequence's K drafted tokens
     __shared__ int s_ok[EESD_MAX_ROWS];
     if ((int)threadIdx.x < K && K <= EESD_MAX_ROWS) {   // one test per thread: their loads are in flight together
         const int j = threadIdx.x, t = x[j];
@@ -375,28 +375,29 @@ size_t accept_scratch_bytes(int B, int K) {
 
 void launch_accept(cudaStream_t s, const float *p_logits, const float *q_logits, const int32_t *tokens,
                    const float *u_acc, const float *u_res, int B, int K, int V, float T, void *scratch,
-                   int32_t *n_acc, int32_t *y, int32_t *pending_out) {
+                   int32_t *n_acc, int32_t *y, int32_t *pending_out, int tok_stride) {
     unsigned int *counters = (unsigned int *)scratch;
     RowStat *stats = (RowStat *)((char *)scratch + ((size_t)B * sizeof(unsigned int) + 15) / 16 * 16);
     accept_kernel<<<B * (2 * K + 1), kAccThreads, 0, s>>>(p_logits, q_logits, tokens, u_acc, u_res, K, V, T,
-                                                         stats, counters, n_acc, y, pending_out);
+                                                         stats, counters, n_acc, y, pending_out, tok_stride ? tok_stride : K);
 }
 
 // ---- draft-token sampler -------------------------------------------------------------------------
 __global__ void __launch_bounds__(kAccThreads) sample_rows_kernel(const float *logits, const float *u, int V, float T,
-                                                                  int32_t *out) {
+                                                                  int32_t *out, size_t logit_stride, int out_stride) {
     __shared__ AccSmem sm;
     const int b = blockIdx.x;
-    const float *l = logits + (size_t)b * V;
+    const float *l = logits + (size_t)b * logit_stride;
     const bool greedy = (T == 0.0f);
     RowStat st = row_stat(l, V, greedy ? 1.0f : T, !greedy, sm);
     int tok = st.arg;
     if (!greedy) tok = block_draw(l, st, nullptr, st, T, V, u[b], sm);
-    if (threadIdx.x == 0) out[b] = tok;
+    if (threadIdx.x == 0) out[(size_t)b * out_stride] = tok;
 }
 
-void launch_sample_rows(cudaStream_t s, const float *logits, const float *u, int B, int V, float T, int32_t *out) {
-    sample_rows_kernel<<<B, kAccThreads, 0, s>>>(logits, u, V, T, out);
+void launch_sample_rows(cudaStream_t s, const float *logits, const float *u, int B, int V, float T, int32_t *out,
+                        size_t logit_stride, int out_stride) {
+    sample_rows_kernel<<<B, kAccThreads, 0, s>>>(logits, u, V, T, out, logit_stride ? logit_stride : (size_t)V, out_stride);
 }
 
 }  // namespace eesd

@@ -92,6 +92,9 @@ int prefill_rows(const eesd_config *c) {
 // arrival counters of the attention merge: one per (KV head, batch of (head, row) pairs)
 size_t ticket_count(const eesd_config *c) { return 1024 + (size_t)c->n_heads; }
 
+// entries of one sequence's page table
+size_t table_len(const eesd_config *c) { return (size_t)c->max_ctx / c->page_tokens + 2; }
+
 Workspace carve(const eesd_config *c) {
     Workspace w;
     const size_t R = EESD_MAX_ROWS;
@@ -123,12 +126,12 @@ Workspace carve(const eesd_config *c) {
     w.logits_p = take(R * (size_t)c->vocab * 4);
     w.logits_q = take(R * (size_t)c->vocab * 4);
     w.rope = take((size_t)c->max_ctx * (c->head_dim / 2) * 8);
-    w.page_table = take(((size_t)c->max_ctx / c->page_tokens + 2) * 4);
+    w.page_table = take(table_len(c) * kMaxSeqs * 4);   // one table per sequence of a batch (one sequence: the first)
     w.ints = take(kIntSlots * 4);
     w.u_dev = take((size_t)3 * c->max_ctx * 4);
     w.u_stage = take(64 * 4);
     w.err = take(16);
-    w.accept = take(accept_scratch_bytes(1, EESD_MAX_ROWS));
+    w.accept = take(accept_scratch_bytes(kMaxSeqs, EESD_MAX_ROWS));
     w.hT = take((size_t)c->d_model * 4);
     w.xs_cali = take(2 * R * (size_t)c->d_model * 2);
     w.theta = take(16);
@@ -156,7 +159,7 @@ Workspace carve(const eesd_config *c) {
 // offsets inside the device integer area
 constexpr int kRoundTok = 0;   // [17]: pending token, then the round's draft tokens
 constexpr int kRowTok = 20;    // [16]: token rows of a prefill chunk / verify_only
-constexpr int kResult = 40;    // [3]: n_accept, next token, row of the kept leaf (tree verification) or -1
+constexpr int kResult = 40;    // [3]: n_accept, next token, row of the kept leaf (tree verification) or -1; batch mode: [8] n_accept, [8] next tokens
 constexpr int kLeafTok = 64;   // [15]: tree verification: leaves of depth 1, depth 2, ... (width - 1 each)
 constexpr int kTreeTop = 80;   // [16]: tree verification: the target's top-1 token of every row
 
@@ -208,6 +211,13 @@ struct eesd_ctx {
     // sequence state
     std::vector<int32_t> tokens;
     bool prefilled;
+    // batch mode (several sequences decoded together): the other sequences' state is parked here while one is
+    // selected; page_table points at the selected sequence's table inside the array starting at page_table0
+    struct Seq { std::vector<int32_t> tokens, page_of; bool prefilled; };
+    std::vector<Seq> seqs;       // empty: batch mode off
+    int32_t *page_table0;
+    const BatchRows *batch_cur;  // geometry of the pass being enqueued (null: one sequence)
+    BatchRows batch_rows;
     int round_k;
     int64_t alpha, beta;
     int64_t launches;
@@ -243,7 +253,7 @@ int check_launch(eesd_ctx *c) {
 KvGeom kv_geom(eesd_ctx *c, int slot) {
     KvGeom g;
     g.slot_base = (char *)c->buf.kv_pool + (size_t)slot * c->slot_bytes;
-    g.page_table = c->page_table;
+    g.page_table = c->batch_cur ? c->page_table0 : c->page_table;   // a batch pass offsets it per sequence
     g.Hkv = c->cfg.n_kv_heads;
     g.D = c->cfg.head_dim;
     g.page_tokens = c->cfg.page_tokens;
@@ -327,7 +337,7 @@ void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const fl
     const RowScale rs = norm_scale(c);
     PartView pv = run_proj(c, w.wqkv, &w.m_qkv, P_QKV, X_NORM, M, qd + 2 * kvd, d);
     launch_attention(s, f.dtype, pv, rs, c->rope, kv_geom(c, slot), c->apart, c->tickets, c->use_tc ? nullptr : c->attn,
-                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, true, c->err, c->tree_cur, c->wait_polls);
+                     c->xs[X_ATTN], M, pos0, f.n_heads, c->n_sm, kAttnSplits, true, c->err, c->tree_cur, c->wait_polls, c->batch_cur);
     pv = run_proj(c, w.wo, &w.m_o, P_O, X_ATTN, M, d, qd);
     run_resid(c, &pv, w.g_ffn, nullptr, M);
     pv = run_proj(c, w.wgu, &w.m_gu, P_GU, X_NORM, M, 2 * F, d);
@@ -364,8 +374,19 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
             for (int e = 0; e + 1 < E; e++) run_layer(c, c->layers[L + e], L + e, M, pos0, c->layers[L + e + 1].g_attn, nullptr);
             const char *wkv = c->layers[L + E - 1].wqkv + (size_t)qd * d * c->es;
             PartView pv = run_proj(c, wkv, &c->m_exit_kv, P_EXIT_KV, X_NORM, M, 2 * kvd, d);
-            launch_qkv_post(s, f.dtype, pv, norm_scale(c), M, pos0, f.n_heads, kv_geom(c, L + E - 1), c->rope, nullptr, true, c->err, 0,
-                            c->tree_cur);
+            if (c->batch_cur) {   // every sequence's rows go to its own positions and pages
+                const BatchRows &br = *c->batch_cur;
+                for (int b = 0; b < br.n_seq; b++) {
+                    KvGeom g = kv_geom(c, L + E - 1);
+                    g.page_table += br.table_off[b];
+                    launch_qkv_post(s, f.dtype, pv, norm_scale(c), br.rows[b], br.pos0[b], f.n_heads, g, c->rope, nullptr, true, c->err, 0,
+                                    nullptr, br.row0[b]);
+                }
+                c->launches += br.n_seq - 1;
+            } else {
+                launch_qkv_post(s, f.dtype, pv, norm_scale(c), M, pos0, f.n_heads, kv_geom(c, L + E - 1), c->rope, nullptr, true, c->err, 0,
+                                c->tree_cur);
+            }
             if (E > 1) CU(c, cudaMemcpyAsync(c->x, c->x_save, (size_t)M * d * 4, cudaMemcpyDeviceToDevice, s));
             const float *g_next = l + 1 < L ? c->layers[l + 1].g_attn : c->g_final;
             run_resid(c, nullptr, g_next, nullptr, M);
@@ -671,6 +692,128 @@ int finish_round(eesd_ctx *c, const int32_t *draft_tokens_host, int *n_accept, i
     return EESD_OK;
 }
 
+
+// ------------------------------------------------------------------------------------ batch mode
+// Several sequences decoded together (an extension; the paper decodes one at a time): the rows of a
+// pass are split among the sequences, every sequence has its own pages, positions and tokens, and
+// the weights cross HBM once per pass for all of them.  Host state of the sequences that are not
+// selected is parked in c->seqs; select_seq swaps one in, so that the single-sequence code
+// (prefill, page bookkeeping) works on it unchanged.
+bool batch_on(const eesd_ctx *c) { return !c->seqs.empty(); }
+
+void select_seq(eesd_ctx *c, int b) {
+    std::swap(c->tokens, c->seqs[b].tokens);
+    std::swap(c->page_of, c->seqs[b].page_of);
+    std::swap(c->prefilled, c->seqs[b].prefilled);
+    c->page_table = c->page_table0 + (size_t)b * table_len(&c->cfg);
+}
+void park_seq(eesd_ctx *c, int b) {
+    select_seq(c, b);   // the swap is its own inverse
+    c->page_table = c->page_table0;
+}
+
+// rows of a pass: sequence act[i] gets `rows` rows starting `back` positions before the end of its
+// context (its tokens.size() counts the pending token, which takes position size - 1)
+void batch_geometry(eesd_ctx *c, const int *act, int n_act, int rows, int step) {
+    BatchRows &br = c->batch_rows;
+    br.n_seq = n_act;
+    for (int i = 0; i < n_act; i++) {
+        br.row0[i] = i * rows;
+        br.rows[i] = rows;
+        br.pos0[i] = (int)c->seqs[act[i]].tokens.size() - 1 + step;
+        br.table_off[i] = (int)((size_t)act[i] * table_len(&c->cfg));
+    }
+}
+
+// pages for `extra` more rows after the pending token of every active sequence
+int batch_ensure_pages(eesd_ctx *c, const int *act, int n_act, int extra) {
+    for (int i = 0; i < n_act; i++) {
+        select_seq(c, act[i]);
+        const int st = ensure_pages(c, (int)c->tokens.size() + extra);
+        park_seq(c, act[i]);
+        if (st) return st;
+    }
+    return EESD_OK;
+}
+
+// Draft step i of a round of draft length K on the active sequences (one row each): token
+// chain[a][i] at position T_a - 1 + i; logits into logits_q[a][i], chosen token into chain[a][i + 1]
+// (chain = ints + kRowTok, [n_act][K + 1]).  d_u: one uniform per sequence for this step.
+int run_batch_draft_step(eesd_ctx *c, const int *act, int n_act, int i, int K, const float *d_u) {
+    const eesd_config &f = c->cfg;
+    cudaStream_t s = c->stream;
+    const int L = f.n_layers, d = f.d_model, N = f.n_early;
+    int32_t *chain = c->ints + kRowTok;
+    batch_geometry(c, act, n_act, 1, i);
+    c->batch_cur = &c->batch_rows;
+    launch_embed(s, f.dtype, chain + i, c->embed, c->x, nullptr, n_act, d, f.vocab, c->err, K + 1);
+    run_resid(c, nullptr, c->layers[0].g_attn, nullptr, n_act);
+    for (int l = 0; l < N; l++)
+        run_layer(c, c->layers[l], l, n_act, 0, l + 1 < N ? c->layers[l + 1].g_attn : c->layers[L].g_attn, nullptr);
+    for (int e = 0; e < c->E; e++)
+        run_layer(c, c->layers[L + e], L + e, n_act, 0, e + 1 < c->E ? c->layers[L + e + 1].g_attn : c->g_exit, nullptr);
+    c->batch_cur = nullptr;
+    float *lq = c->logits_q + (size_t)i * f.vocab;   // row a of this step is row a * K + i of [n_act][K][V]
+    PartView pv = run_proj(c, c->exit_head, &c->m_exit_head, P_HEAD, X_NORM, n_act, f.vocab, d);
+    launch_reduce_partials(s, pv, norm_scale(c), lq, n_act, f.vocab, (size_t)K * f.vocab);
+    launch_sample_rows(s, lq, d_u, n_act, f.vocab, f.temperature, chain + i + 1, (size_t)K * f.vocab, K + 1);
+    c->launches += 3;
+    return check_launch(c);
+}
+
+// One round of the active sequences: K draft steps, one verification pass of K + 1 rows per
+// sequence, the acceptance step for all of them; the result (n_accept and next token per
+// sequence, the chains, the error word) is on its way to h_result when this returns.
+// h_result: [2] error word, [8..23] the chains, [32..39] n_accept, [40..47] next tokens.
+int batch_round(eesd_ctx *c, const int *act, int n_act, int K, const eesd_uniforms *u) {
+    const eesd_config &f = c->cfg;
+    const bool greedy = f.temperature == 0.f;
+    int32_t *chain = c->ints + kRowTok;
+    int st = batch_ensure_pages(c, act, n_act, K);
+    if (st) return st;
+    IntList16 first;   // the pending tokens: chain[a][0]
+    for (int i = 0; i < 16; i++) first.v[i] = 0;
+    for (int a = 0; a < n_act; a++) first.v[a * (K + 1)] = c->seqs[act[a]].tokens.back();
+    launch_set_ints(c->stream, chain, first, n_act * (K + 1));
+    c->launches++;
+    float *d_ud = c->u_stage, *d_ua = c->u_stage + 16, *d_ur = c->u_stage + 32;
+    if (!greedy) {   // this round's uniforms: draft [K][n_act], accept [n_act][K], resample [n_act]
+        float h[40];
+        for (int a = 0; a < n_act; a++) {
+            const int T = (int)c->seqs[act[a]].tokens.size();
+            for (int i = 0; i < K; i++) {
+                h[i * n_act + a] = u[act[a]].u_draft[T + i];
+                h[16 + a * K + i] = u[act[a]].u_accept[T + i];
+            }
+            h[32 + a] = u[act[a]].u_resample[T];
+        }
+        CU(c, cudaMemcpyAsync(c->u_stage, h, sizeof(h), cudaMemcpyHostToDevice, c->stream));
+    }
+    CU(c, cudaEventRecord(c->ev[2], c->stream));
+    for (int i = 0; i < K; i++) {
+        st = run_batch_draft_step(c, act, n_act, i, K, greedy ? nullptr : d_ud + i * n_act);
+        if (st) return st;
+    }
+    CU(c, cudaEventRecord(c->ev[3], c->stream));
+    batch_geometry(c, act, n_act, K + 1, 0);
+    c->batch_cur = &c->batch_rows;
+    st = run_target(c, chain, n_act * (K + 1), 0, true);
+    c->batch_cur = nullptr;
+    if (st) return st;
+    CU(c, cudaEventRecord(c->ev[5], c->stream));
+    launch_accept(c->stream, c->logits_p, c->logits_q, chain + 1, d_ua, d_ur, n_act, K, f.vocab, f.temperature, c->accept_scratch,
+                  c->ints + kResult, c->ints + kResult + kMaxSeqs, nullptr, K + 1);
+    CU(c, cudaEventRecord(c->ev[6], c->stream));
+    c->launches++;
+    st = check_launch(c);
+    if (st) return st;
+    CU(c, cudaMemcpyAsync(c->h_result + 32, c->ints + kResult, 2 * kMaxSeqs * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaMemcpyAsync(c->h_result + 8, chain, 16 * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaMemcpyAsync(c->h_result + 2, c->err, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaEventRecord(c->ev[4], c->stream));
+    return EESD_OK;
+}
+
 }  // namespace
 
 // =====================================================================================  C ABI
@@ -772,7 +915,8 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     c->x = (float *)(ws + w.x); c->x_save = (float *)(ws + w.x_save); c->xn = (float *)(ws + w.xn); c->attn = (float *)(ws + w.attn);
     c->h = (float *)(ws + w.h); c->part = (float *)(ws + w.part); c->apart = (float *)(ws + w.apart);
     c->logits_p = (float *)(ws + w.logits_p); c->logits_q = (float *)(ws + w.logits_q);
-    c->rope = (float2 *)(ws + w.rope); c->page_table = (int32_t *)(ws + w.page_table);
+    c->rope = (float2 *)(ws + w.rope); c->page_table = c->page_table0 = (int32_t *)(ws + w.page_table);
+    c->batch_cur = nullptr;
     c->ints = (int32_t *)(ws + w.ints); c->u_dev = (float *)(ws + w.u_dev); c->u_stage = (float *)(ws + w.u_stage);
     c->err = (int *)(ws + w.err); c->accept_scratch = ws + w.accept;
     c->ssq = (float *)(ws + w.ssq); c->tickets = (unsigned int *)(ws + w.tickets);
@@ -860,7 +1004,7 @@ int eesd_init(const eesd_config *cfg, const eesd_buffers *b, void *cuda_stream, 
     cudaMemsetAsync(c->err, 0, 16, c->stream);
     cudaMemsetAsync(c->tickets, 0, ticket_count(cfg) * 4, c->stream);
     cudaMemsetAsync(c->ints, 0, kIntSlots * 4, c->stream);
-    cudaMemsetAsync(c->accept_scratch, 0, accept_scratch_bytes(1, EESD_MAX_ROWS), c->stream);
+    cudaMemsetAsync(c->accept_scratch, 0, accept_scratch_bytes(kMaxSeqs, EESD_MAX_ROWS), c->stream);
     // The tensor-core attention multiplies cached values past the end of a slice by weights that are
     // exactly zero; that is only harmless while every value the pool ever holds is finite, so the pool
     // starts as zeros (afterwards only this library writes it).
@@ -893,6 +1037,7 @@ int eesd_reset(eesd_ctx *c) {
 
 int eesd_prefill(eesd_ctx *c, const int32_t *prompt, int n_prompt) {
     if (!c) return EESD_ERR_BADARG;
+    if (batch_on(c)) return EESD_ERR_STATE;   // the sequences of a batch are fed with eesd_batch_prefill
     int st = prefill_impl(c, prompt, n_prompt);
     if (st) return st;
     CU(c, cudaMemcpyAsync(c->h_result + 2, c->err, 4, cudaMemcpyDeviceToHost, c->stream));
@@ -1069,6 +1214,158 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
     return EESD_OK;
 }
 
+// ---- batch mode: several sequences decoded together (an extension; the paper's batch is 1) ----
+
+int eesd_batch_begin(eesd_ctx *c, int n_seq) {
+    if (!c || n_seq < 0 || n_seq > kMaxSeqs) return EESD_ERR_BADARG;
+    // the bf16-cache attention kernel is the one that knows about batches; trees and the per-sequence
+    // stopping rules of the controllers have no batch counterpart here
+    if (n_seq > 0 && (c->cfg.dtype != EESD_BF16 || tree_on(c))) return EESD_ERR_UNSUPPORTED;
+    if (batch_on(c)) {   // leave batch mode: give every sequence's pages back
+        for (size_t b = 0; b < c->seqs.size(); b++) {
+            select_seq(c, (int)b);
+            trim_pages(c, 0);
+            park_seq(c, (int)b);
+        }
+        c->seqs.clear();
+    }
+    reset_sequence(c);
+    c->page_table = c->page_table0;
+    c->seqs.resize((size_t)n_seq);
+    for (auto &q : c->seqs) q.prefilled = false;
+    return EESD_OK;
+}
+
+int eesd_batch_prefill(eesd_ctx *c, int seq, const int32_t *prompt, int n_prompt) {
+    if (!c || !batch_on(c) || seq < 0 || seq >= (int)c->seqs.size()) return EESD_ERR_BADARG;
+    select_seq(c, seq);
+    int st = prefill_impl(c, prompt, n_prompt);   // (resets the selected sequence first)
+    if (!st) {
+        cudaError_t e = cudaMemcpyAsync(c->h_result + 2, c->err, 4, cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+        st = e != cudaSuccess ? EESD_ERR_CUDA : read_error_word(c);
+    }
+    park_seq(c, seq);
+    return st;
+}
+
+int eesd_batch_context_len(const eesd_ctx *c, int seq, int *n_tokens, int *pages_in_use) {
+    if (!c || !batch_on(c) || seq < 0 || seq >= (int)c->seqs.size()) return EESD_ERR_BADARG;
+    if (n_tokens) *n_tokens = (int)c->seqs[seq].tokens.size();
+    if (pages_in_use) *pages_in_use = (int)c->seqs[seq].page_of.size();
+    return EESD_OK;
+}
+
+int eesd_batch_verify_only(eesd_ctx *c, const int32_t *tokens, int m) {
+    if (!c || !batch_on(c) || !tokens || m < 1) return EESD_ERR_BADARG;
+    const int B = (int)c->seqs.size();
+    if (B * m > EESD_MAX_ROWS) return EESD_ERR_BADARG;
+    int act[kMaxSeqs];
+    for (int b = 0; b < B; b++) {
+        if (!c->seqs[b].prefilled) return EESD_ERR_STATE;
+        if ((int)c->seqs[b].tokens.size() - 1 + m > c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
+        act[b] = b;
+    }
+    int st = batch_ensure_pages(c, act, B, m - 1);
+    if (st) return st;
+    st = set_device_ints(c, kRowTok, tokens, B * m);
+    if (st) return st;
+    batch_geometry(c, act, B, m, 0);
+    c->batch_cur = &c->batch_rows;
+    st = run_target(c, c->ints + kRowTok, B * m, 0, true);
+    c->batch_cur = nullptr;
+    return st;
+}
+
+int eesd_batch_decode(eesd_ctx *c, int max_new, const int32_t *k_schedule, int n_schedule, const eesd_uniforms *u,
+                      int32_t *out, eesd_stats *stats, eesd_round *trace, int trace_cap, int *n_rounds) {
+    if (!c || !batch_on(c) || !out || max_new < 1) return EESD_ERR_BADARG;
+    const eesd_config &f = c->cfg;
+    const int B = (int)c->seqs.size();
+    const bool greedy = f.temperature == 0.f;
+    int n0[kMaxSeqs], got[kMaxSeqs], rounds_of[kMaxSeqs];
+    for (int b = 0; b < B; b++) {
+        if (!c->seqs[b].prefilled) return EESD_ERR_STATE;
+        if (!greedy && (!u || !u[b].u_draft || !u[b].u_accept || !u[b].u_resample)) return EESD_ERR_RNG;
+        n0[b] = (int)c->seqs[b].tokens.size();
+        if (n0[b] + max_new + 1 > f.max_ctx) return EESD_ERR_CTX_FULL;
+        got[b] = 0;
+        rounds_of[b] = 0;
+    }
+    const host_clock::time_point wall0 = host_clock::now();
+    const int64_t launches0 = c->launches;
+    eesd_stats sacc;
+    memset(&sacc, 0, sizeof(sacc));
+    int rounds = 0;
+    for (;;) {
+        int act[kMaxSeqs], n_act = 0;   // sequences that still owe tokens
+        for (int b = 0; b < B; b++)
+            if (got[b] < max_new) act[n_act++] = b;
+        if (!n_act) break;
+        // one draft length for the whole round: the schedule's or the configured one, as far as the
+        // rows of a pass (n_act * (K + 1) <= 16), the round cap and every sequence's context allow
+        int K = (k_schedule && rounds < n_schedule) ? k_schedule[rounds] : f.fixed_k;
+        if (K > f.k_cap) K = f.k_cap;
+        if (K > EESD_MAX_ROWS / n_act - 1) K = EESD_MAX_ROWS / n_act - 1;
+        for (int a = 0; a < n_act; a++) {
+            const int room = f.max_ctx - 1 - (int)c->seqs[act[a]].tokens.size();
+            if (room < K) K = room;
+        }
+        if (K < 1) return EESD_ERR_CTX_FULL;
+        int st = batch_round(c, act, n_act, K, u);
+        if (st) return st;
+        CU(c, cudaStreamSynchronize(c->stream));
+        if (read_error_word(c)) {
+            snprintf(c->cuda_err, sizeof(c->cuda_err), "device error word 0x%x in a batch round", c->h_result[2]);
+            return EESD_ERR_DEVICE;
+        }
+        const int32_t *chain = c->h_result + 8, *n_acc = c->h_result + 32, *next = c->h_result + 32 + kMaxSeqs;
+        for (int a = 0; a < n_act; a++) {
+            const int b = act[a], acc = n_acc[a], y = next[a];
+            if (acc < 0 || acc > K || y < 0 || y >= f.vocab) {
+                snprintf(c->cuda_err, sizeof(c->cuda_err), "batch round result n_accept=%d next=%d (K=%d, sequence %d)", acc, y, K, b);
+                return EESD_ERR_DEVICE;
+            }
+            select_seq(c, b);
+            for (int i = 0; i < acc; i++) c->tokens.push_back(chain[a * (K + 1) + 1 + i]);
+            c->tokens.push_back(y);
+            trim_pages(c, (int)c->tokens.size() - 1);   // rows of rejected tokens are dropped
+            park_seq(c, b);
+            if (trace && rounds_of[b] < trace_cap) {
+                eesd_round &r = trace[(size_t)b * trace_cap + rounds_of[b]];
+                r.k = K; r.n_accept = acc; r.next_token = y;
+            }
+            rounds_of[b]++;
+            sacc.drafted += K;
+            sacc.accepted += acc < max_new - got[b] ? acc : max_new - got[b];
+            got[b] += acc + 1;
+        }
+        float ms_d = 0.f, ms_v = 0.f, ms_a = 0.f;
+        cudaEventElapsedTime(&ms_d, c->ev[2], c->ev[3]);
+        cudaEventElapsedTime(&ms_v, c->ev[3], c->ev[4]);
+        cudaEventElapsedTime(&ms_a, c->ev[5], c->ev[6]);
+        sacc.ms_draft += ms_d;
+        sacc.ms_verify += ms_v - ms_a;
+        sacc.ms_sampling += ms_a;
+        rounds++;
+    }
+    for (int b = 0; b < B; b++) {
+        for (int i = 0; i < max_new; i++) out[(size_t)b * max_new + i] = c->seqs[b].tokens[(size_t)n0[b] + i];
+        if (n_rounds) n_rounds[b] = rounds_of[b];
+    }
+    if (stats) {
+        sacc.rounds = rounds;
+        sacc.emitted = (int64_t)B * max_new;
+        sacc.ms_total = ms_since(wall0);
+        sacc.ms_other = sacc.ms_total - (sacc.ms_draft + sacc.ms_verify + sacc.ms_sampling);
+        sacc.kernel_launches = c->launches - launches0;
+        sacc.alpha = c->alpha;
+        sacc.beta = c->beta;
+        *stats = sacc;
+    }
+    return EESD_OK;
+}
+
 int eesd_decode(eesd_ctx *c, int max_new, const int32_t *k_schedule, int n_schedule, const eesd_uniforms *u,
                 int32_t *out, eesd_stats *stats, eesd_round *trace, int trace_cap, int *n_rounds) {
     if (!c || !out || max_new < 1) return EESD_ERR_BADARG;
@@ -1080,6 +1377,7 @@ int eesd_generate(eesd_ctx *c, const int32_t *prompt, int n_prompt, int max_new,
                   int n_schedule, const eesd_uniforms *u, int32_t *out, eesd_stats *stats, eesd_round *trace,
                   int trace_cap, int *n_rounds) {
     if (!c || !out || max_new < 1) return EESD_ERR_BADARG;
+    if (batch_on(c)) return EESD_ERR_STATE;
     if (n_prompt + max_new + 1 > c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
     const int64_t launches0 = c->launches;
     const host_clock::time_point wall0 = host_clock::now();
@@ -1217,8 +1515,25 @@ int eesd_posterior(const eesd_ctx *c, int64_t *alpha, int64_t *beta) {
     return EESD_OK;
 }
 
+int eesd_batch_assume_context(eesd_ctx *c, int seq, int n_ctx, int32_t pending) {
+    if (!c || !batch_on(c) || seq < 0 || seq >= (int)c->seqs.size()) return EESD_ERR_BADARG;
+    if (n_ctx < 1 || pending < 0 || pending >= c->cfg.vocab) return EESD_ERR_BADARG;
+    if (n_ctx >= c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
+    select_seq(c, seq);
+    trim_pages(c, 0);
+    int st = ensure_pages(c, n_ctx);
+    if (!st) {
+        c->tokens.assign(n_ctx, 0);
+        c->tokens[n_ctx - 1] = pending;
+        c->prefilled = true;
+    }
+    park_seq(c, seq);
+    return st;
+}
+
 int eesd_assume_context(eesd_ctx *c, int n_ctx, int32_t pending) {
     if (!c || n_ctx < 1 || pending < 0 || pending >= c->cfg.vocab) return EESD_ERR_BADARG;
+    if (batch_on(c)) return EESD_ERR_STATE;
     if (n_ctx >= c->cfg.max_ctx) return EESD_ERR_CTX_FULL;
     reset_sequence(c);
     int st = ensure_pages(c, n_ctx);

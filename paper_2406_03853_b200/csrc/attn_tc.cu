@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
                                                           float *__restrict__ apart, unsigned int *tickets,
                                                           float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
                                                           int M, int pos0, int H, int pps, int n_split, float scale2, int *err,
-                                                          TreeRows tr, uint32_t spin) {
+                                                          TreeRows tr, uint32_t spin, BatchRows br) {
     constexpr int HALF = D / 2;
     constexpr uint32_t LBO_C = Opnd<NC>::LBO;          // query / numerator operands
     constexpr uint32_t GRP = (D / 8) * 128;            // bytes of one 8-position group of a key / value tile
@@ -134,7 +134,8 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
     extern __shared__ __align__(128) unsigned char smem[];
     const int PT = kv.page_tokens, ptl = 31 - __clz(PT), group = H / kv.Hkv;
     const int cap = pps * PT;
-    const Smem lay = carve(cap, D, NC, n_split);
+    const int ns_stride = n_split;   // slices in the scratch layouts (batch mode: those of the longest sequence)
+    const Smem lay = carve(cap, D, NC, ns_stride);
     unsigned char *sK = smem + lay.k, *sV = smem + lay.v, *sQ = smem + lay.q, *sP = smem + lay.p;
     float *wgt = reinterpret_cast<float *>(smem + lay.wgt);       // [NC][n_split] merge weights
     float *s_mx = reinterpret_cast<float *>(smem + lay.red);      // [8][NC] per-warp column maxima
@@ -153,7 +154,19 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
-    const int bz = blockIdx.z;
+    // Batch mode: grid z runs over (sequence, column batch); a sequence is an independent problem with its
+    // own rows of the pass, positions, page table and slice count.
+    int bz = blockIdx.z, row_base = 0;
+    if (br.n_seq > 0) {
+        const int nbat = gridDim.z / br.n_seq, seq = blockIdx.z / nbat;
+        bz = blockIdx.z - seq * nbat;
+        M = br.rows[seq];
+        pos0 = br.pos0[seq];
+        row_base = br.row0[seq];
+        kv.page_table += br.table_off[seq];
+        n_split = (((pos0 + M + PT - 1) >> ptl) + pps - 1) / pps;
+        if (sp >= n_split || group * M <= bz * NC) return;   // a shorter sequence fills fewer slices and batches
+    }
     // per-slice (maximum, sum) pairs live behind the outputs: [H][16][kMaxSlices]
     float2 *ml = reinterpret_cast<float2 *>(apart + (size_t)H * kMaxSlices * kMaxRows * D);
     const int r0 = bz * NC;                  // first column ((head, row) pair) of this block's batch
@@ -237,7 +250,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
     pdl_wait();   // from here on the QKV projection's partial sums are read
     // One round of global loads: the RMSNorm statistics (threads 0..M-1) and the raw partial
     // sums of this block's queries and of the new keys / values that fall into its slice.
-    if (tid < M) s_rstd[tid] = row_rstd(rs, tid);
+    if (tid < M) s_rstd[tid] = row_rstd(rs, row_base + tid);
     float raw_a[kNewMax], raw_b[kNewMax];
     int new_page[kNewMax];
 #pragma unroll
@@ -248,7 +261,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
             const int pn = idx / D, w = idx - pn * D;
             new_page[it] = kv.page_table[(p_first + pn) >> ptl];
             const int isV = w >= HALF, i = isV ? w - HALF : w;
-            const float2 pr = gather_pair(p_first + pn - pos0, (H + (isV ? kv.Hkv : 0) + kh) * D + 2 * i);
+            const float2 pr = gather_pair(row_base + p_first + pn - pos0, (H + (isV ? kv.Hkv : 0) + kh) * D + 2 * i);
             raw_a[it] = pr.x;
             raw_b[it] = pr.y;
         }
@@ -260,7 +273,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
         const int idx = tid + it * THREADS;
         if (idx < n_q) {
             const int rl = idx / HALF, i = idx - rl * HALF;
-            const float2 pr = gather_pair(s_colm[rl], s_colh[rl] * D + 2 * i);
+            const float2 pr = gather_pair(row_base + s_colm[rl], s_colh[rl] * D + 2 * i);
             qraw_a[it] = pr.x;
             qraw_b[it] = pr.y;
         }
@@ -318,7 +331,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
                 const int page = new_page[it];
                 if (page < 0 || page >= kv.n_pages_total) { atomicOr(err, kErrBadPage); continue; }
                 bf16 *blk = (bf16 *)kv.slot_base + ((((size_t)page * 2 + isV) * kv.Hkv + kh) << ptl) * D;
-                const bool append = blockIdx.z == 0;   // every batch needs the row in its tile; one block writes the cache
+                const bool append = bz == 0;   // every batch needs the row in its tile; one block writes the cache
                 const int pp = pos & (PT - 1);
                 // a slice's pages sit one after the other in shared memory: token j of the slice is token j of one long block
                 if (isV) {
@@ -334,6 +347,16 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
                     *reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(sK) + k_index<bf16>(j, e, PT, D)) = w2;
                     if (append) *reinterpret_cast<uint32_t *>(blk + k_index<bf16>(pp, e, PT, D)) = w2;
                 }
+            }
+        }
+        // The output MMAs take the slice in steps of 16 positions.  With 8-token pages a slice may end on an odd
+        // page: the 8 positions after it were never copied, and their weights being zero does not help if the
+        // bytes there look like a NaN.  Clear those value rows (one 8-position group, contiguous).
+        {
+            const int loaded = (page_hi - page_lo) << ptl, need = ((npos + 15) >> 4) << 4;
+            if (loaded < need) {
+                uint4 *z = reinterpret_cast<uint4 *>(sV + (size_t)(loaded >> 3) * GRP);
+                for (int i = tid; i < (int)(((need - loaded) >> 3) * GRP / 16); i += THREADS) z[i] = make_uint4(0u, 0u, 0u, 0u);
             }
         }
         fence_async_smem();   // generic-proxy writes (queries, new rows) before the MMAs read them
@@ -449,7 +472,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
             for (int w = 0; w < 8; w++) l += s_sm[w * NC + c];
 #pragma unroll
             for (int w = 1; w < 8; w++) mx = fmaxf(mx, s_mx[w * NC + c]);
-            ml[((size_t)s_colh[c] * kMaxRows + s_colm[c]) * kMaxSlices + sp] = make_float2(mx, l);
+            ml[((size_t)s_colh[c] * kMaxRows + row_base + s_colm[c]) * kMaxSlices + sp] = make_float2(mx, l);
         }
         __syncwarp();
         mbar_wait(bar_o, 0, abort_flag, spin, 32);
@@ -469,7 +492,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
 #pragma unroll
                 for (int c = 0; c < HC; c++) {
                     if (c0 + c >= nb) break;
-                    apart[(((size_t)s_colh[c0 + c] * n_split + sp) * kMaxRows + s_colm[c0 + c]) * D + lane_id] =
+                    apart[(((size_t)s_colh[c0 + c] * ns_stride + sp) * kMaxRows + row_base + s_colm[c0 + c]) * D + lane_id] =
                         __uint_as_float(rl[c]) + __uint_as_float(rh[c]);
                 }
             }
@@ -492,7 +515,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
     }
     // ---- merge: the block that arrives last for this (KV head, batch) combines all slices
     if (tid == 0) {
-        unsigned int *tkt = tickets + (size_t)kh * gridDim.z + bz;   // one counter per (KV head, batch)
+        unsigned int *tkt = tickets + (size_t)kh * gridDim.z + blockIdx.z;   // one counter per (KV head, sequence, batch)
         const unsigned int prev = atomicAdd(tkt, 1u);
         *s_last = (prev == (unsigned int)n_split - 1);
         if (*s_last) *tkt = 0;
@@ -506,7 +529,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
     float4 pre[8];
     {
         const int rl = min(tid / (D / 4), nb - 1), dd = (tid % (D / 4)) * 4;
-        const float *src = apart + ((size_t)s_colh[rl] * n_split * kMaxRows + s_colm[rl]) * D + dd;
+        const float *src = apart + ((size_t)s_colh[rl] * ns_stride * kMaxRows + row_base + s_colm[rl]) * D + dd;
 #pragma unroll
         for (int u = 0; u < 8; u++)
             pre[u] = (tid < nb * (D / 4) && u < n_split) ? __ldcg(reinterpret_cast<const float4 *>(src + (size_t)u * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -518,7 +541,7 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
 #pragma unroll
         for (int i = 0; i < CPW; i++) {
             const int rl = min(warp + 8 * i, nb - 1);
-            const float2 *src = ml + ((size_t)s_colh[rl] * kMaxRows + s_colm[rl]) * kMaxSlices;
+            const float2 *src = ml + ((size_t)s_colh[rl] * kMaxRows + row_base + s_colm[rl]) * kMaxSlices;
             v0[i] = (warp + 8 * i < nb && lane < n_split) ? __ldcg(src + lane) : none;
             v1[i] = (warp + 8 * i < nb && lane + 32 < n_split) ? __ldcg(src + lane + 32) : none;
         }
@@ -537,8 +560,8 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
     __syncthreads();
     for (int idx = tid; idx < nb * (D / 4); idx += THREADS) {   // four output dimensions per item
         const int rl = idx / (D / 4), dd = (idx - rl * (D / 4)) * 4;
-        const int m = s_colm[rl], h = s_colh[rl];
-        const float *src = apart + ((size_t)h * n_split * kMaxRows + m) * D + dd;
+        const int m = row_base + s_colm[rl], h = s_colh[rl];   // row of the pass
+        const float *src = apart + ((size_t)h * ns_stride * kMaxRows + m) * D + dd;
         const float *wr = wgt + rl * n_split;
         float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int s2 = 0; s2 < n_split; s2 += 8) {   // eight slices in flight, added in slice order
@@ -571,15 +594,16 @@ __global__ void __launch_bounds__(THREADS) attn_tc_kernel(PartView pv, RowScale 
 template <int D, int NC, bool TR>
 static void launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv, float *apart,
                    unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H, int pps, int n_split,
-                   float scale, bool early, int *err, const TreeRows &tr, uint32_t wait_polls) {
+                   float scale, bool early, int *err, const TreeRows &tr, uint32_t wait_polls, const BatchRows &br) {
     const int rows = (H / kv.Hkv) * M, nbat = (rows + NC - 1) / NC;
     const Smem lay = carve(pps * kv.page_tokens, D, NC, n_split);
     // once per instantiation (thread-safe static initialisation)
     static const cudaError_t configured =
         cudaFuncSetAttribute(attn_tc_kernel<D, NC, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
     (void)configured;
-    launch_k(attn_tc_kernel<D, NC, TR>, dim3(kv.Hkv, n_split, nbat), dim3(THREADS), (size_t)lay.total, s, early && pdl_enabled(),
-             pv, rs, rope, kv, apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, tr, wait_polls);
+    launch_k(attn_tc_kernel<D, NC, TR>, dim3(kv.Hkv, n_split, nbat * (br.n_seq > 0 ? br.n_seq : 1)), dim3(THREADS), (size_t)lay.total, s,
+             early && pdl_enabled(), pv, rs, rope, kv, apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, tr,
+             wait_polls, br);
 }
 
 }  // namespace at
@@ -605,13 +629,15 @@ int attention_tc_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, in
 
 void launch_attention_tc(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv, float *apart,
                          unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H, int pps, int n_split,
-                         bool early, int *err, const TreeRows *tree, uint32_t wait_polls) {
+                         bool early, int *err, const TreeRows *tree, uint32_t wait_polls, const BatchRows *batch) {
     // queries are scaled by 1 / sqrt(D) and by log2 e: the softmax numerators are powers of two
     const float scale = 1.4426950408889634f / sqrtf((float)kv.D);
     const int rows = (H / kv.Hkv) * M;
     const TreeRows tr = tree ? *tree : chain_rows();
+    BatchRows br = {};
+    if (batch) br = *batch;
     const bool wide = attention_tc_columns(rows) == 32;
-#define EESD_AT(D, NC, TR) at::launch<D, NC, TR>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls)
+#define EESD_AT(D, NC, TR) at::launch<D, NC, TR>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls, br)
     if (kv.D == 64) {
         if (tree) { if (wide) EESD_AT(64, 32, true); else EESD_AT(64, 16, true); }
         else { if (wide) EESD_AT(64, 32, false); else EESD_AT(64, 16, false); }

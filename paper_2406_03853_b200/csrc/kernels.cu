@@ -45,11 +45,11 @@ void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float 
 
 // ------------------------------------------------------------------------------------ embedding gather
 template <typename WT>
-__global__ void embed_kernel(const int32_t *tok, const WT *E, float *x, float *cap, int d, int V, int *err) {
+__global__ void embed_kernel(const int32_t *tok, const WT *E, float *x, float *cap, int d, int V, int *err, int tok_stride) {
     const int m = blockIdx.x;
     pdl_trigger();
     pdl_wait();
-    int t = tok[m];
+    int t = tok[(size_t)m * tok_stride];
     if (t < 0 || t >= V) {
         if (threadIdx.x == 0) atomicOr(err, kErrBadToken);
         t = 0;
@@ -62,9 +62,9 @@ __global__ void embed_kernel(const int32_t *tok, const WT *E, float *x, float *c
     }
 }
 void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
-                  int M, int d, int V, int *err) {
-    if (dtype == 0) launch_k(embed_kernel<float>, dim3(M), dim3(256), 0, s, pdl_enabled(), tok, (const float *)E, x, cap, d, V, err);
-    else launch_k(embed_kernel<bf16>, dim3(M), dim3(256), 0, s, pdl_enabled(), tok, (const bf16 *)E, x, cap, d, V, err);
+                  int M, int d, int V, int *err, int tok_stride) {
+    if (dtype == 0) launch_k(embed_kernel<float>, dim3(M), dim3(256), 0, s, pdl_enabled(), tok, (const float *)E, x, cap, d, V, err, tok_stride);
+    else launch_k(embed_kernel<bf16>, dim3(M), dim3(256), 0, s, pdl_enabled(), tok, (const bf16 *)E, x, cap, d, V, err, tok_stride);
 }
 
 // ------------------------------------------------------------------------------------ residual + RMSNorm
@@ -194,14 +194,14 @@ int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float 
 // grid (heads, M), block D/2: one thread per rotation pair.
 template <typename AT>
 __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeom kv, const float2 *rope, float *q,
-                                int head_off, int col_off, int *err, TreeRows tr, int tree_on) {
+                                int head_off, int col_off, int *err, TreeRows tr, int tree_on, int row0) {
     const int hh = blockIdx.x + head_off;  // 0..H-1 q, H..H+Hkv-1 k, then v
-    const int m = blockIdx.y, i = threadIdx.x, D = kv.D;
+    const int m = blockIdx.y, i = threadIdx.x, D = kv.D;   // row row0 + m of the pass is position pos0 + m
     const int col = col_off + blockIdx.x * D + 2 * i;
     pdl_trigger();
     pdl_wait();
-    const float2 pr = part_gather_n<2>(pv, m, col);
-    const float rstd = row_rstd(rs, m);
+    const float2 pr = part_gather_n<2>(pv, row0 + m, col);
+    const float rstd = row_rstd(rs, row0 + m);
     float a = pr.x * rstd, b = pr.y * rstd;
     const int pos = pos0 + m;   // where the row is stored; a tree row is rotated as its depth's position
     if (hh < H + kv.Hkv) {
@@ -210,7 +210,7 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
         a = ra; b = rb;
     }
     if (hh < H) {
-        float *dst = q + (size_t)m * H * D + (size_t)hh * D + 2 * i;
+        float *dst = q + (size_t)(row0 + m) * H * D + (size_t)hh * D + 2 * i;
         dst[0] = a; dst[1] = b;
         return;
     }
@@ -232,13 +232,13 @@ __global__ void qkv_post_kernel(PartView pv, RowScale rs, int pos0, int H, KvGeo
 }
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
                      const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0,
-                     const TreeRows *tree) {
+                     const TreeRows *tree, int row0) {
     const int heads = only_kv ? 2 * kv.Hkv : H + 2 * kv.Hkv;
     dim3 grid(heads, M);
     const TreeRows tr = tree ? *tree : chain_rows();
     const int tree_on = tree && M <= 16 ? 1 : 0;
-    if (dtype == 0) launch_k(qkv_post_kernel<float>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on);
-    else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on);
+    if (dtype == 0) launch_k(qkv_post_kernel<float>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on, row0);
+    else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on, row0);
 }
 
 // ------------------------------------------------------------------------------------ paged decode attention, fp32 cache
@@ -714,8 +714,24 @@ int attention_max_ctx(int dtype, int page_tokens) {
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
                       int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err, const TreeRows *tree,
-                      uint32_t wait_polls) {
+                      uint32_t wait_polls, const BatchRows *batch) {
     int pps;
+    if (batch && batch->n_seq > 0) {   // several sequences: plan for the one with the most rows / the longest context
+        M = 0;
+        int ctx = 0;
+        for (int b = 0; b < batch->n_seq; b++) {
+            if (batch->rows[b] > M) M = batch->rows[b];
+            if (batch->pos0[b] + batch->rows[b] > ctx) ctx = batch->pos0[b] + batch->rows[b];
+        }
+        pos0 = ctx - M;
+        if (dtype == 0 || tree) {   // only the bf16-cache kernel knows about batches
+            const int e = kErrPlan;
+            cudaMemcpyAsync(err, &e, sizeof(e), cudaMemcpyHostToDevice, s);
+            return;
+        }
+    } else {
+        batch = nullptr;
+    }
     const int rows = (H / kv.Hkv) * M;
     auto refuse = [&](int n_split) {   // more slices than the merge can take: report, launch nothing
         if (n_split <= kMaxSlices && n_split <= max_splits) return false;
@@ -725,10 +741,11 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
     };
     if (dtype != 0) {   // bf16 cache: tensor-core kernel
         const int nc = attention_tc_columns(rows);
-        const int n_split = attention_tc_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + nc - 1) / nc, n_sm, max_splits, &pps);
+        const int n_split = attention_tc_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + nc - 1) / nc * (batch ? batch->n_seq : 1), n_sm,
+                                                max_splits, &pps);
         if (refuse(n_split)) return;
         launch_attention_tc(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, early, err, tree,
-                            wait_polls);
+                            wait_polls, batch);
         return;
     }
     const int rb = rows <= 8 ? 8 : rows <= kRows16 ? 16 : 32;
@@ -943,15 +960,16 @@ void launch_cali_theta(cudaStream_t s, const PartView &pv, const float *Wp, cons
     launch_k(cali_theta_kernel, dim3(1), dim3(256), 0, s, pdl_enabled(), pv, Wp, hD, d, theta);
 }
 
-__global__ void reduce_partials_kernel(PartView pv, RowScale rs, float *out, int R) {
+__global__ void reduce_partials_kernel(PartView pv, RowScale rs, float *out, int R, size_t out_stride) {
     const int m = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;
     pdl_trigger();
     pdl_wait();
     if (r >= R) return;
-    out[(size_t)m * R + r] = part_gather(pv, m, r) * row_rstd(rs, m);
+    out[(size_t)m * out_stride + r] = part_gather(pv, m, r) * row_rstd(rs, m);
 }
-void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R) {
-    launch_k(reduce_partials_kernel, dim3((R + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, out, R);
+void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R, size_t out_stride) {
+    launch_k(reduce_partials_kernel, dim3((R + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, out, R,
+             out_stride ? out_stride : (size_t)R);
 }
 
 }  // namespace eesd

@@ -63,6 +63,16 @@ struct TreeRows {
     uint16_t vis[16];
     uint8_t depth[16];
 };
+// Rows of a pass that belong to several sequences decoded together (batch mode; an extension, the
+// paper decodes one sequence at a time).  Sequence b owns rows row0[b] .. row0[b] + rows[b] - 1 of
+// the pass, at consecutive positions pos0[b] .. of its own context, whose page table starts
+// table_off[b] entries into the page-table array.  n_seq == 0: one sequence (the launcher's own
+// M, pos0 and page table apply).
+constexpr int kMaxSeqs = 8;
+struct BatchRows {
+    int n_seq;
+    int row0[kMaxSeqs], rows[kMaxSeqs], pos0[kMaxSeqs], table_off[kMaxSeqs];
+};
 inline TreeRows chain_rows() {
     TreeRows t;
     for (int m = 0; m < 16; m++) { t.vis[m] = (uint16_t)((2u << m) - 1u); t.depth[m] = (uint8_t)m; }
@@ -71,8 +81,9 @@ inline TreeRows chain_rows() {
 
 void launch_set_ints(cudaStream_t s, int32_t *dst, const IntList16 &vals, int n);
 void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float theta);
+// row m takes token tok[m * tok_stride]
 void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
-                  int M, int d, int V, int *err);
+                  int M, int d, int V, int *err, int tok_stride = 1);
 // x[m] += partial sums (if pv); y = x[m] * g -> xn (fp32, may be null) and xs (two bf16 terms,
 // [chunk of 16 rows][hi | lo][16][d], may be null); ssq[m][b] = sum of squares of block b (1024
 // columns) of x[m]; cap[m] = x[m] (if cap).  The RMSNorm scale itself is applied by the consumers.
@@ -85,19 +96,21 @@ int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float 
 // tree (optional, M <= 16): row m is rotated as position pos0 + depth[m] and stored at pos0 + m.
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
                      const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0 = 0,
-                     const TreeRows *tree = nullptr);
+                     const TreeRows *tree = nullptr, int row0 = 0);
 // Fused attention step of one layer on M new rows: q/k/v of the new rows are taken from the
 // QKV projection's partial sums (scaled by rs, rotated), the new keys/values are appended to
 // the paged cache, every KV head's cached slice is read once, and the slices are merged into
 // attn_out (fp32 [M][H*D], may be null) and attn_split (two bf16 terms, may be null).
 // apart: H * max_splits * 16 * (D + 2) floats; tickets: zero-initialised counters, one per
 // (KV head, batch of 32 (head, row) pairs): at most H_kv * 4.
+// batch (optional, bf16 cache only, no tree): the rows belong to several sequences; M, pos0 and kv.page_table
+// are then taken per sequence from it, and `M` is the largest row count of a sequence.
 // early: the kernel may start (and read cached rows) while the kernel before it still runs;
 // must be false when that kernel appends rows to the same cache slot.
 void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, const float2 *rope,
                       const KvGeom &kv, float *apart, unsigned int *tickets, float *attn_out, void *attn_split,
                       int M, int pos0, int H, int n_sm, int max_splits, bool early, int *err,
-                      const TreeRows *tree, uint32_t wait_polls);
+                      const TreeRows *tree, uint32_t wait_polls, const BatchRows *batch = nullptr);
 // most context tokens the attention kernel of `dtype` can serve with pages of page_tokens
 int attention_max_ctx(int dtype, int page_tokens);
 // tensor-core attention (attn_tc.cu; bf16 cache): columns ((head, row) pairs) per block for `rows` pairs per KV head,
@@ -106,7 +119,7 @@ int attention_tc_columns(int rows);
 int attention_tc_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out);
 void launch_attention_tc(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv, float *apart,
                          unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H, int pps, int n_split,
-                         bool early, int *err, const TreeRows *tree, uint32_t wait_polls);
+                         bool early, int *err, const TreeRows *tree, uint32_t wait_polls, const BatchRows *batch = nullptr);
 int attention_splits(int ctx_len, int page_tokens, int Hkv, int n_batches, int n_sm, int max_splits, int *pps_out);
 // Causal prompt attention (attn_prompt.cu; bf16 cache, D = 64 or 128): Mtot rows at positions pos0.., 128 rows per
 // block; the rows' keys / values must be in the cache already (launch_qkv_post with only_kv on the QKV
@@ -135,7 +148,8 @@ void launch_tree_walk(cudaStream_t s, const int32_t *top, int32_t *chain, const 
 void launch_kv_move(cudaStream_t s, int dtype, const KvGeom &kv0, size_t slot_bytes, int slots, int pos0,
                     const int32_t *result, int *err);
 void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F);
-void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R);
+// out_stride: floats between consecutive output rows (0: R)
+void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R, size_t out_stride = 0);
 // programmatic dependent launch (kernels start early and wait on-device for their producer):
 // on by default, off when the environment variable EESD_NO_PDL is set
 bool pdl_enabled();
@@ -163,8 +177,9 @@ void launch_split_rows(cudaStream_t s, const float *x, void *xs, int M, int K);
 size_t accept_scratch_bytes(int B, int K);
 void launch_accept(cudaStream_t s, const float *p_logits, const float *q_logits, const int32_t *tokens,
                    const float *u_acc, const float *u_res, int B, int K, int V, float T, void *scratch,
-                   int32_t *n_acc, int32_t *y, int32_t *pending_out);
+                   int32_t *n_acc, int32_t *y, int32_t *pending_out, int tok_stride = 0);   // tok_stride: ints between the sequences' token lists (0: K)
+// logit_stride: floats between rows (0: V); out_stride: ints between results
 void launch_sample_rows(cudaStream_t s, const float *logits, const float *u, int B, int V, float T,
-                        int32_t *out);
+                        int32_t *out, size_t logit_stride = 0, int out_stride = 1);
 
 }  // namespace eesd

@@ -1,0 +1,111 @@
+"""Batch mode: several sequences share the rows of every pass.
+
+Drafting, verification and acceptance of a sequence never look at another sequence (Algorithm 1),
+so per sequence the batch must give what the CPU oracle gives for that sequence alone: logits of
+a batched verification pass row by row against the oracle, and whole generations (tokens and the
+per-round trace) against single-sequence decoding with the draft lengths the batch used and the
+same uniforms."""
+import numpy as np
+import pytest
+import torch
+
+import eesd_synth as synth
+from tests.helpers import engine_from_spec, oracle_from_spec
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+BASE = synth.TINY.with_(dtype="bf16", ffn_dim=640)          # every projection tile-aligned: the tensor-core kernels
+SPECS = {"mha": BASE, "gqa8": BASE.with_(n_heads=8, n_kv_heads=1, head_dim=64, n_layers=2),
+         "wide_head": BASE.with_(n_heads=2, n_kv_heads=1, head_dim=128, n_layers=2)}
+
+
+@pytest.mark.parametrize("variant,lens,m,pt,max_ctx", [
+    ("mha", (37, 16, 5), 5, 16, 96),            # three sequences, one ending on a page boundary, 15 rows
+    ("mha", (9, 3, 30, 17, 2, 8, 33, 1), 2, 8, 64),   # eight sequences of two rows (a one-token prompt among them)
+    ("gqa8", (40, 23), 8, 16, 96),              # 64 (head, row) pairs per sequence: two column batches each
+    ("wide_head", (300, 150, 2), 4, 16, 384),   # contexts of very different length: 1 to several slices per sequence
+    ("mha", (200, 90), 3, 128, 384),            # one page holds the whole context
+])
+def test_batched_verification_pass_matches_the_oracle_row_by_row(variant, lens, m, pt, max_ctx):
+    spec = SPECS[variant]
+    B = len(lens)
+    eng = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, page_tokens=pt, kv_pages=B * (max_ctx // pt))   # one pool for all
+    eng.batch_begin(B)
+    prompts = [synth.prompt_tokens(40 + b, n, spec.vocab).numpy() for b, n in enumerate(lens)]
+    for b, p in enumerate(prompts):
+        eng.batch_prefill(b, p)
+    rows = np.stack([np.concatenate([p[-1:], synth.prompt_tokens(70 + b, m - 1, spec.vocab).numpy()]) for b, p in enumerate(prompts)])
+    eng.batch_verify_only(rows.astype(np.int32))
+    torch.cuda.synchronize()
+    got = eng.logits(0, B * m).cpu().numpy().reshape(B, m, spec.vocab)
+    for b, p in enumerate(prompts):
+        o = oracle_from_spec(spec, max_ctx)
+        if len(p) > 1:
+            o.target_rows(p[:-1], 0, want_logits=False)
+        _, lg = o.target_rows(rows[b].astype(np.int32), len(p) - 1)
+        err = np.abs(got[b] - lg).max()
+        assert err < TOL, (b, err)
+        n_tok, pages = eng.batch_context_len(b)
+        assert n_tok == len(p) and pages == (len(p) - 1 + m + pt - 1) // pt
+    eng.batch_begin(0)
+    assert eng.context_len() == (0, 0)
+    eng.close()
+
+
+@pytest.mark.parametrize("temperature", [0.0, 1.0])
+@pytest.mark.parametrize("variant,lens", [("mha", (21, 40, 7)), ("gqa8", (12, 33, 5, 18, 26))])
+def test_batch_decode_equals_single_sequence_decoding(variant, lens, temperature):
+    spec = SPECS[variant]
+    max_new, max_ctx = 40, 128
+    B = len(lens)
+    eng = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, temperature=temperature, page_tokens=16, kv_pages=B * 8)
+    prompts = [synth.prompt_tokens(90 + b, n, spec.vocab).numpy() for b, n in enumerate(lens)]
+    unis = [{k: v.numpy() for k, v in synth.generate_uniforms(max_ctx, 64, seed=300 + b).items()} for b in range(B)]
+    eng.batch_begin(B)
+    for b, p in enumerate(prompts):
+        eng.batch_prefill(b, p)
+    schedule = [3, 1, 7, 2, 4, 4, 1, 5] * 6
+    out, traces, st = eng.batch_decode(max_new, k_schedule=schedule, uniforms=unis if temperature else None)
+    for b in range(B):
+        n_tok, pages = eng.batch_context_len(b)
+        assert n_tok == lens[b] + sum(a + 1 for _, a, _ in traces[b]) and pages == (n_tok - 1 + 15) // 16
+        assert all(k * len(lens) <= 16 for k, _, _ in traces[b][:1])     # the first round holds every sequence
+    assert st.emitted == B * max_new and st.drafted == sum(k for t in traces for k, _, _ in t)
+    eng.batch_begin(0)
+    # the same sequences one at a time, with the draft lengths the batch used for each
+    for b, p in enumerate(prompts):
+        ks = [k for k, _, _ in traces[b]]
+        ref, rtrace, _ = eng.generate(p, max_new, k_schedule=ks + [3] * 8, uniforms=unis[b] if temperature else None)
+        np.testing.assert_array_equal(out[b], ref)
+        assert traces[b] == rtrace[:len(traces[b])]
+    eng.close()
+
+
+def test_batch_mode_errors():
+    from paper_2406_03853_b200 import EesdError
+    f32 = engine_from_spec(synth.TINY, max_ctx=64)
+    with pytest.raises(EesdError) as e:
+        f32.batch_begin(2)                                  # fp32 cache: the SIMT attention kernel has no batch form
+    assert e.value.status == -8
+    f32.close()
+    eng = engine_from_spec(BASE, max_ctx=64, page_tokens=16, kv_pages=8)
+    with pytest.raises(EesdError):
+        eng.batch_begin(9)
+    eng.batch_begin(2)
+    p = synth.prompt_tokens(1, 9, BASE.vocab).numpy()
+    with pytest.raises(EesdError) as e:
+        eng.prefill(p)                                      # single-sequence calls are closed while the batch is open
+    assert e.value.status == -4
+    eng.batch_prefill(0, p)
+    with pytest.raises(EesdError) as e:
+        eng.batch_decode(8)                                 # sequence 1 has no prompt
+    assert e.value.status == -4
+    with pytest.raises(EesdError):
+        eng.batch_prefill(2, p)
+    eng.batch_prefill(1, p[:4])
+    out, traces, _ = eng.batch_decode(8)
+    assert out.shape == (2, 8)
+    eng.batch_begin(0)
+    out1, _, _ = eng.generate(p, 8)                         # and open again afterwards
+    np.testing.assert_array_equal(out1, out[0])
+    eng.close()
