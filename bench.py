@@ -108,11 +108,14 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None, cali=False, tree_width=0, n_exit=1):
+def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_early=None, cali=False, tree_width=0, n_exit=1,
+                 spec_edit=None, kv_seqs=1):
     from paper_2406_03853_b200 import Engine
     from paper_2406_03853_b200 import binding as b
     spec_name, n_prompt, max_new, damp, _ = WORKLOADS[wl]
     spec = synth.SPECS[spec_name].with_(damp=damp if alpha is None else alpha)
+    if spec_edit:
+        spec = spec.with_(**spec_edit)
     if n_early:
         spec = spec.with_(n_early=n_early)
     if n_layers:
@@ -124,7 +127,8 @@ def build_engine(wl, temperature, controller, device, n_layers=0, alpha=None, n_
                         k_cap=10 if tree_width < 2 else 15 // tree_width,
                         temperature=temperature, controller=b.CTRL_CALI_TS if cali else controller, fixed_k=5, page_tokens=16,
                         tree_width=tree_width, n_exit_layers=n_exit)
-    eng = Engine(cfg, device=device)
+    # (kv_seqs > 1: one page pool that holds that many sequences, for batch mode)
+    eng = Engine(cfg, device=device, kv_pages=None if kv_seqs == 1 else kv_seqs * (max_ctx // 16 + 2))
     # synthetic weights, generated on the device by the shared seeded generator
     for l in range(spec.n_layers):
         v = eng.layer_views(l)
@@ -408,6 +412,35 @@ def run_sweep(args, device):
             eng.close()
             del eng
             torch.cuda.empty_cache()
+    elif args.sweep == "batch":
+        # Several sequences sharing every pass (an extension: the paper's batch is 1).  The rows of a pass are capped
+        # at 16, so more sequences mean shorter drafts: B x (K + 1) <= 16.  One JSON line per (B, K): tokens/s summed
+        # over the sequences, against single-sequence decoding with the same fixed draft length.
+        edit = {"dtype": "bf16", "ffn_dim": 640} if synth.SPECS[spec_name].dtype == "f32" else None   # batch mode is bf16 only
+        eng, spec, _, _ = build_engine(args.workload, args.temperature, b.CTRL_FIXED_K, device, alpha=args.alpha, spec_edit=edit, kv_seqs=8)
+        u = [{k: v.numpy() for k, v in synth.generate_uniforms(eng.cfg.max_ctx, 64, seed=synth.SEED + 50 + i).items()} for i in range(8)]
+        for B, K in ((1, 3), (1, 1), (2, 3), (2, 7), (4, 3), (4, 1), (8, 1)):
+            ms, tot = 0.0, {"drafted": 0, "accepted": 0, "emitted": 0, "rounds": 0}
+            for i in range(args.steps):
+                eng.batch_begin(B)
+                for q in range(B):
+                    eng.batch_prefill(q, synth.prompt_tokens(synth.SEED + 8 * i + q, n_prompt, spec.vocab).numpy())
+                torch.cuda.synchronize()
+                e0.record()
+                _, _, st = eng.batch_decode(max_new, k_schedule=[K] * (4 * max_new), uniforms=u[:B] if args.temperature else None)
+                e1.record()
+                torch.cuda.synchronize()
+                ms += e0.elapsed_time(e1)
+                for k in tot:
+                    tot[k] += st.as_dict()[k]
+            eng.batch_begin(0)
+            q = report.run_quality(tot["drafted"], tot["accepted"], tot["emitted"])
+            print(json.dumps({"sweep": "batch", "setting": f"B={B}, K={K}", "workload": args.workload, "sequences": B, "k": K,
+                              "rows_per_verify_pass": B * (K + 1), "tokens_per_s": round(args.steps * B * max_new / (ms / 1e3), 2),
+                              "tokens_per_s_per_sequence": round(args.steps * max_new / (ms / 1e3), 2),
+                              "v_d": round(q["v_d"], 4), "r_d": round(q["r_d"], 4), "batch_rounds": tot["rounds"],
+                              "steps": args.steps}), flush=True)
+        eng.close()
     elif args.sweep == "exit":
         # the paper's experiment on the number of early-exit layers: a deeper draft head accepts more and costs more
         for E in (1, 2, 3):
@@ -524,9 +557,9 @@ def main():
                          "bracket, for ncu --profile-from-start off")
     ap.add_argument("--controller", choices=["beta", "cali"], default="beta",
                     help="draft-length controller: Beta-TS (default) or TS with calibration (random-init predictor)")
-    ap.add_argument("--sweep", choices=["k", "n", "tree", "exit"], default=None,
+    ap.add_argument("--sweep", choices=["k", "n", "tree", "exit", "batch"], default=None,
                     help="method sweep instead of the benchmark line: fixed K = 1..10 against Beta-TS, the exit depth N, "
-                         "tree verification widths, or the number of early-exit layers")
+                         "tree verification widths, the number of early-exit layers, or the number of sequences decoded together")
     ap.add_argument("--profile-prefill", action="store_true",
                     help="only run one prompt pass inside a cudaProfilerStart/Stop region (for ncu)")
     ap.add_argument("--profile-tree", type=int, default=0, metavar="W",
@@ -694,7 +727,8 @@ def main():
         torch.cuda.empty_cache()
         tv, outs = {}, {}
         for W in (1, 2):
-            eng_t, _, _, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, alpha=args.alpha, tree_width=W)
+            eng_t, _, _, _ = build_engine(args.workload, 0.0, b.CTRL_FIXED_K, device, alpha=args.alpha, tree_width=W,
+                                          kv_seqs=4 if W == 1 else 1)
             ms_t, tot = 0.0, {"drafted": 0, "accepted": 0, "rounds": 0, "leaves_kept": 0}
             for i in range(args.steps):
                 eng_t.prefill(prompts[i])
@@ -711,6 +745,25 @@ def main():
                 "tokens_per_s": round(args.steps * max_new / (ms_t * 1e-3), 2),
                 "v_d": round(tot["accepted"] / max(1, tot["drafted"]), 4),
                 "leaves_kept_per_round": round(tot["leaves_kept"] / max(1, tot["rounds"]), 4)}
+            if W == 1 and spec.dtype == "bf16" and args.steps >= 4:
+                # batch mode (an extension: the paper's batch is 1): the first four prompts decoded together, three
+                # drafts per round (16 rows per verification pass), against the same prompts decoded one by one above
+                for timed in (False, True):   # once untimed: the first launches of the batched kernels load them
+                    eng_t.batch_begin(4)
+                    for q in range(4):
+                        eng_t.batch_prefill(q, prompts[q])
+                    if not timed:
+                        eng_t.batch_decode(8, k_schedule=[3] * 32)
+                torch.cuda.synchronize()
+                e0.record()
+                out_b, _, st_b = eng_t.batch_decode(max_new, k_schedule=[3] * (4 * max_new))
+                e1.record()
+                torch.cuda.synchronize()
+                eng_t.batch_begin(0)
+                line["batch_decode"] = {"sequences": 4, "k": 3, "rows_per_verify_pass": 16,
+                                        "tokens_per_s": round(4 * max_new / (e0.elapsed_time(e1) * 1e-3), 2),
+                                        "v_d": round(st_b.accepted / max(1, st_b.drafted), 4),
+                                        "same_tokens_as_one_by_one": all((out_b[q] == outs[1][q]).all() for q in range(4))}
             eng_t.close()
             del eng_t
             torch.cuda.empty_cache()

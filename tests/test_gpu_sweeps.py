@@ -51,3 +51,14 @@ def test_tree_width_sweep():
     wide = [r for r in rows if r["setting"].startswith("width 2,")]
     assert all(r["leaves_kept_per_round"] == 0.0 for r in chain)
     assert any(r["leaves_kept_per_round"] > 0.0 for r in wide)          # the second-best candidate is the target's choice now and then
+
+
+def test_batch_sweep():
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--sweep", "batch", "--workload", "tiny-eesd", "--steps", "1"],
+                       capture_output=True, text=True, timeout=900, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    rows = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert [(x["sequences"], x["k"]) for x in rows] == [(1, 3), (1, 1), (2, 3), (2, 7), (4, 3), (4, 1), (8, 1)]
+    for x in rows:
+        assert x["rows_per_verify_pass"] <= 16 and x["tokens_per_s"] > 0 and 0.0 <= x["v_d"] <= 1.0
+        assert abs(x["tokens_per_s"] - x["sequences"] * x["tokens_per_s_per_sequence"]) < 0.02 * x["tokens_per_s"]
