@@ -413,7 +413,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
         if (idx < n_new) {
             const int pn = idx / D, w = idx - pn * D;
             const int pos = p_first + pn, m = pos - pos0;
-            const int isV = w >= HALF, i = isV ? w - HALF : w;
+            const int isV = w >= HALF;
             float a = raw_a[it] * s_rstd[m], b = raw_b[it] * s_rstd[m];
             if (!isV) {
                 const float2 cs = cs_new[it];
