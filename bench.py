@@ -549,6 +549,7 @@ def main():
                     help="scale of the upper layers' output projections (draft/target agreement): 0.05 high, "
                          "0.2 medium (default), 0.5 low acceptance")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the temperature-1 / lower-agreement legs")
     ap.add_argument("--no-tree", action="store_true", help="skip the tree-verification leg of the default run")
     ap.add_argument("--no-70b", action="store_true",
                     help="skip the LLaMA-2-70B-shaped leg of the default run (verify passes and a short decode; about a minute)")
@@ -770,6 +771,32 @@ def main():
         # greedy decoding is lossless either way: both runs must have emitted the same tokens
         tv["same_tokens_as_chain"] = all((a == c).all() for a, c in zip(outs[2], outs[1]))
         line["tree_verification"] = tv
+    if world == 1 and greedy and args.controller == "beta" and not args.no_variants and args.alpha is None:
+        # the same workload at temperature 1 (stochastic acceptance and residual resampling on the device) and with
+        # less agreement between draft and target (output projections of the upper layers scaled by 0.2 and 0.5
+        # instead of 0.05): two prompts each, Beta-TS
+        torch.cuda.empty_cache()
+        var = {}
+        for label, alpha_v, temp_v in (("temperature_1", None, 1.0), ("alpha_0.2", 0.2, 0.0), ("alpha_0.5", 0.5, 0.0)):
+            eng_v, _, _, _ = build_engine(args.workload, temp_v, b.CTRL_BETA_TS, device, alpha=alpha_v)
+            ms_v, tot = 0.0, {"drafted": 0, "accepted": 0, "emitted": 0, "rounds": 0}
+            for i in range(min(2, args.steps)):
+                eng_v.prefill(prompts[i])
+                torch.cuda.synchronize()
+                e0.record()
+                _, _, st_v = eng_v.decode(max_new, uniforms=u)
+                e1.record()
+                torch.cuda.synchronize()
+                ms_v += e0.elapsed_time(e1)
+                for k in tot:
+                    tot[k] += st_v.as_dict()[k]
+            qv = report.run_quality(tot["drafted"], tot["accepted"], tot["emitted"])
+            var[label] = {"tokens_per_s": round(tot["emitted"] / (ms_v * 1e-3), 2), "v_d": round(qv["v_d"], 4), "r_d": round(qv["r_d"], 4),
+                          "mean_k": round(tot["drafted"] / max(1, tot["rounds"]), 3), "prompts": min(2, args.steps)}
+            eng_v.close()
+            del eng_v
+            torch.cuda.empty_cache()
+        line["variants"] = var
     if world == 1 and greedy and args.controller == "beta" and not args.no_70b and args.workload == "13b-eesd":
         line["shape_70b"] = leg_70b(device, peaks)
         line["verify_pass_frac_of_8tbs"]["70b"] = {k: v["frac_of_8tbs"] for k, v in line["shape_70b"]["verify_pass"].items()
