@@ -35,13 +35,25 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// the same test, but the thread may be parked by the hardware for up to about `ns` nanoseconds while the
+// phase is incomplete (fewer polls for the same bound in time)
+__device__ __forceinline__ bool mbar_try_parked(uint64_t *bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
 // bounded wait: at most `limit` polls; false (and the abort flag set) when the limit is reached
 // or another role of the CTA gave up
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t limit,
                                           uint32_t sleep_ns = 0) {
     for (uint32_t i = 0; i < limit; i++) {
-        if (mbar_try(bar, parity)) return true;   // non-blocking poll
-        if (sleep_ns) __nanosleep(sleep_ns);
+        if (mbar_try_parked(bar, parity, 200u)) return true;   // parked by the hardware for at most about 200 ns per poll
         if ((i & 1023u) == 1023u && *abort_flag) return false;
     }
     *abort_flag = 1;
