@@ -125,28 +125,61 @@ __global__ void __launch_bounds__(THREADS, 1) attn_prompt_kernel(PartView pv, Ro
         n_k[0]++;
     }
 
-    // ---- queries: item = (row, 8 consecutive dimensions); consecutive lanes take consecutive rows
-    for (int idx = tid; idx < QT * (D / 8); idx += THREADS) {
-        const int row = idx & (QT - 1), c = idx >> 7;
-        uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
-        if (row < n_rows) {
-            const int m = r0 + row;
-            float4 a = part_gather_n<4>(pv, m, h * D + 8 * c), b = part_gather_n<4>(pv, m, h * D + 8 * c + 4);
-            const float2 *cs = rope + (size_t)(pos0 + m) * HALF + 4 * c;
-            const float r = s_rstd[row];
-            const float raw[8] = {a.x * r, a.y * r, a.z * r, a.w * r, b.x * r, b.y * r, b.z * r, b.w * r};
-            float q[8];
+    // ---- queries: item = (row, 8 consecutive dimensions); consecutive lanes take consecutive rows.  Four items at a
+    // time, all their loads requested before the first is used (pv is a plain [split][row][column] result here).
+    constexpr int QI = QT * (D / 8) / THREADS, QB = 4;
+#pragma unroll 1
+    for (int g = 0; g < QI; g += QB) {
+        float4 a[QB], b[QB], w0[QB], w1[QB];
 #pragma unroll
-            for (int i = 0; i < 4; i++) {
-                const float2 w = cs[i];
-                q[2 * i] = (raw[2 * i] * w.x - raw[2 * i + 1] * w.y) * scale2;
-                q[2 * i + 1] = (raw[2 * i] * w.y + raw[2 * i + 1] * w.x) * scale2;
+        for (int k = 0; k < QB; k++) {
+            const int idx = tid + (g + k) * THREADS, row = idx & (QT - 1), c = idx >> 7;
+            a[k] = b[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            w0[k] = w1[k] = make_float4(1.f, 0.f, 1.f, 0.f);
+            if (row < n_rows) {
+                const float4 *cs = reinterpret_cast<const float4 *>(rope + (size_t)(pos0 + r0 + row) * HALF + 4 * c);
+                w0[k] = cs[0];
+                w1[k] = cs[1];
             }
-            split8(q, hi, lo);
         }
-        unsigned char *dst = sQ + (uint32_t)c * ROWS_LBO + (uint32_t)row * 16;   // (row / 8) * 128 + (row % 8) * 16
-        *reinterpret_cast<uint4 *>(dst) = hi;
-        *reinterpret_cast<uint4 *>(dst + Q_BYTES) = lo;
+        for (int sp = 0; sp < pv.S; sp++) {   // the k-range splits of the projection, added in order
+            float4 la[QB], lb[QB];
+#pragma unroll
+            for (int k = 0; k < QB; k++) {
+                const int idx = tid + (g + k) * THREADS, row = idx & (QT - 1), c = idx >> 7;
+                la[k] = lb[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (row < n_rows) {
+                    const float4 *src = reinterpret_cast<const float4 *>(pv.base + (size_t)sp * pv.split_stride + (size_t)(r0 + row) * pv.R + h * D + 8 * c);
+                    la[k] = src[0];
+                    lb[k] = src[1];
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < QB; k++) {
+                a[k].x += la[k].x; a[k].y += la[k].y; a[k].z += la[k].z; a[k].w += la[k].w;
+                b[k].x += lb[k].x; b[k].y += lb[k].y; b[k].z += lb[k].z; b[k].w += lb[k].w;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < QB; k++) {
+            const int idx = tid + (g + k) * THREADS, row = idx & (QT - 1), c = idx >> 7;
+            uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
+            if (row < n_rows) {
+                const float r = s_rstd[row];
+                const float raw[8] = {a[k].x * r, a[k].y * r, a[k].z * r, a[k].w * r, b[k].x * r, b[k].y * r, b[k].z * r, b[k].w * r};
+                const float cw[8] = {w0[k].x, w0[k].y, w0[k].z, w0[k].w, w1[k].x, w1[k].y, w1[k].z, w1[k].w};   // (cos, sin) of four pairs
+                float q[8];
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    q[2 * i] = (raw[2 * i] * cw[2 * i] - raw[2 * i + 1] * cw[2 * i + 1]) * scale2;
+                    q[2 * i + 1] = (raw[2 * i] * cw[2 * i + 1] + raw[2 * i + 1] * cw[2 * i]) * scale2;
+                }
+                split8(q, hi, lo);
+            }
+            unsigned char *dst = sQ + (uint32_t)c * ROWS_LBO + (uint32_t)row * 16;   // (row / 8) * 128 + (row % 8) * 16
+            *reinterpret_cast<uint4 *>(dst) = hi;
+            *reinterpret_cast<uint4 *>(dst + Q_BYTES) = lo;
+        }
     }
     fence_async_smem();
     __syncthreads();
