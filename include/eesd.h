@@ -349,7 +349,7 @@ int eesd_clear_device_error(eesd_ctx *ctx);
  * no batch counterpart and is not consulted.  Per sequence the result is what single-sequence
  * decoding with the same draft lengths and the same uniforms gives (Algorithm 1: drafting,
  * verification and acceptance of a sequence never look at another sequence).
- * bf16 models only (UNSUPPORTED otherwise, and with tree verification).  While batch mode is on,
+ * Not with tree verification (UNSUPPORTED).  While batch mode is on,
  * the single-sequence calls that start or feed a sequence return STATE. */
 #define EESD_MAX_BATCH 8
 /* Enters batch mode with n_seq empty sequences (1..EESD_MAX_BATCH), or leaves it (n_seq = 0); either

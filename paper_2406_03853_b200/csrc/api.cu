@@ -1218,9 +1218,8 @@ static int decode_impl(eesd_ctx *c, int max_new, const int32_t *k_schedule, int 
 
 int eesd_batch_begin(eesd_ctx *c, int n_seq) {
     if (!c || n_seq < 0 || n_seq > kMaxSeqs) return EESD_ERR_BADARG;
-    // the bf16-cache attention kernel is the one that knows about batches; trees and the per-sequence
-    // stopping rules of the controllers have no batch counterpart here
-    if (n_seq > 0 && (c->cfg.dtype != EESD_BF16 || tree_on(c))) return EESD_ERR_UNSUPPORTED;
+    // trees and the per-sequence stopping rules of the controllers have no batch counterpart here
+    if (n_seq > 0 && tree_on(c)) return EESD_ERR_UNSUPPORTED;
     if (batch_on(c)) {   // leave batch mode: give every sequence's pages back
         for (size_t b = 0; b < c->seqs.size(); b++) {
             select_seq(c, (int)b);

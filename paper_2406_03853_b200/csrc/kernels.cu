@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                                                    float *__restrict__ apart, unsigned int *tickets,
                                                    float *__restrict__ attn_out, bf16 *__restrict__ attn_split,
                                                    int M, int pos0, int H, int pps, int n_split, float scale, int *err,
-                                                   int nbat, size_t ml_off, TreeRows tr, uint32_t spin) {
+                                                   int nbat, size_t ml_off, TreeRows tr, uint32_t spin, BatchRows br) {
     typedef float AT;
     typedef float2 KP;   // a pair of adjacent head dimensions of one key
     constexpr int HALF = D / 2;
@@ -300,7 +300,21 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kh = blockIdx.x, sp = blockIdx.y;
-    const int bz = blockIdx.z;   // batch of (head, row) pairs
+    int bz = blockIdx.z;   // batch of (head, row) pairs
+    // Batch mode: grid z runs over (sequence, batch of pairs); a sequence is an independent problem with its own
+    // rows of the pass, positions, page table and slice count (the scratch layouts keep the launch's slice count).
+    const int ns_stride = n_split;
+    int row_base = 0;
+    if (br.n_seq > 0) {
+        const int seq = blockIdx.z / nbat;
+        bz = blockIdx.z - seq * nbat;
+        M = br.rows[seq];
+        pos0 = br.pos0[seq];
+        row_base = br.row0[seq];
+        kv.page_table += br.table_off[seq];
+        n_split = ((pos0 + M + PT - 1) / PT + pps - 1) / pps;
+        if (sp >= n_split || group * M <= bz * RB) return;   // a shorter sequence fills fewer slices and batches
+    }
     // per-slice (maximum, sum) pairs live behind the outputs: [H][16][kMaxSlices]
     float2 *ml = reinterpret_cast<float2 *>(apart + ml_off);
     const int r0 = bz * RB;                  // first (head, row) pair of this block's batch
@@ -348,9 +362,9 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
         s_tb[tid] = tile_blocks(pv.sk, tid < nq ? tq0 + tid : (tid == nq ? tk : tv));
     __syncthreads();
     auto gather_pair = [&](int m, int col) -> float2 {
-        if (pv.mode == 0) return part_gather_n<2>(pv, m, col);
+        if (pv.mode == 0) return part_gather_n<2>(pv, row_base + m, col);
         const int t = col >> 7;
-        return part_gather_blocks<2>(pv, s_tb[t == tk ? nq : (t == tv ? nq + 1 : t - tq0)], m, col);
+        return part_gather_blocks<2>(pv, s_tb[t == tk ? nq : (t == tv ? nq + 1 : t - tq0)], row_base + m, col);
     };
     // rotation factors of the new keys and of this block's queries: a constant table, fetched
     // before the wait so that they are not one more round trip behind the partial sums
@@ -375,7 +389,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     // One round of global loads: the RMSNorm statistics (threads 0..M-1) and the raw partial
     // sums of this block's queries and of the new keys / values that fall into its slice; they
     // are scaled, rotated and rounded after the barrier, while the cached slice is still arriving.
-    if (tid < M) s_rstd[tid] = row_rstd(rs, tid);
+    if (tid < M) s_rstd[tid] = row_rstd(rs, row_base + tid);
     float raw_a[kNewPerThread], raw_b[kNewPerThread];
     int new_page[kNewPerThread];
 #pragma unroll
@@ -460,7 +474,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
             const int page = new_page[it];
             if (page < 0 || page >= kv.n_pages_total) { atomicOr(err, kErrBadPage); continue; }
             AT *blk = (AT *)kv.slot_base + (((size_t)page * 2 + isV) * kv.Hkv + kh) * (size_t)PT * D;
-            const bool append = blockIdx.z == 0;   // every batch needs the row in its tile; one block writes the cache
+            const bool append = bz == 0;   // every batch needs the row in its tile; one block writes the cache
             if (isV) {
                 const int e = v_elem<AT>(pos, 2 * i);
                 AT *tile = sV + (size_t)j * D + e;
@@ -563,10 +577,10 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
                 if (rl < nb) {
                     const int g = (r0 + rl) / M, m = (r0 + rl) - g * M;
                     const int h = kh * group + g;
-                    float *dst = apart + (((size_t)h * n_split + sp) * kMaxRows + m) * D;
+                    float *dst = apart + (((size_t)h * ns_stride + sp) * kMaxRows + row_base + m) * D;
 #pragma unroll
                     for (int e = 0; e < DPL; e++) dst[lane * DPL + e] = o[i][e];
-                    if (lane == 0) ml[((size_t)h * kMaxRows + m) * kMaxSlices + sp] = make_float2(s_m[rl], s_l[rl]);
+                    if (lane == 0) ml[((size_t)h * kMaxRows + row_base + m) * kMaxSlices + sp] = make_float2(s_m[rl], s_l[rl]);
                 }
             }
         }
@@ -576,7 +590,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        unsigned int *tk = tickets + (size_t)kh * nbat + bz;   // one counter per (KV head, batch)
+        unsigned int *tk = tickets + (size_t)kh * gridDim.z + blockIdx.z;   // one counter per (KV head, sequence, batch)
         const unsigned int prev = atomicAdd(tk, 1u);
         s_last = (prev == (unsigned int)n_split - 1);
         if (s_last) *tk = 0;
@@ -593,7 +607,7 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
         for (int i = 0; i < RPW; i++) {
             const int rl = warp + 8 * i, rho = r0 + min(rl, nb - 1);
             const int g = rho / M, m = rho - g * M, h = kh * group + g;
-            const float2 *src = ml + ((size_t)h * kMaxRows + m) * kMaxSlices;
+            const float2 *src = ml + ((size_t)h * kMaxRows + row_base + m) * kMaxSlices;
             v0[i] = (rl < nb && lane < n_split) ? __ldcg(src + lane) : none;
             v1[i] = (rl < nb && lane + 32 < n_split) ? __ldcg(src + lane + 32) : none;
         }
@@ -613,8 +627,8 @@ __global__ void __launch_bounds__(256) attn_kernel(PartView pv, RowScale rs, con
     __syncthreads();
     for (int idx = tid; idx < nb * (D / 4); idx += 256) {   // four output dimensions per item
         const int rl = idx / (D / 4), dd = (idx - rl * (D / 4)) * 4, rho = r0 + rl;
-        const int g = rho / M, m = rho - g * M, h = kh * group + g;
-        const float *src = apart + ((size_t)h * n_split * kMaxRows + m) * D + dd;
+        const int g = rho / M, m = row_base + rho - g * M, h = kh * group + g;   // m: row of the pass
+        const float *src = apart + ((size_t)h * ns_stride * kMaxRows + m) * D + dd;
         const float *wr = wgt + rl * n_split;
         float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int s2 = 0; s2 < n_split; s2 += 16) {   // sixteen slices in flight, added in slice order
@@ -646,7 +660,7 @@ static size_t attn_smem_bytes(int D, int RB, int cap, int n_split) {
 template <int D, int RB, int NM, bool TR>
 static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                         float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                        int pps, int n_split, float scale, bool early, int *err, const TreeRows &tr, uint32_t wait_polls) {
+                        int pps, int n_split, float scale, bool early, int *err, const TreeRows &tr, uint32_t wait_polls, const BatchRows &br) {
     const int rows = (H / kv.Hkv) * M, nbat = (rows + RB - 1) / RB;
     const size_t ml_off = (size_t)H * kMaxSlices * kMaxRows * D;
     const size_t smem = attn_smem_bytes(D, RB, pps * kv.page_tokens, n_split);
@@ -654,18 +668,19 @@ static void attn_launch(cudaStream_t s, const PartView &pv, const RowScale &rs, 
     static const cudaError_t configured =
         cudaFuncSetAttribute(attn_kernel<D, RB, NM, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
     (void)configured;
-    launch_k(attn_kernel<D, RB, NM, TR>, dim3(kv.Hkv, n_split, nbat), dim3(256), smem, s, early && pdl_enabled(), pv, rs, rope, kv,
-             apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, nbat, ml_off, tr, wait_polls);
+    launch_k(attn_kernel<D, RB, NM, TR>, dim3(kv.Hkv, n_split, nbat * (br.n_seq > 0 ? br.n_seq : 1)), dim3(256), smem, s, early && pdl_enabled(),
+             pv, rs, rope, kv, apart, tickets, attn_out, (bf16 *)attn_split, M, pos0, H, pps, n_split, scale, err, nbat, ml_off, tr, wait_polls, br);
 }
 
 template <int D>
 static void attn_dispatch(cudaStream_t s, const PartView &pv, const RowScale &rs, const float2 *rope, const KvGeom &kv,
                           float *apart, unsigned int *tickets, float *attn_out, void *attn_split, int M, int pos0, int H,
-                          int pps, int n_split, float scale, bool early, int *err, const TreeRows *tree, uint32_t wait_polls) {
+                          int pps, int n_split, float scale, bool early, int *err, const TreeRows *tree, uint32_t wait_polls,
+                          const BatchRows &br) {
     const int rows = (H / kv.Hkv) * M;
     const TreeRows tr = tree ? *tree : chain_rows();
-#define EESD_ATTN(RB, NM) attn_launch<D, RB, NM, false>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls)
-#define EESD_ATTN_TREE(RB, NM) attn_launch<D, RB, NM, true>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls)
+#define EESD_ATTN(RB, NM) attn_launch<D, RB, NM, false>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls, br)
+#define EESD_ATTN_TREE(RB, NM) attn_launch<D, RB, NM, true>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tr, wait_polls, br)
     if (tree) {   // tree passes: one instantiation per batch size
         if (rows <= 8) EESD_ATTN_TREE(8, 8);
         else if (rows <= kRows16) EESD_ATTN_TREE(16, 16);
@@ -724,7 +739,7 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
             if (batch->pos0[b] + batch->rows[b] > ctx) ctx = batch->pos0[b] + batch->rows[b];
         }
         pos0 = ctx - M;
-        if (dtype == 0 || tree) {   // only the bf16-cache kernel knows about batches
+        if (tree) {   // a tree's rows belong to one sequence
             const int e = kErrPlan;
             cudaMemcpyAsync(err, &e, sizeof(e), cudaMemcpyHostToDevice, s);
             return;
@@ -749,11 +764,13 @@ void launch_attention(cudaStream_t s, int dtype, const PartView &pv, const RowSc
         return;
     }
     const int rb = rows <= 8 ? 8 : rows <= kRows16 ? 16 : 32;
-    const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb, n_sm, max_splits, &pps);
+    const int n_split = attention_splits(pos0 + M, kv.page_tokens, kv.Hkv, (rows + rb - 1) / rb * (batch ? batch->n_seq : 1), n_sm, max_splits, &pps);
     if (refuse(n_split)) return;
+    BatchRows br = {};
+    if (batch) br = *batch;
     const float scale = 1.0f / sqrtf((float)kv.D);
-    if (kv.D == 64) attn_dispatch<64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls);
-    else attn_dispatch<128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls);
+    if (kv.D == 64) attn_dispatch<64>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls, br);
+    else attn_dispatch<128>(s, pv, rs, rope, kv, apart, tickets, attn_out, attn_split, M, pos0, H, pps, n_split, scale, early, err, tree, wait_polls, br);
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU, partial sums

@@ -16,7 +16,8 @@ pytestmark = pytest.mark.gpu
 TOL = 2e-2
 BASE = synth.TINY.with_(dtype="bf16", ffn_dim=640)          # every projection tile-aligned: the tensor-core kernels
 SPECS = {"mha": BASE, "gqa8": BASE.with_(n_heads=8, n_kv_heads=1, head_dim=64, n_layers=2),
-         "wide_head": BASE.with_(n_heads=2, n_kv_heads=1, head_dim=128, n_layers=2)}
+         "wide_head": BASE.with_(n_heads=2, n_kv_heads=1, head_dim=128, n_layers=2),
+         "f32": synth.TINY, "f32_gqa": synth.TINY.with_(n_kv_heads=2)}                 # fp32 cache: the SIMT attention kernel
 
 
 @pytest.mark.parametrize("variant,lens,m,pt,max_ctx", [
@@ -25,6 +26,8 @@ SPECS = {"mha": BASE, "gqa8": BASE.with_(n_heads=8, n_kv_heads=1, head_dim=64, n
     ("gqa8", (40, 23), 8, 16, 96),              # 64 (head, row) pairs per sequence: two column batches each
     ("wide_head", (300, 150, 2), 4, 16, 384),   # contexts of very different length: 1 to several slices per sequence
     ("mha", (200, 90), 3, 128, 384),            # one page holds the whole context
+    ("f32", (37, 16, 5), 5, 16, 96),
+    ("f32_gqa", (300, 9, 120, 1), 4, 8, 384),   # fp32 cache, 8-token pages: up to 13 slices for one sequence, one for another
 ])
 def test_batched_verification_pass_matches_the_oracle_row_by_row(variant, lens, m, pt, max_ctx):
     spec = SPECS[variant]
@@ -44,11 +47,34 @@ def test_batched_verification_pass_matches_the_oracle_row_by_row(variant, lens, 
             o.target_rows(p[:-1], 0, want_logits=False)
         _, lg = o.target_rows(rows[b].astype(np.int32), len(p) - 1)
         err = np.abs(got[b] - lg).max()
-        assert err < TOL, (b, err)
+        assert err < (TOL if spec.dtype == "bf16" else 2e-4), (b, err)
         n_tok, pages = eng.batch_context_len(b)
         assert n_tok == len(p) and pages == (len(p) - 1 + m + pt - 1) // pt
     eng.batch_begin(0)
     assert eng.context_len() == (0, 0)
+    eng.close()
+
+
+@pytest.mark.parametrize("temperature", [0.0, 1.0])
+@pytest.mark.parametrize("lens,pt", [((21, 40, 7), 8), ((12, 33, 5, 18, 26, 1, 9, 64), 16)])
+def test_batch_decode_fp32_model_equals_the_oracle(lens, pt, temperature):
+    # the fp32 tiny model is the configuration whose tokens equal the oracle's exactly: every sequence of a batch
+    # must reproduce the oracle's own generation for its prompt, uniforms and draft lengths, token by token
+    spec = synth.TINY
+    max_new, max_ctx, B = 32, 128, len(lens)
+    eng = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, temperature=temperature, page_tokens=pt, kv_pages=B * (max_ctx // pt))
+    prompts = [synth.prompt_tokens(190 + b, n, spec.vocab).numpy() for b, n in enumerate(lens)]
+    unis = [{k: v.numpy() for k, v in synth.generate_uniforms(max_ctx, 64, seed=500 + b).items()} for b in range(B)]
+    eng.batch_begin(B)
+    for b, p in enumerate(prompts):
+        eng.batch_prefill(b, p)
+    out, traces, _ = eng.batch_decode(max_new, k_schedule=[2, 5, 1, 3, 7, 4] * 8, uniforms=unis if temperature else None)
+    for b, p in enumerate(prompts):
+        ks = [k for k, _, _ in traces[b]]
+        ref, rtrace, _ = oracle_from_spec(spec, max_ctx).generate(p, max_new, temperature=temperature, k_schedule=ks + [3] * 8, fixed_k=3,
+                                                                  uniforms=unis[b] if temperature else None)
+        np.testing.assert_array_equal(out[b], ref)
+        assert traces[b] == rtrace[:len(traces[b])]
     eng.close()
 
 
@@ -83,11 +109,11 @@ def test_batch_decode_equals_single_sequence_decoding(variant, lens, temperature
 
 def test_batch_mode_errors():
     from paper_2406_03853_b200 import EesdError
-    f32 = engine_from_spec(synth.TINY, max_ctx=64)
+    tree = engine_from_spec(synth.TINY, max_ctx=64, tree_width=2, k_cap=5)
     with pytest.raises(EesdError) as e:
-        f32.batch_begin(2)                                  # fp32 cache: the SIMT attention kernel has no batch form
+        tree.batch_begin(2)                                 # a tree's rows belong to one sequence
     assert e.value.status == -8
-    f32.close()
+    tree.close()
     eng = engine_from_spec(BASE, max_ctx=64, page_tokens=16, kv_pages=8)
     with pytest.raises(EesdError):
         eng.batch_begin(9)
