@@ -135,3 +135,40 @@ def test_batch_mode_errors():
     out1, _, _ = eng.generate(p, 8)                         # and open again afterwards
     np.testing.assert_array_equal(out1, out[0])
     eng.close()
+
+
+def test_batch_decode_continues_and_page_pool_exhaustion_is_reported():
+    from paper_2406_03853_b200 import EesdError
+    spec = BASE
+    prompts = [synth.prompt_tokens(140 + b, n, spec.vocab).numpy() for b, n in enumerate((11, 30, 19))]
+    eng = engine_from_spec(spec, max_ctx=128, k_cap=10, fixed_k=2, page_tokens=16, kv_pages=24)
+    eng.batch_begin(3)
+    for b, p in enumerate(prompts):
+        eng.batch_prefill(b, p)
+    whole, _, _ = eng.batch_decode(30)
+    eng.batch_begin(3)
+    for b, p in enumerate(prompts):
+        eng.batch_prefill(b, p)
+    first, traces, _ = eng.batch_decode(12)
+    # a second call goes on from where every sequence stands (the surplus tokens of its last round included)
+    have = [sum(a + 1 for _, a, _ in t) for t in traces]
+    rest, _, _ = eng.batch_decode(30 - min(have))
+    for b in range(3):
+        n_tok, _ = eng.batch_context_len(b)
+        np.testing.assert_array_equal(first[b], whole[b][:12])
+        extra = have[b] - 12                                  # tokens the first call produced beyond its 12
+        np.testing.assert_array_equal(rest[b][:30 - have[b]], whole[b][have[b]:30])
+        assert extra >= 0 and n_tok >= len(prompts[b]) + 30
+    eng.close()
+    # a pool too small for the three contexts: the call says so, and the engine is usable afterwards
+    small = engine_from_spec(spec, max_ctx=128, k_cap=10, fixed_k=2, page_tokens=16, kv_pages=8)
+    small.batch_begin(3)
+    for b, p in enumerate(prompts):
+        small.batch_prefill(b, p)                             # 1 + 2 + 2 pages
+    with pytest.raises(EesdError) as e:
+        small.batch_decode(60)                                # needs about 5 + 6 + 5 pages
+    assert e.value.status == -5
+    small.batch_begin(0)
+    out, _, _ = small.generate(prompts[0], 20)
+    np.testing.assert_array_equal(out, whole[0][:20])
+    small.close()
