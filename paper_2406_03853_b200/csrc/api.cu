@@ -89,8 +89,9 @@ int prefill_rows(const eesd_config *c) {
     return need < kPrefillRows ? need : kPrefillRows;
 }
 
-// arrival counters of the attention merge: one per (KV head, batch of (head, row) pairs)
-size_t ticket_count(const eesd_config *c) { return 1024 + (size_t)c->n_heads; }
+// arrival counters of the attention merge: one per (KV head, sequence of a batch, batch of (head, row) pairs); at most
+// n_kv_heads * 8 * (pairs of a sequence / 16 + 1) <= n_heads + 8 * n_kv_heads of them are in use
+size_t ticket_count(const eesd_config *c) { return 1024 + (size_t)9 * c->n_heads; }
 
 // entries of one sequence's page table
 size_t table_len(const eesd_config *c) { return (size_t)c->max_ctx / c->page_tokens + 2; }

@@ -102,7 +102,7 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
 // the paged cache, every KV head's cached slice is read once, and the slices are merged into
 // attn_out (fp32 [M][H*D], may be null) and attn_split (two bf16 terms, may be null).
 // apart: H * max_splits * 16 * (D + 2) floats; tickets: zero-initialised counters, one per
-// (KV head, batch of 32 (head, row) pairs): at most H_kv * 4.
+// (KV head, sequence of a batch, batch of 16 or 32 (head, row) pairs).
 // batch (optional, no tree): the rows belong to several sequences; M, pos0 and kv.page_table
 // are then taken per sequence from it, and `M` is the largest row count of a sequence.
 // early: the kernel may start (and read cached rows) while the kernel before it still runs;
