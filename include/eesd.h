@@ -335,7 +335,8 @@ int eesd_capture_hidden(eesd_ctx *ctx, float *device_buf, size_t bytes);
  * first wait of every block give up at once: no result is produced, nothing is left in flight, and
  * the error path can be exercised without stalling anything.
  * eesd_clear_device_error: zeroes the error word and the counters a failed pass may have left half
- * counted, and forgets the sequence (as eesd_reset); the context is usable again afterwards. */
+ * counted, and forgets the sequence (as eesd_reset; in batch mode all sequences: the context is back in
+ * single-sequence mode); the context is usable again afterwards. */
 int eesd_set_wait_limit(eesd_ctx *ctx, uint32_t polls);
 int eesd_clear_device_error(eesd_ctx *ctx);
 

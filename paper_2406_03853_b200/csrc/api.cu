@@ -1475,6 +1475,7 @@ int eesd_clear_device_error(eesd_ctx *c) {
     CU(c, cudaMemsetAsync(c->tickets, 0, ticket_count(&c->cfg) * 4, c->stream));
     CU(c, cudaStreamSynchronize(c->stream));
     c->h_result[2] = 0;
+    if (batch_on(c)) return eesd_batch_begin(c, 0);   // a round that failed half way leaves the sequences of a batch inconsistent: forget them all
     reset_sequence(c);
     return EESD_OK;
 }

@@ -172,3 +172,29 @@ def test_batch_decode_continues_and_page_pool_exhaustion_is_reported():
     out, _, _ = small.generate(prompts[0], 20)
     np.testing.assert_array_equal(out, whole[0][:20])
     small.close()
+
+
+def test_a_wait_that_runs_out_in_a_batch_round_is_reported_and_cleared():
+    from paper_2406_03853_b200 import EesdError
+    eng = engine_from_spec(BASE, max_ctx=96, k_cap=10, fixed_k=3, page_tokens=16, kv_pages=18)
+    prompts = [synth.prompt_tokens(160 + b, n, BASE.vocab).numpy() for b, n in enumerate((14, 29, 6))]
+    eng.batch_begin(3)
+    for b, p in enumerate(prompts):
+        eng.batch_prefill(b, p)
+    ref, _, _ = eng.batch_decode(16)
+    eng.batch_begin(3)
+    for b, p in enumerate(prompts):
+        eng.batch_prefill(b, p)
+    eng.set_wait_limit(0)                                   # every bounded wait gives up at once: nothing is stalled
+    with pytest.raises(EesdError) as e:
+        eng.batch_decode(16)
+    assert e.value.status == -7
+    eng.set_wait_limit(None)
+    eng.clear_device_error()                                # leaves batch mode, all pages free
+    assert eng.context_len() == (0, 0)
+    eng.batch_begin(3)
+    for b, p in enumerate(prompts):
+        eng.batch_prefill(b, p)
+    out, _, _ = eng.batch_decode(16)
+    np.testing.assert_array_equal(out, ref)
+    eng.close()
