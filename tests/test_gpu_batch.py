@@ -79,12 +79,13 @@ def test_batch_decode_fp32_model_equals_the_oracle(lens, pt, temperature):
 
 
 @pytest.mark.parametrize("temperature", [0.0, 1.0])
-@pytest.mark.parametrize("variant,lens", [("mha", (21, 40, 7)), ("gqa8", (12, 33, 5, 18, 26))])
-def test_batch_decode_equals_single_sequence_decoding(variant, lens, temperature):
+@pytest.mark.parametrize("variant,lens,n_exit", [("mha", (21, 40, 7), 1), ("gqa8", (12, 33, 5, 18, 26), 1), ("mha", (9, 30), 2)])
+def test_batch_decode_equals_single_sequence_decoding(variant, lens, n_exit, temperature):
     spec = SPECS[variant]
     max_new, max_ctx = 40, 128
     B = len(lens)
-    eng = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, temperature=temperature, page_tokens=16, kv_pages=B * 8)
+    eng = engine_from_spec(spec, max_ctx=max_ctx, k_cap=10, fixed_k=3, temperature=temperature, page_tokens=16, kv_pages=B * 8,
+                           n_exit_layers=n_exit)     # (two early-exit layers: their caches are synchronised per sequence as well)
     prompts = [synth.prompt_tokens(90 + b, n, spec.vocab).numpy() for b, n in enumerate(lens)]
     unis = [{k: v.numpy() for k, v in synth.generate_uniforms(max_ctx, 64, seed=300 + b).items()} for b in range(B)]
     eng.batch_begin(B)
