@@ -433,7 +433,7 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
     auto layer = [&](const LayerW &w, int slot, const float *g_after) {
         PartView pv = proj(w.m_qkv, X_NORM, qd + 2 * kvd, d);
         // keys / values of all rows into the cache first, then the causal attention of all rows
-        launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, slot), c->rope, nullptr, true, c->err, qd);
+        launch_kv_append_wide(s, pv, rs, Mtot, p0, kv_geom(c, slot), c->rope, qd, c->err);
         launch_attention_prompt(s, pv, rs, c->rope, kv_geom(c, slot), c->wxs[X_ATTN], Mtot, p0, H, c->err, c->wait_polls);
         c->launches += 2;
         pv = proj(w.m_o, X_ATTN, d, qd);
@@ -452,7 +452,7 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
             if (E > 1) CU(c, cudaMemcpyAsync(c->wx_save, c->wx, (size_t)Mtot * d * 4, cudaMemcpyDeviceToDevice, s));
             for (int e = 0; e + 1 < E; e++) layer(c->layers[L + e], L + e, c->layers[L + e + 1].g_attn);
             PartView pv = proj(c->m_exit_kv, X_NORM, 2 * kvd, d);
-            launch_qkv_post(s, f.dtype, pv, rs, Mtot, p0, H, kv_geom(c, L + E - 1), c->rope, nullptr, true, c->err);
+            launch_kv_append_wide(s, pv, rs, Mtot, p0, kv_geom(c, L + E - 1), c->rope, 0, c->err);
             c->launches++;
             if (E > 1) CU(c, cudaMemcpyAsync(c->wx, c->wx_save, (size_t)Mtot * d * 4, cudaMemcpyDeviceToDevice, s));
             resid(nullptr, l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);

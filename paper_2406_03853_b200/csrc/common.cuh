@@ -109,4 +109,15 @@ __device__ __forceinline__ void store_split(__nv_bfloat16 *xs, int m, size_t K, 
     xs[(row + kMaxRows) * K + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
+// four consecutive elements at once (i % 4 == 0): one 8-byte store per term
+__device__ __forceinline__ void store_split4(__nv_bfloat16 *xs, int m, size_t K, size_t i, float4 v) {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(v.x), h1 = __float2bfloat16_rn(v.y), h2 = __float2bfloat16_rn(v.z), h3 = __float2bfloat16_rn(v.w);
+    const __nv_bfloat16 l0 = __float2bfloat16_rn(v.x - __bfloat162float(h0)), l1 = __float2bfloat16_rn(v.y - __bfloat162float(h1));
+    const __nv_bfloat16 l2 = __float2bfloat16_rn(v.z - __bfloat162float(h2)), l3 = __float2bfloat16_rn(v.w - __bfloat162float(h3));
+    auto pack = [](__nv_bfloat16 a, __nv_bfloat16 b) { return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16); };
+    const size_t row = (size_t)(m / kMaxRows) * (2 * kMaxRows) + (size_t)(m % kMaxRows);
+    *reinterpret_cast<uint2 *>(xs + row * K + i) = make_uint2(pack(h0, h1), pack(h2, h3));
+    *reinterpret_cast<uint2 *>(xs + (row + kMaxRows) * K + i) = make_uint2(pack(l0, l1), pack(l2, l3));
+}
+
 }  // namespace eesd

@@ -91,10 +91,7 @@ __global__ void __launch_bounds__(256) resid_kernel(float *x, PartView pv, int h
         const float4 g4 = *reinterpret_cast<const float4 *>(g + i);
         const float4 y = make_float4(v.x * g4.x, v.y * g4.y, v.z * g4.z, v.w * g4.w);
         if (xn) *reinterpret_cast<float4 *>(xn + (size_t)m * d + i) = y;
-        if (xs) {
-            store_split(xs, m, d, i, y.x); store_split(xs, m, d, i + 1, y.y);
-            store_split(xs, m, d, i + 2, y.z); store_split(xs, m, d, i + 3, y.w);
-        }
+        if (xs) store_split4(xs, m, d, i, y);
     }
     ss = block_sum(ss, scratch);
     if (threadIdx.x == 0) ssq[m * kSsqBlocks + blockIdx.x] = ss;
@@ -239,6 +236,89 @@ void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowSca
     const int tree_on = tree && M <= 16 ? 1 : 0;
     if (dtype == 0) launch_k(qkv_post_kernel<float>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on, row0);
     else launch_k(qkv_post_kernel<bf16>, grid, dim3(kv.D / 2), 0, s, pdl_enabled(), pv, rs, pos0, H, kv, rope, q, only_kv ? H : 0, kv_col0, err, tr, tree_on, row0);
+}
+
+// Prompt passes (bf16 cache, plain [split][row][column] projection result): keys / values of many rows into the
+// cache, one block per (KV head, group of 8 consecutive positions = one row of core matrices).  Threads
+// 0 .. D - 1 take (token, 8 key dimensions): scale, rotate, one 16-byte store; threads 128 .. 128 + D - 1 take one
+// value dimension of the 8 tokens: one 16-byte store (the row of a value core matrix), keeping what the
+// cache holds for tokens of the group that are not part of this pass.
+template <int D>
+__global__ void __launch_bounds__(256) kv_append_wide_kernel(PartView pv, RowScale rs, int Mtot, int pos0, KvGeom kv, const float2 *rope,
+                                                             int kcol0, int *err) {
+    __shared__ float s_rstd[8];
+    const int kh = blockIdx.x, grp = (pos0 >> 3) + blockIdx.y, tid = threadIdx.x;
+    const int PT = kv.page_tokens;
+    pdl_trigger();
+    pdl_wait();
+    if (tid < 8) {
+        const int m = grp * 8 + tid - pos0;
+        s_rstd[tid] = (m >= 0 && m < Mtot) ? row_rstd(rs, m) : 0.f;
+    }
+    __syncthreads();
+    const int page = kv.page_table[(grp * 8) / PT], pp = (grp * 8) & (PT - 1);   // the group lies inside one page
+    if (page < 0 || page >= kv.n_pages_total) {
+        if (tid == 0) atomicOr(err, kErrBadPage);
+        return;
+    }
+    unsigned char *blk_k = (unsigned char *)kv.slot_base + (((size_t)page * 2) * kv.Hkv + kh) * (size_t)PT * D * 2;
+    unsigned char *blk_v = blk_k + (size_t)kv.Hkv * PT * D * 2;
+    if (tid < D) {   // keys: token tt, dimensions 8 c .. 8 c + 7
+        const int tt = tid & 7, c = tid >> 3, m = grp * 8 + tt - pos0;
+        if (m >= 0 && m < Mtot) {
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+            for (int sp = 0; sp < pv.S; sp++) {
+                const float4 *src = reinterpret_cast<const float4 *>(pv.base + (size_t)sp * pv.split_stride + (size_t)m * pv.R + kcol0 + kh * D + 8 * c);
+                const float4 la = src[0], lb = src[1];
+                a.x += la.x; a.y += la.y; a.z += la.z; a.w += la.w;
+                b.x += lb.x; b.y += lb.y; b.z += lb.z; b.w += lb.w;
+            }
+            const float r = s_rstd[tt];
+            const float raw[8] = {a.x * r, a.y * r, a.z * r, a.w * r, b.x * r, b.y * r, b.z * r, b.w * r};
+            const float4 *cs = reinterpret_cast<const float4 *>(rope + (size_t)(pos0 + m) * (D / 2) + 4 * c);
+            const float4 w0 = cs[0], w1 = cs[1];
+            const float cw[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};   // (cos, sin) of four pairs
+            uint32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                const float x0 = raw[2 * i], x1 = raw[2 * i + 1];
+                const float ra = x0 * cw[2 * i] - x1 * cw[2 * i + 1], rb = x0 * cw[2 * i + 1] + x1 * cw[2 * i];
+                o[i] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(ra)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(rb)) << 16);
+            }
+            *reinterpret_cast<uint4 *>(blk_k + ((size_t)(pp >> 3) * (D / 8) + c) * 128 + tt * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    } else if (tid >= 128 && tid < 128 + D) {   // values: dimension d of the group's 8 tokens
+        const int d = tid - 128;
+        uint4 *dst = reinterpret_cast<uint4 *>(blk_v + ((size_t)(pp >> 3) * (D / 8) + (d >> 3)) * 128 + (d & 7) * 16);
+        const int m0 = grp * 8 - pos0;
+        const bool whole = m0 >= 0 && m0 + 8 <= Mtot;
+        uint4 old = make_uint4(0u, 0u, 0u, 0u);
+        if (!whole) old = *dst;
+        unsigned short h[8] = {(unsigned short)old.x, (unsigned short)(old.x >> 16), (unsigned short)old.y, (unsigned short)(old.y >> 16),
+                               (unsigned short)old.z, (unsigned short)(old.z >> 16), (unsigned short)old.w, (unsigned short)(old.w >> 16)};
+        float v[8];
+#pragma unroll
+        for (int tt = 0; tt < 8; tt++) {
+            const int m = m0 + tt;
+            v[tt] = 0.f;
+            if (m >= 0 && m < Mtot)
+                for (int sp = 0; sp < pv.S; sp++)
+                    v[tt] += pv.base[(size_t)sp * pv.split_stride + (size_t)m * pv.R + kcol0 + (kv.Hkv + kh) * D + d];
+        }
+#pragma unroll
+        for (int tt = 0; tt < 8; tt++) {
+            const int m = m0 + tt;
+            if (m >= 0 && m < Mtot) h[tt] = __bfloat16_as_ushort(__float2bfloat16_rn(v[tt] * s_rstd[tt]));
+        }
+        *dst = make_uint4((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16),
+                          (uint32_t)h[4] | ((uint32_t)h[5] << 16), (uint32_t)h[6] | ((uint32_t)h[7] << 16));
+    }
+}
+void launch_kv_append_wide(cudaStream_t s, const PartView &pv, const RowScale &rs, int Mtot, int pos0, const KvGeom &kv,
+                           const float2 *rope, int kcol0, int *err) {
+    const dim3 grid(kv.Hkv, ((pos0 + Mtot - 1) >> 3) - (pos0 >> 3) + 1);
+    if (kv.D == 64) launch_k(kv_append_wide_kernel<64>, grid, dim3(256), 0, s, pdl_enabled(), pv, rs, Mtot, pos0, kv, rope, kcol0, err);
+    else launch_k(kv_append_wide_kernel<128>, grid, dim3(256), 0, s, pdl_enabled(), pv, rs, Mtot, pos0, kv, rope, kcol0, err);
 }
 
 // ------------------------------------------------------------------------------------ paged decode attention, fp32 cache
@@ -783,12 +863,11 @@ __global__ void swiglu_kernel(PartView pv, RowScale rs, float *h, bf16 *hs, int 
     const float rstd = row_rstd(rs, m);
     const float gg[4] = {g.x * rstd, g.y * rstd, g.z * rstd, g.w * rstd};
     const float uu[4] = {u.x * rstd, u.y * rstd, u.z * rstd, u.w * rstd};
+    float v[4];
 #pragma unroll
-    for (int k = 0; k < 4; k++) {
-        const float v = gg[k] / (1.0f + expf(-gg[k])) * uu[k];
-        if (h) h[(size_t)m * F + i + k] = v;
-        if (hs) store_split(hs, m, F, i + k, v);
-    }
+    for (int k = 0; k < 4; k++) v[k] = gg[k] / (1.0f + expf(-gg[k])) * uu[k];
+    if (h) *reinterpret_cast<float4 *>(h + (size_t)m * F + i) = make_float4(v[0], v[1], v[2], v[3]);
+    if (hs) store_split4(hs, m, F, i, make_float4(v[0], v[1], v[2], v[3]));
 }
 void launch_swiglu(cudaStream_t s, const PartView &pv, const RowScale &rs, float *h, void *h_split, int M, int F) {
     launch_k(swiglu_kernel, dim3((F / 4 + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, h, (bf16 *)h_split, F);

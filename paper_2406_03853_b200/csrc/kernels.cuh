@@ -97,6 +97,10 @@ int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float 
 void launch_qkv_post(cudaStream_t s, int dtype, const PartView &pv, const RowScale &rs, int M, int pos0, int H,
                      const KvGeom &kv, const float2 *rope, float *q, bool only_kv, int *err, int kv_col0 = 0,
                      const TreeRows *tree = nullptr, int row0 = 0);
+// The same for the rows of a prompt pass (bf16 cache, D = 64 or 128, pv a plain [split][row][column] result): keys at
+// columns kcol0 + kh * D, values H_kv * D columns further; whole 16-byte rows of the cache's core matrices per thread.
+void launch_kv_append_wide(cudaStream_t s, const PartView &pv, const RowScale &rs, int Mtot, int pos0, const KvGeom &kv,
+                           const float2 *rope, int kcol0, int *err);
 // Fused attention step of one layer on M new rows: q/k/v of the new rows are taken from the
 // QKV projection's partial sums (scaled by rs, rotated), the new keys/values are appended to
 // the paged cache, every KV head's cached slice is read once, and the slices are merged into
