@@ -1056,16 +1056,27 @@ void launch_cali_theta(cudaStream_t s, const PartView &pv, const float *Wp, cons
     launch_k(cali_theta_kernel, dim3(1), dim3(256), 0, s, pdl_enabled(), pv, Wp, hD, d, theta);
 }
 
+// four consecutive outputs per thread (R % 4 == 0: tensor-core shapes are multiples of 128), else one
+template <int VEC>
 __global__ void reduce_partials_kernel(PartView pv, RowScale rs, float *out, int R, size_t out_stride) {
-    const int m = blockIdx.y, r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int m = blockIdx.y, r = (blockIdx.x * blockDim.x + threadIdx.x) * VEC;
     pdl_trigger();
     pdl_wait();
     if (r >= R) return;
-    out[(size_t)m * out_stride + r] = part_gather(pv, m, r) * row_rstd(rs, m);
+    if (VEC == 4) {
+        const float4 v = part_gather4(pv, m, r);
+        const float s = row_rstd(rs, m);
+        *reinterpret_cast<float4 *>(out + (size_t)m * out_stride + r) = make_float4(v.x * s, v.y * s, v.z * s, v.w * s);
+    } else {
+        out[(size_t)m * out_stride + r] = part_gather(pv, m, r) * row_rstd(rs, m);
+    }
 }
 void launch_reduce_partials(cudaStream_t s, const PartView &pv, const RowScale &rs, float *out, int M, int R, size_t out_stride) {
-    launch_k(reduce_partials_kernel, dim3((R + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, out, R,
-             out_stride ? out_stride : (size_t)R);
+    const size_t stride = out_stride ? out_stride : (size_t)R;
+    if (R % 4 == 0 && stride % 4 == 0)
+        launch_k(reduce_partials_kernel<4>, dim3((R / 4 + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, out, R, stride);
+    else
+        launch_k(reduce_partials_kernel<1>, dim3((R + 255) / 256, M), dim3(256), 0, s, pdl_enabled(), pv, rs, out, R, stride);
 }
 
 }  // namespace eesd
