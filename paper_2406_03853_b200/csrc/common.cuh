@@ -78,6 +78,18 @@ __device__ __forceinline__ float block_sum(float v, float *scratch /* >= 33 floa
     return scratch[32];
 }
 
+// the same sum (same order of additions) delivered to thread 0 only: one barrier instead of three
+__device__ __forceinline__ float block_sum_thread0(float v, float *scratch /* >= 32 floats */) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_sum(v);
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    if (threadIdx.x == 0)
+        for (int i = 0; i < nw; i++) t += scratch[i];
+    return t;
+}
+
 // Programmatic dependent launch.  pdl_trigger lets the next kernel in the stream be scheduled
 // early; pdl_wait blocks until every kernel this one depends on has completed and its writes
 // are visible.  Both are no-ops for kernels launched without the attribute.

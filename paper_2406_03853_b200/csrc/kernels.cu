@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(256) resid_kernel(float *x, PartView pv, int h
         if (xn) *reinterpret_cast<float4 *>(xn + (size_t)m * d + i) = y;
         if (xs) store_split4(xs, m, d, i, y);
     }
-    ss = block_sum(ss, scratch);
+    ss = block_sum_thread0(ss, scratch);
     if (threadIdx.x == 0) ssq[m * kSsqBlocks + blockIdx.x] = ss;
 }
 void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
