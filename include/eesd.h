@@ -328,7 +328,7 @@ int eesd_logits(const eesd_ctx *ctx, int which, const float **device_ptr);
 int eesd_capture_hidden(eesd_ctx *ctx, float *device_buf, size_t bytes);
 
 /* Bound of the waits inside the kernels.  Every wait of a kernel on data in flight (a bulk copy
- * into shared memory, a tensor-core operation) polls at most `polls` times (about a second's worth
+ * into shared memory, a tensor-core operation) polls at most `polls` times (a second or two's worth
  * by default; 0xffffffff restores the default); a wait that runs out makes its thread block raise
  * the context's error word, skip the rest of its work, let the copies it has already requested land
  * and return, and the call that reads results next returns EESD_ERR_DEVICE.  polls = 0 makes the

@@ -70,7 +70,7 @@ constexpr int kIntSlots = 128;   // small device integer area
 constexpr int kMaxSm = 256;      // upper bound on the SM count the work splits are planned for
 constexpr int kCtasPerSm = 2;    // projection CTAs per SM (gemm_tc.cu: two 4-stage rings fit one SM)
 constexpr int kPrefillRows = 512; // most prompt rows per pass of the wide (prompt) path
-constexpr uint32_t kDefaultWaitPolls = 1u << 25;   // polls before a wait inside a kernel gives up (about a second)
+constexpr uint32_t kDefaultWaitPolls = 1u << 23;   // polls before a wait inside a kernel gives up (a poll parks the thread for up to about 200 ns: under two seconds)
 
 // early-exit layers of the draft model (0 in the configuration reads as 1, the paper's setting)
 int n_exit(const eesd_config *c) { return c->n_exit_layers < 1 ? 1 : c->n_exit_layers; }
