@@ -329,6 +329,13 @@ void run_resid(eesd_ctx *c, const PartView *pv, const float *g, float *cap, int 
     c->launches++;
 }
 
+// embedding rows of M tokens (tok[m * tok_stride]) and, in the same kernel, the first layer's normalised rows
+void run_embed(eesd_ctx *c, const int32_t *tok, int tok_stride, int M, float *cap) {
+    launch_embed_resid(c->stream, c->cfg.dtype, tok, tok_stride, c->embed, c->cfg.vocab, c->x, c->layers[0].g_attn,
+                       c->use_tc ? nullptr : c->xn, c->xs[X_NORM], cap, c->ssq, M, c->cfg.d_model, c->err);
+    c->launches++;
+}
+
 // one decoder layer on M rows at positions pos0.. ; on entry y = x * g_attn of this layer (and
 // its sums of squares) are in place; on exit x holds the layer output and y = x * g_next.
 void run_layer(eesd_ctx *c, const LayerW &w, int slot, int M, int pos0, const float *g_next, float *cap) {
@@ -358,9 +365,7 @@ int run_target(eesd_ctx *c, const int32_t *d_tok, int M, int pos0, bool want_log
     const eesd_config &f = c->cfg;
     cudaStream_t s = c->stream;
     const int L = f.n_layers, d = f.d_model;
-    launch_embed(s, f.dtype, d_tok, c->embed, c->x, cap_slot(c, 0), M, d, f.vocab, c->err);
-    run_resid(c, nullptr, c->layers[0].g_attn, nullptr, M);
-    c->launches += 1;
+    run_embed(c, d_tok, 1, M, cap_slot(c, 0));
     for (int l = 0; l < L; l++) {
         const bool exit_here = (l == f.n_early - 1);
         const float *g_after = exit_here ? c->layers[L].g_attn : (l + 1 < L ? c->layers[l + 1].g_attn : c->g_final);
@@ -427,9 +432,8 @@ int run_prompt_pass(eesd_ctx *c, const int32_t *prompt_host, int p0, int Mtot) {
         launch_resid(s, c->wx, pv, g, nullptr, c->wxs[X_NORM], nullptr, c->wssq, Mtot, d);
         c->launches++;
     };
-    launch_embed(s, f.dtype, c->wtok, c->embed, c->wx, nullptr, Mtot, d, f.vocab, c->err);
+    launch_embed_resid(s, f.dtype, c->wtok, 1, c->embed, f.vocab, c->wx, c->layers[0].g_attn, nullptr, c->wxs[X_NORM], nullptr, c->wssq, Mtot, d, c->err);
     c->launches++;
-    resid(nullptr, c->layers[0].g_attn);
     auto layer = [&](const LayerW &w, int slot, const float *g_after) {
         PartView pv = proj(w.m_qkv, X_NORM, qd + 2 * kvd, d);
         // keys / values of all rows into the cache first, then the causal attention of all rows
@@ -467,8 +471,7 @@ int run_draft_step(eesd_ctx *c, int i, int pos, const float *d_u) {
     const eesd_config &f = c->cfg;
     cudaStream_t s = c->stream;
     const int L = f.n_layers, d = f.d_model, N = f.n_early;
-    launch_embed(s, f.dtype, c->ints + kRoundTok + i, c->embed, c->x, cap_slot(c, 0), 1, d, f.vocab, c->err);
-    run_resid(c, nullptr, c->layers[0].g_attn, nullptr, 1);
+    run_embed(c, c->ints + kRoundTok + i, 1, 1, cap_slot(c, 0));
     for (int l = 0; l < N; l++) {
         const float *g_after = l + 1 < N ? c->layers[l + 1].g_attn : c->layers[L].g_attn;
         run_layer(c, c->layers[l], l, 1, pos, g_after, cap_slot(c, l + 1));
@@ -747,8 +750,7 @@ int run_batch_draft_step(eesd_ctx *c, const int *act, int n_act, int i, int K, c
     int32_t *chain = c->ints + kRowTok;
     batch_geometry(c, act, n_act, 1, i);
     c->batch_cur = &c->batch_rows;
-    launch_embed(s, f.dtype, chain + i, c->embed, c->x, nullptr, n_act, d, f.vocab, c->err, K + 1);
-    run_resid(c, nullptr, c->layers[0].g_attn, nullptr, n_act);
+    run_embed(c, chain + i, K + 1, n_act, nullptr);
     for (int l = 0; l < N; l++)
         run_layer(c, c->layers[l], l, n_act, 0, l + 1 < N ? c->layers[l + 1].g_attn : c->layers[L].g_attn, nullptr);
     for (int e = 0; e < c->E; e++)

@@ -103,6 +103,43 @@ void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, 
              (int)(pv != nullptr), g, xn, (bf16 *)xs, cap, ssq, d);
 }
 
+// Embedding gather and the first layer's rows in one kernel: x[m] = E[token]; then what resid_kernel does with x
+// (y = x * g as fp32 and / or two bf16 terms, the sums of squares per 1024 columns, the captured copy).  Same grid
+// and the same arithmetic as resid_kernel, so the rows are those of embed_kernel followed by resid_kernel.
+template <typename WT>
+__global__ void __launch_bounds__(256) embed_resid_kernel(const int32_t *tok, int tok_stride, const WT *E, int V, float *x, const float *g,
+                                                          float *xn, bf16 *xs, float *cap, float *ssq, int d, int *err) {
+    __shared__ float scratch[33];
+    const int m = blockIdx.y, i = blockIdx.x * 1024 + threadIdx.x * 4;
+    pdl_trigger();
+    pdl_wait();
+    int t = tok[(size_t)m * tok_stride];
+    if (t < 0 || t >= V) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(err, kErrBadToken);
+        t = 0;
+    }
+    float ss = 0.f;
+    if (i < d) {
+        const WT *row = E + (size_t)t * d + i;
+        const float4 v = make_float4(to_f(row[0]), to_f(row[1]), to_f(row[2]), to_f(row[3]));
+        *reinterpret_cast<float4 *>(x + (size_t)m * d + i) = v;
+        if (cap) *reinterpret_cast<float4 *>(cap + (size_t)m * d + i) = v;
+        ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        const float4 g4 = *reinterpret_cast<const float4 *>(g + i);
+        const float4 y = make_float4(v.x * g4.x, v.y * g4.y, v.z * g4.z, v.w * g4.w);
+        if (xn) *reinterpret_cast<float4 *>(xn + (size_t)m * d + i) = y;
+        if (xs) store_split4(xs, m, d, i, y);
+    }
+    ss = block_sum_thread0(ss, scratch);
+    if (threadIdx.x == 0) ssq[m * kSsqBlocks + blockIdx.x] = ss;
+}
+void launch_embed_resid(cudaStream_t s, int dtype, const int32_t *tok, int tok_stride, const void *E, int V, float *x, const float *g,
+                        float *xn, void *xs, float *cap, float *ssq, int M, int d, int *err) {
+    const dim3 grid((d + 1023) / 1024, M);
+    if (dtype == 0) launch_k(embed_resid_kernel<float>, grid, dim3(256), 0, s, pdl_enabled(), tok, tok_stride, (const float *)E, V, x, g, xn, (bf16 *)xs, cap, ssq, d, err);
+    else launch_k(embed_resid_kernel<bf16>, grid, dim3(256), 0, s, pdl_enabled(), tok, tok_stride, (const bf16 *)E, V, x, g, xn, (bf16 *)xs, cap, ssq, d, err);
+}
+
 // ------------------------------------------------------------------------------------ skinny projection (SIMT)
 // out[m][r] = sum_k A[m][k] W[r][k] for m < M <= MT rows.  Each warp owns 4 weight rows and
 // streams them with 16-byte loads; the token rows sit in shared memory as fp32.  The k order

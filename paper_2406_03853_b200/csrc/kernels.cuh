@@ -89,6 +89,9 @@ void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, 
 // columns) of x[m]; cap[m] = x[m] (if cap).  The RMSNorm scale itself is applied by the consumers.
 void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
                   float *ssq, int M, int d);
+// launch_embed followed by launch_resid(x, no partial sums, g, ...) as one kernel (d % 4 == 0)
+void launch_embed_resid(cudaStream_t s, int dtype, const int32_t *tok, int tok_stride, const void *E, int V, float *x, const float *g,
+                        float *xn, void *xs, float *cap, float *ssq, int M, int d, int *err);
 // out[sp][m][r] = sum_{k in split sp} A[m][k] * W[r][k]; returns the number of K splits written
 int launch_gemm(cudaStream_t s, int dtype, const float *A, const void *W, float *out, int M, int R, int K);
 // RoPE + KV append (+ q store).  part rows are [q heads | k heads | v heads] or, when
