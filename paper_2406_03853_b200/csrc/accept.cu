@@ -389,6 +389,8 @@ __global__ void __launch_bounds__(kAccThreads) sample_rows_kernel(const float *l
     const int b = blockIdx.x;
     const float *l = logits + (size_t)b * logit_stride;
     const bool greedy = (T == 0.0f);
+    pdl_trigger();   // (programmatic dependent launch: resident early, reads the logits only once their producer is done)
+    pdl_wait();
     RowStat st = row_stat(l, V, greedy ? 1.0f : T, !greedy, sm);
     int tok = st.arg;
     if (!greedy) tok = block_draw(l, st, nullptr, st, T, V, u[b], sm);
@@ -397,7 +399,8 @@ __global__ void __launch_bounds__(kAccThreads) sample_rows_kernel(const float *l
 
 void launch_sample_rows(cudaStream_t s, const float *logits, const float *u, int B, int V, float T, int32_t *out,
                         size_t logit_stride, int out_stride) {
-    sample_rows_kernel<<<B, kAccThreads, 0, s>>>(logits, u, V, T, out, logit_stride ? logit_stride : (size_t)V, out_stride);
+    launch_k(sample_rows_kernel, dim3(B), dim3(kAccThreads), 0, s, pdl_enabled(), logits, u, V, T, out, logit_stride ? logit_stride : (size_t)V,
+             out_stride);
 }
 
 }  // namespace eesd
