@@ -922,6 +922,8 @@ __global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict
     __shared__ float s_pv;
     __shared__ int s_pi;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    pdl_trigger();
+    pdl_wait();
     float pv = INFINITY;
     int pi = -1;
     auto better = [](float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); };
@@ -984,7 +986,7 @@ __global__ void __launch_bounds__(1024) next_best_kernel(const float *__restrict
     }
 }
 void launch_next_best(cudaStream_t s, const float *logits, int V, int width, int32_t *first, int32_t *out) {
-    next_best_kernel<<<1, 1024, 0, s>>>(logits, V, width, first, out);
+    launch_k(next_best_kernel, dim3(1), dim3(1024), 0, s, pdl_enabled(), logits, V, width, first, out);
 }
 
 __global__ void tree_rows_kernel(const int32_t *chain, const int32_t *leaf, int K, int width, int32_t *rows) {
