@@ -43,30 +43,6 @@ void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float 
     rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(table, max_ctx, D / 2, log((double)theta), D);
 }
 
-// ------------------------------------------------------------------------------------ embedding gather
-template <typename WT>
-__global__ void embed_kernel(const int32_t *tok, const WT *E, float *x, float *cap, int d, int V, int *err, int tok_stride) {
-    const int m = blockIdx.x;
-    pdl_trigger();
-    pdl_wait();
-    int t = tok[(size_t)m * tok_stride];
-    if (t < 0 || t >= V) {
-        if (threadIdx.x == 0) atomicOr(err, kErrBadToken);
-        t = 0;
-    }
-    const WT *row = E + (size_t)t * d;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float v = to_f(row[i]);
-        x[(size_t)m * d + i] = v;
-        if (cap) cap[(size_t)m * d + i] = v;
-    }
-}
-void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
-                  int M, int d, int V, int *err, int tok_stride) {
-    if (dtype == 0) launch_k(embed_kernel<float>, dim3(M), dim3(256), 0, s, pdl_enabled(), tok, (const float *)E, x, cap, d, V, err, tok_stride);
-    else launch_k(embed_kernel<bf16>, dim3(M), dim3(256), 0, s, pdl_enabled(), tok, (const bf16 *)E, x, cap, d, V, err, tok_stride);
-}
-
 // ------------------------------------------------------------------------------------ residual + RMSNorm
 // grid (ceil(d / 1024), M), 256 threads, four elements per thread.
 // x[m] += partial sums; y = x[m] * g (fp32 and / or two bf16 terms); ssq[m][block] = sum x^2.
@@ -105,7 +81,7 @@ void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, 
 
 // Embedding gather and the first layer's rows in one kernel: x[m] = E[token]; then what resid_kernel does with x
 // (y = x * g as fp32 and / or two bf16 terms, the sums of squares per 1024 columns, the captured copy).  Same grid
-// and the same arithmetic as resid_kernel, so the rows are those of embed_kernel followed by resid_kernel.
+// and the same arithmetic as resid_kernel, so the rows are those of a plain gather followed by resid_kernel.
 template <typename WT>
 __global__ void __launch_bounds__(256) embed_resid_kernel(const int32_t *tok, int tok_stride, const WT *E, int V, float *x, const float *g,
                                                           float *xn, bf16 *xs, float *cap, float *ssq, int d, int *err) {

@@ -81,15 +81,13 @@ inline TreeRows chain_rows() {
 
 void launch_set_ints(cudaStream_t s, int32_t *dst, const IntList16 &vals, int n);
 void launch_rope_table(cudaStream_t s, float2 *table, int max_ctx, int D, float theta);
-// row m takes token tok[m * tok_stride]
-void launch_embed(cudaStream_t s, int dtype, const int32_t *tok, const void *E, float *x, float *cap,
-                  int M, int d, int V, int *err, int tok_stride = 1);
 // x[m] += partial sums (if pv); y = x[m] * g -> xn (fp32, may be null) and xs (two bf16 terms,
 // [chunk of 16 rows][hi | lo][16][d], may be null); ssq[m][b] = sum of squares of block b (1024
 // columns) of x[m]; cap[m] = x[m] (if cap).  The RMSNorm scale itself is applied by the consumers.
 void launch_resid(cudaStream_t s, float *x, const PartView *pv, const float *g, float *xn, void *xs, float *cap,
                   float *ssq, int M, int d);
-// launch_embed followed by launch_resid(x, no partial sums, g, ...) as one kernel (d % 4 == 0)
+// Embedding gather (row m takes token tok[m * tok_stride]) and launch_resid(x, no partial sums, g, ...) on the rows, in one
+// kernel (d % 4 == 0)
 void launch_embed_resid(cudaStream_t s, int dtype, const int32_t *tok, int tok_stride, const void *E, int V, float *x, const float *g,
                         float *xn, void *xs, float *cap, float *ssq, int M, int d, int *err);
 // out[sp][m][r] = sum_{k in split sp} A[m][k] * W[r][k]; returns the number of K splits written
