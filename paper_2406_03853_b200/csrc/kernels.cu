@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(256) resid_kernel(float *x, PartView pv, int h
             *reinterpret_cast<float4 *>(xr + i) = v;
         }
         if (cap) *reinterpret_cast<float4 *>(cap + (size_t)m * d + i) = v;
-        ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        ss = fmaf(v.w, v.w, fmaf(v.z, v.z, fmaf(v.y, v.y, v.x * v.x)));   // one fixed form wherever these sums are taken
         const float4 g4 = *reinterpret_cast<const float4 *>(g + i);
         const float4 y = make_float4(v.x * g4.x, v.y * g4.y, v.z * g4.z, v.w * g4.w);
         if (xn) *reinterpret_cast<float4 *>(xn + (size_t)m * d + i) = y;
@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(256) embed_resid_kernel(const int32_t *tok, in
         const float4 v = make_float4(to_f(row[0]), to_f(row[1]), to_f(row[2]), to_f(row[3]));
         *reinterpret_cast<float4 *>(x + (size_t)m * d + i) = v;
         if (cap) *reinterpret_cast<float4 *>(cap + (size_t)m * d + i) = v;
-        ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        ss = fmaf(v.w, v.w, fmaf(v.z, v.z, fmaf(v.y, v.y, v.x * v.x)));   // one fixed form wherever these sums are taken
         const float4 g4 = *reinterpret_cast<const float4 *>(g + i);
         const float4 y = make_float4(v.x * g4.x, v.y * g4.y, v.z * g4.z, v.w * g4.w);
         if (xn) *reinterpret_cast<float4 *>(xn + (size_t)m * d + i) = y;
